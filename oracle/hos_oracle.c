@@ -1,0 +1,302 @@
+/*
+ * CPU oracle for the hybrid offline-online scheduler (arXiv 2502.15763).
+ * TEST INFRASTRUCTURE ONLY -- see hos_oracle.h.  Single thread, no blocking,
+ * no fusion: each function takes the steps of the definition in order.
+ */
+#include "hos_oracle.h"
+
+#include <stdlib.h>
+#include <string.h>
+
+/* ------------------------------------------------------------------------- */
+/* Offline part: Minimizing-Makespan Bin Packing, Eq. 26-30                   */
+/* ------------------------------------------------------------------------- */
+
+void ora_estimate(int n, const uint32_t* p, const uint32_t* o, const ora_cost* c, int64_t* T)
+{
+    for (int i = 0; i < n; ++i)
+        T[i] = (int64_t)c->est_per_prompt_token * (int64_t)p[i]
+             + (int64_t)c->est_per_output_token * (int64_t)o[i];
+}
+
+typedef struct { int64_t key; int32_t idx; } ora_keyed;
+
+/* larger key first; equal keys: smaller index first */
+static int cmp_key_desc_idx_asc(const void* a, const void* b)
+{
+    const ora_keyed* x = (const ora_keyed*)a;
+    const ora_keyed* y = (const ora_keyed*)b;
+    if (x->key != y->key) return (x->key > y->key) ? -1 : 1;
+    if (x->idx != y->idx) return (x->idx < y->idx) ? -1 : 1;
+    return 0;
+}
+
+void ora_order(int n, const int64_t* T, int32_t* order)
+{
+    ora_keyed* a = (ora_keyed*)malloc(sizeof(ora_keyed) * (size_t)(n > 0 ? n : 1));
+    for (int i = 0; i < n; ++i) { a[i].key = T[i]; a[i].idx = i; }
+    qsort(a, (size_t)n, sizeof(ora_keyed), cmp_key_desc_idx_asc);   /* keys (T, i) are unique */
+    for (int r = 0; r < n; ++r) order[r] = a[r].idx;
+    free(a);
+}
+
+void ora_lpt(int n, int M, const int64_t* T, const int32_t* order, int32_t* assign, int64_t* load)
+{
+    for (int j = 0; j < M; ++j) load[j] = 0;
+    for (int r = 0; r < n; ++r) {
+        int i = order[r];
+        int best = 0;                               /* smallest j attaining the minimum load */
+        for (int j = 1; j < M; ++j)
+            if (load[j] < load[best]) best = j;
+        assign[i] = best;
+        load[best] += T[i];
+    }
+}
+
+/* One round: enumerate EVERY candidate (i, k, u) and keep the lexicographic minimum of
+ * (v, i, k, u), u = -1 meaning "move".  Returns 1 and applies it when v < Lmax. */
+static int local_search_round(int n, int M, const int64_t* T, int32_t* assign, int64_t* load,
+                              ora_move* out)
+{
+    int jmax = 0;                                   /* smallest j attaining the maximum load */
+    for (int j = 1; j < M; ++j)
+        if (load[j] > load[jmax]) jmax = j;
+    const int64_t Lmax = load[jmax];
+
+    int have = 0;
+    int64_t bv = 0; int bi = -1, bk = -1, bu = -1;
+
+    for (int i = 0; i < n; ++i) {
+        if (assign[i] != jmax) continue;
+        /* u = -1 .. n-1; u = -1 stands for "move i", tried once for every other client k;
+         * u >= 0 is a swap with request u, whose client fixes k; needs d = T_i - T_u > 0 */
+        for (int u = -1; u < n; ++u) {
+            int k_first, k_last;
+            if (u < 0) { k_first = 0; k_last = M - 1; }
+            else {
+                if (assign[u] == jmax) continue;
+                k_first = k_last = assign[u];
+            }
+            for (int k = k_first; k <= k_last; ++k) {
+                if (k == jmax) continue;
+                int64_t d = (u < 0) ? T[i] : T[i] - T[u];
+                if (u >= 0 && d <= 0) continue;
+                int64_t a = Lmax - d, b = load[k] + d;
+                int64_t v = (a > b) ? a : b;
+                int better;
+                if (!have) better = 1;
+                else if (v != bv) better = v < bv;
+                else if (i != bi) better = i < bi;
+                else if (k != bk) better = k < bk;
+                else better = u < bu;
+                if (better) { have = 1; bv = v; bi = i; bk = k; bu = u; }
+            }
+        }
+    }
+    if (!have || bv >= Lmax) {
+        out->i = -1; out->u = -1; out->k = -1; out->v = Lmax;
+        return 0;
+    }
+    int64_t d = (bu < 0) ? T[bi] : T[bi] - T[bu];
+    assign[bi] = bk;
+    if (bu >= 0) assign[bu] = jmax;
+    load[jmax] -= d;
+    load[bk]   += d;
+    out->i = bi; out->u = bu; out->k = bk; out->v = bv;
+    return 1;
+}
+
+int ora_local_search(int n, int M, const int64_t* T, int32_t* assign, int64_t* load,
+                     int rounds, ora_move* log)
+{
+    int applied = 0;
+    for (int r = 0; r < rounds; ++r) {
+        ora_move mv;
+        int ok = local_search_round(n, M, T, assign, load, &mv);
+        if (log) log[r] = mv;
+        if (ok) { ++applied; continue; }
+        /* a no-op round leaves the state unchanged, so every later round is the same no-op */
+        if (log) for (int s = r + 1; s < rounds; ++s) log[s] = mv;
+        break;
+    }
+    return applied;
+}
+
+/* ------------------------------------------------------------------------- */
+/* Lower bounds, Eq. 31-32                                                    */
+/* ------------------------------------------------------------------------- */
+
+static int64_t ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
+
+void ora_lower_bound(int n, int M, int cap, const uint32_t* p, const uint32_t* o,
+                     const ora_cost* c, ora_lb* out)
+{
+    const int64_t ap = c->prefill_fixed_us, bp = c->prefill_per_token_us;
+    const int64_t ad = c->decode_fixed_us,  bd = c->decode_per_seq_us, q = c->decode_kv_div;
+
+    /* --- packing bound: the optimum of Eq. 26 is at least the mean load, the largest
+     *     item, and the two smallest of the M+1 largest items together --- */
+    int64_t* T = (int64_t*)malloc(sizeof(int64_t) * (size_t)(n > 0 ? n : 1));
+    int32_t* order = (int32_t*)malloc(sizeof(int32_t) * (size_t)(n > 0 ? n : 1));
+    ora_estimate(n, p, o, c, T);
+    ora_order(n, T, order);
+    int64_t sumT = 0, maxT = 0;
+    for (int i = 0; i < n; ++i) { sumT += T[i]; if (T[i] > maxT) maxT = T[i]; }
+    int64_t pairT = (n > M) ? T[order[M - 1]] + T[order[M]] : 0;
+    int64_t lb = ceil_div(sumT, M);
+    if (maxT > lb) lb = maxT;
+    if (pairT > lb) lb = pairT;
+    out->lb_pack = lb; out->sum_T = sumT; out->max_T = maxT; out->pair_T = pairT;
+
+    /* --- simulation bound T^LB = t^p* + t^d*: prefill work and decode work taken as two
+     *     separate groups, each with the fewest possible iterations --- */
+    int64_t P = 0, O = 0, K = 0, chain = 0;
+    for (int i = 0; i < n; ++i) {
+        P += p[i];
+        O += o[i];
+        int64_t alone = ap + bp * (int64_t)p[i];    /* request i served alone on a client */
+        for (int64_t s = 0; s < (int64_t)o[i]; ++s) {
+            K += (int64_t)p[i] + s;                 /* KV tokens attended by decode step s */
+            alone += ad + bd + ((int64_t)p[i] + s) / q;
+        }
+        if (alone > chain) chain = alone;
+    }
+    /* every prefill iteration admits at most cap prompts and pays a_p once */
+    int64_t tp_star = ap * ceil_div(n, cap) + bp * P;
+    /* every decode iteration advances at most cap requests; floor(S/q) > S/q - 1 */
+    int64_t td_q = q * ((ad - 1) * ceil_div(O, cap) + bd * O) + K;      /* q * t^d*  */
+    int64_t work = ceil_div(q * tp_star + td_q, q * (int64_t)M);        /* mean client time */
+    out->tp_star_us = ceil_div(tp_star, M);
+    out->td_star_us = ceil_div(td_q, q * (int64_t)M);
+    out->chain_us   = chain;
+    out->lb_sim_us  = (work > chain) ? work : chain;
+    free(T); free(order);
+}
+
+/* ------------------------------------------------------------------------- */
+/* Online part: Algorithm 1 (queue order) and the iteration simulator         */
+/* ------------------------------------------------------------------------- */
+
+void ora_queue_build(int n, int M, const int32_t* assign, const uint32_t* p, const uint32_t* o,
+                     int mode, int32_t* q_off, int32_t* q_req)
+{
+    int pos = 0;
+    ora_keyed* a = (ora_keyed*)malloc(sizeof(ora_keyed) * (size_t)(n > 0 ? n : 1));
+    for (int j = 0; j < M; ++j) {
+        q_off[j] = pos;
+        int m = 0;
+        for (int i = 0; i < n; ++i)
+            if (assign[i] == j) {
+                /* SORTED: longest N^p + N^d first; FCFS: arrival (index) order */
+                a[m].key = (mode == ORA_QUEUE_SORTED) ? (int64_t)p[i] + (int64_t)o[i] : 0;
+                a[m].idx = i;
+                ++m;
+            }
+        qsort(a, (size_t)m, sizeof(ora_keyed), cmp_key_desc_idx_asc);
+        for (int r = 0; r < m; ++r) q_req[pos++] = a[r].idx;
+    }
+    q_off[M] = pos;
+    free(a);
+}
+
+#define ORA_HASH_INIT  0xCBF29CE484222325ull
+#define ORA_HASH_BASE  0x9E3779B97F4A7C15ull
+#define ORA_HASH_W0    0xBF58476D1CE4E5B9ull
+#define ORA_HASH_W1    0x94D049BB133111EBull
+#define ORA_HASH_W2    0xD6E8FEB86659FD93ull
+#define ORA_HASH_W3    0xA0761D6478BD642Full
+#define ORA_HASH_W4    0xE7037ED1A0B428DBull
+
+typedef struct { int64_t kv, rem, total; } ora_running;
+
+void ora_simulate_client(int qn, const int32_t* q_req, const uint32_t* p, const uint32_t* o,
+                         const ora_cost* c, int cap, int64_t kv_budget, uint32_t lambda_q16,
+                         uint32_t max_iters, ora_client* res, ora_rec* trace, int64_t trace_cap)
+{
+    const int64_t ap = c->prefill_fixed_us, bp = c->prefill_per_token_us;
+    const int64_t ad = c->decode_fixed_us,  bd = c->decode_per_seq_us, q = c->decode_kv_div;
+
+    ora_running* R = (ora_running*)malloc(sizeof(ora_running) * (size_t)(cap > 0 ? cap : 1));
+    int nR = 0;                 /* |R| */
+    int head = 0;               /* next queue position */
+    int64_t reserved = 0;       /* sum over R of (p + o) */
+    int64_t t = 0, busy = 0, Cd = 0;
+    uint64_t hash = ORA_HASH_INIT, pw = 1;
+    uint32_t n_pre = 0, n_dec = 0;
+    uint64_t iters = 0;
+    int32_t status = 0;
+
+    while (nR > 0 || head < qn) {
+        /* 1. candidates: a prefix of the queue, no skipping */
+        int nA = 0; int64_t sumP = 0, sumTot = 0;
+        while (head + nA < qn && nR + nA < cap) {
+            int i = q_req[head + nA];
+            int64_t tot = (int64_t)p[i] + (int64_t)o[i];
+            if (reserved + sumTot + tot > kv_budget) break;
+            sumTot += tot; sumP += p[i]; ++nA;
+        }
+        /* 2. decide */
+        int prefill;
+        int64_t Cp = ap + bp * sumP;
+        if (nA == 0) prefill = 0;
+        else if (nR == 0) prefill = 1;
+        else prefill = ((uint64_t)lambda_q16 * (uint64_t)Cd) > (((uint64_t)Cp) << 16);
+        if (nA == 0 && nR == 0) { status |= 1; break; }     /* head can never fit: invalid input */
+
+        if (iters == (uint64_t)max_iters) { status |= 1; break; }
+
+        ora_rec rec;
+        int64_t dur;
+        if (prefill) {
+            /* 3. prefill iteration: running decodes stall (PD competition) */
+            dur = Cp;
+            busy += dur * nA;
+            rec.dur_us = (uint32_t)dur; rec.kind_n = 0x80000000u | (uint32_t)nA;
+            rec.tokens = (uint32_t)sumP; rec.aux = (uint32_t)head;
+            for (int a = 0; a < nA; ++a) {
+                int i = q_req[head + a];
+                R[nR].kv = p[i]; R[nR].rem = o[i]; R[nR].total = (int64_t)p[i] + (int64_t)o[i];
+                ++nR;
+            }
+            head += nA;
+            reserved += sumTot;
+            Cd = 0;
+            ++n_pre;
+        } else {
+            /* 4. decode iteration: one token for every running request */
+            int64_t B = nR, S = 0;
+            for (int s = 0; s < nR; ++s) S += R[s].kv;       /* KV lengths before the step */
+            dur = ad + bd * B + S / q;
+            busy += dur * B;
+            int f = 0, w = 0;
+            for (int s = 0; s < nR; ++s) {
+                R[s].kv += 1; R[s].rem -= 1;
+                if (R[s].rem == 0) { reserved -= R[s].total; ++f; }
+                else R[w++] = R[s];
+            }
+            nR = w;
+            Cd += dur;
+            if (Cd > 2147483647ll) Cd = 2147483647ll;
+            rec.dur_us = (uint32_t)dur; rec.kind_n = (uint32_t)B;
+            rec.tokens = (uint32_t)S; rec.aux = (uint32_t)f;
+            ++n_dec;
+        }
+        /* 5. clock, trace, hash */
+        t += dur;
+        if ((int64_t)iters < trace_cap) { if (trace) trace[iters] = rec; }
+        else if (trace) status |= 2;
+        uint64_t g = ORA_HASH_W0 * rec.dur_us + ORA_HASH_W1 * rec.kind_n
+                   + ORA_HASH_W2 * rec.tokens + ORA_HASH_W3 * rec.aux + ORA_HASH_W4;
+        hash += g * pw;
+        pw *= ORA_HASH_BASE;
+        ++iters;
+        if (t >= ((int64_t)1 << 39)) { status |= 1; break; }
+    }
+    res->makespan_us = t;
+    res->busy_slot_us = busy;
+    res->n_prefill_iters = n_pre;
+    res->n_decode_iters = n_dec;
+    res->trace_hash = hash;
+    res->status = status;
+    free(R);
+}

@@ -1,0 +1,79 @@
+"""The five synthetic workloads (sizes, length distributions, seeds, multipliers).
+
+Pure description of inputs: no scheduling arithmetic lives here.  Every number
+is an input to the method (request-table shape, client count, caps, the
+integer-microsecond cost coefficients, the Q16.16 multipliers to sweep).
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass, field
+from typing import List, Tuple
+
+import numpy as np
+
+from .gen import LengthDist, batch_lengths
+
+# (prefill_fixed_us, prefill_per_token_us, decode_fixed_us, decode_per_seq_us,
+#  decode_kv_div, est_per_prompt_token, est_per_output_token)
+COST_MODEL: Tuple[int, ...] = (20000, 40, 15000, 300, 16, 40, 350)
+
+SHORT_P = LengthDist(120.0, 0.4, 16, 512)
+SHORT_O = LengthDist(130.0, 0.5, 8, 512)
+LONG_P = LengthDist(300.0, 0.6, 16, 4096)
+LONG_O = LengthDist(250.0, 0.7, 8, 2048)
+
+LAMBDA_ONE = 1 << 16            # 1.0 in Q16.16
+LAMBDA_PREFILL_FIRST = 0xFFFFFFFF
+LAMBDA_NEVER_PREEMPT = 0
+
+
+@dataclass(frozen=True)
+class Workload:
+    name: str
+    seeds: Tuple[int, ...]
+    n_req: int
+    n_clients: int
+    batch_cap: int
+    kv_budget: int
+    dist_p: LengthDist
+    dist_o: LengthDist
+    lambdas_q16: Tuple[int, ...] = (LAMBDA_ONE,)
+    ls_rounds: int = 0
+    cost_model: Tuple[int, ...] = COST_MODEL
+
+    @property
+    def n_inst(self) -> int:
+        return len(self.seeds)
+
+    def subset(self, first: int, count: int) -> "Workload":
+        """The same workload restricted to instances [first, first+count)."""
+        return Workload(self.name, self.seeds[first:first + count], self.n_req, self.n_clients,
+                        self.batch_cap, self.kv_budget, self.dist_p, self.dist_o,
+                        self.lambdas_q16, self.ls_rounds, self.cost_model)
+
+    def lengths(self):
+        """uint32 tables p, o of shape [n_inst][n_req]."""
+        return batch_lengths(self.seeds, self.n_req, self.dist_p, self.dist_o)
+
+
+def workload(name: str) -> Workload:
+    if name == "c0":      # one small instance
+        return Workload("c0", (0,), 200, 4, 16, 32768, SHORT_P, SHORT_O)
+    if name == "c1":      # one math-QA-batch-shaped instance
+        return Workload("c1", (1,), 1300, 8, 32, 65536, SHORT_P, SHORT_O)
+    if name == "c2":      # 100-case study
+        return Workload("c2", tuple(range(100, 200)), 1300, 8, 32, 65536, SHORT_P, SHORT_O)
+    if name == "c3":      # multiplier sweep, 64 values k/16, 20 local-search rounds
+        return Workload("c3", tuple(range(100, 200)), 1300, 8, 32, 65536, SHORT_P, SHORT_O,
+                        tuple(k * 4096 for k in range(1, 65)), 20)
+    if name == "c4":      # scale-out stress
+        return Workload("c4", tuple(range(1000, 2024)), 20000, 64, 128, 262144, LONG_P, LONG_O,
+                        (LAMBDA_ONE,), 100)
+    raise KeyError(name)
+
+
+def shard(n_units: int, world_size: int, rank: int) -> Tuple[int, int]:
+    """Contiguous block [first, first+count) of n_units owned by this rank (sizes differ by <= 1)."""
+    base, extra = divmod(n_units, world_size)
+    first = rank * base + min(rank, extra)
+    return first, base + (1 if rank < extra else 0)
