@@ -1,0 +1,191 @@
+/*
+ * hos -- batched evaluation of the hybrid offline-online LLM-inference scheduler
+ * of arXiv 2502.15763 on one NVIDIA B200 (sm_100a).
+ *
+ * C ABI.  Conventions shared by every call:
+ *   - `hos_batch`, `hos_cost_model` and every `const T*` marked HOST are read on
+ *     the host during the call.  Every other pointer is DEVICE memory owned by
+ *     the caller; the library allocates nothing, keeps no state between calls,
+ *     enqueues its kernels on `stream` (a cudaStream_t passed as void*) and
+ *     returns without synchronising.  Results are valid once `stream` has
+ *     reached the point of the call's return.
+ *   - Tables are row-major.  A batch holds `n_inst` independent scheduling
+ *     instances of the same shape: `n_req` requests, `n_clients` clients, each
+ *     client with `batch_cap` slots and `kv_budget` KV tokens.
+ *   - Return value: HOS_OK or a negative HOS_E_* code found on the host before
+ *     anything is enqueued (bad sizes, null pointers, workspace too small,
+ *     unsupported shape, CUDA launch error).  Problems that depend on the data
+ *     (a zero length, a request larger than the KV budget, an iteration limit,
+ *     a trace buffer that is too small) never trap: they set bits of the
+ *     per-unit `status` word on the device and the unit's results are zeroed
+ *     (HOS_ST_INVALID) or truncated (HOS_ST_LIMIT, HOS_ST_TRACE).
+ *   - Workspaces are scratch: contents are undefined before and after a call;
+ *     base must be 256-byte aligned.  Two calls that share a workspace or an
+ *     output buffer must be ordered on the stream.
+ *   - Shape limits of this build: n_clients <= 256, batch_cap <= 256,
+ *     n_req <= 24576, kv_budget < 2^31, estimated times T_i < 2^32.
+ */
+#ifndef HOS_H
+#define HOS_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+enum {
+    HOS_OK            =  0,
+    HOS_E_INVALID     = -1,   /* null pointer, non-positive size, inconsistent arguments        */
+    HOS_E_WORKSPACE   = -2,   /* workspace smaller than hos_*_workspace_bytes, or misaligned     */
+    HOS_E_CUDA        = -3,   /* a CUDA runtime call failed (see cudaGetLastError)               */
+    HOS_E_UNSUPPORTED = -4    /* shape outside the limits listed above                           */
+};
+
+/* bits of the per-unit device status words */
+enum {
+    HOS_ST_LIMIT   = 1,       /* iteration limit or 2^39 us clock limit reached; results partial */
+    HOS_ST_TRACE   = 2,       /* more iterations than trace slots; extra records dropped         */
+    HOS_ST_INVALID = 4        /* instance data invalid (p_i = 0, o_i = 0, p_i + o_i > kv_budget,
+                                 T_i >= 2^32, assignment outside [0, n_clients))                */
+};
+
+enum { HOS_QUEUE_SORTED = 0, HOS_QUEUE_FCFS = 1 };
+
+/* Integer-microsecond cost model.  The paper profiles both stage times as affine in the
+ * token counts (Numerical Experiment, "Experiment settings"); the KV term is this build's
+ * workload definition.  prefill iteration = prefill_fixed_us + prefill_per_token_us * sum p;
+ * decode iteration = decode_fixed_us + decode_per_seq_us * B + floor(sum KV / decode_kv_div);
+ * estimated request time T_i = est_per_prompt_token * p_i + est_per_output_token * o_i.
+ * Requires decode_fixed_us >= 1, decode_kv_div >= 1, and both iteration durations < 2^31
+ * for any admissible batch. */
+typedef struct hos_cost_model {
+    uint32_t prefill_fixed_us, prefill_per_token_us;
+    uint32_t decode_fixed_us, decode_per_seq_us, decode_kv_div;
+    uint32_t est_per_prompt_token, est_per_output_token;
+} hos_cost_model;
+
+/* HOST struct; p and o are DEVICE tables [n_inst][n_req] of prompt lengths N^p_i and output
+ * lengths N^d_i (both >= 1, Notation table of the paper). */
+typedef struct hos_batch {
+    int32_t n_inst, n_req, n_clients, batch_cap;
+    int64_t kv_budget;
+    const uint32_t* p;
+    const uint32_t* o;
+} hos_batch;
+
+/* One local-search round: request i left the critical client for client k; u >= 0 came back
+ * in exchange (swap), u = -1 is a plain move; v = max of the two changed loads afterwards.
+ * A round that found no improving step is {-1, -1, -1, current maximum load}. */
+typedef struct hos_ls_move { int32_t i, u, k; int64_t v; } hos_ls_move;
+
+/* Lower bounds of one instance.  lb_pack (units of T) bounds the optimum of the offline
+ * model, Eq. 26-30: max(ceil(sum_T / M), max_T, pair_T), pair_T = T_(M) + T_(M+1) when
+ * n_req > M.  lb_sim_us bounds every simulated makespan: max(work, chain_us), where work
+ * is Eq. 32's t^p* + t^d* for M clients (tp_star_us, td_star_us are the two terms, each
+ * rounded up) and chain_us is the longest request served alone. */
+typedef struct hos_lb {
+    int64_t lb_pack, sum_T, max_T, pair_T;
+    int64_t lb_sim_us, tp_star_us, td_star_us, chain_us;
+} hos_lb;
+
+typedef struct hos_client_result {
+    int64_t  makespan_us;        /* this client's clock when its last request retired        */
+    int64_t  busy_slot_us;       /* sum over iterations of duration * requests advanced       */
+    uint32_t n_prefill_iters, n_decode_iters;
+    uint64_t trace_hash;         /* polynomial hash of the trace, produced with or without it */
+    double   utilisation;        /* busy_slot_us / (batch_cap * makespan of the simulation)   */
+} hos_client_result;
+
+typedef struct hos_sim_result {
+    int64_t makespan_us;         /* max over clients                                          */
+    int64_t busy_slot_us;        /* sum over clients                                          */
+    double  utilisation;         /* busy / (n_clients * batch_cap * makespan)                 */
+    double  tokens_per_s;        /* sum o_i * 1e6 / makespan                                  */
+} hos_sim_result;
+
+/* One iteration of one client.  prefill: {duration, 2^31 | admitted requests, sum of their
+ * prompt tokens, queue position of the first admitted}.  decode: {duration, B, sum of KV
+ * lengths before the step, requests retired by the step}. */
+typedef struct hos_iter_rec { uint32_t dur_us, kind_n, tokens, aux; } hos_iter_rec;
+
+/*
+ * Offline request scheduling, Eq. 26-30 (Minimizing-Makespan Bin Packing): T_i, per-instance
+ * order by (T descending, index ascending), longest-first list scheduling onto the least
+ * loaded client (ties: lowest client), then `ls_rounds` rounds of local search, each applying
+ * the single move or pairwise swap off the most loaded client that minimises
+ * (v, i, k, u) lexicographically, if v is below the current maximum load.
+ *   assign         [n_inst][n_req]     out  client of every request (-1 in invalid instances)
+ *   load           [n_inst][n_clients] out  sum of T_i per client
+ *   makespan_est   [n_inst]            out  max_j load
+ *   rounds_applied [n_inst]            out  local-search rounds that changed the assignment
+ *   ls_log         [n_inst][ls_rounds] out, nullable
+ *   status         [n_inst]            out  0 or HOS_ST_INVALID
+ */
+int hos_offline_pack(const hos_batch* batch, const hos_cost_model* cm, int ls_rounds,
+                     int32_t* assign, int64_t* load, int64_t* makespan_est,
+                     int32_t* rounds_applied, hos_ls_move* ls_log, int32_t* status,
+                     void* ws, size_t ws_bytes, void* stream);
+
+/*
+ * Local-search rounds only, from given assignments (same rule as in hos_offline_pack).
+ * Every instance carries `n_copies` independent assignments (for instance one per
+ * multiplier value of a sweep); request data are shared by the copies.
+ *   assign [n_inst][n_copies][n_req] in/out;  load, makespan_est, rounds_applied, ls_log
+ *   are laid out [n_inst][n_copies][...];  load is recomputed from assign on entry.
+ *   status [n_inst] out.
+ */
+int hos_local_search(const hos_batch* batch, const hos_cost_model* cm, int n_copies, int ls_rounds,
+                     int32_t* assign, int64_t* load, int64_t* makespan_est,
+                     int32_t* rounds_applied, hos_ls_move* ls_log, int32_t* status,
+                     void* ws, size_t ws_bytes, void* stream);
+
+/* Theoretical lower bounds, Eq. 31-32 and the relaxations of Eq. 26-30.  out [n_inst],
+ * status [n_inst]. */
+int hos_lower_bound(const hos_batch* batch, const hos_cost_model* cm, hos_lb* out, int32_t* status,
+                    void* ws, size_t ws_bytes, void* stream);
+
+/*
+ * Online scheduling.  Queues: the requests of each client in the order of Algorithm 1
+ * (N^p + N^d descending, ties by index; HOS_QUEUE_FCFS: index order).  Then one simulation
+ * per (instance, multiplier, client): every iteration either prefills the longest
+ * admissible queue prefix (batch cap and KV budget, p+o reserved per request) or decodes one
+ * token for every running request; with candidates and a non-empty batch it prefills iff
+ * lambda * C_d > C_p (Section "Online requests and iteration scheduling": C_p = cost of
+ * that prefill, C_d = decode time waited since the last prefill; lambda = 1.0 is the
+ * paper's rule), lambda in Q16.16.
+ *   assign     [n_inst][n_req]                  in
+ *   lambda_q16 [n_lambda]                       in (DEVICE)
+ *   cres       [n_inst][n_lambda][n_clients]    out
+ *   sres       [n_inst][n_lambda]               out
+ *   status     [n_inst][n_lambda][n_clients]    out  HOS_ST_* bits
+ *   trace      nullable; with trace_off [n_inst*n_lambda*n_clients + 1] (DEVICE, ascending):
+ *              unit x = (inst*n_lambda + l)*n_clients + c writes its iterations, in order, to
+ *              trace[trace_off[x] .. trace_off[x+1]).  Sizes come from a first call with
+ *              trace = NULL (n_prefill_iters + n_decode_iters) and hos_trace_offsets, or from
+ *              any upper bound the caller chooses.
+ *   max_iters  at most this many iterations per client (then HOS_ST_LIMIT).
+ */
+int hos_online_simulate(const hos_batch* batch, const int32_t* assign, const hos_cost_model* cm,
+                        const uint32_t* lambda_q16, int n_lambda, int queue_order, uint32_t max_iters,
+                        hos_client_result* cres, hos_sim_result* sres,
+                        hos_iter_rec* trace, const int64_t* trace_off, int32_t* status,
+                        void* ws, size_t ws_bytes, void* stream);
+
+/* trace_off[0] = 0, trace_off[x+1] = trace_off[x] + iterations of unit x (exclusive scan of
+ * n_prefill_iters + n_decode_iters over cres[0..n_units)).  The trace protocol of
+ * hos_online_simulate; no counterpart in the paper beyond "the Gantt chart is recorded". */
+int hos_trace_offsets(const hos_client_result* cres, int64_t n_units, int64_t* trace_off,
+                      void* stream);
+
+size_t hos_offline_workspace_bytes(const hos_batch* batch, int n_copies, int ls_rounds);
+size_t hos_lower_bound_workspace_bytes(const hos_batch* batch);
+size_t hos_online_workspace_bytes(const hos_batch* batch, int n_lambda);
+
+const char* hos_strerror(int code);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* HOS_H */

@@ -1,0 +1,250 @@
+"""ctypes binding of libhos.so: same names as the C entry points, argument marshalling only.
+
+Every array argument is a torch CUDA tensor (torch supplies device memory and
+the current stream); every result is a torch CUDA tensor.  Structured results
+are returned as uint8 tensors of shape [..., sizeof(struct)] whose host copy can
+be viewed with the numpy dtypes below (`view_struct`).
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Optional, Sequence
+
+import numpy as np
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+
+HOS_QUEUE_SORTED, HOS_QUEUE_FCFS = 0, 1
+HOS_ST_LIMIT, HOS_ST_TRACE, HOS_ST_INVALID = 1, 2, 4
+
+LS_MOVE_DTYPE = np.dtype([("i", "<i4"), ("u", "<i4"), ("k", "<i4"), ("v", "<i8")], align=True)
+LB_DTYPE = np.dtype([(n, "<i8") for n in ("lb_pack", "sum_T", "max_T", "pair_T", "lb_sim_us",
+                                           "tp_star_us", "td_star_us", "chain_us")])
+CLIENT_RESULT_DTYPE = np.dtype([("makespan_us", "<i8"), ("busy_slot_us", "<i8"),
+                                ("n_prefill_iters", "<u4"), ("n_decode_iters", "<u4"),
+                                ("trace_hash", "<u8"), ("utilisation", "<f8")])
+SIM_RESULT_DTYPE = np.dtype([("makespan_us", "<i8"), ("busy_slot_us", "<i8"),
+                             ("utilisation", "<f8"), ("tokens_per_s", "<f8")])
+ITER_REC_DTYPE = np.dtype([("dur_us", "<u4"), ("kind_n", "<u4"), ("tokens", "<u4"), ("aux", "<u4")])
+
+_SYMBOLS = ("hos_offline_pack", "hos_local_search", "hos_lower_bound", "hos_online_simulate",
+            "hos_trace_offsets", "hos_offline_workspace_bytes", "hos_lower_bound_workspace_bytes",
+            "hos_online_workspace_bytes", "hos_strerror")
+
+
+class HosError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__(f"{where}: {hos_strerror(code)} ({code})")
+
+
+class _CostModel(C.Structure):
+    _fields_ = [(n, C.c_uint32) for n in (
+        "prefill_fixed_us", "prefill_per_token_us", "decode_fixed_us", "decode_per_seq_us",
+        "decode_kv_div", "est_per_prompt_token", "est_per_output_token")]
+
+
+class _Batch(C.Structure):
+    _fields_ = [("n_inst", C.c_int32), ("n_req", C.c_int32), ("n_clients", C.c_int32),
+                ("batch_cap", C.c_int32), ("kv_budget", C.c_int64),
+                ("p", C.c_void_p), ("o", C.c_void_p)]
+
+
+_lib = None
+
+
+def lib_path() -> str:
+    return os.path.join(_PKG, "libhos.so")
+
+
+def lib():
+    """Load libhos.so (building it first if the sources are newer).  Raises if it cannot be had."""
+    global _lib
+    if _lib is None:
+        from . import _build
+        path = _build.build() if _build.is_stale() else lib_path()
+        L = C.CDLL(path)
+        for name in ("hos_offline_workspace_bytes", "hos_lower_bound_workspace_bytes",
+                     "hos_online_workspace_bytes"):
+            getattr(L, name).restype = C.c_size_t
+        L.hos_strerror.restype = C.c_char_p
+        for name in ("hos_offline_pack", "hos_local_search", "hos_lower_bound",
+                     "hos_online_simulate", "hos_trace_offsets"):
+            getattr(L, name).restype = C.c_int
+        _lib = L
+    return _lib
+
+
+def exported_symbols() -> Sequence[str]:
+    return _SYMBOLS
+
+
+def hos_strerror(code: int) -> str:
+    return lib().hos_strerror(C.c_int(code)).decode()
+
+
+def _torch():
+    import torch
+    if not torch.cuda.is_available():
+        raise RuntimeError("paper_2502_15763_b200 needs a CUDA device; there is no CPU fallback")
+    return torch
+
+
+def _dev(t, dtype, what: str):
+    torch = _torch()
+    if not (isinstance(t, torch.Tensor) and t.is_cuda and t.dtype == dtype and t.is_contiguous()):
+        raise TypeError(f"{what}: expected a contiguous CUDA tensor of {dtype}")
+    return t
+
+
+def _ptr(t) -> C.c_void_p:
+    return C.c_void_p(t.data_ptr() if t is not None else None)
+
+
+def _stream():
+    return C.c_void_p(_torch().cuda.current_stream().cuda_stream)
+
+
+def _batch(p, o, n_clients: int, batch_cap: int, kv_budget: int) -> _Batch:
+    torch = _torch()
+    # uint32 tables travel as int32 tensors (same bits)
+    p = _dev(p, torch.int32, "p")
+    o = _dev(o, torch.int32, "o")
+    if p.dim() != 2 or p.shape != o.shape:
+        raise ValueError("p and o must be [n_inst][n_req] tables of the same shape")
+    return _Batch(p.shape[0], p.shape[1], n_clients, batch_cap, kv_budget, p.data_ptr(), o.data_ptr())
+
+
+def _cost(cm: Sequence[int]) -> _CostModel:
+    return _CostModel(*[int(x) for x in cm])
+
+
+def _workspace(nbytes: int, like):
+    torch = _torch()
+    return torch.empty(max(int(nbytes), 256), dtype=torch.uint8, device=like.device)
+
+
+def _check(rc: int, where: str):
+    if rc != 0:
+        raise HosError(rc, where)
+
+
+def view_struct(t, dtype: np.dtype) -> np.ndarray:
+    """Host copy of a [..., sizeof] uint8 result tensor viewed as a structured numpy array."""
+    a = t.detach().cpu().numpy()
+    return a.view(dtype).reshape(a.shape[:-1])
+
+
+def hos_offline_pack(p, o, n_clients: int, batch_cap: int, kv_budget: int, cost_model, ls_rounds: int = 0,
+                     want_log: bool = False, ws=None):
+    """Eq. 26-30: estimate, order, LPT, `ls_rounds` local-search rounds.  Returns a dict of tensors."""
+    torch = _torch()
+    b = _batch(p, o, n_clients, batch_cap, kv_budget)
+    cm = _cost(cost_model)
+    L = lib()
+    need = L.hos_offline_workspace_bytes(C.byref(b), C.c_int(1), C.c_int(ls_rounds))
+    ws = ws if ws is not None else _workspace(need, p)
+    dev = p.device
+    assign = torch.empty((b.n_inst, b.n_req), dtype=torch.int32, device=dev)
+    load = torch.empty((b.n_inst, n_clients), dtype=torch.int64, device=dev)
+    makespan = torch.empty((b.n_inst,), dtype=torch.int64, device=dev)
+    applied = torch.empty((b.n_inst,), dtype=torch.int32, device=dev)
+    status = torch.empty((b.n_inst,), dtype=torch.int32, device=dev)
+    log = (torch.empty((b.n_inst, ls_rounds, LS_MOVE_DTYPE.itemsize), dtype=torch.uint8, device=dev)
+           if want_log and ls_rounds > 0 else None)
+    rc = L.hos_offline_pack(C.byref(b), C.byref(cm), C.c_int(ls_rounds), _ptr(assign), _ptr(load),
+                            _ptr(makespan), _ptr(applied), _ptr(log), _ptr(status), _ptr(ws),
+                            C.c_size_t(ws.numel()), _stream())
+    _check(rc, "hos_offline_pack")
+    return dict(assign=assign, load=load, makespan_est=makespan, rounds_applied=applied, ls_log=log,
+                status=status)
+
+
+def hos_local_search(p, o, n_clients: int, batch_cap: int, kv_budget: int, cost_model, assign,
+                     ls_rounds: int, want_log: bool = False, ws=None):
+    """Local-search rounds from given assignments [n_inst][n_copies][n_req] (modified in place)."""
+    torch = _torch()
+    b = _batch(p, o, n_clients, batch_cap, kv_budget)
+    cm = _cost(cost_model)
+    assign = _dev(assign, torch.int32, "assign")
+    if assign.dim() != 3 or assign.shape[0] != b.n_inst or assign.shape[2] != b.n_req:
+        raise ValueError("assign must be [n_inst][n_copies][n_req]")
+    n_copies = assign.shape[1]
+    L = lib()
+    need = L.hos_offline_workspace_bytes(C.byref(b), C.c_int(n_copies), C.c_int(ls_rounds))
+    ws = ws if ws is not None else _workspace(need, p)
+    dev = p.device
+    load = torch.empty((b.n_inst, n_copies, n_clients), dtype=torch.int64, device=dev)
+    makespan = torch.empty((b.n_inst, n_copies), dtype=torch.int64, device=dev)
+    applied = torch.empty((b.n_inst, n_copies), dtype=torch.int32, device=dev)
+    status = torch.empty((b.n_inst,), dtype=torch.int32, device=dev)
+    log = (torch.empty((b.n_inst, n_copies, ls_rounds, LS_MOVE_DTYPE.itemsize), dtype=torch.uint8, device=dev)
+           if want_log and ls_rounds > 0 else None)
+    rc = L.hos_local_search(C.byref(b), C.byref(cm), C.c_int(n_copies), C.c_int(ls_rounds), _ptr(assign),
+                            _ptr(load), _ptr(makespan), _ptr(applied), _ptr(log), _ptr(status), _ptr(ws),
+                            C.c_size_t(ws.numel()), _stream())
+    _check(rc, "hos_local_search")
+    return dict(assign=assign, load=load, makespan_est=makespan, rounds_applied=applied, ls_log=log,
+                status=status)
+
+
+def hos_lower_bound(p, o, n_clients: int, batch_cap: int, kv_budget: int, cost_model, ws=None):
+    """Eq. 31-32 and the packing relaxations; returns {'lb': uint8 [n_inst][64], 'status': ...}."""
+    torch = _torch()
+    b = _batch(p, o, n_clients, batch_cap, kv_budget)
+    cm = _cost(cost_model)
+    L = lib()
+    need = L.hos_lower_bound_workspace_bytes(C.byref(b))
+    ws = ws if ws is not None else _workspace(need, p)
+    out = torch.empty((b.n_inst, LB_DTYPE.itemsize), dtype=torch.uint8, device=p.device)
+    status = torch.empty((b.n_inst,), dtype=torch.int32, device=p.device)
+    rc = L.hos_lower_bound(C.byref(b), C.byref(cm), _ptr(out), _ptr(status), _ptr(ws),
+                           C.c_size_t(ws.numel()), _stream())
+    _check(rc, "hos_lower_bound")
+    return dict(lb=out, status=status)
+
+
+def hos_trace_offsets(cres, n_units: Optional[int] = None):
+    """Exclusive scan of the per-client iteration counts -> int64 [n_units + 1]."""
+    torch = _torch()
+    cres = _dev(cres, torch.uint8, "cres")
+    n = int(cres.numel() // CLIENT_RESULT_DTYPE.itemsize) if n_units is None else int(n_units)
+    off = torch.empty((n + 1,), dtype=torch.int64, device=cres.device)
+    _check(lib().hos_trace_offsets(_ptr(cres), C.c_int64(n), _ptr(off), _stream()), "hos_trace_offsets")
+    return off
+
+
+def hos_online_simulate(p, o, n_clients: int, batch_cap: int, kv_budget: int, cost_model, assign,
+                        lambda_q16, queue_order: int = HOS_QUEUE_SORTED, max_iters: int = 0x7FFFFFFF,
+                        trace=None, trace_off=None, ws=None):
+    """Queues + iteration simulation for every (instance, multiplier, client).
+
+    trace: None, or a uint8 tensor [n_records][16] with trace_off (int64 [n_units + 1]).
+    """
+    torch = _torch()
+    b = _batch(p, o, n_clients, batch_cap, kv_budget)
+    cm = _cost(cost_model)
+    assign = _dev(assign, torch.int32, "assign")
+    if tuple(assign.shape) != (b.n_inst, b.n_req):
+        raise ValueError("assign must be [n_inst][n_req]")
+    lambda_q16 = _dev(lambda_q16, torch.int32, "lambda_q16")       # uint32 bits
+    n_lambda = int(lambda_q16.numel())
+    L = lib()
+    need = L.hos_online_workspace_bytes(C.byref(b), C.c_int(n_lambda))
+    ws = ws if ws is not None else _workspace(need, p)
+    dev = p.device
+    cres = torch.empty((b.n_inst, n_lambda, n_clients, CLIENT_RESULT_DTYPE.itemsize), dtype=torch.uint8, device=dev)
+    sres = torch.empty((b.n_inst, n_lambda, SIM_RESULT_DTYPE.itemsize), dtype=torch.uint8, device=dev)
+    status = torch.empty((b.n_inst, n_lambda, n_clients), dtype=torch.int32, device=dev)
+    if trace is not None:
+        trace = _dev(trace, torch.uint8, "trace")
+        trace_off = _dev(trace_off, torch.int64, "trace_off")
+        if trace_off.numel() != b.n_inst * n_lambda * n_clients + 1:
+            raise ValueError("trace_off must have n_units + 1 entries")
+    rc = L.hos_online_simulate(C.byref(b), _ptr(assign), C.byref(cm), _ptr(lambda_q16), C.c_int(n_lambda),
+                               C.c_int(queue_order), C.c_uint32(max_iters), _ptr(cres), _ptr(sres),
+                               _ptr(trace), _ptr(trace_off), _ptr(status), _ptr(ws),
+                               C.c_size_t(ws.numel()), _stream())
+    _check(rc, "hos_online_simulate")
+    return dict(cres=cres, sres=sres, status=status, ws=ws)

@@ -1,0 +1,215 @@
+// C-ABI layer: argument validation, workspace carving, kernel sequencing.
+#include <cuda_runtime.h>
+
+#include "hos.h"
+#include "hos_common.cuh"
+#include "hos_kernels.h"
+
+namespace {
+
+using namespace hos;
+
+constexpr size_t WS_ALIGN = 256;
+inline size_t up(size_t x) { return (x + WS_ALIGN - 1) & ~(WS_ALIGN - 1); }
+inline int pad4(int n) { return (n + 3) & ~3; }
+inline int bit_width_host(unsigned long long v) { int b = 0; while (v) { ++b; v >>= 1; } return b; }
+
+int check_batch(const hos_batch* b) {
+    if (!b || !b->p || !b->o) return HOS_E_INVALID;
+    if (b->n_inst < 1 || b->n_req < 1 || b->n_clients < 1 || b->batch_cap < 1 || b->kv_budget < 1)
+        return HOS_E_INVALID;
+    if (b->n_clients > MAX_CLIENTS || b->batch_cap > MAX_CAP || b->n_req > MAX_REQ ||
+        b->kv_budget >= (1ll << 31))
+        return HOS_E_UNSUPPORTED;
+    if ((long long)b->n_inst * (long long)pad4(b->n_req) >= (1ll << 40)) return HOS_E_UNSUPPORTED;
+    return HOS_OK;
+}
+
+int check_cost(const hos_cost_model* cm, const hos_batch* b) {
+    if (!cm) return HOS_E_INVALID;
+    if (cm->decode_fixed_us < 1 || cm->decode_kv_div < 1) return HOS_E_INVALID;
+    // longest possible iterations must stay below 2^31 us
+    const unsigned long long kv = (unsigned long long)b->kv_budget;
+    const unsigned long long pre = cm->prefill_fixed_us + (unsigned long long)cm->prefill_per_token_us * kv;
+    const unsigned long long dec = cm->decode_fixed_us +
+                                   (unsigned long long)cm->decode_per_seq_us * (unsigned long long)b->batch_cap +
+                                   kv / cm->decode_kv_div;
+    if (pre >= (1ull << 31) || dec >= (1ull << 31)) return HOS_E_INVALID;
+    return HOS_OK;
+}
+
+int check_ws(const void* ws, size_t have, size_t need) {
+    if (!ws || have < need || (reinterpret_cast<uintptr_t>(ws) & (WS_ALIGN - 1))) return HOS_E_WORKSPACE;
+    return HOS_OK;
+}
+
+struct OfflineWs {
+    uint32_t* T_sorted;
+    uint32_t* order;
+    InstInfo* info;
+    size_t bytes;
+};
+OfflineWs carve_offline(const hos_batch* b, void* ws) {
+    OfflineWs w;
+    const size_t rows = (size_t)b->n_inst * pad4(b->n_req);
+    unsigned char* base = static_cast<unsigned char*>(ws);
+    size_t off = 0;
+    w.T_sorted = reinterpret_cast<uint32_t*>(base + off); off += up(rows * 4);
+    w.order = reinterpret_cast<uint32_t*>(base + off);    off += up(rows * 4);
+    w.info = reinterpret_cast<InstInfo*>(base + off);     off += up((size_t)b->n_inst * sizeof(InstInfo));
+    w.bytes = off;
+    return w;
+}
+
+struct OnlineWs {
+    uint2* q_po;
+    uint32_t* q_req;
+    int32_t* q_off;
+    unsigned long long* inst_O;
+    int32_t* inst_status;
+    size_t bytes;
+};
+OnlineWs carve_online(const hos_batch* b, void* ws) {
+    OnlineWs w;
+    const size_t rows = (size_t)b->n_inst * pad4(b->n_req);
+    unsigned char* base = static_cast<unsigned char*>(ws);
+    size_t off = 0;
+    w.q_po = reinterpret_cast<uint2*>(base + off);                off += up(rows * 8);
+    w.q_req = reinterpret_cast<uint32_t*>(base + off);            off += up(rows * 4);
+    w.q_off = reinterpret_cast<int32_t*>(base + off);             off += up((size_t)b->n_inst * (b->n_clients + 1) * 4);
+    w.inst_O = reinterpret_cast<unsigned long long*>(base + off); off += up((size_t)b->n_inst * 8);
+    w.inst_status = reinterpret_cast<int32_t*>(base + off);       off += up((size_t)b->n_inst * 4);
+    w.bytes = off;
+    return w;
+}
+
+inline int cuda_rc(cudaError_t e) { return e == cudaSuccess ? HOS_OK : HOS_E_CUDA; }
+
+}  // namespace
+
+extern "C" {
+
+size_t hos_offline_workspace_bytes(const hos_batch* b, int /*n_copies*/, int /*ls_rounds*/) {
+    if (!b || b->n_inst < 1 || b->n_req < 1) return 0;
+    return carve_offline(b, nullptr).bytes;
+}
+size_t hos_lower_bound_workspace_bytes(const hos_batch* b) {
+    if (!b || b->n_inst < 1 || b->n_req < 1) return 0;
+    return carve_offline(b, nullptr).bytes;
+}
+size_t hos_online_workspace_bytes(const hos_batch* b, int /*n_lambda*/) {
+    if (!b || b->n_inst < 1 || b->n_req < 1 || b->n_clients < 1) return 0;
+    return carve_online(b, nullptr).bytes;
+}
+
+int hos_offline_pack(const hos_batch* b, const hos_cost_model* cm, int ls_rounds, int32_t* assign,
+                     int64_t* load, int64_t* makespan_est, int32_t* rounds_applied,
+                     hos_ls_move* ls_log, int32_t* status, void* ws, size_t ws_bytes, void* stream) {
+    int rc = check_batch(b);
+    if (rc) return rc;
+    if ((rc = check_cost(cm, b))) return rc;
+    if (!assign || !load || !makespan_est || !rounds_applied || !status || ls_rounds < 0) return HOS_E_INVALID;
+    if (estimate_sort_smem(b->n_req) > SMEM_LIMIT || local_search_smem(b->n_req) > SMEM_LIMIT)
+        return HOS_E_UNSUPPORTED;
+    if ((rc = check_ws(ws, ws_bytes, hos_offline_workspace_bytes(b, 1, ls_rounds)))) return rc;
+    const OfflineWs w = carve_offline(b, ws);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const int n_pad = pad4(b->n_req);
+    if ((rc = cuda_rc(launch_estimate_sort(*b, *cm, w.T_sorted, w.order, w.info, status, n_pad, st)))) return rc;
+    if ((rc = cuda_rc(launch_lpt(*b, w.T_sorted, w.order, w.info, n_pad, assign,
+                                 reinterpret_cast<long long*>(load),
+                                 reinterpret_cast<long long*>(makespan_est), st))))
+        return rc;
+    if (ls_rounds == 0)
+        return cuda_rc(cudaMemsetAsync(rounds_applied, 0, (size_t)b->n_inst * sizeof(int32_t), st));
+    return cuda_rc(launch_local_search(*b, w.T_sorted, w.order, w.info, n_pad, 1, ls_rounds, false, assign,
+                                       reinterpret_cast<long long*>(load),
+                                       reinterpret_cast<long long*>(makespan_est), rounds_applied,
+                                       ls_log, status, st));
+}
+
+int hos_local_search(const hos_batch* b, const hos_cost_model* cm, int n_copies, int ls_rounds,
+                     int32_t* assign, int64_t* load, int64_t* makespan_est, int32_t* rounds_applied,
+                     hos_ls_move* ls_log, int32_t* status, void* ws, size_t ws_bytes, void* stream) {
+    int rc = check_batch(b);
+    if (rc) return rc;
+    if ((rc = check_cost(cm, b))) return rc;
+    if (!assign || !load || !makespan_est || !rounds_applied || !status || ls_rounds < 0 || n_copies < 1)
+        return HOS_E_INVALID;
+    if ((long long)b->n_inst * n_copies > 0x7FFFFFFFll) return HOS_E_UNSUPPORTED;
+    if (estimate_sort_smem(b->n_req) > SMEM_LIMIT || local_search_smem(b->n_req) > SMEM_LIMIT)
+        return HOS_E_UNSUPPORTED;
+    if ((rc = check_ws(ws, ws_bytes, hos_offline_workspace_bytes(b, n_copies, ls_rounds)))) return rc;
+    const OfflineWs w = carve_offline(b, ws);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const int n_pad = pad4(b->n_req);
+    if ((rc = cuda_rc(launch_estimate_sort(*b, *cm, w.T_sorted, w.order, w.info, status, n_pad, st)))) return rc;
+    return cuda_rc(launch_local_search(*b, w.T_sorted, w.order, w.info, n_pad, n_copies, ls_rounds, true,
+                                       assign, reinterpret_cast<long long*>(load),
+                                       reinterpret_cast<long long*>(makespan_est), rounds_applied,
+                                       ls_log, status, st));
+}
+
+int hos_lower_bound(const hos_batch* b, const hos_cost_model* cm, hos_lb* out, int32_t* status, void* ws,
+                    size_t ws_bytes, void* stream) {
+    int rc = check_batch(b);
+    if (rc) return rc;
+    if ((rc = check_cost(cm, b))) return rc;
+    if (!out || !status) return HOS_E_INVALID;
+    if (estimate_sort_smem(b->n_req) > SMEM_LIMIT) return HOS_E_UNSUPPORTED;
+    if ((rc = check_ws(ws, ws_bytes, hos_lower_bound_workspace_bytes(b)))) return rc;
+    const OfflineWs w = carve_offline(b, ws);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const int n_pad = pad4(b->n_req);
+    if ((rc = cuda_rc(launch_estimate_sort(*b, *cm, w.T_sorted, w.order, w.info, status, n_pad, st)))) return rc;
+    return cuda_rc(launch_lower_bound(*b, *cm, w.T_sorted, w.info, n_pad, out, st));
+}
+
+int hos_online_simulate(const hos_batch* b, const int32_t* assign, const hos_cost_model* cm,
+                        const uint32_t* lambda_q16, int n_lambda, int queue_order, uint32_t max_iters,
+                        hos_client_result* cres, hos_sim_result* sres, hos_iter_rec* trace,
+                        const int64_t* trace_off, int32_t* status, void* ws, size_t ws_bytes,
+                        void* stream) {
+    int rc = check_batch(b);
+    if (rc) return rc;
+    if ((rc = check_cost(cm, b))) return rc;
+    if (!assign || !lambda_q16 || n_lambda < 1 || !cres || !sres || !status) return HOS_E_INVALID;
+    if (queue_order != HOS_QUEUE_SORTED && queue_order != HOS_QUEUE_FCFS) return HOS_E_INVALID;
+    if (trace && !trace_off) return HOS_E_INVALID;
+    if (queue_build_smem(b->n_req) > SMEM_LIMIT) return HOS_E_UNSUPPORTED;
+    if (bit_width_host((unsigned long long)b->kv_budget) + bit_width_host((unsigned long long)(b->n_clients - 1)) > 32)
+        return HOS_E_UNSUPPORTED;
+    if ((long long)b->n_inst * n_lambda > 0x7FFFFFFFll / 4) return HOS_E_UNSUPPORTED;
+    if ((rc = check_ws(ws, ws_bytes, hos_online_workspace_bytes(b, n_lambda)))) return rc;
+    const OnlineWs w = carve_online(b, ws);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const int n_pad = pad4(b->n_req);
+    if (max_iters > 0x7FFFFFFFu) max_iters = 0x7FFFFFFFu;
+    if ((rc = cuda_rc(launch_queue_build(*b, assign, queue_order, w.q_po, w.q_req, w.q_off, w.inst_O,
+                                         w.inst_status, n_pad, st))))
+        return rc;
+    if ((rc = cuda_rc(launch_simulate(*b, *cm, lambda_q16, n_lambda, max_iters, w.q_po, w.q_off,
+                                      w.inst_status, n_pad, cres, trace,
+                                      reinterpret_cast<const long long*>(trace_off), status, st))))
+        return rc;
+    return cuda_rc(launch_finalize(*b, n_lambda, w.inst_O, cres, sres, st));
+}
+
+int hos_trace_offsets(const hos_client_result* cres, int64_t n_units, int64_t* trace_off, void* stream) {
+    if (!cres || !trace_off || n_units < 0) return HOS_E_INVALID;
+    return cuda_rc(launch_trace_offsets(cres, (long long)n_units, reinterpret_cast<long long*>(trace_off),
+                                        static_cast<cudaStream_t>(stream)));
+}
+
+const char* hos_strerror(int code) {
+    switch (code) {
+        case HOS_OK: return "ok";
+        case HOS_E_INVALID: return "invalid argument";
+        case HOS_E_WORKSPACE: return "workspace missing, too small or not 256-byte aligned";
+        case HOS_E_CUDA: return "CUDA runtime error";
+        case HOS_E_UNSUPPORTED: return "shape outside the supported limits";
+        default: return "unknown error code";
+    }
+}
+
+}  // extern "C"

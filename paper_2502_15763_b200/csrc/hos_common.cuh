@@ -1,0 +1,78 @@
+// Shared device helpers of the hos kernels (sm_100a).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "hos.h"
+
+namespace hos {
+
+constexpr unsigned FULL = 0xFFFFFFFFu;
+constexpr int SORT_THREADS = 1024;          // one CTA per instance for the smem-resident kernels
+constexpr int SORT_WARPS = SORT_THREADS / 32;
+constexpr int RADIX_BITS = 8;
+constexpr int RADIX = 1 << RADIX_BITS;
+constexpr int MAX_CLIENTS = 256;
+constexpr int MAX_CAP = 256;
+constexpr int MAX_REQ = 24576;
+constexpr size_t SMEM_LIMIT = 227 * 1024;
+
+// Per-instance facts left in the workspace by the estimate+sort kernel.
+struct InstInfo {
+    unsigned long long sum_T;
+    uint32_t max_T;
+    int32_t status;
+};
+
+__device__ __forceinline__ int lane_id() { return threadIdx.x & 31; }
+__device__ __forceinline__ int warp_id() { return threadIdx.x >> 5; }
+
+__device__ __forceinline__ unsigned long long warp_sum_u64(unsigned long long v) {
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) v += __shfl_xor_sync(FULL, v, d);
+    return v;
+}
+__device__ __forceinline__ long long warp_max_i64(long long v) {
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) {
+        long long w = __shfl_xor_sync(FULL, v, d);
+        v = w > v ? w : v;
+    }
+    return v;
+}
+__device__ __forceinline__ unsigned long long warp_max_u64(unsigned long long v) {
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) {
+        unsigned long long w = __shfl_xor_sync(FULL, v, d);
+        v = w > v ? w : v;
+    }
+    return v;
+}
+
+// Block-wide reductions for blocks of up to 1024 threads; `scratch` holds 32 entries.
+// Every thread gets the result.  Contains __syncthreads().
+__device__ __forceinline__ unsigned long long block_sum_u64(unsigned long long v,
+                                                            unsigned long long* scratch) {
+    v = warp_sum_u64(v);
+    __syncthreads();
+    if (lane_id() == 0) scratch[warp_id()] = v;
+    __syncthreads();
+    int nw = (blockDim.x + 31) >> 5;
+    unsigned long long t = (lane_id() < nw) ? scratch[lane_id()] : 0ull;
+    return warp_sum_u64(t);
+}
+__device__ __forceinline__ unsigned long long block_max_u64(unsigned long long v,
+                                                            unsigned long long* scratch) {
+    v = warp_max_u64(v);
+    __syncthreads();
+    if (lane_id() == 0) scratch[warp_id()] = v;
+    __syncthreads();
+    int nw = (blockDim.x + 31) >> 5;
+    unsigned long long t = (lane_id() < nw) ? scratch[lane_id()] : 0ull;
+    return warp_max_u64(t);
+}
+
+__device__ __forceinline__ int bit_width_u32(uint32_t v) { return 32 - __clz(v); }
+
+}  // namespace hos

@@ -1,0 +1,44 @@
+// Internal launch interface between the C-ABI layer and the kernel translation units.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "hos.h"
+
+namespace hos {
+
+struct InstInfo;
+
+size_t estimate_sort_smem(int n_req);
+size_t local_search_smem(int n_req);
+size_t queue_build_smem(int n_req);
+
+cudaError_t launch_estimate_sort(const hos_batch& b, const hos_cost_model& cm, uint32_t* T_sorted,
+                                 uint32_t* order, InstInfo* info, int32_t* status_out, int n_pad,
+                                 cudaStream_t st);
+cudaError_t launch_lpt(const hos_batch& b, const uint32_t* T_sorted, const uint32_t* order,
+                       const InstInfo* info, int n_pad, int32_t* assign, long long* load,
+                       long long* makespan, cudaStream_t st);
+cudaError_t launch_local_search(const hos_batch& b, const uint32_t* T_sorted, const uint32_t* order,
+                                const InstInfo* info, int n_pad, int n_copies, int rounds,
+                                bool load_from_assign, int32_t* assign, long long* load,
+                                long long* makespan, int32_t* rounds_applied, hos_ls_move* ls_log,
+                                int32_t* status, cudaStream_t st);
+cudaError_t launch_lower_bound(const hos_batch& b, const hos_cost_model& cm, const uint32_t* T_sorted,
+                               const InstInfo* info, int n_pad, hos_lb* out, cudaStream_t st);
+
+cudaError_t launch_queue_build(const hos_batch& b, const int32_t* assign, int queue_order, uint2* q_po,
+                               uint32_t* q_req, int32_t* q_off, unsigned long long* inst_O,
+                               int32_t* inst_status, int n_pad, cudaStream_t st);
+cudaError_t launch_simulate(const hos_batch& b, const hos_cost_model& cm, const uint32_t* lambda_q16,
+                            int n_lambda, uint32_t max_iters, const uint2* q_po, const int32_t* q_off,
+                            const int32_t* inst_status, int n_pad, hos_client_result* cres,
+                            hos_iter_rec* trace, const long long* trace_off, int32_t* status,
+                            cudaStream_t st);
+cudaError_t launch_finalize(const hos_batch& b, int n_lambda, const unsigned long long* inst_O,
+                            hos_client_result* cres, hos_sim_result* sres, cudaStream_t st);
+cudaError_t launch_trace_offsets(const hos_client_result* cres, long long n_units, long long* trace_off,
+                                 cudaStream_t st);
+
+}  // namespace hos

@@ -1,0 +1,400 @@
+// Online scheduling kernels (Section "Online requests and iteration scheduling"):
+//   k_queue_build    per-client queues in the order of Algorithm 1
+//   k_simulate       iteration-level simulation, one warp per (instance, multiplier, client)
+//   k_finalize       per-simulation makespan, utilisation, generation speed
+//   k_trace_offsets  exclusive scan of the per-client iteration counts
+#include "hos_common.cuh"
+#include "hos_kernels.h"
+#include "hos_sort.cuh"
+
+namespace hos {
+
+// ---------------------------------------------------------------------------------------
+// Queue build: a segmented sort of the instance's requests by (client ascending,
+// N^p + N^d descending, index ascending) -- one stable radix sort on the composite key
+// client << kb | (2^kb - 1 - (p + o)).  HOS_QUEUE_FCFS sorts by client only.
+// ---------------------------------------------------------------------------------------
+template <typename IdxT>
+__global__ void __launch_bounds__(SORT_THREADS, 1)
+k_queue_build(const uint32_t* __restrict__ p, const uint32_t* __restrict__ o,
+              const int32_t* __restrict__ assign, int n_req, int n_clients, long long kv_budget,
+              int queue_order, uint2* __restrict__ q_po, uint32_t* __restrict__ q_req,
+              int32_t* __restrict__ q_off, unsigned long long* __restrict__ inst_O,
+              int32_t* __restrict__ inst_status, int n_pad) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    __shared__ unsigned long long red[32];
+    SortSmem<IdxT> s = sort_smem_carve<IdxT>(smem_raw, n_req);
+    const int inst = blockIdx.x;
+    const uint32_t* pi = p + (size_t)inst * n_req;
+    const uint32_t* oi = o + (size_t)inst * n_req;
+    const int32_t* ai = assign + (size_t)inst * n_req;
+
+    unsigned long long sumO = 0, mx = 0, bad = 0;
+    for (int i = threadIdx.x; i < n_req; i += SORT_THREADS) {
+        const uint32_t pp = pi[i], oo = oi[i];
+        const int c = ai[i];
+        const unsigned long long tot = (unsigned long long)pp + oo;
+        if (pp == 0 || oo == 0 || (long long)tot > kv_budget || c < 0 || c >= n_clients) bad = 1;
+        s.key[i] = (uint32_t)tot;
+        s.buf1[i] = (IdxT)(c & 0xFF);                 // parked until the keys are composed
+        sumO += oo;
+        mx = tot > mx ? tot : mx;
+    }
+    sumO = block_sum_u64(sumO, red);
+    mx = block_max_u64(mx, red);
+    bad = block_max_u64(bad, red);
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        inst_O[inst] = sumO;
+        inst_status[inst] = bad ? HOS_ST_INVALID : 0;
+    }
+    if (bad) return;
+
+    const int kb = (queue_order == HOS_QUEUE_SORTED) ? bit_width_u32((uint32_t)mx) : 0;
+    const uint32_t kmask = kb >= 32 ? 0xFFFFFFFFu : ((1u << kb) - 1u);
+    const int nbits = kb + bit_width_u32((uint32_t)(n_clients - 1));
+    for (int i = threadIdx.x; i < n_req; i += SORT_THREADS) {
+        const uint32_t c = (uint32_t)s.buf1[i];
+        s.key[i] = (kb >= 32 ? 0u : (c << kb)) | (kmask - (s.key[i] & kmask));
+    }
+    __syncthreads();
+    const IdxT* sorted = block_radix_sort_ids<IdxT>(s, n_req, nbits, 0u);
+
+    uint2* qp = q_po + (size_t)inst * n_pad;
+    uint32_t* qr = q_req + (size_t)inst * n_pad;
+    int32_t* qo = q_off + (size_t)inst * (n_clients + 1);
+    for (int r = threadIdx.x; r < n_req; r += SORT_THREADS) {
+        const uint32_t id = sorted[r];
+        qr[r] = id;
+        qp[r] = make_uint2(pi[id], oi[id]);
+        const int c = (int)(s.key[id] >> kb);
+        const int cprev = r > 0 ? (int)(s.key[sorted[r - 1]] >> kb) : -1;
+        for (int cc = cprev + 1; cc <= c; ++cc) qo[cc] = r;
+        if (r == n_req - 1)
+            for (int cc = c + 1; cc <= n_clients; ++cc) qo[cc] = n_req;
+    }
+}
+
+// ---------------------------------------------------------------------------------------
+// Iteration-level simulator.  One warp per (instance, multiplier, client).  The running
+// batch lives in registers: slot = (lane, k), k < SPL, batch_cap <= 32 * SPL.  A slot keeps
+// the decode-iteration count at which its request retires (`fin`) and the request's p + o
+// (`tot`): the KV length at count c is tot - fin + c, so a decode iteration touches no slot
+// unless someone retires, and sum KV is carried along (S += B - sum of retired tot).
+// ---------------------------------------------------------------------------------------
+constexpr uint32_t EMPTY = 0xFFFFFFFFu;
+constexpr unsigned long long HASH_INIT = 0xCBF29CE484222325ull;
+constexpr unsigned long long HASH_BASE = 0x9E3779B97F4A7C15ull;
+constexpr unsigned long long HASH_W0 = 0xBF58476D1CE4E5B9ull;
+constexpr unsigned long long HASH_W1 = 0x94D049BB133111EBull;
+constexpr unsigned long long HASH_W2 = 0xD6E8FEB86659FD93ull;
+constexpr unsigned long long HASH_W3 = 0xA0761D6478BD642Full;
+constexpr unsigned long long HASH_W4 = 0xE7037ED1A0B428DBull;
+constexpr int SIM_WARPS = 4;
+
+template <int SPL>
+__global__ void __launch_bounds__(SIM_WARPS * 32)
+k_simulate(const uint2* __restrict__ q_po, const int32_t* __restrict__ q_off,
+           const int32_t* __restrict__ inst_status, const uint32_t* __restrict__ lambda_q16,
+           int n_lambda, int n_clients, int n_pad, long long n_units, int cap, uint32_t kv_budget,
+           hos_cost_model cm, uint32_t max_iters, hos_client_result* __restrict__ cres,
+           hos_iter_rec* __restrict__ trace, const long long* __restrict__ trace_off,
+           int32_t* __restrict__ status_out) {
+    const long long unit = (long long)blockIdx.x * SIM_WARPS + warp_id();
+    if (unit >= n_units) return;
+    const int lane = lane_id();
+    const int c = (int)(unit % n_clients);
+    const int l = (int)((unit / n_clients) % n_lambda);
+    const int inst = (int)(unit / ((long long)n_clients * n_lambda));
+
+    if (inst_status[inst]) {
+        if (lane == 0) {
+            cres[unit] = hos_client_result{0, 0, 0u, 0u, 0ull, 0.0};
+            status_out[unit] = inst_status[inst];
+        }
+        return;
+    }
+    const int q0 = q_off[(size_t)inst * (n_clients + 1) + c];
+    const int qn = q_off[(size_t)inst * (n_clients + 1) + c + 1] - q0;
+    const uint2* q = q_po + (size_t)inst * n_pad + q0;
+    const uint32_t lam = lambda_q16[l];
+    const uint32_t ap = cm.prefill_fixed_us, bp = cm.prefill_per_token_us;
+    const uint32_t ad = cm.decode_fixed_us, bd = cm.decode_per_seq_us, qd = cm.decode_kv_div;
+
+    uint32_t fin[SPL], tot[SPL];
+#pragma unroll
+    for (int k = 0; k < SPL; ++k) { fin[k] = EMPTY; tot[k] = 0; }
+
+    long long t = 0, busy = 0;
+    uint32_t Cd = 0, cnt = 0, B = 0, S = 0, reserved = 0, iters = 0, n_pre = 0, n_dec = 0;
+    uint32_t next_fin = EMPTY;
+    int head = 0;
+    unsigned long long hash = HASH_INIT, pw = 1ull;
+    uint32_t nA = 0, sumP = 0, sumTot = 0;
+    bool dirty = true;
+    int32_t status = 0;
+
+    hos_iter_rec* tr = nullptr;
+    long long tr_cap = 0;
+    if (trace) {
+        const long long t0 = trace_off[unit];
+        tr = trace + t0;
+        tr_cap = trace_off[unit + 1] - t0;
+    }
+    uint4 held = make_uint4(0, 0, 0, 0);                 // lane x holds record (iters & ~31) + x
+
+    while (true) {
+        if (dirty) {
+            // candidates: longest queue prefix that fits the free slots and the KV budget
+            nA = 0; sumP = 0; sumTot = 0;
+            int pos = head;
+            while (pos < qn && B + nA < (uint32_t)cap) {
+                const int e = pos + lane;
+                uint2 po = make_uint2(0u, 0u);
+                if (e < qn) po = __ldg(&q[e]);
+                unsigned long long it = (unsigned long long)po.x + po.y;   // inclusive sums
+                unsigned long long ip = po.x;
+#pragma unroll
+                for (int d = 1; d < 32; d <<= 1) {
+                    const unsigned long long yt = __shfl_up_sync(FULL, it, d);
+                    const unsigned long long yp = __shfl_up_sync(FULL, ip, d);
+                    if (lane >= d) { it += yt; ip += yp; }
+                }
+                const bool ok = e < qn && (B + nA + (uint32_t)lane < (uint32_t)cap) &&
+                                ((unsigned long long)reserved + sumTot + it <= (unsigned long long)kv_budget);
+                const unsigned okm = __ballot_sync(FULL, ok);
+                const int take = (okm == FULL) ? 32 : (__ffs(~okm) - 1);
+                if (take > 0) {
+                    sumTot += (uint32_t)__shfl_sync(FULL, it, take - 1);
+                    sumP += (uint32_t)__shfl_sync(FULL, ip, take - 1);
+                    nA += take;
+                }
+                if (take < 32) break;
+                pos += 32;
+            }
+            dirty = false;
+        }
+        if (B == 0 && nA == 0) break;                    // queue empty and nothing running
+        if (iters == max_iters) { status |= HOS_ST_LIMIT; break; }
+
+        const uint32_t Cp = ap + bp * sumP;
+        const bool prefill =
+            nA > 0 && (B == 0 || (unsigned long long)lam * Cd > ((unsigned long long)Cp << 16));
+        uint32_t dur, r1, r2, r3;
+        if (prefill) {
+            // admit queue[head .. head + nA) into free slots
+            int nfree = 0;
+#pragma unroll
+            for (int k = 0; k < SPL; ++k) nfree += (fin[k] == EMPTY);
+            int g = nfree;
+#pragma unroll
+            for (int d = 1; d < 32; d <<= 1) {
+                const int y = __shfl_up_sync(FULL, g, d);
+                if (lane >= d) g += y;
+            }
+            g -= nfree;                                   // exclusive: free slots in lower lanes
+#pragma unroll
+            for (int k = 0; k < SPL; ++k) {
+                if (fin[k] == EMPTY) {
+                    if ((uint32_t)g < nA) {
+                        const uint2 po = __ldg(&q[head + g]);
+                        fin[k] = cnt + po.y;
+                        tot[k] = po.x + po.y;
+                    }
+                    ++g;
+                }
+            }
+            dur = Cp; r1 = 0x80000000u | nA; r2 = sumP; r3 = (uint32_t)head;
+            busy += (long long)dur * nA;
+            S += sumP; B += nA; reserved += sumTot; head += (int)nA;
+            Cd = 0; ++n_pre;
+            nA = 0; sumP = 0; sumTot = 0;                 // nothing more fits until someone retires
+            uint32_t m = fin[0];
+#pragma unroll
+            for (int k = 1; k < SPL; ++k) m = min(m, fin[k]);
+            next_fin = __reduce_min_sync(FULL, m);
+        } else {
+            dur = ad + bd * B + S / qd;
+            r1 = B; r2 = S; r3 = 0;
+            busy += (long long)dur * B;
+            ++cnt;
+            if (cnt == next_fin) {
+                uint32_t rel = 0, nf = 0;
+#pragma unroll
+                for (int k = 0; k < SPL; ++k)
+                    if (fin[k] == cnt) { rel += tot[k]; ++nf; fin[k] = EMPTY; }
+                // rel < 2^31 in total (reserved <= kv_budget), nf <= cap: pack both in one reduction
+                const unsigned long long both =
+                    warp_sum_u64(((unsigned long long)nf << 32) | rel);
+                rel = (uint32_t)both; nf = (uint32_t)(both >> 32);
+                S = S + B - rel;
+                B -= nf; reserved -= rel; r3 = nf;
+                uint32_t m = fin[0];
+#pragma unroll
+                for (int k = 1; k < SPL; ++k) m = min(m, fin[k]);
+                next_fin = __reduce_min_sync(FULL, m);
+                dirty = head < qn;
+            } else {
+                S += B;
+            }
+            const unsigned long long w = (unsigned long long)Cd + dur;
+            Cd = w > 0x7FFFFFFFull ? 0x7FFFFFFFu : (uint32_t)w;
+            ++n_dec;
+        }
+        t += dur;
+        hash += (HASH_W0 * dur + HASH_W1 * r1 + HASH_W2 * r2 + HASH_W3 * r3 + HASH_W4) * pw;
+        pw *= HASH_BASE;
+        if (tr) {
+            if (lane == (int)(iters & 31u)) held = make_uint4(dur, r1, r2, r3);
+            if ((iters & 31u) == 31u) {
+                const long long idx = (long long)(iters & ~31u) + lane;
+                if (idx < tr_cap) reinterpret_cast<uint4*>(tr)[idx] = held;
+                else status |= HOS_ST_TRACE;
+            }
+        }
+        ++iters;
+        if (t >= (1ll << 39)) { status |= HOS_ST_LIMIT; break; }
+    }
+    if (tr && (iters & 31u) != 0u) {                      // records of the last, partial row
+        const long long idx = (long long)(iters & ~31u) + lane;
+        if (lane < (int)(iters & 31u)) {
+            if (idx < tr_cap) reinterpret_cast<uint4*>(tr)[idx] = held;
+            else status |= HOS_ST_TRACE;
+        }
+    }
+    status = __reduce_or_sync(FULL, status);
+    if (lane == 0) {
+        cres[unit] = hos_client_result{t, busy, n_pre, n_dec, hash, 0.0};
+        status_out[unit] = status;
+    }
+}
+
+// ---------------------------------------------------------------------------------------
+// Per-simulation figures: makespan = max over clients, busy = sum, utilisation = busy slot
+// time over offered slot time, generation speed = output tokens per second of makespan.
+// One warp per (instance, multiplier).
+// ---------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(128)
+k_finalize(int n_sims, int n_lambda, int n_clients, int cap,
+           const unsigned long long* __restrict__ inst_O, hos_client_result* __restrict__ cres,
+           hos_sim_result* __restrict__ sres) {
+    const int sim = blockIdx.x * 4 + warp_id();
+    if (sim >= n_sims) return;
+    const int lane = lane_id();
+    hos_client_result* cr = cres + (size_t)sim * n_clients;
+    long long mk = 0;
+    unsigned long long busy = 0;
+    for (int j = lane; j < n_clients; j += 32) {
+        mk = cr[j].makespan_us > mk ? cr[j].makespan_us : mk;
+        busy += (unsigned long long)cr[j].busy_slot_us;
+    }
+    mk = warp_max_i64(mk);
+    busy = warp_sum_u64(busy);
+    const double dm = (double)mk;
+    for (int j = lane; j < n_clients; j += 32)
+        cr[j].utilisation = mk > 0 ? (double)cr[j].busy_slot_us / ((double)cap * dm) : 0.0;
+    if (lane == 0) {
+        hos_sim_result r;
+        r.makespan_us = mk;
+        r.busy_slot_us = (long long)busy;
+        r.utilisation = mk > 0 ? (double)(long long)busy / (((double)n_clients * (double)cap) * dm) : 0.0;
+        r.tokens_per_s = mk > 0 ? ((double)inst_O[sim / n_lambda] * 1.0e6) / dm : 0.0;
+        sres[sim] = r;
+    }
+}
+
+// Exclusive scan of the iteration counts; one CTA walks the array in tiles of 1024.
+__global__ void __launch_bounds__(1024)
+k_trace_offsets(const hos_client_result* __restrict__ cres, long long n_units,
+                long long* __restrict__ trace_off) {
+    __shared__ unsigned long long wsum[32];
+    __shared__ unsigned long long carry_s;
+    if (threadIdx.x == 0) { carry_s = 0; trace_off[0] = 0; }
+    __syncthreads();
+    for (long long base = 0; base < n_units; base += 1024) {
+        const long long x = base + threadIdx.x;
+        const unsigned long long v =
+            x < n_units ? (unsigned long long)cres[x].n_prefill_iters + cres[x].n_decode_iters : 0ull;
+        unsigned long long inc = v;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const unsigned long long y = __shfl_up_sync(FULL, inc, d);
+            if (lane_id() >= d) inc += y;
+        }
+        if (lane_id() == 31) wsum[warp_id()] = inc;
+        __syncthreads();
+        if (warp_id() == 0) {
+            const unsigned long long w = wsum[lane_id()];
+            unsigned long long winc = w;
+#pragma unroll
+            for (int d = 1; d < 32; d <<= 1) {
+                const unsigned long long y = __shfl_up_sync(FULL, winc, d);
+                if (lane_id() >= d) winc += y;
+            }
+            wsum[lane_id()] = winc - w;
+        }
+        __syncthreads();
+        const unsigned long long carry = carry_s;
+        const unsigned long long mine = carry + wsum[warp_id()] + inc;       // inclusive
+        if (x < n_units) trace_off[x + 1] = (long long)mine;
+        __syncthreads();
+        if (threadIdx.x == 1023) carry_s = mine;
+        __syncthreads();
+    }
+}
+
+// ---------------------------------------------------------------------------------------
+// launchers
+// ---------------------------------------------------------------------------------------
+size_t queue_build_smem(int n_req) {
+    return n_req <= 65536 ? sort_smem_bytes<uint16_t>(n_req) : sort_smem_bytes<uint32_t>(n_req);
+}
+
+cudaError_t launch_queue_build(const hos_batch& b, const int32_t* assign, int queue_order, uint2* q_po,
+                               uint32_t* q_req, int32_t* q_off, unsigned long long* inst_O,
+                               int32_t* inst_status, int n_pad, cudaStream_t st) {
+    const size_t smem = queue_build_smem(b.n_req);
+    auto kern = b.n_req <= 65536 ? k_queue_build<uint16_t> : k_queue_build<uint32_t>;
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    kern<<<b.n_inst, SORT_THREADS, smem, st>>>(b.p, b.o, assign, b.n_req, b.n_clients,
+                                               (long long)b.kv_budget, queue_order, q_po, q_req, q_off,
+                                               inst_O, inst_status, n_pad);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_simulate(const hos_batch& b, const hos_cost_model& cm, const uint32_t* lambda_q16,
+                            int n_lambda, uint32_t max_iters, const uint2* q_po, const int32_t* q_off,
+                            const int32_t* inst_status, int n_pad, hos_client_result* cres,
+                            hos_iter_rec* trace, const long long* trace_off, int32_t* status,
+                            cudaStream_t st) {
+    const long long n_units = (long long)b.n_inst * n_lambda * b.n_clients;
+    const unsigned grid = (unsigned)((n_units + SIM_WARPS - 1) / SIM_WARPS);
+#define HOS_SIM(SPL)                                                                               \
+    k_simulate<SPL><<<grid, SIM_WARPS * 32, 0, st>>>(q_po, q_off, inst_status, lambda_q16, n_lambda, \
+                                                     b.n_clients, n_pad, n_units, b.batch_cap,     \
+                                                     (uint32_t)b.kv_budget, cm, max_iters, cres,   \
+                                                     trace, trace_off, status)
+    if (b.batch_cap <= 32) HOS_SIM(1);
+    else if (b.batch_cap <= 64) HOS_SIM(2);
+    else if (b.batch_cap <= 128) HOS_SIM(4);
+    else HOS_SIM(8);
+#undef HOS_SIM
+    return cudaGetLastError();
+}
+
+cudaError_t launch_finalize(const hos_batch& b, int n_lambda, const unsigned long long* inst_O,
+                            hos_client_result* cres, hos_sim_result* sres, cudaStream_t st) {
+    const int n_sims = b.n_inst * n_lambda;
+    k_finalize<<<(n_sims + 3) / 4, 128, 0, st>>>(n_sims, n_lambda, b.n_clients, b.batch_cap, inst_O,
+                                                 cres, sres);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_trace_offsets(const hos_client_result* cres, long long n_units, long long* trace_off,
+                                 cudaStream_t st) {
+    k_trace_offsets<<<1, 1024, 0, st>>>(cres, n_units, trace_off);
+    return cudaGetLastError();
+}
+
+}  // namespace hos

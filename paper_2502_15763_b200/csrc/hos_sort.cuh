@@ -1,0 +1,142 @@
+// CTA-wide stable LSD radix sort of item ids by a 32-bit key table held in shared memory.
+//
+// One CTA of SORT_THREADS threads owns one instance.  The ids 0..n-1 are sorted
+// ascending by (key[id] ^ flip), `nbits` low bits significant, 8 bits per pass; equal keys
+// keep id order (the first pass reads ids in natural order, every pass is stable).  Each
+// warp owns a contiguous chunk of positions; a pass is (1) per-warp digit counts,
+// (2) one exclusive scan over the [digit][warp] count matrix, (3) a stable scatter in which
+// the rank of an item among the equal digits of its 32-wide row comes from match_any.
+#pragma once
+
+#include "hos_common.cuh"
+
+namespace hos {
+
+template <typename IdxT>
+struct SortSmem {
+    // layout inside dynamic shared memory, all 16-byte aligned
+    uint32_t* key;      // [n]
+    IdxT* buf0;         // [n]
+    IdxT* buf1;         // [n]
+    uint32_t* cnt;      // [RADIX * SORT_WARPS]
+    uint32_t* wsum;     // [SORT_WARPS]
+};
+
+__host__ __device__ inline size_t align16(size_t x) { return (x + 15) & ~size_t(15); }
+
+template <typename IdxT>
+__host__ __device__ inline size_t sort_smem_bytes(int n) {
+    return align16(size_t(n) * 4) + 2 * align16(size_t(n) * sizeof(IdxT)) +
+           size_t(RADIX) * SORT_WARPS * 4 + SORT_WARPS * 4;
+}
+
+template <typename IdxT>
+__device__ inline SortSmem<IdxT> sort_smem_carve(unsigned char* base, int n) {
+    SortSmem<IdxT> s;
+    s.key = reinterpret_cast<uint32_t*>(base);
+    base += align16(size_t(n) * 4);
+    s.buf0 = reinterpret_cast<IdxT*>(base);
+    base += align16(size_t(n) * sizeof(IdxT));
+    s.buf1 = reinterpret_cast<IdxT*>(base);
+    base += align16(size_t(n) * sizeof(IdxT));
+    s.cnt = reinterpret_cast<uint32_t*>(base);
+    base += size_t(RADIX) * SORT_WARPS * 4;
+    s.wsum = reinterpret_cast<uint32_t*>(base);
+    return s;
+}
+
+// Exclusive scan of cnt[0 .. RADIX*SORT_WARPS) in place.  All SORT_THREADS threads call it.
+__device__ inline void scan_counts(uint32_t* cnt, uint32_t* wsum) {
+    constexpr int PER = RADIX * SORT_WARPS / SORT_THREADS;   // 8 consecutive entries per thread
+    const int t = threadIdx.x;
+    uint32_t v[PER];
+    uint32_t run = 0;
+#pragma unroll
+    for (int k = 0; k < PER; ++k) {
+        uint32_t c = cnt[t * PER + k];
+        v[k] = run;
+        run += c;
+    }
+    // inclusive warp scan of the thread totals
+    uint32_t inc = run;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+        uint32_t y = __shfl_up_sync(FULL, inc, d);
+        if (lane_id() >= d) inc += y;
+    }
+    if (lane_id() == 31) wsum[warp_id()] = inc;
+    __syncthreads();
+    if (warp_id() == 0) {
+        uint32_t w = wsum[lane_id()];
+        uint32_t winc = w;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            uint32_t y = __shfl_up_sync(FULL, winc, d);
+            if (lane_id() >= d) winc += y;
+        }
+        wsum[lane_id()] = winc - w;                          // exclusive warp offsets
+    }
+    __syncthreads();
+    uint32_t base = wsum[warp_id()] + inc - run;
+#pragma unroll
+    for (int k = 0; k < PER; ++k) cnt[t * PER + k] = base + v[k];
+    __syncthreads();
+}
+
+// Returns the buffer (buf0 or buf1) that holds the sorted ids.  nbits == 0 leaves ids in
+// natural order.  Ends with a __syncthreads().
+template <typename IdxT>
+__device__ inline IdxT* block_radix_sort_ids(const SortSmem<IdxT>& s, int n, int nbits,
+                                             uint32_t flip) {
+    const int lane = lane_id(), warp = warp_id();
+    const int chunk = (((n + SORT_WARPS - 1) / SORT_WARPS) + 31) & ~31;   // positions per warp
+    const int lo = warp * chunk;
+    const int hi = min(n, lo + chunk);
+    IdxT* src = s.buf1;
+    IdxT* dst = s.buf0;
+    bool natural = true;                                     // first pass reads id = position
+
+    if (nbits <= 0) {
+        for (int i = threadIdx.x; i < n; i += SORT_THREADS) dst[i] = (IdxT)i;
+        __syncthreads();
+        return dst;
+    }
+    for (int shift = 0; shift < nbits; shift += RADIX_BITS) {
+        for (int i = threadIdx.x; i < RADIX * SORT_WARPS; i += SORT_THREADS) s.cnt[i] = 0;
+        __syncthreads();
+        // (1) per-warp digit counts
+        for (int row = lo; row < hi; row += 32) {
+            const int pos = row + lane;
+            const bool valid = pos < hi;
+            uint32_t id = valid ? (natural ? (uint32_t)pos : (uint32_t)src[pos]) : 0u;
+            uint32_t dig = valid ? (((s.key[id] ^ flip) >> shift) & (RADIX - 1)) : (uint32_t)RADIX;
+            unsigned m = __match_any_sync(FULL, dig);
+            if (valid && lane == (__ffs(m) - 1)) s.cnt[dig * SORT_WARPS + warp] += __popc(m);
+            __syncwarp();
+        }
+        __syncthreads();
+        // (2) offsets
+        scan_counts(s.cnt, s.wsum);
+        // (3) stable scatter
+        for (int row = lo; row < hi; row += 32) {
+            const int pos = row + lane;
+            const bool valid = pos < hi;
+            uint32_t id = valid ? (natural ? (uint32_t)pos : (uint32_t)src[pos]) : 0u;
+            uint32_t dig = valid ? (((s.key[id] ^ flip) >> shift) & (RADIX - 1)) : (uint32_t)RADIX;
+            unsigned m = __match_any_sync(FULL, dig);
+            uint32_t base = valid ? s.cnt[dig * SORT_WARPS + warp] : 0u;
+            __syncwarp();
+            if (valid) {
+                dst[base + __popc(m & ((1u << lane) - 1u))] = (IdxT)id;
+                if (lane == (__ffs(m) - 1)) s.cnt[dig * SORT_WARPS + warp] = base + __popc(m);
+            }
+            __syncwarp();
+        }
+        __syncthreads();
+        IdxT* t = src; src = dst; dst = t;
+        natural = false;
+    }
+    return src;
+}
+
+}  // namespace hos

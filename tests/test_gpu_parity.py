@@ -1,0 +1,202 @@
+"""CUDA path against the CPU oracle, element by element, through the C ABI (needs a GPU)."""
+import numpy as np
+import pytest
+
+from oracle import hos_oracle as ora
+from tests import gpu_harness as H
+from workload import LAMBDA_NEVER_PREEMPT, LAMBDA_ONE, LAMBDA_PREFILL_FIRST, LengthDist, batch_lengths, workload
+
+pytestmark = pytest.mark.gpu
+
+LAMS = (LAMBDA_NEVER_PREEMPT, 20000, LAMBDA_ONE, 5 << 16, LAMBDA_PREFILL_FIRST)
+
+
+@pytest.fixture(scope="module")
+def hos():
+    import torch
+    assert torch.cuda.is_available(), "GPU tests need a CUDA device"
+    import paper_2502_15763_b200 as m
+    m.lib()
+    return m
+
+
+def full_pipeline(hos, w, ls_rounds, lambdas, insts=None, modes=(ora.QUEUE_SORTED, ora.QUEUE_FCFS)):
+    p, o = w.lengths()
+    M, cap, kv, cm = w.n_clients, w.batch_cap, w.kv_budget, w.cost_model
+    g = H.check_offline(hos, p, o, M, cap, kv, cm, ls_rounds, insts)
+    H.check_lower_bound(hos, p, o, M, cap, kv, cm, insts)
+    for mode in modes:
+        H.check_simulate(hos, p, o, M, cap, kv, cm, g["assign"], lambdas, mode, insts)
+    return p, o, g
+
+
+def test_config0(hos):
+    full_pipeline(hos, workload("c0"), 10, LAMS)
+
+
+def test_config1(hos):
+    full_pipeline(hos, workload("c1"), 20, LAMS)
+
+
+def test_config2_hybrid_and_baseline(hos):
+    w = workload("c2")
+    p, o, g = full_pipeline(hos, w, 0, (LAMBDA_ONE,), modes=(ora.QUEUE_SORTED,))
+    rr = (np.arange(w.n_req, dtype=np.int32) % w.n_clients)[None, :].repeat(w.n_inst, 0)
+    base = H.check_simulate(hos, p, o, w.n_clients, w.batch_cap, w.kv_budget, w.cost_model, rr,
+                            (LAMBDA_PREFILL_FIRST, LAMBDA_NEVER_PREEMPT), ora.QUEUE_FCFS)
+    hyb = H.gpu_simulate(hos, p, o, w.n_clients, w.batch_cap, w.kv_budget, w.cost_model, g["assign"],
+                         (LAMBDA_ONE,), ora.QUEUE_SORTED, want_trace=False)
+    gain = hyb["sres"]["utilisation"][:, 0] - base["sres"]["utilisation"][:, 0]
+    assert gain.mean() > 0           # direction of the paper's 100-case study
+
+
+def test_config3_sweep(hos):
+    w = workload("c3")
+    p, o = w.lengths()
+    M, cap, kv, cm = w.n_clients, w.batch_cap, w.kv_budget, w.cost_model
+    g = H.check_offline(hos, p, o, M, cap, kv, cm, 0)
+    H.check_simulate(hos, p, o, M, cap, kv, cm, g["assign"], w.lambdas_q16, ora.QUEUE_SORTED,
+                     insts=range(0, 100, 9), want_trace=False)
+    H.check_simulate(hos, p, o, M, cap, kv, cm, g["assign"], w.lambdas_q16[::13], ora.QUEUE_SORTED,
+                     insts=(3, 50))
+    # 20 local-search rounds on a private copy of the LPT assignment per (instance, multiplier)
+    import torch
+    from paper_2502_15763_b200.binding import view_struct
+    nl = len(w.lambdas_q16)
+    copies = torch.from_numpy(g["assign"]).cuda()[:, None, :].repeat(1, nl, 1).contiguous()
+    r = hos.hos_local_search(H.to_dev(p), H.to_dev(o), M, cap, kv, cm, copies, w.ls_rounds, want_log=True)
+    a, l = r["assign"].cpu().numpy(), r["load"].cpu().numpy()
+    log = view_struct(r["ls_log"], hos.LS_MOVE_DTYPE)
+    assert (r["status"].cpu().numpy() == 0).all()
+    for k in range(w.n_inst):
+        T = ora.estimate(p[k], o[k], cm)
+        ea, el, applied, elog = ora.local_search(T, g["assign"][k], g["load"][k], w.ls_rounds)
+        for c in range(nl):                                    # the copies agree bit for bit
+            assert np.array_equal(a[k, c], ea) and np.array_equal(l[k, c], el)
+            assert int(r["rounds_applied"][k, c]) == applied
+            assert int(r["makespan_est"][k, c]) == int(el.max())
+        for f in ("i", "u", "k", "v"):
+            assert np.array_equal(log[k, 0][f], elog[f]) and np.array_equal(log[k, nl - 1][f], elog[f])
+
+
+@pytest.mark.parametrize("n,M,cap", [(1, 1, 1), (2, 3, 1), (31, 4, 2), (33, 32, 16), (97, 33, 33),
+                                     (257, 64, 64), (1000, 65, 100), (1301, 130, 128), (2050, 256, 200),
+                                     (515, 7, 256), (64, 100, 5)])
+def test_ragged_shapes(hos, n, M, cap):
+    rng = np.random.default_rng(n * 1000 + M)
+    n_inst = 3
+    p = rng.integers(1, 300, size=(n_inst, n)).astype(np.uint32)
+    o = rng.integers(1, 120, size=(n_inst, n)).astype(np.uint32)
+    o[:, ::7] = 1                                              # many ties and one-token outputs
+    p[:, ::5] = p[:, :1]
+    cm = (20000, 40, 15000, 300, 16, 40, 350)
+    kv = int((p.astype(np.int64) + o).max()) * int(rng.choice([1, 3, 1000]))
+    g = H.check_offline(hos, p, o, M, cap, kv, cm, 6)
+    H.check_lower_bound(hos, p, o, M, cap, kv, cm)
+    rand_assign = rng.integers(0, M, size=(n_inst, n)).astype(np.int32)
+    for assign in (g["assign"], rand_assign):
+        for mode in (ora.QUEUE_SORTED, ora.QUEUE_FCFS):
+            H.check_simulate(hos, p, o, M, cap, kv, cm, assign, LAMS, mode)
+
+
+def test_local_search_from_bad_assignments(hos):
+    import torch
+    from paper_2502_15763_b200.binding import view_struct
+    rng = np.random.default_rng(77)
+    n_inst, n, M, rounds = 4, 700, 9, 40
+    p = rng.integers(1, 50, size=(n_inst, n)).astype(np.uint32)      # few distinct T: many ties
+    o = rng.integers(1, 6, size=(n_inst, n)).astype(np.uint32)
+    cm = (20000, 40, 15000, 300, 16, 40, 350)
+    assign = rng.integers(0, M, size=(n_inst, 2, n)).astype(np.int32)
+    assign[:, 1, :] = 0                                              # everything on one client
+    r = hos.hos_local_search(H.to_dev(p), H.to_dev(o), M, 8, 10 ** 6, cm, torch.from_numpy(assign).cuda(),
+                             rounds, want_log=True)
+    log = view_struct(r["ls_log"], hos.LS_MOVE_DTYPE)
+    for k in range(n_inst):
+        T = ora.estimate(p[k], o[k], cm)
+        for c in range(2):
+            l0 = np.array([int(T[assign[k, c] == j].sum()) for j in range(M)], dtype=np.int64)
+            ea, el, applied, elog = ora.local_search(T, assign[k, c], l0, rounds)
+            assert np.array_equal(r["assign"][k, c].cpu().numpy(), ea)
+            assert np.array_equal(r["load"][k, c].cpu().numpy(), el)
+            assert int(r["rounds_applied"][k, c]) == applied
+            for f in ("i", "u", "k", "v"):
+                assert np.array_equal(log[k, c][f], elog[f])
+
+
+def test_wide_estimates_take_the_64bit_packing_path(hos):
+    # T_i up to ~2^31: the packed 32-bit load keys cannot be used
+    rng = np.random.default_rng(5)
+    n_inst, n, M = 2, 400, 5
+    p = rng.integers(1, 2000, size=(n_inst, n)).astype(np.uint32)
+    o = rng.integers(1, 2000, size=(n_inst, n)).astype(np.uint32)
+    cm = (20000, 40, 15000, 300, 16, 500000, 500000)
+    H.check_offline(hos, p, o, M, 8, 10 ** 6, cm, 5)
+    H.check_lower_bound(hos, p, o, M, 8, 10 ** 6, cm)
+
+
+def test_limits_and_bad_data(hos):
+    w = workload("c0")
+    p, o = w.lengths()
+    M, cap, kv, cm = w.n_clients, w.batch_cap, w.kv_budget, w.cost_model
+    g = H.gpu_offline(hos, p, o, M, cap, kv, cm, 0)
+    # iteration limit: truncated exactly like the oracle
+    H.check_simulate(hos, p, o, M, cap, kv, cm, g["assign"], (LAMBDA_ONE,), ora.QUEUE_SORTED, max_iters=37)
+    # trace slots too small: records dropped, hash and counts intact, status bit set
+    full = H.gpu_simulate(hos, p, o, M, cap, kv, cm, g["assign"], (LAMBDA_ONE,), ora.QUEUE_SORTED)
+    small = H.gpu_simulate(hos, p, o, M, cap, kv, cm, g["assign"], (LAMBDA_ONE,), ora.QUEUE_SORTED, trace_slots=40)
+    assert (small["status_traced"] == hos.HOS_ST_TRACE).all()
+    assert np.array_equal(small["cres"]["trace_hash"], full["cres"]["trace_hash"])
+    for j in range(M):
+        t0 = int(full["trace_off"][j])
+        assert np.array_equal(small["trace"][40 * j:40 * j + 40], full["trace"][t0:t0 + 40])
+    # a zero-length output marks the instance invalid without touching the others
+    p2 = np.concatenate([p, p]); o2 = np.concatenate([o, o]).copy(); o2[1, 5] = 0
+    g2 = H.gpu_offline(hos, p2, o2, M, cap, kv, cm, 3)
+    assert g2["status"].tolist() == [0, hos.HOS_ST_INVALID]
+    assert np.array_equal(g2["assign"][0], ora.offline_pack(p[0], o[0], M, cm, 3)["assign"])
+    assert (g2["assign"][1] == -1).all() and g2["makespan_est"][1] == 0
+    s2 = H.gpu_simulate(hos, p2, o2, M, cap, kv, cm, np.concatenate([g["assign"], g["assign"]]),
+                        (LAMBDA_ONE,), ora.QUEUE_SORTED, want_trace=False)
+    assert (s2["status"][1] == hos.HOS_ST_INVALID).all() and (s2["status"][0] == 0).all()
+    assert s2["sres"]["makespan_us"][1, 0] == 0 and s2["sres"]["makespan_us"][0, 0] == full["sres"]["makespan_us"][0, 0]
+    # host-side rejections
+    with pytest.raises(hos.HosError):
+        hos.hos_offline_pack(H.to_dev(p), H.to_dev(o), 0, cap, kv, cm)
+    with pytest.raises(hos.HosError):
+        hos.hos_offline_pack(H.to_dev(p), H.to_dev(o), 300, cap, kv, cm)
+
+
+def test_config4_full_size_sampled(hos):
+    """All 1,024 instances on the GPU in the benchmark's launch shape; the oracle checks a sample
+    element by element and size-independent properties are checked on everything."""
+    import multiprocessing as mp
+    w = workload("c4")
+    p, o = w.lengths()
+    M, cap, kv, cm = w.n_clients, w.batch_cap, w.kv_budget, w.cost_model
+    sample = (0, 341, 1023)
+    g = H.check_offline(hos, p, o, M, cap, kv, cm, w.ls_rounds, insts=sample)
+    lb = H.check_lower_bound(hos, p, o, M, cap, kv, cm, insts=sample)
+    s = H.check_simulate(hos, p, o, M, cap, kv, cm, g["assign"], w.lambdas_q16, ora.QUEUE_SORTED, insts=sample)
+    # properties on every instance
+    T = 40 * p.astype(np.int64) + 350 * o.astype(np.int64)
+    assert (g["status"] == 0).all() and (s["status"] == 0).all()
+    assert np.array_equal(g["load"].sum(1), T.sum(1))
+    assert (g["makespan_est"] == g["load"].max(1)).all()
+    assert (lb["lb_pack"] <= g["makespan_est"]).all()
+    assert (M * g["makespan_est"] <= T.sum(1) + (M - 1) * T.max(1)).all()      # list-scheduling bound
+    for k in (5, 500):
+        for j in range(M):
+            assert g["load"][k, j] == T[k][g["assign"][k] == j].sum()
+    assert (lb["lb_sim_us"] <= s["sres"]["makespan_us"][:, 0]).all()
+    assert ((s["sres"]["utilisation"] > 0) & (s["sres"]["utilisation"] <= 1)).all()
+    n_dec_tokens = o.astype(np.int64).sum(1)
+    # every decode iteration advances its B requests by one token: sum over the trace of B = sum o_i
+    tr, off = s["trace"], s["trace_off"]
+    for k in (7, 777):
+        a, b = int(off[k * M]), int(off[(k + 1) * M])
+        rows = tr[a:b]
+        dec = (rows["kind_n"] >> 31) == 0
+        assert int(rows["kind_n"][dec].astype(np.int64).sum()) == int(n_dec_tokens[k])
+        assert int(rows["tokens"][~dec].astype(np.int64).sum()) == int(p[k].astype(np.int64).sum())
+        assert int(rows["dur_us"].astype(np.int64).sum()) == int(s["cres"]["makespan_us"][k, 0].sum())
