@@ -1,0 +1,439 @@
+#!/usr/bin/env python
+"""Benchmark of the batched scheduler evaluation (offline pack + lower bound + online simulation).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c0..c4] [--impl ours|reference]
+
+One step is one pass of the whole path over one batch of synthetic instances:
+hos_offline_pack (sort, LPT, local search) -> hos_lower_bound -> hos_online_simulate
+(count pass) -> hos_trace_offsets -> hos_online_simulate (traced pass).  Prints ONE JSON line.
+With N > 1 (under torchrun) every rank runs the same number of instances with its own seeds
+(weak scaling, no data-path collective); the time is the max over ranks.
+`--impl reference` times the CPU oracle on a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from workload import Workload, workload  # noqa: E402
+
+METRIC = "instances/sec"
+UNIT = "instances/s"
+DTYPE = "int64"            # integer microseconds / Q16.16; utilisation is one f64 division
+L2_FLUSH_BYTES = 256 << 20
+
+# algorithmic bytes per unit of work of each kernel (what a streaming implementation of that
+# step alone must move once)
+BYTES_PER_REQ = {"k_estimate_sort": 16, "k_lpt": 12, "k_lower_bound": 8, "k_queue_build": 16}
+
+
+def describe(w: Workload) -> str:
+    return (f"{w.name}: {w.n_inst} instances x {w.n_req} requests, {w.n_clients} clients, batch cap "
+            f"{w.batch_cap}, KV budget {w.kv_budget}, {len(w.lambdas_q16)} multiplier value(s), "
+            f"{w.ls_rounds} local-search rounds")
+
+
+def rank_workload(name: str, rank: int) -> Workload:
+    """Rank r evaluates the same number of instances with seeds shifted by r * n_inst."""
+    w = workload(name)
+    if rank == 0:
+        return w
+    seeds = tuple(s + rank * w.n_inst for s in w.seeds)
+    return Workload(w.name, seeds, w.n_req, w.n_clients, w.batch_cap, w.kv_budget, w.dist_p, w.dist_o,
+                    w.lambdas_q16, w.ls_rounds, w.cost_model)
+
+
+# ------------------------------------------------------------------------------------------
+# clocks
+# ------------------------------------------------------------------------------------------
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.rows = []
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "100",
+                 "-i", str(self.index)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            threading.Thread(target=self._read, daemon=True).start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append(line.strip())
+
+    def stop(self) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        for row in self.rows:
+            parts = [x.strip() for x in row.split(",")]
+            if len(parts) != 6:
+                continue
+            try:
+                sm.append(float(parts[0])); mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, parts[2:]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ------------------------------------------------------------------------------------------
+# our arm
+# ------------------------------------------------------------------------------------------
+class Pipeline:
+    """Device buffers of one workload and the step that runs the whole path through the C ABI."""
+
+    def __init__(self, w: Workload, device):
+        import torch
+        import paper_2502_15763_b200 as hos
+        self.torch, self.hos, self.w, self.dev = torch, hos, w, device
+        p, o = w.lengths()
+        self.p_host = torch.from_numpy(p.view(np.int32)).pin_memory()
+        self.o_host = torch.from_numpy(o.view(np.int32)).pin_memory()
+        self.lam_host = torch.from_numpy(np.asarray(w.lambdas_q16, dtype=np.uint32).view(np.int32)).pin_memory()
+        self.p = self.p_host.to(device)
+        self.o = self.o_host.to(device)
+        self.lam = self.lam_host.to(device)
+        self.ws_off = None
+        self.ws_on = None
+        self.trace = None
+        self.out = None
+        self.n_iters = 0
+
+    def args(self):
+        w = self.w
+        return (self.p, self.o, w.n_clients, w.batch_cap, w.kv_budget, w.cost_model)
+
+    def step(self):
+        hos, w = self.hos, self.w
+        sweep = len(w.lambdas_q16) > 1
+        # a multiplier sweep runs its local-search rounds per (instance, multiplier) copy, below
+        pk = hos.hos_offline_pack(*self.args(), 0 if sweep else w.ls_rounds, ws=self.ws_off)
+        lb = hos.hos_lower_bound(*self.args(), ws=self.ws_off)
+        s1 = hos.hos_online_simulate(*self.args(), pk["assign"], self.lam, hos.HOS_QUEUE_SORTED, ws=self.ws_on)
+        off = hos.hos_trace_offsets(s1["cres"])
+        if self.trace is None:                      # first (warm-up) step sizes the trace buffer
+            self.n_iters = int(off[-1].item())
+            self.trace = self.torch.empty((max(self.n_iters, 1), 16), dtype=self.torch.uint8, device=self.dev)
+        s2 = hos.hos_online_simulate(*self.args(), pk["assign"], self.lam, hos.HOS_QUEUE_SORTED,
+                                     trace=self.trace, trace_off=off, ws=self.ws_on)
+        self.out = dict(pk=pk, lb=lb, sim=s2, off=off)
+        if sweep and w.ls_rounds > 0:
+            copies = pk["assign"][:, None, :].expand(-1, len(w.lambdas_q16), -1).contiguous()
+            self.out["ls"] = hos.hos_local_search(*self.args(), copies, w.ls_rounds, ws=self.ws_off)
+        return self.out
+
+    def prepare(self):
+        """Workspaces (allocated once; the library itself allocates nothing)."""
+        import ctypes as C
+        from paper_2502_15763_b200 import binding as B
+        b = B._batch(*self.args()[:5])
+        L = self.hos.lib()
+        n_off = L.hos_offline_workspace_bytes(C.byref(b), 1, self.w.ls_rounds)
+        n_on = L.hos_online_workspace_bytes(C.byref(b), len(self.w.lambdas_q16))
+        self.ws_off = self.torch.empty(n_off, dtype=self.torch.uint8, device=self.dev)
+        self.ws_on = self.torch.empty(n_on, dtype=self.torch.uint8, device=self.dev)
+
+    def e2e_step(self, host_out):
+        """The same step from pinned host tables to pinned host results."""
+        self.p.copy_(self.p_host, non_blocking=True)
+        self.o.copy_(self.o_host, non_blocking=True)
+        self.lam.copy_(self.lam_host, non_blocking=True)
+        r = self.step()
+        srcs = (r["pk"]["assign"], r["pk"]["load"], r["pk"]["makespan_est"], r["pk"]["status"],
+                r["lb"]["lb"], r["sim"]["cres"], r["sim"]["sres"], r["sim"]["status"])
+        if not host_out:
+            host_out.extend(self.torch.empty(t.shape, dtype=t.dtype).pin_memory() for t in srcs)
+        for h, d in zip(host_out, srcs):
+            h.copy_(d, non_blocking=True)
+        h2d = sum(t.numel() * t.element_size() for t in (self.p_host, self.o_host, self.lam_host))
+        d2h = sum(t.numel() * t.element_size() for t in srcs)
+        return h2d, d2h
+
+
+def timed_steps(torch, fn, steps, flush):
+    """Sum of per-step CUDA-event times (ms); L2 is flushed between steps outside the timed spans."""
+    spans = []
+    for _ in range(steps):
+        if flush is not None:
+            flush.fill_(1)
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        fn()
+        b.record()
+        spans.append((a, b))
+    torch.cuda.synchronize()
+    return sum(a.elapsed_time(b) for a, b in spans)
+
+
+def kernel_profile(torch, hos, pipe, steps, flush):
+    """Per-kernel device time from CUDA events recorded by the library's launch hook."""
+    events = []
+
+    def hook(name, phase, stream, user):
+        ev = torch.cuda.Event(enable_timing=True)
+        ev.record()                                  # the binding launches on torch's current stream
+        events.append((name.decode(), phase, ev))
+
+    cb = hos.hos_set_launch_hook(hook)
+    try:
+        for _ in range(steps):
+            if flush is not None:
+                flush.fill_(1)
+            pipe.step()
+        torch.cuda.synchronize()
+    finally:
+        hos.hos_set_launch_hook(None)
+    del cb
+    table, order, pending = {}, [], {}
+    for name, phase, ev in events:
+        if phase == 0:
+            pending[name] = ev
+        else:
+            ms = pending.pop(name).elapsed_time(ev)
+            if name not in table:
+                table[name] = [0, 0.0]
+                order.append(name)
+            table[name][0] += 1
+            table[name][1] += ms
+    return {n: {"launches_per_step": table[n][0] / steps, "ms_per_launch": table[n][1] / table[n][0]}
+            for n in order}
+
+
+def algorithmic_bytes(w: Workload, name: str, pipe) -> float:
+    """Bytes one launch of `name` must move at least (see the design notes for the per-unit figures)."""
+    n_req_total = w.n_inst * w.n_req
+    if name in BYTES_PER_REQ:
+        extra = 64 * w.n_inst if name == "k_lower_bound" else 0
+        return BYTES_PER_REQ[name] * n_req_total + extra
+    if name == "k_local_search":
+        src = pipe.out["ls"] if "ls" in pipe.out else pipe.out["pk"]
+        applied = src["rounds_applied"].to("cpu").numpy().astype(np.int64)
+        executed = np.minimum(applied + 1, w.ls_rounds).sum()          # the no-op round is evaluated too
+        return float(executed) * (8 * w.n_req + 8 * w.n_clients)
+    if name == "k_simulate":
+        n_sims = w.n_inst * len(w.lambdas_q16)
+        # two launches per step (count pass, traced pass): each reads the queue entries and writes
+        # the client results; the traced one also writes the trace -> average per launch
+        return (8.0 * w.n_req * n_sims + 48.0 * n_sims * w.n_clients) + 16.0 * pipe.n_iters / 2
+    if name == "k_finalize":
+        return 40.0 * w.n_inst * len(w.lambdas_q16) * w.n_clients
+    if name == "k_trace_offsets":
+        return 48.0 * w.n_inst * len(w.lambdas_q16) * w.n_clients
+    return 0.0
+
+
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        try:
+            return float(json.load(open(path))["hbm_gbs"]), "measured"
+        except (OSError, KeyError, ValueError):
+            pass
+    return 6650.0, "fallback"
+
+
+def oracle_sample(w: Workload, n_sample: int):
+    """Time the CPU oracle (one thread) on the first n_sample instances: the whole path."""
+    from oracle import hos_oracle as ora
+    sub = w.subset(0, n_sample)
+    p, o = sub.lengths()
+    t0 = time.perf_counter()
+    iters = 0
+    for k in range(sub.n_inst):
+        sweep = len(w.lambdas_q16) > 1
+        pk = ora.offline_pack(p[k], o[k], w.n_clients, w.cost_model, 0 if sweep else w.ls_rounds)
+        ora.lower_bound(p[k], o[k], w.n_clients, w.batch_cap, w.cost_model)
+        for lam in w.lambdas_q16:
+            s = ora.simulate(pk["assign"], p[k], o[k], w.n_clients, w.cost_model, w.batch_cap, w.kv_budget,
+                             lam, ora.QUEUE_SORTED, want_trace=True)
+            iters += sum(c.n_prefill_iters + c.n_decode_iters for c in s.clients)
+            if sweep and w.ls_rounds > 0:      # local search on a private copy per multiplier value
+                ora.local_search(pk["T"], pk["assign"], pk["load"], w.ls_rounds)
+    dt = time.perf_counter() - t0
+    return sub.n_inst / dt, iters / dt, dt
+
+
+def sample_size(w: Workload) -> int:
+    # about 5 s of single-thread oracle work per instance at the largest size, milliseconds at the others
+    per_inst = 5.0 if w.n_req >= 10000 else 0.025 * max(1, len(w.lambdas_q16)) + 0.03
+    return max(1, min(w.n_inst, int(12.0 / per_inst)))
+
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    import paper_2502_15763_b200 as hos
+    hos.lib()
+
+    w = rank_workload(args.workload, rank)
+    pipe = Pipeline(w, dev)
+    pipe.prepare()
+    input_bytes = 2 * w.n_inst * w.n_req * 4
+    flush = None
+    if input_bytes <= (128 << 20):
+        flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=dev)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(max(args.warmup, 1)):
+        pipe.step()
+    barrier()
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    ms = timed_steps(torch, pipe.step, args.steps, flush)
+    barrier()
+    clocks = sampler.stop() if rank == 0 else None
+    ms_t = torch.tensor([ms], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(ms_t, op=dist.ReduceOp.MAX)
+    ms = float(ms_t.item())
+
+    # end to end: pinned host tables in, pinned host results out, every step
+    host_out = []
+    h2d, d2h = pipe.e2e_step(host_out)
+    barrier()
+    ms_e2e = timed_steps(torch, lambda: pipe.e2e_step(host_out), args.steps, flush)
+    barrier()
+    e_t = torch.tensor([ms_e2e], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(e_t, op=dist.ReduceOp.MAX)
+    ms_e2e = float(e_t.item())
+
+    st = pipe.out
+    bad = int((st["pk"]["status"] != 0).sum().item()) + int((st["sim"]["status"] != 0).sum().item())
+    if bad:
+        raise SystemExit(f"bench: {bad} units finished with a non-zero status")
+
+    if rank == 0:
+        prof = kernel_profile(torch, hos, pipe, max(2, min(args.steps, 5)), flush)
+        peak, peak_kind = measured_peak()
+        rows = {}
+        for name, r in prof.items():
+            by = algorithmic_bytes(w, name, pipe)
+            gbs = by / (r["ms_per_launch"] * 1e-3) / 1e9
+            rows[name] = dict(r, algorithmic_bytes=by, achieved_gbs=gbs, frac=gbs / peak,
+                              ms_per_step=r["ms_per_launch"] * r["launches_per_step"])
+        top = max(rows, key=lambda n: rows[n]["ms_per_step"])
+        roofline = {"kernel": top, "bound": "hbm", "achieved": rows[top]["achieved_gbs"], "peak": peak,
+                    "unit": "GB/s", "frac": rows[top]["frac"], "traffic": None,
+                    "peak_source": f"of {peak_kind}", "ms_per_launch": rows[top]["ms_per_launch"]}
+        launches = sum(r["launches_per_step"] for r in prof.values())
+        n_s = sample_size(w)
+        cpu_inst, cpu_iters, cpu_dt = oracle_sample(w, n_s)
+        total_inst = w.n_inst * world
+        line = {
+            "metric": METRIC, "value": total_inst * args.steps / (ms * 1e-3), "unit": UNIT,
+            "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms / args.steps,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": DTYPE,
+            "data": "synthetic",
+            "config": {"workload": describe(w), "instances_per_gpu": w.n_inst,
+                       "l2": ("inputs larger than L2" if flush is None else "L2 flushed between steps")},
+            "sim_iterations_per_step": pipe.n_iters * world,
+            "sim_iterations_per_s": 2 * pipe.n_iters * world * args.steps / (ms * 1e-3),
+            "clocks": clocks,
+            "e2e": {"value": total_inst * args.steps / (ms_e2e * 1e-3), "unit": UNIT,
+                    "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                    "note": "results copied back: assignment, loads, bounds, client and simulation results; "
+                            "the iteration trace stays on the device"},
+            "gpu_launches": int(round(launches * args.steps)),
+            "roofline": roofline,
+            "kernels": rows,
+            "cpu_baseline": {"value": cpu_inst, "unit": UNIT, "cores": 1, "kind": "oracle",
+                             "sample": f"first {n_s} instance(s) of the workload, whole path, {cpu_dt:.1f} s",
+                             "sim_iterations_per_s": cpu_iters},
+        }
+        print(json.dumps(line))
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def run_reference(args):
+    """The CPU oracle as it stands, one thread, on a bounded sample of the workload per step."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    w = workload(args.workload)
+    n_s = max(1, sample_size(w) // 2)
+    for _ in range(args.warmup):
+        oracle_sample(w, 1)
+    t0 = time.perf_counter()
+    iters_per_s = 0.0
+    for _ in range(args.steps):
+        _, it, _ = oracle_sample(w, n_s)
+        iters_per_s += it / args.steps
+    dt = time.perf_counter() - t0
+    value = n_s * args.steps / dt
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT,
+        "n_gpus": int(os.environ.get("WORLD_SIZE", "1")), "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": dt * 1e3 / args.steps, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": DTYPE, "data": "synthetic",
+        "config": {"workload": describe(w), "sample_instances_per_step": n_s},
+        "sim_iterations_per_s": iters_per_s,
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle",
+                         "sample": f"first {n_s} instance(s) of the workload per step, whole path"},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--workload", default="c4", choices=["c0", "c1", "c2", "c3", "c4"])
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -185,6 +185,17 @@ size_t hos_online_workspace_bytes(const hos_batch* batch, int n_lambda);
 
 const char* hos_strerror(int code);
 
+/*
+ * Measurement aid (no counterpart in the paper).  When a hook is set, every kernel launch of
+ * the library is bracketed by hook(kernel_name, 0, stream, user) and
+ * hook(kernel_name, 1, stream, user), called on the host from the launching thread, so that
+ * a caller can record CUDA events on the launching stream and count launches.  Process-wide
+ * and not thread-safe: set it only while no other thread is inside the library; pass NULL
+ * to remove it.  With no hook set the library keeps no state between calls.
+ */
+typedef void (*hos_launch_hook)(const char* kernel, int phase, void* stream, void* user);
+void hos_set_launch_hook(hos_launch_hook hook, void* user);
+
 #ifdef __cplusplus
 }
 #endif

@@ -30,7 +30,9 @@ ITER_REC_DTYPE = np.dtype([("dur_us", "<u4"), ("kind_n", "<u4"), ("tokens", "<u4
 
 _SYMBOLS = ("hos_offline_pack", "hos_local_search", "hos_lower_bound", "hos_online_simulate",
             "hos_trace_offsets", "hos_offline_workspace_bytes", "hos_lower_bound_workspace_bytes",
-            "hos_online_workspace_bytes", "hos_strerror")
+            "hos_online_workspace_bytes", "hos_strerror", "hos_set_launch_hook")
+
+LAUNCH_HOOK = C.CFUNCTYPE(None, C.c_char_p, C.c_int, C.c_void_p, C.c_void_p)
 
 
 class HosError(RuntimeError):
@@ -74,6 +76,19 @@ def lib():
             getattr(L, name).restype = C.c_int
         _lib = L
     return _lib
+
+
+def hos_set_launch_hook(fn):
+    """fn(kernel_name: bytes, phase: int, stream: int, user) around every kernel launch; None removes it.
+
+    Returns the ctypes callback object, which the caller must keep alive while it is set."""
+    L = lib()
+    if fn is None:
+        L.hos_set_launch_hook(None, None)
+        return None
+    cb = LAUNCH_HOOK(fn)
+    L.hos_set_launch_hook(cb, None)
+    return cb
 
 
 def exported_symbols() -> Sequence[str]:

@@ -85,7 +85,16 @@ OnlineWs carve_online(const hos_batch* b, void* ws) {
 
 inline int cuda_rc(cudaError_t e) { return e == cudaSuccess ? HOS_OK : HOS_E_CUDA; }
 
+hos_launch_hook g_hook = nullptr;
+void* g_hook_user = nullptr;
+
 }  // namespace
+
+namespace hos {
+void launch_hook(const char* kernel, int phase, cudaStream_t st) {
+    if (g_hook) g_hook(kernel, phase, static_cast<void*>(st), g_hook_user);
+}
+}  // namespace hos
 
 extern "C" {
 
@@ -199,6 +208,11 @@ int hos_trace_offsets(const hos_client_result* cres, int64_t n_units, int64_t* t
     if (!cres || !trace_off || n_units < 0) return HOS_E_INVALID;
     return cuda_rc(launch_trace_offsets(cres, (long long)n_units, reinterpret_cast<long long*>(trace_off),
                                         static_cast<cudaStream_t>(stream)));
+}
+
+void hos_set_launch_hook(hos_launch_hook hook, void* user) {
+    g_hook = hook;
+    g_hook_user = user;
 }
 
 const char* hos_strerror(int code) {

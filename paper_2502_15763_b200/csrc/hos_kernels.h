@@ -10,6 +10,9 @@ namespace hos {
 
 struct InstInfo;
 
+// Calls the user's launch hook, if one is set (see hos_set_launch_hook).
+void launch_hook(const char* kernel, int phase, cudaStream_t st);
+
 size_t estimate_sort_smem(int n_req);
 size_t local_search_smem(int n_req);
 size_t queue_build_smem(int n_req);

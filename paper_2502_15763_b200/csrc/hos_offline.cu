@@ -522,9 +522,11 @@ cudaError_t launch_estimate_sort(const hos_batch& b, const hos_cost_model& cm, u
     auto kern = b.n_req <= 65536 ? k_estimate_sort<uint16_t> : k_estimate_sort<uint32_t>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
+    launch_hook("k_estimate_sort", 0, st);
     kern<<<b.n_inst, SORT_THREADS, smem, st>>>(b.p, b.o, b.n_req, (long long)b.kv_budget,
                                                cm.est_per_prompt_token, cm.est_per_output_token,
                                                T_sorted, order, info, status_out, n_pad);
+    launch_hook("k_estimate_sort", 1, st);
     return cudaGetLastError();
 }
 
@@ -535,11 +537,13 @@ cudaError_t launch_lpt(const hos_batch& b, const uint32_t* T_sorted, const uint3
 #define HOS_LPT(KPL)                                                                               \
     k_lpt<KPL><<<b.n_inst, 32, 0, st>>>(T_sorted, order, info, b.n_req, n_pad, M, assign, load,    \
                                          makespan)
+    launch_hook("k_lpt", 0, st);
     if (M <= 32) HOS_LPT(1);
     else if (M <= 64) HOS_LPT(2);
     else if (M <= 128) HOS_LPT(4);
     else HOS_LPT(8);
 #undef HOS_LPT
+    launch_hook("k_lpt", 1, st);
     return cudaGetLastError();
 }
 
@@ -552,17 +556,21 @@ cudaError_t launch_local_search(const hos_batch& b, const uint32_t* T_sorted, co
     auto kern = b.n_req <= 65536 ? k_local_search<uint16_t> : k_local_search<uint32_t>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
+    launch_hook("k_local_search", 0, st);
     kern<<<b.n_inst * n_copies, SORT_THREADS, smem, st>>>(T_sorted, order, info, b.n_req, n_pad,
                                                           b.n_clients, n_copies, rounds,
                                                           load_from_assign, assign, load, makespan,
                                                           rounds_applied, ls_log, status);
+    launch_hook("k_local_search", 1, st);
     return cudaGetLastError();
 }
 
 cudaError_t launch_lower_bound(const hos_batch& b, const hos_cost_model& cm, const uint32_t* T_sorted,
                                const InstInfo* info, int n_pad, hos_lb* out, cudaStream_t st) {
+    launch_hook("k_lower_bound", 0, st);
     k_lower_bound<<<b.n_inst, 256, 0, st>>>(b.p, b.o, b.n_req, n_pad, b.n_clients, b.batch_cap, cm,
                                             T_sorted, info, out);
+    launch_hook("k_lower_bound", 1, st);
     return cudaGetLastError();
 }
 

@@ -357,9 +357,11 @@ cudaError_t launch_queue_build(const hos_batch& b, const int32_t* assign, int qu
     auto kern = b.n_req <= 65536 ? k_queue_build<uint16_t> : k_queue_build<uint32_t>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
+    launch_hook("k_queue_build", 0, st);
     kern<<<b.n_inst, SORT_THREADS, smem, st>>>(b.p, b.o, assign, b.n_req, b.n_clients,
                                                (long long)b.kv_budget, queue_order, q_po, q_req, q_off,
                                                inst_O, inst_status, n_pad);
+    launch_hook("k_queue_build", 1, st);
     return cudaGetLastError();
 }
 
@@ -375,25 +377,31 @@ cudaError_t launch_simulate(const hos_batch& b, const hos_cost_model& cm, const 
                                                      b.n_clients, n_pad, n_units, b.batch_cap,     \
                                                      (uint32_t)b.kv_budget, cm, max_iters, cres,   \
                                                      trace, trace_off, status)
+    launch_hook("k_simulate", 0, st);
     if (b.batch_cap <= 32) HOS_SIM(1);
     else if (b.batch_cap <= 64) HOS_SIM(2);
     else if (b.batch_cap <= 128) HOS_SIM(4);
     else HOS_SIM(8);
 #undef HOS_SIM
+    launch_hook("k_simulate", 1, st);
     return cudaGetLastError();
 }
 
 cudaError_t launch_finalize(const hos_batch& b, int n_lambda, const unsigned long long* inst_O,
                             hos_client_result* cres, hos_sim_result* sres, cudaStream_t st) {
     const int n_sims = b.n_inst * n_lambda;
+    launch_hook("k_finalize", 0, st);
     k_finalize<<<(n_sims + 3) / 4, 128, 0, st>>>(n_sims, n_lambda, b.n_clients, b.batch_cap, inst_O,
                                                  cres, sres);
+    launch_hook("k_finalize", 1, st);
     return cudaGetLastError();
 }
 
 cudaError_t launch_trace_offsets(const hos_client_result* cres, long long n_units, long long* trace_off,
                                  cudaStream_t st) {
+    launch_hook("k_trace_offsets", 0, st);
     k_trace_offsets<<<1, 1024, 0, st>>>(cres, n_units, trace_off);
+    launch_hook("k_trace_offsets", 1, st);
     return cudaGetLastError();
 }
 
