@@ -44,9 +44,11 @@ def describe(w: Workload) -> str:
             f"{w.ls_rounds} local-search rounds")
 
 
-def rank_workload(name: str, rank: int) -> Workload:
+def rank_workload(name: str, rank: int, instances: int = 0) -> Workload:
     """Rank r evaluates the same number of instances with seeds shifted by r * n_inst."""
     w = workload(name)
+    if instances > 0:
+        w = w.subset(0, min(instances, w.n_inst))
     if rank == 0:
         return w
     seeds = tuple(s + rank * w.n_inst for s in w.seeds)
@@ -303,7 +305,7 @@ def run_ours(args):
     import paper_2502_15763_b200 as hos
     hos.lib()
 
-    w = rank_workload(args.workload, rank)
+    w = rank_workload(args.workload, rank, args.instances)
     pipe = Pipeline(w, dev)
     pipe.prepare()
     input_bytes = 2 * w.n_inst * w.n_req * 4
@@ -362,7 +364,10 @@ def run_ours(args):
                     "peak_source": f"of {peak_kind}", "ms_per_launch": rows[top]["ms_per_launch"]}
         launches = sum(r["launches_per_step"] for r in prof.values())
         n_s = sample_size(w)
-        cpu_inst, cpu_iters, cpu_dt = oracle_sample(w, n_s)
+        if args.skip_cpu_baseline:
+            cpu_inst, cpu_iters, cpu_dt = None, None, 0.0
+        else:
+            cpu_inst, cpu_iters, cpu_dt = oracle_sample(w, n_s)
         total_inst = w.n_inst * world
         line = {
             "metric": METRIC, "value": total_inst * args.steps / (ms * 1e-3), "unit": UNIT,
@@ -428,6 +433,10 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--workload", default="c4", choices=["c0", "c1", "c2", "c3", "c4"])
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--instances", type=int, default=0,
+                    help="use only the first N instances of the workload (profiling captures)")
+    ap.add_argument("--skip-cpu-baseline", action="store_true",
+                    help="do not time the CPU oracle (profiling captures)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
