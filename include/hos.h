@@ -40,7 +40,8 @@ enum {
     HOS_E_INVALID     = -1,   /* null pointer, non-positive size, inconsistent arguments        */
     HOS_E_WORKSPACE   = -2,   /* workspace smaller than hos_*_workspace_bytes, or misaligned     */
     HOS_E_CUDA        = -3,   /* a CUDA runtime call failed (see cudaGetLastError)               */
-    HOS_E_UNSUPPORTED = -4    /* shape outside the limits listed above                           */
+    HOS_E_UNSUPPORTED = -4,   /* shape outside the limits listed above                           */
+    HOS_E_TOO_LARGE   = -5    /* batch needs more scratch than hos_lower_bound_static has built in */
 };
 
 /* bits of the per-unit device status words */
@@ -172,6 +173,35 @@ int hos_online_simulate(const hos_batch* batch, const int32_t* assign, const hos
                         hos_client_result* cres, hos_sim_result* sres,
                         hos_iter_rec* trace, const int64_t* trace_off, int32_t* status,
                         void* ws, size_t ws_bytes, void* stream);
+
+/*
+ * The lower bounds again, for callers that must not allocate.  (The paper has no counterpart:
+ * this is a packaging variant of hos_lower_bound, same results bit for bit.)
+ *
+ * Who needs it: a scheduler that runs next to an inference engine usually finds the device
+ * already carved up -- the engine reserved nearly all of HBM for weights and KV cache at
+ * start-up, so a cudaMalloc may fail, and even a successful one synchronises the device in the
+ * middle of a serving loop.  The same holds for plug-ins that live inside another framework's
+ * memory pool and have no allocator of their own.  Such callers pass only inputs and outputs;
+ * the scratch that hos_lower_bound asks its caller for sits in a fixed array of
+ * HOS_STATIC_SCRATCH_BYTES inside the library's device image.  Every GPU that loads the
+ * library carries that array until the process exits, whether or not this call is used.
+ *
+ *   - The call itself allocates and frees nothing, on host or device.
+ *   - Size limit: hos_lower_bound_workspace_bytes(batch) must not exceed
+ *     HOS_STATIC_SCRATCH_BYTES (about n_inst * n_req <= 1,000,000 requests); larger batches
+ *     get HOS_E_TOO_LARGE and nothing is enqueued.  Split them, or use hos_lower_bound.
+ *   - The first call on each device looks up the array's device address (with that device
+ *     current) and remembers it.  Make that first call outside any stream capture.
+ *   - All calls on one device share the one array and find the previous call's leftovers in
+ *     it; the kernels overwrite everything they later read, so no clearing is needed.  Two
+ *     calls that may run at the same time on the same GPU (different streams, or different
+ *     host threads without ordering) race on the array: order them on one stream.
+ * out [n_inst], status [n_inst] as in hos_lower_bound.
+ */
+#define HOS_STATIC_SCRATCH_BYTES (8u << 20)
+int hos_lower_bound_static(const hos_batch* batch, const hos_cost_model* cm, hos_lb* out,
+                           int32_t* status, void* stream);
 
 /* trace_off[0] = 0, trace_off[x+1] = trace_off[x] + iterations of unit x (exclusive scan of
  * n_prefill_iters + n_decode_iters over cres[0..n_units)).  The trace protocol of

@@ -30,7 +30,8 @@ ITER_REC_DTYPE = np.dtype([("dur_us", "<u4"), ("kind_n", "<u4"), ("tokens", "<u4
 
 _SYMBOLS = ("hos_offline_pack", "hos_local_search", "hos_lower_bound", "hos_online_simulate",
             "hos_trace_offsets", "hos_offline_workspace_bytes", "hos_lower_bound_workspace_bytes",
-            "hos_online_workspace_bytes", "hos_strerror", "hos_set_launch_hook")
+            "hos_online_workspace_bytes", "hos_strerror", "hos_set_launch_hook",
+            "hos_lower_bound_static")
 
 LAUNCH_HOOK = C.CFUNCTYPE(None, C.c_char_p, C.c_int, C.c_void_p, C.c_void_p)
 
@@ -72,7 +73,7 @@ def lib():
             getattr(L, name).restype = C.c_size_t
         L.hos_strerror.restype = C.c_char_p
         for name in ("hos_offline_pack", "hos_local_search", "hos_lower_bound",
-                     "hos_online_simulate", "hos_trace_offsets"):
+                     "hos_online_simulate", "hos_trace_offsets", "hos_lower_bound_static"):
             getattr(L, name).restype = C.c_int
         _lib = L
     return _lib
@@ -217,6 +218,20 @@ def hos_lower_bound(p, o, n_clients: int, batch_cap: int, kv_budget: int, cost_m
     rc = L.hos_lower_bound(C.byref(b), C.byref(cm), _ptr(out), _ptr(status), _ptr(ws),
                            C.c_size_t(ws.numel()), _stream())
     _check(rc, "hos_lower_bound")
+    return dict(lb=out, status=status)
+
+
+def hos_lower_bound_static(p, o, n_clients: int, batch_cap: int, kv_budget: int, cost_model):
+    """hos_lower_bound without a caller workspace: for code that may not allocate device memory
+    (the scratch is a fixed array inside the library; batches beyond it raise HosError -5).
+    The result tensors here are the caller's outputs; the C call itself allocates nothing."""
+    torch = _torch()
+    b = _batch(p, o, n_clients, batch_cap, kv_budget)
+    cm = _cost(cost_model)
+    out = torch.empty((b.n_inst, LB_DTYPE.itemsize), dtype=torch.uint8, device=p.device)
+    status = torch.empty((b.n_inst,), dtype=torch.int32, device=p.device)
+    rc = lib().hos_lower_bound_static(C.byref(b), C.byref(cm), _ptr(out), _ptr(status), _stream())
+    _check(rc, "hos_lower_bound_static")
     return dict(lb=out, status=status)
 
 

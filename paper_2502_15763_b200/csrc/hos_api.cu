@@ -222,6 +222,7 @@ const char* hos_strerror(int code) {
         case HOS_E_WORKSPACE: return "workspace missing, too small or not 256-byte aligned";
         case HOS_E_CUDA: return "CUDA runtime error";
         case HOS_E_UNSUPPORTED: return "shape outside the supported limits";
+        case HOS_E_TOO_LARGE: return "batch exceeds the built-in scratch of hos_lower_bound_static";
         default: return "unknown error code";
     }
 }
