@@ -103,10 +103,16 @@ k_lpt(const uint32_t* __restrict__ T_sorted, const uint32_t* __restrict__ order,
             const int j = k * 32 + lane;
             key[k] = (j < n_clients) ? (uint32_t)j : 0xFFFFFFFFu;
         }
+        unsigned long long rebased = 0;                 // sum of the bases subtracted so far
+        uint32_t tv_next = (lane < n_req) ? Ts[lane] : 0u;
+        uint32_t rq_next = (lane < n_req) ? od[lane] : 0u;
         for (int r0 = 0; r0 < n_req; r0 += 32) {
             const int r = r0 + lane;
-            const uint32_t tv = (r < n_req) ? Ts[r] : 0u;
-            const uint32_t rq = (r < n_req) ? od[r] : 0u;
+            const uint32_t tsh = tv_next << JB;         // this chunk's items, already in key units
+            const uint32_t rq = rq_next;
+            const int rn = r + 32;                      // prefetch the next chunk behind the chain
+            tv_next = (rn < n_req) ? Ts[rn] : 0u;
+            rq_next = (rn < n_req) ? od[rn] : 0u;
             const int steps = min(32, n_req - r0);
             uint32_t mine = 0;
             for (int sidx = 0; sidx < steps; ++sidx) {
@@ -115,13 +121,11 @@ k_lpt(const uint32_t* __restrict__ T_sorted, const uint32_t* __restrict__ order,
                 for (int k = 1; k < KPL; ++k) m = min(m, key[k]);
                 const uint32_t g = __reduce_min_sync(FULL, m);
                 const uint32_t j = g & ((1u << JB) - 1u);
-                const uint32_t t = __shfl_sync(FULL, tv, sidx);
-                if (lane == (int)(j & 31u)) {
+                const uint32_t t = __shfl_sync(FULL, tsh, sidx);
+                const bool own = lane == (int)(j & 31u);
 #pragma unroll
-                    for (int k = 0; k < KPL; ++k)
-                        if ((int)(j >> 5) == k) { key[k] += t << JB; load[k] += t; }
-                }
-                if (lane == sidx) mine = j;
+                for (int k = 0; k < KPL; ++k) key[k] += (own && (int)(j >> 5) == k) ? t : 0u;
+                mine = (lane == sidx) ? j : mine;
             }
             if (r < n_req) asg[rq] = (int32_t)mine;
             // re-base: subtract the current least relative load from every real key
@@ -129,10 +133,14 @@ k_lpt(const uint32_t* __restrict__ T_sorted, const uint32_t* __restrict__ order,
 #pragma unroll
             for (int k = 1; k < KPL; ++k) m = min(m, key[k]);
             const uint32_t base = (__reduce_min_sync(FULL, m) >> JB) << JB;
+            rebased += base >> JB;
 #pragma unroll
             for (int k = 0; k < KPL; ++k)
                 if (k * 32 + lane < n_clients) key[k] -= base;
         }
+#pragma unroll
+        for (int k = 0; k < KPL; ++k)
+            if (k * 32 + lane < n_clients) load[k] = (long long)(rebased + (key[k] >> JB));
     } else {
         for (int r0 = 0; r0 < n_req; r0 += 32) {
             const int r = r0 + lane;
@@ -155,12 +163,10 @@ k_lpt(const uint32_t* __restrict__ T_sorted, const uint32_t* __restrict__ order,
                     if (ol < bl || (ol == bl && oj < bj)) { bl = ol; bj = oj; }
                 }
                 const uint32_t t = __shfl_sync(FULL, tv, sidx);
-                if (lane == (bj & 31)) {
+                const bool own = lane == (bj & 31);
 #pragma unroll
-                    for (int k = 0; k < KPL; ++k)
-                        if ((bj >> 5) == k) load[k] += t;
-                }
-                if (lane == sidx) mine = (uint32_t)bj;
+                for (int k = 0; k < KPL; ++k) load[k] += (own && (bj >> 5) == k) ? (long long)t : 0ll;
+                mine = (lane == sidx) ? (uint32_t)bj : mine;
             }
             if (r < n_req) asg[rq] = (int32_t)mine;
         }
@@ -229,7 +235,8 @@ k_local_search(const uint32_t* __restrict__ T_sorted, const uint32_t* __restrict
     __shared__ long long s_load[MAX_CLIENTS];
     __shared__ Cand s_cand[32];
     __shared__ int s_wcnt[32];
-    __shared__ int s_jmax, s_nm;
+    __shared__ int s_jmax, s_nm, s_kmin;
+    __shared__ long long s_vb[32];
     __shared__ long long s_lmax;
 
     const int inst = blockIdx.x / n_copies;
@@ -304,6 +311,19 @@ k_local_search(const uint32_t* __restrict__ T_sorted, const uint32_t* __restrict
                 if (ol > bl || (ol == bl && oj < bj)) { bl = ol; bj = oj; }
             }
             if (lane == 0) { s_jmax = bj; s_lmax = bl; }
+            // least loaded other client (any of them on ties: it only seeds the pruning bound)
+            const int jm = __shfl_sync(FULL, bj, 0);
+            long long ml = NO_V;
+            int mj = -1;
+            for (int j = lane; j < n_clients; j += 32)
+                if (j != jm && s_load[j] < ml) { ml = s_load[j]; mj = j; }
+#pragma unroll
+            for (int d = 16; d > 0; d >>= 1) {
+                const long long ol = __shfl_xor_sync(FULL, ml, d);
+                const int oj = __shfl_xor_sync(FULL, mj, d);
+                if (ol < ml) { ml = ol; mj = oj; }
+            }
+            if (lane == 0) s_kmin = mj;
         }
         __syncthreads();
         const int jmax = s_jmax;
@@ -341,18 +361,20 @@ k_local_search(const uint32_t* __restrict__ T_sorted, const uint32_t* __restrict
         const int nm = s_nm;
 
         // (c) candidates: work item w < n_req is "swap with the request of rank w";
-        //     w >= n_req is "move to client w - n_req"
-        Cand best;
-        best.v = NO_V; best.i = NO_I; best.k = NO_I; best.u = NO_I; best.ri = -1; best.ru = -1;
-        for (int w = threadIdx.x; w < n_req + n_clients; w += SORT_THREADS) {
+        //     w >= n_req is "move to client w - n_req".
+        //     Any step onto client k ends with v >= ceil((Lmax + load_k) / 2).  A first sweep over
+        //     the least loaded client alone gives an achievable v (`vbound`); the full sweep then
+        //     skips every client whose floor is above it.  Ties in v survive the filter.
+        auto evaluate = [&](int w, Cand& best, long long vbound) {
             int k, u, ru;
             long long Tu;
-            if (w < n_req) { k = bins[w]; u = (int)ord[w]; ru = w; Tu = Ts[w]; }
+            if (w < n_req) { k = bins[w]; u = -2; ru = w; Tu = Ts[w]; }
             else { k = w - n_req; u = -1; ru = -1; Tu = 0; }
-            if (k == jmax) continue;
+            if (k == jmax) return;
             const long long lk = s_load[k];
             const long long slack = Lmax - lk;
-            if (slack <= 0) continue;
+            if (slack <= 0 || ((Lmax + lk + 1) >> 1) > vbound) return;
+            if (u == -2) u = (int)ord[w];
             const long long thr = Tu + ((slack + 1) >> 1);      // T_i >= thr  <=>  2 d >= slack
             // b = number of members with T >= thr (members are sorted by T descending)
             int a = 0, z = nm;
@@ -385,7 +407,27 @@ k_local_search(const uint32_t* __restrict__ T_sorted, const uint32_t* __restrict
                     if (cand_less(c, best)) best = c;
                 }
             }
+        };
+        Cand best;
+        best.v = NO_V; best.i = NO_I; best.k = NO_I; best.u = NO_I; best.ri = -1; best.ru = -1;
+        const int kmin = s_kmin;
+        if (kmin >= 0) {
+            for (int w = threadIdx.x; w < n_req + n_clients; w += SORT_THREADS) {
+                const int k = (w < n_req) ? (int)bins[w] : w - n_req;
+                if (k == kmin) evaluate(w, best, NO_V);
+            }
         }
+        long long vb = best.v;
+#pragma unroll
+        for (int d = 16; d > 0; d >>= 1) vb = min(vb, __shfl_xor_sync(FULL, vb, d));
+        if (lane == 0) s_vb[warp] = vb;
+        __syncthreads();
+        vb = s_vb[lane];
+#pragma unroll
+        for (int d = 16; d > 0; d >>= 1) vb = min(vb, __shfl_xor_sync(FULL, vb, d));
+        const long long vbound = vb;
+        best.v = NO_V; best.i = NO_I; best.k = NO_I; best.u = NO_I; best.ri = -1; best.ru = -1;
+        for (int w = threadIdx.x; w < n_req + n_clients; w += SORT_THREADS) evaluate(w, best, vbound);
         // (d) CTA-wide lexicographic minimum
 #pragma unroll
         for (int d = 16; d > 0; d >>= 1) {

@@ -76,11 +76,14 @@ k_queue_build(const uint32_t* __restrict__ p, const uint32_t* __restrict__ o,
 }
 
 // ---------------------------------------------------------------------------------------
-// Iteration-level simulator.  One warp per (instance, multiplier, client).  The running
-// batch lives in registers: slot = (lane, k), k < SPL, batch_cap <= 32 * SPL.  A slot keeps
-// the decode-iteration count at which its request retires (`fin`) and the request's p + o
-// (`tot`): the KV length at count c is tot - fin + c, so a decode iteration touches no slot
-// unless someone retires, and sum KV is carried along (S += B - sum of retired tot).
+// Iteration-level simulator.  One THREAD per (instance, multiplier, client): the per-client
+// recurrence (duration, clock, waited decode time, decision, hash) is scalar work, so every
+// lane of a warp runs a client of its own.  The running batch of a client is a binary
+// min-heap in shared memory, keyed by the decode-iteration count at which a request retires
+// (`fin`) with the request's p + o (`tot`) as payload, laid out [slot][lane] so that lanes
+// never collide on a bank whatever slots they touch.  The KV length of a request at count c
+// is tot - fin + c, so a decode iteration touches the heap only when someone retires, and
+// sum KV is carried along: S += B - sum of retired tot.
 // ---------------------------------------------------------------------------------------
 constexpr uint32_t EMPTY = 0xFFFFFFFFu;
 constexpr unsigned long long HASH_INIT = 0xCBF29CE484222325ull;
@@ -90,28 +93,27 @@ constexpr unsigned long long HASH_W1 = 0x94D049BB133111EBull;
 constexpr unsigned long long HASH_W2 = 0xD6E8FEB86659FD93ull;
 constexpr unsigned long long HASH_W3 = 0xA0761D6478BD642Full;
 constexpr unsigned long long HASH_W4 = 0xE7037ED1A0B428DBull;
-constexpr int SIM_WARPS = 4;
+constexpr int SIM_THREADS = 32;          // one warp per CTA: a warp leaves as soon as its clients are done
 
-template <int SPL>
-__global__ void __launch_bounds__(SIM_WARPS * 32)
+__global__ void __launch_bounds__(SIM_THREADS)
 k_simulate(const uint2* __restrict__ q_po, const int32_t* __restrict__ q_off,
            const int32_t* __restrict__ inst_status, const uint32_t* __restrict__ lambda_q16,
            int n_lambda, int n_clients, int n_pad, long long n_units, int cap, uint32_t kv_budget,
-           hos_cost_model cm, uint32_t max_iters, hos_client_result* __restrict__ cres,
+           hos_cost_model cm, int q_shift, uint32_t max_iters, hos_client_result* __restrict__ cres,
            hos_iter_rec* __restrict__ trace, const long long* __restrict__ trace_off,
            int32_t* __restrict__ status_out) {
-    const long long unit = (long long)blockIdx.x * SIM_WARPS + warp_id();
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    unsigned long long* heap = reinterpret_cast<unsigned long long*>(smem_raw) + threadIdx.x;
+#define HEAP(s) heap[(s) * SIM_THREADS]
+    const long long unit = (long long)blockIdx.x * SIM_THREADS + threadIdx.x;
     if (unit >= n_units) return;
-    const int lane = lane_id();
     const int c = (int)(unit % n_clients);
     const int l = (int)((unit / n_clients) % n_lambda);
     const int inst = (int)(unit / ((long long)n_clients * n_lambda));
 
     if (inst_status[inst]) {
-        if (lane == 0) {
-            cres[unit] = hos_client_result{0, 0, 0u, 0u, 0ull, 0.0};
-            status_out[unit] = inst_status[inst];
-        }
+        cres[unit] = hos_client_result{0, 0, 0u, 0u, 0ull, 0.0};
+        status_out[unit] = inst_status[inst];
         return;
     }
     const int q0 = q_off[(size_t)inst * (n_clients + 1) + c];
@@ -121,58 +123,34 @@ k_simulate(const uint2* __restrict__ q_po, const int32_t* __restrict__ q_off,
     const uint32_t ap = cm.prefill_fixed_us, bp = cm.prefill_per_token_us;
     const uint32_t ad = cm.decode_fixed_us, bd = cm.decode_per_seq_us, qd = cm.decode_kv_div;
 
-    uint32_t fin[SPL], tot[SPL];
-#pragma unroll
-    for (int k = 0; k < SPL; ++k) { fin[k] = EMPTY; tot[k] = 0; }
-
     long long t = 0, busy = 0;
     uint32_t Cd = 0, cnt = 0, B = 0, S = 0, reserved = 0, iters = 0, n_pre = 0, n_dec = 0;
     uint32_t next_fin = EMPTY;
     int head = 0;
     unsigned long long hash = HASH_INIT, pw = 1ull;
     uint32_t nA = 0, sumP = 0, sumTot = 0;
-    bool dirty = true;
+    bool grow = true;                        // the candidate prefix may extend
     int32_t status = 0;
 
-    hos_iter_rec* tr = nullptr;
+    uint4* tr = nullptr;
     long long tr_cap = 0;
     if (trace) {
         const long long t0 = trace_off[unit];
-        tr = trace + t0;
+        tr = reinterpret_cast<uint4*>(trace + t0);
         tr_cap = trace_off[unit + 1] - t0;
     }
-    uint4 held = make_uint4(0, 0, 0, 0);                 // lane x holds record (iters & ~31) + x
 
     while (true) {
-        if (dirty) {
-            // candidates: longest queue prefix that fits the free slots and the KV budget
-            nA = 0; sumP = 0; sumTot = 0;
-            int pos = head;
-            while (pos < qn && B + nA < (uint32_t)cap) {
-                const int e = pos + lane;
-                uint2 po = make_uint2(0u, 0u);
-                if (e < qn) po = __ldg(&q[e]);
-                unsigned long long it = (unsigned long long)po.x + po.y;   // inclusive sums
-                unsigned long long ip = po.x;
-#pragma unroll
-                for (int d = 1; d < 32; d <<= 1) {
-                    const unsigned long long yt = __shfl_up_sync(FULL, it, d);
-                    const unsigned long long yp = __shfl_up_sync(FULL, ip, d);
-                    if (lane >= d) { it += yt; ip += yp; }
-                }
-                const bool ok = e < qn && (B + nA + (uint32_t)lane < (uint32_t)cap) &&
-                                ((unsigned long long)reserved + sumTot + it <= (unsigned long long)kv_budget);
-                const unsigned okm = __ballot_sync(FULL, ok);
-                const int take = (okm == FULL) ? 32 : (__ffs(~okm) - 1);
-                if (take > 0) {
-                    sumTot += (uint32_t)__shfl_sync(FULL, it, take - 1);
-                    sumP += (uint32_t)__shfl_sync(FULL, ip, take - 1);
-                    nA += take;
-                }
-                if (take < 32) break;
-                pos += 32;
+        if (grow) {
+            // candidates: the longest queue prefix that fits the free slots and the KV budget.
+            // A retirement only loosens both limits, so the prefix found earlier stays valid.
+            while (head + (int)nA < qn && B + nA < (uint32_t)cap) {
+                const uint2 po = __ldg(&q[head + nA]);
+                const uint32_t tt = po.x + po.y;
+                if ((unsigned long long)reserved + sumTot + tt > (unsigned long long)kv_budget) break;
+                sumTot += tt; sumP += po.x; ++nA;
             }
-            dirty = false;
+            grow = false;
         }
         if (B == 0 && nA == 0) break;                    // queue empty and nothing running
         if (iters == max_iters) { status |= HOS_ST_LIMIT; break; }
@@ -182,60 +160,57 @@ k_simulate(const uint2* __restrict__ q_po, const int32_t* __restrict__ q_off,
             nA > 0 && (B == 0 || (unsigned long long)lam * Cd > ((unsigned long long)Cp << 16));
         uint32_t dur, r1, r2, r3;
         if (prefill) {
-            // admit queue[head .. head + nA) into free slots
-            int nfree = 0;
-#pragma unroll
-            for (int k = 0; k < SPL; ++k) nfree += (fin[k] == EMPTY);
-            int g = nfree;
-#pragma unroll
-            for (int d = 1; d < 32; d <<= 1) {
-                const int y = __shfl_up_sync(FULL, g, d);
-                if (lane >= d) g += y;
-            }
-            g -= nfree;                                   // exclusive: free slots in lower lanes
-#pragma unroll
-            for (int k = 0; k < SPL; ++k) {
-                if (fin[k] == EMPTY) {
-                    if ((uint32_t)g < nA) {
-                        const uint2 po = __ldg(&q[head + g]);
-                        fin[k] = cnt + po.y;
-                        tot[k] = po.x + po.y;
-                    }
-                    ++g;
+            for (uint32_t a = 0; a < nA; ++a) {          // push queue[head .. head + nA)
+                const uint2 po = __ldg(&q[head + a]);
+                const unsigned long long x = ((unsigned long long)(cnt + po.y) << 32) | (po.x + po.y);
+                uint32_t i = B + a;
+                while (i > 0) {
+                    const uint32_t par = (i - 1) >> 1;
+                    const unsigned long long y = HEAP(par);
+                    if (y <= x) break;
+                    HEAP(i) = y;
+                    i = par;
                 }
+                HEAP(i) = x;
             }
             dur = Cp; r1 = 0x80000000u | nA; r2 = sumP; r3 = (uint32_t)head;
             busy += (long long)dur * nA;
             S += sumP; B += nA; reserved += sumTot; head += (int)nA;
             Cd = 0; ++n_pre;
             nA = 0; sumP = 0; sumTot = 0;                 // nothing more fits until someone retires
-            uint32_t m = fin[0];
-#pragma unroll
-            for (int k = 1; k < SPL; ++k) m = min(m, fin[k]);
-            next_fin = __reduce_min_sync(FULL, m);
+            next_fin = (uint32_t)(HEAP(0) >> 32);
         } else {
-            dur = ad + bd * B + S / qd;
+            dur = ad + bd * B + (q_shift >= 0 ? (S >> q_shift) : (S / qd));
             r1 = B; r2 = S; r3 = 0;
             busy += (long long)dur * B;
             ++cnt;
+            S += B;
             if (cnt == next_fin) {
-                uint32_t rel = 0, nf = 0;
-#pragma unroll
-                for (int k = 0; k < SPL; ++k)
-                    if (fin[k] == cnt) { rel += tot[k]; ++nf; fin[k] = EMPTY; }
-                // rel < 2^31 in total (reserved <= kv_budget), nf <= cap: pack both in one reduction
-                const unsigned long long both =
-                    warp_sum_u64(((unsigned long long)nf << 32) | rel);
-                rel = (uint32_t)both; nf = (uint32_t)(both >> 32);
-                S = S + B - rel;
-                B -= nf; reserved -= rel; r3 = nf;
-                uint32_t m = fin[0];
-#pragma unroll
-                for (int k = 1; k < SPL; ++k) m = min(m, fin[k]);
-                next_fin = __reduce_min_sync(FULL, m);
-                dirty = head < qn;
-            } else {
-                S += B;
+                uint32_t n = B;
+                do {                                      // pop every request that retires now
+                    S -= (uint32_t)HEAP(0);
+                    reserved -= (uint32_t)HEAP(0);
+                    ++r3;
+                    --n;
+                    const unsigned long long x = HEAP(n);
+                    uint32_t i = 0;
+                    while (true) {
+                        uint32_t ch = 2 * i + 1;
+                        if (ch >= n) break;
+                        unsigned long long y = HEAP(ch);
+                        if (ch + 1 < n) {
+                            const unsigned long long y2 = HEAP(ch + 1);
+                            if (y2 < y) { y = y2; ++ch; }
+                        }
+                        if (x <= y) break;
+                        HEAP(i) = y;
+                        i = ch;
+                    }
+                    if (n > 0) HEAP(i) = x;
+                } while (n > 0 && (uint32_t)(HEAP(0) >> 32) == cnt);
+                B = n;
+                next_fin = n > 0 ? (uint32_t)(HEAP(0) >> 32) : EMPTY;
+                grow = head + (int)nA < qn;
             }
             const unsigned long long w = (unsigned long long)Cd + dur;
             Cd = w > 0x7FFFFFFFull ? 0x7FFFFFFFu : (uint32_t)w;
@@ -245,28 +220,15 @@ k_simulate(const uint2* __restrict__ q_po, const int32_t* __restrict__ q_off,
         hash += (HASH_W0 * dur + HASH_W1 * r1 + HASH_W2 * r2 + HASH_W3 * r3 + HASH_W4) * pw;
         pw *= HASH_BASE;
         if (tr) {
-            if (lane == (int)(iters & 31u)) held = make_uint4(dur, r1, r2, r3);
-            if ((iters & 31u) == 31u) {
-                const long long idx = (long long)(iters & ~31u) + lane;
-                if (idx < tr_cap) reinterpret_cast<uint4*>(tr)[idx] = held;
-                else status |= HOS_ST_TRACE;
-            }
+            if ((long long)iters < tr_cap) tr[iters] = make_uint4(dur, r1, r2, r3);
+            else status |= HOS_ST_TRACE;
         }
         ++iters;
         if (t >= (1ll << 39)) { status |= HOS_ST_LIMIT; break; }
     }
-    if (tr && (iters & 31u) != 0u) {                      // records of the last, partial row
-        const long long idx = (long long)(iters & ~31u) + lane;
-        if (lane < (int)(iters & 31u)) {
-            if (idx < tr_cap) reinterpret_cast<uint4*>(tr)[idx] = held;
-            else status |= HOS_ST_TRACE;
-        }
-    }
-    status = __reduce_or_sync(FULL, status);
-    if (lane == 0) {
-        cres[unit] = hos_client_result{t, busy, n_pre, n_dec, hash, 0.0};
-        status_out[unit] = status;
-    }
+    cres[unit] = hos_client_result{t, busy, n_pre, n_dec, hash, 0.0};
+    status_out[unit] = status;
+#undef HEAP
 }
 
 // ---------------------------------------------------------------------------------------
@@ -371,18 +333,18 @@ cudaError_t launch_simulate(const hos_batch& b, const hos_cost_model& cm, const 
                             hos_iter_rec* trace, const long long* trace_off, int32_t* status,
                             cudaStream_t st) {
     const long long n_units = (long long)b.n_inst * n_lambda * b.n_clients;
-    const unsigned grid = (unsigned)((n_units + SIM_WARPS - 1) / SIM_WARPS);
-#define HOS_SIM(SPL)                                                                               \
-    k_simulate<SPL><<<grid, SIM_WARPS * 32, 0, st>>>(q_po, q_off, inst_status, lambda_q16, n_lambda, \
-                                                     b.n_clients, n_pad, n_units, b.batch_cap,     \
-                                                     (uint32_t)b.kv_budget, cm, max_iters, cres,   \
-                                                     trace, trace_off, status)
+    const unsigned grid = (unsigned)((n_units + SIM_THREADS - 1) / SIM_THREADS);
+    const size_t smem = (size_t)b.batch_cap * SIM_THREADS * sizeof(unsigned long long);
+    int q_shift = -1;                                    // power-of-two KV divisor -> shift
+    if ((cm.decode_kv_div & (cm.decode_kv_div - 1)) == 0)
+        for (q_shift = 0; (1u << q_shift) != cm.decode_kv_div; ++q_shift) {}
+    cudaError_t e = cudaFuncSetAttribute(k_simulate, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
     launch_hook("k_simulate", 0, st);
-    if (b.batch_cap <= 32) HOS_SIM(1);
-    else if (b.batch_cap <= 64) HOS_SIM(2);
-    else if (b.batch_cap <= 128) HOS_SIM(4);
-    else HOS_SIM(8);
-#undef HOS_SIM
+    k_simulate<<<grid, SIM_THREADS, smem, st>>>(q_po, q_off, inst_status, lambda_q16, n_lambda,
+                                               b.n_clients, n_pad, n_units, b.batch_cap,
+                                               (uint32_t)b.kv_budget, cm, q_shift, max_iters, cres,
+                                               trace, trace_off, status);
     launch_hook("k_simulate", 1, st);
     return cudaGetLastError();
 }
