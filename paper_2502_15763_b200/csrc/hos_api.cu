@@ -118,7 +118,7 @@ int hos_offline_pack(const hos_batch* b, const hos_cost_model* cm, int ls_rounds
     if (rc) return rc;
     if ((rc = check_cost(cm, b))) return rc;
     if (!assign || !load || !makespan_est || !rounds_applied || !status || ls_rounds < 0) return HOS_E_INVALID;
-    if (estimate_sort_smem(b->n_req) > SMEM_LIMIT || local_search_smem(b->n_req) > SMEM_LIMIT)
+    if (estimate_sort_smem(b->n_req) > SMEM_LIMIT || local_search_smem(b->n_req, b->n_clients) > SMEM_LIMIT)
         return HOS_E_UNSUPPORTED;
     if ((rc = check_ws(ws, ws_bytes, hos_offline_workspace_bytes(b, 1, ls_rounds)))) return rc;
     const OfflineWs w = carve_offline(b, ws);
@@ -146,7 +146,7 @@ int hos_local_search(const hos_batch* b, const hos_cost_model* cm, int n_copies,
     if (!assign || !load || !makespan_est || !rounds_applied || !status || ls_rounds < 0 || n_copies < 1)
         return HOS_E_INVALID;
     if ((long long)b->n_inst * n_copies > 0x7FFFFFFFll) return HOS_E_UNSUPPORTED;
-    if (estimate_sort_smem(b->n_req) > SMEM_LIMIT || local_search_smem(b->n_req) > SMEM_LIMIT)
+    if (estimate_sort_smem(b->n_req) > SMEM_LIMIT || local_search_smem(b->n_req, b->n_clients) > SMEM_LIMIT)
         return HOS_E_UNSUPPORTED;
     if ((rc = check_ws(ws, ws_bytes, hos_offline_workspace_bytes(b, n_copies, ls_rounds)))) return rc;
     const OfflineWs w = carve_offline(b, ws);

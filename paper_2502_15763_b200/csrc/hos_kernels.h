@@ -14,7 +14,7 @@ struct InstInfo;
 void launch_hook(const char* kernel, int phase, cudaStream_t st);
 
 size_t estimate_sort_smem(int n_req);
-size_t local_search_smem(int n_req);
+size_t local_search_smem(int n_req, int n_clients);
 size_t queue_build_smem(int n_req);
 
 cudaError_t launch_estimate_sort(const hos_batch& b, const hos_cost_model& cm, uint32_t* T_sorted,

@@ -186,42 +186,145 @@ k_lpt(const uint32_t* __restrict__ T_sorted, const uint32_t* __restrict__ order,
 
 // ---------------------------------------------------------------------------------------
 // Local search.  One CTA per (instance, copy); the instance stays in shared memory for all
-// rounds: T by rank, client by rank, request index by rank, the critical client's members.
+// rounds: T by rank, request index by rank, client by rank, and the clients' member lists
+// (CSR: for every client its ranks in ascending order, i.e. T descending, index ascending
+// inside equal T).
 //
 // A round looks for the minimum of (v, i, k, u) over every move (u = -1, d = T_i) and swap
 // (d = T_i - T_u > 0) off the critical client jmax, v = max(Lmax - d, load_k + d).  For a
 // fixed (k, u), v falls while 2 d < Lmax - load_k and rises afterwards, so only two members
 // of jmax can win: the one with the largest T below the turning point and the one with the
-// smallest T at or above it (first index of its run of equal T).  Each thread owns the
-// requests u of some ranks, finds those two members by binary search in the member list
-// (sorted by T) and keeps its best tuple; a CTA-wide lexicographic min picks the step.
+// smallest T at or above it (first index of its run of equal T); both come from one binary
+// search in jmax's member list.  Any step onto client k ends with
+// v >= ceil((Lmax + load_k) / 2): the least loaded client is evaluated first, its best v
+// bounds the optimum, and only clients whose floor does not exceed that bound are looked at
+// (ties in v survive the filter).  Work items are taken from the member lists, so every lane
+// of the evaluating warps has an item.  A swap keeps both list lengths: the two lists are
+// patched in place; a move rebuilds the lists.
 // ---------------------------------------------------------------------------------------
+// A candidate step, ordered by (v, i, k, u) through three words that compare the same way:
+// inv = ~(Lmax - v) (every useful candidate has 0 < Lmax - v <= T_i < 2^32), ik = i << 8 | k,
+// u1 = u + 1 (0 for a move).  n_req < 2^15 and n_clients <= 2^8 keep ik inside 23 bits.
 struct Cand {
-    long long v;
-    int i, k, u;       // request indices / client
-    int ri, ru;        // ranks of i and u (ru = -1 for a move)
+    uint32_t inv, ik, u1;
+    int pi, pu;        // positions of i in jmax's list and of u in k's list (pu = -1 for a move)
 };
+constexpr uint32_t NO_CAND = 0xFFFFFFFFu;
 
 __device__ __forceinline__ bool cand_less(const Cand& a, const Cand& b) {
-    if (a.v != b.v) return a.v < b.v;
-    if (a.i != b.i) return a.i < b.i;
-    if (a.k != b.k) return a.k < b.k;
-    return a.u < b.u;
+    if (a.inv != b.inv) return a.inv < b.inv;
+    if (a.ik != b.ik) return a.ik < b.ik;
+    return a.u1 < b.u1;
 }
 
-__device__ __forceinline__ Cand cand_shfl_xor(const Cand& c, int d) {
+// Warp-wide minimum by three integer reductions; every lane gets the winner.
+__device__ __forceinline__ Cand cand_warp_min(const Cand& c) {
+    const uint32_t m0 = __reduce_min_sync(FULL, c.inv);
+    const uint32_t m1 = __reduce_min_sync(FULL, c.inv == m0 ? c.ik : 0xFFFFFFFFu);
+    const uint32_t m2 = __reduce_min_sync(FULL, (c.inv == m0 && c.ik == m1) ? c.u1 : 0xFFFFFFFFu);
+    const unsigned who = __ballot_sync(FULL, c.inv == m0 && c.ik == m1 && c.u1 == m2);
+    const int src = __ffs(who) - 1;
     Cand r;
-    r.v = __shfl_xor_sync(FULL, c.v, d);
-    r.i = __shfl_xor_sync(FULL, c.i, d);
-    r.k = __shfl_xor_sync(FULL, c.k, d);
-    r.u = __shfl_xor_sync(FULL, c.u, d);
-    r.ri = __shfl_xor_sync(FULL, c.ri, d);
-    r.ru = __shfl_xor_sync(FULL, c.ru, d);
+    r.inv = m0; r.ik = m1; r.u1 = m2;
+    r.pi = __shfl_sync(FULL, c.pi, src);
+    r.pu = __shfl_sync(FULL, c.pu, src);
     return r;
 }
 
 constexpr long long NO_V = 0x7FFFFFFFFFFFFFFFll;
 constexpr int NO_I = 0x7FFFFFFF;
+
+// Exclusive scan of a[0 .. len) in place by the whole CTA; `wsum` holds 32 words.
+__device__ inline void block_scan_u32(uint32_t* a, int len, uint32_t* wsum) {
+    const int per = (len + SORT_THREADS - 1) / SORT_THREADS;
+    const int lo = min(len, (int)threadIdx.x * per), hi = min(len, lo + per);
+    uint32_t run = 0;
+    for (int x = lo; x < hi; ++x) run += a[x];
+    uint32_t inc = run;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+        const uint32_t y = __shfl_up_sync(FULL, inc, d);
+        if (lane_id() >= d) inc += y;
+    }
+    if (lane_id() == 31) wsum[warp_id()] = inc;
+    __syncthreads();
+    if (warp_id() == 0) {
+        const uint32_t w = wsum[lane_id()];
+        uint32_t winc = w;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const uint32_t y = __shfl_up_sync(FULL, winc, d);
+            if (lane_id() >= d) winc += y;
+        }
+        wsum[lane_id()] = winc - w;
+    }
+    __syncthreads();
+    uint32_t acc = wsum[warp_id()] + inc - run;
+    for (int x = lo; x < hi; ++x) { const uint32_t c = a[x]; a[x] = acc; acc += c; }
+    __syncthreads();
+}
+
+// Member lists of all clients from bins[]: a stable split of the ranks 0..n-1 by client.
+// cnt holds n_clients * SORT_WARPS words.  off[k] = start of client k's list, off[M] = n.
+template <typename IdxT>
+__device__ inline void build_member_lists(const uint8_t* bins, IdxT* cl, int n, int n_clients,
+                                          uint32_t* cnt, uint32_t* wsum, int* off) {
+    const int lane = lane_id(), warp = warp_id();
+    const int chunk = (((n + SORT_WARPS - 1) / SORT_WARPS) + 31) & ~31;
+    const int lo = warp * chunk, hi = min(n, lo + chunk);
+    for (int x = threadIdx.x; x < n_clients * SORT_WARPS; x += SORT_THREADS) cnt[x] = 0;
+    __syncthreads();
+    for (int row = lo; row < hi; row += 32) {
+        const int r = row + lane;
+        const bool valid = r < hi;
+        const uint32_t dig = valid ? (uint32_t)bins[r] : 0xFFFFu;
+        const unsigned m = __match_any_sync(FULL, dig);
+        if (valid && lane == (__ffs(m) - 1)) cnt[dig * SORT_WARPS + warp] += __popc(m);
+        __syncwarp();
+    }
+    __syncthreads();
+    block_scan_u32(cnt, n_clients * SORT_WARPS, wsum);
+    for (int k = threadIdx.x; k <= n_clients; k += SORT_THREADS)
+        off[k] = k < n_clients ? (int)cnt[k * SORT_WARPS] : n;
+    __syncthreads();
+    for (int row = lo; row < hi; row += 32) {
+        const int r = row + lane;
+        const bool valid = r < hi;
+        const uint32_t dig = valid ? (uint32_t)bins[r] : 0xFFFFu;
+        const unsigned m = __match_any_sync(FULL, dig);
+        const uint32_t base = valid ? cnt[dig * SORT_WARPS + warp] : 0u;
+        __syncwarp();
+        if (valid) {
+            cl[base + __popc(m & ((1u << lane) - 1u))] = (IdxT)r;
+            if (lane == (__ffs(m) - 1)) cnt[dig * SORT_WARPS + warp] = base + __popc(m);
+        }
+        __syncwarp();
+    }
+    __syncthreads();
+}
+
+// In the ascending list seg[0 .. len): drop the element at position `gone`, insert `val`.
+// Called by `nthr` threads (tid 0 .. nthr-1) of the CTA; the caller places a __syncthreads()
+// between the returned read phase and `patch_write`.
+template <typename IdxT>
+struct ListPatch {
+    int dst_lo, dst_hi, shift, at;     // elements at [dst_lo, dst_hi) move by `shift`; val lands at `at`
+};
+template <typename IdxT>
+__device__ inline ListPatch<IdxT> patch_plan(const IdxT* seg, int len, int gone, int val) {
+    int a = 0, z = len;                                  // lower bound of val
+    while (a < z) {
+        const int mid = (a + z) >> 1;
+        if ((int)seg[mid] < val) a = mid + 1; else z = mid;
+    }
+    const int at = a - ((int)seg[gone] < val ? 1 : 0);   // position among the remaining elements
+    ListPatch<IdxT> p;
+    p.at = at;
+    if (at > gone) { p.dst_lo = gone + 1; p.dst_hi = at + 1; p.shift = -1; }
+    else if (at < gone) { p.dst_lo = at; p.dst_hi = gone; p.shift = +1; }
+    else { p.dst_lo = 0; p.dst_hi = 0; p.shift = 0; }
+    return p;
+}
 
 template <typename IdxT>
 __global__ void __launch_bounds__(SORT_THREADS, 1)
@@ -233,10 +336,13 @@ k_local_search(const uint32_t* __restrict__ T_sorted, const uint32_t* __restrict
                hos_ls_move* __restrict__ ls_log, int32_t* __restrict__ status_out) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     __shared__ long long s_load[MAX_CLIENTS];
+    __shared__ int s_off[MAX_CLIENTS + 1];
     __shared__ Cand s_cand[32];
-    __shared__ int s_wcnt[32];
-    __shared__ int s_jmax, s_nm, s_kmin;
-    __shared__ long long s_vb[32];
+    __shared__ uint32_t s_inv[32];
+    __shared__ uint32_t s_wsum[32];
+    __shared__ int s_as[MAX_CLIENTS];
+    __shared__ uint8_t s_ak[MAX_CLIENTS];
+    __shared__ int s_jmax, s_kmin, s_na, s_nitems;
     __shared__ long long s_lmax;
 
     const int inst = blockIdx.x / n_copies;
@@ -261,8 +367,9 @@ k_local_search(const uint32_t* __restrict__ T_sorted, const uint32_t* __restrict
     unsigned char* base = smem_raw;
     uint32_t* Ts = reinterpret_cast<uint32_t*>(base);   base += align16((size_t)n_req * 4);
     IdxT* ord = reinterpret_cast<IdxT*>(base);          base += align16((size_t)n_req * sizeof(IdxT));
-    IdxT* mem = reinterpret_cast<IdxT*>(base);          base += align16((size_t)n_req * sizeof(IdxT));
-    uint8_t* bins = reinterpret_cast<uint8_t*>(base);
+    IdxT* cl = reinterpret_cast<IdxT*>(base);           base += align16((size_t)n_req * sizeof(IdxT));
+    uint8_t* bins = reinterpret_cast<uint8_t*>(base);   base += align16((size_t)n_req);
+    uint32_t* cnt = reinterpret_cast<uint32_t*>(base);
 
     const uint32_t* gT = T_sorted + (size_t)inst * n_pad;
     const uint32_t* gO = order + (size_t)inst * n_pad;
@@ -291,14 +398,16 @@ k_local_search(const uint32_t* __restrict__ T_sorted, const uint32_t* __restrict
             for (int r = threadIdx.x; r < rounds; r += SORT_THREADS) log[r] = hos_ls_move{-1, -1, -1, 0};
         return;
     }
+    build_member_lists<IdxT>(bins, cl, n_req, n_clients, cnt, s_wsum, s_off);
 
-    const int chunk = (((n_req + SORT_WARPS - 1) / SORT_WARPS) + 31) & ~31;
-    const int lo = warp * chunk, hi = min(n_req, lo + chunk);
     int applied = 0;
     int done_at = rounds;
 
     for (int round = 0; round < rounds; ++round) {
-        // (a) critical client: largest load, ties to the lowest client
+        // (a) critical client: largest load, ties to the lowest client (warp 0); the least loaded
+        //     other client, any of them on ties, seeds the pruning bound (warp 1, once jmax is known
+        //     it only has to skip it, and the least loaded client is never the critical one unless
+        //     all loads are equal, in which case no step can improve)
         if (warp == 0) {
             long long bl = -1;
             int bj = NO_I;
@@ -311,159 +420,187 @@ k_local_search(const uint32_t* __restrict__ T_sorted, const uint32_t* __restrict
                 if (ol > bl || (ol == bl && oj < bj)) { bl = ol; bj = oj; }
             }
             if (lane == 0) { s_jmax = bj; s_lmax = bl; }
-            // least loaded other client (any of them on ties: it only seeds the pruning bound)
-            const int jm = __shfl_sync(FULL, bj, 0);
+        } else if (warp == 1) {
             long long ml = NO_V;
             int mj = -1;
             for (int j = lane; j < n_clients; j += 32)
-                if (j != jm && s_load[j] < ml) { ml = s_load[j]; mj = j; }
+                if (s_load[j] < ml) { ml = s_load[j]; mj = j; }
 #pragma unroll
             for (int d = 16; d > 0; d >>= 1) {
                 const long long ol = __shfl_xor_sync(FULL, ml, d);
                 const int oj = __shfl_xor_sync(FULL, mj, d);
-                if (ol < ml) { ml = ol; mj = oj; }
+                if (ol < ml || (ol == ml && oj > mj)) { ml = ol; mj = oj; }   // highest client on ties
             }
             if (lane == 0) s_kmin = mj;
         }
         __syncthreads();
         const int jmax = s_jmax;
         const long long Lmax = s_lmax;
+        // all loads equal: kmin may coincide with jmax; then nothing can improve anyway
+        const int kmin = (s_kmin != jmax && s_load[s_kmin] < Lmax) ? s_kmin : -1;
+        const IdxT* mem = cl + s_off[jmax];                 // jmax's members, T descending
+        const int nm = s_off[jmax + 1] - s_off[jmax];
 
-        // (b) members of jmax, in rank order (T descending, index ascending inside equal T)
-        int cnt = 0;
-        for (int row = lo; row < hi; row += 32) {
-            const int r = row + lane;
-            cnt += __popc(__ballot_sync(FULL, r < hi && bins[r] == jmax));
-        }
-        if (lane == 0) s_wcnt[warp] = cnt;
-        __syncthreads();
-        if (warp == 0) {
-            const int c = s_wcnt[lane];
-            int inc = c;
-#pragma unroll
-            for (int d = 1; d < 32; d <<= 1) {
-                const int y = __shfl_up_sync(FULL, inc, d);
-                if (lane >= d) inc += y;
-            }
-            s_wcnt[lane] = inc - c;
-            if (lane == 31) s_nm = inc;
-        }
-        __syncthreads();
-        int off = s_wcnt[warp];
-        for (int row = lo; row < hi; row += 32) {
-            const int r = row + lane;
-            const bool is = r < hi && bins[r] == jmax;
-            const unsigned b = __ballot_sync(FULL, is);
-            if (is) mem[off + __popc(b & ((1u << lane) - 1u))] = (IdxT)r;
-            off += __popc(b);
-        }
-        __syncthreads();
-        const int nm = s_nm;
-
-        // (c) candidates: work item w < n_req is "swap with the request of rank w";
-        //     w >= n_req is "move to client w - n_req".
-        //     Any step onto client k ends with v >= ceil((Lmax + load_k) / 2).  A first sweep over
-        //     the least loaded client alone gives an achievable v (`vbound`); the full sweep then
-        //     skips every client whose floor is above it.  Ties in v survive the filter.
-        auto evaluate = [&](int w, Cand& best, long long vbound) {
-            int k, u, ru;
-            long long Tu;
-            if (w < n_req) { k = bins[w]; u = -2; ru = w; Tu = Ts[w]; }
-            else { k = w - n_req; u = -1; ru = -1; Tu = 0; }
-            if (k == jmax) return;
+        // (b) one work item: client k, position idx in its list (idx == its length: the move)
+        auto evaluate = [&](int k, int idx, int len, Cand& best) {
             const long long lk = s_load[k];
             const long long slack = Lmax - lk;
-            if (slack <= 0 || ((Lmax + lk + 1) >> 1) > vbound) return;
-            if (u == -2) u = (int)ord[w];
+            uint32_t u1 = 0;
+            int pu = -1;
+            long long Tu = 0;
+            if (idx < len) {
+                const int w = (int)cl[s_off[k] + idx];
+                u1 = (uint32_t)ord[w] + 1u; pu = idx; Tu = Ts[w];
+            }
             const long long thr = Tu + ((slack + 1) >> 1);      // T_i >= thr  <=>  2 d >= slack
-            // b = number of members with T >= thr (members are sorted by T descending)
-            int a = 0, z = nm;
+            int a = 0, z = nm;                                  // b = members with T >= thr
             while (a < z) {
                 const int mid = (a + z) >> 1;
                 if ((long long)Ts[mem[mid]] >= thr) a = mid + 1; else z = mid;
             }
             const int b = a;
             if (b > 0) {                                        // rising side: smallest T >= thr
-                const long long Ti = Ts[mem[b - 1]];
-                const long long d = Ti - Tu;
+                const uint32_t Ti = Ts[mem[b - 1]];
+                const long long d = (long long)Ti - Tu;
                 if (d < slack) {
-                    // first member of the run of equal T (smallest request index)
-                    int a2 = 0, z2 = b - 1;
-                    while (a2 < z2) {
-                        const int mid = (a2 + z2) >> 1;
-                        if ((long long)Ts[mem[mid]] > Ti) a2 = mid + 1; else z2 = mid;
+                    int a2 = b - 1;                             // first member of the run of equal T
+                    if (b >= 2 && Ts[mem[b - 2]] == Ti) {
+                        int z2 = b - 2;
+                        a2 = 0;
+                        while (a2 < z2) {
+                            const int mid = (a2 + z2) >> 1;
+                            if (Ts[mem[mid]] > Ti) a2 = mid + 1; else z2 = mid;
+                        }
                     }
-                    Cand c;
-                    c.v = lk + d; c.ri = (int)mem[a2]; c.i = (int)ord[c.ri]; c.k = k; c.u = u; c.ru = ru;
+                    Cand c;                                     // v = lk + d, Lmax - v = slack - d
+                    c.inv = ~(uint32_t)(slack - d); c.pi = a2; c.ik = ((uint32_t)ord[mem[a2]] << 8) | (uint32_t)k;
+                    c.u1 = u1; c.pu = pu;
                     if (cand_less(c, best)) best = c;
                 }
             }
             if (b < nm) {                                       // falling side: largest T < thr
-                const long long Ti = Ts[mem[b]];
-                const long long d = Ti - Tu;
+                const long long d = (long long)Ts[mem[b]] - Tu;
                 if (d > 0) {
-                    Cand c;
-                    c.v = Lmax - d; c.ri = (int)mem[b]; c.i = (int)ord[c.ri]; c.k = k; c.u = u; c.ru = ru;
+                    Cand c;                                     // v = Lmax - d
+                    c.inv = ~(uint32_t)d; c.pi = b; c.ik = ((uint32_t)ord[mem[b]] << 8) | (uint32_t)k;
+                    c.u1 = u1; c.pu = pu;
                     if (cand_less(c, best)) best = c;
                 }
             }
         };
         Cand best;
-        best.v = NO_V; best.i = NO_I; best.k = NO_I; best.u = NO_I; best.ri = -1; best.ru = -1;
-        const int kmin = s_kmin;
+        best.inv = NO_CAND; best.ik = NO_CAND; best.u1 = NO_CAND; best.pi = -1; best.pu = -1;
+        // (c) the least loaded client first: its best step is achievable, hence bounds the optimum
         if (kmin >= 0) {
-            for (int w = threadIdx.x; w < n_req + n_clients; w += SORT_THREADS) {
-                const int k = (w < n_req) ? (int)bins[w] : w - n_req;
-                if (k == kmin) evaluate(w, best, NO_V);
+            const int len = s_off[kmin + 1] - s_off[kmin];
+            for (int idx = threadIdx.x; idx <= len; idx += SORT_THREADS) evaluate(kmin, idx, len, best);
+        }
+        {
+            const uint32_t wi = __reduce_min_sync(FULL, best.inv);
+            if (lane == 0) s_inv[warp] = wi;
+        }
+        __syncthreads();
+        // (d) warp 0 lists the other clients whose floor ceil((Lmax + load_k) / 2) does not exceed
+        //     the bound, with the running count of their work items (list length + 1 move)
+        if (warp == 0) {
+            const uint32_t inv = __reduce_min_sync(FULL, s_inv[lane]);
+            const long long vbound = Lmax - (long long)(~inv);          // no candidate: gain 0 -> Lmax
+            int n_alive = 0, n_items = 0;
+            for (int k0 = 0; k0 < n_clients; k0 += 32) {
+                const int k = k0 + lane;
+                bool alive = false;
+                int sz = 0;
+                if (k < n_clients && k != jmax && k != kmin) {
+                    const long long lk = s_load[k];
+                    alive = lk < Lmax && ((Lmax + lk + 1) >> 1) <= vbound;
+                    sz = alive ? s_off[k + 1] - s_off[k] + 1 : 0;
+                }
+                const unsigned am = __ballot_sync(FULL, alive);
+                int inc = sz;
+#pragma unroll
+                for (int d = 1; d < 32; d <<= 1) {
+                    const int y = __shfl_up_sync(FULL, inc, d);
+                    if (lane >= d) inc += y;
+                }
+                if (alive) {
+                    const int pos = n_alive + __popc(am & ((1u << lane) - 1u));
+                    s_ak[pos] = (uint8_t)k;
+                    s_as[pos] = n_items + inc - sz;
+                }
+                n_alive += __popc(am);
+                n_items += __shfl_sync(FULL, inc, 31);
+            }
+            if (lane == 0) { s_na = n_alive; s_nitems = n_items; }
+        }
+        __syncthreads();
+        {
+            const int n_alive = s_na, n_items = s_nitems;
+            for (int x = threadIdx.x; x < n_items; x += SORT_THREADS) {
+                int a = 0, z = n_alive;                         // last listed client with start <= x
+                while (z - a > 1) {
+                    const int mid = (a + z) >> 1;
+                    if (s_as[mid] <= x) a = mid; else z = mid;
+                }
+                const int k = s_ak[a];
+                evaluate(k, x - s_as[a], s_off[k + 1] - s_off[k], best);
             }
         }
-        long long vb = best.v;
-#pragma unroll
-        for (int d = 16; d > 0; d >>= 1) vb = min(vb, __shfl_xor_sync(FULL, vb, d));
-        if (lane == 0) s_vb[warp] = vb;
-        __syncthreads();
-        vb = s_vb[lane];
-#pragma unroll
-        for (int d = 16; d > 0; d >>= 1) vb = min(vb, __shfl_xor_sync(FULL, vb, d));
-        const long long vbound = vb;
-        best.v = NO_V; best.i = NO_I; best.k = NO_I; best.u = NO_I; best.ri = -1; best.ru = -1;
-        for (int w = threadIdx.x; w < n_req + n_clients; w += SORT_THREADS) evaluate(w, best, vbound);
-        // (d) CTA-wide lexicographic minimum
-#pragma unroll
-        for (int d = 16; d > 0; d >>= 1) {
-            const Cand oc = cand_shfl_xor(best, d);
-            if (cand_less(oc, best)) best = oc;
-        }
+        // (e) CTA-wide lexicographic minimum: per warp, then every warp reduces the 32 records
+        best = cand_warp_min(best);
         if (lane == 0) s_cand[warp] = best;
         __syncthreads();
-        if (warp == 0) {
-            best = s_cand[lane];
-#pragma unroll
-            for (int d = 16; d > 0; d >>= 1) {
-                const Cand oc = cand_shfl_xor(best, d);
-                if (cand_less(oc, best)) best = oc;
-            }
-            if (lane == 0) s_cand[0] = best;
+        best = cand_warp_min(s_cand[lane]);
+        const bool ok = best.inv != NO_CAND;                    // a candidate always has v < Lmax
+        if (!ok) {
+            if (threadIdx.x == 0 && log) log[round] = hos_ls_move{-1, -1, -1, Lmax};
+            done_at = round;
+            break;
         }
-        __syncthreads();
-        best = s_cand[0];
-        const bool ok = best.v < Lmax;                          // NO_V when there was no candidate
-        // (e) apply
+        const int best_k = (int)(best.ik & 0xFFu);
+        const int best_i = (int)(best.ik >> 8);
+        const int best_u = (int)best.u1 - 1;
+        const long long best_v = Lmax - (long long)(~best.inv);
+        // (f) apply
+        const int ri = (int)mem[best.pi];
+        const int ru = best.pu >= 0 ? (int)cl[s_off[best_k] + best.pu] : -1;
+        if (best.pu >= 0) {
+            // swap: jmax's list loses ri and gains ru, k's list loses ru and gains ri
+            const bool first = threadIdx.x < SORT_THREADS / 2;
+            IdxT* seg = cl + s_off[first ? jmax : best_k];
+            const int len = first ? nm : s_off[best_k + 1] - s_off[best_k];
+            const int gone = first ? best.pi : best.pu;
+            const int val = first ? ru : ri;
+            const ListPatch<IdxT> pp = patch_plan<IdxT>(seg, len, gone, val);
+            const int tid = threadIdx.x & (SORT_THREADS / 2 - 1);
+            // every thread moves at most ceil(range / 512) elements: read, barrier, write
+            IdxT keep[4];
+            int nk = 0;
+            const int span = pp.dst_hi - pp.dst_lo;
+            const bool big = span > 4 * (SORT_THREADS / 2);     // generic path for very long ranges
+            if (!big)
+                for (int x = pp.dst_lo + tid; x < pp.dst_hi; x += SORT_THREADS / 2) keep[nk++] = seg[x];
+            __syncthreads();
+            if (!big) {
+                nk = 0;
+                for (int x = pp.dst_lo + tid; x < pp.dst_hi; x += SORT_THREADS / 2) seg[x + pp.shift] = keep[nk++];
+            } else if (tid == 0) {                              // serial shift, direction-safe
+                if (pp.shift < 0) for (int x = pp.dst_lo; x < pp.dst_hi; ++x) seg[x - 1] = seg[x];
+                else for (int x = pp.dst_hi - 1; x >= pp.dst_lo; --x) seg[x + 1] = seg[x];
+            }
+            __syncthreads();
+            if (tid == 0) seg[pp.at] = (IdxT)val;
+        }
         if (threadIdx.x == 0) {
-            if (ok) {
-                const long long d = (long long)Ts[best.ri] - (best.ru >= 0 ? (long long)Ts[best.ru] : 0ll);
-                bins[best.ri] = (uint8_t)best.k;
-                asg[best.i] = best.k;
-                if (best.ru >= 0) { bins[best.ru] = (uint8_t)jmax; asg[best.u] = jmax; }
-                s_load[jmax] -= d;
-                s_load[best.k] += d;
-                if (log) log[round] = hos_ls_move{best.i, best.u, best.k, best.v};
-            } else if (log) {
-                log[round] = hos_ls_move{-1, -1, -1, Lmax};
-            }
+            const long long d = (long long)Ts[ri] - (ru >= 0 ? (long long)Ts[ru] : 0ll);
+            bins[ri] = (uint8_t)best_k;
+            asg[best_i] = best_k;
+            if (ru >= 0) { bins[ru] = (uint8_t)jmax; asg[best_u] = jmax; }
+            s_load[jmax] -= d;
+            s_load[best_k] += d;
+            if (log) log[round] = hos_ls_move{best_i, best_u, best_k, best_v};
         }
         __syncthreads();
-        if (!ok) { done_at = round; break; }
+        if (best.pu < 0) build_member_lists<IdxT>(bins, cl, n_req, n_clients, cnt, s_wsum, s_off);
         ++applied;
     }
     // a round without an improving step leaves the state as it is: all later rounds are the same
@@ -471,9 +608,9 @@ k_local_search(const uint32_t* __restrict__ T_sorted, const uint32_t* __restrict
         const hos_ls_move noop = hos_ls_move{-1, -1, -1, s_lmax};
         for (int r = done_at + 1 + threadIdx.x; r < rounds; r += SORT_THREADS) log[r] = noop;
     }
-    long long mx = 0;
     for (int j = threadIdx.x; j < n_clients; j += SORT_THREADS) { ld[j] = s_load[j]; }
     if (warp == 0) {
+        long long mx = 0;
         for (int j = lane; j < n_clients; j += 32) mx = s_load[j] > mx ? s_load[j] : mx;
         mx = warp_max_i64(mx);
         if (lane == 0) { makespan_out[unit] = mx; rounds_applied[unit] = applied; }
@@ -548,14 +685,17 @@ k_lower_bound(const uint32_t* __restrict__ p, const uint32_t* __restrict__ o, in
 // ---------------------------------------------------------------------------------------
 // launchers
 // ---------------------------------------------------------------------------------------
-static size_t ls_smem_bytes(int n_req, size_t isz) {
-    return align16((size_t)n_req * 4) + 2 * align16((size_t)n_req * isz) + align16((size_t)n_req);
+static size_t ls_smem_bytes(int n_req, int n_clients, size_t isz) {
+    return align16((size_t)n_req * 4) + 2 * align16((size_t)n_req * isz) + align16((size_t)n_req) +
+           (size_t)n_clients * SORT_WARPS * 4;
 }
 
 size_t estimate_sort_smem(int n_req) {
     return n_req <= 65536 ? sort_smem_bytes<uint16_t>(n_req) : sort_smem_bytes<uint32_t>(n_req);
 }
-size_t local_search_smem(int n_req) { return ls_smem_bytes(n_req, n_req <= 65536 ? 2 : 4); }
+size_t local_search_smem(int n_req, int n_clients) {
+    return ls_smem_bytes(n_req, n_clients, n_req <= 65536 ? 2 : 4);
+}
 
 cudaError_t launch_estimate_sort(const hos_batch& b, const hos_cost_model& cm, uint32_t* T_sorted,
                                  uint32_t* order, InstInfo* info, int32_t* status_out, int n_pad,
@@ -594,7 +734,7 @@ cudaError_t launch_local_search(const hos_batch& b, const uint32_t* T_sorted, co
                                 bool load_from_assign, int32_t* assign, long long* load,
                                 long long* makespan, int32_t* rounds_applied, hos_ls_move* ls_log,
                                 int32_t* status, cudaStream_t st) {
-    const size_t smem = local_search_smem(b.n_req);
+    const size_t smem = local_search_smem(b.n_req, b.n_clients);
     auto kern = b.n_req <= 65536 ? k_local_search<uint16_t> : k_local_search<uint32_t>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;

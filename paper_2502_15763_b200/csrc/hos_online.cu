@@ -9,6 +9,8 @@
 
 namespace hos {
 
+constexpr int INST_WIDE = 0x100;         // internal flag in the workspace's per-instance status word
+
 // ---------------------------------------------------------------------------------------
 // Queue build: a segmented sort of the instance's requests by (client ascending,
 // N^p + N^d descending, index ascending) -- one stable radix sort on the composite key
@@ -46,7 +48,8 @@ k_queue_build(const uint32_t* __restrict__ p, const uint32_t* __restrict__ o,
     __syncthreads();
     if (threadIdx.x == 0) {
         inst_O[inst] = sumO;
-        inst_status[inst] = bad ? HOS_ST_INVALID : 0;
+        // bit 8 (internal): some p + o needs more than 16 bits -> the simulator's wide heap entries
+        inst_status[inst] = bad ? HOS_ST_INVALID : (mx >= 65536ull ? INST_WIDE : 0);
     }
     if (bad) return;
 
@@ -95,6 +98,26 @@ constexpr unsigned long long HASH_W3 = 0xA0761D6478BD642Full;
 constexpr unsigned long long HASH_W4 = 0xE7037ED1A0B428DBull;
 constexpr int SIM_THREADS = 32;          // one warp per CTA: a warp leaves as soon as its clients are done
 
+// Heap entries.  Narrow: (fin mod 2^16) << 16 | tot, usable when every p + o of the instance is
+// below 2^16 (then fin - cnt < 2^16 too, and entries compare correctly after subtracting
+// cnt << 16).  Wide: fin << 32 | tot.  Half the shared memory per client doubles the resident
+// warps, and the recurrence is latency-bound.
+struct NarrowEntry {
+    typedef uint32_t T;
+    static __device__ __forceinline__ T make(uint32_t fin, uint32_t tot) { return (fin << 16) | tot; }
+    static __device__ __forceinline__ T rel(T x, uint32_t cnt) { return x - (cnt << 16); }
+    static __device__ __forceinline__ uint32_t tot(T x) { return x & 0xFFFFu; }
+    static __device__ __forceinline__ uint32_t fin(T x, uint32_t cnt) { return cnt + (rel(x, cnt) >> 16); }
+};
+struct WideEntry {
+    typedef unsigned long long T;
+    static __device__ __forceinline__ T make(uint32_t fin, uint32_t tot) { return ((T)fin << 32) | tot; }
+    static __device__ __forceinline__ T rel(T x, uint32_t) { return x; }
+    static __device__ __forceinline__ uint32_t tot(T x) { return (uint32_t)x; }
+    static __device__ __forceinline__ uint32_t fin(T x, uint32_t) { return (uint32_t)(x >> 32); }
+};
+
+template <typename E>
 __global__ void __launch_bounds__(SIM_THREADS)
 k_simulate(const uint2* __restrict__ q_po, const int32_t* __restrict__ q_off,
            const int32_t* __restrict__ inst_status, const uint32_t* __restrict__ lambda_q16,
@@ -102,8 +125,9 @@ k_simulate(const uint2* __restrict__ q_po, const int32_t* __restrict__ q_off,
            hos_cost_model cm, int q_shift, uint32_t max_iters, hos_client_result* __restrict__ cres,
            hos_iter_rec* __restrict__ trace, const long long* __restrict__ trace_off,
            int32_t* __restrict__ status_out) {
+    typedef typename E::T entry_t;
     extern __shared__ __align__(16) unsigned char smem_raw[];
-    unsigned long long* heap = reinterpret_cast<unsigned long long*>(smem_raw) + threadIdx.x;
+    entry_t* heap = reinterpret_cast<entry_t*>(smem_raw) + threadIdx.x;
 #define HEAP(s) heap[(s) * SIM_THREADS]
     const long long unit = (long long)blockIdx.x * SIM_THREADS + threadIdx.x;
     if (unit >= n_units) return;
@@ -111,9 +135,11 @@ k_simulate(const uint2* __restrict__ q_po, const int32_t* __restrict__ q_off,
     const int l = (int)((unit / n_clients) % n_lambda);
     const int inst = (int)(unit / ((long long)n_clients * n_lambda));
 
-    if (inst_status[inst]) {
+    const int ist = inst_status[inst];
+    if (((ist & INST_WIDE) != 0) != (sizeof(entry_t) == 8)) return;   // the other instantiation's instance
+    if (ist & HOS_ST_INVALID) {
         cres[unit] = hos_client_result{0, 0, 0u, 0u, 0ull, 0.0};
-        status_out[unit] = inst_status[inst];
+        status_out[unit] = HOS_ST_INVALID;
         return;
     }
     const int q0 = q_off[(size_t)inst * (n_clients + 1) + c];
@@ -162,12 +188,13 @@ k_simulate(const uint2* __restrict__ q_po, const int32_t* __restrict__ q_off,
         if (prefill) {
             for (uint32_t a = 0; a < nA; ++a) {          // push queue[head .. head + nA)
                 const uint2 po = __ldg(&q[head + a]);
-                const unsigned long long x = ((unsigned long long)(cnt + po.y) << 32) | (po.x + po.y);
+                const entry_t x = E::make(cnt + po.y, po.x + po.y);
+                const entry_t xr = E::rel(x, cnt);
                 uint32_t i = B + a;
                 while (i > 0) {
                     const uint32_t par = (i - 1) >> 1;
-                    const unsigned long long y = HEAP(par);
-                    if (y <= x) break;
+                    const entry_t y = HEAP(par);
+                    if (E::rel(y, cnt) <= xr) break;
                     HEAP(i) = y;
                     i = par;
                 }
@@ -178,7 +205,7 @@ k_simulate(const uint2* __restrict__ q_po, const int32_t* __restrict__ q_off,
             S += sumP; B += nA; reserved += sumTot; head += (int)nA;
             Cd = 0; ++n_pre;
             nA = 0; sumP = 0; sumTot = 0;                 // nothing more fits until someone retires
-            next_fin = (uint32_t)(HEAP(0) >> 32);
+            next_fin = E::fin(HEAP(0), cnt);
         } else {
             dur = ad + bd * B + (q_shift >= 0 ? (S >> q_shift) : (S / qd));
             r1 = B; r2 = S; r3 = 0;
@@ -188,28 +215,30 @@ k_simulate(const uint2* __restrict__ q_po, const int32_t* __restrict__ q_off,
             if (cnt == next_fin) {
                 uint32_t n = B;
                 do {                                      // pop every request that retires now
-                    S -= (uint32_t)HEAP(0);
-                    reserved -= (uint32_t)HEAP(0);
+                    const uint32_t gone = E::tot(HEAP(0));
+                    S -= gone;
+                    reserved -= gone;
                     ++r3;
                     --n;
-                    const unsigned long long x = HEAP(n);
+                    const entry_t x = HEAP(n);
+                    const entry_t xr = E::rel(x, cnt);
                     uint32_t i = 0;
                     while (true) {
                         uint32_t ch = 2 * i + 1;
                         if (ch >= n) break;
-                        unsigned long long y = HEAP(ch);
+                        entry_t y = HEAP(ch);
                         if (ch + 1 < n) {
-                            const unsigned long long y2 = HEAP(ch + 1);
-                            if (y2 < y) { y = y2; ++ch; }
+                            const entry_t y2 = HEAP(ch + 1);
+                            if (E::rel(y2, cnt) < E::rel(y, cnt)) { y = y2; ++ch; }
                         }
-                        if (x <= y) break;
+                        if (xr <= E::rel(y, cnt)) break;
                         HEAP(i) = y;
                         i = ch;
                     }
                     if (n > 0) HEAP(i) = x;
-                } while (n > 0 && (uint32_t)(HEAP(0) >> 32) == cnt);
+                } while (n > 0 && E::fin(HEAP(0), cnt) == cnt);
                 B = n;
-                next_fin = n > 0 ? (uint32_t)(HEAP(0) >> 32) : EMPTY;
+                next_fin = n > 0 ? E::fin(HEAP(0), cnt) : EMPTY;
                 grow = head + (int)nA < qn;
             }
             const unsigned long long w = (unsigned long long)Cd + dur;
@@ -334,18 +363,29 @@ cudaError_t launch_simulate(const hos_batch& b, const hos_cost_model& cm, const 
                             cudaStream_t st) {
     const long long n_units = (long long)b.n_inst * n_lambda * b.n_clients;
     const unsigned grid = (unsigned)((n_units + SIM_THREADS - 1) / SIM_THREADS);
-    const size_t smem = (size_t)b.batch_cap * SIM_THREADS * sizeof(unsigned long long);
     int q_shift = -1;                                    // power-of-two KV divisor -> shift
     if ((cm.decode_kv_div & (cm.decode_kv_div - 1)) == 0)
         for (q_shift = 0; (1u << q_shift) != cm.decode_kv_div; ++q_shift) {}
-    cudaError_t e = cudaFuncSetAttribute(k_simulate, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    // Both instantiations are launched; each one runs the instances whose entries it can hold and
+    // returns at once for the others (the flag is per instance, on the device).
+    const size_t smem_n = (size_t)b.batch_cap * SIM_THREADS * sizeof(uint32_t);
+    const size_t smem_w = (size_t)b.batch_cap * SIM_THREADS * sizeof(unsigned long long);
+    cudaError_t e = cudaFuncSetAttribute(k_simulate<NarrowEntry>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_n);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(k_simulate<WideEntry>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_w);
     if (e != cudaSuccess) return e;
     launch_hook("k_simulate", 0, st);
-    k_simulate<<<grid, SIM_THREADS, smem, st>>>(q_po, q_off, inst_status, lambda_q16, n_lambda,
-                                               b.n_clients, n_pad, n_units, b.batch_cap,
-                                               (uint32_t)b.kv_budget, cm, q_shift, max_iters, cres,
-                                               trace, trace_off, status);
+    k_simulate<NarrowEntry><<<grid, SIM_THREADS, smem_n, st>>>(
+        q_po, q_off, inst_status, lambda_q16, n_lambda, b.n_clients, n_pad, n_units, b.batch_cap,
+        (uint32_t)b.kv_budget, cm, q_shift, max_iters, cres, trace, trace_off, status);
     launch_hook("k_simulate", 1, st);
+    if (b.kv_budget >= 65536) {                          // otherwise no p + o can reach 2^16
+        launch_hook("k_simulate_wide", 0, st);
+        k_simulate<WideEntry><<<grid, SIM_THREADS, smem_w, st>>>(
+            q_po, q_off, inst_status, lambda_q16, n_lambda, b.n_clients, n_pad, n_units, b.batch_cap,
+            (uint32_t)b.kv_budget, cm, q_shift, max_iters, cres, trace, trace_off, status);
+        launch_hook("k_simulate_wide", 1, st);
+    }
     return cudaGetLastError();
 }
 

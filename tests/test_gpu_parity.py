@@ -135,6 +135,22 @@ def test_wide_estimates_take_the_64bit_packing_path(hos):
     H.check_lower_bound(hos, p, o, M, 8, 10 ** 6, cm)
 
 
+def test_long_requests_use_the_wide_heap_entries(hos):
+    # p + o >= 2^16 in instance 1 only: the two simulator instantiations split the batch between them
+    rng = np.random.default_rng(11)
+    n_inst, n, M, cap = 3, 300, 5, 12
+    p = rng.integers(1, 3000, size=(n_inst, n)).astype(np.uint32)
+    o = rng.integers(1, 60, size=(n_inst, n)).astype(np.uint32)
+    p[1, ::9] = rng.integers(65000, 90000, size=p[1, ::9].shape)
+    cm = (20000, 40, 15000, 300, 16, 40, 350)
+    kv = 300000
+    g = H.check_offline(hos, p, o, M, cap, kv, cm, 4)
+    for mode in (ora.QUEUE_SORTED, ora.QUEUE_FCFS):
+        H.check_simulate(hos, p, o, M, cap, kv, cm, g["assign"], LAMS, mode)
+    # a divisor that is not a power of two takes the division path
+    H.check_simulate(hos, p, o, M, cap, kv, (20000, 40, 15000, 300, 7, 40, 350), g["assign"], LAMS, ora.QUEUE_SORTED)
+
+
 def test_limits_and_bad_data(hos):
     w = workload("c0")
     p, o = w.lengths()
