@@ -199,13 +199,13 @@ void ora_queue_build(int n, int M, const int32_t* assign, const uint32_t* p, con
     free(a);
 }
 
+/* Trace hash (this build's own definition; the paper has none): h <- (h + dur + C1 kind_n +
+ * C2 tokens + C3 aux) * M  mod 2^64 per record, in trace order, from h = INIT. */
 #define ORA_HASH_INIT  0xCBF29CE484222325ull
-#define ORA_HASH_BASE  0x9E3779B97F4A7C15ull
-#define ORA_HASH_W0    0xBF58476D1CE4E5B9ull
-#define ORA_HASH_W1    0x94D049BB133111EBull
-#define ORA_HASH_W2    0xD6E8FEB86659FD93ull
-#define ORA_HASH_W3    0xA0761D6478BD642Full
-#define ORA_HASH_W4    0xE7037ED1A0B428DBull
+#define ORA_HASH_C1    0x9E3779B1ull
+#define ORA_HASH_C2    0x85EBCA77ull
+#define ORA_HASH_C3    0xC2B2AE3Dull
+#define ORA_HASH_M     0x27D4EB2Full
 
 typedef struct { int64_t kv, rem, total; } ora_running;
 
@@ -221,7 +221,7 @@ void ora_simulate_client(int qn, const int32_t* q_req, const uint32_t* p, const 
     int head = 0;               /* next queue position */
     int64_t reserved = 0;       /* sum over R of (p + o) */
     int64_t t = 0, busy = 0, Cd = 0;
-    uint64_t hash = ORA_HASH_INIT, pw = 1;
+    uint64_t hash = ORA_HASH_INIT;
     uint32_t n_pre = 0, n_dec = 0;
     uint64_t iters = 0;
     int32_t status = 0;
@@ -285,10 +285,8 @@ void ora_simulate_client(int qn, const int32_t* q_req, const uint32_t* p, const 
         t += dur;
         if ((int64_t)iters < trace_cap) { if (trace) trace[iters] = rec; }
         else if (trace) status |= 2;
-        uint64_t g = ORA_HASH_W0 * rec.dur_us + ORA_HASH_W1 * rec.kind_n
-                   + ORA_HASH_W2 * rec.tokens + ORA_HASH_W3 * rec.aux + ORA_HASH_W4;
-        hash += g * pw;
-        pw *= ORA_HASH_BASE;
+        hash = (hash + (uint64_t)rec.dur_us + ORA_HASH_C1 * rec.kind_n + ORA_HASH_C2 * rec.tokens
+                     + ORA_HASH_C3 * rec.aux) * ORA_HASH_M;
         ++iters;
         if (t >= ((int64_t)1 << 39)) { status |= 1; break; }
     }

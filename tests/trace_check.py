@@ -89,17 +89,14 @@ def replay(queue, p, o, cm, cap, kv_budget, lambda_q16, trace):
 
 
 HASH_INIT = 0xCBF29CE484222325
-HASH_BASE = 0x9E3779B97F4A7C15
-HASH_W = (0xBF58476D1CE4E5B9, 0x94D049BB133111EB, 0xD6E8FEB86659FD93, 0xA0761D6478BD642F,
-          0xE7037ED1A0B428DB)
+HASH_C = (1, 0x9E3779B1, 0x85EBCA77, 0xC2B2AE3D)
+HASH_M = 0x27D4EB2F
 
 
 def trace_hash(trace):
-    """hash = INIT + sum_k (W0 dur + W1 kind_n + W2 tokens + W3 aux + W4) * BASE^k  (mod 2^64)."""
+    """h <- (h + dur + C1*kind_n + C2*tokens + C3*aux) * M  (mod 2^64) per record, from h = INIT."""
     mask = (1 << 64) - 1
-    h, pw = HASH_INIT, 1
+    h = HASH_INIT
     for rec in trace:
-        g = sum(w * int(x) for w, x in zip(HASH_W, rec)) + HASH_W[4]
-        h = (h + g * pw) & mask
-        pw = (pw * HASH_BASE) & mask
+        h = ((h + sum(c * int(x) for c, x in zip(HASH_C, rec))) * HASH_M) & mask
     return h
