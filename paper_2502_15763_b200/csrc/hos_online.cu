@@ -90,12 +90,7 @@ k_queue_build(const uint32_t* __restrict__ p, const uint32_t* __restrict__ o,
 // ---------------------------------------------------------------------------------------
 constexpr uint32_t EMPTY = 0xFFFFFFFFu;
 constexpr unsigned long long HASH_INIT = 0xCBF29CE484222325ull;
-constexpr unsigned long long HASH_BASE = 0x9E3779B97F4A7C15ull;
-constexpr unsigned long long HASH_W0 = 0xBF58476D1CE4E5B9ull;
-constexpr unsigned long long HASH_W1 = 0x94D049BB133111EBull;
-constexpr unsigned long long HASH_W2 = 0xD6E8FEB86659FD93ull;
-constexpr unsigned long long HASH_W3 = 0xA0761D6478BD642Full;
-constexpr unsigned long long HASH_W4 = 0xE7037ED1A0B428DBull;
+constexpr uint32_t HASH_C1 = 0x9E3779B1u, HASH_C2 = 0x85EBCA77u, HASH_C3 = 0xC2B2AE3Du, HASH_M = 0x27D4EB2Fu;
 constexpr int SIM_THREADS = 32;          // one warp per CTA: a warp leaves as soon as its clients are done
 
 // Heap entries.  Narrow: (fin mod 2^16) << 16 | tot, usable when every p + o of the instance is
@@ -108,6 +103,7 @@ struct NarrowEntry {
     static __device__ __forceinline__ T rel(T x, uint32_t cnt) { return x - (cnt << 16); }
     static __device__ __forceinline__ uint32_t tot(T x) { return x & 0xFFFFu; }
     static __device__ __forceinline__ uint32_t fin(T x, uint32_t cnt) { return cnt + (rel(x, cnt) >> 16); }
+    static __device__ __forceinline__ T rebase(T staged, uint32_t cnt) { return staged + (cnt << 16); }
 };
 struct WideEntry {
     typedef unsigned long long T;
@@ -115,6 +111,7 @@ struct WideEntry {
     static __device__ __forceinline__ T rel(T x, uint32_t) { return x; }
     static __device__ __forceinline__ uint32_t tot(T x) { return (uint32_t)x; }
     static __device__ __forceinline__ uint32_t fin(T x, uint32_t) { return (uint32_t)(x >> 32); }
+    static __device__ __forceinline__ T rebase(T staged, uint32_t cnt) { return staged + ((T)cnt << 32); }
 };
 
 template <typename E>
@@ -150,49 +147,69 @@ k_simulate(const uint2* __restrict__ q_po, const int32_t* __restrict__ q_off,
     const uint32_t ad = cm.decode_fixed_us, bd = cm.decode_per_seq_us, qd = cm.decode_kv_div;
 
     long long t = 0, busy = 0;
-    uint32_t Cd = 0, cnt = 0, B = 0, S = 0, reserved = 0, iters = 0, n_pre = 0, n_dec = 0;
+    uint32_t Cd = 0, cnt = 0, B = 0, S = 0, reserved = 0, n_pre = 0;   // iterations = n_pre + cnt
     uint32_t next_fin = EMPTY;
     int head = 0;
-    unsigned long long hash = HASH_INIT, pw = 1ull;
+    unsigned long long hash = HASH_INIT;
     uint32_t nA = 0, sumP = 0, sumTot = 0;
     bool grow = true;                        // the candidate prefix may extend
     int32_t status = 0;
 
     uint4* tr = nullptr;
-    long long tr_cap = 0;
+    uint32_t tr_lim = 0;                     // records that fit the caller's slots
     if (trace) {
         const long long t0 = trace_off[unit];
+        const long long capr = trace_off[unit + 1] - t0;
         tr = reinterpret_cast<uint4*>(trace + t0);
-        tr_cap = trace_off[unit + 1] - t0;
+        tr_lim = capr > 0x7FFFFFFFll ? 0x7FFFFFFFu : (uint32_t)(capr < 0 ? 0 : capr);
     }
+    uint2 nxt = make_uint2(0u, 0u);          // queue entry head + nA, fetched ahead of its use
+    if (qn > 0) nxt = __ldg(&q[0]);
 
+    // one iteration's bookkeeping: clock, hash, trace
+    auto emit = [&](uint32_t dur, uint32_t r1, uint32_t r2, uint32_t r3) {
+        const uint32_t it = n_pre + cnt;                 // index of this record (cnt not yet bumped)
+        t += dur;
+        hash = (hash + dur + (unsigned long long)HASH_C1 * r1 + (unsigned long long)HASH_C2 * r2 +
+                (unsigned long long)HASH_C3 * r3) * HASH_M;
+        if (it < tr_lim) tr[it] = make_uint4(dur, r1, r2, r3);
+    };
+
+    // Every pass of this loop is one "event" iteration (a prefill, or a decode that may retire
+    // requests) followed by a quiet run of decode iterations in which nobody retires and the
+    // decision cannot change.  The lanes of a warp meet again at every event, so the heap and
+    // queue work is done by all of them together and the quiet runs are short scalar loops.
+    // The heap is 4-ary: half the depth of a binary heap, and the four children of a node are
+    // independent loads.
     while (true) {
         if (grow) {
             // candidates: the longest queue prefix that fits the free slots and the KV budget.
             // A retirement only loosens both limits, so the prefix found earlier stays valid.
+            // Candidate j waits at heap slot cap-1-j as (o, p+o); B + nA <= cap keeps it clear of
+            // the heap itself.
             while (head + (int)nA < qn && B + nA < (uint32_t)cap) {
-                const uint2 po = __ldg(&q[head + nA]);
-                const uint32_t tt = po.x + po.y;
+                const uint32_t tt = nxt.x + nxt.y;
                 if ((unsigned long long)reserved + sumTot + tt > (unsigned long long)kv_budget) break;
-                sumTot += tt; sumP += po.x; ++nA;
+                HEAP(cap - 1 - (int)nA) = E::make(nxt.y, tt);
+                sumTot += tt; sumP += nxt.x; ++nA;
+                if (head + (int)nA < qn) nxt = __ldg(&q[head + nA]);
             }
             grow = false;
         }
         if (B == 0 && nA == 0) break;                    // queue empty and nothing running
-        if (iters == max_iters) { status |= HOS_ST_LIMIT; break; }
+        if (n_pre + cnt == max_iters) { status |= HOS_ST_LIMIT; break; }
 
         const uint32_t Cp = ap + bp * sumP;
-        const bool prefill =
-            nA > 0 && (B == 0 || (unsigned long long)lam * Cd > ((unsigned long long)Cp << 16));
-        uint32_t dur, r1, r2, r3;
-        if (prefill) {
-            for (uint32_t a = 0; a < nA; ++a) {          // push queue[head .. head + nA)
-                const uint2 po = __ldg(&q[head + a]);
-                const entry_t x = E::make(cnt + po.y, po.x + po.y);
+        const unsigned long long Cp16 = (unsigned long long)Cp << 16;
+        if (nA > 0 && (B == 0 || (unsigned long long)lam * Cd > Cp16)) {
+            // prefill: push the candidates, last staged first (its slot is the lowest, so the
+            // growing heap never reaches a candidate that is still waiting)
+            for (uint32_t j = 0; j < nA; ++j) {
+                const entry_t x = E::rebase(HEAP(cap - (int)nA + (int)j), cnt);
                 const entry_t xr = E::rel(x, cnt);
-                uint32_t i = B + a;
+                uint32_t i = B + j;
                 while (i > 0) {
-                    const uint32_t par = (i - 1) >> 1;
+                    const uint32_t par = (i - 1) >> 2;
                     const entry_t y = HEAP(par);
                     if (E::rel(y, cnt) <= xr) break;
                     HEAP(i) = y;
@@ -200,61 +217,85 @@ k_simulate(const uint2* __restrict__ q_po, const int32_t* __restrict__ q_off,
                 }
                 HEAP(i) = x;
             }
-            dur = Cp; r1 = 0x80000000u | nA; r2 = sumP; r3 = (uint32_t)head;
-            busy += (long long)dur * nA;
+            busy += (long long)Cp * nA;
+            emit(Cp, 0x80000000u | nA, sumP, (uint32_t)head);
             S += sumP; B += nA; reserved += sumTot; head += (int)nA;
             Cd = 0; ++n_pre;
             nA = 0; sumP = 0; sumTot = 0;                 // nothing more fits until someone retires
             next_fin = E::fin(HEAP(0), cnt);
         } else {
-            dur = ad + bd * B + (q_shift >= 0 ? (S >> q_shift) : (S / qd));
-            r1 = B; r2 = S; r3 = 0;
+            const uint32_t dur = ad + bd * B + (q_shift >= 0 ? (S >> q_shift) : (S / qd));
+            const uint32_t B0 = B, S0 = S;
+            uint32_t gone_n = 0;
             busy += (long long)dur * B;
-            ++cnt;
             S += B;
-            if (cnt == next_fin) {
+            if (cnt + 1 == next_fin) {
+                const uint32_t c1 = cnt + 1;
                 uint32_t n = B;
                 do {                                      // pop every request that retires now
                     const uint32_t gone = E::tot(HEAP(0));
                     S -= gone;
                     reserved -= gone;
-                    ++r3;
+                    ++gone_n;
                     --n;
                     const entry_t x = HEAP(n);
-                    const entry_t xr = E::rel(x, cnt);
+                    const entry_t xr = E::rel(x, c1);
                     uint32_t i = 0;
                     while (true) {
-                        uint32_t ch = 2 * i + 1;
+                        const uint32_t ch = 4 * i + 1;
                         if (ch >= n) break;
-                        entry_t y = HEAP(ch);
-                        if (ch + 1 < n) {
-                            const entry_t y2 = HEAP(ch + 1);
-                            if (E::rel(y2, cnt) < E::rel(y, cnt)) { y = y2; ++ch; }
+                        // children beyond the heap's end compare as +infinity
+                        entry_t y0 = HEAP(ch), ym = y0;
+                        entry_t m = E::rel(y0, c1);
+                        uint32_t at = ch;
+#pragma unroll
+                        for (uint32_t k = 1; k < 4; ++k) {
+                            if (ch + k < n) {
+                                const entry_t y = HEAP(ch + k);
+                                const entry_t r = E::rel(y, c1);
+                                if (r < m) { m = r; ym = y; at = ch + k; }
+                            }
                         }
-                        if (xr <= E::rel(y, cnt)) break;
-                        HEAP(i) = y;
-                        i = ch;
+                        if (xr <= m) break;
+                        HEAP(i) = ym;
+                        i = at;
                     }
                     if (n > 0) HEAP(i) = x;
-                } while (n > 0 && E::fin(HEAP(0), cnt) == cnt);
+                } while (n > 0 && E::fin(HEAP(0), c1) == c1);
                 B = n;
-                next_fin = n > 0 ? E::fin(HEAP(0), cnt) : EMPTY;
+                next_fin = n > 0 ? E::fin(HEAP(0), c1) : EMPTY;
                 grow = head + (int)nA < qn;
             }
-            const unsigned long long w = (unsigned long long)Cd + dur;
-            Cd = w > 0x7FFFFFFFull ? 0x7FFFFFFFu : (uint32_t)w;
-            ++n_dec;
+            emit(dur, B0, S0, gone_n);
+            ++cnt;
+            Cd = min(Cd + dur, 0x7FFFFFFFu);              // both below 2^31: no wrap
         }
-        t += dur;
-        hash += (HASH_W0 * dur + HASH_W1 * r1 + HASH_W2 * r2 + HASH_W3 * r3 + HASH_W4) * pw;
-        pw *= HASH_BASE;
-        if (tr) {
-            if ((long long)iters < tr_cap) tr[iters] = make_uint4(dur, r1, r2, r3);
-            else status |= HOS_ST_TRACE;
+        if (t >= (1ll << 39)) { status |= HOS_ST_LIMIT; break; }
+        if (grow || B == 0) continue;
+        // quiet run: at most `room` iterations (next retirement, iteration limit), while the waited
+        // decode time stays at or below the largest value that still says "decode"
+        uint32_t room = min(next_fin - cnt - 1u, max_iters - (n_pre + cnt));
+        uint32_t Cd_max = 0x7FFFFFFFu;                    // Cd saturates there: never above it
+        if (nA > 0 && lam != 0u) {
+            const unsigned long long lim = Cp16 / lam;    // lam * Cd > Cp16  <=>  Cd > floor(Cp16 / lam)
+            Cd_max = lim > 0x7FFFFFFFull ? 0x7FFFFFFFu : (uint32_t)lim;
         }
-        ++iters;
+        const uint32_t base = ad + bd * B;
+        const long long t_run = t;
+        while (room > 0 && Cd <= Cd_max) {
+            const uint32_t dur = base + (q_shift >= 0 ? (S >> q_shift) : (S / qd));
+            emit(dur, B, S, 0u);
+            ++cnt;
+            S += B;
+            Cd = min(Cd + dur, 0x7FFFFFFFu);
+            --room;
+            if (t >= (1ll << 39)) break;
+        }
+        busy += (t - t_run) * (long long)B;
         if (t >= (1ll << 39)) { status |= HOS_ST_LIMIT; break; }
     }
+    if (tr && n_pre + cnt > tr_lim) status |= HOS_ST_TRACE;
+    const uint32_t n_dec = cnt;
     cres[unit] = hos_client_result{t, busy, n_pre, n_dec, hash, 0.0};
     status_out[unit] = status;
 #undef HEAP
