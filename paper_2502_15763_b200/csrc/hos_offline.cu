@@ -272,15 +272,12 @@ __device__ inline void build_member_lists(const uint8_t* bins, IdxT* cl, int n, 
     const int lane = lane_id(), warp = warp_id();
     const int chunk = (((n + SORT_WARPS - 1) / SORT_WARPS) + 31) & ~31;
     const int lo = warp * chunk, hi = min(n, lo + chunk);
+    const int nb = bit_width_u32((uint32_t)(n_clients - 1));
     for (int x = threadIdx.x; x < n_clients * SORT_WARPS; x += SORT_THREADS) cnt[x] = 0;
     __syncthreads();
     for (int row = lo; row < hi; row += 32) {
         const int r = row + lane;
-        const bool valid = r < hi;
-        const uint32_t dig = valid ? (uint32_t)bins[r] : 0xFFFFu;
-        const unsigned m = __match_any_sync(FULL, dig);
-        if (valid && lane == (__ffs(m) - 1)) cnt[dig * SORT_WARPS + warp] += __popc(m);
-        __syncwarp();
+        if (r < hi) atomicAdd(&cnt[(uint32_t)bins[r] * SORT_WARPS + warp], 1u);
     }
     __syncthreads();
     block_scan_u32(cnt, n_clients * SORT_WARPS, wsum);
@@ -290,8 +287,13 @@ __device__ inline void build_member_lists(const uint8_t* bins, IdxT* cl, int n, 
     for (int row = lo; row < hi; row += 32) {
         const int r = row + lane;
         const bool valid = r < hi;
-        const uint32_t dig = valid ? (uint32_t)bins[r] : 0xFFFFu;
-        const unsigned m = __match_any_sync(FULL, dig);
+        const uint32_t dig = valid ? (uint32_t)bins[r] : 0u;
+        unsigned m = __ballot_sync(FULL, valid);             // lanes of this row on my client
+        for (int b = 0; b < nb; ++b) {
+            const bool bit = (dig >> b) & 1u;
+            const unsigned bal = __ballot_sync(FULL, bit);
+            m &= bit ? bal : ~bal;
+        }
         const uint32_t base = valid ? cnt[dig * SORT_WARPS + warp] : 0u;
         __syncwarp();
         if (valid) {

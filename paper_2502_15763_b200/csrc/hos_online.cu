@@ -119,13 +119,15 @@ __global__ void __launch_bounds__(SIM_THREADS)
 k_simulate(const uint2* __restrict__ q_po, const int32_t* __restrict__ q_off,
            const int32_t* __restrict__ inst_status, const uint32_t* __restrict__ lambda_q16,
            int n_lambda, int n_clients, int n_pad, long long n_units, int cap, uint32_t kv_budget,
-           hos_cost_model cm, int q_shift, uint32_t max_iters, hos_client_result* __restrict__ cres,
+           hos_cost_model cm, int q_shift, uint32_t max_iters,
+           hos_client_result* __restrict__ cres,
            hos_iter_rec* __restrict__ trace, const long long* __restrict__ trace_off,
            int32_t* __restrict__ status_out) {
     typedef typename E::T entry_t;
     extern __shared__ __align__(16) unsigned char smem_raw[];
     entry_t* heap = reinterpret_cast<entry_t*>(smem_raw) + threadIdx.x;
-#define HEAP(s) heap[(s) * SIM_THREADS]
+    auto heap_ld = [&](int sl) -> entry_t { return heap[sl * SIM_THREADS]; };
+    auto heap_st = [&](int sl, entry_t v) { heap[sl * SIM_THREADS] = v; };
     const long long unit = (long long)blockIdx.x * SIM_THREADS + threadIdx.x;
     if (unit >= n_units) return;
     const int c = (int)(unit % n_clients);
@@ -163,8 +165,10 @@ k_simulate(const uint2* __restrict__ q_po, const int32_t* __restrict__ q_off,
         tr = reinterpret_cast<uint4*>(trace + t0);
         tr_lim = capr > 0x7FFFFFFFll ? 0x7FFFFFFFu : (uint32_t)(capr < 0 ? 0 : capr);
     }
-    uint2 nxt = make_uint2(0u, 0u);          // queue entry head + nA, fetched ahead of its use
+    uint2 nxt = make_uint2(0u, 0u);          // queue entries head + nA and head + nA + 1,
+    uint2 nxt2 = make_uint2(0u, 0u);         // fetched ahead of their use
     if (qn > 0) nxt = __ldg(&q[0]);
+    if (qn > 1) nxt2 = __ldg(&q[1]);
 
     // one iteration's bookkeeping: clock, hash, trace
     auto emit = [&](uint32_t dur, uint32_t r1, uint32_t r2, uint32_t r3) {
@@ -189,10 +193,11 @@ k_simulate(const uint2* __restrict__ q_po, const int32_t* __restrict__ q_off,
             // the heap itself.
             while (head + (int)nA < qn && B + nA < (uint32_t)cap) {
                 const uint32_t tt = nxt.x + nxt.y;
-                if ((unsigned long long)reserved + sumTot + tt > (unsigned long long)kv_budget) break;
-                HEAP(cap - 1 - (int)nA) = E::make(nxt.y, tt);
+                if (reserved + sumTot + tt > kv_budget) break;   // each term < 2^31 and reserved + sumTot <= budget: no wrap
+                heap_st(cap - 1 - (int)nA, E::make(nxt.y, tt));
                 sumTot += tt; sumP += nxt.x; ++nA;
-                if (head + (int)nA < qn) nxt = __ldg(&q[head + nA]);
+                nxt = nxt2;
+                if (head + (int)nA + 1 < qn) nxt2 = __ldg(&q[head + nA + 1]);
             }
             grow = false;
         }
@@ -201,31 +206,31 @@ k_simulate(const uint2* __restrict__ q_po, const int32_t* __restrict__ q_off,
 
         const uint32_t Cp = ap + bp * sumP;
         const unsigned long long Cp16 = (unsigned long long)Cp << 16;
+        uint32_t dur, r1, r2, r3;
         if (nA > 0 && (B == 0 || (unsigned long long)lam * Cd > Cp16)) {
             // prefill: push the candidates, last staged first (its slot is the lowest, so the
             // growing heap never reaches a candidate that is still waiting)
             for (uint32_t j = 0; j < nA; ++j) {
-                const entry_t x = E::rebase(HEAP(cap - (int)nA + (int)j), cnt);
+                const entry_t x = E::rebase(heap_ld(cap - (int)nA + (int)j), cnt);
                 const entry_t xr = E::rel(x, cnt);
                 uint32_t i = B + j;
                 while (i > 0) {
                     const uint32_t par = (i - 1) >> 2;
-                    const entry_t y = HEAP(par);
+                    const entry_t y = heap_ld((int)par);
                     if (E::rel(y, cnt) <= xr) break;
-                    HEAP(i) = y;
+                    heap_st((int)i, y);
                     i = par;
                 }
-                HEAP(i) = x;
+                heap_st((int)i, x);
             }
+            dur = Cp; r1 = 0x80000000u | nA; r2 = sumP; r3 = (uint32_t)head;
             busy += (long long)Cp * nA;
-            emit(Cp, 0x80000000u | nA, sumP, (uint32_t)head);
             S += sumP; B += nA; reserved += sumTot; head += (int)nA;
-            Cd = 0; ++n_pre;
             nA = 0; sumP = 0; sumTot = 0;                 // nothing more fits until someone retires
-            next_fin = E::fin(HEAP(0), cnt);
+            next_fin = E::fin(heap_ld(0), cnt);
         } else {
-            const uint32_t dur = ad + bd * B + (q_shift >= 0 ? (S >> q_shift) : (S / qd));
-            const uint32_t B0 = B, S0 = S;
+            dur = ad + bd * B + (q_shift >= 0 ? (S >> q_shift) : (S / qd));
+            r1 = B; r2 = S;
             uint32_t gone_n = 0;
             busy += (long long)dur * B;
             S += B;
@@ -233,63 +238,61 @@ k_simulate(const uint2* __restrict__ q_po, const int32_t* __restrict__ q_off,
                 const uint32_t c1 = cnt + 1;
                 uint32_t n = B;
                 do {                                      // pop every request that retires now
-                    const uint32_t gone = E::tot(HEAP(0));
+                    const uint32_t gone = E::tot(heap_ld(0));
                     S -= gone;
                     reserved -= gone;
                     ++gone_n;
                     --n;
-                    const entry_t x = HEAP(n);
+                    const entry_t x = heap_ld((int)n);
                     const entry_t xr = E::rel(x, c1);
                     uint32_t i = 0;
                     while (true) {
                         const uint32_t ch = 4 * i + 1;
                         if (ch >= n) break;
                         // children beyond the heap's end compare as +infinity
-                        entry_t y0 = HEAP(ch), ym = y0;
+                        entry_t y0 = heap_ld((int)ch), ym = y0;
                         entry_t m = E::rel(y0, c1);
                         uint32_t at = ch;
 #pragma unroll
                         for (uint32_t k = 1; k < 4; ++k) {
                             if (ch + k < n) {
-                                const entry_t y = HEAP(ch + k);
+                                const entry_t y = heap_ld((int)(ch + k));
                                 const entry_t r = E::rel(y, c1);
                                 if (r < m) { m = r; ym = y; at = ch + k; }
                             }
                         }
                         if (xr <= m) break;
-                        HEAP(i) = ym;
+                        heap_st((int)i, ym);
                         i = at;
                     }
-                    if (n > 0) HEAP(i) = x;
-                } while (n > 0 && E::fin(HEAP(0), c1) == c1);
+                    if (n > 0) heap_st((int)i, x);
+                } while (n > 0 && E::fin(heap_ld(0), c1) == c1);
                 B = n;
-                next_fin = n > 0 ? E::fin(HEAP(0), c1) : EMPTY;
+                next_fin = n > 0 ? E::fin(heap_ld(0), c1) : EMPTY;
                 grow = head + (int)nA < qn;
             }
-            emit(dur, B0, S0, gone_n);
-            ++cnt;
-            Cd = min(Cd + dur, 0x7FFFFFFFu);              // both below 2^31: no wrap
+            r3 = gone_n;
         }
+        emit(dur, r1, r2, r3);
+        if (r1 >> 31) { Cd = 0; ++n_pre; }
+        else { ++cnt; Cd = min(Cd + dur, 0x7FFFFFFFu); }  // both below 2^31: no wrap
         if (t >= (1ll << 39)) { status |= HOS_ST_LIMIT; break; }
         if (grow || B == 0) continue;
-        // quiet run: at most `room` iterations (next retirement, iteration limit), while the waited
-        // decode time stays at or below the largest value that still says "decode"
-        uint32_t room = min(next_fin - cnt - 1u, max_iters - (n_pre + cnt));
-        uint32_t Cd_max = 0x7FFFFFFFu;                    // Cd saturates there: never above it
-        if (nA > 0 && lam != 0u) {
-            const unsigned long long lim = Cp16 / lam;    // lam * Cd > Cp16  <=>  Cd > floor(Cp16 / lam)
-            Cd_max = lim > 0x7FFFFFFFull ? 0x7FFFFFFFu : (uint32_t)lim;
-        }
+        // quiet run: at most `room` iterations -- up to the next retirement, the iteration limit,
+        // and so few that only the last of them can take the clock past its limit (every
+        // iteration adds less than 2^31) -- and only while the rule keeps saying "decode"
+        const uint32_t room_t = (uint32_t)(((1ll << 39) - 1 - t) >> 31) + 1u;
+        uint32_t room = min(min(next_fin - cnt - 1u, max_iters - (n_pre + cnt)), room_t);
+        const uint32_t lam_run = nA > 0 ? lam : 0u;      // no candidates: nothing to prefill
         const uint32_t base = ad + bd * B;
         const long long t_run = t;
-        while (room > 0 && Cd <= Cd_max) {
-            const uint32_t dur = base + (q_shift >= 0 ? (S >> q_shift) : (S / qd));
-            emit(dur, B, S, 0u);
+        while (room > 0 && (unsigned long long)lam_run * Cd <= Cp16) {
+            const uint32_t dq = base + (q_shift >= 0 ? (S >> q_shift) : (S / qd));
+            emit(dq, B, S, 0u);
             ++cnt;
             S += B;
-            Cd = min(Cd + dur, 0x7FFFFFFFu);
+            Cd = min(Cd + dq, 0x7FFFFFFFu);
             --room;
-            if (t >= (1ll << 39)) break;
         }
         busy += (t - t_run) * (long long)B;
         if (t >= (1ll << 39)) { status |= HOS_ST_LIMIT; break; }
@@ -298,7 +301,6 @@ k_simulate(const uint2* __restrict__ q_po, const int32_t* __restrict__ q_off,
     const uint32_t n_dec = cnt;
     cres[unit] = hos_client_result{t, busy, n_pre, n_dec, hash, 0.0};
     status_out[unit] = status;
-#undef HEAP
 }
 
 // ---------------------------------------------------------------------------------------
@@ -409,8 +411,9 @@ cudaError_t launch_simulate(const hos_batch& b, const hos_cost_model& cm, const 
         for (q_shift = 0; (1u << q_shift) != cm.decode_kv_div; ++q_shift) {}
     // Both instantiations are launched; each one runs the instances whose entries it can hold and
     // returns at once for the others (the flag is per instance, on the device).
-    const size_t smem_n = (size_t)b.batch_cap * SIM_THREADS * sizeof(uint32_t);
-    const size_t smem_w = (size_t)b.batch_cap * SIM_THREADS * sizeof(unsigned long long);
+    const int slots_n = b.batch_cap, slots_w = b.batch_cap;
+    const size_t smem_n = (size_t)slots_n * SIM_THREADS * sizeof(uint32_t);
+    const size_t smem_w = (size_t)slots_w * SIM_THREADS * sizeof(unsigned long long);
     cudaError_t e = cudaFuncSetAttribute(k_simulate<NarrowEntry>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_n);
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(k_simulate<WideEntry>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_w);

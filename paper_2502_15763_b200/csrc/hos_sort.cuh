@@ -3,9 +3,11 @@
 // One CTA of SORT_THREADS threads owns one instance.  The ids 0..n-1 are sorted
 // ascending by (key[id] ^ flip), `nbits` low bits significant, 8 bits per pass; equal keys
 // keep id order (the first pass reads ids in natural order, every pass is stable).  Each
-// warp owns a contiguous chunk of positions; a pass is (1) per-warp digit counts,
-// (2) one exclusive scan over the [digit][warp] count matrix, (3) a stable scatter in which
-// the rank of an item among the equal digits of its 32-wide row comes from match_any.
+// warp owns a contiguous chunk of positions; a pass is (1) per-warp digit counts by shared
+// memory atomics, (2) one exclusive scan over the [digit][warp] count matrix, (3) a stable
+// scatter in which the rank of an item among the equal digits of its 32-wide row comes from
+// one ballot per digit bit.  The count matrix has a row stride of 33 words so that the 32
+// lanes of a warp, which all address their own warp's column, spread over the banks.
 #pragma once
 
 #include "hos_common.cuh"
@@ -18,16 +20,20 @@ struct SortSmem {
     uint32_t* key;      // [n]
     IdxT* buf0;         // [n]
     IdxT* buf1;         // [n]
-    uint32_t* cnt;      // [RADIX * SORT_WARPS]
+    uint32_t* cnt;      // [CNT_WORDS], entry (digit, warp) at digit * CNT_STRIDE + warp
     uint32_t* wsum;     // [SORT_WARPS]
 };
+
+constexpr int CNT_STRIDE = SORT_WARPS + 1;
+constexpr int CNT_PER_THREAD = (RADIX * CNT_STRIDE + SORT_THREADS - 1) / SORT_THREADS;
+constexpr int CNT_WORDS = CNT_PER_THREAD * SORT_THREADS;     // padded; the padding stays zero
 
 __host__ __device__ inline size_t align16(size_t x) { return (x + 15) & ~size_t(15); }
 
 template <typename IdxT>
 __host__ __device__ inline size_t sort_smem_bytes(int n) {
     return align16(size_t(n) * 4) + 2 * align16(size_t(n) * sizeof(IdxT)) +
-           size_t(RADIX) * SORT_WARPS * 4 + SORT_WARPS * 4;
+           size_t(CNT_WORDS) * 4 + SORT_WARPS * 4;
 }
 
 template <typename IdxT>
@@ -40,14 +46,14 @@ __device__ inline SortSmem<IdxT> sort_smem_carve(unsigned char* base, int n) {
     s.buf1 = reinterpret_cast<IdxT*>(base);
     base += align16(size_t(n) * sizeof(IdxT));
     s.cnt = reinterpret_cast<uint32_t*>(base);
-    base += size_t(RADIX) * SORT_WARPS * 4;
+    base += size_t(CNT_WORDS) * 4;
     s.wsum = reinterpret_cast<uint32_t*>(base);
     return s;
 }
 
-// Exclusive scan of cnt[0 .. RADIX*SORT_WARPS) in place.  All SORT_THREADS threads call it.
+// Exclusive scan of cnt[0 .. CNT_WORDS) in place.  All SORT_THREADS threads call it.
 __device__ inline void scan_counts(uint32_t* cnt, uint32_t* wsum) {
-    constexpr int PER = RADIX * SORT_WARPS / SORT_THREADS;   // 8 consecutive entries per thread
+    constexpr int PER = CNT_PER_THREAD;                      // consecutive entries per thread
     const int t = threadIdx.x;
     uint32_t v[PER];
     uint32_t run = 0;
@@ -102,35 +108,58 @@ __device__ inline IdxT* block_radix_sort_ids(const SortSmem<IdxT>& s, int n, int
         return dst;
     }
     for (int shift = 0; shift < nbits; shift += RADIX_BITS) {
-        for (int i = threadIdx.x; i < RADIX * SORT_WARPS; i += SORT_THREADS) s.cnt[i] = 0;
+        const int nb = min(RADIX_BITS, nbits - shift);       // significant bits of this digit
+        const uint32_t dmask = (1u << nb) - 1u;
+        for (int i = threadIdx.x; i < CNT_WORDS; i += SORT_THREADS) s.cnt[i] = 0;
         __syncthreads();
         // (1) per-warp digit counts
         for (int row = lo; row < hi; row += 32) {
             const int pos = row + lane;
-            const bool valid = pos < hi;
-            uint32_t id = valid ? (natural ? (uint32_t)pos : (uint32_t)src[pos]) : 0u;
-            uint32_t dig = valid ? (((s.key[id] ^ flip) >> shift) & (RADIX - 1)) : (uint32_t)RADIX;
-            unsigned m = __match_any_sync(FULL, dig);
-            if (valid && lane == (__ffs(m) - 1)) s.cnt[dig * SORT_WARPS + warp] += __popc(m);
-            __syncwarp();
+            if (pos < hi) {
+                const uint32_t id = natural ? (uint32_t)pos : (uint32_t)src[pos];
+                const uint32_t dig = ((s.key[id] ^ flip) >> shift) & dmask;
+                atomicAdd(&s.cnt[dig * CNT_STRIDE + warp], 1u);
+            }
         }
         __syncthreads();
         // (2) offsets
         scan_counts(s.cnt, s.wsum);
-        // (3) stable scatter
-        for (int row = lo; row < hi; row += 32) {
-            const int pos = row + lane;
-            const bool valid = pos < hi;
-            uint32_t id = valid ? (natural ? (uint32_t)pos : (uint32_t)src[pos]) : 0u;
-            uint32_t dig = valid ? (((s.key[id] ^ flip) >> shift) & (RADIX - 1)) : (uint32_t)RADIX;
-            unsigned m = __match_any_sync(FULL, dig);
-            uint32_t base = valid ? s.cnt[dig * SORT_WARPS + warp] : 0u;
-            __syncwarp();
-            if (valid) {
-                dst[base + __popc(m & ((1u << lane) - 1u))] = (IdxT)id;
-                if (lane == (__ffs(m) - 1)) s.cnt[dig * SORT_WARPS + warp] = base + __popc(m);
+        // (3) stable scatter, four rows at a time: the key loads and ballots of the four rows
+        //     are independent of each other; only the counter updates run row after row
+        constexpr int G = 4;
+        for (int row = lo; row < hi; row += 32 * G) {
+            uint32_t id[G], dig[G];
+            unsigned m[G];
+            bool valid[G];
+#pragma unroll
+            for (int g = 0; g < G; ++g) {
+                const int pos = row + 32 * g + lane;
+                valid[g] = pos < hi;
+                id[g] = valid[g] ? (natural ? (uint32_t)pos : (uint32_t)src[pos]) : 0u;
             }
-            __syncwarp();
+#pragma unroll
+            for (int g = 0; g < G; ++g) {
+                dig[g] = valid[g] ? (((s.key[id[g]] ^ flip) >> shift) & dmask) : 0u;
+                m[g] = __ballot_sync(FULL, valid[g]);        // lanes of this row with my digit
+            }
+            for (int b = 0; b < nb; ++b) {
+#pragma unroll
+                for (int g = 0; g < G; ++g) {
+                    const bool bit = (dig[g] >> b) & 1u;
+                    const unsigned bal = __ballot_sync(FULL, bit);
+                    m[g] &= bit ? bal : ~bal;
+                }
+            }
+#pragma unroll
+            for (int g = 0; g < G; ++g) {
+                const uint32_t base = valid[g] ? s.cnt[dig[g] * CNT_STRIDE + warp] : 0u;
+                __syncwarp();
+                if (valid[g]) {
+                    dst[base + __popc(m[g] & ((1u << lane) - 1u))] = (IdxT)id[g];
+                    if (lane == (__ffs(m[g]) - 1)) s.cnt[dig[g] * CNT_STRIDE + warp] = base + __popc(m[g]);
+                }
+                __syncwarp();
+            }
         }
         __syncthreads();
         IdxT* t = src; src = dst; dst = t;
