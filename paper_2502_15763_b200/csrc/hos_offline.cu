@@ -264,11 +264,13 @@ __device__ inline void block_scan_u32(uint32_t* a, int len, uint32_t* wsum) {
     __syncthreads();
 }
 
-// Member lists of all clients from bins[]: a stable split of the ranks 0..n-1 by client.
+// Member lists of all clients from bins[]: a stable split of the ranks 0..n-1 by client, with the
+// members' T beside them (clT).
 // cnt holds n_clients * SORT_WARPS words.  off[k] = start of client k's list, off[M] = n.
 template <typename IdxT>
-__device__ inline void build_member_lists(const uint8_t* bins, IdxT* cl, int n, int n_clients,
-                                          uint32_t* cnt, uint32_t* wsum, int* off) {
+__device__ inline void build_member_lists(const uint8_t* bins, const uint32_t* __restrict__ gT, IdxT* cl,
+                                          uint32_t* clT, int n, int n_clients, uint32_t* cnt,
+                                          uint32_t* wsum, int* off) {
     const int lane = lane_id(), warp = warp_id();
     const int chunk = (((n + SORT_WARPS - 1) / SORT_WARPS) + 31) & ~31;
     const int lo = warp * chunk, hi = min(n, lo + chunk);
@@ -288,6 +290,7 @@ __device__ inline void build_member_lists(const uint8_t* bins, IdxT* cl, int n, 
         const int r = row + lane;
         const bool valid = r < hi;
         const uint32_t dig = valid ? (uint32_t)bins[r] : 0u;
+        const uint32_t tr = valid ? gT[r] : 0u;
         unsigned m = __ballot_sync(FULL, valid);             // lanes of this row on my client
         for (int b = 0; b < nb; ++b) {
             const bool bit = (dig >> b) & 1u;
@@ -297,7 +300,9 @@ __device__ inline void build_member_lists(const uint8_t* bins, IdxT* cl, int n, 
         const uint32_t base = valid ? cnt[dig * SORT_WARPS + warp] : 0u;
         __syncwarp();
         if (valid) {
-            cl[base + __popc(m & ((1u << lane) - 1u))] = (IdxT)r;
+            const uint32_t at = base + __popc(m & ((1u << lane) - 1u));
+            cl[at] = (IdxT)r;
+            clT[at] = tr;
             if (lane == (__ffs(m) - 1)) cnt[dig * SORT_WARPS + warp] = base + __popc(m);
         }
         __syncwarp();
@@ -340,10 +345,10 @@ k_local_search(const uint32_t* __restrict__ T_sorted, const uint32_t* __restrict
     __shared__ long long s_load[MAX_CLIENTS];
     __shared__ int s_off[MAX_CLIENTS + 1];
     __shared__ Cand s_cand[32];
-    __shared__ uint32_t s_inv[32];
     __shared__ uint32_t s_wsum[32];
     __shared__ int s_as[MAX_CLIENTS];
     __shared__ uint8_t s_ak[MAX_CLIENTS];
+    __shared__ uint8_t s_listed[MAX_CLIENTS];
     __shared__ int s_jmax, s_kmin, s_na, s_nitems;
     __shared__ long long s_lmax;
 
@@ -367,7 +372,7 @@ k_local_search(const uint32_t* __restrict__ T_sorted, const uint32_t* __restrict
     }
 
     unsigned char* base = smem_raw;
-    uint32_t* Ts = reinterpret_cast<uint32_t*>(base);   base += align16((size_t)n_req * 4);
+    uint32_t* clT = reinterpret_cast<uint32_t*>(base);  base += align16((size_t)n_req * 4);
     IdxT* ord = reinterpret_cast<IdxT*>(base);          base += align16((size_t)n_req * sizeof(IdxT));
     IdxT* cl = reinterpret_cast<IdxT*>(base);           base += align16((size_t)n_req * sizeof(IdxT));
     uint8_t* bins = reinterpret_cast<uint8_t*>(base);   base += align16((size_t)n_req);
@@ -381,7 +386,6 @@ k_local_search(const uint32_t* __restrict__ T_sorted, const uint32_t* __restrict
     for (int r = threadIdx.x; r < n_req; r += SORT_THREADS) {
         const uint32_t t = gT[r], id = gO[r];
         const int c = asg[id];
-        Ts[r] = t;
         ord[r] = (IdxT)id;
         if (c < 0 || c >= n_clients) { bad_assign = true; bins[r] = 0; }
         else {
@@ -400,50 +404,46 @@ k_local_search(const uint32_t* __restrict__ T_sorted, const uint32_t* __restrict
             for (int r = threadIdx.x; r < rounds; r += SORT_THREADS) log[r] = hos_ls_move{-1, -1, -1, 0};
         return;
     }
-    build_member_lists<IdxT>(bins, cl, n_req, n_clients, cnt, s_wsum, s_off);
+    build_member_lists<IdxT>(bins, gT, cl, clT, n_req, n_clients, cnt, s_wsum, s_off);
 
     int applied = 0;
     int done_at = rounds;
+    long long margin = 64;                  // how far above the least loaded client's floor to look first
+
+    // critical client (largest load, ties to the lowest client) and least loaded client (ties to the
+    // highest, so that it differs from the critical one unless all loads are equal); one warp
+    auto find_extremes = [&]() {
+        long long bl = -1, ml = NO_V;
+        int bj = NO_I, mj = -1;
+        for (int j = lane; j < n_clients; j += 32) {
+            const long long l = s_load[j];
+            if (l > bl) { bl = l; bj = j; }
+            if (l <= ml) { ml = l; mj = j; }
+        }
+#pragma unroll
+        for (int d = 16; d > 0; d >>= 1) {
+            const long long ol = __shfl_xor_sync(FULL, bl, d);
+            const int oj = __shfl_xor_sync(FULL, bj, d);
+            if (ol > bl || (ol == bl && oj < bj)) { bl = ol; bj = oj; }
+            const long long pl = __shfl_xor_sync(FULL, ml, d);
+            const int pj = __shfl_xor_sync(FULL, mj, d);
+            if (pl < ml || (pl == ml && pj > mj)) { ml = pl; mj = pj; }
+        }
+        if (lane == 0) { s_jmax = bj; s_lmax = bl; s_kmin = mj; }
+    };
+    if (warp == 0) find_extremes();
+    __syncthreads();
 
     for (int round = 0; round < rounds; ++round) {
-        // (a) critical client: largest load, ties to the lowest client (warp 0); the least loaded
-        //     other client, any of them on ties, seeds the pruning bound (warp 1, once jmax is known
-        //     it only has to skip it, and the least loaded client is never the critical one unless
-        //     all loads are equal, in which case no step can improve)
-        if (warp == 0) {
-            long long bl = -1;
-            int bj = NO_I;
-            for (int j = lane; j < n_clients; j += 32)
-                if (s_load[j] > bl) { bl = s_load[j]; bj = j; }
-#pragma unroll
-            for (int d = 16; d > 0; d >>= 1) {
-                const long long ol = __shfl_xor_sync(FULL, bl, d);
-                const int oj = __shfl_xor_sync(FULL, bj, d);
-                if (ol > bl || (ol == bl && oj < bj)) { bl = ol; bj = oj; }
-            }
-            if (lane == 0) { s_jmax = bj; s_lmax = bl; }
-        } else if (warp == 1) {
-            long long ml = NO_V;
-            int mj = -1;
-            for (int j = lane; j < n_clients; j += 32)
-                if (s_load[j] < ml) { ml = s_load[j]; mj = j; }
-#pragma unroll
-            for (int d = 16; d > 0; d >>= 1) {
-                const long long ol = __shfl_xor_sync(FULL, ml, d);
-                const int oj = __shfl_xor_sync(FULL, mj, d);
-                if (ol < ml || (ol == ml && oj > mj)) { ml = ol; mj = oj; }   // highest client on ties
-            }
-            if (lane == 0) s_kmin = mj;
-        }
-        __syncthreads();
         const int jmax = s_jmax;
         const long long Lmax = s_lmax;
-        // all loads equal: kmin may coincide with jmax; then nothing can improve anyway
+        // all loads equal: the least loaded client is as loaded as the critical one; nothing can improve
         const int kmin = (s_kmin != jmax && s_load[s_kmin] < Lmax) ? s_kmin : -1;
         const IdxT* mem = cl + s_off[jmax];                 // jmax's members, T descending
+        const uint32_t* memT = clT + s_off[jmax];
         const int nm = s_off[jmax + 1] - s_off[jmax];
 
-        // (b) one work item: client k, position idx in its list (idx == its length: the move)
+        // (a) one work item: client k, position idx in its list (idx == its length: the move)
         auto evaluate = [&](int k, int idx, int len, Cand& best) {
             const long long lk = s_load[k];
             const long long slack = Lmax - lk;
@@ -451,27 +451,27 @@ k_local_search(const uint32_t* __restrict__ T_sorted, const uint32_t* __restrict
             int pu = -1;
             long long Tu = 0;
             if (idx < len) {
-                const int w = (int)cl[s_off[k] + idx];
-                u1 = (uint32_t)ord[w] + 1u; pu = idx; Tu = Ts[w];
+                const int at = s_off[k] + idx;
+                u1 = (uint32_t)ord[cl[at]] + 1u; pu = idx; Tu = clT[at];
             }
             const long long thr = Tu + ((slack + 1) >> 1);      // T_i >= thr  <=>  2 d >= slack
             int a = 0, z = nm;                                  // b = members with T >= thr
             while (a < z) {
                 const int mid = (a + z) >> 1;
-                if ((long long)Ts[mem[mid]] >= thr) a = mid + 1; else z = mid;
+                if ((long long)memT[mid] >= thr) a = mid + 1; else z = mid;
             }
             const int b = a;
             if (b > 0) {                                        // rising side: smallest T >= thr
-                const uint32_t Ti = Ts[mem[b - 1]];
+                const uint32_t Ti = memT[b - 1];
                 const long long d = (long long)Ti - Tu;
                 if (d < slack) {
                     int a2 = b - 1;                             // first member of the run of equal T
-                    if (b >= 2 && Ts[mem[b - 2]] == Ti) {
+                    if (b >= 2 && memT[b - 2] == Ti) {
                         int z2 = b - 2;
                         a2 = 0;
                         while (a2 < z2) {
                             const int mid = (a2 + z2) >> 1;
-                            if (Ts[mem[mid]] > Ti) a2 = mid + 1; else z2 = mid;
+                            if (memT[mid] > Ti) a2 = mid + 1; else z2 = mid;
                         }
                     }
                     Cand c;                                     // v = lk + d, Lmax - v = slack - d
@@ -481,7 +481,7 @@ k_local_search(const uint32_t* __restrict__ T_sorted, const uint32_t* __restrict
                 }
             }
             if (b < nm) {                                       // falling side: largest T < thr
-                const long long d = (long long)Ts[mem[b]] - Tu;
+                const long long d = (long long)memT[b] - Tu;
                 if (d > 0) {
                     Cand c;                                     // v = Lmax - d
                     c.inv = ~(uint32_t)d; c.pi = b; c.ik = ((uint32_t)ord[mem[b]] << 8) | (uint32_t)k;
@@ -490,32 +490,25 @@ k_local_search(const uint32_t* __restrict__ T_sorted, const uint32_t* __restrict
                 }
             }
         };
-        Cand best;
-        best.inv = NO_CAND; best.ik = NO_CAND; best.u1 = NO_CAND; best.pi = -1; best.pu = -1;
-        // (c) the least loaded client first: its best step is achievable, hence bounds the optimum
-        if (kmin >= 0) {
-            const int len = s_off[kmin + 1] - s_off[kmin];
-            for (int idx = threadIdx.x; idx <= len; idx += SORT_THREADS) evaluate(kmin, idx, len, best);
-        }
-        {
-            const uint32_t wi = __reduce_min_sync(FULL, best.inv);
-            if (lane == 0) s_inv[warp] = wi;
-        }
-        __syncthreads();
-        // (d) warp 0 lists the other clients whose floor ceil((Lmax + load_k) / 2) does not exceed
-        //     the bound, with the running count of their work items (list length + 1 move)
-        if (warp == 0) {
-            const uint32_t inv = __reduce_min_sync(FULL, s_inv[lane]);
-            const long long vbound = Lmax - (long long)(~inv);          // no candidate: gain 0 -> Lmax
+        // (b) warp 0 lists the clients to look at, with the running count of their work items (list
+        //     length + 1 move).  Any step onto client k ends with v >= floor_k = ceil((Lmax + load_k) / 2),
+        //     so a client whose floor is above an achieved v cannot win or tie.  First pass: the
+        //     clients whose floor is within `margin` of the least loaded client's; after the
+        //     reduction, any client left out whose floor does not exceed the best v found is
+        //     evaluated in a second pass (vlimit = that v), which makes the result exact whatever
+        //     the margin was.
+        auto list_clients = [&](long long vlimit, bool skip_listed) {
             int n_alive = 0, n_items = 0;
             for (int k0 = 0; k0 < n_clients; k0 += 32) {
                 const int k = k0 + lane;
                 bool alive = false;
                 int sz = 0;
-                if (k < n_clients && k != jmax && k != kmin) {
+                if (k < n_clients && k != jmax) {
                     const long long lk = s_load[k];
-                    alive = lk < Lmax && ((Lmax + lk + 1) >> 1) <= vbound;
+                    alive = lk < Lmax && ((Lmax + lk + 1) >> 1) <= vlimit && !(skip_listed && s_listed[k]);
                     sz = alive ? s_off[k + 1] - s_off[k] + 1 : 0;
+                    if (!skip_listed) s_listed[k] = alive;
+                    else if (alive) s_listed[k] = 1;
                 }
                 const unsigned am = __ballot_sync(FULL, alive);
                 int inc = sz;
@@ -533,9 +526,8 @@ k_local_search(const uint32_t* __restrict__ T_sorted, const uint32_t* __restrict
                 n_items += __shfl_sync(FULL, inc, 31);
             }
             if (lane == 0) { s_na = n_alive; s_nitems = n_items; }
-        }
-        __syncthreads();
-        {
+        };
+        auto evaluate_listed = [&](Cand& best) {
             const int n_alive = s_na, n_items = s_nitems;
             for (int x = threadIdx.x; x < n_items; x += SORT_THREADS) {
                 int a = 0, z = n_alive;                         // last listed client with start <= x
@@ -546,63 +538,98 @@ k_local_search(const uint32_t* __restrict__ T_sorted, const uint32_t* __restrict
                 const int k = s_ak[a];
                 evaluate(k, x - s_as[a], s_off[k + 1] - s_off[k], best);
             }
-        }
-        // (e) CTA-wide lexicographic minimum: per warp, then every warp reduces the 32 records
-        best = cand_warp_min(best);
-        if (lane == 0) s_cand[warp] = best;
+        };
+        Cand best;
+        best.inv = NO_CAND; best.ik = NO_CAND; best.u1 = NO_CAND; best.pi = -1; best.pu = -1;
+        const long long floor_min = kmin >= 0 ? ((Lmax + s_load[kmin] + 1) >> 1) : Lmax;
+        if (warp == 0) list_clients(floor_min + margin, false);
         __syncthreads();
-        best = cand_warp_min(s_cand[lane]);
+        long long best_v = Lmax;
+        for (int pass = 0; pass < 2; ++pass) {
+            evaluate_listed(best);
+            // CTA-wide lexicographic minimum: per warp, then every warp reduces the 32 records
+            best = cand_warp_min(best);
+            if (lane == 0) s_cand[warp] = best;
+            __syncthreads();
+            best = cand_warp_min(s_cand[lane]);
+            best_v = best.inv != NO_CAND ? Lmax - (long long)(~best.inv) : Lmax;
+            if (pass == 1) break;
+            // is a client that was left out still able to reach best_v?
+            bool missed = false;
+            if (threadIdx.x < n_clients && (int)threadIdx.x != jmax && !s_listed[threadIdx.x]) {
+                const long long lk = s_load[threadIdx.x];
+                missed = lk < Lmax && ((Lmax + lk + 1) >> 1) <= best_v;
+            }
+            if (!__syncthreads_or(missed)) break;
+            if (warp == 0) list_clients(best_v, true);
+            __syncthreads();
+        }
         const bool ok = best.inv != NO_CAND;                    // a candidate always has v < Lmax
         if (!ok) {
             if (threadIdx.x == 0 && log) log[round] = hos_ls_move{-1, -1, -1, Lmax};
             done_at = round;
             break;
         }
+        margin = (best_v - floor_min) + 2;                      // uniform: every thread holds the same best
         const int best_k = (int)(best.ik & 0xFFu);
         const int best_i = (int)(best.ik >> 8);
         const int best_u = (int)best.u1 - 1;
-        const long long best_v = Lmax - (long long)(~best.inv);
-        // (f) apply
+        // (c) apply.  Warp 0 updates the two loads and finds the next round's extremes while the
+        //     other warps patch the member lists (a swap keeps both list lengths).
         const int ri = (int)mem[best.pi];
         const int ru = best.pu >= 0 ? (int)cl[s_off[best_k] + best.pu] : -1;
-        if (best.pu >= 0) {
-            // swap: jmax's list loses ri and gains ru, k's list loses ru and gains ri
-            const bool first = threadIdx.x < SORT_THREADS / 2;
-            IdxT* seg = cl + s_off[first ? jmax : best_k];
+        const uint32_t Ti_w = memT[best.pi];
+        const uint32_t Tu_w = best.pu >= 0 ? clT[s_off[best_k] + best.pu] : 0u;
+        const long long dT = (long long)Ti_w - (long long)Tu_w;
+        ListPatch<IdxT> pp;
+        IdxT* seg = nullptr;
+        uint32_t* segT = nullptr;
+        IdxT keep[4];
+        uint32_t keepT[4];
+        int nk = 0, gtid = 0, val = 0;
+        uint32_t valT = 0;
+        bool big = false;
+        constexpr int GROUP = (SORT_THREADS - 64) / 2;          // threads per list: warps 2..16 and 17..31
+        const bool patcher = best.pu >= 0 && warp >= 2;
+        if (patcher) {
+            const bool first = (int)threadIdx.x - 64 < GROUP;
+            seg = cl + s_off[first ? jmax : best_k];
+            segT = clT + s_off[first ? jmax : best_k];
             const int len = first ? nm : s_off[best_k + 1] - s_off[best_k];
             const int gone = first ? best.pi : best.pu;
-            const int val = first ? ru : ri;
-            const ListPatch<IdxT> pp = patch_plan<IdxT>(seg, len, gone, val);
-            const int tid = threadIdx.x & (SORT_THREADS / 2 - 1);
-            // every thread moves at most ceil(range / 512) elements: read, barrier, write
-            IdxT keep[4];
-            int nk = 0;
-            const int span = pp.dst_hi - pp.dst_lo;
-            const bool big = span > 4 * (SORT_THREADS / 2);     // generic path for very long ranges
+            val = first ? ru : ri;
+            valT = first ? Tu_w : Ti_w;
+            pp = patch_plan<IdxT>(seg, len, gone, val);
+            gtid = ((int)threadIdx.x - 64) % GROUP;
+            big = pp.dst_hi - pp.dst_lo > 4 * GROUP;            // generic path for very long ranges
             if (!big)
-                for (int x = pp.dst_lo + tid; x < pp.dst_hi; x += SORT_THREADS / 2) keep[nk++] = seg[x];
-            __syncthreads();
-            if (!big) {
-                nk = 0;
-                for (int x = pp.dst_lo + tid; x < pp.dst_hi; x += SORT_THREADS / 2) seg[x + pp.shift] = keep[nk++];
-            } else if (tid == 0) {                              // serial shift, direction-safe
-                if (pp.shift < 0) for (int x = pp.dst_lo; x < pp.dst_hi; ++x) seg[x - 1] = seg[x];
-                else for (int x = pp.dst_hi - 1; x >= pp.dst_lo; --x) seg[x + 1] = seg[x];
-            }
-            __syncthreads();
-            if (tid == 0) seg[pp.at] = (IdxT)val;
-        }
-        if (threadIdx.x == 0) {
-            const long long d = (long long)Ts[ri] - (ru >= 0 ? (long long)Ts[ru] : 0ll);
-            bins[ri] = (uint8_t)best_k;
+                for (int x = pp.dst_lo + gtid; x < pp.dst_hi; x += GROUP) { keep[nk] = seg[x]; keepT[nk] = segT[x]; ++nk; }
+        } else if (warp == 0) {
+            if (lane == 0) { s_load[jmax] -= dT; s_load[best_k] += dT; }
+            __syncwarp();
+            find_extremes();
+        } else if (threadIdx.x == 32) {
             asg[best_i] = best_k;
-            if (ru >= 0) { bins[ru] = (uint8_t)jmax; asg[best_u] = jmax; }
-            s_load[jmax] -= d;
-            s_load[best_k] += d;
+            if (ru >= 0) asg[best_u] = jmax;
             if (log) log[round] = hos_ls_move{best_i, best_u, best_k, best_v};
         }
         __syncthreads();
-        if (best.pu < 0) build_member_lists<IdxT>(bins, cl, n_req, n_clients, cnt, s_wsum, s_off);
+        if (patcher) {
+            if (!big) {
+                nk = 0;
+                for (int x = pp.dst_lo + gtid; x < pp.dst_hi; x += GROUP) { seg[x + pp.shift] = keep[nk]; segT[x + pp.shift] = keepT[nk]; ++nk; }
+            } else if (gtid == 0) {                             // serial shift, direction-safe
+                if (pp.shift < 0) for (int x = pp.dst_lo; x < pp.dst_hi; ++x) { seg[x - 1] = seg[x]; segT[x - 1] = segT[x]; }
+                else for (int x = pp.dst_hi - 1; x >= pp.dst_lo; --x) { seg[x + 1] = seg[x]; segT[x + 1] = segT[x]; }
+            }
+            if (gtid == 0) { seg[pp.at] = (IdxT)val; segT[pp.at] = valT; }   // never a destination of the shift
+        }
+        if (threadIdx.x == 0) {
+            bins[ri] = (uint8_t)best_k;
+            if (ru >= 0) bins[ru] = (uint8_t)jmax;
+        }
+        __syncthreads();
+        if (best.pu < 0) build_member_lists<IdxT>(bins, gT, cl, clT, n_req, n_clients, cnt, s_wsum, s_off);
         ++applied;
     }
     // a round without an improving step leaves the state as it is: all later rounds are the same
