@@ -5,7 +5,7 @@
 
 One step is one pass of the whole path over one batch of synthetic instances:
 hos_offline_pack (sort, LPT, local search) -> hos_lower_bound -> hos_online_simulate
-(count pass) -> hos_trace_offsets -> hos_online_simulate (traced pass).  Prints ONE JSON line.
+(with its event log) -> hos_trace_offsets -> hos_trace_fill (the iteration trace).  Prints ONE JSON line.
 With N > 1 (under torchrun) every rank runs the same number of instances with its own seeds
 (weak scaling, no data-path collective); the time is the max over ranks.
 `--impl reference` times the CPU oracle on a bounded sample of the same workload.
@@ -140,14 +140,14 @@ class Pipeline:
         # a multiplier sweep runs its local-search rounds per (instance, multiplier) copy, below
         pk = hos.hos_offline_pack(*self.args(), 0 if sweep else w.ls_rounds, ws=self.ws_off)
         lb = hos.hos_lower_bound(*self.args(), ws=self.ws_off)
-        s1 = hos.hos_online_simulate(*self.args(), pk["assign"], self.lam, hos.HOS_QUEUE_SORTED, ws=self.ws_on)
+        s1 = hos.hos_online_simulate(*self.args(), pk["assign"], self.lam, hos.HOS_QUEUE_SORTED,
+                                     keep_events=True, ws=self.ws_on)
         off = hos.hos_trace_offsets(s1["cres"])
         if self.trace is None:                      # first (warm-up) step sizes the trace buffer
             self.n_iters = int(off[-1].item())
             self.trace = self.torch.empty((max(self.n_iters, 1), 16), dtype=self.torch.uint8, device=self.dev)
-        s2 = hos.hos_online_simulate(*self.args(), pk["assign"], self.lam, hos.HOS_QUEUE_SORTED,
-                                     trace=self.trace, trace_off=off, ws=self.ws_on)
-        self.out = dict(pk=pk, lb=lb, sim=s2, off=off)
+        hos.hos_trace_fill(*self.args(), len(w.lambdas_q16), s1, self.trace, off)
+        self.out = dict(pk=pk, lb=lb, sim=s1, off=off)
         if sweep and w.ls_rounds > 0:
             copies = pk["assign"][:, None, :].expand(-1, len(w.lambdas_q16), -1).contiguous()
             self.out["ls"] = hos.hos_local_search(*self.args(), copies, w.ls_rounds, ws=self.ws_off)
@@ -160,7 +160,7 @@ class Pipeline:
         b = B._batch(*self.args()[:5])
         L = self.hos.lib()
         n_off = L.hos_offline_workspace_bytes(C.byref(b), 1, self.w.ls_rounds)
-        n_on = L.hos_online_workspace_bytes(C.byref(b), len(self.w.lambdas_q16))
+        n_on = L.hos_online_workspace_bytes(C.byref(b), len(self.w.lambdas_q16), 1)
         self.ws_off = self.torch.empty(n_off, dtype=self.torch.uint8, device=self.dev)
         self.ws_on = self.torch.empty(n_on, dtype=self.torch.uint8, device=self.dev)
 
@@ -243,9 +243,10 @@ def algorithmic_bytes(w: Workload, name: str, pipe) -> float:
         return float(executed) * (8 * w.n_req + 8 * w.n_clients)
     if name == "k_simulate":
         n_sims = w.n_inst * len(w.lambdas_q16)
-        # two launches per step (count pass, traced pass): each reads the queue entries and writes
-        # the client results; the traced one also writes the trace -> average per launch
-        return (8.0 * w.n_req * n_sims + 48.0 * n_sims * w.n_clients) + 16.0 * pipe.n_iters / 2
+        # reads the queue entries, writes the client results
+        return 8.0 * w.n_req * n_sims + 48.0 * n_sims * w.n_clients
+    if name == "k_trace_fill":
+        return 16.0 * pipe.n_iters
     if name == "k_finalize":
         return 40.0 * w.n_inst * len(w.lambdas_q16) * w.n_clients
     if name == "k_trace_offsets":
@@ -377,7 +378,7 @@ def run_ours(args):
             "config": {"workload": describe(w), "instances_per_gpu": w.n_inst,
                        "l2": ("inputs larger than L2" if flush is None else "L2 flushed between steps")},
             "sim_iterations_per_step": pipe.n_iters * world,
-            "sim_iterations_per_s": 2 * pipe.n_iters * world * args.steps / (ms * 1e-3),
+            "sim_iterations_per_s": pipe.n_iters * world * args.steps / (ms * 1e-3),
             "clocks": clocks,
             "e2e": {"value": total_inst * args.steps / (ms_e2e * 1e-3), "unit": UNIT,
                     "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,

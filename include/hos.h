@@ -165,14 +165,33 @@ int hos_lower_bound(const hos_batch* batch, const hos_cost_model* cm, hos_lb* ou
  *              unit x = (inst*n_lambda + l)*n_clients + c writes its iterations, in order, to
  *              trace[trace_off[x] .. trace_off[x+1]).  Sizes come from a first call with
  *              trace = NULL (n_prefill_iters + n_decode_iters) and hos_trace_offsets, or from
- *              any upper bound the caller chooses.
+ *              any upper bound the caller chooses.  (With sizes from a first call, hos_trace_fill
+ *              below is the cheaper way to get the trace.)
  *   max_iters  at most this many iterations per client (then HOS_ST_LIMIT).
+ *   keep_events  non-zero: also leave in `ws` the log of the iterations in which something
+ *              changes (prefills and decodes that retire requests; at most two per request),
+ *              from which hos_trace_fill rebuilds the full trace without simulating again.
+ *              Needs the larger workspace of hos_online_workspace_bytes(.., keep_events = 1).
  */
 int hos_online_simulate(const hos_batch* batch, const int32_t* assign, const hos_cost_model* cm,
                         const uint32_t* lambda_q16, int n_lambda, int queue_order, uint32_t max_iters,
                         hos_client_result* cres, hos_sim_result* sres,
                         hos_iter_rec* trace, const int64_t* trace_off, int32_t* status,
-                        void* ws, size_t ws_bytes, void* stream);
+                        int keep_events, void* ws, size_t ws_bytes, void* stream);
+
+/*
+ * The iteration trace from the event log of a hos_online_simulate call made with
+ * keep_events != 0: between two logged iterations a client only decodes, with a constant
+ * batch and sum KV growing by B per iteration, so every record in between follows from the
+ * log (same records, bit for bit, as a traced simulation).  `batch`, `cm`, `n_lambda`, `cres`
+ * and `ws` must be those of that call, and `ws` untouched since.  trace / trace_off as in
+ * hos_online_simulate; status [n_units] gets HOS_ST_TRACE OR-ed in where the slots are too few.
+ * The usual sequence: simulate (trace = NULL, keep_events = 1) -> hos_trace_offsets ->
+ * allocate -> hos_trace_fill.
+ */
+int hos_trace_fill(const hos_batch* batch, const hos_cost_model* cm, int n_lambda,
+                   const hos_client_result* cres, hos_iter_rec* trace, const int64_t* trace_off,
+                   int32_t* status, const void* ws, size_t ws_bytes, void* stream);
 
 /*
  * The lower bounds again, for callers that must not allocate.  (The paper has no counterpart:
@@ -211,7 +230,7 @@ int hos_trace_offsets(const hos_client_result* cres, int64_t n_units, int64_t* t
 
 size_t hos_offline_workspace_bytes(const hos_batch* batch, int n_copies, int ls_rounds);
 size_t hos_lower_bound_workspace_bytes(const hos_batch* batch);
-size_t hos_online_workspace_bytes(const hos_batch* batch, int n_lambda);
+size_t hos_online_workspace_bytes(const hos_batch* batch, int n_lambda, int keep_events);
 
 const char* hos_strerror(int code);
 

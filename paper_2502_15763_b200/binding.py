@@ -31,7 +31,7 @@ ITER_REC_DTYPE = np.dtype([("dur_us", "<u4"), ("kind_n", "<u4"), ("tokens", "<u4
 _SYMBOLS = ("hos_offline_pack", "hos_local_search", "hos_lower_bound", "hos_online_simulate",
             "hos_trace_offsets", "hos_offline_workspace_bytes", "hos_lower_bound_workspace_bytes",
             "hos_online_workspace_bytes", "hos_strerror", "hos_set_launch_hook",
-            "hos_lower_bound_static")
+            "hos_lower_bound_static", "hos_trace_fill")
 
 LAUNCH_HOOK = C.CFUNCTYPE(None, C.c_char_p, C.c_int, C.c_void_p, C.c_void_p)
 
@@ -73,7 +73,7 @@ def lib():
             getattr(L, name).restype = C.c_size_t
         L.hos_strerror.restype = C.c_char_p
         for name in ("hos_offline_pack", "hos_local_search", "hos_lower_bound",
-                     "hos_online_simulate", "hos_trace_offsets", "hos_lower_bound_static"):
+                     "hos_online_simulate", "hos_trace_offsets", "hos_lower_bound_static", "hos_trace_fill"):
             getattr(L, name).restype = C.c_int
         _lib = L
     return _lib
@@ -247,10 +247,11 @@ def hos_trace_offsets(cres, n_units: Optional[int] = None):
 
 def hos_online_simulate(p, o, n_clients: int, batch_cap: int, kv_budget: int, cost_model, assign,
                         lambda_q16, queue_order: int = HOS_QUEUE_SORTED, max_iters: int = 0x7FFFFFFF,
-                        trace=None, trace_off=None, ws=None):
+                        trace=None, trace_off=None, keep_events: bool = False, ws=None):
     """Queues + iteration simulation for every (instance, multiplier, client).
 
     trace: None, or a uint8 tensor [n_records][16] with trace_off (int64 [n_units + 1]).
+    keep_events: leave the event log in the returned workspace `ws` for hos_trace_fill.
     """
     torch = _torch()
     b = _batch(p, o, n_clients, batch_cap, kv_budget)
@@ -261,7 +262,7 @@ def hos_online_simulate(p, o, n_clients: int, batch_cap: int, kv_budget: int, co
     lambda_q16 = _dev(lambda_q16, torch.int32, "lambda_q16")       # uint32 bits
     n_lambda = int(lambda_q16.numel())
     L = lib()
-    need = L.hos_online_workspace_bytes(C.byref(b), C.c_int(n_lambda))
+    need = L.hos_online_workspace_bytes(C.byref(b), C.c_int(n_lambda), C.c_int(int(keep_events)))
     ws = ws if ws is not None else _workspace(need, p)
     dev = p.device
     cres = torch.empty((b.n_inst, n_lambda, n_clients, CLIENT_RESULT_DTYPE.itemsize), dtype=torch.uint8, device=dev)
@@ -274,7 +275,26 @@ def hos_online_simulate(p, o, n_clients: int, batch_cap: int, kv_budget: int, co
             raise ValueError("trace_off must have n_units + 1 entries")
     rc = L.hos_online_simulate(C.byref(b), _ptr(assign), C.byref(cm), _ptr(lambda_q16), C.c_int(n_lambda),
                                C.c_int(queue_order), C.c_uint32(max_iters), _ptr(cres), _ptr(sres),
-                               _ptr(trace), _ptr(trace_off), _ptr(status), _ptr(ws),
+                               _ptr(trace), _ptr(trace_off), _ptr(status), C.c_int(int(keep_events)), _ptr(ws),
                                C.c_size_t(ws.numel()), _stream())
     _check(rc, "hos_online_simulate")
     return dict(cres=cres, sres=sres, status=status, ws=ws)
+
+
+def hos_trace_fill(p, o, n_clients: int, batch_cap: int, kv_budget: int, cost_model, n_lambda: int,
+                   sim, trace, trace_off):
+    """The full iteration trace from the event log of `sim`, the dict returned by
+    hos_online_simulate(..., keep_events=True) for the same batch.  ORs HOS_ST_TRACE into
+    sim["status"] where the slots are too few.  Returns `trace`."""
+    torch = _torch()
+    b = _batch(p, o, n_clients, batch_cap, kv_budget)
+    cm = _cost(cost_model)
+    trace = _dev(trace, torch.uint8, "trace")
+    trace_off = _dev(trace_off, torch.int64, "trace_off")
+    if trace_off.numel() != b.n_inst * n_lambda * n_clients + 1:
+        raise ValueError("trace_off must have n_units + 1 entries")
+    ws = sim["ws"]
+    rc = lib().hos_trace_fill(C.byref(b), C.byref(cm), C.c_int(n_lambda), _ptr(sim["cres"]), _ptr(trace),
+                              _ptr(trace_off), _ptr(sim["status"]), _ptr(ws), C.c_size_t(ws.numel()), _stream())
+    _check(rc, "hos_trace_fill")
+    return trace

@@ -67,9 +67,11 @@ struct OnlineWs {
     int32_t* q_off;
     unsigned long long* inst_O;
     int32_t* inst_status;
+    uint32_t* event_count;      // [n_units]                      (keep_events only)
+    uint4* events;              // [n_sims][n_pad][2 events][2]   (keep_events only)
     size_t bytes;
 };
-OnlineWs carve_online(const hos_batch* b, void* ws) {
+OnlineWs carve_online(const hos_batch* b, void* ws, int n_lambda, int keep_events) {
     OnlineWs w;
     const size_t rows = (size_t)b->n_inst * pad4(b->n_req);
     unsigned char* base = static_cast<unsigned char*>(ws);
@@ -79,6 +81,13 @@ OnlineWs carve_online(const hos_batch* b, void* ws) {
     w.q_off = reinterpret_cast<int32_t*>(base + off);             off += up((size_t)b->n_inst * (b->n_clients + 1) * 4);
     w.inst_O = reinterpret_cast<unsigned long long*>(base + off); off += up((size_t)b->n_inst * 8);
     w.inst_status = reinterpret_cast<int32_t*>(base + off);       off += up((size_t)b->n_inst * 4);
+    w.event_count = nullptr;
+    w.events = nullptr;
+    if (keep_events) {
+        const size_t sims = (size_t)b->n_inst * (size_t)n_lambda;
+        w.event_count = reinterpret_cast<uint32_t*>(base + off);  off += up(sims * b->n_clients * 4);
+        w.events = reinterpret_cast<uint4*>(base + off);          off += up(sims * pad4(b->n_req) * 2 * 32);
+    }
     w.bytes = off;
     return w;
 }
@@ -106,9 +115,9 @@ size_t hos_lower_bound_workspace_bytes(const hos_batch* b) {
     if (!b || b->n_inst < 1 || b->n_req < 1) return 0;
     return carve_offline(b, nullptr).bytes;
 }
-size_t hos_online_workspace_bytes(const hos_batch* b, int /*n_lambda*/) {
-    if (!b || b->n_inst < 1 || b->n_req < 1 || b->n_clients < 1) return 0;
-    return carve_online(b, nullptr).bytes;
+size_t hos_online_workspace_bytes(const hos_batch* b, int n_lambda, int keep_events) {
+    if (!b || b->n_inst < 1 || b->n_req < 1 || b->n_clients < 1 || n_lambda < 1) return 0;
+    return carve_online(b, nullptr, n_lambda, keep_events).bytes;
 }
 
 int hos_offline_pack(const hos_batch* b, const hos_cost_model* cm, int ls_rounds, int32_t* assign,
@@ -177,8 +186,8 @@ int hos_lower_bound(const hos_batch* b, const hos_cost_model* cm, hos_lb* out, i
 int hos_online_simulate(const hos_batch* b, const int32_t* assign, const hos_cost_model* cm,
                         const uint32_t* lambda_q16, int n_lambda, int queue_order, uint32_t max_iters,
                         hos_client_result* cres, hos_sim_result* sres, hos_iter_rec* trace,
-                        const int64_t* trace_off, int32_t* status, void* ws, size_t ws_bytes,
-                        void* stream) {
+                        const int64_t* trace_off, int32_t* status, int keep_events, void* ws,
+                        size_t ws_bytes, void* stream) {
     int rc = check_batch(b);
     if (rc) return rc;
     if ((rc = check_cost(cm, b))) return rc;
@@ -189,8 +198,8 @@ int hos_online_simulate(const hos_batch* b, const int32_t* assign, const hos_cos
     if (bit_width_host((unsigned long long)b->kv_budget) + bit_width_host((unsigned long long)(b->n_clients - 1)) > 32)
         return HOS_E_UNSUPPORTED;
     if ((long long)b->n_inst * n_lambda > 0x7FFFFFFFll / 4) return HOS_E_UNSUPPORTED;
-    if ((rc = check_ws(ws, ws_bytes, hos_online_workspace_bytes(b, n_lambda)))) return rc;
-    const OnlineWs w = carve_online(b, ws);
+    if ((rc = check_ws(ws, ws_bytes, hos_online_workspace_bytes(b, n_lambda, keep_events)))) return rc;
+    const OnlineWs w = carve_online(b, ws, n_lambda, keep_events);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const int n_pad = pad4(b->n_req);
     if (max_iters > 0x7FFFFFFFu) max_iters = 0x7FFFFFFFu;
@@ -199,9 +208,25 @@ int hos_online_simulate(const hos_batch* b, const int32_t* assign, const hos_cos
         return rc;
     if ((rc = cuda_rc(launch_simulate(*b, *cm, lambda_q16, n_lambda, max_iters, w.q_po, w.q_off,
                                       w.inst_status, n_pad, cres, trace,
-                                      reinterpret_cast<const long long*>(trace_off), status, st))))
+                                      reinterpret_cast<const long long*>(trace_off), status, w.events,
+                                      w.event_count, st))))
         return rc;
     return cuda_rc(launch_finalize(*b, n_lambda, w.inst_O, cres, sres, st));
+}
+
+int hos_trace_fill(const hos_batch* b, const hos_cost_model* cm, int n_lambda, const hos_client_result* cres,
+                   hos_iter_rec* trace, const int64_t* trace_off, int32_t* status, const void* ws,
+                   size_t ws_bytes, void* stream) {
+    int rc = check_batch(b);
+    if (rc) return rc;
+    if ((rc = check_cost(cm, b))) return rc;
+    if (!cres || !trace || !trace_off || !status || n_lambda < 1) return HOS_E_INVALID;
+    if ((long long)b->n_inst * n_lambda > 0x7FFFFFFFll / 4) return HOS_E_UNSUPPORTED;
+    if ((rc = check_ws(ws, ws_bytes, hos_online_workspace_bytes(b, n_lambda, 1)))) return rc;
+    const OnlineWs w = carve_online(b, const_cast<void*>(ws), n_lambda, 1);
+    return cuda_rc(launch_trace_fill(*b, *cm, n_lambda, w.q_off, pad4(b->n_req), cres, w.events, w.event_count,
+                                     trace, reinterpret_cast<const long long*>(trace_off), status,
+                                     static_cast<cudaStream_t>(stream)));
 }
 
 int hos_trace_offsets(const hos_client_result* cres, int64_t n_units, int64_t* trace_off, void* stream) {

@@ -38,7 +38,11 @@ cudaError_t launch_simulate(const hos_batch& b, const hos_cost_model& cm, const 
                             int n_lambda, uint32_t max_iters, const uint2* q_po, const int32_t* q_off,
                             const int32_t* inst_status, int n_pad, hos_client_result* cres,
                             hos_iter_rec* trace, const long long* trace_off, int32_t* status,
-                            cudaStream_t st);
+                            uint4* events, uint32_t* event_count, cudaStream_t st);
+cudaError_t launch_trace_fill(const hos_batch& b, const hos_cost_model& cm, int n_lambda,
+                              const int32_t* q_off, int n_pad, const hos_client_result* cres,
+                              const uint4* events, const uint32_t* event_count, hos_iter_rec* trace,
+                              const long long* trace_off, int32_t* status, cudaStream_t st);
 cudaError_t launch_finalize(const hos_batch& b, int n_lambda, const unsigned long long* inst_O,
                             hos_client_result* cres, hos_sim_result* sres, cudaStream_t st);
 cudaError_t launch_trace_offsets(const hos_client_result* cres, long long n_units, long long* trace_off,

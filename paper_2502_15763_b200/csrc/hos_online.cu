@@ -122,7 +122,8 @@ k_simulate(const uint2* __restrict__ q_po, const int32_t* __restrict__ q_off,
            hos_cost_model cm, int q_shift, uint32_t max_iters,
            hos_client_result* __restrict__ cres,
            hos_iter_rec* __restrict__ trace, const long long* __restrict__ trace_off,
-           int32_t* __restrict__ status_out) {
+           int32_t* __restrict__ status_out, uint4* __restrict__ events,
+           uint32_t* __restrict__ event_count) {
     typedef typename E::T entry_t;
     extern __shared__ __align__(16) unsigned char smem_raw[];
     entry_t* heap = reinterpret_cast<entry_t*>(smem_raw) + threadIdx.x;
@@ -139,6 +140,7 @@ k_simulate(const uint2* __restrict__ q_po, const int32_t* __restrict__ q_off,
     if (ist & HOS_ST_INVALID) {
         cres[unit] = hos_client_result{0, 0, 0u, 0u, 0ull, 0.0};
         status_out[unit] = HOS_ST_INVALID;
+        if (event_count) event_count[unit] = 0;
         return;
     }
     const int q0 = q_off[(size_t)inst * (n_clients + 1) + c];
@@ -165,6 +167,9 @@ k_simulate(const uint2* __restrict__ q_po, const int32_t* __restrict__ q_off,
         tr = reinterpret_cast<uint4*>(trace + t0);
         tr_lim = capr > 0x7FFFFFFFll ? 0x7FFFFFFFu : (uint32_t)(capr < 0 ? 0 : capr);
     }
+    // event log of this client: two 16-byte words per logged iteration, at most 2 per request
+    uint4* ev = events ? events + ((size_t)(inst * n_lambda + l) * n_pad + q0) * 4 : nullptr;
+    uint32_t n_ev = 0;
     uint2 nxt = make_uint2(0u, 0u);          // queue entries head + nA and head + nA + 1,
     uint2 nxt2 = make_uint2(0u, 0u);         // fetched ahead of their use
     if (qn > 0) nxt = __ldg(&q[0]);
@@ -273,6 +278,11 @@ k_simulate(const uint2* __restrict__ q_po, const int32_t* __restrict__ q_off,
             }
             r3 = gone_n;
         }
+        if (ev && ((r1 >> 31) || r3 != 0u)) {          // something changed: log it with the state after it
+            ev[2 * n_ev] = make_uint4(n_pre + cnt, B, S, 0u);
+            ev[2 * n_ev + 1] = make_uint4(dur, r1, r2, r3);
+            ++n_ev;
+        }
         emit(dur, r1, r2, r3);
         if (r1 >> 31) { Cd = 0; ++n_pre; }
         else { ++cnt; Cd = min(Cd + dur, 0x7FFFFFFFu); }  // both below 2^31: no wrap
@@ -301,7 +311,65 @@ k_simulate(const uint2* __restrict__ q_po, const int32_t* __restrict__ q_off,
     const uint32_t n_dec = cnt;
     cres[unit] = hos_client_result{t, busy, n_pre, n_dec, hash, 0.0};
     status_out[unit] = status;
+    if (event_count) event_count[unit] = n_ev;
 }
+
+// ---------------------------------------------------------------------------------------
+// Trace from the event log.  One warp per (instance, multiplier, client); a lane per iteration.
+// Iteration `it` belongs to the last logged iteration k with it_k <= it: it is that record
+// itself, or the (it - it_k)-th plain decode after it, with the batch B logged there and
+// sum KV = S_k + (it - it_k - 1) * B.  A chunk of 32 consecutive iterations can only reach the
+// next 32 log entries, so one coalesced load of their iteration numbers and a bit mask place
+// every lane.
+// ---------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(128)
+k_trace_fill(const int32_t* __restrict__ q_off, int n_lambda, int n_clients, int n_pad, long long n_units,
+             hos_cost_model cm, int q_shift, const hos_client_result* __restrict__ cres,
+             const uint4* __restrict__ events, const uint32_t* __restrict__ event_count,
+             hos_iter_rec* __restrict__ trace, const long long* __restrict__ trace_off,
+             int32_t* __restrict__ status_out) {
+    const long long unit = (long long)blockIdx.x * 4 + warp_id();
+    if (unit >= n_units) return;
+    const int lane = lane_id();
+    const int c = (int)(unit % n_clients);
+    const int sim = (int)(unit / n_clients);
+    const int inst = sim / n_lambda;
+    const int q0 = q_off[(size_t)inst * (n_clients + 1) + c];
+    const uint4* ev = events + ((size_t)sim * n_pad + q0) * 4;
+    const uint32_t n_ev = event_count[unit];
+    const uint32_t n_total = cres[unit].n_prefill_iters + cres[unit].n_decode_iters;
+    const long long t0 = trace_off[unit];
+    const long long capr = trace_off[unit + 1] - t0;
+    uint4* tr = reinterpret_cast<uint4*>(trace + t0);
+    const uint32_t lim = capr > (long long)n_total ? n_total : (uint32_t)(capr < 0 ? 0 : capr);
+    if (lane == 0 && (long long)n_total > capr) atomicOr(&status_out[unit], HOS_ST_TRACE);
+    const uint32_t ad = cm.decode_fixed_us, bd = cm.decode_per_seq_us, qd = cm.decode_kv_div;
+
+    uint32_t k_next = 0;                       // log entries before k_next have it < base
+    for (uint32_t base = 0; base < lim; base += 32) {
+        const uint32_t it = base + lane;
+        // iteration numbers of the next 32 log entries
+        const uint32_t kw = k_next + lane;
+        const uint32_t itw = kw < n_ev ? ev[2 * (size_t)kw].x : 0xFFFFFFFFu;
+        const uint32_t dw = itw - base;                                  // >= 0 by construction
+        const uint32_t mask = __reduce_or_sync(FULL, dw < 32u ? (1u << dw) : 0u);
+        const uint32_t upto = mask & (0xFFFFFFFFu >> (31 - lane));       // logged iterations <= it
+        const uint32_t k = k_next + __popc(upto) - 1u;                   // iteration 0 is always logged
+        if (it < lim) {
+            const uint4 st = ev[2 * (size_t)k];
+            uint4 rec;
+            if (st.x == it) rec = ev[2 * (size_t)k + 1];
+            else {
+                const uint32_t Bk = st.y;
+                const uint32_t Sk = st.z + (it - st.x - 1u) * Bk;
+                rec = make_uint4(ad + bd * Bk + (q_shift >= 0 ? (Sk >> q_shift) : (Sk / qd)), Bk, Sk, 0u);
+            }
+            tr[it] = rec;
+        }
+        k_next += __popc(mask);
+    }
+}
+
 
 // ---------------------------------------------------------------------------------------
 // Per-simulation figures: makespan = max over clients, busy = sum, utilisation = busy slot
@@ -403,7 +471,7 @@ cudaError_t launch_simulate(const hos_batch& b, const hos_cost_model& cm, const 
                             int n_lambda, uint32_t max_iters, const uint2* q_po, const int32_t* q_off,
                             const int32_t* inst_status, int n_pad, hos_client_result* cres,
                             hos_iter_rec* trace, const long long* trace_off, int32_t* status,
-                            cudaStream_t st) {
+                            uint4* events, uint32_t* event_count, cudaStream_t st) {
     const long long n_units = (long long)b.n_inst * n_lambda * b.n_clients;
     const unsigned grid = (unsigned)((n_units + SIM_THREADS - 1) / SIM_THREADS);
     int q_shift = -1;                                    // power-of-two KV divisor -> shift
@@ -421,15 +489,31 @@ cudaError_t launch_simulate(const hos_batch& b, const hos_cost_model& cm, const 
     launch_hook("k_simulate", 0, st);
     k_simulate<NarrowEntry><<<grid, SIM_THREADS, smem_n, st>>>(
         q_po, q_off, inst_status, lambda_q16, n_lambda, b.n_clients, n_pad, n_units, b.batch_cap,
-        (uint32_t)b.kv_budget, cm, q_shift, max_iters, cres, trace, trace_off, status);
+        (uint32_t)b.kv_budget, cm, q_shift, max_iters, cres, trace, trace_off, status, events, event_count);
     launch_hook("k_simulate", 1, st);
     if (b.kv_budget >= 65536) {                          // otherwise no p + o can reach 2^16
         launch_hook("k_simulate_wide", 0, st);
         k_simulate<WideEntry><<<grid, SIM_THREADS, smem_w, st>>>(
             q_po, q_off, inst_status, lambda_q16, n_lambda, b.n_clients, n_pad, n_units, b.batch_cap,
-            (uint32_t)b.kv_budget, cm, q_shift, max_iters, cres, trace, trace_off, status);
+            (uint32_t)b.kv_budget, cm, q_shift, max_iters, cres, trace, trace_off, status, events, event_count);
         launch_hook("k_simulate_wide", 1, st);
     }
+    return cudaGetLastError();
+}
+
+cudaError_t launch_trace_fill(const hos_batch& b, const hos_cost_model& cm, int n_lambda,
+                              const int32_t* q_off, int n_pad, const hos_client_result* cres,
+                              const uint4* events, const uint32_t* event_count, hos_iter_rec* trace,
+                              const long long* trace_off, int32_t* status, cudaStream_t st) {
+    const long long n_units = (long long)b.n_inst * n_lambda * b.n_clients;
+    int q_shift = -1;
+    if ((cm.decode_kv_div & (cm.decode_kv_div - 1)) == 0)
+        for (q_shift = 0; (1u << q_shift) != cm.decode_kv_div; ++q_shift) {}
+    launch_hook("k_trace_fill", 0, st);
+    k_trace_fill<<<(unsigned)((n_units + 3) / 4), 128, 0, st>>>(q_off, n_lambda, b.n_clients, n_pad, n_units,
+                                                                cm, q_shift, cres, events, event_count,
+                                                                trace, trace_off, status);
+    launch_hook("k_trace_fill", 1, st);
     return cudaGetLastError();
 }
 

@@ -57,12 +57,14 @@ def check_lower_bound(hos, p, o, M, cap, kv, cm, insts=None):
 
 def gpu_simulate(hos, p, o, M, cap, kv, cm, assign, lambdas, mode, max_iters=0x7FFFFFFF, want_trace=True,
                  trace_slots=None):
-    """Two-pass protocol: counts, offsets, then the traced run.  Returns host-side views."""
+    """Counts (with the event log), offsets, then the trace twice: rebuilt from the event log by
+    hos_trace_fill and written directly by a traced simulation; the two must be the same bytes.
+    Returns host-side views."""
     import torch
     from paper_2502_15763_b200.binding import view_struct
     dp, do, da = to_dev(p), to_dev(o), to_dev(assign)
     dl = to_dev(np.asarray(lambdas, dtype=np.uint32))
-    r = hos.hos_online_simulate(dp, do, M, cap, kv, cm, da, dl, mode, max_iters)
+    r = hos.hos_online_simulate(dp, do, M, cap, kv, cm, da, dl, mode, max_iters, keep_events=want_trace)
     out = dict(cres=view_struct(r["cres"], hos.CLIENT_RESULT_DTYPE),
                sres=view_struct(r["sres"], hos.SIM_RESULT_DTYPE), status=r["status"].cpu().numpy())
     if want_trace:
@@ -79,6 +81,10 @@ def gpu_simulate(hos, p, o, M, cap, kv, cm, assign, lambdas, mode, max_iters=0x7
         for f in out["cres"].dtype.names:
             assert np.array_equal(out["cres"][f], out2["cres"][f]), f"traced run changed cres.{f}"
         out["status_traced"] = out2["status"]
+        filled = torch.zeros_like(trace)
+        hos.hos_trace_fill(dp, do, M, cap, kv, cm, len(lambdas), r, filled, off)
+        assert torch.equal(filled, trace), "trace rebuilt from the event log differs from the traced simulation"
+        assert np.array_equal(r["status"].cpu().numpy(), out2["status"]), "status after hos_trace_fill differs"
         out["trace"] = view_struct(trace, hos.ITER_REC_DTYPE)
         out["trace_off"] = off.cpu().numpy()
     return out
