@@ -298,3 +298,137 @@ void ora_simulate_client(int qn, const int32_t* q_req, const uint32_t* p, const 
     res->status = status;
     free(R);
 }
+
+/* ------------------------------------------------------------------------- */
+/* Algorithm 1, second part: idle clients take the longest request of the     */
+/* client with the most remaining tokens                                      */
+/* ------------------------------------------------------------------------- */
+
+typedef struct {
+    ora_running* R; int nR;
+    int32_t* cand; int nA; int64_t sumP, sumTot;   /* claimed, not yet prefilled */
+    int ustart, qend;                               /* own queue: unclaimed part [ustart, qend) */
+    int64_t remain;                                 /* sum of p+o over the unclaimed part */
+    int head;                                       /* requests prefilled so far */
+    int64_t reserved, t, busy, Cd;
+    uint64_t hash, iters;
+    uint32_t n_pre, n_dec;
+    int32_t status;
+    int finished;
+} ora_cstate;
+
+void ora_simulate_steal(int n, int M, const int32_t* q_off, const int32_t* q_req,
+                        const uint32_t* p, const uint32_t* o, const ora_cost* c, int cap,
+                        int64_t kv_budget, uint32_t lambda_q16, uint32_t max_iters,
+                        ora_client* res, ora_rec** traces, const int64_t* trace_cap,
+                        int32_t* served_by)
+{
+    const int64_t ap = c->prefill_fixed_us, bp = c->prefill_per_token_us;
+    const int64_t ad = c->decode_fixed_us,  bd = c->decode_per_seq_us, q = c->decode_kv_div;
+    ora_cstate* C = (ora_cstate*)calloc((size_t)M, sizeof(ora_cstate));
+    (void)n;
+    for (int j = 0; j < M; ++j) {
+        C[j].R = (ora_running*)malloc(sizeof(ora_running) * (size_t)cap);
+        C[j].cand = (int32_t*)malloc(sizeof(int32_t) * (size_t)cap);
+        C[j].ustart = q_off[j]; C[j].qend = q_off[j + 1];
+        for (int x = q_off[j]; x < q_off[j + 1]; ++x)
+            C[j].remain += (int64_t)p[q_req[x]] + (int64_t)o[q_req[x]];
+        C[j].hash = ORA_HASH_INIT;
+    }
+    for (;;) {
+        /* the unfinished client with the earliest clock, ties to the lower client */
+        int cur = -1;
+        for (int j = 0; j < M; ++j)
+            if (!C[j].finished && (cur < 0 || C[j].t < C[cur].t)) cur = j;
+        if (cur < 0) break;
+        ora_cstate* s = &C[cur];
+
+        /* 1. claim from the own queue: a prefix, no skipping */
+        while (s->ustart < s->qend && s->nR + s->nA < cap) {
+            int i = q_req[s->ustart];
+            int64_t tot = (int64_t)p[i] + (int64_t)o[i];
+            if (s->reserved + s->sumTot + tot > kv_budget) break;
+            s->cand[s->nA++] = i; s->sumTot += tot; s->sumP += p[i];
+            s->ustart += 1; s->remain -= tot;
+            if (served_by) served_by[i] = cur;
+        }
+        /* 1b. own queue exhausted and a slot free: take the longest waiting request of the client
+         *     with the most remaining tokens */
+        if (s->ustart == s->qend) {
+            while (s->nR + s->nA < cap) {
+                int d = -1;
+                for (int j = 0; j < M; ++j)
+                    if (C[j].remain > 0 && (d < 0 || C[j].remain > C[d].remain)) d = j;
+                if (d < 0) break;
+                int i = q_req[C[d].ustart];
+                int64_t tot = (int64_t)p[i] + (int64_t)o[i];
+                if (s->reserved + s->sumTot + tot > kv_budget) break;
+                s->cand[s->nA++] = i; s->sumTot += tot; s->sumP += p[i];
+                C[d].ustart += 1; C[d].remain -= tot;
+                if (served_by) served_by[i] = cur;
+            }
+        }
+        if (s->nR == 0 && s->nA == 0) { s->finished = 1; continue; }   /* nothing left anywhere */
+        if (s->iters == (uint64_t)max_iters) { s->status |= 1; s->finished = 1; continue; }
+
+        /* 2. decide */
+        int64_t Cp = ap + bp * s->sumP;
+        int prefill;
+        if (s->nA == 0) prefill = 0;
+        else if (s->nR == 0) prefill = 1;
+        else prefill = ((uint64_t)lambda_q16 * (uint64_t)s->Cd) > (((uint64_t)Cp) << 16);
+
+        ora_rec rec;
+        int64_t dur;
+        if (prefill) {
+            dur = Cp;
+            s->busy += dur * s->nA;
+            rec.dur_us = (uint32_t)dur; rec.kind_n = 0x80000000u | (uint32_t)s->nA;
+            rec.tokens = (uint32_t)s->sumP; rec.aux = (uint32_t)s->head;
+            for (int a = 0; a < s->nA; ++a) {
+                int i = s->cand[a];
+                s->R[s->nR].kv = p[i]; s->R[s->nR].rem = o[i];
+                s->R[s->nR].total = (int64_t)p[i] + (int64_t)o[i];
+                s->nR += 1;
+            }
+            s->head += s->nA;
+            s->reserved += s->sumTot;
+            s->nA = 0; s->sumP = 0; s->sumTot = 0;
+            s->Cd = 0;
+            s->n_pre += 1;
+        } else {
+            int64_t B = s->nR, S = 0;
+            for (int x = 0; x < s->nR; ++x) S += s->R[x].kv;
+            dur = ad + bd * B + S / q;
+            s->busy += dur * B;
+            int f = 0, w = 0;
+            for (int x = 0; x < s->nR; ++x) {
+                s->R[x].kv += 1; s->R[x].rem -= 1;
+                if (s->R[x].rem == 0) { s->reserved -= s->R[x].total; ++f; }
+                else s->R[w++] = s->R[x];
+            }
+            s->nR = w;
+            s->Cd += dur;
+            if (s->Cd > 2147483647ll) s->Cd = 2147483647ll;
+            rec.dur_us = (uint32_t)dur; rec.kind_n = (uint32_t)B;
+            rec.tokens = (uint32_t)S; rec.aux = (uint32_t)f;
+            s->n_dec += 1;
+        }
+        s->t += dur;
+        if (traces && traces[cur]) {
+            if ((int64_t)s->iters < trace_cap[cur]) traces[cur][s->iters] = rec;
+            else s->status |= 2;
+        }
+        s->hash = (s->hash + (uint64_t)rec.dur_us + ORA_HASH_C1 * rec.kind_n + ORA_HASH_C2 * rec.tokens
+                           + ORA_HASH_C3 * rec.aux) * ORA_HASH_M;
+        s->iters += 1;
+        if (s->t >= ((int64_t)1 << 39)) { s->status |= 1; s->finished = 1; }
+    }
+    for (int j = 0; j < M; ++j) {
+        res[j].makespan_us = C[j].t; res[j].busy_slot_us = C[j].busy;
+        res[j].n_prefill_iters = C[j].n_pre; res[j].n_decode_iters = C[j].n_dec;
+        res[j].trace_hash = C[j].hash; res[j].status = C[j].status;
+        free(C[j].R); free(C[j].cand);
+    }
+    free(C);
+}

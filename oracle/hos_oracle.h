@@ -81,6 +81,18 @@ void ora_simulate_client(int qn, const int32_t* q_req, const uint32_t* p, const 
                          const ora_cost* c, int cap, int64_t kv_budget, uint32_t lambda_q16,
                          uint32_t max_iters, ora_client* res, ora_rec* trace, int64_t trace_cap);
 
+/* The same simulation with Algorithm 1's second part: all M clients of one instance advance in
+ * global time order (earliest clock first, ties to the lower client); a client whose own queue
+ * is exhausted and that still has a free slot takes the head of the queue of the client with
+ * the most queued tokens (ties to the lower client).  q_off/q_req: queues from ora_queue_build.
+ * res [M]; traces [M] (nullable, each with trace_cap[c] slots); served_by [n] (nullable) gets the
+ * client that finally served each request. */
+void ora_simulate_steal(int n, int M, const int32_t* q_off, const int32_t* q_req,
+                        const uint32_t* p, const uint32_t* o, const ora_cost* c, int cap,
+                        int64_t kv_budget, uint32_t lambda_q16, uint32_t max_iters,
+                        ora_client* res, ora_rec** traces, const int64_t* trace_cap,
+                        int32_t* served_by);
+
 #ifdef __cplusplus
 }
 #endif

@@ -217,6 +217,48 @@ def simulate(assign, p, o, M: int, cm, cap: int, kv_budget: int, lambda_q16: int
     return SimResult(makespan, busy, util, tps, clients)
 
 
+def simulate_steal(assign, p, o, M: int, cm, cap: int, kv_budget: int, lambda_q16: int, mode: int,
+                   max_iters: int = 0xFFFFFFFF, want_trace: bool = False):
+    """One (instance, multiplier) simulation with Algorithm 1's request stealing: clients advance
+    in global time order and an idle client takes the longest waiting request of the client with
+    the most queued tokens.  Returns (SimResult, served_by)."""
+    p, o = _u32(p), _u32(o)
+    n = p.shape[0]
+    q_off, q_req = queue_build(assign, p, o, M, mode)
+    cost = _cost(cm)
+    res = (_Client * M)()
+    served = np.full(n, -1, dtype=np.int32)
+
+    def run(traces, caps):
+        tp = (C.c_void_p * M)(*[t.ctypes.data if t is not None else None for t in traces]) if traces else None
+        cp = (C.c_int64 * M)(*caps) if traces else None
+        lib().ora_simulate_steal(
+            C.c_int(n), C.c_int(M), _ptr(q_off, C.c_int32), _ptr(q_req, C.c_int32), _ptr(p, C.c_uint32),
+            _ptr(o, C.c_uint32), C.byref(cost), C.c_int(cap), C.c_int64(kv_budget), C.c_uint32(lambda_q16),
+            C.c_uint32(max_iters), res, tp, cp, _ptr(served, C.c_int32))
+
+    run(None, None)
+    traces = [None] * M
+    if want_trace:
+        caps = [int(r.n_prefill_iters + r.n_decode_iters) for r in res]
+        traces = [np.zeros(max(k, 1), dtype=REC_DTYPE) for k in caps]
+        run(traces, caps)
+        traces = [t[:k] for t, k in zip(traces, caps)]
+    clients = [ClientResult(int(r.makespan_us), int(r.busy_slot_us), int(r.n_prefill_iters),
+                            int(r.n_decode_iters), int(r.trace_hash), int(r.status), traces[j])
+               for j, r in enumerate(res)]
+    makespan = max(c.makespan_us for c in clients)
+    busy = sum(c.busy_slot_us for c in clients)
+    if makespan > 0:
+        for c in clients:
+            c.utilisation = float(c.busy_slot_us) / (float(cap) * float(makespan))
+        util = float(busy) / (float(M) * float(cap) * float(makespan))
+        tps = float(int(o.astype(np.int64).sum())) * 1.0e6 / float(makespan)
+    else:
+        util, tps = 0.0, 0.0
+    return SimResult(makespan, busy, util, tps, clients), served
+
+
 def offline_pack(p, o, M: int, cm, ls_rounds: int = 0):
     """estimate -> order -> LPT -> local search.  Returns dict with T, order, assign, load, ..."""
     T = estimate(p, o, cm)
