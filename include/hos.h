@@ -180,6 +180,25 @@ int hos_online_simulate(const hos_batch* batch, const int32_t* assign, const hos
                         int keep_events, void* ws, size_t ws_bytes, void* stream);
 
 /*
+ * Online scheduling with the second part of Algorithm 1 ("sorting and online preemptive
+ * method"): the clients of an instance are advanced together in global time order (earliest
+ * clock first, ties to the lower client), and a client whose own queue is used up while it
+ * still has a free slot takes the longest waiting request (the head of the queue) of the
+ * client with the most queued tokens, sum of p+o (ties to the lower client), as long as it
+ * fits its KV budget.  A request counts as taken from the moment a client has picked it as a
+ * candidate for its next prefill.  Everything else -- queues, iteration rule, results, trace,
+ * status bits -- is as in hos_online_simulate.
+ *   served_by [n_inst][n_lambda][n_req]  out, nullable: the client that served each request.
+ * Limit of this build: n_clients (rounded up to 32) * batch_cap heap entries of one simulation
+ * must fit one CTA's shared memory (HOS_E_UNSUPPORTED otherwise).
+ */
+int hos_online_simulate_steal(const hos_batch* batch, const int32_t* assign, const hos_cost_model* cm,
+                              const uint32_t* lambda_q16, int n_lambda, int queue_order,
+                              uint32_t max_iters, hos_client_result* cres, hos_sim_result* sres,
+                              hos_iter_rec* trace, const int64_t* trace_off, int32_t* status,
+                              int32_t* served_by, void* ws, size_t ws_bytes, void* stream);
+
+/*
  * The iteration trace from the event log of a hos_online_simulate call made with
  * keep_events != 0: between two logged iterations a client only decodes, with a constant
  * batch and sum KV growing by B per iteration, so every record in between follows from the

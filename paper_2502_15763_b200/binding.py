@@ -31,7 +31,7 @@ ITER_REC_DTYPE = np.dtype([("dur_us", "<u4"), ("kind_n", "<u4"), ("tokens", "<u4
 _SYMBOLS = ("hos_offline_pack", "hos_local_search", "hos_lower_bound", "hos_online_simulate",
             "hos_trace_offsets", "hos_offline_workspace_bytes", "hos_lower_bound_workspace_bytes",
             "hos_online_workspace_bytes", "hos_strerror", "hos_set_launch_hook",
-            "hos_lower_bound_static", "hos_trace_fill")
+            "hos_lower_bound_static", "hos_trace_fill", "hos_online_simulate_steal")
 
 LAUNCH_HOOK = C.CFUNCTYPE(None, C.c_char_p, C.c_int, C.c_void_p, C.c_void_p)
 
@@ -73,7 +73,8 @@ def lib():
             getattr(L, name).restype = C.c_size_t
         L.hos_strerror.restype = C.c_char_p
         for name in ("hos_offline_pack", "hos_local_search", "hos_lower_bound",
-                     "hos_online_simulate", "hos_trace_offsets", "hos_lower_bound_static", "hos_trace_fill"):
+                     "hos_online_simulate", "hos_trace_offsets", "hos_lower_bound_static", "hos_trace_fill",
+                     "hos_online_simulate_steal"):
             getattr(L, name).restype = C.c_int
         _lib = L
     return _lib
@@ -279,6 +280,39 @@ def hos_online_simulate(p, o, n_clients: int, batch_cap: int, kv_budget: int, co
                                C.c_size_t(ws.numel()), _stream())
     _check(rc, "hos_online_simulate")
     return dict(cres=cres, sres=sres, status=status, ws=ws)
+
+
+def hos_online_simulate_steal(p, o, n_clients: int, batch_cap: int, kv_budget: int, cost_model, assign,
+                              lambda_q16, queue_order: int = HOS_QUEUE_SORTED, max_iters: int = 0x7FFFFFFF,
+                              trace=None, trace_off=None, want_served_by: bool = False, ws=None):
+    """hos_online_simulate with Algorithm 1's request stealing between the clients of an instance."""
+    torch = _torch()
+    b = _batch(p, o, n_clients, batch_cap, kv_budget)
+    cm = _cost(cost_model)
+    assign = _dev(assign, torch.int32, "assign")
+    if tuple(assign.shape) != (b.n_inst, b.n_req):
+        raise ValueError("assign must be [n_inst][n_req]")
+    lambda_q16 = _dev(lambda_q16, torch.int32, "lambda_q16")
+    n_lambda = int(lambda_q16.numel())
+    L = lib()
+    need = L.hos_online_workspace_bytes(C.byref(b), C.c_int(n_lambda), C.c_int(0))
+    ws = ws if ws is not None else _workspace(need, p)
+    dev = p.device
+    cres = torch.empty((b.n_inst, n_lambda, n_clients, CLIENT_RESULT_DTYPE.itemsize), dtype=torch.uint8, device=dev)
+    sres = torch.empty((b.n_inst, n_lambda, SIM_RESULT_DTYPE.itemsize), dtype=torch.uint8, device=dev)
+    status = torch.empty((b.n_inst, n_lambda, n_clients), dtype=torch.int32, device=dev)
+    served = torch.empty((b.n_inst, n_lambda, b.n_req), dtype=torch.int32, device=dev) if want_served_by else None
+    if trace is not None:
+        trace = _dev(trace, torch.uint8, "trace")
+        trace_off = _dev(trace_off, torch.int64, "trace_off")
+        if trace_off.numel() != b.n_inst * n_lambda * n_clients + 1:
+            raise ValueError("trace_off must have n_units + 1 entries")
+    rc = L.hos_online_simulate_steal(C.byref(b), _ptr(assign), C.byref(cm), _ptr(lambda_q16), C.c_int(n_lambda),
+                                     C.c_int(queue_order), C.c_uint32(max_iters), _ptr(cres), _ptr(sres),
+                                     _ptr(trace), _ptr(trace_off), _ptr(status), _ptr(served), _ptr(ws),
+                                     C.c_size_t(ws.numel()), _stream())
+    _check(rc, "hos_online_simulate_steal")
+    return dict(cres=cres, sres=sres, status=status, served_by=served, ws=ws)
 
 
 def hos_trace_fill(p, o, n_clients: int, batch_cap: int, kv_budget: int, cost_model, n_lambda: int,

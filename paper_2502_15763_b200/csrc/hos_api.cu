@@ -214,6 +214,40 @@ int hos_online_simulate(const hos_batch* b, const int32_t* assign, const hos_cos
     return cuda_rc(launch_finalize(*b, n_lambda, w.inst_O, cres, sres, st));
 }
 
+int hos_online_simulate_steal(const hos_batch* b, const int32_t* assign, const hos_cost_model* cm,
+                              const uint32_t* lambda_q16, int n_lambda, int queue_order, uint32_t max_iters,
+                              hos_client_result* cres, hos_sim_result* sres, hos_iter_rec* trace,
+                              const int64_t* trace_off, int32_t* status, int32_t* served_by, void* ws,
+                              size_t ws_bytes, void* stream) {
+    int rc = check_batch(b);
+    if (rc) return rc;
+    if ((rc = check_cost(cm, b))) return rc;
+    if (!assign || !lambda_q16 || n_lambda < 1 || !cres || !sres || !status) return HOS_E_INVALID;
+    if (queue_order != HOS_QUEUE_SORTED && queue_order != HOS_QUEUE_FCFS) return HOS_E_INVALID;
+    if (trace && !trace_off) return HOS_E_INVALID;
+    if (queue_build_smem(b->n_req) > SMEM_LIMIT) return HOS_E_UNSUPPORTED;
+    if (bit_width_host((unsigned long long)b->kv_budget) + bit_width_host((unsigned long long)(b->n_clients - 1)) > 32)
+        return HOS_E_UNSUPPORTED;
+    if ((long long)b->n_inst * n_lambda > 0x7FFFFFFFll / 4) return HOS_E_UNSUPPORTED;
+    // every client's heap of one simulation shares a CTA's shared memory
+    const bool may_be_wide = b->kv_budget >= 65536;
+    if (simulate_steal_smem(b->n_clients, b->batch_cap, may_be_wide) + 8 * 1024 > SMEM_LIMIT) return HOS_E_UNSUPPORTED;
+    if ((rc = check_ws(ws, ws_bytes, hos_online_workspace_bytes(b, n_lambda, 0)))) return rc;
+    const OnlineWs w = carve_online(b, ws, n_lambda, 0);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const int n_pad = pad4(b->n_req);
+    if (max_iters > 0x7FFFFFFFu) max_iters = 0x7FFFFFFFu;
+    if ((rc = cuda_rc(launch_queue_build(*b, assign, queue_order, w.q_po, w.q_req, w.q_off, w.inst_O,
+                                         w.inst_status, n_pad, st))))
+        return rc;
+    if ((rc = cuda_rc(launch_simulate_steal(*b, *cm, lambda_q16, n_lambda, max_iters, w.q_po, w.q_req, w.q_off,
+                                            w.inst_status, n_pad, cres, trace,
+                                            reinterpret_cast<const long long*>(trace_off), status, served_by,
+                                            st))))
+        return rc;
+    return cuda_rc(launch_finalize(*b, n_lambda, w.inst_O, cres, sres, st));
+}
+
 int hos_trace_fill(const hos_batch* b, const hos_cost_model* cm, int n_lambda, const hos_client_result* cres,
                    hos_iter_rec* trace, const int64_t* trace_off, int32_t* status, const void* ws,
                    size_t ws_bytes, void* stream) {

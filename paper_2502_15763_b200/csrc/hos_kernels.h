@@ -39,6 +39,12 @@ cudaError_t launch_simulate(const hos_batch& b, const hos_cost_model& cm, const 
                             const int32_t* inst_status, int n_pad, hos_client_result* cres,
                             hos_iter_rec* trace, const long long* trace_off, int32_t* status,
                             uint4* events, uint32_t* event_count, cudaStream_t st);
+size_t simulate_steal_smem(int n_clients, int cap, bool wide);
+cudaError_t launch_simulate_steal(const hos_batch& b, const hos_cost_model& cm, const uint32_t* lambda_q16,
+                                  int n_lambda, uint32_t max_iters, const uint2* q_po, const uint32_t* q_req,
+                                  const int32_t* q_off, const int32_t* inst_status, int n_pad,
+                                  hos_client_result* cres, hos_iter_rec* trace, const long long* trace_off,
+                                  int32_t* status, int32_t* served_by, cudaStream_t st);
 cudaError_t launch_trace_fill(const hos_batch& b, const hos_cost_model& cm, int n_lambda,
                               const int32_t* q_off, int n_pad, const hos_client_result* cres,
                               const uint4* events, const uint32_t* event_count, hos_iter_rec* trace,

@@ -315,6 +315,248 @@ k_simulate(const uint2* __restrict__ q_po, const int32_t* __restrict__ q_off,
 }
 
 // ---------------------------------------------------------------------------------------
+// Simulation with Algorithm 1's request stealing.  One CTA per (instance, multiplier), one
+// thread per client.  Clients advance in global time order (earliest clock first, ties to the
+// lower client); a client whose own queue is used up and that still has a free slot takes the
+// longest waiting request of the client with the most queued tokens.
+//
+// Only a stealing client touches other clients' queues, so iterations that provably start
+// before any steal can happen run side by side, one thread each; the client at the front of
+// the global order runs alone when it might steal (see the horizon H below).  Plain decode
+// iterations claim nothing and commute with everything, so they follow their event iteration
+// at once.
+// ---------------------------------------------------------------------------------------
+template <typename E>
+__global__ void __launch_bounds__(MAX_CLIENTS)
+k_simulate_steal(const uint2* __restrict__ q_po, const uint32_t* __restrict__ q_req,
+                 const int32_t* __restrict__ q_off, const int32_t* __restrict__ inst_status,
+                 const uint32_t* __restrict__ lambda_q16, int n_lambda, int n_clients, int n_req,
+                 int n_pad, int cap, uint32_t kv_budget, hos_cost_model cm, int q_shift,
+                 uint32_t max_iters, hos_client_result* __restrict__ cres,
+                 hos_iter_rec* __restrict__ trace, const long long* __restrict__ trace_off,
+                 int32_t* __restrict__ status_out, int32_t* __restrict__ served_by) {
+    typedef typename E::T entry_t;
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    __shared__ int s_ustart[MAX_CLIENTS];                 // first unclaimed position of each queue
+    __shared__ unsigned long long s_remain[MAX_CLIENTS];  // p+o still unclaimed in each queue
+    __shared__ unsigned long long s_total;                // sum of s_remain
+    __shared__ unsigned long long s_horizon;
+    const int sim = blockIdx.x;
+    const int inst = sim / n_lambda, l = sim % n_lambda;
+    const int c = threadIdx.x;
+    const int stride = blockDim.x;
+    const long long unit = (long long)sim * n_clients + c;
+    const bool is_client = c < n_clients;
+    entry_t* heap = reinterpret_cast<entry_t*>(smem_raw) + c;
+    auto heap_ld = [&](int sl) -> entry_t { return heap[sl * stride]; };
+    auto heap_st = [&](int sl, entry_t v) { heap[sl * stride] = v; };
+
+    const int ist = inst_status[inst];
+    if (((ist & INST_WIDE) != 0) != (sizeof(entry_t) == 8)) return;   // the other instantiation's instance
+    if (ist & HOS_ST_INVALID) {
+        if (is_client) {
+            cres[unit] = hos_client_result{0, 0, 0u, 0u, 0ull, 0.0};
+            status_out[unit] = HOS_ST_INVALID;
+        }
+        if (served_by)
+            for (int i = c; i < n_req; i += stride) served_by[(size_t)sim * n_req + i] = -1;
+        return;
+    }
+    const int32_t* qo = q_off + (size_t)inst * (n_clients + 1);
+    const uint2* q = q_po + (size_t)inst * n_pad;          // all queues of the instance, CSR by client
+    const uint32_t* qr = q_req + (size_t)inst * n_pad;
+    int32_t* served = served_by ? served_by + (size_t)sim * n_req : nullptr;
+    const int qend = is_client ? qo[c + 1] : 0;
+    const uint32_t lam = lambda_q16[l];
+    const uint32_t ap = cm.prefill_fixed_us, bp = cm.prefill_per_token_us;
+    const uint32_t ad = cm.decode_fixed_us, bd = cm.decode_per_seq_us, qd = cm.decode_kv_div;
+
+    if (is_client) {
+        unsigned long long r = 0;
+        for (int x = qo[c]; x < qend; ++x) { const uint2 po = q[x]; r += (unsigned long long)po.x + po.y; }
+        s_ustart[c] = qo[c];
+        s_remain[c] = r;
+    }
+    if (c == 0) { s_total = 0; s_horizon = ~0ull; }
+    if (served)                                           // requests nobody gets to (iteration limit)
+        for (int i = c; i < n_req; i += stride) served[i] = -1;
+    __syncthreads();
+    if (is_client) atomicAdd(&s_total, s_remain[c]);
+
+    long long t = 0, busy = 0;
+    uint32_t Cd = 0, cnt = 0, B = 0, S = 0, reserved = 0, n_pre = 0;
+    uint32_t next_fin = EMPTY, nA = 0, sumP = 0, sumTot = 0, head = 0;
+    unsigned long long hash = HASH_INIT;
+    int32_t status = 0;
+    bool finished = !is_client;
+    uint4* tr = nullptr;
+    uint32_t tr_lim = 0;
+    if (trace && is_client) {
+        const long long t0 = trace_off[unit];
+        const long long capr = trace_off[unit + 1] - t0;
+        tr = reinterpret_cast<uint4*>(trace + t0);
+        tr_lim = capr > 0x7FFFFFFFll ? 0x7FFFFFFFu : (uint32_t)(capr < 0 ? 0 : capr);
+    }
+    auto emit = [&](uint32_t dur, uint32_t r1, uint32_t r2, uint32_t r3) {
+        const uint32_t it = n_pre + cnt;
+        t += dur;
+        hash = (hash + dur + (unsigned long long)HASH_C1 * r1 + (unsigned long long)HASH_C2 * r2 +
+                (unsigned long long)HASH_C3 * r3) * HASH_M;
+        if (it < tr_lim) tr[it] = make_uint4(dur, r1, r2, r3);
+    };
+    // claim the request at position x of some queue as my next candidate, if it fits
+    auto claim = [&](int owner, int x) -> bool {
+        const uint2 po = q[x];
+        const uint32_t tt = po.x + po.y;
+        if (reserved + sumTot + tt > kv_budget) return false;
+        heap_st(cap - 1 - (int)nA, E::make(po.y, tt));
+        sumTot += tt; sumP += po.x; ++nA;
+        s_ustart[owner] = x + 1;
+        s_remain[owner] -= tt;
+        atomicAdd(&s_total, 0ull - (unsigned long long)tt);
+        if (served) served[qr[x]] = c;
+        return true;
+    };
+
+    // No iteration lasts less than d_min, and a client claims at most `cap` requests per iteration,
+    // so a client with u unclaimed own requests cannot use them up -- and so cannot steal -- before
+    // es = clock + (ceil(u / cap) - 1) * d_min.  Nothing is stolen before H = min es over the
+    // unfinished clients, hence every iteration that starts before H only touches its own client
+    // and all of them may run side by side.  When none starts before H, the client that attains H
+    // is at the front of the global order and may steal: it runs alone.
+    const unsigned long long d_min = min((unsigned long long)ap, (unsigned long long)ad + bd);
+    while (true) {
+        __syncthreads();                                   // last step's queue updates are visible
+        const unsigned long long key = ((unsigned long long)t << 9) | (unsigned)c;
+        unsigned long long es_key = ~0ull;
+        if (!finished && s_total > s_remain[c]) {          // somebody else still has queued requests
+            const unsigned long long u = (unsigned long long)(qend - s_ustart[c]);
+            const unsigned long long k = u > (unsigned long long)cap ? (u + cap - 1) / cap - 1 : 0ull;
+            es_key = (((unsigned long long)t + k * d_min) << 9) | (unsigned)c;
+            atomicMin(&s_horizon, es_key);
+        }
+        if (__syncthreads_and(finished)) break;
+        const unsigned long long H = s_horizon;
+        bool run = !finished && key < H;
+        const int ahead = __syncthreads_or(run);           // also orders the read of s_horizon
+        if (!ahead) run = !finished && es_key == H;        // the front of the global order: may steal
+        if (c == 0) s_horizon = ~0ull;                   // for the next step (after the barrier above)
+        if (!run) continue;
+
+        // ---- one iteration of my client (and, for a client that cannot steal, the plain decodes
+        //      that follow that follow it) ----
+        while (s_ustart[c] < qend && B + nA < (uint32_t)cap) {
+            if (!claim(c, s_ustart[c])) break;
+        }
+        if (s_ustart[c] == qend) {
+            while (B + nA < (uint32_t)cap && s_total > 0) {    // only reached when running alone
+                int d = -1;
+                unsigned long long best = 0;
+                for (int j = 0; j < n_clients; ++j)
+                    if (s_remain[j] > best) { best = s_remain[j]; d = j; }
+                if (d < 0 || !claim(d, s_ustart[d])) break;
+            }
+        }
+        if (B == 0 && nA == 0) { finished = true; continue; }
+        if (n_pre + cnt == max_iters) { status |= HOS_ST_LIMIT; finished = true; continue; }
+
+        const uint32_t Cp = ap + bp * sumP;
+        const unsigned long long Cp16 = (unsigned long long)Cp << 16;
+        uint32_t dur, r1, r2, r3;
+        if (nA > 0 && (B == 0 || (unsigned long long)lam * Cd > Cp16)) {
+            for (uint32_t j = 0; j < nA; ++j) {
+                const entry_t x = E::rebase(heap_ld(cap - (int)nA + (int)j), cnt);
+                const entry_t xr = E::rel(x, cnt);
+                uint32_t i = B + j;
+                while (i > 0) {
+                    const uint32_t par = (i - 1) >> 2;
+                    const entry_t y = heap_ld((int)par);
+                    if (E::rel(y, cnt) <= xr) break;
+                    heap_st((int)i, y);
+                    i = par;
+                }
+                heap_st((int)i, x);
+            }
+            dur = Cp; r1 = 0x80000000u | nA; r2 = sumP; r3 = head;
+            busy += (long long)Cp * nA;
+            S += sumP; B += nA; reserved += sumTot; head += nA;
+            nA = 0; sumP = 0; sumTot = 0;
+            next_fin = E::fin(heap_ld(0), cnt);
+        } else {
+            dur = ad + bd * B + (q_shift >= 0 ? (S >> q_shift) : (S / qd));
+            r1 = B; r2 = S; r3 = 0;
+            busy += (long long)dur * B;
+            S += B;
+            if (cnt + 1 == next_fin) {
+                const uint32_t c1 = cnt + 1;
+                uint32_t n = B;
+                do {
+                    const uint32_t gone = E::tot(heap_ld(0));
+                    S -= gone;
+                    reserved -= gone;
+                    ++r3;
+                    --n;
+                    const entry_t x = heap_ld((int)n);
+                    const entry_t xr = E::rel(x, c1);
+                    uint32_t i = 0;
+                    while (true) {
+                        const uint32_t ch = 4 * i + 1;
+                        if (ch >= n) break;
+                        entry_t y0 = heap_ld((int)ch), ym = y0;
+                        entry_t m = E::rel(y0, c1);
+                        uint32_t at = ch;
+#pragma unroll
+                        for (uint32_t k = 1; k < 4; ++k) {
+                            if (ch + k < n) {
+                                const entry_t y = heap_ld((int)(ch + k));
+                                const entry_t r = E::rel(y, c1);
+                                if (r < m) { m = r; ym = y; at = ch + k; }
+                            }
+                        }
+                        if (xr <= m) break;
+                        heap_st((int)i, ym);
+                        i = at;
+                    }
+                    if (n > 0) heap_st((int)i, x);
+                } while (n > 0 && E::fin(heap_ld(0), c1) == c1);
+                B = n;
+                next_fin = n > 0 ? E::fin(heap_ld(0), c1) : EMPTY;
+            }
+        }
+        emit(dur, r1, r2, r3);
+        if (r1 >> 31) { Cd = 0; ++n_pre; }
+        else { ++cnt; Cd = min(Cd + dur, 0x7FFFFFFFu); }
+        if (t >= (1ll << 39)) { status |= HOS_ST_LIMIT; finished = true; continue; }
+        // plain decodes may follow at once while nothing can be claimed: they touch no queue, so
+        // their order against other clients' claims does not matter.  Nothing can be claimed when no
+        // slot is free, or when the own queue is used up and no queue has anything left (s_total
+        // only ever falls, so a zero read here is final).
+        if (B == 0) continue;
+        if (B + nA < (uint32_t)cap && (s_ustart[c] < qend || s_total > 0)) continue;
+        const uint32_t room_t = (uint32_t)(((1ll << 39) - 1 - t) >> 31) + 1u;
+        uint32_t room = min(min(next_fin - cnt - 1u, max_iters - (n_pre + cnt)), room_t);
+        const uint32_t lam_run = nA > 0 ? lam : 0u;
+        const uint32_t base = ad + bd * B;
+        const long long t_run = t;
+        while (room > 0 && (unsigned long long)lam_run * Cd <= Cp16) {
+            const uint32_t dq = base + (q_shift >= 0 ? (S >> q_shift) : (S / qd));
+            emit(dq, B, S, 0u);
+            ++cnt;
+            S += B;
+            Cd = min(Cd + dq, 0x7FFFFFFFu);
+            --room;
+        }
+        busy += (t - t_run) * (long long)B;
+        if (t >= (1ll << 39)) { status |= HOS_ST_LIMIT; finished = true; }
+    }
+    if (is_client) {
+        if (tr && n_pre + cnt > tr_lim) status |= HOS_ST_TRACE;
+        cres[unit] = hos_client_result{t, busy, n_pre, cnt, hash, 0.0};
+        status_out[unit] = status;
+    }
+}
+
+// ---------------------------------------------------------------------------------------
 // Trace from the event log.  One warp per (instance, multiplier, client); a lane per iteration.
 // Iteration `it` belongs to the last logged iteration k with it_k <= it: it is that record
 // itself, or the (it - it_k)-th plain decode after it, with the batch B logged there and
@@ -497,6 +739,42 @@ cudaError_t launch_simulate(const hos_batch& b, const hos_cost_model& cm, const 
             q_po, q_off, inst_status, lambda_q16, n_lambda, b.n_clients, n_pad, n_units, b.batch_cap,
             (uint32_t)b.kv_budget, cm, q_shift, max_iters, cres, trace, trace_off, status, events, event_count);
         launch_hook("k_simulate_wide", 1, st);
+    }
+    return cudaGetLastError();
+}
+
+size_t simulate_steal_smem(int n_clients, int cap, bool wide) {
+    const int threads = (n_clients + 31) & ~31;
+    return (size_t)cap * threads * (wide ? sizeof(unsigned long long) : sizeof(uint32_t));
+}
+
+cudaError_t launch_simulate_steal(const hos_batch& b, const hos_cost_model& cm, const uint32_t* lambda_q16,
+                                  int n_lambda, uint32_t max_iters, const uint2* q_po, const uint32_t* q_req,
+                                  const int32_t* q_off, const int32_t* inst_status, int n_pad,
+                                  hos_client_result* cres, hos_iter_rec* trace, const long long* trace_off,
+                                  int32_t* status, int32_t* served_by, cudaStream_t st) {
+    const int threads = (b.n_clients + 31) & ~31;
+    const unsigned grid = (unsigned)(b.n_inst * n_lambda);
+    int q_shift = -1;
+    if ((cm.decode_kv_div & (cm.decode_kv_div - 1)) == 0)
+        for (q_shift = 0; (1u << q_shift) != cm.decode_kv_div; ++q_shift) {}
+    const size_t smem_n = simulate_steal_smem(b.n_clients, b.batch_cap, false);
+    const size_t smem_w = simulate_steal_smem(b.n_clients, b.batch_cap, true);
+    cudaError_t e = cudaFuncSetAttribute(k_simulate_steal<NarrowEntry>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_n);
+    if (e != cudaSuccess) return e;
+    launch_hook("k_simulate_steal", 0, st);
+    k_simulate_steal<NarrowEntry><<<grid, threads, smem_n, st>>>(
+        q_po, q_req, q_off, inst_status, lambda_q16, n_lambda, b.n_clients, b.n_req, n_pad, b.batch_cap,
+        (uint32_t)b.kv_budget, cm, q_shift, max_iters, cres, trace, trace_off, status, served_by);
+    launch_hook("k_simulate_steal", 1, st);
+    if (b.kv_budget >= 65536) {                          // otherwise no p + o can reach 2^16
+        e = cudaFuncSetAttribute(k_simulate_steal<WideEntry>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_w);
+        if (e != cudaSuccess) return e;
+        launch_hook("k_simulate_steal_wide", 0, st);
+        k_simulate_steal<WideEntry><<<grid, threads, smem_w, st>>>(
+            q_po, q_req, q_off, inst_status, lambda_q16, n_lambda, b.n_clients, b.n_req, n_pad, b.batch_cap,
+            (uint32_t)b.kv_budget, cm, q_shift, max_iters, cres, trace, trace_off, status, served_by);
+        launch_hook("k_simulate_steal_wide", 1, st);
     }
     return cudaGetLastError();
 }

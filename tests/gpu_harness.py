@@ -119,3 +119,46 @@ def check_simulate(hos, p, o, M, cap, kv, cm, assign, lambdas, mode, insts=None,
                     for f in ("dur_us", "kind_n", "tokens", "aux"):
                         assert np.array_equal(gt[f], ec.trace[f]), f"trace.{f} differs: inst {k} lambda {li} client {j}"
     return g
+
+
+def check_simulate_steal(hos, p, o, M, cap, kv, cm, assign, lambdas, mode, insts=None, max_iters=0x7FFFFFFF):
+    """hos_online_simulate_steal (counts, then a traced run with exact slots) against the oracle."""
+    import torch
+    from paper_2502_15763_b200.binding import view_struct
+    dp, do, da = to_dev(p), to_dev(o), to_dev(assign)
+    dl = to_dev(np.asarray(lambdas, dtype=np.uint32))
+    r = hos.hos_online_simulate_steal(dp, do, M, cap, kv, cm, da, dl, mode, max_iters, want_served_by=True)
+    off = hos.hos_trace_offsets(r["cres"])
+    trace = torch.zeros((max(int(off[-1].item()), 1), 16), dtype=torch.uint8, device="cuda")
+    r2 = hos.hos_online_simulate_steal(dp, do, M, cap, kv, cm, da, dl, mode, max_iters, trace=trace, trace_off=off,
+                                       want_served_by=True)
+    assert torch.equal(r["cres"][..., :32], r2["cres"][..., :32]) and torch.equal(r["served_by"], r2["served_by"])
+    cres = view_struct(r2["cres"], hos.CLIENT_RESULT_DTYPE)
+    sres = view_struct(r2["sres"], hos.SIM_RESULT_DTYPE)
+    st = r2["status"].cpu().numpy()
+    served = r2["served_by"].cpu().numpy()
+    tr = view_struct(trace, hos.ITER_REC_DTYPE)
+    toff = off.cpu().numpy()
+    insts = range(p.shape[0]) if insts is None else insts
+    nl = len(lambdas)
+    for k in insts:
+        for li, lam in enumerate(lambdas):
+            e, eserved = ora.simulate_steal(assign[k], p[k], o[k], M, cm, cap, kv, int(lam), mode, max_iters, True)
+            assert np.array_equal(served[k, li], eserved), f"served_by differs: inst {k} lambda {li}"
+            s = sres[k, li]
+            assert int(s["makespan_us"]) == e.makespan_us and int(s["busy_slot_us"]) == e.busy_slot_us
+            assert abs(float(s["utilisation"]) - e.utilisation) <= 1e-9 * abs(e.utilisation)
+            assert abs(float(s["tokens_per_s"]) - e.tokens_per_s) <= 1e-9 * abs(e.tokens_per_s)
+            for j, ec in enumerate(e.clients):
+                c = cres[k, li, j]
+                got = (int(c["makespan_us"]), int(c["busy_slot_us"]), int(c["n_prefill_iters"]),
+                       int(c["n_decode_iters"]), int(c["trace_hash"]), int(st[k, li, j]))
+                want = (ec.makespan_us, ec.busy_slot_us, ec.n_prefill_iters, ec.n_decode_iters, ec.trace_hash,
+                        ec.status)
+                assert got == want, f"client result differs: inst {k} lambda {li} client {j}: {got} != {want}"
+                x = (k * nl + li) * M + j
+                gt = tr[int(toff[x]):int(toff[x + 1])]
+                assert len(gt) == len(ec.trace)
+                for f in ("dur_us", "kind_n", "tokens", "aux"):
+                    assert np.array_equal(gt[f], ec.trace[f]), f"trace.{f} differs: inst {k} lambda {li} client {j}"
+    return dict(cres=cres, sres=sres, status=st, served_by=served)

@@ -151,6 +151,39 @@ def test_long_requests_use_the_wide_heap_entries(hos):
     H.check_simulate(hos, p, o, M, cap, kv, (20000, 40, 15000, 300, 7, 40, 350), g["assign"], LAMS, ora.QUEUE_SORTED)
 
 
+@pytest.mark.parametrize("n,M,cap", [(3, 2, 1), (40, 1, 4), (97, 5, 3), (300, 8, 16), (515, 33, 7), (1000, 64, 40),
+                                     (700, 100, 128)])
+def test_request_stealing(hos, n, M, cap):
+    rng = np.random.default_rng(n * 7 + M)
+    n_inst = 3
+    p = rng.integers(1, 300, size=(n_inst, n)).astype(np.uint32)
+    o = rng.integers(1, 90, size=(n_inst, n)).astype(np.uint32)
+    cm = (20000, 40, 15000, 300, 16, 40, 350)
+    kv = int((p.astype(np.int64) + o).max()) * int(rng.choice([1, 4, 1000]))
+    g = H.gpu_offline(hos, p, o, M, cap, kv, cm, 0)
+    lopsided = np.zeros((n_inst, n), dtype=np.int32)               # everything queued on client 0
+    lopsided[1] = rng.integers(0, max(1, M // 2), size=n)
+    for assign in (g["assign"], lopsided):
+        for mode in (ora.QUEUE_SORTED, ora.QUEUE_FCFS):
+            H.check_simulate_steal(hos, p, o, M, cap, kv, cm, assign, LAMS, mode)
+    H.check_simulate_steal(hos, p, o, M, cap, kv, cm, g["assign"], (LAMBDA_ONE,), ora.QUEUE_SORTED, max_iters=25)
+
+
+def test_request_stealing_config1_and_wide(hos):
+    w = workload("c1")
+    p, o = w.lengths()
+    M, cap, kv, cm = w.n_clients, w.batch_cap, w.kv_budget, w.cost_model
+    g = H.gpu_offline(hos, p, o, M, cap, kv, cm, 0)
+    H.check_simulate_steal(hos, p, o, M, cap, kv, cm, g["assign"], LAMS, ora.QUEUE_SORTED)
+    rr = (np.arange(w.n_req, dtype=np.int32) % M)[None, :]
+    r = H.check_simulate_steal(hos, p, o, M, cap, kv, cm, rr, (LAMBDA_PREFILL_FIRST,), ora.QUEUE_FCFS)
+    plain = H.gpu_simulate(hos, p, o, M, cap, kv, cm, rr, (LAMBDA_PREFILL_FIRST,), ora.QUEUE_FCFS, want_trace=False)
+    assert r["sres"]["makespan_us"][0, 0] <= plain["sres"]["makespan_us"][0, 0]
+    # long requests: the 64-bit heap entries
+    p2 = p.copy(); p2[0, ::50] = 70000
+    H.check_simulate_steal(hos, p2, o, M, cap, 300000, cm, g["assign"], (LAMBDA_ONE,), ora.QUEUE_SORTED)
+
+
 def test_limits_and_bad_data(hos):
     w = workload("c0")
     p, o = w.lengths()
