@@ -345,6 +345,15 @@ def run_ours(args):
         dist.all_reduce(e_t, op=dist.ReduceOp.MAX)
     ms_e2e = float(e_t.item())
 
+    # the widened path: the same batch with Algorithm 1's request stealing between clients
+    steal_ms = None
+    if rank == 0 and not args.skip_steal:
+        run_steal = lambda: hos.hos_online_simulate_steal(*pipe.args(), pipe.out["pk"]["assign"], pipe.lam,
+                                                          hos.HOS_QUEUE_SORTED, ws=pipe.ws_on)
+        run_steal()
+        torch.cuda.synchronize()
+        steal_ms = timed_steps(torch, run_steal, 3, flush) / 3
+
     st = pipe.out
     bad = int((st["pk"]["status"] != 0).sum().item()) + int((st["sim"]["status"] != 0).sum().item())
     if bad:
@@ -387,6 +396,10 @@ def run_ours(args):
             "gpu_launches": int(round(launches * args.steps)),
             "roofline": roofline,
             "kernels": rows,
+            "request_stealing": None if steal_ms is None else {
+                "call": "hos_online_simulate_steal", "ms_per_call": steal_ms,
+                "simulations_per_s": w.n_inst * len(w.lambdas_q16) / (steal_ms * 1e-3),
+                "plain_simulate_ms": rows.get("k_simulate", {}).get("ms_per_launch")},
             "cpu_baseline": {"value": cpu_inst, "unit": UNIT, "cores": 1, "kind": "oracle",
                              "sample": f"first {n_s} instance(s) of the workload, whole path, {cpu_dt:.1f} s",
                              "sim_iterations_per_s": cpu_iters},
@@ -436,6 +449,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--instances", type=int, default=0,
                     help="use only the first N instances of the workload (profiling captures)")
+    ap.add_argument("--skip-steal", action="store_true",
+                    help="do not time the request-stealing simulation (profiling captures)")
     ap.add_argument("--skip-cpu-baseline", action="store_true",
                     help="do not time the CPU oracle (profiling captures)")
     args = ap.parse_args()

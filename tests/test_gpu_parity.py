@@ -184,6 +184,22 @@ def test_request_stealing_config1_and_wide(hos):
     H.check_simulate_steal(hos, p2, o, M, cap, 300000, cm, g["assign"], (LAMBDA_ONE,), ora.QUEUE_SORTED)
 
 
+def test_request_stealing_config4_sampled(hos):
+    w = workload("c4").subset(0, 40)
+    p, o = w.lengths()
+    M, cap, kv, cm = w.n_clients, w.batch_cap, w.kv_budget, w.cost_model
+    g = H.gpu_offline(hos, p, o, M, cap, kv, cm, 0)
+    r = H.check_simulate_steal(hos, p, o, M, cap, kv, cm, g["assign"], w.lambdas_q16, ora.QUEUE_SORTED, insts=(0, 39))
+    plain = H.gpu_simulate(hos, p, o, M, cap, kv, cm, g["assign"], w.lambdas_q16, ora.QUEUE_SORTED, want_trace=False)
+    lb = H.check_lower_bound(hos, p, o, M, cap, kv, cm, insts=(0,))
+    assert (r["status"] == 0).all()
+    assert (lb["lb_sim_us"] <= r["sres"]["makespan_us"][:, 0]).all()
+    # every request is served by exactly one client
+    assert ((r["served_by"] >= 0) & (r["served_by"] < M)).all()
+    # with balanced queues stealing only matters at the very end: it cannot be much worse
+    assert (r["sres"]["makespan_us"][:, 0] <= 1.02 * plain["sres"]["makespan_us"][:, 0]).all()
+
+
 def test_limits_and_bad_data(hos):
     w = workload("c0")
     p, o = w.lengths()
