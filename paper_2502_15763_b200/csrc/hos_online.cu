@@ -340,7 +340,9 @@ k_simulate_steal(const uint2* __restrict__ q_po, const uint32_t* __restrict__ q_
     __shared__ int s_ustart[MAX_CLIENTS];                 // first unclaimed position of each queue
     __shared__ unsigned long long s_remain[MAX_CLIENTS];  // p+o still unclaimed in each queue
     __shared__ unsigned long long s_total;                // sum of s_remain
-    __shared__ unsigned long long s_horizon;
+    __shared__ unsigned long long s_horizon;              // earliest possible steal (conservative bound)
+    __shared__ unsigned long long s_first;                // earliest possible steal (from the dry run)
+    __shared__ unsigned long long s_front;                // earliest unfinished client
     const int sim = blockIdx.x;
     const int inst = sim / n_lambda, l = sim % n_lambda;
     const int c = threadIdx.x;
@@ -377,7 +379,7 @@ k_simulate_steal(const uint2* __restrict__ q_po, const uint32_t* __restrict__ q_
         s_ustart[c] = qo[c];
         s_remain[c] = r;
     }
-    if (c == 0) { s_total = 0; s_horizon = ~0ull; }
+    if (c == 0) { s_total = 0; s_horizon = ~0ull; s_first = ~0ull; s_front = ~0ull; }
     if (served)                                           // requests nobody gets to (iteration limit)
         for (int i = c; i < n_req; i += stride) served[i] = -1;
     __syncthreads();
@@ -404,61 +406,45 @@ k_simulate_steal(const uint2* __restrict__ q_po, const uint32_t* __restrict__ q_
                 (unsigned long long)HASH_C3 * r3) * HASH_M;
         if (it < tr_lim) tr[it] = make_uint4(dur, r1, r2, r3);
     };
-    // claim the request at position x of some queue as my next candidate, if it fits
-    auto claim = [&](int owner, int x) -> bool {
+    // claim the request at position x of some queue as my next candidate, if it fits.  A dry run
+    // keeps its hands off everything the clients share.
+    auto claim = [&](int owner, int x, bool dry) -> bool {
         const uint2 po = q[x];
         const uint32_t tt = po.x + po.y;
         if (reserved + sumTot + tt > kv_budget) return false;
         heap_st(cap - 1 - (int)nA, E::make(po.y, tt));
         sumTot += tt; sumP += po.x; ++nA;
-        s_ustart[owner] = x + 1;
-        s_remain[owner] -= tt;
-        atomicAdd(&s_total, 0ull - (unsigned long long)tt);
-        if (served) served[qr[x]] = c;
+        if (!dry) {
+            s_ustart[owner] = x + 1;
+            s_remain[owner] -= tt;
+            atomicAdd(&s_total, 0ull - (unsigned long long)tt);
+            if (served) served[qr[x]] = c;
+        }
         return true;
     };
+    int u_dry = is_client ? qo[c] : 0;                      // the dry run's own queue position
 
-    // No iteration lasts less than d_min, and a client claims at most `cap` requests per iteration,
-    // so a client with u unclaimed own requests cannot use them up -- and so cannot steal -- before
-    // es = clock + (ceil(u / cap) - 1) * d_min.  Nothing is stolen before H = min es over the
-    // unfinished clients, hence every iteration that starts before H only touches its own client
-    // and all of them may run side by side.  When none starts before H, the client that attains H
-    // is at the front of the global order and may steal: it runs alone.
-    const unsigned long long d_min = min((unsigned long long)ap, (unsigned long long)ad + bd);
-    while (true) {
-        __syncthreads();                                   // last step's queue updates are visible
-        const unsigned long long key = ((unsigned long long)t << 9) | (unsigned)c;
-        unsigned long long es_key = ~0ull;
-        if (!finished && s_total > s_remain[c]) {          // somebody else still has queued requests
-            const unsigned long long u = (unsigned long long)(qend - s_ustart[c]);
-            const unsigned long long k = u > (unsigned long long)cap ? (u + cap - 1) / cap - 1 : 0ull;
-            es_key = (((unsigned long long)t + k * d_min) << 9) | (unsigned)c;
-            atomicMin(&s_horizon, es_key);
+    // One event iteration of my client -- claims (and, when `may_steal`, requests taken from other
+    // queues), the decision, the prefill or decode -- and the plain decodes that follow it while
+    // nothing can be claimed.  Sets `finished` when the client is done or hits a limit.
+    auto advance = [&](bool dry) {
+        int up = dry ? u_dry : s_ustart[c];
+        while (up < qend && B + nA < (uint32_t)cap) {
+            if (!claim(c, up, dry)) break;
+            ++up;
         }
-        if (__syncthreads_and(finished)) break;
-        const unsigned long long H = s_horizon;
-        bool run = !finished && key < H;
-        const int ahead = __syncthreads_or(run);           // also orders the read of s_horizon
-        if (!ahead) run = !finished && es_key == H;        // the front of the global order: may steal
-        if (c == 0) s_horizon = ~0ull;                   // for the next step (after the barrier above)
-        if (!run) continue;
-
-        // ---- one iteration of my client (and, for a client that cannot steal, the plain decodes
-        //      that follow that follow it) ----
-        while (s_ustart[c] < qend && B + nA < (uint32_t)cap) {
-            if (!claim(c, s_ustart[c])) break;
-        }
-        if (s_ustart[c] == qend) {
+        if (dry) u_dry = up;
+        if (!dry && up == qend) {
             while (B + nA < (uint32_t)cap && s_total > 0) {    // only reached when running alone
                 int d = -1;
                 unsigned long long best = 0;
                 for (int j = 0; j < n_clients; ++j)
                     if (s_remain[j] > best) { best = s_remain[j]; d = j; }
-                if (d < 0 || !claim(d, s_ustart[d])) break;
+                if (d < 0 || !claim(d, s_ustart[d], false)) break;
             }
         }
-        if (B == 0 && nA == 0) { finished = true; continue; }
-        if (n_pre + cnt == max_iters) { status |= HOS_ST_LIMIT; finished = true; continue; }
+        if (B == 0 && nA == 0) { finished = true; return; }
+        if (n_pre + cnt == max_iters) { status |= HOS_ST_LIMIT; finished = true; return; }
 
         const uint32_t Cp = ap + bp * sumP;
         const unsigned long long Cp16 = (unsigned long long)Cp << 16;
@@ -526,13 +512,13 @@ k_simulate_steal(const uint2* __restrict__ q_po, const uint32_t* __restrict__ q_
         emit(dur, r1, r2, r3);
         if (r1 >> 31) { Cd = 0; ++n_pre; }
         else { ++cnt; Cd = min(Cd + dur, 0x7FFFFFFFu); }
-        if (t >= (1ll << 39)) { status |= HOS_ST_LIMIT; finished = true; continue; }
+        if (t >= (1ll << 39)) { status |= HOS_ST_LIMIT; finished = true; return; }
         // plain decodes may follow at once while nothing can be claimed: they touch no queue, so
         // their order against other clients' claims does not matter.  Nothing can be claimed when no
         // slot is free, or when the own queue is used up and no queue has anything left (s_total
         // only ever falls, so a zero read here is final).
-        if (B == 0) continue;
-        if (B + nA < (uint32_t)cap && (s_ustart[c] < qend || s_total > 0)) continue;
+        if (B == 0) return;
+        if (B + nA < (uint32_t)cap && ((dry ? u_dry : s_ustart[c]) < qend || s_total > 0)) return;
         const uint32_t room_t = (uint32_t)(((1ll << 39) - 1 - t) >> 31) + 1u;
         uint32_t room = min(min(next_fin - cnt - 1u, max_iters - (n_pre + cnt)), room_t);
         const uint32_t lam_run = nA > 0 ? lam : 0u;
@@ -548,6 +534,48 @@ k_simulate_steal(const uint2* __restrict__ q_po, const uint32_t* __restrict__ q_
         }
         busy += (t - t_run) * (long long)B;
         if (t >= (1ll << 39)) { status |= HOS_ST_LIMIT; finished = true; }
+    };
+
+    // Dry run: every client alone, until the iteration in which it could use up its own queue
+    // (unclaimed requests <= free slots).  As long as nothing has been stolen the real run is these
+    // independent runs, so nothing can be stolen before the earliest such iteration, s_first.
+    {
+        const uint32_t keep_lim = tr_lim;
+        tr_lim = 0;                                         // no trace from the dry run
+        while (!finished && (uint32_t)(qend - u_dry) > (uint32_t)cap - B - nA) advance(true);
+        if (is_client) atomicMin(&s_first, ((unsigned long long)t << 9) | (unsigned)c);
+        tr_lim = keep_lim;
+        t = 0; busy = 0; Cd = 0; cnt = 0; B = 0; S = 0; reserved = 0; n_pre = 0;
+        next_fin = EMPTY; nA = 0; sumP = 0; sumTot = 0; head = 0;
+        hash = HASH_INIT; status = 0; finished = !is_client;
+    }
+
+    // After s_first the conservative bound: no iteration lasts less than d_min and a client claims
+    // at most `cap` requests per iteration, so a client with u unclaimed own requests cannot use
+    // them up -- and so cannot steal -- before es = clock + (ceil(u / cap) - 1) * d_min.  Nothing is
+    // stolen before H = max(s_first, min es over the unfinished clients), hence every iteration that
+    // starts before H only touches its own client and all of them may run side by side.  When none
+    // starts before H, the client at the front of the global order may steal: it runs alone.
+    const unsigned long long d_min = min((unsigned long long)ap, (unsigned long long)ad + bd);
+    while (true) {
+        __syncthreads();                                   // last step's queue updates are visible
+        const unsigned long long key = ((unsigned long long)t << 9) | (unsigned)c;
+        unsigned long long es_key = ~0ull;
+        if (!finished && s_total > s_remain[c]) {          // somebody else still has queued requests
+            const unsigned long long u = (unsigned long long)(qend - s_ustart[c]);
+            const unsigned long long k = u > (unsigned long long)cap ? (u + cap - 1) / cap - 1 : 0ull;
+            es_key = (((unsigned long long)t + k * d_min) << 9) | (unsigned)c;
+            atomicMin(&s_horizon, es_key);
+        }
+        if (!finished) atomicMin(&s_front, key);
+        if (__syncthreads_and(finished)) break;
+        const unsigned long long H = max(s_horizon, s_first);
+        const unsigned long long front = s_front;
+        bool run = !finished && key < H;
+        const int ahead = __syncthreads_or(run);           // also orders the reads of the shared keys
+        if (!ahead) run = !finished && key == front;       // the front of the global order: may steal
+        if (c == 0) { s_horizon = ~0ull; s_front = ~0ull; } // for the next step (after the barrier above)
+        if (run) advance(false);
     }
     if (is_client) {
         if (tr && n_pre + cnt > tr_lim) status |= HOS_ST_TRACE;
