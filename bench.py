@@ -129,6 +129,9 @@ class Pipeline:
         self.trace = None
         self.out = None
         self.n_iters = 0
+        self.copy_stream = None
+        self.chunks = None
+        self.pk_out = None
 
     def args(self):
         w = self.w
@@ -139,19 +142,7 @@ class Pipeline:
         sweep = len(w.lambdas_q16) > 1
         # a multiplier sweep runs its local-search rounds per (instance, multiplier) copy, below
         pk = hos.hos_offline_pack(*self.args(), 0 if sweep else w.ls_rounds, ws=self.ws_off)
-        lb = hos.hos_lower_bound(*self.args(), ws=self.ws_off)
-        s1 = hos.hos_online_simulate(*self.args(), pk["assign"], self.lam, hos.HOS_QUEUE_SORTED,
-                                     keep_events=True, ws=self.ws_on)
-        off = hos.hos_trace_offsets(s1["cres"])
-        if self.trace is None:                      # first (warm-up) step sizes the trace buffer
-            self.n_iters = int(off[-1].item())
-            self.trace = self.torch.empty((max(self.n_iters, 1), 16), dtype=self.torch.uint8, device=self.dev)
-        hos.hos_trace_fill(*self.args(), len(w.lambdas_q16), s1, self.trace, off)
-        self.out = dict(pk=pk, lb=lb, sim=s1, off=off)
-        if sweep and w.ls_rounds > 0:
-            copies = pk["assign"][:, None, :].expand(-1, len(w.lambdas_q16), -1).contiguous()
-            self.out["ls"] = hos.hos_local_search(*self.args(), copies, w.ls_rounds, ws=self.ws_off)
-        return self.out
+        return self.online(pk)
 
     def prepare(self):
         """Workspaces (allocated once; the library itself allocates nothing)."""
@@ -164,20 +155,82 @@ class Pipeline:
         self.ws_off = self.torch.empty(n_off, dtype=self.torch.uint8, device=self.dev)
         self.ws_on = self.torch.empty(n_on, dtype=self.torch.uint8, device=self.dev)
 
+    def online(self, pk):
+        """Lower bound, simulation with event log, trace offsets, trace (and the sweep's local search)."""
+        hos, w = self.hos, self.w
+        lb = hos.hos_lower_bound(*self.args(), ws=self.ws_off)
+        s1 = hos.hos_online_simulate(*self.args(), pk["assign"], self.lam, hos.HOS_QUEUE_SORTED,
+                                     keep_events=True, ws=self.ws_on)
+        off = hos.hos_trace_offsets(s1["cres"])
+        if self.trace is None:                      # first (warm-up) step sizes the trace buffer
+            self.n_iters = int(off[-1].item())
+            self.trace = self.torch.empty((max(self.n_iters, 1), 16), dtype=self.torch.uint8, device=self.dev)
+        hos.hos_trace_fill(*self.args(), len(w.lambdas_q16), s1, self.trace, off)
+        self.out = dict(pk=pk, lb=lb, sim=s1, off=off)
+        if len(w.lambdas_q16) > 1 and w.ls_rounds > 0:
+            copies = pk["assign"][:, None, :].expand(-1, len(w.lambdas_q16), -1).contiguous()
+            self.out["ls"] = hos.hos_local_search(*self.args(), copies, w.ls_rounds, ws=self.ws_off)
+        return self.out
+
     def e2e_step(self, host_out):
-        """The same step from pinned host tables to pinned host results."""
-        self.p.copy_(self.p_host, non_blocking=True)
-        self.o.copy_(self.o_host, non_blocking=True)
-        self.lam.copy_(self.lam_host, non_blocking=True)
-        r = self.step()
-        srcs = (r["pk"]["assign"], r["pk"]["load"], r["pk"]["makespan_est"], r["pk"]["status"],
-                r["lb"]["lb"], r["sim"]["cres"], r["sim"]["sres"], r["sim"]["status"])
-        if not host_out:
-            host_out.extend(self.torch.empty(t.shape, dtype=t.dtype).pin_memory() for t in srcs)
-        for h, d in zip(host_out, srcs):
+        """The same step from pinned host tables to pinned host results.
+
+        The instances are independent, so the offline part runs on a first chunk (two full waves of
+        one-CTA-per-instance kernels) while the rest of the tables are still on their way up,
+        and the offline results go down while the simulation runs; everything is inside the step."""
+        torch, hos, w = self.torch, self.hos, self.w
+        sweep = len(w.lambdas_q16) > 1
+        main = torch.cuda.current_stream()
+        if self.copy_stream is None:
+            self.copy_stream = torch.cuda.Stream()
+            sm = torch.cuda.get_device_properties(self.dev).multi_processor_count
+            # two chunks: a first one of two waves so that little of the upload is exposed, then the
+            # rest (every offline call pays the packing chain's latency once, so few chunks)
+            first = min(w.n_inst, 2 * sm)
+            self.chunks = [(0, first)] + ([(first, w.n_inst - first)] if w.n_inst > first else [])
+            self.pk_out = dict(
+                assign=torch.empty((w.n_inst, w.n_req), dtype=torch.int32, device=self.dev),
+                load=torch.empty((w.n_inst, w.n_clients), dtype=torch.int64, device=self.dev),
+                makespan_est=torch.empty((w.n_inst,), dtype=torch.int64, device=self.dev),
+                rounds_applied=torch.empty((w.n_inst,), dtype=torch.int32, device=self.dev),
+                status=torch.empty((w.n_inst,), dtype=torch.int32, device=self.dev))
+        cs = self.copy_stream
+        cs.wait_stream(main)
+        arrived = []
+        with torch.cuda.stream(cs):
+            self.lam.copy_(self.lam_host, non_blocking=True)
+            for f, n in self.chunks:
+                self.p[f:f + n].copy_(self.p_host[f:f + n], non_blocking=True)
+                self.o[f:f + n].copy_(self.o_host[f:f + n], non_blocking=True)
+                ev = torch.cuda.Event()
+                ev.record(cs)
+                arrived.append(ev)
+        pk = self.pk_out
+        for (f, n), ev in zip(self.chunks, arrived):
+            main.wait_event(ev)
+            hos.hos_offline_pack(self.p[f:f + n], self.o[f:f + n], w.n_clients, w.batch_cap, w.kv_budget,
+                                 w.cost_model, 0 if sweep else w.ls_rounds, ws=self.ws_off,
+                                 out={k: v[f:f + n] for k, v in pk.items()})
+        packed = torch.cuda.Event()
+        packed.record(main)
+        early = (pk["assign"], pk["load"], pk["makespan_est"], pk["status"])
+        r = None
+        if not host_out:                            # first call: run once to learn the result shapes
+            r = self.online(pk)
+            late = (r["lb"]["lb"], r["sim"]["cres"], r["sim"]["sres"], r["sim"]["status"])
+            host_out.extend(torch.empty(t.shape, dtype=t.dtype).pin_memory() for t in early + late)
+        with torch.cuda.stream(cs):                 # offline results go down while the simulation runs
+            cs.wait_event(packed)
+            for h, d in zip(host_out[:4], early):
+                h.copy_(d, non_blocking=True)
+        if r is None:
+            r = self.online(pk)
+        late = (r["lb"]["lb"], r["sim"]["cres"], r["sim"]["sres"], r["sim"]["status"])
+        for h, d in zip(host_out[4:], late):
             h.copy_(d, non_blocking=True)
+        main.wait_stream(cs)
         h2d = sum(t.numel() * t.element_size() for t in (self.p_host, self.o_host, self.lam_host))
-        d2h = sum(t.numel() * t.element_size() for t in srcs)
+        d2h = sum(t.numel() * t.element_size() for t in early + late)
         return h2d, d2h
 
 
@@ -392,7 +445,8 @@ def run_ours(args):
             "e2e": {"value": total_inst * args.steps / (ms_e2e * 1e-3), "unit": UNIT,
                     "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                     "note": "results copied back: assignment, loads, bounds, client and simulation results; "
-                            "the iteration trace stays on the device"},
+                            "the iteration trace stays on the device; uploads and the offline part are pipelined by "
+                            "chunks of instances, offline results go down while the simulation runs"},
             "gpu_launches": int(round(launches * args.steps)),
             "roofline": roofline,
             "kernels": rows,

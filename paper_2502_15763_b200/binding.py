@@ -154,8 +154,11 @@ def view_struct(t, dtype: np.dtype) -> np.ndarray:
 
 
 def hos_offline_pack(p, o, n_clients: int, batch_cap: int, kv_budget: int, cost_model, ls_rounds: int = 0,
-                     want_log: bool = False, ws=None):
-    """Eq. 26-30: estimate, order, LPT, `ls_rounds` local-search rounds.  Returns a dict of tensors."""
+                     want_log: bool = False, ws=None, out=None):
+    """Eq. 26-30: estimate, order, LPT, `ls_rounds` local-search rounds.  Returns a dict of tensors.
+
+    out: optional dict with preallocated 'assign', 'load', 'makespan_est', 'rounds_applied', 'status'
+    (for instance row slices of larger tensors) to write into instead of new tensors."""
     torch = _torch()
     b = _batch(p, o, n_clients, batch_cap, kv_budget)
     cm = _cost(cost_model)
@@ -163,11 +166,21 @@ def hos_offline_pack(p, o, n_clients: int, batch_cap: int, kv_budget: int, cost_
     need = L.hos_offline_workspace_bytes(C.byref(b), C.c_int(1), C.c_int(ls_rounds))
     ws = ws if ws is not None else _workspace(need, p)
     dev = p.device
-    assign = torch.empty((b.n_inst, b.n_req), dtype=torch.int32, device=dev)
-    load = torch.empty((b.n_inst, n_clients), dtype=torch.int64, device=dev)
-    makespan = torch.empty((b.n_inst,), dtype=torch.int64, device=dev)
-    applied = torch.empty((b.n_inst,), dtype=torch.int32, device=dev)
-    status = torch.empty((b.n_inst,), dtype=torch.int32, device=dev)
+    if out is not None:
+        assign = _dev(out["assign"], torch.int32, "out.assign")
+        load = _dev(out["load"], torch.int64, "out.load")
+        makespan = _dev(out["makespan_est"], torch.int64, "out.makespan_est")
+        applied = _dev(out["rounds_applied"], torch.int32, "out.rounds_applied")
+        status = _dev(out["status"], torch.int32, "out.status")
+        if (tuple(assign.shape) != (b.n_inst, b.n_req) or tuple(load.shape) != (b.n_inst, n_clients)
+                or makespan.numel() != b.n_inst or applied.numel() != b.n_inst or status.numel() != b.n_inst):
+            raise ValueError("out tensors do not match the batch")
+    else:
+        assign = torch.empty((b.n_inst, b.n_req), dtype=torch.int32, device=dev)
+        load = torch.empty((b.n_inst, n_clients), dtype=torch.int64, device=dev)
+        makespan = torch.empty((b.n_inst,), dtype=torch.int64, device=dev)
+        applied = torch.empty((b.n_inst,), dtype=torch.int32, device=dev)
+        status = torch.empty((b.n_inst,), dtype=torch.int32, device=dev)
     log = (torch.empty((b.n_inst, ls_rounds, LS_MOVE_DTYPE.itemsize), dtype=torch.uint8, device=dev)
            if want_log and ls_rounds > 0 else None)
     rc = L.hos_offline_pack(C.byref(b), C.byref(cm), C.c_int(ls_rounds), _ptr(assign), _ptr(load),
