@@ -91,7 +91,7 @@ k_queue_build(const uint32_t* __restrict__ p, const uint32_t* __restrict__ o,
 constexpr uint32_t EMPTY = 0xFFFFFFFFu;
 constexpr unsigned long long HASH_INIT = 0xCBF29CE484222325ull;
 constexpr uint32_t HASH_C1 = 0x9E3779B1u, HASH_C2 = 0x85EBCA77u, HASH_C3 = 0xC2B2AE3Du, HASH_M = 0x27D4EB2Fu;
-constexpr int SIM_THREADS = 32;          // one warp per CTA: a warp leaves as soon as its clients are done
+constexpr int SIM_THREADS = 32;          // heap stride: the 32 clients of one warp sit side by side
 
 // Heap entries.  Narrow: (fin mod 2^16) << 16 | tot, usable when every p + o of the instance is
 // below 2^16 (then fin - cnt < 2^16 too, and entries compare correctly after subtracting
@@ -115,7 +115,7 @@ struct WideEntry {
 };
 
 template <typename E>
-__global__ void __launch_bounds__(SIM_THREADS)
+__global__ void __launch_bounds__(1024)
 k_simulate(const uint2* __restrict__ q_po, const int32_t* __restrict__ q_off,
            const int32_t* __restrict__ inst_status, const uint32_t* __restrict__ lambda_q16,
            int n_lambda, int n_clients, int n_pad, long long n_units, int cap, uint32_t kv_budget,
@@ -126,10 +126,11 @@ k_simulate(const uint2* __restrict__ q_po, const int32_t* __restrict__ q_off,
            uint32_t* __restrict__ event_count) {
     typedef typename E::T entry_t;
     extern __shared__ __align__(16) unsigned char smem_raw[];
-    entry_t* heap = reinterpret_cast<entry_t*>(smem_raw) + threadIdx.x;
+    // warps of a CTA are independent; each has its own block of cap * 32 heap entries
+    entry_t* heap = reinterpret_cast<entry_t*>(smem_raw) + (size_t)warp_id() * cap * SIM_THREADS + lane_id();
     auto heap_ld = [&](int sl) -> entry_t { return heap[sl * SIM_THREADS]; };
     auto heap_st = [&](int sl, entry_t v) { heap[sl * SIM_THREADS] = v; };
-    const long long unit = (long long)blockIdx.x * SIM_THREADS + threadIdx.x;
+    const long long unit = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     if (unit >= n_units) return;
     const int c = (int)(unit % n_clients);
     const int l = (int)((unit / n_clients) % n_lambda);
@@ -743,27 +744,47 @@ cudaError_t launch_simulate(const hos_batch& b, const hos_cost_model& cm, const 
                             hos_iter_rec* trace, const long long* trace_off, int32_t* status,
                             uint4* events, uint32_t* event_count, cudaStream_t st) {
     const long long n_units = (long long)b.n_inst * n_lambda * b.n_clients;
-    const unsigned grid = (unsigned)((n_units + SIM_THREADS - 1) / SIM_THREADS);
+    const long long n_warps = (n_units + SIM_THREADS - 1) / SIM_THREADS;
     int q_shift = -1;                                    // power-of-two KV divisor -> shift
     if ((cm.decode_kv_div & (cm.decode_kv_div - 1)) == 0)
         for (q_shift = 0; (1u << q_shift) != cm.decode_kv_div; ++q_shift) {}
     // Both instantiations are launched; each one runs the instances whose entries it can hold and
     // returns at once for the others (the flag is per instance, on the device).
-    const int slots_n = b.batch_cap, slots_w = b.batch_cap;
-    const size_t smem_n = (size_t)slots_n * SIM_THREADS * sizeof(uint32_t);
-    const size_t smem_w = (size_t)slots_w * SIM_THREADS * sizeof(unsigned long long);
+    //
+    // Warps per CTA.  The recurrence is latency-bound and shared memory (one heap per client) limits
+    // the resident warps, so what matters is how many fit at once.  Every CTA costs 1 KB of shared
+    // memory on top of its own: one-warp CTAs free their SM slot as soon as they finish, which is
+    // best over many waves, but when all the work fits the GPU at once only with fewer, larger
+    // CTAs (one per SM), those are used.
+    int n_sm = 148, dev = 0;
+    if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev);
+    auto warps_per_cta = [&](size_t per_warp) {
+        const size_t budget = 227 * 1024, fixed = 1024;
+        const long long small_ctas = (long long)(budget / (per_warp + fixed));
+        const long long cap_small = (long long)n_sm * (small_ctas < 32 ? small_ctas : 32);
+        long long wide = (long long)((budget - fixed) / per_warp);
+        if (wide > 32) wide = 32;
+        if (n_warps > cap_small && wide >= 1 && n_warps <= (long long)n_sm * wide) return (int)wide;
+        return 1;
+    };
+    const size_t warp_n = (size_t)b.batch_cap * SIM_THREADS * sizeof(uint32_t);
+    const size_t warp_w = (size_t)b.batch_cap * SIM_THREADS * sizeof(unsigned long long);
+    const int wpc_n = warps_per_cta(warp_n), wpc_w = warps_per_cta(warp_w);
+    const size_t smem_n = warp_n * wpc_n, smem_w = warp_w * wpc_w;
+    const unsigned grid_n = (unsigned)((n_warps + wpc_n - 1) / wpc_n);
+    const unsigned grid_w = (unsigned)((n_warps + wpc_w - 1) / wpc_w);
     cudaError_t e = cudaFuncSetAttribute(k_simulate<NarrowEntry>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_n);
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(k_simulate<WideEntry>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_w);
     if (e != cudaSuccess) return e;
     launch_hook("k_simulate", 0, st);
-    k_simulate<NarrowEntry><<<grid, SIM_THREADS, smem_n, st>>>(
+    k_simulate<NarrowEntry><<<grid_n, SIM_THREADS * wpc_n, smem_n, st>>>(
         q_po, q_off, inst_status, lambda_q16, n_lambda, b.n_clients, n_pad, n_units, b.batch_cap,
         (uint32_t)b.kv_budget, cm, q_shift, max_iters, cres, trace, trace_off, status, events, event_count);
     launch_hook("k_simulate", 1, st);
     if (b.kv_budget >= 65536) {                          // otherwise no p + o can reach 2^16
         launch_hook("k_simulate_wide", 0, st);
-        k_simulate<WideEntry><<<grid, SIM_THREADS, smem_w, st>>>(
+        k_simulate<WideEntry><<<grid_w, SIM_THREADS * wpc_w, smem_w, st>>>(
             q_po, q_off, inst_status, lambda_q16, n_lambda, b.n_clients, n_pad, n_units, b.batch_cap,
             (uint32_t)b.kv_budget, cm, q_shift, max_iters, cres, trace, trace_off, status, events, event_count);
         launch_hook("k_simulate_wide", 1, st);
