@@ -4,7 +4,7 @@
     python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c0..c4] [--impl ours|reference]
 
 One step is one pass of the whole path over one batch of synthetic instances:
-hos_offline_pack (sort, LPT, local search) -> hos_lower_bound -> hos_online_simulate
+hos_offline_pack (sort, lower bounds, LPT, local search) -> hos_online_simulate
 (with its event log) -> hos_trace_offsets -> hos_trace_fill (the iteration trace).  Prints ONE JSON line.
 With N > 1 (under torchrun) every rank runs the same number of instances with its own seeds
 (weak scaling, no data-path collective); the time is the max over ranks.
@@ -141,7 +141,7 @@ class Pipeline:
         hos, w = self.hos, self.w
         sweep = len(w.lambdas_q16) > 1
         # a multiplier sweep runs its local-search rounds per (instance, multiplier) copy, below
-        pk = hos.hos_offline_pack(*self.args(), 0 if sweep else w.ls_rounds, ws=self.ws_off)
+        pk = hos.hos_offline_pack(*self.args(), 0 if sweep else w.ls_rounds, ws=self.ws_off, want_lb=True)
         return self.online(pk)
 
     def prepare(self):
@@ -158,7 +158,7 @@ class Pipeline:
     def online(self, pk):
         """Lower bound, simulation with event log, trace offsets, trace (and the sweep's local search)."""
         hos, w = self.hos, self.w
-        lb = hos.hos_lower_bound(*self.args(), ws=self.ws_off)
+        lb = dict(lb=pk["lb"])                      # Eq. 31-32 bounds, computed inside hos_offline_pack
         s1 = hos.hos_online_simulate(*self.args(), pk["assign"], self.lam, hos.HOS_QUEUE_SORTED,
                                      keep_events=True, ws=self.ws_on)
         off = hos.hos_trace_offsets(s1["cres"])
@@ -193,7 +193,8 @@ class Pipeline:
                 load=torch.empty((w.n_inst, w.n_clients), dtype=torch.int64, device=self.dev),
                 makespan_est=torch.empty((w.n_inst,), dtype=torch.int64, device=self.dev),
                 rounds_applied=torch.empty((w.n_inst,), dtype=torch.int32, device=self.dev),
-                status=torch.empty((w.n_inst,), dtype=torch.int32, device=self.dev))
+                status=torch.empty((w.n_inst,), dtype=torch.int32, device=self.dev),
+                lb=torch.empty((w.n_inst, 64), dtype=torch.uint8, device=self.dev))
         cs = self.copy_stream
         cs.wait_stream(main)
         arrived = []

@@ -122,11 +122,13 @@ typedef struct hos_iter_rec { uint32_t dur_us, kind_n, tokens, aux; } hos_iter_r
  *   makespan_est   [n_inst]            out  max_j load
  *   rounds_applied [n_inst]            out  local-search rounds that changed the assignment
  *   ls_log         [n_inst][ls_rounds] out, nullable
+ *   lb             [n_inst]            out, nullable: the lower bounds of hos_lower_bound, from the
+ *                                      sort this call does anyway (saves the separate call its own)
  *   status         [n_inst]            out  0 or HOS_ST_INVALID
  */
 int hos_offline_pack(const hos_batch* batch, const hos_cost_model* cm, int ls_rounds,
                      int32_t* assign, int64_t* load, int64_t* makespan_est,
-                     int32_t* rounds_applied, hos_ls_move* ls_log, int32_t* status,
+                     int32_t* rounds_applied, hos_ls_move* ls_log, hos_lb* lb, int32_t* status,
                      void* ws, size_t ws_bytes, void* stream);
 
 /*

@@ -154,11 +154,12 @@ def view_struct(t, dtype: np.dtype) -> np.ndarray:
 
 
 def hos_offline_pack(p, o, n_clients: int, batch_cap: int, kv_budget: int, cost_model, ls_rounds: int = 0,
-                     want_log: bool = False, ws=None, out=None):
+                     want_log: bool = False, ws=None, out=None, want_lb: bool = False):
     """Eq. 26-30: estimate, order, LPT, `ls_rounds` local-search rounds.  Returns a dict of tensors.
 
     out: optional dict with preallocated 'assign', 'load', 'makespan_est', 'rounds_applied', 'status'
-    (for instance row slices of larger tensors) to write into instead of new tensors."""
+    (for instance row slices of larger tensors) to write into instead of new tensors, optionally 'lb'.
+    want_lb: also return the lower bounds (uint8 [n_inst][64]) computed from the same sort."""
     torch = _torch()
     b = _batch(p, o, n_clients, batch_cap, kv_budget)
     cm = _cost(cost_model)
@@ -183,12 +184,17 @@ def hos_offline_pack(p, o, n_clients: int, batch_cap: int, kv_budget: int, cost_
         status = torch.empty((b.n_inst,), dtype=torch.int32, device=dev)
     log = (torch.empty((b.n_inst, ls_rounds, LS_MOVE_DTYPE.itemsize), dtype=torch.uint8, device=dev)
            if want_log and ls_rounds > 0 else None)
+    lb = None
+    if out is not None and out.get("lb") is not None:
+        lb = _dev(out["lb"], torch.uint8, "out.lb")
+    elif want_lb:
+        lb = torch.empty((b.n_inst, LB_DTYPE.itemsize), dtype=torch.uint8, device=dev)
     rc = L.hos_offline_pack(C.byref(b), C.byref(cm), C.c_int(ls_rounds), _ptr(assign), _ptr(load),
-                            _ptr(makespan), _ptr(applied), _ptr(log), _ptr(status), _ptr(ws),
+                            _ptr(makespan), _ptr(applied), _ptr(log), _ptr(lb), _ptr(status), _ptr(ws),
                             C.c_size_t(ws.numel()), _stream())
     _check(rc, "hos_offline_pack")
     return dict(assign=assign, load=load, makespan_est=makespan, rounds_applied=applied, ls_log=log,
-                status=status)
+                lb=lb, status=status)
 
 
 def hos_local_search(p, o, n_clients: int, batch_cap: int, kv_budget: int, cost_model, assign,

@@ -122,7 +122,8 @@ size_t hos_online_workspace_bytes(const hos_batch* b, int n_lambda, int keep_eve
 
 int hos_offline_pack(const hos_batch* b, const hos_cost_model* cm, int ls_rounds, int32_t* assign,
                      int64_t* load, int64_t* makespan_est, int32_t* rounds_applied,
-                     hos_ls_move* ls_log, int32_t* status, void* ws, size_t ws_bytes, void* stream) {
+                     hos_ls_move* ls_log, hos_lb* lb, int32_t* status, void* ws, size_t ws_bytes,
+                     void* stream) {
     int rc = check_batch(b);
     if (rc) return rc;
     if ((rc = check_cost(cm, b))) return rc;
@@ -134,6 +135,7 @@ int hos_offline_pack(const hos_batch* b, const hos_cost_model* cm, int ls_rounds
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const int n_pad = pad4(b->n_req);
     if ((rc = cuda_rc(launch_estimate_sort(*b, *cm, w.T_sorted, w.order, w.info, status, n_pad, st)))) return rc;
+    if (lb && (rc = cuda_rc(launch_lower_bound(*b, *cm, w.T_sorted, w.info, n_pad, lb, st)))) return rc;
     if ((rc = cuda_rc(launch_lpt(*b, w.T_sorted, w.order, w.info, n_pad, assign,
                                  reinterpret_cast<long long*>(load),
                                  reinterpret_cast<long long*>(makespan_est), st))))

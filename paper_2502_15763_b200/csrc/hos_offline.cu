@@ -431,6 +431,37 @@ k_local_search(const uint32_t* __restrict__ T_sorted, const uint32_t* __restrict
         }
         if (lane == 0) { s_jmax = bj; s_lmax = bl; s_kmin = mj; }
     };
+    // warp 0: the clients a round looks at first, with the running count of their work items (see (b))
+    auto list_clients = [&](int jmax, long long Lmax, long long vlimit, bool skip_listed) {
+        int n_alive = 0, n_items = 0;
+        for (int k0 = 0; k0 < n_clients; k0 += 32) {
+            const int k = k0 + lane;
+            bool alive = false;
+            int sz = 0;
+            if (k < n_clients && k != jmax) {
+                const long long lk = s_load[k];
+                alive = lk < Lmax && ((Lmax + lk + 1) >> 1) <= vlimit && !(skip_listed && s_listed[k]);
+                sz = alive ? s_off[k + 1] - s_off[k] + 1 : 0;
+                if (!skip_listed) s_listed[k] = alive;
+                else if (alive) s_listed[k] = 1;
+            }
+            const unsigned am = __ballot_sync(FULL, alive);
+            int inc = sz;
+#pragma unroll
+            for (int d = 1; d < 32; d <<= 1) {
+                const int y = __shfl_up_sync(FULL, inc, d);
+                if (lane >= d) inc += y;
+            }
+            if (alive) {
+                const int pos = n_alive + __popc(am & ((1u << lane) - 1u));
+                s_ak[pos] = (uint8_t)k;
+                s_as[pos] = n_items + inc - sz;
+            }
+            n_alive += __popc(am);
+            n_items += __shfl_sync(FULL, inc, 31);
+        }
+        if (lane == 0) { s_na = n_alive; s_nitems = n_items; }
+    };
     if (warp == 0) find_extremes();
     __syncthreads();
 
@@ -497,36 +528,6 @@ k_local_search(const uint32_t* __restrict__ T_sorted, const uint32_t* __restrict
         //     reduction, any client left out whose floor does not exceed the best v found is
         //     evaluated in a second pass (vlimit = that v), which makes the result exact whatever
         //     the margin was.
-        auto list_clients = [&](long long vlimit, bool skip_listed) {
-            int n_alive = 0, n_items = 0;
-            for (int k0 = 0; k0 < n_clients; k0 += 32) {
-                const int k = k0 + lane;
-                bool alive = false;
-                int sz = 0;
-                if (k < n_clients && k != jmax) {
-                    const long long lk = s_load[k];
-                    alive = lk < Lmax && ((Lmax + lk + 1) >> 1) <= vlimit && !(skip_listed && s_listed[k]);
-                    sz = alive ? s_off[k + 1] - s_off[k] + 1 : 0;
-                    if (!skip_listed) s_listed[k] = alive;
-                    else if (alive) s_listed[k] = 1;
-                }
-                const unsigned am = __ballot_sync(FULL, alive);
-                int inc = sz;
-#pragma unroll
-                for (int d = 1; d < 32; d <<= 1) {
-                    const int y = __shfl_up_sync(FULL, inc, d);
-                    if (lane >= d) inc += y;
-                }
-                if (alive) {
-                    const int pos = n_alive + __popc(am & ((1u << lane) - 1u));
-                    s_ak[pos] = (uint8_t)k;
-                    s_as[pos] = n_items + inc - sz;
-                }
-                n_alive += __popc(am);
-                n_items += __shfl_sync(FULL, inc, 31);
-            }
-            if (lane == 0) { s_na = n_alive; s_nitems = n_items; }
-        };
         auto evaluate_listed = [&](Cand& best) {
             const int n_alive = s_na, n_items = s_nitems;
             for (int x = threadIdx.x; x < n_items; x += SORT_THREADS) {
@@ -542,7 +543,7 @@ k_local_search(const uint32_t* __restrict__ T_sorted, const uint32_t* __restrict
         Cand best;
         best.inv = NO_CAND; best.ik = NO_CAND; best.u1 = NO_CAND; best.pi = -1; best.pu = -1;
         const long long floor_min = kmin >= 0 ? ((Lmax + s_load[kmin] + 1) >> 1) : Lmax;
-        if (warp == 0) list_clients(floor_min + margin, false);
+        if (warp == 0) list_clients(jmax, Lmax, floor_min + margin, false);
         __syncthreads();
         long long best_v = Lmax;
         for (int pass = 0; pass < 2; ++pass) {
@@ -561,7 +562,7 @@ k_local_search(const uint32_t* __restrict__ T_sorted, const uint32_t* __restrict
                 missed = lk < Lmax && ((Lmax + lk + 1) >> 1) <= best_v;
             }
             if (!__syncthreads_or(missed)) break;
-            if (warp == 0) list_clients(best_v, true);
+            if (warp == 0) list_clients(jmax, Lmax, best_v, true);
             __syncthreads();
         }
         const bool ok = best.inv != NO_CAND;                    // a candidate always has v < Lmax

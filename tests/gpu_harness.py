@@ -15,8 +15,11 @@ def to_dev(a, dtype=np.int32):
 
 
 def gpu_offline(hos, p, o, M, cap, kv, cm, ls_rounds):
-    r = hos.hos_offline_pack(to_dev(p), to_dev(o), M, cap, kv, cm, ls_rounds, want_log=True)
-    out = {k: (v.cpu().numpy() if v is not None and k != "ls_log" else v) for k, v in r.items()}
+    r = hos.hos_offline_pack(to_dev(p), to_dev(o), M, cap, kv, cm, ls_rounds, want_log=True, want_lb=True)
+    import torch
+    sep = hos.hos_lower_bound(to_dev(p), to_dev(o), M, cap, kv, cm)
+    assert torch.equal(r["lb"], sep["lb"]), "bounds from hos_offline_pack differ from hos_lower_bound"
+    out = {k: (v.cpu().numpy() if v is not None and k not in ("ls_log", "lb") else v) for k, v in r.items()}
     if r["ls_log"] is not None:
         from paper_2502_15763_b200.binding import view_struct
         out["ls_log"] = view_struct(r["ls_log"], hos.LS_MOVE_DTYPE)

@@ -27,7 +27,7 @@ def test_strerror_and_host_side_validation():
     assert "workspace" in hos.hos_strerror(-2)
     L = hos.lib()
     # null batch is rejected on the host, before any CUDA call
-    assert L.hos_offline_pack(None, None, 0, None, None, None, None, None, None, None, C.c_size_t(0), None) == -1
+    assert L.hos_offline_pack(None, None, 0, None, None, None, None, None, None, None, None, C.c_size_t(0), None) == -1
     assert L.hos_lower_bound(None, None, None, None, None, C.c_size_t(0), None) == -1
     assert L.hos_online_workspace_bytes(None, 1, 0) == 0
 
