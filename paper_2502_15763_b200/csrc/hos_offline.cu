@@ -97,6 +97,11 @@ k_lpt(const uint32_t* __restrict__ T_sorted, const uint32_t* __restrict__ order,
     const bool packed = (span << JB) < 0xFFFFFFFFull;
 
     if (packed) {
+        // Wave form of the chain.  With the keys sorted, s_0 < s_1 < ..., the next items t_0 >= t_1 >= ...
+        // go to s_0, s_1, ... one each for as long as s_a is still below every updated key
+        // s_b + t_b, b < a: exactly what the one-by-one rule does, found for up to 32 items at once by
+        // one sort of the keys (bitonic, across the warp) and one prefix minimum.  Keys carry their
+        // client in the low bits, so they may sit in any lane.
         uint32_t key[KPL];
 #pragma unroll
         for (int k = 0; k < KPL; ++k) {
@@ -115,17 +120,56 @@ k_lpt(const uint32_t* __restrict__ T_sorted, const uint32_t* __restrict__ order,
             rq_next = (rn < n_req) ? od[rn] : 0u;
             const int steps = min(32, n_req - r0);
             uint32_t mine = 0;
-            for (int sidx = 0; sidx < steps; ++sidx) {
-                uint32_t m = key[0];
+            int pos = 0;
+            while (pos < steps) {
+                // sort all 32 * KPL keys ascending: element e = k * 32 + lane
 #pragma unroll
-                for (int k = 1; k < KPL; ++k) m = min(m, key[k]);
-                const uint32_t g = __reduce_min_sync(FULL, m);
-                const uint32_t j = g & ((1u << JB) - 1u);
-                const uint32_t t = __shfl_sync(FULL, tsh, sidx);
-                const bool own = lane == (int)(j & 31u);
+                for (int size = 2; size <= 32 * KPL; size <<= 1) {
 #pragma unroll
-                for (int k = 0; k < KPL; ++k) key[k] += (own && (int)(j >> 5) == k) ? t : 0u;
-                mine = (lane == sidx) ? j : mine;
+                    for (int stride = size >> 1; stride > 0; stride >>= 1) {
+                        if (stride < 32) {
+#pragma unroll
+                            for (int k = 0; k < KPL; ++k) {
+                                const uint32_t other = __shfl_xor_sync(FULL, key[k], stride);
+                                const bool up = ((k * 32 + lane) & size) == 0;
+                                const bool lower = (lane & stride) == 0;
+                                key[k] = (lower == up) ? min(key[k], other) : max(key[k], other);
+                            }
+                        } else {
+                            const int kk = stride >> 5;
+#pragma unroll
+                            for (int k = 0; k < KPL; ++k) {
+                                if ((k & kk) == 0) {
+                                    const uint32_t a = key[k], b = key[k | kk];
+                                    const bool up = ((k * 32) & size) == 0;
+                                    key[k] = up ? min(a, b) : max(a, b);
+                                    key[k | kk] = up ? max(a, b) : min(a, b);
+                                }
+                            }
+                        }
+                    }
+                }
+                // lane a now holds the a-th smallest key in key[0]; item pos + a is its candidate
+                const int src = pos + lane;
+                const bool have = src < steps;
+                const uint32_t t = __shfl_sync(FULL, tsh, src & 31);
+                const uint32_t s_a = key[0];
+                const uint32_t u_a = s_a + (have ? t : 0u);
+                uint32_t inc = u_a;
+#pragma unroll
+                for (int d = 1; d < 32; d <<= 1) {
+                    const uint32_t y = __shfl_up_sync(FULL, inc, d);
+                    if (lane >= d) inc = min(inc, y);
+                }
+                uint32_t before = __shfl_up_sync(FULL, inc, 1);     // min of the updated keys of lower lanes
+                if (lane == 0) before = 0xFFFFFFFFu;
+                const bool ok = have && s_a != 0xFFFFFFFFu && (lane == 0 || s_a < before);
+                const unsigned okm = __ballot_sync(FULL, ok);
+                const int W = (okm == FULL) ? 32 : (__ffs(~okm) - 1);  // >= 1: lane 0 always qualifies
+                if (lane < W) key[0] = u_a;
+                const uint32_t jv = __shfl_sync(FULL, s_a & ((1u << JB) - 1u), (lane - pos) & 31);
+                if (lane >= pos && lane < pos + W) mine = jv;
+                pos += W;
             }
             if (r < n_req) asg[rq] = (int32_t)mine;
             // re-base: subtract the current least relative load from every real key
@@ -136,11 +180,20 @@ k_lpt(const uint32_t* __restrict__ T_sorted, const uint32_t* __restrict__ order,
             rebased += base >> JB;
 #pragma unroll
             for (int k = 0; k < KPL; ++k)
-                if (k * 32 + lane < n_clients) key[k] -= base;
+                if (key[k] != 0xFFFFFFFFu) key[k] -= base;
         }
+        long long mx = 0;
 #pragma unroll
-        for (int k = 0; k < KPL; ++k)
-            if (k * 32 + lane < n_clients) load[k] = (long long)(rebased + (key[k] >> JB));
+        for (int k = 0; k < KPL; ++k) {
+            if (key[k] != 0xFFFFFFFFu) {
+                const long long l = (long long)(rebased + (key[k] >> JB));
+                load_out[(size_t)inst * n_clients + (key[k] & ((1u << JB) - 1u))] = l;
+                mx = l > mx ? l : mx;
+            }
+        }
+        mx = warp_max_i64(mx);
+        if (lane == 0) makespan_out[inst] = mx;
+        return;
     } else {
         for (int r0 = 0; r0 < n_req; r0 += 32) {
             const int r = r0 + lane;
