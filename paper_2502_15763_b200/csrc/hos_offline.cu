@@ -538,11 +538,12 @@ k_local_search(const uint32_t* __restrict__ T_sorted, const uint32_t* __restrict
                 const int at = s_off[k] + idx;
                 u1 = (uint32_t)ord[cl[at]] + 1u; pu = idx; Tu = clT[at];
             }
-            const long long thr = Tu + ((slack + 1) >> 1);      // T_i >= thr  <=>  2 d >= slack
-            int a = 0, z = nm;                                  // b = members with T >= thr
-            while (a < z) {
+            const long long thr64 = Tu + ((slack + 1) >> 1);    // T_i >= thr  <=>  2 d >= slack
+            const uint32_t thr = (uint32_t)thr64;
+            int a = 0, z = thr64 > 0xFFFFFFFFll ? 0 : nm;       // b = members with T >= thr (none if it
+            while (a < z) {                                     // is beyond every T)
                 const int mid = (a + z) >> 1;
-                if ((long long)memT[mid] >= thr) a = mid + 1; else z = mid;
+                if (memT[mid] >= thr) a = mid + 1; else z = mid;
             }
             const int b = a;
             if (b > 0) {                                        // rising side: smallest T >= thr
