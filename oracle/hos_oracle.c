@@ -128,10 +128,25 @@ int ora_local_search(int n, int M, const int64_t* T, int32_t* assign, int64_t* l
 
 static int64_t ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
 
+/* Duration of a prefill stage over `tokens` prompt tokens: affine, or by level (Eq. 5-7). */
+static int64_t prefill_us(const ora_cost* c, int64_t tokens)
+{
+    if (c->n_levels == 0)
+        return (int64_t)c->prefill_fixed_us + (int64_t)c->prefill_per_token_us * tokens;
+    for (uint32_t l = 0; l < c->n_levels; ++l)
+        if (tokens <= (int64_t)c->level_cap[l]) return (int64_t)c->level_time[l];
+    return (int64_t)c->level_time[c->n_levels - 1];        /* not reached: admission stops at the largest level */
+}
+
+/* Does a prefill stage that already holds `have` tokens take `more` on top?  (largest level's capacity) */
+static int stage_holds(const ora_cost* c, int64_t have, int64_t more)
+{
+    return c->n_levels == 0 || have + more <= (int64_t)c->level_cap[c->n_levels - 1];
+}
+
 void ora_lower_bound(int n, int M, int cap, const uint32_t* p, const uint32_t* o,
                      const ora_cost* c, ora_lb* out)
 {
-    const int64_t ap = c->prefill_fixed_us, bp = c->prefill_per_token_us;
     const int64_t ad = c->decode_fixed_us,  bd = c->decode_per_seq_us, q = c->decode_kv_div;
 
     /* --- packing bound: the optimum of Eq. 26 is at least the mean load, the largest
@@ -154,15 +169,31 @@ void ora_lower_bound(int n, int M, int cap, const uint32_t* p, const uint32_t* o
     for (int i = 0; i < n; ++i) {
         P += p[i];
         O += o[i];
-        int64_t alone = ap + bp * (int64_t)p[i];    /* request i served alone on a client */
+        int64_t alone = prefill_us(c, p[i]);        /* request i served alone on a client */
         for (int64_t s = 0; s < (int64_t)o[i]; ++s) {
             K += (int64_t)p[i] + s;                 /* KV tokens attended by decode step s */
             alone += ad + bd + ((int64_t)p[i] + s) / q;
         }
         if (alone > chain) chain = alone;
     }
-    /* every prefill iteration admits at most cap prompts and pays a_p once */
-    int64_t tp_star = ap * ceil_div(n, cap) + bp * P;
+    int64_t tp_star, tp_paper = 0;
+    if (c->n_levels == 0) {
+        /* every prefill iteration admits at most cap prompts and pays a_p once */
+        tp_star = (int64_t)c->prefill_fixed_us * ceil_div(n, cap) + (int64_t)c->prefill_per_token_us * P;
+    } else {
+        /* by level: at least ceil(n/cap) stages of at least the smallest level's time; and a stage
+         * of level l carries at most N^cap_l tokens, so the P tokens cost at least
+         * min_l floor(P / N^cap_l) T^p_l.  Eq. 31 as printed takes l = L only. */
+        int64_t by_count = (int64_t)c->level_time[0] * ceil_div(n, cap);
+        int64_t by_tokens = -1;
+        for (uint32_t l = 0; l < c->n_levels; ++l) {
+            int64_t v = (P / (int64_t)c->level_cap[l]) * (int64_t)c->level_time[l];
+            if (by_tokens < 0 || v < by_tokens) by_tokens = v;
+        }
+        tp_star = by_count > by_tokens ? by_count : by_tokens;
+        tp_paper = (P / (int64_t)c->level_cap[c->n_levels - 1]) * (int64_t)c->level_time[c->n_levels - 1];
+    }
+    out->tp_paper_us = tp_paper;
     /* every decode iteration advances at most cap requests; floor(S/q) > S/q - 1 */
     int64_t td_q = q * ((ad - 1) * ceil_div(O, cap) + bd * O) + K;      /* q * t^d*  */
     int64_t work = ceil_div(q * tp_star + td_q, q * (int64_t)M);        /* mean client time */
@@ -213,7 +244,6 @@ void ora_simulate_client(int qn, const int32_t* q_req, const uint32_t* p, const 
                          const ora_cost* c, int cap, int64_t kv_budget, uint32_t lambda_q16,
                          uint32_t max_iters, ora_client* res, ora_rec* trace, int64_t trace_cap)
 {
-    const int64_t ap = c->prefill_fixed_us, bp = c->prefill_per_token_us;
     const int64_t ad = c->decode_fixed_us,  bd = c->decode_per_seq_us, q = c->decode_kv_div;
 
     ora_running* R = (ora_running*)malloc(sizeof(ora_running) * (size_t)(cap > 0 ? cap : 1));
@@ -233,11 +263,12 @@ void ora_simulate_client(int qn, const int32_t* q_req, const uint32_t* p, const 
             int i = q_req[head + nA];
             int64_t tot = (int64_t)p[i] + (int64_t)o[i];
             if (reserved + sumTot + tot > kv_budget) break;
+            if (!stage_holds(c, sumP, p[i])) break;
             sumTot += tot; sumP += p[i]; ++nA;
         }
         /* 2. decide */
         int prefill;
-        int64_t Cp = ap + bp * sumP;
+        int64_t Cp = prefill_us(c, sumP);
         if (nA == 0) prefill = 0;
         else if (nR == 0) prefill = 1;
         else prefill = ((uint64_t)lambda_q16 * (uint64_t)Cd) > (((uint64_t)Cp) << 16);
@@ -323,7 +354,6 @@ void ora_simulate_steal(int n, int M, const int32_t* q_off, const int32_t* q_req
                         ora_client* res, ora_rec** traces, const int64_t* trace_cap,
                         int32_t* served_by)
 {
-    const int64_t ap = c->prefill_fixed_us, bp = c->prefill_per_token_us;
     const int64_t ad = c->decode_fixed_us,  bd = c->decode_per_seq_us, q = c->decode_kv_div;
     ora_cstate* C = (ora_cstate*)calloc((size_t)M, sizeof(ora_cstate));
     (void)n;
@@ -348,6 +378,7 @@ void ora_simulate_steal(int n, int M, const int32_t* q_off, const int32_t* q_req
             int i = q_req[s->ustart];
             int64_t tot = (int64_t)p[i] + (int64_t)o[i];
             if (s->reserved + s->sumTot + tot > kv_budget) break;
+            if (!stage_holds(c, s->sumP, p[i])) break;
             s->cand[s->nA++] = i; s->sumTot += tot; s->sumP += p[i];
             s->ustart += 1; s->remain -= tot;
             if (served_by) served_by[i] = cur;
@@ -363,6 +394,7 @@ void ora_simulate_steal(int n, int M, const int32_t* q_off, const int32_t* q_req
                 int i = q_req[C[d].ustart];
                 int64_t tot = (int64_t)p[i] + (int64_t)o[i];
                 if (s->reserved + s->sumTot + tot > kv_budget) break;
+                if (!stage_holds(c, s->sumP, p[i])) break;
                 s->cand[s->nA++] = i; s->sumTot += tot; s->sumP += p[i];
                 C[d].ustart += 1; C[d].remain -= tot;
                 if (served_by) served_by[i] = cur;
@@ -372,7 +404,7 @@ void ora_simulate_steal(int n, int M, const int32_t* q_off, const int32_t* q_req
         if (s->iters == (uint64_t)max_iters) { s->status |= 1; s->finished = 1; continue; }
 
         /* 2. decide */
-        int64_t Cp = ap + bp * s->sumP;
+        int64_t Cp = prefill_us(c, s->sumP);
         int prefill;
         if (s->nA == 0) prefill = 0;
         else if (s->nR == 0) prefill = 1;

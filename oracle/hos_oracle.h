@@ -32,6 +32,11 @@ typedef struct {
     uint32_t decode_kv_div;         /* q: decode adds floor(sum KV / q) */
     uint32_t est_per_prompt_token;  /* e_p */
     uint32_t est_per_output_token;  /* e_o */
+    /* Eq. 5-7: with n_levels > 0 a prefill stage is at the smallest level l whose capacity
+     * N^cap_l holds its tokens and lasts T^p_l (a_p, b_p unused); no stage exceeds the largest. */
+    uint32_t n_levels;
+    uint32_t level_cap[8];          /* N^cap_l, ascending */
+    uint32_t level_time[8];         /* T^p_l, non-decreasing */
 } ora_cost;
 
 typedef struct { int32_t i, u, k; int64_t v; } ora_move;
@@ -39,6 +44,7 @@ typedef struct { int32_t i, u, k; int64_t v; } ora_move;
 typedef struct {
     int64_t lb_pack, sum_T, max_T, pair_T;
     int64_t lb_sim_us, tp_star_us, td_star_us, chain_us;
+    int64_t tp_paper_us;            /* Eq. 31 as printed: T^p_L * floor(sum N^p / N^cap_L); 0 without levels */
 } ora_lb;
 
 typedef struct { uint32_t dur_us, kind_n, tokens, aux; } ora_rec;

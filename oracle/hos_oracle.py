@@ -39,7 +39,8 @@ def build(force: bool = False) -> str:
 class _Cost(C.Structure):
     _fields_ = [(n, C.c_uint32) for n in (
         "prefill_fixed_us", "prefill_per_token_us", "decode_fixed_us", "decode_per_seq_us",
-        "decode_kv_div", "est_per_prompt_token", "est_per_output_token")]
+        "decode_kv_div", "est_per_prompt_token", "est_per_output_token", "n_levels")] + [
+        ("level_cap", C.c_uint32 * 8), ("level_time", C.c_uint32 * 8)]
 
 
 class _Move(C.Structure):
@@ -48,7 +49,8 @@ class _Move(C.Structure):
 
 class _Lb(C.Structure):
     _fields_ = [(n, C.c_int64) for n in (
-        "lb_pack", "sum_T", "max_T", "pair_T", "lb_sim_us", "tp_star_us", "td_star_us", "chain_us")]
+        "lb_pack", "sum_T", "max_T", "pair_T", "lb_sim_us", "tp_star_us", "td_star_us", "chain_us",
+        "tp_paper_us")]
 
 
 class _Client(C.Structure):
@@ -71,8 +73,15 @@ def lib():
     return _lib
 
 
-def _cost(cm: Sequence[int]) -> _Cost:
-    return _Cost(*[int(x) for x in cm])
+def _cost(cm: Sequence) -> _Cost:
+    """cm: the seven coefficients, optionally followed by the prefill levels ((cap_tokens, time_us), ...)."""
+    c = _Cost(*[int(x) for x in cm[:7]])
+    levels = list(cm[7]) if len(cm) > 7 else []
+    c.n_levels = len(levels)
+    for l, (cap_tokens, time_us) in enumerate(levels):
+        c.level_cap[l] = int(cap_tokens)
+        c.level_time[l] = int(time_us)
+    return c
 
 
 def _ptr(a: np.ndarray, ty):

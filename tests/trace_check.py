@@ -23,6 +23,12 @@ PREFILL_FLAG = 1 << 31
 
 def replay(queue, p, o, cm, cap, kv_budget, lambda_q16, trace):
     ap, bp, ad, bd, q = (int(x) for x in cm[:5])
+    levels = [(int(a), int(b)) for a, b in cm[7]] if len(cm) > 7 else []
+
+    def prefill_cost(tokens):              # Eq. 5-7: smallest level that holds the tokens
+        if not levels:
+            return ap + bp * tokens
+        return next(t for c_, t in levels if tokens <= c_)
     queue = [int(i) for i in queue]
     running = {}                      # request -> [kv, remaining]
     head = 0
@@ -41,9 +47,11 @@ def replay(queue, p, o, cm, cap, kv_budget, lambda_q16, trace):
             need = int(p[i]) + int(o[i])
             if reserved + extra + need > kv_budget:
                 break
+            if levels and sum(int(p[x]) for x in cand) + int(p[i]) > levels[-1][0]:
+                break
             cand.append(i)
             extra += need
-        cp = ap + bp * sum(int(p[i]) for i in cand)
+        cp = prefill_cost(sum(int(p[i]) for i in cand))
         wants_prefill = lambda_q16 * waited > (cp << 16)
         if kind_n & PREFILL_FLAG:
             assert cand, f"record {k}: prefill with nothing admissible"
