@@ -194,7 +194,7 @@ class Pipeline:
                 makespan_est=torch.empty((w.n_inst,), dtype=torch.int64, device=self.dev),
                 rounds_applied=torch.empty((w.n_inst,), dtype=torch.int32, device=self.dev),
                 status=torch.empty((w.n_inst,), dtype=torch.int32, device=self.dev),
-                lb=torch.empty((w.n_inst, 64), dtype=torch.uint8, device=self.dev))
+                lb=torch.empty((w.n_inst, hos.LB_DTYPE.itemsize), dtype=torch.uint8, device=self.dev))
         cs = self.copy_stream
         cs.wait_stream(main)
         arrived = []

@@ -61,10 +61,20 @@ enum { HOS_QUEUE_SORTED = 0, HOS_QUEUE_FCFS = 1 };
  * estimated request time T_i = est_per_prompt_token * p_i + est_per_output_token * o_i.
  * Requires decode_fixed_us >= 1, decode_kv_div >= 1, and both iteration durations < 2^31
  * for any admissible batch. */
+#define HOS_MAX_LEVELS 8
 typedef struct hos_cost_model {
     uint32_t prefill_fixed_us, prefill_per_token_us;
     uint32_t decode_fixed_us, decode_per_seq_us, decode_kv_div;
     uint32_t est_per_prompt_token, est_per_output_token;
+    /* Stepped prefill cost, Eq. 5-7: with n_levels > 0 (at most HOS_MAX_LEVELS) a prefill stage is
+     * at the smallest level l whose capacity level_cap_tokens[l] (N^cap_l, strictly ascending)
+     * holds its prompt tokens and lasts level_time_us[l] (T^p_l, non-decreasing, < 2^31); the two
+     * prefill_* coefficients are then unused, no stage takes more than the largest level's
+     * tokens, and a prompt longer than that makes its instance HOS_ST_INVALID.  n_levels = 0:
+     * the affine cost above. */
+    uint32_t n_levels;
+    uint32_t level_cap_tokens[HOS_MAX_LEVELS];
+    uint32_t level_time_us[HOS_MAX_LEVELS];
 } hos_cost_model;
 
 /* HOST struct; p and o are DEVICE tables [n_inst][n_req] of prompt lengths N^p_i and output
@@ -85,10 +95,14 @@ typedef struct hos_ls_move { int32_t i, u, k; int64_t v; } hos_ls_move;
  * model, Eq. 26-30: max(ceil(sum_T / M), max_T, pair_T), pair_T = T_(M) + T_(M+1) when
  * n_req > M.  lb_sim_us bounds every simulated makespan: max(work, chain_us), where work
  * is Eq. 32's t^p* + t^d* for M clients (tp_star_us, td_star_us are the two terms, each
- * rounded up) and chain_us is the longest request served alone. */
+ * rounded up) and chain_us is the longest request served alone.  With prefill levels t^p* is
+ * max(T^p_1 * ceil(n_req / batch_cap), min_l floor(P / N^cap_l) * T^p_l), valid for any level
+ * table; tp_paper_us is Eq. 31 as printed, T^p_L * floor(P / N^cap_L) for the largest level (not
+ * divided by the number of clients; 0 without levels). */
 typedef struct hos_lb {
     int64_t lb_pack, sum_T, max_T, pair_T;
     int64_t lb_sim_us, tp_star_us, td_star_us, chain_us;
+    int64_t tp_paper_us;
 } hos_lb;
 
 typedef struct hos_client_result {

@@ -20,7 +20,7 @@ HOS_ST_LIMIT, HOS_ST_TRACE, HOS_ST_INVALID = 1, 2, 4
 
 LS_MOVE_DTYPE = np.dtype([("i", "<i4"), ("u", "<i4"), ("k", "<i4"), ("v", "<i8")], align=True)
 LB_DTYPE = np.dtype([(n, "<i8") for n in ("lb_pack", "sum_T", "max_T", "pair_T", "lb_sim_us",
-                                           "tp_star_us", "td_star_us", "chain_us")])
+                                           "tp_star_us", "td_star_us", "chain_us", "tp_paper_us")])
 CLIENT_RESULT_DTYPE = np.dtype([("makespan_us", "<i8"), ("busy_slot_us", "<i8"),
                                 ("n_prefill_iters", "<u4"), ("n_decode_iters", "<u4"),
                                 ("trace_hash", "<u8"), ("utilisation", "<f8")])
@@ -45,7 +45,8 @@ class HosError(RuntimeError):
 class _CostModel(C.Structure):
     _fields_ = [(n, C.c_uint32) for n in (
         "prefill_fixed_us", "prefill_per_token_us", "decode_fixed_us", "decode_per_seq_us",
-        "decode_kv_div", "est_per_prompt_token", "est_per_output_token")]
+        "decode_kv_div", "est_per_prompt_token", "est_per_output_token", "n_levels")] + [
+        ("level_cap_tokens", C.c_uint32 * 8), ("level_time_us", C.c_uint32 * 8)]
 
 
 class _Batch(C.Structure):
@@ -133,8 +134,17 @@ def _batch(p, o, n_clients: int, batch_cap: int, kv_budget: int) -> _Batch:
     return _Batch(p.shape[0], p.shape[1], n_clients, batch_cap, kv_budget, p.data_ptr(), o.data_ptr())
 
 
-def _cost(cm: Sequence[int]) -> _CostModel:
-    return _CostModel(*[int(x) for x in cm])
+def _cost(cm: Sequence) -> _CostModel:
+    """cm: the seven coefficients, optionally followed by the prefill levels ((cap_tokens, time_us), ...)."""
+    c = _CostModel(*[int(x) for x in cm[:7]])
+    levels = list(cm[7]) if len(cm) > 7 else []
+    if len(levels) > 8:
+        raise ValueError("at most 8 prefill levels")
+    c.n_levels = len(levels)
+    for l, (cap_tokens, time_us) in enumerate(levels):
+        c.level_cap_tokens[l] = int(cap_tokens)
+        c.level_time_us[l] = int(time_us)
+    return c
 
 
 def _workspace(nbytes: int, like):

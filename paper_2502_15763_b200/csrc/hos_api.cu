@@ -28,9 +28,17 @@ int check_batch(const hos_batch* b) {
 int check_cost(const hos_cost_model* cm, const hos_batch* b) {
     if (!cm) return HOS_E_INVALID;
     if (cm->decode_fixed_us < 1 || cm->decode_kv_div < 1) return HOS_E_INVALID;
+    if (cm->n_levels > HOS_MAX_LEVELS) return HOS_E_INVALID;
+    for (uint32_t l = 0; l < cm->n_levels; ++l) {
+        if (cm->level_cap_tokens[l] < 1 || cm->level_time_us[l] >= (1u << 31)) return HOS_E_INVALID;
+        if (l > 0 && (cm->level_cap_tokens[l] <= cm->level_cap_tokens[l - 1] ||
+                      cm->level_time_us[l] < cm->level_time_us[l - 1]))
+            return HOS_E_INVALID;
+    }
     // longest possible iterations must stay below 2^31 us
     const unsigned long long kv = (unsigned long long)b->kv_budget;
-    const unsigned long long pre = cm->prefill_fixed_us + (unsigned long long)cm->prefill_per_token_us * kv;
+    const unsigned long long pre = cm->n_levels ? 0ull :
+        cm->prefill_fixed_us + (unsigned long long)cm->prefill_per_token_us * kv;
     const unsigned long long dec = cm->decode_fixed_us +
                                    (unsigned long long)cm->decode_per_seq_us * (unsigned long long)b->batch_cap +
                                    kv / cm->decode_kv_div;
@@ -205,7 +213,7 @@ int hos_online_simulate(const hos_batch* b, const int32_t* assign, const hos_cos
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const int n_pad = pad4(b->n_req);
     if (max_iters > 0x7FFFFFFFu) max_iters = 0x7FFFFFFFu;
-    if ((rc = cuda_rc(launch_queue_build(*b, assign, queue_order, w.q_po, w.q_req, w.q_off, w.inst_O,
+    if ((rc = cuda_rc(launch_queue_build(*b, assign, stage_cap_tokens(*cm), queue_order, w.q_po, w.q_req, w.q_off, w.inst_O,
                                          w.inst_status, n_pad, st))))
         return rc;
     if ((rc = cuda_rc(launch_simulate(*b, *cm, lambda_q16, n_lambda, max_iters, w.q_po, w.q_off,
@@ -239,7 +247,7 @@ int hos_online_simulate_steal(const hos_batch* b, const int32_t* assign, const h
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const int n_pad = pad4(b->n_req);
     if (max_iters > 0x7FFFFFFFu) max_iters = 0x7FFFFFFFu;
-    if ((rc = cuda_rc(launch_queue_build(*b, assign, queue_order, w.q_po, w.q_req, w.q_off, w.inst_O,
+    if ((rc = cuda_rc(launch_queue_build(*b, assign, stage_cap_tokens(*cm), queue_order, w.q_po, w.q_req, w.q_off, w.inst_O,
                                          w.inst_status, n_pad, st))))
         return rc;
     if ((rc = cuda_rc(launch_simulate_steal(*b, *cm, lambda_q16, n_lambda, max_iters, w.q_po, w.q_req, w.q_off,

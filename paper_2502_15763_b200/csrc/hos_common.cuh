@@ -75,4 +75,17 @@ __device__ __forceinline__ unsigned long long block_max_u64(unsigned long long v
 
 __device__ __forceinline__ int bit_width_u32(uint32_t v) { return 32 - __clz(v); }
 
+// Duration of a prefill stage over `tokens` prompt tokens: affine, or by level (Eq. 5-7).
+__device__ __forceinline__ uint32_t prefill_us(const hos_cost_model& cm, uint32_t tokens) {
+    if (cm.n_levels == 0) return cm.prefill_fixed_us + cm.prefill_per_token_us * tokens;
+    uint32_t t = cm.level_time_us[cm.n_levels - 1];
+    for (int l = (int)cm.n_levels - 2; l >= 0; --l)
+        if (tokens <= cm.level_cap_tokens[l]) t = cm.level_time_us[l];
+    return t;
+}
+// Most prompt tokens one prefill stage can take (and the longest admissible prompt).
+__host__ __device__ __forceinline__ uint32_t stage_cap_tokens(const hos_cost_model& cm) {
+    return cm.n_levels ? cm.level_cap_tokens[cm.n_levels - 1] : 0xFFFFFFFFu;
+}
+
 }  // namespace hos

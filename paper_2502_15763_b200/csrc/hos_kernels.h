@@ -31,7 +31,7 @@ cudaError_t launch_local_search(const hos_batch& b, const uint32_t* T_sorted, co
 cudaError_t launch_lower_bound(const hos_batch& b, const hos_cost_model& cm, const uint32_t* T_sorted,
                                const InstInfo* info, int n_pad, hos_lb* out, cudaStream_t st);
 
-cudaError_t launch_queue_build(const hos_batch& b, const int32_t* assign, int queue_order, uint2* q_po,
+cudaError_t launch_queue_build(const hos_batch& b, const int32_t* assign, uint32_t p_max, int queue_order, uint2* q_po,
                                uint32_t* q_req, int32_t* q_off, unsigned long long* inst_O,
                                int32_t* inst_status, int n_pad, cudaStream_t st);
 cudaError_t launch_simulate(const hos_batch& b, const hos_cost_model& cm, const uint32_t* lambda_q16,

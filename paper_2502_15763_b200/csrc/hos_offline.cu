@@ -16,7 +16,7 @@ namespace hos {
 template <typename IdxT>
 __global__ void __launch_bounds__(SORT_THREADS, 1)
 k_estimate_sort(const uint32_t* __restrict__ p, const uint32_t* __restrict__ o, int n_req,
-                long long kv_budget, uint32_t e_p, uint32_t e_o,
+                long long kv_budget, uint32_t e_p, uint32_t e_o, uint32_t p_max,
                 uint32_t* __restrict__ T_sorted, uint32_t* __restrict__ order,
                 InstInfo* __restrict__ info, int32_t* __restrict__ status_out, int n_pad) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -30,7 +30,7 @@ k_estimate_sort(const uint32_t* __restrict__ p, const uint32_t* __restrict__ o, 
     for (int i = threadIdx.x; i < n_req; i += SORT_THREADS) {
         const uint32_t pp = pi[i], oo = oi[i];
         const unsigned long long t = (unsigned long long)e_p * pp + (unsigned long long)e_o * oo;
-        if (pp == 0 || oo == 0 || (long long)pp + (long long)oo > kv_budget || t > 0xFFFFFFFFull) bad = 1;
+        if (pp == 0 || oo == 0 || pp > p_max || (long long)pp + (long long)oo > kv_budget || t > 0xFFFFFFFFull) bad = 1;
         s.key[i] = (uint32_t)t;
         sum += t;
         mx = t > mx ? t : mx;
@@ -719,12 +719,11 @@ k_lower_bound(const uint32_t* __restrict__ p, const uint32_t* __restrict__ o, in
     const int inst = blockIdx.x;
     const InstInfo inf = info[inst];
     if (inf.status) {
-        if (threadIdx.x == 0) out[inst] = hos_lb{0, 0, 0, 0, 0, 0, 0, 0};
+        if (threadIdx.x == 0) out[inst] = hos_lb{0, 0, 0, 0, 0, 0, 0, 0, 0};
         return;
     }
     const uint32_t* pi = p + (size_t)inst * n_req;
     const uint32_t* oi = o + (size_t)inst * n_req;
-    const unsigned long long ap = cm.prefill_fixed_us, bp = cm.prefill_per_token_us;
     const unsigned long long ad = cm.decode_fixed_us, bd = cm.decode_per_seq_us, q = cm.decode_kv_div;
     unsigned long long P = 0, O = 0, K = 0, chain = 0;
     for (int i = threadIdx.x; i < n_req; i += blockDim.x) {
@@ -732,7 +731,7 @@ k_lower_bound(const uint32_t* __restrict__ p, const uint32_t* __restrict__ o, in
         P += pp;
         O += oo;
         K += oo * pp + oo * (oo - 1ull) / 2ull;
-        const unsigned long long alone = ap + bp * pp + oo * (ad + bd) +
+        const unsigned long long alone = (unsigned long long)prefill_us(cm, (uint32_t)pp) + oo * (ad + bd) +
                                          floor_sum_below(pp + oo, q) - floor_sum_below(pp, q);
         chain = alone > chain ? alone : chain;
     }
@@ -754,7 +753,22 @@ k_lower_bound(const uint32_t* __restrict__ p, const uint32_t* __restrict__ o, in
         lb = pairT > lb ? pairT : lb;
         const unsigned long long n_pre = ((unsigned long long)n_req + C - 1ull) / C;
         const unsigned long long n_dec = (O + C - 1ull) / C;
-        const unsigned long long tp_star = ap * n_pre + bp * P;
+        unsigned long long tp_star, tp_paper = 0;
+        if (cm.n_levels == 0) {
+            tp_star = (unsigned long long)cm.prefill_fixed_us * n_pre + (unsigned long long)cm.prefill_per_token_us * P;
+        } else {
+            // at least n_pre stages of at least the smallest level's time; a stage of level l carries
+            // at most N^cap_l tokens, so P tokens cost at least min_l floor(P / N^cap_l) T^p_l
+            const unsigned long long by_count = (unsigned long long)cm.level_time_us[0] * n_pre;
+            unsigned long long by_tokens = ~0ull;
+            for (uint32_t l = 0; l < cm.n_levels; ++l) {
+                const unsigned long long v = (P / cm.level_cap_tokens[l]) * cm.level_time_us[l];
+                by_tokens = v < by_tokens ? v : by_tokens;
+            }
+            tp_star = by_count > by_tokens ? by_count : by_tokens;
+            tp_paper = (P / cm.level_cap_tokens[cm.n_levels - 1]) * cm.level_time_us[cm.n_levels - 1];
+        }
+        r.tp_paper_us = (long long)tp_paper;
         const unsigned long long td_q = q * ((ad - 1ull) * n_dec + bd * O) + K;
         const unsigned long long work = (q * tp_star + td_q + q * M - 1ull) / (q * M);
         r.lb_pack = (long long)lb; r.sum_T = (long long)sumT; r.max_T = (long long)maxT; r.pair_T = (long long)pairT;
@@ -790,7 +804,7 @@ cudaError_t launch_estimate_sort(const hos_batch& b, const hos_cost_model& cm, u
     if (e != cudaSuccess) return e;
     launch_hook("k_estimate_sort", 0, st);
     kern<<<b.n_inst, SORT_THREADS, smem, st>>>(b.p, b.o, b.n_req, (long long)b.kv_budget,
-                                               cm.est_per_prompt_token, cm.est_per_output_token,
+                                               cm.est_per_prompt_token, cm.est_per_output_token, stage_cap_tokens(cm),
                                                T_sorted, order, info, status_out, n_pad);
     launch_hook("k_estimate_sort", 1, st);
     return cudaGetLastError();

@@ -20,7 +20,7 @@ template <typename IdxT>
 __global__ void __launch_bounds__(SORT_THREADS, 1)
 k_queue_build(const uint32_t* __restrict__ p, const uint32_t* __restrict__ o,
               const int32_t* __restrict__ assign, int n_req, int n_clients, long long kv_budget,
-              int queue_order, uint2* __restrict__ q_po, uint32_t* __restrict__ q_req,
+              uint32_t p_max, int queue_order, uint2* __restrict__ q_po, uint32_t* __restrict__ q_req,
               int32_t* __restrict__ q_off, unsigned long long* __restrict__ inst_O,
               int32_t* __restrict__ inst_status, int n_pad) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -36,7 +36,7 @@ k_queue_build(const uint32_t* __restrict__ p, const uint32_t* __restrict__ o,
         const uint32_t pp = pi[i], oo = oi[i];
         const int c = ai[i];
         const unsigned long long tot = (unsigned long long)pp + oo;
-        if (pp == 0 || oo == 0 || (long long)tot > kv_budget || c < 0 || c >= n_clients) bad = 1;
+        if (pp == 0 || oo == 0 || pp > p_max || (long long)tot > kv_budget || c < 0 || c >= n_clients) bad = 1;
         s.key[i] = (uint32_t)tot;
         s.buf1[i] = (IdxT)(c & 0xFF);                 // parked until the keys are composed
         sumO += oo;
@@ -148,7 +148,7 @@ k_simulate(const uint2* __restrict__ q_po, const int32_t* __restrict__ q_off,
     const int qn = q_off[(size_t)inst * (n_clients + 1) + c + 1] - q0;
     const uint2* q = q_po + (size_t)inst * n_pad + q0;
     const uint32_t lam = lambda_q16[l];
-    const uint32_t ap = cm.prefill_fixed_us, bp = cm.prefill_per_token_us;
+    const uint32_t stage_cap = stage_cap_tokens(cm);
     const uint32_t ad = cm.decode_fixed_us, bd = cm.decode_per_seq_us, qd = cm.decode_kv_div;
 
     long long t = 0, busy = 0;
@@ -200,6 +200,7 @@ k_simulate(const uint2* __restrict__ q_po, const int32_t* __restrict__ q_off,
             while (head + (int)nA < qn && B + nA < (uint32_t)cap) {
                 const uint32_t tt = nxt.x + nxt.y;
                 if (reserved + sumTot + tt > kv_budget) break;   // each term < 2^31 and reserved + sumTot <= budget: no wrap
+                if (sumP + nxt.x > stage_cap) break;             // the largest prefill level is full
                 heap_st(cap - 1 - (int)nA, E::make(nxt.y, tt));
                 sumTot += tt; sumP += nxt.x; ++nA;
                 nxt = nxt2;
@@ -210,7 +211,7 @@ k_simulate(const uint2* __restrict__ q_po, const int32_t* __restrict__ q_off,
         if (B == 0 && nA == 0) break;                    // queue empty and nothing running
         if (n_pre + cnt == max_iters) { status |= HOS_ST_LIMIT; break; }
 
-        const uint32_t Cp = ap + bp * sumP;
+        const uint32_t Cp = prefill_us(cm, sumP);
         const unsigned long long Cp16 = (unsigned long long)Cp << 16;
         uint32_t dur, r1, r2, r3;
         if (nA > 0 && (B == 0 || (unsigned long long)lam * Cd > Cp16)) {
@@ -232,7 +233,10 @@ k_simulate(const uint2* __restrict__ q_po, const int32_t* __restrict__ q_off,
             dur = Cp; r1 = 0x80000000u | nA; r2 = sumP; r3 = (uint32_t)head;
             busy += (long long)Cp * nA;
             S += sumP; B += nA; reserved += sumTot; head += (int)nA;
-            nA = 0; sumP = 0; sumTot = 0;                 // nothing more fits until someone retires
+            nA = 0; sumP = 0; sumTot = 0;
+            // slots and KV budget are as full as before, but a stage that stopped at the largest
+            // prefill level's capacity has room again
+            grow = stage_cap != 0xFFFFFFFFu && head < qn;
             next_fin = E::fin(heap_ld(0), cnt);
         } else {
             dur = ad + bd * B + (q_shift >= 0 ? (S >> q_shift) : (S / qd));
@@ -371,7 +375,7 @@ k_simulate_steal(const uint2* __restrict__ q_po, const uint32_t* __restrict__ q_
     int32_t* served = served_by ? served_by + (size_t)sim * n_req : nullptr;
     const int qend = is_client ? qo[c + 1] : 0;
     const uint32_t lam = lambda_q16[l];
-    const uint32_t ap = cm.prefill_fixed_us, bp = cm.prefill_per_token_us;
+    const uint32_t stage_cap = stage_cap_tokens(cm);
     const uint32_t ad = cm.decode_fixed_us, bd = cm.decode_per_seq_us, qd = cm.decode_kv_div;
 
     if (is_client) {
@@ -413,6 +417,7 @@ k_simulate_steal(const uint2* __restrict__ q_po, const uint32_t* __restrict__ q_
         const uint2 po = q[x];
         const uint32_t tt = po.x + po.y;
         if (reserved + sumTot + tt > kv_budget) return false;
+        if (sumP + po.x > stage_cap) return false;          // the largest prefill level is full
         heap_st(cap - 1 - (int)nA, E::make(po.y, tt));
         sumTot += tt; sumP += po.x; ++nA;
         if (!dry) {
@@ -447,7 +452,7 @@ k_simulate_steal(const uint2* __restrict__ q_po, const uint32_t* __restrict__ q_
         if (B == 0 && nA == 0) { finished = true; return; }
         if (n_pre + cnt == max_iters) { status |= HOS_ST_LIMIT; finished = true; return; }
 
-        const uint32_t Cp = ap + bp * sumP;
+        const uint32_t Cp = prefill_us(cm, sumP);
         const unsigned long long Cp16 = (unsigned long long)Cp << 16;
         uint32_t dur, r1, r2, r3;
         if (nA > 0 && (B == 0 || (unsigned long long)lam * Cd > Cp16)) {
@@ -557,7 +562,8 @@ k_simulate_steal(const uint2* __restrict__ q_po, const uint32_t* __restrict__ q_
     // stolen before H = max(s_first, min es over the unfinished clients), hence every iteration that
     // starts before H only touches its own client and all of them may run side by side.  When none
     // starts before H, the client at the front of the global order may steal: it runs alone.
-    const unsigned long long d_min = min((unsigned long long)ap, (unsigned long long)ad + bd);
+    // shortest possible iteration: a prefill of one token, or a decode of one request
+    const unsigned long long d_min = min((unsigned long long)prefill_us(cm, 1u), (unsigned long long)ad + bd);
     while (true) {
         __syncthreads();                                   // last step's queue updates are visible
         const unsigned long long key = ((unsigned long long)t << 9) | (unsigned)c;
@@ -723,7 +729,7 @@ size_t queue_build_smem(int n_req) {
     return n_req <= 65536 ? sort_smem_bytes<uint16_t>(n_req) : sort_smem_bytes<uint32_t>(n_req);
 }
 
-cudaError_t launch_queue_build(const hos_batch& b, const int32_t* assign, int queue_order, uint2* q_po,
+cudaError_t launch_queue_build(const hos_batch& b, const int32_t* assign, uint32_t p_max, int queue_order, uint2* q_po,
                                uint32_t* q_req, int32_t* q_off, unsigned long long* inst_O,
                                int32_t* inst_status, int n_pad, cudaStream_t st) {
     const size_t smem = queue_build_smem(b.n_req);
@@ -732,7 +738,7 @@ cudaError_t launch_queue_build(const hos_batch& b, const int32_t* assign, int qu
     if (e != cudaSuccess) return e;
     launch_hook("k_queue_build", 0, st);
     kern<<<b.n_inst, SORT_THREADS, smem, st>>>(b.p, b.o, assign, b.n_req, b.n_clients,
-                                               (long long)b.kv_budget, queue_order, q_po, q_req, q_off,
+                                               (long long)b.kv_budget, p_max, queue_order, q_po, q_req, q_off,
                                                inst_O, inst_status, n_pad);
     launch_hook("k_queue_build", 1, st);
     return cudaGetLastError();

@@ -34,7 +34,7 @@ def test_strerror_and_host_side_validation():
 
 def test_struct_sizes_match_the_header():
     assert hos.LS_MOVE_DTYPE.itemsize == 24
-    assert hos.LB_DTYPE.itemsize == 64
+    assert hos.LB_DTYPE.itemsize == 72
     assert hos.CLIENT_RESULT_DTYPE.itemsize == 40
     assert hos.SIM_RESULT_DTYPE.itemsize == 32
     assert hos.ITER_REC_DTYPE.itemsize == 16

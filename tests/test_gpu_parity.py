@@ -200,6 +200,42 @@ def test_request_stealing_config4_sampled(hos):
     assert (r["sres"]["makespan_us"][:, 0] <= 1.02 * plain["sres"]["makespan_us"][:, 0]).all()
 
 
+def test_prefill_levels(hos):
+    # stepped prefill cost (Eq. 5-7) in the simulators and the bounds
+    rng = np.random.default_rng(21)
+    n_inst, n, M, cap = 3, 400, 4, 24
+    p = rng.integers(1, 300, size=(n_inst, n)).astype(np.uint32)
+    o = rng.integers(1, 60, size=(n_inst, n)).astype(np.uint32)
+    for levels in ([(300, 30000)], [(400, 20000), (900, 41000), (2500, 90000)]):
+        cm = (5, 5, 15000, 300, 16, 40, 350, levels)
+        g = H.check_offline(hos, p, o, M, cap, 10 ** 6, cm, 3)
+        lb = H.check_lower_bound(hos, p, o, M, cap, 10 ** 6, cm)
+        assert (lb["tp_paper_us"] > 0).all()
+        for mode in (ora.QUEUE_SORTED, ora.QUEUE_FCFS):
+            H.check_simulate(hos, p, o, M, cap, 10 ** 6, cm, g["assign"], LAMS, mode)
+            H.check_simulate_steal(hos, p, o, M, cap, 10 ** 6, cm, g["assign"], (LAMBDA_NEVER_PREEMPT, LAMBDA_ONE), mode)
+    # a prompt longer than the largest level can never be prefilled: the instance is invalid
+    p2 = p.copy(); p2[2, 7] = 301
+    cm = (5, 5, 15000, 300, 16, 40, 350, [(300, 30000)])
+    g2 = H.gpu_simulate(hos, p2, o, M, cap, 10 ** 6, cm, g["assign"], (LAMBDA_ONE,), ora.QUEUE_SORTED, want_trace=False)
+    assert (g2["status"][2] == hos.HOS_ST_INVALID).all() and (g2["status"][:2] == 0).all()
+    with pytest.raises(hos.HosError):                        # caps must ascend
+        hos.hos_lower_bound(H.to_dev(p), H.to_dev(o), M, cap, 10 ** 6, (5, 5, 15000, 300, 16, 40, 350, [(300, 1), (300, 2)]))
+
+
+def test_paper_shaped_workload(hos):
+    from workload import paper_shaped
+    w = paper_shaped(n_inst=6)
+    p, o = w.lengths()
+    M, cap, kv, cm = w.n_clients, w.batch_cap, w.kv_budget, w.cost_model
+    g = H.check_offline(hos, p, o, M, cap, kv, cm, 0)
+    lb = H.check_lower_bound(hos, p, o, M, cap, kv, cm)
+    hyb = H.check_simulate(hos, p, o, M, cap, kv, cm, g["assign"], (LAMBDA_ONE,), ora.QUEUE_SORTED)
+    base = H.check_simulate(hos, p, o, M, cap, kv, cm, g["assign"], (LAMBDA_PREFILL_FIRST,), ora.QUEUE_FCFS)
+    assert (lb["lb_sim_us"] <= hyb["sres"]["makespan_us"][:, 0]).all()
+    assert (hyb["sres"]["utilisation"][:, 0] > base["sres"]["utilisation"][:, 0]).mean() >= 0.5
+
+
 def test_limits_and_bad_data(hos):
     w = workload("c0")
     p, o = w.lengths()

@@ -69,7 +69,26 @@ def workload(name: str) -> Workload:
     if name == "c4":      # scale-out stress
         return Workload("c4", tuple(range(1000, 2024)), 20000, 64, 128, 262144, LONG_P, LONG_O,
                         (LAMBDA_ONE,), 100)
+    if name == "paper":   # shaped like the paper's own experiment (Table "Experiment settings")
+        return paper_shaped()
     raise KeyError(name)
+
+
+# Lengths with the paper's moments: input 68.43 +- 25.04 tokens, output 344.83 +- 187.99 capped at
+# 512 (log-normals with those means and deviations before clipping).
+PAPER_P = LengthDist(64.26, 0.3545, 4, 512)
+PAPER_O = LengthDist(302.8, 0.5101, 1, 512)
+# 0.13 ms per prompt token + 25 ms as a level table (Eq. 5-7), 0.21 ms per running request + 29 ms
+# per decode round, no KV term; estimates count output tokens only.
+PAPER_LEVELS = tuple((cap, 25000 + 130 * cap) for cap in (512, 1024, 2048, 4096, 8192, 16384))
+PAPER_COST = (25000, 130, 29000, 210, 0x7FFFFFFF, 0, 71000, PAPER_LEVELS)
+
+
+def paper_shaped(n_inst: int = 100, first_seed: int = 5000) -> Workload:
+    """One client = the paper's whole system: 200 concurrent requests (1024 KV blocks of 128 tokens,
+    five blocks per request), 1,319 requests per instance, lambda = 1.0."""
+    return Workload("paper", tuple(range(first_seed, first_seed + n_inst)), 1319, 1, 200, 1024 * 128,
+                    PAPER_P, PAPER_O, (LAMBDA_ONE,), 0, PAPER_COST)
 
 
 def shard(n_units: int, world_size: int, rank: int) -> Tuple[int, int]:
