@@ -500,7 +500,7 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=10)
     ap.add_argument("--warmup", type=int, default=3)
-    ap.add_argument("--workload", default="c4", choices=["c0", "c1", "c2", "c3", "c4"])
+    ap.add_argument("--workload", default="c4", choices=["c0", "c1", "c2", "c3", "c4", "paper"])
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--instances", type=int, default=0,
                     help="use only the first N instances of the workload (profiling captures)")
