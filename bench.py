@@ -150,7 +150,7 @@ class Pipeline:
         from paper_2502_15763_b200 import binding as B
         b = B._batch(*self.args()[:5])
         L = self.hos.lib()
-        n_off = L.hos_offline_workspace_bytes(C.byref(b), 1, self.w.ls_rounds)
+        n_off = L.hos_offline_workspace_bytes(C.byref(b), len(self.w.lambdas_q16), self.w.ls_rounds)
         n_on = L.hos_online_workspace_bytes(C.byref(b), len(self.w.lambdas_q16), 1)
         self.ws_off = self.torch.empty(n_off, dtype=self.torch.uint8, device=self.dev)
         self.ws_on = self.torch.empty(n_on, dtype=self.torch.uint8, device=self.dev)

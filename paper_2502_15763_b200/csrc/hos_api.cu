@@ -55,9 +55,11 @@ struct OfflineWs {
     uint32_t* T_sorted;
     uint32_t* order;
     InstInfo* info;
+    uint32_t* ls_T;             // local search, per (instance, copy): the member lists' T
+    void* ls_I;                 // and request indices
     size_t bytes;
 };
-OfflineWs carve_offline(const hos_batch* b, void* ws) {
+OfflineWs carve_offline(const hos_batch* b, void* ws, int n_copies, int ls_rounds) {
     OfflineWs w;
     const size_t rows = (size_t)b->n_inst * pad4(b->n_req);
     unsigned char* base = static_cast<unsigned char*>(ws);
@@ -65,6 +67,12 @@ OfflineWs carve_offline(const hos_batch* b, void* ws) {
     w.T_sorted = reinterpret_cast<uint32_t*>(base + off); off += up(rows * 4);
     w.order = reinterpret_cast<uint32_t*>(base + off);    off += up(rows * 4);
     w.info = reinterpret_cast<InstInfo*>(base + off);     off += up((size_t)b->n_inst * sizeof(InstInfo));
+    w.ls_T = nullptr; w.ls_I = nullptr;
+    if (ls_rounds > 0) {
+        const size_t units = rows * (size_t)(n_copies > 0 ? n_copies : 1);
+        w.ls_T = reinterpret_cast<uint32_t*>(base + off);  off += up(units * 4);
+        w.ls_I = base + off;                               off += up(units * local_search_index_bytes(b->n_req));
+    }
     w.bytes = off;
     return w;
 }
@@ -115,13 +123,13 @@ void launch_hook(const char* kernel, int phase, cudaStream_t st) {
 
 extern "C" {
 
-size_t hos_offline_workspace_bytes(const hos_batch* b, int /*n_copies*/, int /*ls_rounds*/) {
+size_t hos_offline_workspace_bytes(const hos_batch* b, int n_copies, int ls_rounds) {
     if (!b || b->n_inst < 1 || b->n_req < 1) return 0;
-    return carve_offline(b, nullptr).bytes;
+    return carve_offline(b, nullptr, n_copies, ls_rounds).bytes;
 }
 size_t hos_lower_bound_workspace_bytes(const hos_batch* b) {
     if (!b || b->n_inst < 1 || b->n_req < 1) return 0;
-    return carve_offline(b, nullptr).bytes;
+    return carve_offline(b, nullptr, 1, 0).bytes;
 }
 size_t hos_online_workspace_bytes(const hos_batch* b, int n_lambda, int keep_events) {
     if (!b || b->n_inst < 1 || b->n_req < 1 || b->n_clients < 1 || n_lambda < 1) return 0;
@@ -136,10 +144,9 @@ int hos_offline_pack(const hos_batch* b, const hos_cost_model* cm, int ls_rounds
     if (rc) return rc;
     if ((rc = check_cost(cm, b))) return rc;
     if (!assign || !load || !makespan_est || !rounds_applied || !status || ls_rounds < 0) return HOS_E_INVALID;
-    if (estimate_sort_smem(b->n_req) > SMEM_LIMIT || local_search_smem(b->n_req, b->n_clients) > SMEM_LIMIT)
-        return HOS_E_UNSUPPORTED;
+    if (estimate_sort_smem(b->n_req) > SMEM_LIMIT) return HOS_E_UNSUPPORTED;
     if ((rc = check_ws(ws, ws_bytes, hos_offline_workspace_bytes(b, 1, ls_rounds)))) return rc;
-    const OfflineWs w = carve_offline(b, ws);
+    const OfflineWs w = carve_offline(b, ws, 1, ls_rounds);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const int n_pad = pad4(b->n_req);
     if ((rc = cuda_rc(launch_estimate_sort(*b, *cm, w.T_sorted, w.order, w.info, status, n_pad, st)))) return rc;
@@ -153,7 +160,7 @@ int hos_offline_pack(const hos_batch* b, const hos_cost_model* cm, int ls_rounds
     return cuda_rc(launch_local_search(*b, w.T_sorted, w.order, w.info, n_pad, 1, ls_rounds, false, assign,
                                        reinterpret_cast<long long*>(load),
                                        reinterpret_cast<long long*>(makespan_est), rounds_applied,
-                                       ls_log, status, st));
+                                       ls_log, status, w.ls_T, w.ls_I, st));
 }
 
 int hos_local_search(const hos_batch* b, const hos_cost_model* cm, int n_copies, int ls_rounds,
@@ -165,17 +172,16 @@ int hos_local_search(const hos_batch* b, const hos_cost_model* cm, int n_copies,
     if (!assign || !load || !makespan_est || !rounds_applied || !status || ls_rounds < 0 || n_copies < 1)
         return HOS_E_INVALID;
     if ((long long)b->n_inst * n_copies > 0x7FFFFFFFll) return HOS_E_UNSUPPORTED;
-    if (estimate_sort_smem(b->n_req) > SMEM_LIMIT || local_search_smem(b->n_req, b->n_clients) > SMEM_LIMIT)
-        return HOS_E_UNSUPPORTED;
+    if (estimate_sort_smem(b->n_req) > SMEM_LIMIT) return HOS_E_UNSUPPORTED;
     if ((rc = check_ws(ws, ws_bytes, hos_offline_workspace_bytes(b, n_copies, ls_rounds)))) return rc;
-    const OfflineWs w = carve_offline(b, ws);
+    const OfflineWs w = carve_offline(b, ws, n_copies, ls_rounds);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const int n_pad = pad4(b->n_req);
     if ((rc = cuda_rc(launch_estimate_sort(*b, *cm, w.T_sorted, w.order, w.info, status, n_pad, st)))) return rc;
     return cuda_rc(launch_local_search(*b, w.T_sorted, w.order, w.info, n_pad, n_copies, ls_rounds, true,
                                        assign, reinterpret_cast<long long*>(load),
                                        reinterpret_cast<long long*>(makespan_est), rounds_applied,
-                                       ls_log, status, st));
+                                       ls_log, status, w.ls_T, w.ls_I, st));
 }
 
 int hos_lower_bound(const hos_batch* b, const hos_cost_model* cm, hos_lb* out, int32_t* status, void* ws,
@@ -186,7 +192,7 @@ int hos_lower_bound(const hos_batch* b, const hos_cost_model* cm, hos_lb* out, i
     if (!out || !status) return HOS_E_INVALID;
     if (estimate_sort_smem(b->n_req) > SMEM_LIMIT) return HOS_E_UNSUPPORTED;
     if ((rc = check_ws(ws, ws_bytes, hos_lower_bound_workspace_bytes(b)))) return rc;
-    const OfflineWs w = carve_offline(b, ws);
+    const OfflineWs w = carve_offline(b, ws, 1, 0);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const int n_pad = pad4(b->n_req);
     if ((rc = cuda_rc(launch_estimate_sort(*b, *cm, w.T_sorted, w.order, w.info, status, n_pad, st)))) return rc;

@@ -238,10 +238,12 @@ k_lpt(const uint32_t* __restrict__ T_sorted, const uint32_t* __restrict__ order,
 }
 
 // ---------------------------------------------------------------------------------------
-// Local search.  One CTA per (instance, copy); the instance stays in shared memory for all
-// rounds: T by rank, request index by rank, client by rank, and the clients' member lists
-// (CSR: for every client its ranks in ascending order, i.e. T descending, index ascending
-// inside equal T).
+// Local search.  One small CTA per (instance, copy), many CTAs per SM: a round is a chain of
+// short dependent phases, so throughput comes from running many instances side by side, not
+// from a wide CTA.  The state of an instance is the clients' member lists in global memory
+// (CSR: for every client its requests with T descending, index ascending inside equal T, as
+// two arrays: T and request index); a round touches a few KB of them, which stay in L1/L2.
+// Shared memory holds the loads, the list offsets and a copy of the critical client's list.
 //
 // A round looks for the minimum of (v, i, k, u) over every move (u = -1, d = T_i) and swap
 // (d = T_i - T_u > 0) off the critical client jmax, v = max(Lmax - d, load_k + d).  For a
@@ -252,8 +254,8 @@ k_lpt(const uint32_t* __restrict__ T_sorted, const uint32_t* __restrict__ order,
 // v >= ceil((Lmax + load_k) / 2): the least loaded client is evaluated first, its best v
 // bounds the optimum, and only clients whose floor does not exceed that bound are looked at
 // (ties in v survive the filter).  Work items are taken from the member lists, so every lane
-// of the evaluating warps has an item.  A swap keeps both list lengths: the two lists are
-// patched in place; a move rebuilds the lists.
+// has an item.  A swap keeps both list lengths: one warp per list shifts the entries between
+// the old and the new position; a move rebuilds the lists from the assignment.
 // ---------------------------------------------------------------------------------------
 // A candidate step, ordered by (v, i, k, u) through three words that compare the same way:
 // inv = ~(Lmax - v) (every useful candidate has 0 < Lmax - v <= T_i < 2^32), ik = i << 8 | k,
@@ -287,9 +289,13 @@ __device__ __forceinline__ Cand cand_warp_min(const Cand& c) {
 constexpr long long NO_V = 0x7FFFFFFFFFFFFFFFll;
 constexpr int NO_I = 0x7FFFFFFF;
 
-// Exclusive scan of a[0 .. len) in place by the whole CTA; `wsum` holds 32 words.
+constexpr int LS_THREADS = 128;
+constexpr int LS_WARPS = LS_THREADS / 32;
+constexpr int LS_STAGE = 512;             // longest critical list that is copied to shared memory
+
+// Exclusive scan of a[0 .. len) in place by the whole CTA; `wsum` holds LS_WARPS words.
 __device__ inline void block_scan_u32(uint32_t* a, int len, uint32_t* wsum) {
-    const int per = (len + SORT_THREADS - 1) / SORT_THREADS;
+    const int per = (len + LS_THREADS - 1) / LS_THREADS;
     const int lo = min(len, (int)threadIdx.x * per), hi = min(len, lo + per);
     uint32_t run = 0;
     for (int x = lo; x < hi; ++x) run += a[x];
@@ -301,107 +307,135 @@ __device__ inline void block_scan_u32(uint32_t* a, int len, uint32_t* wsum) {
     }
     if (lane_id() == 31) wsum[warp_id()] = inc;
     __syncthreads();
-    if (warp_id() == 0) {
-        const uint32_t w = wsum[lane_id()];
-        uint32_t winc = w;
+    uint32_t before = 0;                                     // total of the warps before mine
 #pragma unroll
-        for (int d = 1; d < 32; d <<= 1) {
-            const uint32_t y = __shfl_up_sync(FULL, winc, d);
-            if (lane_id() >= d) winc += y;
-        }
-        wsum[lane_id()] = winc - w;
-    }
-    __syncthreads();
-    uint32_t acc = wsum[warp_id()] + inc - run;
+    for (int w = 0; w < LS_WARPS; ++w) before += w < warp_id() ? wsum[w] : 0u;
+    uint32_t acc = before + inc - run;
     for (int x = lo; x < hi; ++x) { const uint32_t c = a[x]; a[x] = acc; acc += c; }
     __syncthreads();
 }
 
-// Member lists of all clients from bins[]: a stable split of the ranks 0..n-1 by client, with the
-// members' T beside them (clT).
-// cnt holds n_clients * SORT_WARPS words.  off[k] = start of client k's list, off[M] = n.
-template <typename IdxT>
-__device__ inline void build_member_lists(const uint8_t* bins, const uint32_t* __restrict__ gT, IdxT* cl,
-                                          uint32_t* clT, int n, int n_clients, uint32_t* cnt,
-                                          uint32_t* wsum, int* off) {
+// Member lists of all clients from the assignment: a stable split of the ranks 0..n-1 by
+// client, as the members' request index (clI) and T (clT).  cnt holds n_clients * LS_WARPS
+// words.  off[k] = start of client k's list, off[M] = n.  With CHECK, an assignment outside
+// [0, M) makes every thread return true (lists not built), and `load`, if given, receives the
+// clients' summed T.
+template <typename IdxT, bool CHECK>
+__device__ inline bool build_member_lists(const int32_t* asg, const uint32_t* __restrict__ gO,
+                                          const uint32_t* __restrict__ gT, IdxT* clI, uint32_t* clT,
+                                          int n, int n_clients, uint32_t* cnt, uint32_t* wsum, int* off,
+                                          long long* load) {
     const int lane = lane_id(), warp = warp_id();
-    const int chunk = (((n + SORT_WARPS - 1) / SORT_WARPS) + 31) & ~31;
+    const int chunk = (((n + LS_WARPS - 1) / LS_WARPS) + 31) & ~31;
     const int lo = warp * chunk, hi = min(n, lo + chunk);
     const int nb = bit_width_u32((uint32_t)(n_clients - 1));
-    for (int x = threadIdx.x; x < n_clients * SORT_WARPS; x += SORT_THREADS) cnt[x] = 0;
+    for (int x = threadIdx.x; x < n_clients * LS_WARPS; x += LS_THREADS) cnt[x] = 0;
     __syncthreads();
+    bool bad = false;
     for (int row = lo; row < hi; row += 32) {
         const int r = row + lane;
-        if (r < hi) atomicAdd(&cnt[(uint32_t)bins[r] * SORT_WARPS + warp], 1u);
+        if (r < hi) {
+            const int c = asg[__ldg(&gO[r])];
+            if (CHECK && (c < 0 || c >= n_clients)) bad = true;
+            else {
+                atomicAdd(&cnt[(uint32_t)c * LS_WARPS + warp], 1u);
+                if (CHECK && load)
+                    atomicAdd(reinterpret_cast<unsigned long long*>(&load[c]), (unsigned long long)__ldg(&gT[r]));
+            }
+        }
     }
-    __syncthreads();
-    block_scan_u32(cnt, n_clients * SORT_WARPS, wsum);
-    for (int k = threadIdx.x; k <= n_clients; k += SORT_THREADS)
-        off[k] = k < n_clients ? (int)cnt[k * SORT_WARPS] : n;
+    if (CHECK) { if (__syncthreads_or(bad)) return true; }
+    else __syncthreads();
+    block_scan_u32(cnt, n_clients * LS_WARPS, wsum);
+    for (int k = threadIdx.x; k <= n_clients; k += LS_THREADS)
+        off[k] = k < n_clients ? (int)cnt[k * LS_WARPS] : n;
     __syncthreads();
     for (int row = lo; row < hi; row += 32) {
         const int r = row + lane;
         const bool valid = r < hi;
-        const uint32_t dig = valid ? (uint32_t)bins[r] : 0u;
-        const uint32_t tr = valid ? gT[r] : 0u;
+        const uint32_t id = valid ? __ldg(&gO[r]) : 0u;
+        const uint32_t dig = valid ? (uint32_t)asg[id] : 0u;
+        const uint32_t tr = valid ? __ldg(&gT[r]) : 0u;
         unsigned m = __ballot_sync(FULL, valid);             // lanes of this row on my client
         for (int b = 0; b < nb; ++b) {
             const bool bit = (dig >> b) & 1u;
             const unsigned bal = __ballot_sync(FULL, bit);
             m &= bit ? bal : ~bal;
         }
-        const uint32_t base = valid ? cnt[dig * SORT_WARPS + warp] : 0u;
+        const uint32_t base = valid ? cnt[dig * LS_WARPS + warp] : 0u;
         __syncwarp();
         if (valid) {
             const uint32_t at = base + __popc(m & ((1u << lane) - 1u));
-            cl[at] = (IdxT)r;
+            clI[at] = (IdxT)id;
             clT[at] = tr;
-            if (lane == (__ffs(m) - 1)) cnt[dig * SORT_WARPS + warp] = base + __popc(m);
+            if (lane == (__ffs(m) - 1)) cnt[dig * LS_WARPS + warp] = base + __popc(m);
         }
         __syncwarp();
     }
     __syncthreads();
+    return false;
 }
 
-// In the ascending list seg[0 .. len): drop the element at position `gone`, insert `val`.
-// Called by `nthr` threads (tid 0 .. nthr-1) of the CTA; the caller places a __syncthreads()
-// between the returned read phase and `patch_write`.
+// One warp: in the list (segT, segI)[0 .. len), ordered by (T descending, index ascending),
+// drop the entry at position `gone` and insert (valT, valI) at its place in the order.
 template <typename IdxT>
-struct ListPatch {
-    int dst_lo, dst_hi, shift, at;     // elements at [dst_lo, dst_hi) move by `shift`; val lands at `at`
-};
-template <typename IdxT>
-__device__ inline ListPatch<IdxT> patch_plan(const IdxT* seg, int len, int gone, int val) {
-    int a = 0, z = len;                                  // lower bound of val
+__device__ inline void warp_patch_list(uint32_t* segT, IdxT* segI, int len, int gone, uint32_t valT,
+                                       uint32_t valI) {
+    const int lane = lane_id();
+    int a = 0, z = len;                                      // entries that come before the new one
     while (a < z) {
         const int mid = (a + z) >> 1;
-        if ((int)seg[mid] < val) a = mid + 1; else z = mid;
+        const uint32_t t = segT[mid];
+        const bool before = t > valT || (t == valT && (uint32_t)segI[mid] < valI);
+        if (before) a = mid + 1; else z = mid;
     }
-    const int at = a - ((int)seg[gone] < val ? 1 : 0);   // position among the remaining elements
-    ListPatch<IdxT> p;
-    p.at = at;
-    if (at > gone) { p.dst_lo = gone + 1; p.dst_hi = at + 1; p.shift = -1; }
-    else if (at < gone) { p.dst_lo = at; p.dst_hi = gone; p.shift = +1; }
-    else { p.dst_lo = 0; p.dst_hi = 0; p.shift = 0; }
-    return p;
+    const uint32_t tg = segT[gone];
+    const bool gone_before = tg > valT || (tg == valT && (uint32_t)segI[gone] < valI);
+    const int at = a - (gone_before ? 1 : 0);                // position among the remaining entries
+    if (at > gone) {                                         // entries (gone, at] move down by one
+        for (int x0 = gone + 1; x0 <= at; x0 += 32) {
+            const int x = x0 + lane;
+            const bool ok = x <= at;
+            const uint32_t t = ok ? segT[x] : 0u;
+            const IdxT i = ok ? segI[x] : (IdxT)0;
+            __syncwarp();
+            if (ok) { segT[x - 1] = t; segI[x - 1] = i; }
+        }
+    } else if (at < gone) {                                  // entries [at, gone) move up by one
+        for (int x1 = gone - 1; x1 >= at; x1 -= 32) {
+            const int x = x1 - lane;
+            const bool ok = x >= at;
+            const uint32_t t = ok ? segT[x] : 0u;
+            const IdxT i = ok ? segI[x] : (IdxT)0;
+            __syncwarp();
+            if (ok) { segT[x + 1] = t; segI[x + 1] = i; }
+        }
+    }
+    __syncwarp();
+    if (lane == 0) { segT[at] = valT; segI[at] = (IdxT)valI; }
 }
 
 template <typename IdxT>
-__global__ void __launch_bounds__(SORT_THREADS, 1)
+__global__ void __launch_bounds__(LS_THREADS, 8)
 k_local_search(const uint32_t* __restrict__ T_sorted, const uint32_t* __restrict__ order,
                const InstInfo* __restrict__ info, int n_req, int n_pad, int n_clients,
                int n_copies, int rounds, bool load_from_assign,
                int32_t* __restrict__ assign, long long* __restrict__ load_io,
                long long* __restrict__ makespan_out, int32_t* __restrict__ rounds_applied,
-               hos_ls_move* __restrict__ ls_log, int32_t* __restrict__ status_out) {
+               hos_ls_move* __restrict__ ls_log, int32_t* __restrict__ status_out,
+               uint32_t* __restrict__ ws_T, IdxT* __restrict__ ws_I) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     __shared__ long long s_load[MAX_CLIENTS];
     __shared__ int s_off[MAX_CLIENTS + 1];
-    __shared__ Cand s_cand[32];
-    __shared__ uint32_t s_wsum[32];
-    __shared__ int s_as[MAX_CLIENTS];
-    __shared__ uint8_t s_ak[MAX_CLIENTS];
+    __shared__ Cand s_cand[LS_WARPS];
+    __shared__ uint32_t s_wsum[LS_WARPS];
+    __shared__ int s_as[MAX_CLIENTS + 1];                   // listed clients: first work item (and the total),
+    __shared__ int s_cb[MAX_CLIENTS];                       // start of the member list,
+    __shared__ uint32_t s_cs[MAX_CLIENTS];                  // Lmax - load (when that fits 31 bits),
+    __shared__ uint8_t s_ak[MAX_CLIENTS];                   // client
     __shared__ uint8_t s_listed[MAX_CLIENTS];
+    __shared__ uint32_t s_T[LS_STAGE + 1];                  // [0] = all ones, [1 .. nm] = jmax's T, then zeros
+    __shared__ IdxT s_I[LS_STAGE];                          // jmax's request indices
     __shared__ int s_jmax, s_kmin, s_na, s_nitems;
     __shared__ long long s_lmax;
 
@@ -415,49 +449,35 @@ k_local_search(const uint32_t* __restrict__ T_sorted, const uint32_t* __restrict
 
     if (inf.status) {
         if (load_from_assign) {
-            for (int j = threadIdx.x; j < n_clients; j += SORT_THREADS) ld[j] = 0;
+            for (int j = threadIdx.x; j < n_clients; j += LS_THREADS) ld[j] = 0;
             if (threadIdx.x == 0) makespan_out[unit] = 0;
         }
         if (threadIdx.x == 0) rounds_applied[unit] = 0;
         if (log)
-            for (int r = threadIdx.x; r < rounds; r += SORT_THREADS) log[r] = hos_ls_move{-1, -1, -1, 0};
+            for (int r = threadIdx.x; r < rounds; r += LS_THREADS) log[r] = hos_ls_move{-1, -1, -1, 0};
         return;
     }
 
-    unsigned char* base = smem_raw;
-    uint32_t* clT = reinterpret_cast<uint32_t*>(base);  base += align16((size_t)n_req * 4);
-    IdxT* ord = reinterpret_cast<IdxT*>(base);          base += align16((size_t)n_req * sizeof(IdxT));
-    IdxT* cl = reinterpret_cast<IdxT*>(base);           base += align16((size_t)n_req * sizeof(IdxT));
-    uint8_t* bins = reinterpret_cast<uint8_t*>(base);   base += align16((size_t)n_req);
-    uint32_t* cnt = reinterpret_cast<uint32_t*>(base);
+    uint32_t* clT = ws_T + unit * n_pad;                   // T of the members, CSR order
+    IdxT* clI = ws_I + unit * n_pad;                       // request index of the members, CSR order
+    uint32_t* cnt = reinterpret_cast<uint32_t*>(smem_raw);
 
     const uint32_t* gT = T_sorted + (size_t)inst * n_pad;
     const uint32_t* gO = order + (size_t)inst * n_pad;
-    for (int j = threadIdx.x; j < n_clients; j += SORT_THREADS) s_load[j] = load_from_assign ? 0 : ld[j];
+    for (int j = threadIdx.x; j < n_clients; j += LS_THREADS) s_load[j] = load_from_assign ? 0 : ld[j];
     __syncthreads();
-    bool bad_assign = false;
-    for (int r = threadIdx.x; r < n_req; r += SORT_THREADS) {
-        const uint32_t t = gT[r], id = gO[r];
-        const int c = asg[id];
-        ord[r] = (IdxT)id;
-        if (c < 0 || c >= n_clients) { bad_assign = true; bins[r] = 0; }
-        else {
-            bins[r] = (uint8_t)c;
-            if (load_from_assign) atomicAdd(reinterpret_cast<unsigned long long*>(&s_load[c]), (unsigned long long)t);
-        }
-    }
-    if (__syncthreads_or(bad_assign)) {
+    if (build_member_lists<IdxT, true>(asg, gO, gT, clI, clT, n_req, n_clients, cnt, s_wsum, s_off,
+                                       load_from_assign ? s_load : nullptr)) {
         if (threadIdx.x == 0) {
             atomicOr(&status_out[inst], HOS_ST_INVALID);
             rounds_applied[unit] = 0;
             makespan_out[unit] = 0;
         }
-        for (int j = threadIdx.x; j < n_clients; j += SORT_THREADS) ld[j] = 0;
+        for (int j = threadIdx.x; j < n_clients; j += LS_THREADS) ld[j] = 0;
         if (log)
-            for (int r = threadIdx.x; r < rounds; r += SORT_THREADS) log[r] = hos_ls_move{-1, -1, -1, 0};
+            for (int r = threadIdx.x; r < rounds; r += LS_THREADS) log[r] = hos_ls_move{-1, -1, -1, 0};
         return;
     }
-    build_member_lists<IdxT>(bins, gT, cl, clT, n_req, n_clients, cnt, s_wsum, s_off);
 
     int applied = 0;
     int done_at = rounds;
@@ -484,7 +504,7 @@ k_local_search(const uint32_t* __restrict__ T_sorted, const uint32_t* __restrict
         }
         if (lane == 0) { s_jmax = bj; s_lmax = bl; s_kmin = mj; }
     };
-    // warp 0: the clients a round looks at first, with the running count of their work items (see (b))
+    // warp 0: the clients a round looks at, with the running count of their work items (see (b))
     auto list_clients = [&](int jmax, long long Lmax, long long vlimit, bool skip_listed) {
         int n_alive = 0, n_items = 0;
         for (int k0 = 0; k0 < n_clients; k0 += 32) {
@@ -509,11 +529,13 @@ k_local_search(const uint32_t* __restrict__ T_sorted, const uint32_t* __restrict
                 const int pos = n_alive + __popc(am & ((1u << lane) - 1u));
                 s_ak[pos] = (uint8_t)k;
                 s_as[pos] = n_items + inc - sz;
+                s_cb[pos] = s_off[k];
+                s_cs[pos] = (uint32_t)(Lmax - s_load[k]);
             }
             n_alive += __popc(am);
             n_items += __shfl_sync(FULL, inc, 31);
         }
-        if (lane == 0) { s_na = n_alive; s_nitems = n_items; }
+        if (lane == 0) { s_na = n_alive; s_nitems = n_items; s_as[n_alive] = n_items; }
     };
     if (warp == 0) find_extremes();
     __syncthreads();
@@ -523,21 +545,19 @@ k_local_search(const uint32_t* __restrict__ T_sorted, const uint32_t* __restrict
         const long long Lmax = s_lmax;
         // all loads equal: the least loaded client is as loaded as the critical one; nothing can improve
         const int kmin = (s_kmin != jmax && s_load[s_kmin] < Lmax) ? s_kmin : -1;
-        const IdxT* mem = cl + s_off[jmax];                 // jmax's members, T descending
-        const uint32_t* memT = clT + s_off[jmax];
-        const int nm = s_off[jmax + 1] - s_off[jmax];
+        const int base_j = s_off[jmax];
+        const int nm = s_off[jmax + 1] - base_j;            // jmax's members, T descending
+        // short critical list and loads below 2^31: the list is copied to shared memory and the
+        // evaluation runs in 32-bit arithmetic; otherwise the general form reads it in place
+        const bool fast = nm >= 1 && nm < LS_STAGE && Lmax <= 0x7FFFFFFFll;
+        const int top = fast ? 1 << (31 - __clz(nm)) : 0;  // largest power of two <= nm
 
-        // (a) one work item: client k, position idx in its list (idx == its length: the move)
-        auto evaluate = [&](int k, int idx, int len, Cand& best) {
-            const long long lk = s_load[k];
-            const long long slack = Lmax - lk;
-            uint32_t u1 = 0;
-            int pu = -1;
-            long long Tu = 0;
-            if (idx < len) {
-                const int at = s_off[k] + idx;
-                u1 = (uint32_t)ord[cl[at]] + 1u; pu = idx; Tu = clT[at];
-            }
+        // (a) one work item: partner (Tu, u1 = u + 1, position pu; the move has Tu = 0, u1 = 0,
+        //     pu = -1) on client k, against jmax's list (memT, memI)
+        auto evaluate = [&](const uint32_t* memT, const IdxT* memI, int k, uint32_t Tu32, uint32_t u1, int pu,
+                            Cand& best) {
+            const long long slack = Lmax - s_load[k];
+            const long long Tu = Tu32;
             const long long thr64 = Tu + ((slack + 1) >> 1);    // T_i >= thr  <=>  2 d >= slack
             const uint32_t thr = (uint32_t)thr64;
             int a = 0, z = thr64 > 0xFFFFFFFFll ? 0 : nm;       // b = members with T >= thr (none if it
@@ -560,7 +580,7 @@ k_local_search(const uint32_t* __restrict__ T_sorted, const uint32_t* __restrict
                         }
                     }
                     Cand c;                                     // v = lk + d, Lmax - v = slack - d
-                    c.inv = ~(uint32_t)(slack - d); c.pi = a2; c.ik = ((uint32_t)ord[mem[a2]] << 8) | (uint32_t)k;
+                    c.inv = ~(uint32_t)(slack - d); c.pi = a2; c.ik = ((uint32_t)memI[a2] << 8) | (uint32_t)k;
                     c.u1 = u1; c.pu = pu;
                     if (cand_less(c, best)) best = c;
                 }
@@ -569,7 +589,7 @@ k_local_search(const uint32_t* __restrict__ T_sorted, const uint32_t* __restrict
                 const long long d = (long long)memT[b] - Tu;
                 if (d > 0) {
                     Cand c;                                     // v = Lmax - d
-                    c.inv = ~(uint32_t)d; c.pi = b; c.ik = ((uint32_t)ord[mem[b]] << 8) | (uint32_t)k;
+                    c.inv = ~(uint32_t)d; c.pi = b; c.ik = ((uint32_t)memI[b] << 8) | (uint32_t)k;
                     c.u1 = u1; c.pu = pu;
                     if (cand_less(c, best)) best = c;
                 }
@@ -581,40 +601,110 @@ k_local_search(const uint32_t* __restrict__ T_sorted, const uint32_t* __restrict
         //     clients whose floor is within `margin` of the least loaded client's; after the
         //     reduction, any client left out whose floor does not exceed the best v found is
         //     evaluated in a second pass (vlimit = that v), which makes the result exact whatever
-        //     the margin was.
+        //     the margin was.  A thread fetches its next item's partner before it works on the
+        //     current one, so the list reads overlap the searches.
         auto evaluate_listed = [&](Cand& best) {
-            const int n_alive = s_na, n_items = s_nitems;
-            for (int x = threadIdx.x; x < n_items; x += SORT_THREADS) {
-                int a = 0, z = n_alive;                         // last listed client with start <= x
-                while (z - a > 1) {
-                    const int mid = (a + z) >> 1;
-                    if (s_as[mid] <= x) a = mid; else z = mid;
+            const int n_items = s_nitems;
+            const uint32_t* memT = clT + base_j;
+            const IdxT* memI = clI + base_j;
+            int ci = 0;
+            for (int x = threadIdx.x; x < n_items; x += LS_THREADS) {
+                while (x >= s_as[ci + 1]) ++ci;                 // s_as[n_alive] = n_items ends the walk
+                const int k = s_ak[ci], idx = x - s_as[ci], at = s_cb[ci] + idx;
+                if (x + 1 < s_as[ci + 1]) evaluate(memT, memI, k, clT[at], (uint32_t)clI[at] + 1u, idx, best);
+                else evaluate(memT, memI, k, 0u, 0u, -1, best);
+            }
+        };
+        // The same over the shared-memory copy.  A = s_T + 1 holds the members' T, then zeros up to
+        // 2 * top entries, and A[-1] is all ones: the number of members with T >= thr comes from
+        // a fixed sequence of probes without bounds tests, and both neighbours of the turning point
+        // can be read unconditionally (the guard values never make a valid step).  Only an item
+        // that reaches the thread's best v so far builds a full candidate.
+        auto count_ge = [&](uint32_t thr) {
+            int cnt_ge = 0;
+            for (int step = top; step > 0; step >>= 1)
+                if (s_T[cnt_ge + step] >= thr) cnt_ge += step;   // A[cnt_ge + step - 1]
+            return cnt_ge;
+        };
+        auto evaluate_listed_fast = [&](Cand& best) {
+            const int n_items = s_nitems;
+            int ci = 0;
+            int x = threadIdx.x;
+            uint32_t Tu = 0;
+            bool is_move = false;
+            auto locate = [&](int xx) {
+                while (xx >= s_as[ci + 1]) ++ci;
+                is_move = xx + 1 == s_as[ci + 1];
+                Tu = is_move ? 0u : clT[s_cb[ci] + (xx - s_as[ci])];
+            };
+            if (x < n_items) locate(x);
+            while (x < n_items) {
+                const int c0 = ci;
+                const uint32_t Tu0 = Tu;
+                const bool move0 = is_move;
+                const int xn = x + LS_THREADS;
+                if (xn < n_items) locate(xn);                   // next item's partner, in flight during this one
+                const uint32_t slack = s_cs[c0];
+                const int b = count_ge(Tu0 + ((slack + 1u) >> 1));
+                const uint32_t Ti = s_T[b];                     // A[b - 1]: smallest T >= thr (rising side)
+                const uint32_t d = Ti - Tu0;
+                const uint32_t inv_r = d < slack ? ~(slack - d) : NO_CAND;
+                const int d2 = (int)(s_T[b + 1] - Tu0);         // A[b]: largest T < thr (falling side)
+                const uint32_t inv_f = d2 > 0 ? ~(uint32_t)d2 : NO_CAND;
+                const uint32_t m = min(inv_r, inv_f);
+                if (m != NO_CAND && m <= best.inv) {
+                    const int idx = x - s_as[c0];
+                    const uint32_t k = s_ak[c0];
+                    Cand c;
+                    c.u1 = move0 ? 0u : (uint32_t)clI[s_cb[c0] + idx] + 1u;
+                    c.pu = move0 ? -1 : idx;
+                    if (inv_r != NO_CAND && inv_r <= best.inv) {
+                        c.inv = inv_r; c.pi = count_ge(Ti + 1u);  // first member of the run of equal T
+                        c.ik = ((uint32_t)s_I[c.pi] << 8) | k;
+                        if (cand_less(c, best)) best = c;
+                    }
+                    if (inv_f != NO_CAND && inv_f <= best.inv) {
+                        c.inv = inv_f; c.pi = b;
+                        c.ik = ((uint32_t)s_I[b] << 8) | k;
+                        if (cand_less(c, best)) best = c;
+                    }
                 }
-                const int k = s_ak[a];
-                evaluate(k, x - s_as[a], s_off[k + 1] - s_off[k], best);
+                x = xn;
             }
         };
         Cand best;
         best.inv = NO_CAND; best.ik = NO_CAND; best.u1 = NO_CAND; best.pi = -1; best.pu = -1;
         const long long floor_min = kmin >= 0 ? ((Lmax + s_load[kmin] + 1) >> 1) : Lmax;
         if (warp == 0) list_clients(jmax, Lmax, floor_min + margin, false);
+        else if (fast)
+            for (int x = threadIdx.x - 32; x <= 2 * top; x += LS_THREADS - 32) {
+                s_T[x] = x == 0 ? 0xFFFFFFFFu : (x <= nm ? clT[base_j + x - 1] : 0u);
+                if (x < nm) s_I[x] = clI[base_j + x];
+            }
         __syncthreads();
         long long best_v = Lmax;
         for (int pass = 0; pass < 2; ++pass) {
-            evaluate_listed(best);
-            // CTA-wide lexicographic minimum: per warp, then every warp reduces the 32 records
+            if (fast) evaluate_listed_fast(best);
+            else evaluate_listed(best);
+            // CTA-wide lexicographic minimum: per warp, then every warp reduces the warps' records
             best = cand_warp_min(best);
             if (lane == 0) s_cand[warp] = best;
             __syncthreads();
-            best = cand_warp_min(s_cand[lane]);
+            {
+                Cand mine;
+                mine.inv = NO_CAND; mine.ik = NO_CAND; mine.u1 = NO_CAND; mine.pi = -1; mine.pu = -1;
+                if (lane < LS_WARPS) mine = s_cand[lane];
+                best = cand_warp_min(mine);
+            }
             best_v = best.inv != NO_CAND ? Lmax - (long long)(~best.inv) : Lmax;
             if (pass == 1) break;
             // is a client that was left out still able to reach best_v?
             bool missed = false;
-            if (threadIdx.x < n_clients && (int)threadIdx.x != jmax && !s_listed[threadIdx.x]) {
-                const long long lk = s_load[threadIdx.x];
-                missed = lk < Lmax && ((Lmax + lk + 1) >> 1) <= best_v;
-            }
+            for (int kk = threadIdx.x; kk < n_clients; kk += LS_THREADS)
+                if (kk != jmax && !s_listed[kk]) {
+                    const long long lk = s_load[kk];
+                    missed |= lk < Lmax && ((Lmax + lk + 1) >> 1) <= best_v;
+                }
             if (!__syncthreads_or(missed)) break;
             if (warp == 0) list_clients(jmax, Lmax, best_v, true);
             __syncthreads();
@@ -629,70 +719,40 @@ k_local_search(const uint32_t* __restrict__ T_sorted, const uint32_t* __restrict
         const int best_k = (int)(best.ik & 0xFFu);
         const int best_i = (int)(best.ik >> 8);
         const int best_u = (int)best.u1 - 1;
-        // (c) apply.  Warp 0 updates the two loads and finds the next round's extremes while the
-        //     other warps patch the member lists (a swap keeps both list lengths).
-        const int ri = (int)mem[best.pi];
-        const int ru = best.pu >= 0 ? (int)cl[s_off[best_k] + best.pu] : -1;
-        const uint32_t Ti_w = memT[best.pi];
-        const uint32_t Tu_w = best.pu >= 0 ? clT[s_off[best_k] + best.pu] : 0u;
-        const long long dT = (long long)Ti_w - (long long)Tu_w;
-        ListPatch<IdxT> pp;
-        IdxT* seg = nullptr;
-        uint32_t* segT = nullptr;
-        IdxT keep[4];
-        uint32_t keepT[4];
-        int nk = 0, gtid = 0, val = 0;
-        uint32_t valT = 0;
-        bool big = false;
-        constexpr int GROUP = (SORT_THREADS - 64) / 2;          // threads per list: warps 2..16 and 17..31
-        const bool patcher = best.pu >= 0 && warp >= 2;
-        if (patcher) {
-            const bool first = (int)threadIdx.x - 64 < GROUP;
-            seg = cl + s_off[first ? jmax : best_k];
-            segT = clT + s_off[first ? jmax : best_k];
-            const int len = first ? nm : s_off[best_k + 1] - s_off[best_k];
-            const int gone = first ? best.pi : best.pu;
-            val = first ? ru : ri;
-            valT = first ? Tu_w : Ti_w;
-            pp = patch_plan<IdxT>(seg, len, gone, val);
-            gtid = ((int)threadIdx.x - 64) % GROUP;
-            big = pp.dst_hi - pp.dst_lo > 4 * GROUP;            // generic path for very long ranges
-            if (!big)
-                for (int x = pp.dst_lo + gtid; x < pp.dst_hi; x += GROUP) { keep[nk] = seg[x]; keepT[nk] = segT[x]; ++nk; }
-        } else if (warp == 0) {
+        // (c) apply.  Warp 0 updates the two loads and finds the next round's extremes, warp 1
+        //     writes the assignment and the log, warps 2 and 3 patch one member list each.
+        const int base_k = s_off[best_k];
+        const uint32_t Ti_w = clT[base_j + best.pi];            // read by every warp before any list changes
+        const uint32_t Tu_w = best.pu >= 0 ? clT[base_k + best.pu] : 0u;
+        __syncthreads();
+        if (warp == 0) {
+            const long long dT = (long long)Ti_w - (long long)Tu_w;
             if (lane == 0) { s_load[jmax] -= dT; s_load[best_k] += dT; }
             __syncwarp();
             find_extremes();
-        } else if (threadIdx.x == 32) {
-            asg[best_i] = best_k;
-            if (ru >= 0) asg[best_u] = jmax;
-            if (log) log[round] = hos_ls_move{best_i, best_u, best_k, best_v};
-        }
-        __syncthreads();
-        if (patcher) {
-            if (!big) {
-                nk = 0;
-                for (int x = pp.dst_lo + gtid; x < pp.dst_hi; x += GROUP) { seg[x + pp.shift] = keep[nk]; segT[x + pp.shift] = keepT[nk]; ++nk; }
-            } else if (gtid == 0) {                             // serial shift, direction-safe
-                if (pp.shift < 0) for (int x = pp.dst_lo; x < pp.dst_hi; ++x) { seg[x - 1] = seg[x]; segT[x - 1] = segT[x]; }
-                else for (int x = pp.dst_hi - 1; x >= pp.dst_lo; --x) { seg[x + 1] = seg[x]; segT[x + 1] = segT[x]; }
+        } else if (warp == 1) {
+            if (lane == 0) {
+                asg[best_i] = best_k;
+                if (best_u >= 0) asg[best_u] = jmax;
+                if (log) log[round] = hos_ls_move{best_i, best_u, best_k, best_v};
             }
-            if (gtid == 0) { seg[pp.at] = (IdxT)val; segT[pp.at] = valT; }   // never a destination of the shift
-        }
-        if (threadIdx.x == 0) {
-            bins[ri] = (uint8_t)best_k;
-            if (ru >= 0) bins[ru] = (uint8_t)jmax;
+        } else if (best.pu >= 0) {
+            if (warp == 2) warp_patch_list<IdxT>(clT + base_j, clI + base_j, nm, best.pi, Tu_w, (uint32_t)best_u);
+            else if (warp == 3)
+                warp_patch_list<IdxT>(clT + base_k, clI + base_k, s_off[best_k + 1] - base_k, best.pu, Ti_w,
+                                      (uint32_t)best_i);
         }
         __syncthreads();
-        if (best.pu < 0) build_member_lists<IdxT>(bins, gT, cl, clT, n_req, n_clients, cnt, s_wsum, s_off);
+        if (best.pu < 0)
+            build_member_lists<IdxT, false>(asg, gO, gT, clI, clT, n_req, n_clients, cnt, s_wsum, s_off, nullptr);
         ++applied;
     }
     // a round without an improving step leaves the state as it is: all later rounds are the same
     if (log && done_at < rounds) {
         const hos_ls_move noop = hos_ls_move{-1, -1, -1, s_lmax};
-        for (int r = done_at + 1 + threadIdx.x; r < rounds; r += SORT_THREADS) log[r] = noop;
+        for (int r = done_at + 1 + threadIdx.x; r < rounds; r += LS_THREADS) log[r] = noop;
     }
-    for (int j = threadIdx.x; j < n_clients; j += SORT_THREADS) { ld[j] = s_load[j]; }
+    for (int j = threadIdx.x; j < n_clients; j += LS_THREADS) { ld[j] = s_load[j]; }
     if (warp == 0) {
         long long mx = 0;
         for (int j = lane; j < n_clients; j += 32) mx = s_load[j] > mx ? s_load[j] : mx;
@@ -783,17 +843,12 @@ k_lower_bound(const uint32_t* __restrict__ p, const uint32_t* __restrict__ o, in
 // ---------------------------------------------------------------------------------------
 // launchers
 // ---------------------------------------------------------------------------------------
-static size_t ls_smem_bytes(int n_req, int n_clients, size_t isz) {
-    return align16((size_t)n_req * 4) + 2 * align16((size_t)n_req * isz) + align16((size_t)n_req) +
-           (size_t)n_clients * SORT_WARPS * 4;
-}
 
 size_t estimate_sort_smem(int n_req) {
     return n_req <= 65536 ? sort_smem_bytes<uint16_t>(n_req) : sort_smem_bytes<uint32_t>(n_req);
 }
-size_t local_search_smem(int n_req, int n_clients) {
-    return ls_smem_bytes(n_req, n_clients, n_req <= 65536 ? 2 : 4);
-}
+size_t local_search_smem(int /*n_req*/, int n_clients) { return (size_t)n_clients * LS_WARPS * 4; }
+size_t local_search_index_bytes(int n_req) { return n_req <= 65536 ? 2 : 4; }
 
 cudaError_t launch_estimate_sort(const hos_batch& b, const hos_cost_model& cm, uint32_t* T_sorted,
                                  uint32_t* order, InstInfo* info, int32_t* status_out, int n_pad,
@@ -831,16 +886,17 @@ cudaError_t launch_local_search(const hos_batch& b, const uint32_t* T_sorted, co
                                 const InstInfo* info, int n_pad, int n_copies, int rounds,
                                 bool load_from_assign, int32_t* assign, long long* load,
                                 long long* makespan, int32_t* rounds_applied, hos_ls_move* ls_log,
-                                int32_t* status, cudaStream_t st) {
+                                int32_t* status, uint32_t* ws_T, void* ws_I, cudaStream_t st) {
     const size_t smem = local_search_smem(b.n_req, b.n_clients);
-    auto kern = b.n_req <= 65536 ? k_local_search<uint16_t> : k_local_search<uint32_t>;
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return e;
     launch_hook("k_local_search", 0, st);
-    kern<<<b.n_inst * n_copies, SORT_THREADS, smem, st>>>(T_sorted, order, info, b.n_req, n_pad,
-                                                          b.n_clients, n_copies, rounds,
-                                                          load_from_assign, assign, load, makespan,
-                                                          rounds_applied, ls_log, status);
+    if (b.n_req <= 65536)
+        k_local_search<uint16_t><<<b.n_inst * n_copies, LS_THREADS, smem, st>>>(
+            T_sorted, order, info, b.n_req, n_pad, b.n_clients, n_copies, rounds, load_from_assign, assign,
+            load, makespan, rounds_applied, ls_log, status, ws_T, static_cast<uint16_t*>(ws_I));
+    else
+        k_local_search<uint32_t><<<b.n_inst * n_copies, LS_THREADS, smem, st>>>(
+            T_sorted, order, info, b.n_req, n_pad, b.n_clients, n_copies, rounds, load_from_assign, assign,
+            load, makespan, rounds_applied, ls_log, status, ws_T, static_cast<uint32_t*>(ws_I));
     launch_hook("k_local_search", 1, st);
     return cudaGetLastError();
 }

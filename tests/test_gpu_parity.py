@@ -124,6 +124,20 @@ def test_local_search_from_bad_assignments(hos):
                 assert np.array_equal(log[k, c][f], elog[f])
 
 
+@pytest.mark.parametrize("n,M,scale", [(1530, 3, 1), (1024, 2, 1), (900, 5, 1), (600, 4, 10000)])
+def test_local_search_short_list_and_general_forms(hos, n, M, scale):
+    # member lists around the length up to which the critical client's list is evaluated from
+    # on-chip memory (511), and loads above 2^31 (scale), which take the 64-bit form
+    rng = np.random.default_rng(n + M)
+    n_inst = 2
+    p = rng.integers(1, 3000, size=(n_inst, n)).astype(np.uint32)
+    o = rng.integers(1, 800, size=(n_inst, n)).astype(np.uint32)
+    p[:, ::9] = p[:, 1:2]                                            # runs of equal T
+    o[:, ::9] = o[:, 1:2]
+    cm = (20000, 40, 15000, 300 * scale, 16, 40 * scale, 350 * scale)
+    H.check_offline(hos, p, o, M, 16, 10 ** 7, cm, 60)
+
+
 def test_wide_estimates_take_the_64bit_packing_path(hos):
     # T_i up to ~2^31: the packed 32-bit load keys cannot be used
     rng = np.random.default_rng(5)
