@@ -292,6 +292,7 @@ constexpr int NO_I = 0x7FFFFFFF;
 constexpr int LS_THREADS = 128;
 constexpr int LS_WARPS = LS_THREADS / 32;
 constexpr int LS_STAGE = 512;             // longest critical list that is copied to shared memory
+constexpr int LS_BATCH = 4;               // work items a thread has in flight
 
 // Exclusive scan of a[0 .. len) in place by the whole CTA; `wsum` holds LS_WARPS words.
 __device__ inline void block_scan_u32(uint32_t* a, int len, uint32_t* wsum) {
@@ -618,8 +619,11 @@ k_local_search(const uint32_t* __restrict__ T_sorted, const uint32_t* __restrict
         // The same over the shared-memory copy.  A = s_T + 1 holds the members' T, then zeros up to
         // 2 * top entries, and A[-1] is all ones: the number of members with T >= thr comes from
         // a fixed sequence of probes without bounds tests, and both neighbours of the turning point
-        // can be read unconditionally (the guard values never make a valid step).  Only an item
-        // that reaches the thread's best v so far builds a full candidate.
+        // can be read unconditionally (the guard values never make a valid step).  A thread takes
+        // LS_BATCH items at a time: their partners' T are fetched together, one batch ahead of their
+        // use, and the searches of a batch advance side by side, so that neither the list reads nor
+        // the probe chains are waited for one by one.  The partner's request index is read only
+        // when (v, i, k) ties, or at the end for the thread's best step.
         auto count_ge = [&](uint32_t thr) {
             int cnt_ge = 0;
             for (int step = top; step > 0; step >>= 1)
@@ -628,49 +632,76 @@ k_local_search(const uint32_t* __restrict__ T_sorted, const uint32_t* __restrict
         };
         auto evaluate_listed_fast = [&](Cand& best) {
             const int n_items = s_nitems;
-            int ci = 0;
-            int x = threadIdx.x;
-            uint32_t Tu = 0;
-            bool is_move = false;
-            auto locate = [&](int xx) {
-                while (xx >= s_as[ci + 1]) ++ci;
-                is_move = xx + 1 == s_as[ci + 1];
-                Tu = is_move ? 0u : clT[s_cb[ci] + (xx - s_as[ci])];
+            int best_at = -1;                                   // where the best partner's index is, if not read yet
+            auto consider = [&](uint32_t inv, int pi, uint32_t k, bool move, int at, int idx) {
+                const uint32_t ik = ((uint32_t)s_I[pi] << 8) | k;
+                if (inv < best.inv || (inv == best.inv && ik < best.ik)) {
+                    best.inv = inv; best.ik = ik; best.pi = pi; best.pu = move ? -1 : idx;
+                    best.u1 = 0u; best_at = move ? -1 : at;
+                } else if (inv == best.inv && ik == best.ik) {
+                    if (best_at >= 0) { best.u1 = (uint32_t)clI[best_at] + 1u; best_at = -1; }
+                    const uint32_t u1 = move ? 0u : (uint32_t)clI[at] + 1u;
+                    if (u1 < best.u1) { best.pi = pi; best.pu = move ? -1 : idx; best.u1 = u1; }
+                }
             };
-            if (x < n_items) locate(x);
-            while (x < n_items) {
-                const int c0 = ci;
-                const uint32_t Tu0 = Tu;
-                const bool move0 = is_move;
-                const int xn = x + LS_THREADS;
-                if (xn < n_items) locate(xn);                   // next item's partner, in flight during this one
-                const uint32_t slack = s_cs[c0];
-                const int b = count_ge(Tu0 + ((slack + 1u) >> 1));
-                const uint32_t Ti = s_T[b];                     // A[b - 1]: smallest T >= thr (rising side)
-                const uint32_t d = Ti - Tu0;
-                const uint32_t inv_r = d < slack ? ~(slack - d) : NO_CAND;
-                const int d2 = (int)(s_T[b + 1] - Tu0);         // A[b]: largest T < thr (falling side)
-                const uint32_t inv_f = d2 > 0 ? ~(uint32_t)d2 : NO_CAND;
-                const uint32_t m = min(inv_r, inv_f);
-                if (m != NO_CAND && m <= best.inv) {
-                    const int idx = x - s_as[c0];
-                    const uint32_t k = s_ak[c0];
-                    Cand c;
-                    c.u1 = move0 ? 0u : (uint32_t)clI[s_cb[c0] + idx] + 1u;
-                    c.pu = move0 ? -1 : idx;
-                    if (inv_r != NO_CAND && inv_r <= best.inv) {
-                        c.inv = inv_r; c.pi = count_ge(Ti + 1u);  // first member of the run of equal T
-                        c.ik = ((uint32_t)s_I[c.pi] << 8) | k;
-                        if (cand_less(c, best)) best = c;
-                    }
-                    if (inv_f != NO_CAND && inv_f <= best.inv) {
-                        c.inv = inv_f; c.pi = b;
-                        c.ik = ((uint32_t)s_I[b] << 8) | k;
-                        if (cand_less(c, best)) best = c;
+            int ci = 0;
+            uint32_t nTu[LS_BATCH];                             // next batch: partner T (0 for the move),
+            int nci[LS_BATCH];                                  // listed-client slot (-1: no item)
+            auto fetch = [&](int x0) {
+#pragma unroll
+                for (int u = 0; u < LS_BATCH; ++u) {
+                    const int xx = x0 + u * LS_THREADS;
+                    nci[u] = -1; nTu[u] = 0u;
+                    if (xx < n_items) {
+                        while (xx >= s_as[ci + 1]) ++ci;        // s_as[n_alive] = n_items ends the walk
+                        nci[u] = ci;
+                        if (xx + 1 != s_as[ci + 1]) nTu[u] = clT[s_cb[ci] + (xx - s_as[ci])];
                     }
                 }
-                x = xn;
+            };
+            int x0 = threadIdx.x;
+            if (x0 < n_items) fetch(x0);
+            while (x0 < n_items) {
+                uint32_t Tu[LS_BATCH], thr[LS_BATCH], slack[LS_BATCH];
+                int cs[LS_BATCH], b[LS_BATCH];
+#pragma unroll
+                for (int u = 0; u < LS_BATCH; ++u) {
+                    Tu[u] = nTu[u]; cs[u] = nci[u];
+                    slack[u] = cs[u] >= 0 ? s_cs[cs[u]] : 0u;
+                    thr[u] = Tu[u] + ((slack[u] + 1u) >> 1);
+                    b[u] = 0;
+                }
+                const int xn = x0 + LS_BATCH * LS_THREADS;
+                if (xn < n_items) fetch(xn);                    // in flight during this batch's searches
+                for (int step = top; step > 0; step >>= 1) {
+#pragma unroll
+                    for (int u = 0; u < LS_BATCH; ++u)
+                        if (s_T[b[u] + step] >= thr[u]) b[u] += step;
+                }
+#pragma unroll
+                for (int u = 0; u < LS_BATCH; ++u) {
+                    if (cs[u] < 0) continue;
+                    const uint32_t Ti = s_T[b[u]];              // A[b - 1]: smallest T >= thr (rising side)
+                    const uint32_t d = Ti - Tu[u];
+                    const uint32_t inv_r = d < slack[u] ? ~(slack[u] - d) : NO_CAND;
+                    const int d2 = (int)(s_T[b[u] + 1] - Tu[u]);   // A[b]: largest T < thr (falling side)
+                    const uint32_t inv_f = d2 > 0 ? ~(uint32_t)d2 : NO_CAND;
+                    if (min(inv_r, inv_f) > best.inv) continue; // NO_CAND is the largest value
+                    const int xx = x0 + u * LS_THREADS;
+                    const int idx = xx - s_as[cs[u]];
+                    const bool move = xx + 1 == s_as[cs[u] + 1];
+                    const int at = s_cb[cs[u]] + idx;
+                    const uint32_t k = s_ak[cs[u]];
+                    if (inv_r != NO_CAND && inv_r <= best.inv) {
+                        // first member of the run of equal T: b - 1 itself unless its predecessor ties
+                        const int pi = s_T[b[u] - 1] != Ti ? b[u] - 1 : count_ge(Ti + 1u);
+                        consider(inv_r, pi, k, move, at, idx);
+                    }
+                    if (inv_f != NO_CAND && inv_f <= best.inv) consider(inv_f, b[u], k, move, at, idx);
+                }
+                x0 = xn;
             }
+            if (best_at >= 0) best.u1 = (uint32_t)clI[best_at] + 1u;
         };
         Cand best;
         best.inv = NO_CAND; best.ik = NO_CAND; best.u1 = NO_CAND; best.pi = -1; best.pu = -1;
