@@ -57,6 +57,7 @@ struct OfflineWs {
     InstInfo* info;
     uint32_t* ls_T;             // local search, per (instance, copy): the member lists' T
     void* ls_I;                 // and request indices
+    uint8_t* ls_C;              // and the client of every rank of the sorted order
     size_t bytes;
 };
 OfflineWs carve_offline(const hos_batch* b, void* ws, int n_copies, int ls_rounds) {
@@ -67,11 +68,12 @@ OfflineWs carve_offline(const hos_batch* b, void* ws, int n_copies, int ls_round
     w.T_sorted = reinterpret_cast<uint32_t*>(base + off); off += up(rows * 4);
     w.order = reinterpret_cast<uint32_t*>(base + off);    off += up(rows * 4);
     w.info = reinterpret_cast<InstInfo*>(base + off);     off += up((size_t)b->n_inst * sizeof(InstInfo));
-    w.ls_T = nullptr; w.ls_I = nullptr;
+    w.ls_T = nullptr; w.ls_I = nullptr; w.ls_C = nullptr;
     if (ls_rounds > 0) {
         const size_t units = rows * (size_t)(n_copies > 0 ? n_copies : 1);
         w.ls_T = reinterpret_cast<uint32_t*>(base + off);  off += up(units * 4);
         w.ls_I = base + off;                               off += up(units * local_search_index_bytes(b->n_req));
+        w.ls_C = base + off;                               off += up(units);
     }
     w.bytes = off;
     return w;
@@ -153,14 +155,14 @@ int hos_offline_pack(const hos_batch* b, const hos_cost_model* cm, int ls_rounds
     if (lb && (rc = cuda_rc(launch_lower_bound(*b, *cm, w.T_sorted, w.info, n_pad, lb, st)))) return rc;
     if ((rc = cuda_rc(launch_lpt(*b, w.T_sorted, w.order, w.info, n_pad, assign,
                                  reinterpret_cast<long long*>(load),
-                                 reinterpret_cast<long long*>(makespan_est), st))))
+                                 reinterpret_cast<long long*>(makespan_est), w.ls_C, st))))
         return rc;
     if (ls_rounds == 0)
         return cuda_rc(cudaMemsetAsync(rounds_applied, 0, (size_t)b->n_inst * sizeof(int32_t), st));
     return cuda_rc(launch_local_search(*b, w.T_sorted, w.order, w.info, n_pad, 1, ls_rounds, false, assign,
                                        reinterpret_cast<long long*>(load),
                                        reinterpret_cast<long long*>(makespan_est), rounds_applied,
-                                       ls_log, status, w.ls_T, w.ls_I, st));
+                                       ls_log, status, w.ls_T, w.ls_I, w.ls_C, st));
 }
 
 int hos_local_search(const hos_batch* b, const hos_cost_model* cm, int n_copies, int ls_rounds,
@@ -181,7 +183,7 @@ int hos_local_search(const hos_batch* b, const hos_cost_model* cm, int n_copies,
     return cuda_rc(launch_local_search(*b, w.T_sorted, w.order, w.info, n_pad, n_copies, ls_rounds, true,
                                        assign, reinterpret_cast<long long*>(load),
                                        reinterpret_cast<long long*>(makespan_est), rounds_applied,
-                                       ls_log, status, w.ls_T, w.ls_I, st));
+                                       ls_log, status, w.ls_T, w.ls_I, w.ls_C, st));
 }
 
 int hos_lower_bound(const hos_batch* b, const hos_cost_model* cm, hos_lb* out, int32_t* status, void* ws,

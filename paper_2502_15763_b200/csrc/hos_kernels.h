@@ -22,12 +22,12 @@ cudaError_t launch_estimate_sort(const hos_batch& b, const hos_cost_model& cm, u
                                  cudaStream_t st);
 cudaError_t launch_lpt(const hos_batch& b, const uint32_t* T_sorted, const uint32_t* order,
                        const InstInfo* info, int n_pad, int32_t* assign, long long* load,
-                       long long* makespan, cudaStream_t st);
+                       long long* makespan, uint8_t* rank_client, cudaStream_t st);
 cudaError_t launch_local_search(const hos_batch& b, const uint32_t* T_sorted, const uint32_t* order,
                                 const InstInfo* info, int n_pad, int n_copies, int rounds,
                                 bool load_from_assign, int32_t* assign, long long* load,
                                 long long* makespan, int32_t* rounds_applied, hos_ls_move* ls_log,
-                                int32_t* status, uint32_t* ws_T, void* ws_I, cudaStream_t st);
+                                int32_t* status, uint32_t* ws_T, void* ws_I, uint8_t* ws_C, cudaStream_t st);
 size_t local_search_index_bytes(int n_req);
 cudaError_t launch_lower_bound(const hos_batch& b, const hos_cost_model& cm, const uint32_t* T_sorted,
                                const InstInfo* info, int n_pad, hos_lb* out, cudaStream_t st);

@@ -7,6 +7,8 @@
 #include "hos_kernels.h"
 #include "hos_sort.cuh"
 
+#include <type_traits>
+
 namespace hos {
 
 // ---------------------------------------------------------------------------------------
@@ -72,7 +74,7 @@ __global__ void __launch_bounds__(32)
 k_lpt(const uint32_t* __restrict__ T_sorted, const uint32_t* __restrict__ order,
       const InstInfo* __restrict__ info, int n_req, int n_pad, int n_clients,
       int32_t* __restrict__ assign, long long* __restrict__ load_out,
-      long long* __restrict__ makespan_out) {
+      long long* __restrict__ makespan_out, uint8_t* __restrict__ rank_client) {
     constexpr int JB = (KPL == 1) ? 5 : (KPL == 2) ? 6 : (KPL == 4) ? 7 : 8;
     const int inst = blockIdx.x;
     const int lane = threadIdx.x;
@@ -86,6 +88,8 @@ k_lpt(const uint32_t* __restrict__ T_sorted, const uint32_t* __restrict__ order,
     }
     const uint32_t* Ts = T_sorted + (size_t)inst * n_pad;
     const uint32_t* od = order + (size_t)inst * n_pad;
+    // nullable: the client of the r-th request in sorted order, for the local search's list build
+    uint8_t* rc = rank_client ? rank_client + (size_t)inst * n_pad : nullptr;
 
     long long load[KPL];
 #pragma unroll
@@ -171,7 +175,10 @@ k_lpt(const uint32_t* __restrict__ T_sorted, const uint32_t* __restrict__ order,
                 if (lane >= pos && lane < pos + W) mine = jv;
                 pos += W;
             }
-            if (r < n_req) asg[rq] = (int32_t)mine;
+            if (r < n_req) {
+                asg[rq] = (int32_t)mine;
+                if (rc) rc[r] = (uint8_t)mine;
+            }
             // re-base: subtract the current least relative load from every real key
             uint32_t m = key[0];
 #pragma unroll
@@ -221,7 +228,10 @@ k_lpt(const uint32_t* __restrict__ T_sorted, const uint32_t* __restrict__ order,
                 for (int k = 0; k < KPL; ++k) load[k] += (own && (bj >> 5) == k) ? (long long)t : 0ll;
                 mine = (lane == sidx) ? (uint32_t)bj : mine;
             }
-            if (r < n_req) asg[rq] = (int32_t)mine;
+            if (r < n_req) {
+                asg[rq] = (int32_t)mine;
+                if (rc) rc[r] = (uint8_t)mine;
+            }
         }
     }
     long long mx = 0;
@@ -318,30 +328,55 @@ __device__ inline void block_scan_u32(uint32_t* a, int len, uint32_t* wsum) {
 
 // Member lists of all clients from the assignment: a stable split of the ranks 0..n-1 by
 // client, as the members' request index (clI) and T (clT).  cnt holds n_clients * LS_WARPS
-// words.  off[k] = start of client k's list, off[M] = n.  With CHECK, an assignment outside
-// [0, M) makes every thread return true (lists not built), and `load`, if given, receives the
-// clients' summed T.
-template <typename IdxT, bool CHECK>
-__device__ inline bool build_member_lists(const int32_t* asg, const uint32_t* __restrict__ gO,
+// words.  off[k] = start of client k's list, off[M] = n.  rcl[r] is the client of rank r: with
+// GATHER it is filled here from the assignment (asg[order[r]]), otherwise it was left by the
+// packing kernel.  With CHECK, an assignment outside [0, M) makes every thread return true
+// (lists not built), and `load`, if given, receives the clients' summed T.  Each warp takes
+// LS_ROWS rows of 32 ranks at a time, so that their reads are in flight together.
+constexpr int LS_ROWS = 4;
+template <typename IdxT, bool CHECK, bool GATHER>
+__device__ inline bool build_member_lists(const int32_t* asg, uint8_t* rcl, const uint32_t* __restrict__ gO,
                                           const uint32_t* __restrict__ gT, IdxT* clI, uint32_t* clT,
                                           int n, int n_clients, uint32_t* cnt, uint32_t* wsum, int* off,
                                           long long* load) {
     const int lane = lane_id(), warp = warp_id();
     const int chunk = (((n + LS_WARPS - 1) / LS_WARPS) + 31) & ~31;
     const int lo = warp * chunk, hi = min(n, lo + chunk);
-    const int nb = bit_width_u32((uint32_t)(n_clients - 1));
     for (int x = threadIdx.x; x < n_clients * LS_WARPS; x += LS_THREADS) cnt[x] = 0;
     __syncthreads();
     bool bad = false;
-    for (int row = lo; row < hi; row += 32) {
-        const int r = row + lane;
-        if (r < hi) {
-            const int c = asg[__ldg(&gO[r])];
-            if (CHECK && (c < 0 || c >= n_clients)) bad = true;
-            else {
-                atomicAdd(&cnt[(uint32_t)c * LS_WARPS + warp], 1u);
-                if (CHECK && load)
-                    atomicAdd(reinterpret_cast<unsigned long long*>(&load[c]), (unsigned long long)__ldg(&gT[r]));
+    for (int row = lo; row < hi; row += 32 * LS_ROWS) {
+        int c[LS_ROWS];
+        uint32_t t[LS_ROWS];
+        if (GATHER) {
+            uint32_t id[LS_ROWS];
+#pragma unroll
+            for (int e = 0; e < LS_ROWS; ++e) {
+                const int r = row + e * 32 + lane;
+                id[e] = r < hi ? __ldg(&gO[r]) : 0u;
+                t[e] = (CHECK && load && r < hi) ? __ldg(&gT[r]) : 0u;
+            }
+#pragma unroll
+            for (int e = 0; e < LS_ROWS; ++e) c[e] = row + e * 32 + lane < hi ? asg[id[e]] : 0;
+        } else {
+#pragma unroll
+            for (int e = 0; e < LS_ROWS; ++e) {
+                const int r = row + e * 32 + lane;
+                c[e] = r < hi ? (int)rcl[r] : 0;
+                t[e] = (CHECK && load && r < hi) ? __ldg(&gT[r]) : 0u;
+            }
+        }
+#pragma unroll
+        for (int e = 0; e < LS_ROWS; ++e) {
+            const int r = row + e * 32 + lane;
+            if (r < hi) {
+                if (CHECK && (c[e] < 0 || c[e] >= n_clients)) bad = true;
+                else {
+                    if (GATHER) rcl[r] = (uint8_t)c[e];
+                    atomicAdd(&cnt[(uint32_t)c[e] * LS_WARPS + warp], 1u);
+                    if (CHECK && load)
+                        atomicAdd(reinterpret_cast<unsigned long long*>(&load[c[e]]), (unsigned long long)t[e]);
+                }
             }
         }
     }
@@ -351,27 +386,30 @@ __device__ inline bool build_member_lists(const int32_t* asg, const uint32_t* __
     for (int k = threadIdx.x; k <= n_clients; k += LS_THREADS)
         off[k] = k < n_clients ? (int)cnt[k * LS_WARPS] : n;
     __syncthreads();
-    for (int row = lo; row < hi; row += 32) {
-        const int r = row + lane;
-        const bool valid = r < hi;
-        const uint32_t id = valid ? __ldg(&gO[r]) : 0u;
-        const uint32_t dig = valid ? (uint32_t)asg[id] : 0u;
-        const uint32_t tr = valid ? __ldg(&gT[r]) : 0u;
-        unsigned m = __ballot_sync(FULL, valid);             // lanes of this row on my client
-        for (int b = 0; b < nb; ++b) {
-            const bool bit = (dig >> b) & 1u;
-            const unsigned bal = __ballot_sync(FULL, bit);
-            m &= bit ? bal : ~bal;
+    for (int row = lo; row < hi; row += 32 * LS_ROWS) {
+        uint32_t id[LS_ROWS], tr[LS_ROWS], dig[LS_ROWS];
+#pragma unroll
+        for (int e = 0; e < LS_ROWS; ++e) {
+            const int r = row + e * 32 + lane;
+            const bool valid = r < hi;
+            id[e] = valid ? __ldg(&gO[r]) : 0u;
+            tr[e] = valid ? __ldg(&gT[r]) : 0u;
+            dig[e] = valid ? (uint32_t)rcl[r] : 0xFFFFFFFFu;      // (written above by this same thread)
         }
-        const uint32_t base = valid ? cnt[dig * LS_WARPS + warp] : 0u;
-        __syncwarp();
-        if (valid) {
-            const uint32_t at = base + __popc(m & ((1u << lane) - 1u));
-            clI[at] = (IdxT)id;
-            clT[at] = tr;
-            if (lane == (__ffs(m) - 1)) cnt[dig * LS_WARPS + warp] = base + __popc(m);
+#pragma unroll
+        for (int e = 0; e < LS_ROWS; ++e) {
+            const bool valid = row + e * 32 + lane < hi;
+            const unsigned m = __match_any_sync(FULL, dig[e]);   // lanes of this row on my client
+            const uint32_t base = valid ? cnt[dig[e] * LS_WARPS + warp] : 0u;
+            __syncwarp();
+            if (valid) {
+                const uint32_t at = base + __popc(m & ((1u << lane) - 1u));
+                clI[at] = (IdxT)id[e];
+                clT[at] = tr[e];
+                if (lane == (__ffs(m) - 1)) cnt[dig[e] * LS_WARPS + warp] = base + __popc(m);
+            }
+            __syncwarp();
         }
-        __syncwarp();
     }
     __syncthreads();
     return false;
@@ -416,28 +454,62 @@ __device__ inline void warp_patch_list(uint32_t* segT, IdxT* segI, int len, int 
     if (lane == 0) { segT[at] = valT; segI[at] = (IdxT)valI; }
 }
 
+// The clients one round looks at (see (b) in the kernel), double-buffered: the next round's list
+// is made while the current step is applied.
+struct LsListing {
+    int as[MAX_CLIENTS + 1];            // first work item of every listed client, then the total
+    int cb[MAX_CLIENTS];                // start of its member list
+    uint32_t cs[MAX_CLIENTS];           // Lmax - load (when that fits 32 bits)
+    uint8_t ak[MAX_CLIENTS];            // the client
+    long long min_unlisted;             // least floor among the clients left out
+    int na, nitems;
+};
+
+// b[u] += members with T >= thr[u], for LS_BATCH searches side by side.  A = s_T + 1 holds the
+// members' T (descending), then zeros up to 2^STEPS entries, and s_T[0] is all ones.
+template <int STEPS>
+__device__ __forceinline__ void count_ge_batch(const uint32_t* s_T, const uint32_t (&thr)[LS_BATCH],
+                                               int (&b)[LS_BATCH], int top) {
+    if (STEPS > 0) {
+#pragma unroll
+        for (int st = STEPS - 1; st >= 0; --st) {
+#pragma unroll
+            for (int u = 0; u < LS_BATCH; ++u)
+                if (s_T[b[u] + (1 << st)] >= thr[u]) b[u] += 1 << st;
+        }
+    } else {
+        for (int step = top; step > 0; step >>= 1) {
+#pragma unroll
+            for (int u = 0; u < LS_BATCH; ++u)
+                if (s_T[b[u] + step] >= thr[u]) b[u] += step;
+        }
+    }
+}
+
+// Named barrier 1 pairs warp 0 (which finds the next critical client) with warp 1 (which copies
+// that client's list) while the other warps patch the lists.
+__device__ __forceinline__ void pair_arrive() { asm volatile("bar.arrive 1, 64;" ::: "memory"); }
+__device__ __forceinline__ void pair_wait() { asm volatile("bar.sync 1, 64;" ::: "memory"); }
+
 template <typename IdxT>
-__global__ void __launch_bounds__(LS_THREADS, 8)
+__global__ void __launch_bounds__(LS_THREADS, 7)
 k_local_search(const uint32_t* __restrict__ T_sorted, const uint32_t* __restrict__ order,
                const InstInfo* __restrict__ info, int n_req, int n_pad, int n_clients,
                int n_copies, int rounds, bool load_from_assign,
                int32_t* __restrict__ assign, long long* __restrict__ load_io,
                long long* __restrict__ makespan_out, int32_t* __restrict__ rounds_applied,
                hos_ls_move* __restrict__ ls_log, int32_t* __restrict__ status_out,
-               uint32_t* __restrict__ ws_T, IdxT* __restrict__ ws_I) {
+               uint32_t* __restrict__ ws_T, IdxT* __restrict__ ws_I, uint8_t* __restrict__ ws_C) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     __shared__ long long s_load[MAX_CLIENTS];
     __shared__ int s_off[MAX_CLIENTS + 1];
     __shared__ Cand s_cand[LS_WARPS];
     __shared__ uint32_t s_wsum[LS_WARPS];
-    __shared__ int s_as[MAX_CLIENTS + 1];                   // listed clients: first work item (and the total),
-    __shared__ int s_cb[MAX_CLIENTS];                       // start of the member list,
-    __shared__ uint32_t s_cs[MAX_CLIENTS];                  // Lmax - load (when that fits 31 bits),
-    __shared__ uint8_t s_ak[MAX_CLIENTS];                   // client
+    __shared__ LsListing s_ls[2];
     __shared__ uint8_t s_listed[MAX_CLIENTS];
     __shared__ uint32_t s_T[LS_STAGE + 1];                  // [0] = all ones, [1 .. nm] = jmax's T, then zeros
     __shared__ IdxT s_I[LS_STAGE];                          // jmax's request indices
-    __shared__ int s_jmax, s_kmin, s_na, s_nitems;
+    __shared__ int s_jmax, s_kmin;
     __shared__ long long s_lmax;
 
     const int inst = blockIdx.x / n_copies;
@@ -461,14 +533,20 @@ k_local_search(const uint32_t* __restrict__ T_sorted, const uint32_t* __restrict
 
     uint32_t* clT = ws_T + unit * n_pad;                   // T of the members, CSR order
     IdxT* clI = ws_I + unit * n_pad;                       // request index of the members, CSR order
+    uint8_t* rcl = ws_C + unit * n_pad;                    // client of every rank in sorted order
     uint32_t* cnt = reinterpret_cast<uint32_t*>(smem_raw);
 
     const uint32_t* gT = T_sorted + (size_t)inst * n_pad;
     const uint32_t* gO = order + (size_t)inst * n_pad;
     for (int j = threadIdx.x; j < n_clients; j += LS_THREADS) s_load[j] = load_from_assign ? 0 : ld[j];
     __syncthreads();
-    if (build_member_lists<IdxT, true>(asg, gO, gT, clI, clT, n_req, n_clients, cnt, s_wsum, s_off,
-                                       load_from_assign ? s_load : nullptr)) {
+    // a caller's assignment is gathered and checked; the packing kernel's comes with the clients by rank
+    const bool lists_failed =
+        load_from_assign ? build_member_lists<IdxT, true, true>(asg, rcl, gO, gT, clI, clT, n_req, n_clients, cnt,
+                                                                s_wsum, s_off, s_load)
+                         : build_member_lists<IdxT, false, false>(asg, rcl, gO, gT, clI, clT, n_req, n_clients, cnt,
+                                                                  s_wsum, s_off, nullptr);
+    if (lists_failed) {
         if (threadIdx.x == 0) {
             atomicOr(&status_out[inst], HOS_ST_INVALID);
             rounds_applied[unit] = 0;
@@ -505,16 +583,20 @@ k_local_search(const uint32_t* __restrict__ T_sorted, const uint32_t* __restrict
         }
         if (lane == 0) { s_jmax = bj; s_lmax = bl; s_kmin = mj; }
     };
-    // warp 0: the clients a round looks at, with the running count of their work items (see (b))
-    auto list_clients = [&](int jmax, long long Lmax, long long vlimit, bool skip_listed) {
+    // One warp: the clients a round looks at, with the running count of their work items (see (b)).
+    // Without skip_listed it also leaves the least floor of the clients it left out.
+    auto list_clients = [&](LsListing& L, int jmax, long long Lmax, long long vlimit, bool skip_listed) {
         int n_alive = 0, n_items = 0;
+        long long min_out = NO_V;
         for (int k0 = 0; k0 < n_clients; k0 += 32) {
             const int k = k0 + lane;
             bool alive = false;
             int sz = 0;
             if (k < n_clients && k != jmax) {
                 const long long lk = s_load[k];
-                alive = lk < Lmax && ((Lmax + lk + 1) >> 1) <= vlimit && !(skip_listed && s_listed[k]);
+                const long long fl = (Lmax + lk + 1) >> 1;
+                alive = lk < Lmax && fl <= vlimit && !(skip_listed && s_listed[k]);
+                if (lk < Lmax && fl > vlimit) min_out = fl < min_out ? fl : min_out;
                 sz = alive ? s_off[k + 1] - s_off[k] + 1 : 0;
                 if (!skip_listed) s_listed[k] = alive;
                 else if (alive) s_listed[k] = 1;
@@ -528,29 +610,56 @@ k_local_search(const uint32_t* __restrict__ T_sorted, const uint32_t* __restrict
             }
             if (alive) {
                 const int pos = n_alive + __popc(am & ((1u << lane) - 1u));
-                s_ak[pos] = (uint8_t)k;
-                s_as[pos] = n_items + inc - sz;
-                s_cb[pos] = s_off[k];
-                s_cs[pos] = (uint32_t)(Lmax - s_load[k]);
+                L.ak[pos] = (uint8_t)k;
+                L.as[pos] = n_items + inc - sz;
+                L.cb[pos] = s_off[k];
+                L.cs[pos] = (uint32_t)(Lmax - s_load[k]);
             }
             n_alive += __popc(am);
             n_items += __shfl_sync(FULL, inc, 31);
         }
-        if (lane == 0) { s_na = n_alive; s_nitems = n_items; s_as[n_alive] = n_items; }
+        if (!skip_listed) {
+#pragma unroll
+            for (int d = 16; d > 0; d >>= 1) {
+                const long long y = __shfl_xor_sync(FULL, min_out, d);
+                min_out = y < min_out ? y : min_out;
+            }
+        }
+        if (lane == 0) {
+            L.na = n_alive; L.nitems = n_items; L.as[n_alive] = n_items;
+            if (!skip_listed) L.min_unlisted = min_out;
+        }
+    };
+    // Copy of a critical client's list to shared memory by `nthr` threads (this one is number `t`).
+    auto copy_list = [&](int base, int nmem, int t, int nthr) {
+        const int top2 = 2 << (31 - __clz(nmem));
+        for (int x = t; x <= top2; x += nthr) {
+            s_T[x] = x == 0 ? 0xFFFFFFFFu : (x <= nmem ? clT[base + x - 1] : 0u);
+            if (x < nmem) s_I[x] = clI[base + x];
+        }
+    };
+    auto is_fast = [&](int nmem, long long Lmax) { return nmem >= 1 && nmem < LS_STAGE && Lmax <= 0x7FFFFFFFll; };
+    auto floor_of_min = [&](int jmax, long long Lmax) {
+        const int km = s_kmin;
+        return (km != jmax && s_load[km] < Lmax) ? ((Lmax + s_load[km] + 1) >> 1) : Lmax;
     };
     if (warp == 0) find_extremes();
     __syncthreads();
 
+    bool have_list = false;                 // this round's listing was made during the last apply
+    bool have_copy = false;                 // and so was the copy of the critical list
+    int buf = 0;
     for (int round = 0; round < rounds; ++round) {
+        LsListing& L = s_ls[buf];
         const int jmax = s_jmax;
         const long long Lmax = s_lmax;
         // all loads equal: the least loaded client is as loaded as the critical one; nothing can improve
-        const int kmin = (s_kmin != jmax && s_load[s_kmin] < Lmax) ? s_kmin : -1;
+        const long long floor_min = floor_of_min(jmax, Lmax);
         const int base_j = s_off[jmax];
         const int nm = s_off[jmax + 1] - base_j;            // jmax's members, T descending
         // short critical list and loads below 2^31: the list is copied to shared memory and the
         // evaluation runs in 32-bit arithmetic; otherwise the general form reads it in place
-        const bool fast = nm >= 1 && nm < LS_STAGE && Lmax <= 0x7FFFFFFFll;
+        const bool fast = is_fast(nm, Lmax);
         const int top = fast ? 1 << (31 - __clz(nm)) : 0;  // largest power of two <= nm
 
         // (a) one work item: partner (Tu, u1 = u + 1, position pu; the move has Tu = 0, u1 = 0,
@@ -596,23 +705,22 @@ k_local_search(const uint32_t* __restrict__ T_sorted, const uint32_t* __restrict
                 }
             }
         };
-        // (b) warp 0 lists the clients to look at, with the running count of their work items (list
+        // (b) The clients to look at are listed with the running count of their work items (list
         //     length + 1 move).  Any step onto client k ends with v >= floor_k = ceil((Lmax + load_k) / 2),
         //     so a client whose floor is above an achieved v cannot win or tie.  First pass: the
         //     clients whose floor is within `margin` of the least loaded client's; after the
-        //     reduction, any client left out whose floor does not exceed the best v found is
-        //     evaluated in a second pass (vlimit = that v), which makes the result exact whatever
-        //     the margin was.  A thread fetches its next item's partner before it works on the
-        //     current one, so the list reads overlap the searches.
+        //     reduction, if a client left out has a floor that does not exceed the best v found, those
+        //     are evaluated in a second pass (vlimit = that v), which makes the result exact whatever
+        //     the margin was.
         auto evaluate_listed = [&](Cand& best) {
-            const int n_items = s_nitems;
+            const int n_items = L.nitems;
             const uint32_t* memT = clT + base_j;
             const IdxT* memI = clI + base_j;
             int ci = 0;
             for (int x = threadIdx.x; x < n_items; x += LS_THREADS) {
-                while (x >= s_as[ci + 1]) ++ci;                 // s_as[n_alive] = n_items ends the walk
-                const int k = s_ak[ci], idx = x - s_as[ci], at = s_cb[ci] + idx;
-                if (x + 1 < s_as[ci + 1]) evaluate(memT, memI, k, clT[at], (uint32_t)clI[at] + 1u, idx, best);
+                while (x >= L.as[ci + 1]) ++ci;                 // as[n_alive] = n_items ends the walk
+                const int k = L.ak[ci], idx = x - L.as[ci], at = L.cb[ci] + idx;
+                if (x + 1 < L.as[ci + 1]) evaluate(memT, memI, k, clT[at], (uint32_t)clI[at] + 1u, idx, best);
                 else evaluate(memT, memI, k, 0u, 0u, -1, best);
             }
         };
@@ -630,8 +738,9 @@ k_local_search(const uint32_t* __restrict__ T_sorted, const uint32_t* __restrict
                 if (s_T[cnt_ge + step] >= thr) cnt_ge += step;   // A[cnt_ge + step - 1]
             return cnt_ge;
         };
-        auto evaluate_listed_fast = [&](Cand& best) {
-            const int n_items = s_nitems;
+        auto evaluate_listed_fast = [&](Cand& best, auto steps_c) {
+            constexpr int STEPS = decltype(steps_c)::value;
+            const int n_items = L.nitems;
             int best_at = -1;                                   // where the best partner's index is, if not read yet
             auto consider = [&](uint32_t inv, int pi, uint32_t k, bool move, int at, int idx) {
                 const uint32_t ik = ((uint32_t)s_I[pi] << 8) | k;
@@ -644,7 +753,8 @@ k_local_search(const uint32_t* __restrict__ T_sorted, const uint32_t* __restrict
                     if (u1 < best.u1) { best.pi = pi; best.pu = move ? -1 : idx; best.u1 = u1; }
                 }
             };
-            int ci = 0;
+            // the listed client the thread's items are in: slot, first item, end, list start - first item
+            int ci = 0, c_lo = 0, c_hi = L.as[1], c_rel = L.cb[0];
             uint32_t nTu[LS_BATCH];                             // next batch: partner T (0 for the move),
             int nci[LS_BATCH];                                  // listed-client slot (-1: no item)
             auto fetch = [&](int x0) {
@@ -653,9 +763,12 @@ k_local_search(const uint32_t* __restrict__ T_sorted, const uint32_t* __restrict
                     const int xx = x0 + u * LS_THREADS;
                     nci[u] = -1; nTu[u] = 0u;
                     if (xx < n_items) {
-                        while (xx >= s_as[ci + 1]) ++ci;        // s_as[n_alive] = n_items ends the walk
+                        while (xx >= c_hi) {                    // as[n_alive] = n_items ends the walk
+                            ++ci;
+                            c_lo = c_hi; c_hi = L.as[ci + 1]; c_rel = L.cb[ci] - c_lo;
+                        }
                         nci[u] = ci;
-                        if (xx + 1 != s_as[ci + 1]) nTu[u] = clT[s_cb[ci] + (xx - s_as[ci])];
+                        if (xx + 1 != c_hi) nTu[u] = clT[c_rel + xx];
                     }
                 }
             };
@@ -667,17 +780,13 @@ k_local_search(const uint32_t* __restrict__ T_sorted, const uint32_t* __restrict
 #pragma unroll
                 for (int u = 0; u < LS_BATCH; ++u) {
                     Tu[u] = nTu[u]; cs[u] = nci[u];
-                    slack[u] = cs[u] >= 0 ? s_cs[cs[u]] : 0u;
+                    slack[u] = cs[u] >= 0 ? L.cs[cs[u]] : 0u;
                     thr[u] = Tu[u] + ((slack[u] + 1u) >> 1);
                     b[u] = 0;
                 }
                 const int xn = x0 + LS_BATCH * LS_THREADS;
                 if (xn < n_items) fetch(xn);                    // in flight during this batch's searches
-                for (int step = top; step > 0; step >>= 1) {
-#pragma unroll
-                    for (int u = 0; u < LS_BATCH; ++u)
-                        if (s_T[b[u] + step] >= thr[u]) b[u] += step;
-                }
+                count_ge_batch<STEPS>(s_T, thr, b, top);
 #pragma unroll
                 for (int u = 0; u < LS_BATCH; ++u) {
                     if (cs[u] < 0) continue;
@@ -688,10 +797,10 @@ k_local_search(const uint32_t* __restrict__ T_sorted, const uint32_t* __restrict
                     const uint32_t inv_f = d2 > 0 ? ~(uint32_t)d2 : NO_CAND;
                     if (min(inv_r, inv_f) > best.inv) continue; // NO_CAND is the largest value
                     const int xx = x0 + u * LS_THREADS;
-                    const int idx = xx - s_as[cs[u]];
-                    const bool move = xx + 1 == s_as[cs[u] + 1];
-                    const int at = s_cb[cs[u]] + idx;
-                    const uint32_t k = s_ak[cs[u]];
+                    const int idx = xx - L.as[cs[u]];
+                    const bool move = xx + 1 == L.as[cs[u] + 1];
+                    const int at = L.cb[cs[u]] + idx;
+                    const uint32_t k = L.ak[cs[u]];
                     if (inv_r != NO_CAND && inv_r <= best.inv) {
                         // first member of the run of equal T: b - 1 itself unless its predecessor ties
                         const int pi = s_T[b[u] - 1] != Ti ? b[u] - 1 : count_ge(Ti + 1u);
@@ -705,18 +814,17 @@ k_local_search(const uint32_t* __restrict__ T_sorted, const uint32_t* __restrict
         };
         Cand best;
         best.inv = NO_CAND; best.ik = NO_CAND; best.u1 = NO_CAND; best.pi = -1; best.pu = -1;
-        const long long floor_min = kmin >= 0 ? ((Lmax + s_load[kmin] + 1) >> 1) : Lmax;
-        if (warp == 0) list_clients(jmax, Lmax, floor_min + margin, false);
-        else if (fast)
-            for (int x = threadIdx.x - 32; x <= 2 * top; x += LS_THREADS - 32) {
-                s_T[x] = x == 0 ? 0xFFFFFFFFu : (x <= nm ? clT[base_j + x - 1] : 0u);
-                if (x < nm) s_I[x] = clI[base_j + x];
-            }
-        __syncthreads();
+        if (!have_list || (fast && !have_copy)) {
+            if (warp == 0) { if (!have_list) list_clients(L, jmax, Lmax, floor_min + margin, false); }
+            else if (fast && !have_copy) copy_list(base_j, nm, (int)threadIdx.x - 32, LS_THREADS - 32);
+            __syncthreads();
+        }
         long long best_v = Lmax;
         for (int pass = 0; pass < 2; ++pass) {
-            if (fast) evaluate_listed_fast(best);
-            else evaluate_listed(best);
+            if (!fast) evaluate_listed(best);
+            else if (top == 256) evaluate_listed_fast(best, std::integral_constant<int, 9>());
+            else if (top == 128) evaluate_listed_fast(best, std::integral_constant<int, 8>());
+            else evaluate_listed_fast(best, std::integral_constant<int, 0>());
             // CTA-wide lexicographic minimum: per warp, then every warp reduces the warps' records
             best = cand_warp_min(best);
             if (lane == 0) s_cand[warp] = best;
@@ -728,16 +836,10 @@ k_local_search(const uint32_t* __restrict__ T_sorted, const uint32_t* __restrict
                 best = cand_warp_min(mine);
             }
             best_v = best.inv != NO_CAND ? Lmax - (long long)(~best.inv) : Lmax;
-            if (pass == 1) break;
-            // is a client that was left out still able to reach best_v?
-            bool missed = false;
-            for (int kk = threadIdx.x; kk < n_clients; kk += LS_THREADS)
-                if (kk != jmax && !s_listed[kk]) {
-                    const long long lk = s_load[kk];
-                    missed |= lk < Lmax && ((Lmax + lk + 1) >> 1) <= best_v;
-                }
-            if (!__syncthreads_or(missed)) break;
-            if (warp == 0) list_clients(jmax, Lmax, best_v, true);
+            // is a client that was left out still able to reach best_v?  (uniform)
+            if (pass == 1 || L.min_unlisted > best_v) break;
+            __syncthreads();                                    // everyone has read the listing
+            if (warp == 0) list_clients(L, jmax, Lmax, best_v, true);
             __syncthreads();
         }
         const bool ok = best.inv != NO_CAND;                    // a candidate always has v < Lmax
@@ -750,32 +852,54 @@ k_local_search(const uint32_t* __restrict__ T_sorted, const uint32_t* __restrict
         const int best_k = (int)(best.ik & 0xFFu);
         const int best_i = (int)(best.ik >> 8);
         const int best_u = (int)best.u1 - 1;
-        // (c) apply.  Warp 0 updates the two loads and finds the next round's extremes, warp 1
-        //     writes the assignment and the log, warps 2 and 3 patch one member list each.
+        const bool swap = best.pu >= 0;
+        // (c) apply.  Warp 0 updates the two loads, finds the next round's extremes and lists its
+        //     clients; warp 1 writes the assignment and the log and, once warp 0 has the next critical
+        //     client, copies its list unless that is one of the two being patched; warps 2 and 3 patch
+        //     one member list each.  (A move rebuilds the lists, so nothing is prepared ahead.)
         const int base_k = s_off[best_k];
         const uint32_t Ti_w = clT[base_j + best.pi];            // read by every warp before any list changes
-        const uint32_t Tu_w = best.pu >= 0 ? clT[base_k + best.pu] : 0u;
+        const uint32_t Tu_w = swap ? clT[base_k + best.pu] : 0u;
         __syncthreads();
         if (warp == 0) {
             const long long dT = (long long)Ti_w - (long long)Tu_w;
             if (lane == 0) { s_load[jmax] -= dT; s_load[best_k] += dT; }
             __syncwarp();
             find_extremes();
+            __syncwarp();
+            __threadfence_block();                              // the extremes are written before warp 1 is let go
+            pair_arrive();
+            if (swap) {
+                const int nj = s_jmax;
+                const long long nL = s_lmax;
+                list_clients(s_ls[buf ^ 1], nj, nL, floor_of_min(nj, nL) + margin, false);
+            }
         } else if (warp == 1) {
             if (lane == 0) {
                 asg[best_i] = best_k;
                 if (best_u >= 0) asg[best_u] = jmax;
                 if (log) log[round] = hos_ls_move{best_i, best_u, best_k, best_v};
             }
-        } else if (best.pu >= 0) {
+            __syncwarp();
+            pair_wait();
+            const int nj = s_jmax;
+            if (swap && nj != jmax && nj != best_k) {
+                const int nb = s_off[nj], nn = s_off[nj + 1] - nb;
+                if (is_fast(nn, s_lmax)) copy_list(nb, nn, lane, 32);
+            }
+        } else if (swap) {
             if (warp == 2) warp_patch_list<IdxT>(clT + base_j, clI + base_j, nm, best.pi, Tu_w, (uint32_t)best_u);
             else if (warp == 3)
                 warp_patch_list<IdxT>(clT + base_k, clI + base_k, s_off[best_k + 1] - base_k, best.pu, Ti_w,
                                       (uint32_t)best_i);
         }
         __syncthreads();
-        if (best.pu < 0)
-            build_member_lists<IdxT, false>(asg, gO, gT, clI, clT, n_req, n_clients, cnt, s_wsum, s_off, nullptr);
+        if (!swap)
+            build_member_lists<IdxT, false, true>(asg, rcl, gO, gT, clI, clT, n_req, n_clients, cnt, s_wsum, s_off,
+                                                  nullptr);
+        have_list = swap;
+        have_copy = swap && s_jmax != jmax && s_jmax != best_k;
+        buf ^= 1;
         ++applied;
     }
     // a round without an improving step leaves the state as it is: all later rounds are the same
@@ -898,11 +1022,11 @@ cudaError_t launch_estimate_sort(const hos_batch& b, const hos_cost_model& cm, u
 
 cudaError_t launch_lpt(const hos_batch& b, const uint32_t* T_sorted, const uint32_t* order,
                        const InstInfo* info, int n_pad, int32_t* assign, long long* load,
-                       long long* makespan, cudaStream_t st) {
+                       long long* makespan, uint8_t* rank_client, cudaStream_t st) {
     const int M = b.n_clients;
 #define HOS_LPT(KPL)                                                                               \
     k_lpt<KPL><<<b.n_inst, 32, 0, st>>>(T_sorted, order, info, b.n_req, n_pad, M, assign, load,    \
-                                         makespan)
+                                         makespan, rank_client)
     launch_hook("k_lpt", 0, st);
     if (M <= 32) HOS_LPT(1);
     else if (M <= 64) HOS_LPT(2);
@@ -917,17 +1041,17 @@ cudaError_t launch_local_search(const hos_batch& b, const uint32_t* T_sorted, co
                                 const InstInfo* info, int n_pad, int n_copies, int rounds,
                                 bool load_from_assign, int32_t* assign, long long* load,
                                 long long* makespan, int32_t* rounds_applied, hos_ls_move* ls_log,
-                                int32_t* status, uint32_t* ws_T, void* ws_I, cudaStream_t st) {
+                                int32_t* status, uint32_t* ws_T, void* ws_I, uint8_t* ws_C, cudaStream_t st) {
     const size_t smem = local_search_smem(b.n_req, b.n_clients);
     launch_hook("k_local_search", 0, st);
     if (b.n_req <= 65536)
         k_local_search<uint16_t><<<b.n_inst * n_copies, LS_THREADS, smem, st>>>(
             T_sorted, order, info, b.n_req, n_pad, b.n_clients, n_copies, rounds, load_from_assign, assign,
-            load, makespan, rounds_applied, ls_log, status, ws_T, static_cast<uint16_t*>(ws_I));
+            load, makespan, rounds_applied, ls_log, status, ws_T, static_cast<uint16_t*>(ws_I), ws_C);
     else
         k_local_search<uint32_t><<<b.n_inst * n_copies, LS_THREADS, smem, st>>>(
             T_sorted, order, info, b.n_req, n_pad, b.n_clients, n_copies, rounds, load_from_assign, assign,
-            load, makespan, rounds_applied, ls_log, status, ws_T, static_cast<uint32_t*>(ws_I));
+            load, makespan, rounds_applied, ls_log, status, ws_T, static_cast<uint32_t*>(ws_I), ws_C);
     launch_hook("k_local_search", 1, st);
     return cudaGetLastError();
 }
