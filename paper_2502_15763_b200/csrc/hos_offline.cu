@@ -740,7 +740,7 @@ k_local_search(const uint32_t* __restrict__ T_sorted, const uint32_t* __restrict
         };
         auto evaluate_listed_fast = [&](Cand& best, auto steps_c) {
             constexpr int STEPS = decltype(steps_c)::value;
-            const int n_items = L.nitems;
+            const int na = L.na;
             int best_at = -1;                                   // where the best partner's index is, if not read yet
             auto consider = [&](uint32_t inv, int pi, uint32_t k, bool move, int at, int idx) {
                 const uint32_t ik = ((uint32_t)s_I[pi] << 8) | k;
@@ -753,62 +753,48 @@ k_local_search(const uint32_t* __restrict__ T_sorted, const uint32_t* __restrict
                     if (u1 < best.u1) { best.pi = pi; best.pu = move ? -1 : idx; best.u1 = u1; }
                 }
             };
-            // the listed client the thread's items are in: slot, first item, end, list start - first item
-            int ci = 0, c_lo = 0, c_hi = L.as[1], c_rel = L.cb[0];
-            uint32_t nTu[LS_BATCH];                             // next batch: partner T (0 for the move),
-            int nci[LS_BATCH];                                  // listed-client slot (-1: no item)
-            auto fetch = [&](int x0) {
+            // The listed clients one after the other, so that client, list start and slack are the
+            // same for the whole CTA; item idx of a client is its idx-th member, idx = len is the move.
+            uint32_t nTu[LS_BATCH];                             // next batch: partner T (0 for the move)
+            auto fetch = [&](int cb, int len, int i0) {
 #pragma unroll
                 for (int u = 0; u < LS_BATCH; ++u) {
-                    const int xx = x0 + u * LS_THREADS;
-                    nci[u] = -1; nTu[u] = 0u;
-                    if (xx < n_items) {
-                        while (xx >= c_hi) {                    // as[n_alive] = n_items ends the walk
-                            ++ci;
-                            c_lo = c_hi; c_hi = L.as[ci + 1]; c_rel = L.cb[ci] - c_lo;
-                        }
-                        nci[u] = ci;
-                        if (xx + 1 != c_hi) nTu[u] = clT[c_rel + xx];
-                    }
+                    const int idx = i0 + u * LS_THREADS + (int)threadIdx.x;
+                    nTu[u] = idx < len ? clT[cb + idx] : 0u;
                 }
             };
-            int x0 = threadIdx.x;
-            if (x0 < n_items) fetch(x0);
-            while (x0 < n_items) {
-                uint32_t Tu[LS_BATCH], thr[LS_BATCH], slack[LS_BATCH];
-                int cs[LS_BATCH], b[LS_BATCH];
+            if (na > 0) fetch(L.cb[0], L.as[1] - L.as[0] - 1, 0);
+            for (int ci = 0; ci < na; ++ci) {
+                const int cb = L.cb[ci], len = L.as[ci + 1] - L.as[ci] - 1;
+                const uint32_t slack = L.cs[ci], half = (slack + 1u) >> 1, k = L.ak[ci];
+                for (int i0 = 0; i0 <= len; i0 += LS_BATCH * LS_THREADS) {
+                    uint32_t Tu[LS_BATCH], thr[LS_BATCH];
+                    int b[LS_BATCH];
 #pragma unroll
-                for (int u = 0; u < LS_BATCH; ++u) {
-                    Tu[u] = nTu[u]; cs[u] = nci[u];
-                    slack[u] = cs[u] >= 0 ? L.cs[cs[u]] : 0u;
-                    thr[u] = Tu[u] + ((slack[u] + 1u) >> 1);
-                    b[u] = 0;
-                }
-                const int xn = x0 + LS_BATCH * LS_THREADS;
-                if (xn < n_items) fetch(xn);                    // in flight during this batch's searches
-                count_ge_batch<STEPS>(s_T, thr, b, top);
+                    for (int u = 0; u < LS_BATCH; ++u) { Tu[u] = nTu[u]; thr[u] = Tu[u] + half; b[u] = 0; }
+                    // the next batch's reads are in flight during this batch's searches
+                    if (i0 + LS_BATCH * LS_THREADS <= len) fetch(cb, len, i0 + LS_BATCH * LS_THREADS);
+                    else if (ci + 1 < na) fetch(L.cb[ci + 1], L.as[ci + 2] - L.as[ci + 1] - 1, 0);
+                    count_ge_batch<STEPS>(s_T, thr, b, top);
 #pragma unroll
-                for (int u = 0; u < LS_BATCH; ++u) {
-                    if (cs[u] < 0) continue;
-                    const uint32_t Ti = s_T[b[u]];              // A[b - 1]: smallest T >= thr (rising side)
-                    const uint32_t d = Ti - Tu[u];
-                    const uint32_t inv_r = d < slack[u] ? ~(slack[u] - d) : NO_CAND;
-                    const int d2 = (int)(s_T[b[u] + 1] - Tu[u]);   // A[b]: largest T < thr (falling side)
-                    const uint32_t inv_f = d2 > 0 ? ~(uint32_t)d2 : NO_CAND;
-                    if (min(inv_r, inv_f) > best.inv) continue; // NO_CAND is the largest value
-                    const int xx = x0 + u * LS_THREADS;
-                    const int idx = xx - L.as[cs[u]];
-                    const bool move = xx + 1 == L.as[cs[u] + 1];
-                    const int at = L.cb[cs[u]] + idx;
-                    const uint32_t k = L.ak[cs[u]];
-                    if (inv_r != NO_CAND && inv_r <= best.inv) {
-                        // first member of the run of equal T: b - 1 itself unless its predecessor ties
-                        const int pi = s_T[b[u] - 1] != Ti ? b[u] - 1 : count_ge(Ti + 1u);
-                        consider(inv_r, pi, k, move, at, idx);
+                    for (int u = 0; u < LS_BATCH; ++u) {
+                        const int idx = i0 + u * LS_THREADS + (int)threadIdx.x;
+                        if (idx > len) continue;
+                        const uint32_t Ti = s_T[b[u]];          // A[b - 1]: smallest T >= thr (rising side)
+                        const uint32_t d = Ti - Tu[u];
+                        const uint32_t inv_r = d < slack ? ~(slack - d) : NO_CAND;
+                        const int d2 = (int)(s_T[b[u] + 1] - Tu[u]);   // A[b]: largest T < thr (falling side)
+                        const uint32_t inv_f = d2 > 0 ? ~(uint32_t)d2 : NO_CAND;
+                        if (min(inv_r, inv_f) > best.inv) continue;     // NO_CAND is the largest value
+                        const bool move = idx == len;
+                        if (inv_r != NO_CAND && inv_r <= best.inv) {
+                            // first member of the run of equal T: b - 1 itself unless its predecessor ties
+                            const int pi = s_T[b[u] - 1] != Ti ? b[u] - 1 : count_ge(Ti + 1u);
+                            consider(inv_r, pi, k, move, cb + idx, idx);
+                        }
+                        if (inv_f != NO_CAND && inv_f <= best.inv) consider(inv_f, b[u], k, move, cb + idx, idx);
                     }
-                    if (inv_f != NO_CAND && inv_f <= best.inv) consider(inv_f, b[u], k, move, at, idx);
                 }
-                x0 = xn;
             }
             if (best_at >= 0) best.u1 = (uint32_t)clI[best_at] + 1u;
         };
