@@ -906,10 +906,11 @@ k_local_search(const uint32_t* __restrict__ T_sorted, const uint32_t* __restrict
 // Lower bounds.  One CTA per instance; reads p, o once, and T_(M), T_(M+1) from the sorted
 // table left by k_estimate_sort.
 // ---------------------------------------------------------------------------------------
-__device__ __forceinline__ unsigned long long floor_sum_below(unsigned long long n, unsigned long long q) {
-    // sum over x in [0, n) of floor(x / q)
-    const unsigned long long m = n / q, r = n % q;
-    return q * (m * (m - 1ull + (m == 0ull)) / 2ull) + m * r;   // m = 0 -> 0
+__device__ __forceinline__ unsigned long long floor_sum_below(uint32_t n, uint32_t q) {
+    // sum over x in [0, n) of floor(x / q); n and q fit 32 bits, so one 32-bit division does
+    const uint32_t m = n / q, r = n - m * q;
+    return (unsigned long long)q * (((unsigned long long)m * (m - 1u + (m == 0u))) >> 1) +
+           (unsigned long long)m * r;                           // m = 0 -> 0
 }
 
 __global__ void __launch_bounds__(256)
@@ -927,15 +928,26 @@ k_lower_bound(const uint32_t* __restrict__ p, const uint32_t* __restrict__ o, in
     const uint32_t* oi = o + (size_t)inst * n_req;
     const unsigned long long ad = cm.decode_fixed_us, bd = cm.decode_per_seq_us, q = cm.decode_kv_div;
     unsigned long long P = 0, O = 0, K = 0, chain = 0;
-    for (int i = threadIdx.x; i < n_req; i += blockDim.x) {
-        const unsigned long long pp = pi[i], oo = oi[i];
+    // a valid instance has p + o <= kv_budget < 2^31
+    auto take = [&](uint32_t pp, uint32_t oo) {
         P += pp;
         O += oo;
-        K += oo * pp + oo * (oo - 1ull) / 2ull;
-        const unsigned long long alone = (unsigned long long)prefill_us(cm, (uint32_t)pp) + oo * (ad + bd) +
-                                         floor_sum_below(pp + oo, q) - floor_sum_below(pp, q);
+        K += (unsigned long long)oo * pp + (((unsigned long long)oo * (oo - 1u)) >> 1);
+        const unsigned long long alone = (unsigned long long)prefill_us(cm, pp) + oo * (ad + bd) +
+                                         floor_sum_below(pp + oo, cm.decode_kv_div) -
+                                         floor_sum_below(pp, cm.decode_kv_div);
         chain = alone > chain ? alone : chain;
+    };
+    constexpr int UN = 4;                                       // reads in flight per thread and table
+    int i = threadIdx.x;
+    for (; i + (UN - 1) * (int)blockDim.x < n_req; i += UN * blockDim.x) {
+        uint32_t pp[UN], oo[UN];
+#pragma unroll
+        for (int u = 0; u < UN; ++u) { pp[u] = pi[i + u * blockDim.x]; oo[u] = oi[i + u * blockDim.x]; }
+#pragma unroll
+        for (int u = 0; u < UN; ++u) take(pp[u], oo[u]);
     }
+    for (; i < n_req; i += blockDim.x) take(pi[i], oi[i]);
     P = block_sum_u64(P, red);
     O = block_sum_u64(O, red);
     K = block_sum_u64(K, red);
