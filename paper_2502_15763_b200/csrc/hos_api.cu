@@ -58,6 +58,8 @@ struct OfflineWs {
     uint32_t* ls_T;             // local search, per (instance, copy): the member lists' T
     void* ls_I;                 // and request indices
     uint8_t* ls_C;              // and the client of every rank of the sorted order
+    int32_t* ls_off;            // list offsets, n_clients + 1 per (instance, copy)
+    int32_t* ls_bad;            // per (instance, copy): assignment outside [0, n_clients)
     size_t bytes;
 };
 OfflineWs carve_offline(const hos_batch* b, void* ws, int n_copies, int ls_rounds) {
@@ -68,12 +70,15 @@ OfflineWs carve_offline(const hos_batch* b, void* ws, int n_copies, int ls_round
     w.T_sorted = reinterpret_cast<uint32_t*>(base + off); off += up(rows * 4);
     w.order = reinterpret_cast<uint32_t*>(base + off);    off += up(rows * 4);
     w.info = reinterpret_cast<InstInfo*>(base + off);     off += up((size_t)b->n_inst * sizeof(InstInfo));
-    w.ls_T = nullptr; w.ls_I = nullptr; w.ls_C = nullptr;
+    w.ls_T = nullptr; w.ls_I = nullptr; w.ls_C = nullptr; w.ls_off = nullptr; w.ls_bad = nullptr;
     if (ls_rounds > 0) {
         const size_t units = rows * (size_t)(n_copies > 0 ? n_copies : 1);
         w.ls_T = reinterpret_cast<uint32_t*>(base + off);  off += up(units * 4);
         w.ls_I = base + off;                               off += up(units * local_search_index_bytes(b->n_req));
         w.ls_C = base + off;                               off += up(units);
+        const size_t n_units = (size_t)b->n_inst * (size_t)(n_copies > 0 ? n_copies : 1);
+        w.ls_off = reinterpret_cast<int32_t*>(base + off); off += up(n_units * (size_t)(b->n_clients + 1) * 4);
+        w.ls_bad = reinterpret_cast<int32_t*>(base + off); off += up(n_units * 4);
     }
     w.bytes = off;
     return w;
@@ -162,7 +167,7 @@ int hos_offline_pack(const hos_batch* b, const hos_cost_model* cm, int ls_rounds
     return cuda_rc(launch_local_search(*b, w.T_sorted, w.order, w.info, n_pad, 1, ls_rounds, false, assign,
                                        reinterpret_cast<long long*>(load),
                                        reinterpret_cast<long long*>(makespan_est), rounds_applied,
-                                       ls_log, status, w.ls_T, w.ls_I, w.ls_C, st));
+                                       ls_log, status, w.ls_T, w.ls_I, w.ls_C, w.ls_off, w.ls_bad, st));
 }
 
 int hos_local_search(const hos_batch* b, const hos_cost_model* cm, int n_copies, int ls_rounds,
@@ -183,7 +188,7 @@ int hos_local_search(const hos_batch* b, const hos_cost_model* cm, int n_copies,
     return cuda_rc(launch_local_search(*b, w.T_sorted, w.order, w.info, n_pad, n_copies, ls_rounds, true,
                                        assign, reinterpret_cast<long long*>(load),
                                        reinterpret_cast<long long*>(makespan_est), rounds_applied,
-                                       ls_log, status, w.ls_T, w.ls_I, w.ls_C, st));
+                                       ls_log, status, w.ls_T, w.ls_I, w.ls_C, w.ls_off, w.ls_bad, st));
 }
 
 int hos_lower_bound(const hos_batch* b, const hos_cost_model* cm, hos_lb* out, int32_t* status, void* ws,

@@ -27,7 +27,8 @@ cudaError_t launch_local_search(const hos_batch& b, const uint32_t* T_sorted, co
                                 const InstInfo* info, int n_pad, int n_copies, int rounds,
                                 bool load_from_assign, int32_t* assign, long long* load,
                                 long long* makespan, int32_t* rounds_applied, hos_ls_move* ls_log,
-                                int32_t* status, uint32_t* ws_T, void* ws_I, uint8_t* ws_C, cudaStream_t st);
+                                int32_t* status, uint32_t* ws_T, void* ws_I, uint8_t* ws_C, int32_t* ws_off,
+                                int32_t* ws_bad, cudaStream_t st);
 size_t local_search_index_bytes(int n_req);
 cudaError_t launch_lower_bound(const hos_batch& b, const hos_cost_model& cm, const uint32_t* T_sorted,
                                const InstInfo* info, int n_pad, hos_lb* out, cudaStream_t st);

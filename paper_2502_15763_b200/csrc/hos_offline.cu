@@ -304,9 +304,10 @@ constexpr int LS_WARPS = LS_THREADS / 32;
 constexpr int LS_STAGE = 512;             // longest critical list that is copied to shared memory
 constexpr int LS_BATCH = 4;               // work items a thread has in flight
 
-// Exclusive scan of a[0 .. len) in place by the whole CTA; `wsum` holds LS_WARPS words.
+// Exclusive scan of a[0 .. len) in place by the whole CTA of NT threads; `wsum` holds NT / 32 words.
+template <int NT>
 __device__ inline void block_scan_u32(uint32_t* a, int len, uint32_t* wsum) {
-    const int per = (len + LS_THREADS - 1) / LS_THREADS;
+    const int per = (len + NT - 1) / NT;
     const int lo = min(len, (int)threadIdx.x * per), hi = min(len, lo + per);
     uint32_t run = 0;
     for (int x = lo; x < hi; ++x) run += a[x];
@@ -320,36 +321,43 @@ __device__ inline void block_scan_u32(uint32_t* a, int len, uint32_t* wsum) {
     __syncthreads();
     uint32_t before = 0;                                     // total of the warps before mine
 #pragma unroll
-    for (int w = 0; w < LS_WARPS; ++w) before += w < warp_id() ? wsum[w] : 0u;
+    for (int w = 0; w < NT / 32; ++w) before += w < warp_id() ? wsum[w] : 0u;
     uint32_t acc = before + inc - run;
     for (int x = lo; x < hi; ++x) { const uint32_t c = a[x]; a[x] = acc; acc += c; }
     __syncthreads();
 }
 
 // Member lists of all clients from the assignment: a stable split of the ranks 0..n-1 by
-// client, as the members' request index (clI) and T (clT).  cnt holds n_clients * LS_WARPS
-// words.  off[k] = start of client k's list, off[M] = n.  rcl[r] is the client of rank r: with
+// client, as the members' request index (clI) and T (clT).  cnt holds n_clients * (NT / 32 + 1)
+// words (NT = threads of the CTA; the odd row stride keeps the lanes of a warp on different banks).  off[k] = start of client k's list, off[M] = n.  rcl[r] is the client of rank r: with
 // GATHER it is filled here from the assignment (asg[order[r]]), otherwise it was left by the
 // packing kernel.  With CHECK, an assignment outside [0, M) makes every thread return true
 // (lists not built), and `load`, if given, receives the clients' summed T.  Each warp takes
 // LS_ROWS rows of 32 ranks at a time, so that their reads are in flight together.
 constexpr int LS_ROWS = 4;
-template <typename IdxT, bool CHECK, bool GATHER>
+template <typename IdxT, bool CHECK, bool GATHER, int NT>
 __device__ inline bool build_member_lists(const int32_t* asg, uint8_t* rcl, const uint32_t* __restrict__ gO,
                                           const uint32_t* __restrict__ gT, IdxT* clI, uint32_t* clT,
                                           int n, int n_clients, uint32_t* cnt, uint32_t* wsum, int* off,
                                           long long* load) {
     const int lane = lane_id(), warp = warp_id();
-    const int chunk = (((n + LS_WARPS - 1) / LS_WARPS) + 31) & ~31;
+    const int chunk = (((n + (NT / 32) - 1) / (NT / 32)) + 31) & ~31;
     const int lo = warp * chunk, hi = min(n, lo + chunk);
-    for (int x = threadIdx.x; x < n_clients * LS_WARPS; x += LS_THREADS) cnt[x] = 0;
+    for (int x = threadIdx.x; x < n_clients * (NT / 32 + 1); x += NT) cnt[x] = 0;
     __syncthreads();
     bool bad = false;
-    for (int row = lo; row < hi; row += 32 * LS_ROWS) {
-        int c[LS_ROWS];
-        uint32_t t[LS_ROWS];
-        if (GATHER) {
-            uint32_t id[LS_ROWS];
+    if (!GATHER) {
+        // counts only: four ranks per lane and read
+        for (int r4 = lo + 4 * lane; r4 < hi; r4 += 128) {
+            const uint32_t w = *reinterpret_cast<const uint32_t*>(rcl + r4);   // rows start at multiples of 4
+#pragma unroll
+            for (int e = 0; e < 4; ++e)
+                if (r4 + e < hi) atomicAdd(&cnt[((w >> (8 * e)) & 0xFFu) * (NT / 32 + 1) + warp], 1u);
+        }
+    } else {
+        for (int row = lo; row < hi; row += 32 * LS_ROWS) {
+            int c[LS_ROWS];
+            uint32_t t[LS_ROWS], id[LS_ROWS];
 #pragma unroll
             for (int e = 0; e < LS_ROWS; ++e) {
                 const int r = row + e * 32 + lane;
@@ -358,55 +366,68 @@ __device__ inline bool build_member_lists(const int32_t* asg, uint8_t* rcl, cons
             }
 #pragma unroll
             for (int e = 0; e < LS_ROWS; ++e) c[e] = row + e * 32 + lane < hi ? asg[id[e]] : 0;
-        } else {
 #pragma unroll
             for (int e = 0; e < LS_ROWS; ++e) {
                 const int r = row + e * 32 + lane;
-                c[e] = r < hi ? (int)rcl[r] : 0;
-                t[e] = (CHECK && load && r < hi) ? __ldg(&gT[r]) : 0u;
-            }
-        }
-#pragma unroll
-        for (int e = 0; e < LS_ROWS; ++e) {
-            const int r = row + e * 32 + lane;
-            if (r < hi) {
-                if (CHECK && (c[e] < 0 || c[e] >= n_clients)) bad = true;
-                else {
-                    if (GATHER) rcl[r] = (uint8_t)c[e];
-                    atomicAdd(&cnt[(uint32_t)c[e] * LS_WARPS + warp], 1u);
-                    if (CHECK && load)
-                        atomicAdd(reinterpret_cast<unsigned long long*>(&load[c[e]]), (unsigned long long)t[e]);
+                if (r < hi) {
+                    if (CHECK && (c[e] < 0 || c[e] >= n_clients)) bad = true;
+                    else {
+                        rcl[r] = (uint8_t)c[e];
+                        atomicAdd(&cnt[(uint32_t)c[e] * (NT / 32 + 1) + warp], 1u);
+                        if (CHECK && load)
+                            atomicAdd(reinterpret_cast<unsigned long long*>(&load[c[e]]), (unsigned long long)t[e]);
+                    }
                 }
             }
         }
     }
     if (CHECK) { if (__syncthreads_or(bad)) return true; }
     else __syncthreads();
-    block_scan_u32(cnt, n_clients * LS_WARPS, wsum);
-    for (int k = threadIdx.x; k <= n_clients; k += LS_THREADS)
-        off[k] = k < n_clients ? (int)cnt[k * LS_WARPS] : n;
+    block_scan_u32<NT>(cnt, n_clients * (NT / 32 + 1), wsum);
+    for (int k = threadIdx.x; k <= n_clients; k += NT)
+        off[k] = k < n_clients ? (int)cnt[k * (NT / 32 + 1)] : n;
     __syncthreads();
-    for (int row = lo; row < hi; row += 32 * LS_ROWS) {
-        uint32_t id[LS_ROWS], tr[LS_ROWS], dig[LS_ROWS];
+    // placement, LS_ROWS rows at a time; the next rows' reads are in flight meanwhile
+    const int nb = bit_width_u32((uint32_t)(n_clients - 1));
+    uint32_t nid[LS_ROWS], ntr[LS_ROWS], ndig[LS_ROWS];
+    auto fetch_rows = [&](int row) {
 #pragma unroll
         for (int e = 0; e < LS_ROWS; ++e) {
             const int r = row + e * 32 + lane;
             const bool valid = r < hi;
-            id[e] = valid ? __ldg(&gO[r]) : 0u;
-            tr[e] = valid ? __ldg(&gT[r]) : 0u;
-            dig[e] = valid ? (uint32_t)rcl[r] : 0xFFFFFFFFu;      // (written above by this same thread)
+            nid[e] = valid ? __ldg(&gO[r]) : 0u;
+            ntr[e] = valid ? __ldg(&gT[r]) : 0u;
+            ndig[e] = valid ? (uint32_t)rcl[r] : 0u;              // (with GATHER: written above by this same thread)
+        }
+    };
+    if (lo < hi) fetch_rows(lo);
+    for (int row = lo; row < hi; row += 32 * LS_ROWS) {
+        uint32_t id[LS_ROWS], tr[LS_ROWS], dig[LS_ROWS];
+        unsigned m[LS_ROWS];
+#pragma unroll
+        for (int e = 0; e < LS_ROWS; ++e) {
+            id[e] = nid[e]; tr[e] = ntr[e]; dig[e] = ndig[e];
+            m[e] = __ballot_sync(FULL, row + e * 32 + lane < hi);
+        }
+        if (row + 32 * LS_ROWS < hi) fetch_rows(row + 32 * LS_ROWS);
+        for (int b = 0; b < nb; ++b) {                           // lanes of each row on my client
+#pragma unroll
+            for (int e = 0; e < LS_ROWS; ++e) {
+                const bool bit = (dig[e] >> b) & 1u;
+                const unsigned bal = __ballot_sync(FULL, bit);
+                m[e] &= bit ? bal : ~bal;
+            }
         }
 #pragma unroll
         for (int e = 0; e < LS_ROWS; ++e) {
             const bool valid = row + e * 32 + lane < hi;
-            const unsigned m = __match_any_sync(FULL, dig[e]);   // lanes of this row on my client
-            const uint32_t base = valid ? cnt[dig[e] * LS_WARPS + warp] : 0u;
+            const uint32_t base = valid ? cnt[dig[e] * (NT / 32 + 1) + warp] : 0u;
             __syncwarp();
             if (valid) {
-                const uint32_t at = base + __popc(m & ((1u << lane) - 1u));
+                const uint32_t at = base + __popc(m[e] & ((1u << lane) - 1u));
                 clI[at] = (IdxT)id[e];
                 clT[at] = tr[e];
-                if (lane == (__ffs(m) - 1)) cnt[dig[e] * LS_WARPS + warp] = base + __popc(m);
+                if (lane == (__ffs(m[e]) - 1)) cnt[dig[e] * (NT / 32 + 1) + warp] = base + __popc(m[e]);
             }
             __syncwarp();
         }
@@ -454,6 +475,46 @@ __device__ inline void warp_patch_list(uint32_t* segT, IdxT* segI, int len, int 
     if (lane == 0) { segT[at] = valT; segI[at] = (IdxT)valI; }
 }
 
+// Member lists before the first round: one CTA per (instance, copy).  Leaves the lists (ws_T,
+// ws_I), their offsets (ws_off, n_clients + 1 per unit) and, for a caller's assignment, the
+// clients' loads; ws_bad[unit] != 0 marks an assignment outside [0, n_clients).
+constexpr int LSB_THREADS = 256;
+template <typename IdxT>
+__global__ void __launch_bounds__(LSB_THREADS)
+k_ls_lists(const uint32_t* __restrict__ T_sorted, const uint32_t* __restrict__ order,
+           const InstInfo* __restrict__ info, int n_req, int n_pad, int n_clients, int n_copies,
+           bool load_from_assign, const int32_t* __restrict__ assign, long long* __restrict__ load_io,
+           uint32_t* __restrict__ ws_T, IdxT* __restrict__ ws_I, uint8_t* __restrict__ ws_C,
+           int32_t* __restrict__ ws_off, int32_t* __restrict__ ws_bad) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    __shared__ long long s_load[MAX_CLIENTS];
+    __shared__ int s_off[MAX_CLIENTS + 1];
+    __shared__ uint32_t s_wsum[LSB_THREADS / 32];
+    const int inst = blockIdx.x / n_copies;
+    const size_t unit = blockIdx.x;
+    if (info[inst].status) return;                          // the search kernel zeroes this unit's results
+    uint32_t* cnt = reinterpret_cast<uint32_t*>(smem_raw);
+    const uint32_t* gT = T_sorted + (size_t)inst * n_pad;
+    const uint32_t* gO = order + (size_t)inst * n_pad;
+    const int32_t* asg = assign + unit * n_req;
+    for (int j = threadIdx.x; j < n_clients; j += LSB_THREADS) s_load[j] = 0;
+    __syncthreads();
+    // a caller's assignment is gathered and checked; the packing kernel's comes with the clients by rank
+    const bool failed =
+        load_from_assign
+            ? build_member_lists<IdxT, true, true, LSB_THREADS>(asg, ws_C + unit * n_pad, gO, gT, ws_I + unit * n_pad,
+                                                                ws_T + unit * n_pad, n_req, n_clients, cnt, s_wsum,
+                                                                s_off, s_load)
+            : build_member_lists<IdxT, false, false, LSB_THREADS>(asg, ws_C + unit * n_pad, gO, gT,
+                                                                  ws_I + unit * n_pad, ws_T + unit * n_pad, n_req,
+                                                                  n_clients, cnt, s_wsum, s_off, nullptr);
+    if (threadIdx.x == 0) ws_bad[unit] = failed ? 1 : 0;
+    if (failed) return;
+    for (int k = threadIdx.x; k <= n_clients; k += LSB_THREADS) ws_off[unit * (n_clients + 1) + k] = s_off[k];
+    if (load_from_assign)
+        for (int j = threadIdx.x; j < n_clients; j += LSB_THREADS) load_io[unit * n_clients + j] = s_load[j];
+}
+
 // The clients one round looks at (see (b) in the kernel), double-buffered: the next round's list
 // is made while the current step is applied.
 struct LsListing {
@@ -499,7 +560,8 @@ k_local_search(const uint32_t* __restrict__ T_sorted, const uint32_t* __restrict
                int32_t* __restrict__ assign, long long* __restrict__ load_io,
                long long* __restrict__ makespan_out, int32_t* __restrict__ rounds_applied,
                hos_ls_move* __restrict__ ls_log, int32_t* __restrict__ status_out,
-               uint32_t* __restrict__ ws_T, IdxT* __restrict__ ws_I, uint8_t* __restrict__ ws_C) {
+               uint32_t* __restrict__ ws_T, IdxT* __restrict__ ws_I, uint8_t* __restrict__ ws_C,
+               const int32_t* __restrict__ ws_off, const int32_t* __restrict__ ws_bad) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     __shared__ long long s_load[MAX_CLIENTS];
     __shared__ int s_off[MAX_CLIENTS + 1];
@@ -538,14 +600,13 @@ k_local_search(const uint32_t* __restrict__ T_sorted, const uint32_t* __restrict
 
     const uint32_t* gT = T_sorted + (size_t)inst * n_pad;
     const uint32_t* gO = order + (size_t)inst * n_pad;
-    for (int j = threadIdx.x; j < n_clients; j += LS_THREADS) s_load[j] = load_from_assign ? 0 : ld[j];
+    // lists, offsets and (for a caller's assignment) loads were left by k_ls_lists
+    const bool lists_failed = ws_bad[unit] != 0;
+    if (!lists_failed) {
+        for (int j = threadIdx.x; j < n_clients; j += LS_THREADS) s_load[j] = ld[j];
+        for (int k = threadIdx.x; k <= n_clients; k += LS_THREADS) s_off[k] = ws_off[unit * (n_clients + 1) + k];
+    }
     __syncthreads();
-    // a caller's assignment is gathered and checked; the packing kernel's comes with the clients by rank
-    const bool lists_failed =
-        load_from_assign ? build_member_lists<IdxT, true, true>(asg, rcl, gO, gT, clI, clT, n_req, n_clients, cnt,
-                                                                s_wsum, s_off, s_load)
-                         : build_member_lists<IdxT, false, false>(asg, rcl, gO, gT, clI, clT, n_req, n_clients, cnt,
-                                                                  s_wsum, s_off, nullptr);
     if (lists_failed) {
         if (threadIdx.x == 0) {
             atomicOr(&status_out[inst], HOS_ST_INVALID);
@@ -881,8 +942,8 @@ k_local_search(const uint32_t* __restrict__ T_sorted, const uint32_t* __restrict
         }
         __syncthreads();
         if (!swap)
-            build_member_lists<IdxT, false, true>(asg, rcl, gO, gT, clI, clT, n_req, n_clients, cnt, s_wsum, s_off,
-                                                  nullptr);
+            build_member_lists<IdxT, false, true, LS_THREADS>(asg, rcl, gO, gT, clI, clT, n_req, n_clients, cnt, s_wsum,
+                                                              s_off, nullptr);
         have_list = swap;
         have_copy = swap && s_jmax != jmax && s_jmax != best_k;
         buf ^= 1;
@@ -1000,7 +1061,7 @@ k_lower_bound(const uint32_t* __restrict__ p, const uint32_t* __restrict__ o, in
 size_t estimate_sort_smem(int n_req) {
     return n_req <= 65536 ? sort_smem_bytes<uint16_t>(n_req) : sort_smem_bytes<uint32_t>(n_req);
 }
-size_t local_search_smem(int /*n_req*/, int n_clients) { return (size_t)n_clients * LS_WARPS * 4; }
+size_t local_search_smem(int /*n_req*/, int n_clients) { return (size_t)n_clients * (LS_WARPS + 1) * 4; }
 size_t local_search_index_bytes(int n_req) { return n_req <= 65536 ? 2 : 4; }
 
 cudaError_t launch_estimate_sort(const hos_batch& b, const hos_cost_model& cm, uint32_t* T_sorted,
@@ -1039,17 +1100,32 @@ cudaError_t launch_local_search(const hos_batch& b, const uint32_t* T_sorted, co
                                 const InstInfo* info, int n_pad, int n_copies, int rounds,
                                 bool load_from_assign, int32_t* assign, long long* load,
                                 long long* makespan, int32_t* rounds_applied, hos_ls_move* ls_log,
-                                int32_t* status, uint32_t* ws_T, void* ws_I, uint8_t* ws_C, cudaStream_t st) {
+                                int32_t* status, uint32_t* ws_T, void* ws_I, uint8_t* ws_C, int32_t* ws_off,
+                                int32_t* ws_bad, cudaStream_t st) {
     const size_t smem = local_search_smem(b.n_req, b.n_clients);
+    const size_t smem_lists = (size_t)b.n_clients * (LSB_THREADS / 32 + 1) * 4;
+    const unsigned grid = (unsigned)(b.n_inst * n_copies);
+    launch_hook("k_ls_lists", 0, st);
+    if (b.n_req <= 65536)
+        k_ls_lists<uint16_t><<<grid, LSB_THREADS, smem_lists, st>>>(
+            T_sorted, order, info, b.n_req, n_pad, b.n_clients, n_copies, load_from_assign, assign, load, ws_T,
+            static_cast<uint16_t*>(ws_I), ws_C, ws_off, ws_bad);
+    else
+        k_ls_lists<uint32_t><<<grid, LSB_THREADS, smem_lists, st>>>(
+            T_sorted, order, info, b.n_req, n_pad, b.n_clients, n_copies, load_from_assign, assign, load, ws_T,
+            static_cast<uint32_t*>(ws_I), ws_C, ws_off, ws_bad);
+    launch_hook("k_ls_lists", 1, st);
     launch_hook("k_local_search", 0, st);
     if (b.n_req <= 65536)
-        k_local_search<uint16_t><<<b.n_inst * n_copies, LS_THREADS, smem, st>>>(
+        k_local_search<uint16_t><<<grid, LS_THREADS, smem, st>>>(
             T_sorted, order, info, b.n_req, n_pad, b.n_clients, n_copies, rounds, load_from_assign, assign,
-            load, makespan, rounds_applied, ls_log, status, ws_T, static_cast<uint16_t*>(ws_I), ws_C);
+            load, makespan, rounds_applied, ls_log, status, ws_T, static_cast<uint16_t*>(ws_I), ws_C, ws_off,
+            ws_bad);
     else
-        k_local_search<uint32_t><<<b.n_inst * n_copies, LS_THREADS, smem, st>>>(
+        k_local_search<uint32_t><<<grid, LS_THREADS, smem, st>>>(
             T_sorted, order, info, b.n_req, n_pad, b.n_clients, n_copies, rounds, load_from_assign, assign,
-            load, makespan, rounds_applied, ls_log, status, ws_T, static_cast<uint32_t*>(ws_I), ws_C);
+            load, makespan, rounds_applied, ls_log, status, ws_T, static_cast<uint32_t*>(ws_I), ws_C, ws_off,
+            ws_bad);
     launch_hook("k_local_search", 1, st);
     return cudaGetLastError();
 }
