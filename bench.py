@@ -53,7 +53,7 @@ def rank_workload(name: str, rank: int, instances: int = 0) -> Workload:
         return w
     seeds = tuple(s + rank * w.n_inst for s in w.seeds)
     return Workload(w.name, seeds, w.n_req, w.n_clients, w.batch_cap, w.kv_budget, w.dist_p, w.dist_o,
-                    w.lambdas_q16, w.ls_rounds, w.cost_model)
+                    w.lambdas_q16, w.ls_rounds, w.cost_model, w.est_sigma, w.kv_reserve)
 
 
 # ------------------------------------------------------------------------------------------

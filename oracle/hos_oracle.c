@@ -240,8 +240,12 @@ void ora_queue_build(int n, int M, const int32_t* assign, const uint32_t* p, con
 
 typedef struct { int64_t kv, rem, total; } ora_running;
 
+/* kv_reserve > 0: every request reserves exactly that many KV tokens from admission to
+ * retirement (the paper's experiment reserves the maximum input + output, five blocks, for each
+ * request, because the output length is not known when it is admitted); 0: it reserves p + o. */
 void ora_simulate_client(int qn, const int32_t* q_req, const uint32_t* p, const uint32_t* o,
-                         const ora_cost* c, int cap, int64_t kv_budget, uint32_t lambda_q16,
+                         const ora_cost* c, int cap, int64_t kv_budget, int64_t kv_reserve,
+                         uint32_t lambda_q16,
                          uint32_t max_iters, ora_client* res, ora_rec* trace, int64_t trace_cap)
 {
     const int64_t ad = c->decode_fixed_us,  bd = c->decode_per_seq_us, q = c->decode_kv_div;
@@ -249,7 +253,7 @@ void ora_simulate_client(int qn, const int32_t* q_req, const uint32_t* p, const 
     ora_running* R = (ora_running*)malloc(sizeof(ora_running) * (size_t)(cap > 0 ? cap : 1));
     int nR = 0;                 /* |R| */
     int head = 0;               /* next queue position */
-    int64_t reserved = 0;       /* sum over R of (p + o) */
+    int64_t reserved = 0;       /* sum over R of the reservations */
     int64_t t = 0, busy = 0, Cd = 0;
     uint64_t hash = ORA_HASH_INIT;
     uint32_t n_pre = 0, n_dec = 0;
@@ -261,7 +265,7 @@ void ora_simulate_client(int qn, const int32_t* q_req, const uint32_t* p, const 
         int nA = 0; int64_t sumP = 0, sumTot = 0;
         while (head + nA < qn && nR + nA < cap) {
             int i = q_req[head + nA];
-            int64_t tot = (int64_t)p[i] + (int64_t)o[i];
+            int64_t tot = kv_reserve > 0 ? kv_reserve : (int64_t)p[i] + (int64_t)o[i];
             if (reserved + sumTot + tot > kv_budget) break;
             if (!stage_holds(c, sumP, p[i])) break;
             sumTot += tot; sumP += p[i]; ++nA;
@@ -286,7 +290,8 @@ void ora_simulate_client(int qn, const int32_t* q_req, const uint32_t* p, const 
             rec.tokens = (uint32_t)sumP; rec.aux = (uint32_t)head;
             for (int a = 0; a < nA; ++a) {
                 int i = q_req[head + a];
-                R[nR].kv = p[i]; R[nR].rem = o[i]; R[nR].total = (int64_t)p[i] + (int64_t)o[i];
+                R[nR].kv = p[i]; R[nR].rem = o[i];
+                R[nR].total = kv_reserve > 0 ? kv_reserve : (int64_t)p[i] + (int64_t)o[i];
                 ++nR;
             }
             head += nA;
@@ -348,9 +353,12 @@ typedef struct {
     int finished;
 } ora_cstate;
 
+/* o_key: the output lengths the scheduler knows (estimates; o itself when they are exact): the
+ * queued tokens of Algorithm 1's remain_token count p + o_key.  kv_reserve as above. */
 void ora_simulate_steal(int n, int M, const int32_t* q_off, const int32_t* q_req,
-                        const uint32_t* p, const uint32_t* o, const ora_cost* c, int cap,
-                        int64_t kv_budget, uint32_t lambda_q16, uint32_t max_iters,
+                        const uint32_t* p, const uint32_t* o, const uint32_t* o_key, const ora_cost* c,
+                        int cap, int64_t kv_budget, int64_t kv_reserve, uint32_t lambda_q16,
+                        uint32_t max_iters,
                         ora_client* res, ora_rec** traces, const int64_t* trace_cap,
                         int32_t* served_by)
 {
@@ -362,7 +370,7 @@ void ora_simulate_steal(int n, int M, const int32_t* q_off, const int32_t* q_req
         C[j].cand = (int32_t*)malloc(sizeof(int32_t) * (size_t)cap);
         C[j].ustart = q_off[j]; C[j].qend = q_off[j + 1];
         for (int x = q_off[j]; x < q_off[j + 1]; ++x)
-            C[j].remain += (int64_t)p[q_req[x]] + (int64_t)o[q_req[x]];
+            C[j].remain += (int64_t)p[q_req[x]] + (int64_t)o_key[q_req[x]];
         C[j].hash = ORA_HASH_INIT;
     }
     for (;;) {
@@ -376,11 +384,11 @@ void ora_simulate_steal(int n, int M, const int32_t* q_off, const int32_t* q_req
         /* 1. claim from the own queue: a prefix, no skipping */
         while (s->ustart < s->qend && s->nR + s->nA < cap) {
             int i = q_req[s->ustart];
-            int64_t tot = (int64_t)p[i] + (int64_t)o[i];
+            int64_t tot = kv_reserve > 0 ? kv_reserve : (int64_t)p[i] + (int64_t)o[i];
             if (s->reserved + s->sumTot + tot > kv_budget) break;
             if (!stage_holds(c, s->sumP, p[i])) break;
             s->cand[s->nA++] = i; s->sumTot += tot; s->sumP += p[i];
-            s->ustart += 1; s->remain -= tot;
+            s->ustart += 1; s->remain -= (int64_t)p[i] + (int64_t)o_key[i];
             if (served_by) served_by[i] = cur;
         }
         /* 1b. own queue exhausted and a slot free: take the longest waiting request of the client
@@ -392,11 +400,11 @@ void ora_simulate_steal(int n, int M, const int32_t* q_off, const int32_t* q_req
                     if (C[j].remain > 0 && (d < 0 || C[j].remain > C[d].remain)) d = j;
                 if (d < 0) break;
                 int i = q_req[C[d].ustart];
-                int64_t tot = (int64_t)p[i] + (int64_t)o[i];
+                int64_t tot = kv_reserve > 0 ? kv_reserve : (int64_t)p[i] + (int64_t)o[i];
                 if (s->reserved + s->sumTot + tot > kv_budget) break;
                 if (!stage_holds(c, s->sumP, p[i])) break;
                 s->cand[s->nA++] = i; s->sumTot += tot; s->sumP += p[i];
-                C[d].ustart += 1; C[d].remain -= tot;
+                C[d].ustart += 1; C[d].remain -= (int64_t)p[i] + (int64_t)o_key[i];
                 if (served_by) served_by[i] = cur;
             }
         }
@@ -420,7 +428,7 @@ void ora_simulate_steal(int n, int M, const int32_t* q_off, const int32_t* q_req
             for (int a = 0; a < s->nA; ++a) {
                 int i = s->cand[a];
                 s->R[s->nR].kv = p[i]; s->R[s->nR].rem = o[i];
-                s->R[s->nR].total = (int64_t)p[i] + (int64_t)o[i];
+                s->R[s->nR].total = kv_reserve > 0 ? kv_reserve : (int64_t)p[i] + (int64_t)o[i];
                 s->nR += 1;
             }
             s->head += s->nA;

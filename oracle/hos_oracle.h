@@ -78,14 +78,16 @@ void ora_lower_bound(int n, int M, int cap, const uint32_t* p, const uint32_t* o
                      const ora_cost* c, ora_lb* out);
 
 /* Per-client queues (Algorithm 1, first part): CSR q_off[M+1], q_req[n]. */
+/* (o here is what the scheduler sorts by: the output lengths it knows, exact or estimated.) */
 void ora_queue_build(int n, int M, const int32_t* assign, const uint32_t* p, const uint32_t* o,
                      int mode, int32_t* q_off, int32_t* q_req);
 
 /* Iteration-level simulation of one client's queue (PD competition + continuous batching,
  * decision rule of the "Online requests and iteration scheduling" section). */
 void ora_simulate_client(int qn, const int32_t* q_req, const uint32_t* p, const uint32_t* o,
-                         const ora_cost* c, int cap, int64_t kv_budget, uint32_t lambda_q16,
-                         uint32_t max_iters, ora_client* res, ora_rec* trace, int64_t trace_cap);
+                         const ora_cost* c, int cap, int64_t kv_budget, int64_t kv_reserve,
+                         uint32_t lambda_q16, uint32_t max_iters, ora_client* res, ora_rec* trace,
+                         int64_t trace_cap);
 
 /* The same simulation with Algorithm 1's second part: all M clients of one instance advance in
  * global time order (earliest clock first, ties to the lower client); a client whose own queue
@@ -94,8 +96,9 @@ void ora_simulate_client(int qn, const int32_t* q_req, const uint32_t* p, const 
  * res [M]; traces [M] (nullable, each with trace_cap[c] slots); served_by [n] (nullable) gets the
  * client that finally served each request. */
 void ora_simulate_steal(int n, int M, const int32_t* q_off, const int32_t* q_req,
-                        const uint32_t* p, const uint32_t* o, const ora_cost* c, int cap,
-                        int64_t kv_budget, uint32_t lambda_q16, uint32_t max_iters,
+                        const uint32_t* p, const uint32_t* o, const uint32_t* o_key, const ora_cost* c,
+                        int cap, int64_t kv_budget, int64_t kv_reserve, uint32_t lambda_q16,
+                        uint32_t max_iters,
                         ora_client* res, ora_rec** traces, const int64_t* trace_cap,
                         int32_t* served_by);
 

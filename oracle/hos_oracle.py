@@ -140,6 +140,7 @@ def lower_bound(p, o, M: int, cap: int, cm) -> dict:
 
 
 def queue_build(assign, p, o, M: int, mode: int):
+    """Queues by (p + o descending, index); o is what the scheduler knows (exact or estimated)."""
     p, o = _u32(p), _u32(o)
     assign = np.ascontiguousarray(assign, dtype=np.int32)
     q_off = np.empty(M + 1, dtype=np.int32)
@@ -164,8 +165,9 @@ class ClientResult:
 
 def simulate_client(queue, p, o, cm, cap: int, kv_budget: int, lambda_q16: int,
                     max_iters: int = 0xFFFFFFFF, want_trace: bool = False,
-                    trace_cap: Optional[int] = None) -> ClientResult:
-    """Simulate one client's queue (array of request indices into p, o)."""
+                    trace_cap: Optional[int] = None, kv_reserve: int = 0) -> ClientResult:
+    """Simulate one client's queue (array of request indices into p, o).  kv_reserve > 0: every
+    request reserves that many KV tokens instead of p + o."""
     p, o = _u32(p), _u32(o)
     queue = np.ascontiguousarray(queue, dtype=np.int32)
     res = _Client()
@@ -174,7 +176,7 @@ def simulate_client(queue, p, o, cm, cap: int, kv_budget: int, lambda_q16: int,
     def run(trace, cap_records):
         lib().ora_simulate_client(
             C.c_int(queue.shape[0]), _ptr(queue, C.c_int32), _ptr(p, C.c_uint32), _ptr(o, C.c_uint32),
-            C.byref(cost), C.c_int(cap), C.c_int64(kv_budget), C.c_uint32(lambda_q16),
+            C.byref(cost), C.c_int(cap), C.c_int64(kv_budget), C.c_int64(kv_reserve), C.c_uint32(lambda_q16),
             C.c_uint32(max_iters), C.byref(res),
             trace.ctypes.data_as(C.c_void_p) if trace is not None else None, C.c_int64(cap_records))
 
@@ -202,18 +204,19 @@ class SimResult:
 
 
 def simulate(assign, p, o, M: int, cm, cap: int, kv_budget: int, lambda_q16: int, mode: int,
-             max_iters: int = 0xFFFFFFFF, want_trace: bool = False) -> SimResult:
+             max_iters: int = 0xFFFFFFFF, want_trace: bool = False, o_est=None, kv_reserve: int = 0) -> SimResult:
     """One (instance, multiplier) simulation: all M clients, then the per-simulation figures.
 
     makespan = max over clients; busy = sum over clients;
     utilisation_c = busy_c / (cap * makespan), utilisation = busy / (M * cap * makespan)
     (busy slot-time over offered slot-time), tokens_per_s = sum(o) * 1e6 / makespan
     (the paper's "generation speed").  All zero when the makespan is zero.
+    o_est: the output lengths the scheduler knows (queue order); the simulation runs on o.
     """
     p, o = _u32(p), _u32(o)
-    q_off, q_req = queue_build(assign, p, o, M, mode)
+    q_off, q_req = queue_build(assign, p, o if o_est is None else _u32(o_est), M, mode)
     clients = [simulate_client(q_req[q_off[j]:q_off[j + 1]], p, o, cm, cap, kv_budget, lambda_q16,
-                               max_iters, want_trace) for j in range(M)]
+                               max_iters, want_trace, kv_reserve=kv_reserve) for j in range(M)]
     makespan = max(c.makespan_us for c in clients)
     busy = sum(c.busy_slot_us for c in clients)
     if makespan > 0:
@@ -227,13 +230,14 @@ def simulate(assign, p, o, M: int, cm, cap: int, kv_budget: int, lambda_q16: int
 
 
 def simulate_steal(assign, p, o, M: int, cm, cap: int, kv_budget: int, lambda_q16: int, mode: int,
-                   max_iters: int = 0xFFFFFFFF, want_trace: bool = False):
+                   max_iters: int = 0xFFFFFFFF, want_trace: bool = False, o_est=None, kv_reserve: int = 0):
     """One (instance, multiplier) simulation with Algorithm 1's request stealing: clients advance
     in global time order and an idle client takes the longest waiting request of the client with
     the most queued tokens.  Returns (SimResult, served_by)."""
     p, o = _u32(p), _u32(o)
     n = p.shape[0]
-    q_off, q_req = queue_build(assign, p, o, M, mode)
+    o_key = o if o_est is None else _u32(o_est)
+    q_off, q_req = queue_build(assign, p, o_key, M, mode)
     cost = _cost(cm)
     res = (_Client * M)()
     served = np.full(n, -1, dtype=np.int32)
@@ -243,7 +247,8 @@ def simulate_steal(assign, p, o, M: int, cm, cap: int, kv_budget: int, lambda_q1
         cp = (C.c_int64 * M)(*caps) if traces else None
         lib().ora_simulate_steal(
             C.c_int(n), C.c_int(M), _ptr(q_off, C.c_int32), _ptr(q_req, C.c_int32), _ptr(p, C.c_uint32),
-            _ptr(o, C.c_uint32), C.byref(cost), C.c_int(cap), C.c_int64(kv_budget), C.c_uint32(lambda_q16),
+            _ptr(o, C.c_uint32), _ptr(o_key, C.c_uint32), C.byref(cost), C.c_int(cap), C.c_int64(kv_budget),
+            C.c_int64(kv_reserve), C.c_uint32(lambda_q16),
             C.c_uint32(max_iters), res, tp, cp, _ptr(served, C.c_int32))
 
     run(None, None)

@@ -16,10 +16,12 @@ def rows(trace):
     return [[int(r["dur_us"]), int(r["kind_n"]), int(r["tokens"]), int(r["aux"])] for r in trace]
 
 
-def python_steal_sim(queues, p, o, cm, cap, kv, lam, max_iters=10 ** 9):
+def python_steal_sim(queues, p, o, cm, cap, kv, lam, max_iters=10 ** 9, o_key=None, kv_reserve=0):
     """Independent plain-Python statement of the same rules (lists and dicts, no shared code)."""
     ap, bp, ad, bd, q = cm[:5]
     M = len(queues)
+    o_key = o if o_key is None else o_key                   # what the scheduler believes
+    holds = (lambda i: kv_reserve) if kv_reserve else (lambda i: int(p[i]) + int(o[i]))
     waiting = [list(qj) for qj in queues]                  # unclaimed requests per client, in order
     st = [dict(run={}, cand=[], clock=0, waited=0, busy=0, admitted=0, trace=[], done=False) for _ in range(M)]
     served = {}
@@ -29,20 +31,20 @@ def python_steal_sim(queues, p, o, cm, cap, kv, lam, max_iters=10 ** 9):
             break
         j = min(live, key=lambda x: (st[x]["clock"], x))
         s = st[j]
-        used = lambda: sum(int(p[i]) + int(o[i]) for i in list(s["run"]) + s["cand"])
+        used = lambda: sum(holds(i) for i in list(s["run"]) + s["cand"])
         while waiting[j] and len(s["run"]) + len(s["cand"]) < cap:
             i = waiting[j][0]
-            if used() + int(p[i]) + int(o[i]) > kv:
+            if used() + holds(i) > kv:
                 break
             s["cand"].append(waiting[j].pop(0)); served[i] = j
         if not waiting[j]:
             while len(s["run"]) + len(s["cand"]) < cap:
-                left = [sum(int(p[i]) + int(o[i]) for i in w) for w in waiting]
+                left = [sum(int(p[i]) + int(o_key[i]) for i in w) for w in waiting]
                 if max(left) <= 0:
                     break
                 d = left.index(max(left))                   # first maximum: lowest client on ties
                 i = waiting[d][0]
-                if used() + int(p[i]) + int(o[i]) > kv:
+                if used() + holds(i) > kv:
                     break
                 s["cand"].append(waiting[d].pop(0)); served[i] = j
         if not s["run"] and not s["cand"]:

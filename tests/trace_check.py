@@ -8,8 +8,9 @@ the last prefill) and asserts that every record is what the rules force:
   decode token for every running request (PD competition);
 * every request is prefilled exactly once, before its first decode token, and
   decodes exactly o_i tokens on the client that prefilled it;
-* the batch cap and the KV budget (p+o reserved from admission to retirement)
-  are never exceeded; admission takes the longest admissible queue prefix;
+* the batch cap and the KV budget (p+o, or a fixed amount per request when the
+  output length is not known at admission, reserved from admission to
+  retirement) are never exceeded; admission takes the longest admissible queue prefix;
 * each decision follows "prefill iff lambda * C_d > C_p" unless forced
   (nothing admissible -> decode, nothing running -> prefill);
 * every duration is recomputable from its own record.
@@ -21,7 +22,7 @@ from __future__ import annotations
 PREFILL_FLAG = 1 << 31
 
 
-def replay(queue, p, o, cm, cap, kv_budget, lambda_q16, trace):
+def replay(queue, p, o, cm, cap, kv_budget, lambda_q16, trace, kv_reserve=0):
     ap, bp, ad, bd, q = (int(x) for x in cm[:5])
     levels = [(int(a), int(b)) for a, b in cm[7]] if len(cm) > 7 else []
 
@@ -30,6 +31,7 @@ def replay(queue, p, o, cm, cap, kv_budget, lambda_q16, trace):
             return ap + bp * tokens
         return next(t for c_, t in levels if tokens <= c_)
     queue = [int(i) for i in queue]
+    holds = (lambda i: kv_reserve) if kv_reserve else (lambda i: int(p[i]) + int(o[i]))
     running = {}                      # request -> [kv, remaining]
     head = 0
     waited = 0                        # C_d
@@ -38,13 +40,13 @@ def replay(queue, p, o, cm, cap, kv_budget, lambda_q16, trace):
     decoded = {i: 0 for i in queue}
     for k, rec in enumerate(trace):
         dur, kind_n, tokens, aux = (int(x) for x in rec)
-        reserved = sum(int(p[i]) + int(o[i]) for i in running)
+        reserved = sum(holds(i) for i in running)
         assert len(running) <= cap and reserved <= kv_budget
         # admissible prefix of the queue
         cand, extra = [], 0
         while head + len(cand) < len(queue) and len(running) + len(cand) < cap:
             i = queue[head + len(cand)]
-            need = int(p[i]) + int(o[i])
+            need = holds(i)
             if reserved + extra + need > kv_budget:
                 break
             if levels and sum(int(p[x]) for x in cand) + int(p[i]) > levels[-1][0]:

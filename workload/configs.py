@@ -11,7 +11,7 @@ from typing import List, Tuple
 
 import numpy as np
 
-from .gen import LengthDist, batch_lengths
+from .gen import LengthDist, batch_lengths, estimated_outputs
 
 # (prefill_fixed_us, prefill_per_token_us, decode_fixed_us, decode_per_seq_us,
 #  decode_kv_div, est_per_prompt_token, est_per_output_token)
@@ -40,6 +40,8 @@ class Workload:
     lambdas_q16: Tuple[int, ...] = (LAMBDA_ONE,)
     ls_rounds: int = 0
     cost_model: Tuple[int, ...] = COST_MODEL
+    est_sigma: float = -1.0          # >= 0: the scheduler sees noisy output-length estimates
+    kv_reserve: int = 0              # > 0: KV tokens reserved per request (needed with estimates)
 
     @property
     def n_inst(self) -> int:
@@ -49,7 +51,15 @@ class Workload:
         """The same workload restricted to instances [first, first+count)."""
         return Workload(self.name, self.seeds[first:first + count], self.n_req, self.n_clients,
                         self.batch_cap, self.kv_budget, self.dist_p, self.dist_o,
-                        self.lambdas_q16, self.ls_rounds, self.cost_model)
+                        self.lambdas_q16, self.ls_rounds, self.cost_model, self.est_sigma, self.kv_reserve)
+
+    def estimates(self):
+        """uint32 table [n_inst][n_req] of estimated output lengths, or None when lengths are exact."""
+        if self.est_sigma < 0:
+            return None
+        _, o = self.lengths()
+        return np.stack([estimated_outputs(int(s), o[k], self.est_sigma, self.dist_o.lo, self.dist_o.hi)
+                         for k, s in enumerate(self.seeds)])
 
     def lengths(self):
         """uint32 tables p, o of shape [n_inst][n_req]."""
@@ -69,6 +79,12 @@ def workload(name: str) -> Workload:
     if name == "c4":      # scale-out stress
         return Workload("c4", tuple(range(1000, 2024)), 20000, 64, 128, 262144, LONG_P, LONG_O,
                         (LAMBDA_ONE,), 100)
+    if name == "c1e":     # c1 with output lengths known only up to a log-normal error (sigma 0.3);
+        # every request reserves the largest prompt + the largest output
+        return Workload("c1e", (1,), 1300, 8, 32, 65536, SHORT_P, SHORT_O, est_sigma=0.3, kv_reserve=1024)
+    if name == "c2e":     # the 100-case study under the same uncertainty
+        return Workload("c2e", tuple(range(100, 200)), 1300, 8, 32, 65536, SHORT_P, SHORT_O,
+                        est_sigma=0.3, kv_reserve=1024)
     if name == "paper":   # shaped like the paper's own experiment (Table "Experiment settings")
         return paper_shaped()
     raise KeyError(name)

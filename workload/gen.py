@@ -78,6 +78,16 @@ def instance_lengths(seed: int, n_req: int, dist_p: LengthDist, dist_o: LengthDi
     return dist_p.draw(_normal(w0, w1)), dist_o.draw(_normal(w2, w3))
 
 
+def estimated_outputs(seed: int, o: np.ndarray, sigma: float, lo: int, hi: int) -> np.ndarray:
+    """Noisy estimates of the output lengths: clip(rint(o * exp(sigma * z)), lo, hi), z standard
+    normal from the same generator under the key (seed mod 2^32, (seed >> 32) xor 0x45535431), words
+    0 and 1.  sigma = 0 returns o clipped."""
+    idx = np.arange(o.shape[0], dtype=np.uint64)
+    w0, w1, _, _ = philox4x32_10(idx, seed & 0xFFFFFFFF, ((seed >> 32) ^ 0x45535431) & 0xFFFFFFFF)
+    x = np.rint(o.astype(np.float64) * np.exp(sigma * _normal(w0, w1)))
+    return np.clip(x, lo, hi).astype(np.uint32)
+
+
 def batch_lengths(seeds, n_req: int, dist_p: LengthDist, dist_o: LengthDist):
     """Row-major [len(seeds)][n_req] uint32 tables p, o; row k is instance_lengths(seeds[k], ...)."""
     seeds = list(seeds)
