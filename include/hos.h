@@ -78,12 +78,26 @@ typedef struct hos_cost_model {
 } hos_cost_model;
 
 /* HOST struct; p and o are DEVICE tables [n_inst][n_req] of prompt lengths N^p_i and output
- * lengths N^d_i (both >= 1, Notation table of the paper). */
+ * lengths N^d_i (both >= 1, Notation table of the paper).
+ *
+ * Output lengths that are only estimated (Section "Problem formulation": the number of output
+ * tokens is not known before inference; the offline model works on an estimate of it): o_est,
+ * nullable, is a DEVICE table of the same shape with the lengths the scheduler believes (>= 1).
+ * With it, the estimated times T_i, the offline packing, the queue order of Algorithm 1 and its
+ * count of queued tokens use o_est, while the simulation decodes the true o_i tokens, and the
+ * lower bounds of the simulated makespan use the true lengths.  A request's KV need is then not
+ * known at admission, so every request reserves kv_reserve_tokens from admission to retirement
+ * (the paper's experiment reserves the blocks of the maximum input plus output for each
+ * request); a request with p_i + o_i above that makes its instance HOS_ST_INVALID.
+ * kv_reserve_tokens = 0: a request reserves p_i + o_i (requires o_est = NULL);
+ * kv_reserve_tokens must not exceed kv_budget. */
 typedef struct hos_batch {
     int32_t n_inst, n_req, n_clients, batch_cap;
     int64_t kv_budget;
     const uint32_t* p;
     const uint32_t* o;
+    const uint32_t* o_est;
+    uint32_t kv_reserve_tokens;
 } hos_batch;
 
 /* One local-search round: request i left the critical client for client k; u >= 0 came back

@@ -52,7 +52,8 @@ class _CostModel(C.Structure):
 class _Batch(C.Structure):
     _fields_ = [("n_inst", C.c_int32), ("n_req", C.c_int32), ("n_clients", C.c_int32),
                 ("batch_cap", C.c_int32), ("kv_budget", C.c_int64),
-                ("p", C.c_void_p), ("o", C.c_void_p)]
+                ("p", C.c_void_p), ("o", C.c_void_p), ("o_est", C.c_void_p),
+                ("kv_reserve_tokens", C.c_uint32)]
 
 
 _lib = None
@@ -124,14 +125,21 @@ def _stream():
     return C.c_void_p(_torch().cuda.current_stream().cuda_stream)
 
 
-def _batch(p, o, n_clients: int, batch_cap: int, kv_budget: int) -> _Batch:
+def _batch(p, o, n_clients: int, batch_cap: int, kv_budget: int, o_est=None, kv_reserve: int = 0) -> _Batch:
+    """o_est: optional table of estimated output lengths (same shape as o); kv_reserve: KV tokens
+    every request reserves (required with o_est), 0 = p + o."""
     torch = _torch()
     # uint32 tables travel as int32 tensors (same bits)
     p = _dev(p, torch.int32, "p")
     o = _dev(o, torch.int32, "o")
     if p.dim() != 2 or p.shape != o.shape:
         raise ValueError("p and o must be [n_inst][n_req] tables of the same shape")
-    return _Batch(p.shape[0], p.shape[1], n_clients, batch_cap, kv_budget, p.data_ptr(), o.data_ptr())
+    if o_est is not None:
+        o_est = _dev(o_est, torch.int32, "o_est")
+        if o_est.shape != o.shape:
+            raise ValueError("o_est must have the shape of o")
+    return _Batch(p.shape[0], p.shape[1], n_clients, batch_cap, kv_budget, p.data_ptr(), o.data_ptr(),
+                  o_est.data_ptr() if o_est is not None else None, int(kv_reserve))
 
 
 def _cost(cm: Sequence) -> _CostModel:
@@ -164,14 +172,14 @@ def view_struct(t, dtype: np.dtype) -> np.ndarray:
 
 
 def hos_offline_pack(p, o, n_clients: int, batch_cap: int, kv_budget: int, cost_model, ls_rounds: int = 0,
-                     want_log: bool = False, ws=None, out=None, want_lb: bool = False):
+                     want_log: bool = False, ws=None, out=None, want_lb: bool = False, o_est=None, kv_reserve: int = 0):
     """Eq. 26-30: estimate, order, LPT, `ls_rounds` local-search rounds.  Returns a dict of tensors.
 
     out: optional dict with preallocated 'assign', 'load', 'makespan_est', 'rounds_applied', 'status'
     (for instance row slices of larger tensors) to write into instead of new tensors, optionally 'lb'.
     want_lb: also return the lower bounds (uint8 [n_inst][64]) computed from the same sort."""
     torch = _torch()
-    b = _batch(p, o, n_clients, batch_cap, kv_budget)
+    b = _batch(p, o, n_clients, batch_cap, kv_budget, o_est, kv_reserve)
     cm = _cost(cost_model)
     L = lib()
     need = L.hos_offline_workspace_bytes(C.byref(b), C.c_int(1), C.c_int(ls_rounds))
@@ -208,10 +216,10 @@ def hos_offline_pack(p, o, n_clients: int, batch_cap: int, kv_budget: int, cost_
 
 
 def hos_local_search(p, o, n_clients: int, batch_cap: int, kv_budget: int, cost_model, assign,
-                     ls_rounds: int, want_log: bool = False, ws=None):
+                     ls_rounds: int, want_log: bool = False, ws=None, o_est=None, kv_reserve: int = 0):
     """Local-search rounds from given assignments [n_inst][n_copies][n_req] (modified in place)."""
     torch = _torch()
-    b = _batch(p, o, n_clients, batch_cap, kv_budget)
+    b = _batch(p, o, n_clients, batch_cap, kv_budget, o_est, kv_reserve)
     cm = _cost(cost_model)
     assign = _dev(assign, torch.int32, "assign")
     if assign.dim() != 3 or assign.shape[0] != b.n_inst or assign.shape[2] != b.n_req:
@@ -235,10 +243,10 @@ def hos_local_search(p, o, n_clients: int, batch_cap: int, kv_budget: int, cost_
                 status=status)
 
 
-def hos_lower_bound(p, o, n_clients: int, batch_cap: int, kv_budget: int, cost_model, ws=None):
+def hos_lower_bound(p, o, n_clients: int, batch_cap: int, kv_budget: int, cost_model, ws=None, o_est=None, kv_reserve: int = 0):
     """Eq. 31-32 and the packing relaxations; returns {'lb': uint8 [n_inst][64], 'status': ...}."""
     torch = _torch()
-    b = _batch(p, o, n_clients, batch_cap, kv_budget)
+    b = _batch(p, o, n_clients, batch_cap, kv_budget, o_est, kv_reserve)
     cm = _cost(cost_model)
     L = lib()
     need = L.hos_lower_bound_workspace_bytes(C.byref(b))
@@ -251,12 +259,12 @@ def hos_lower_bound(p, o, n_clients: int, batch_cap: int, kv_budget: int, cost_m
     return dict(lb=out, status=status)
 
 
-def hos_lower_bound_static(p, o, n_clients: int, batch_cap: int, kv_budget: int, cost_model):
+def hos_lower_bound_static(p, o, n_clients: int, batch_cap: int, kv_budget: int, cost_model, o_est=None, kv_reserve: int = 0):
     """hos_lower_bound without a caller workspace: for code that may not allocate device memory
     (the scratch is a fixed array inside the library; batches beyond it raise HosError -5).
     The result tensors here are the caller's outputs; the C call itself allocates nothing."""
     torch = _torch()
-    b = _batch(p, o, n_clients, batch_cap, kv_budget)
+    b = _batch(p, o, n_clients, batch_cap, kv_budget, o_est, kv_reserve)
     cm = _cost(cost_model)
     out = torch.empty((b.n_inst, LB_DTYPE.itemsize), dtype=torch.uint8, device=p.device)
     status = torch.empty((b.n_inst,), dtype=torch.int32, device=p.device)
@@ -277,14 +285,14 @@ def hos_trace_offsets(cres, n_units: Optional[int] = None):
 
 def hos_online_simulate(p, o, n_clients: int, batch_cap: int, kv_budget: int, cost_model, assign,
                         lambda_q16, queue_order: int = HOS_QUEUE_SORTED, max_iters: int = 0x7FFFFFFF,
-                        trace=None, trace_off=None, keep_events: bool = False, ws=None):
+                        trace=None, trace_off=None, keep_events: bool = False, ws=None, o_est=None, kv_reserve: int = 0):
     """Queues + iteration simulation for every (instance, multiplier, client).
 
     trace: None, or a uint8 tensor [n_records][16] with trace_off (int64 [n_units + 1]).
     keep_events: leave the event log in the returned workspace `ws` for hos_trace_fill.
     """
     torch = _torch()
-    b = _batch(p, o, n_clients, batch_cap, kv_budget)
+    b = _batch(p, o, n_clients, batch_cap, kv_budget, o_est, kv_reserve)
     cm = _cost(cost_model)
     assign = _dev(assign, torch.int32, "assign")
     if tuple(assign.shape) != (b.n_inst, b.n_req):
@@ -313,10 +321,10 @@ def hos_online_simulate(p, o, n_clients: int, batch_cap: int, kv_budget: int, co
 
 def hos_online_simulate_steal(p, o, n_clients: int, batch_cap: int, kv_budget: int, cost_model, assign,
                               lambda_q16, queue_order: int = HOS_QUEUE_SORTED, max_iters: int = 0x7FFFFFFF,
-                              trace=None, trace_off=None, want_served_by: bool = False, ws=None):
+                              trace=None, trace_off=None, want_served_by: bool = False, ws=None, o_est=None, kv_reserve: int = 0):
     """hos_online_simulate with Algorithm 1's request stealing between the clients of an instance."""
     torch = _torch()
-    b = _batch(p, o, n_clients, batch_cap, kv_budget)
+    b = _batch(p, o, n_clients, batch_cap, kv_budget, o_est, kv_reserve)
     cm = _cost(cost_model)
     assign = _dev(assign, torch.int32, "assign")
     if tuple(assign.shape) != (b.n_inst, b.n_req):
@@ -345,12 +353,12 @@ def hos_online_simulate_steal(p, o, n_clients: int, batch_cap: int, kv_budget: i
 
 
 def hos_trace_fill(p, o, n_clients: int, batch_cap: int, kv_budget: int, cost_model, n_lambda: int,
-                   sim, trace, trace_off):
+                   sim, trace, trace_off, o_est=None, kv_reserve: int = 0):
     """The full iteration trace from the event log of `sim`, the dict returned by
     hos_online_simulate(..., keep_events=True) for the same batch.  ORs HOS_ST_TRACE into
     sim["status"] where the slots are too few.  Returns `trace`."""
     torch = _torch()
-    b = _batch(p, o, n_clients, batch_cap, kv_budget)
+    b = _batch(p, o, n_clients, batch_cap, kv_budget, o_est, kv_reserve)
     cm = _cost(cost_model)
     trace = _dev(trace, torch.uint8, "trace")
     trace_off = _dev(trace_off, torch.int64, "trace_off")

@@ -22,6 +22,9 @@ int check_batch(const hos_batch* b) {
         b->kv_budget >= (1ll << 31))
         return HOS_E_UNSUPPORTED;
     if ((long long)b->n_inst * (long long)pad4(b->n_req) >= (1ll << 40)) return HOS_E_UNSUPPORTED;
+    // estimated output lengths need the fixed reservation; a reservation must fit the budget
+    if (b->o_est && b->kv_reserve_tokens == 0) return HOS_E_INVALID;
+    if ((long long)b->kv_reserve_tokens > (long long)b->kv_budget) return HOS_E_INVALID;
     return HOS_OK;
 }
 
@@ -86,6 +89,7 @@ OfflineWs carve_offline(const hos_batch* b, void* ws, int n_copies, int ls_round
 
 struct OnlineWs {
     uint2* q_po;
+    uint32_t* q_key;            // p + estimated o per queue position (only with hos_batch::o_est)
     uint32_t* q_req;
     int32_t* q_off;
     unsigned long long* inst_O;
@@ -101,6 +105,8 @@ OnlineWs carve_online(const hos_batch* b, void* ws, int n_lambda, int keep_event
     size_t off = 0;
     w.q_po = reinterpret_cast<uint2*>(base + off);                off += up(rows * 8);
     w.q_req = reinterpret_cast<uint32_t*>(base + off);            off += up(rows * 4);
+    w.q_key = nullptr;
+    if (b->o_est) { w.q_key = reinterpret_cast<uint32_t*>(base + off); off += up(rows * 4); }
     w.q_off = reinterpret_cast<int32_t*>(base + off);             off += up((size_t)b->n_inst * (b->n_clients + 1) * 4);
     w.inst_O = reinterpret_cast<unsigned long long*>(base + off); off += up((size_t)b->n_inst * 8);
     w.inst_status = reinterpret_cast<int32_t*>(base + off);       off += up((size_t)b->n_inst * 4);
@@ -226,7 +232,7 @@ int hos_online_simulate(const hos_batch* b, const int32_t* assign, const hos_cos
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const int n_pad = pad4(b->n_req);
     if (max_iters > 0x7FFFFFFFu) max_iters = 0x7FFFFFFFu;
-    if ((rc = cuda_rc(launch_queue_build(*b, assign, stage_cap_tokens(*cm), queue_order, w.q_po, w.q_req, w.q_off, w.inst_O,
+    if ((rc = cuda_rc(launch_queue_build(*b, assign, stage_cap_tokens(*cm), queue_order, w.q_po, w.q_key, w.q_req, w.q_off, w.inst_O,
                                          w.inst_status, n_pad, st))))
         return rc;
     if ((rc = cuda_rc(launch_simulate(*b, *cm, lambda_q16, n_lambda, max_iters, w.q_po, w.q_off,
@@ -260,10 +266,10 @@ int hos_online_simulate_steal(const hos_batch* b, const int32_t* assign, const h
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const int n_pad = pad4(b->n_req);
     if (max_iters > 0x7FFFFFFFu) max_iters = 0x7FFFFFFFu;
-    if ((rc = cuda_rc(launch_queue_build(*b, assign, stage_cap_tokens(*cm), queue_order, w.q_po, w.q_req, w.q_off, w.inst_O,
+    if ((rc = cuda_rc(launch_queue_build(*b, assign, stage_cap_tokens(*cm), queue_order, w.q_po, w.q_key, w.q_req, w.q_off, w.inst_O,
                                          w.inst_status, n_pad, st))))
         return rc;
-    if ((rc = cuda_rc(launch_simulate_steal(*b, *cm, lambda_q16, n_lambda, max_iters, w.q_po, w.q_req, w.q_off,
+    if ((rc = cuda_rc(launch_simulate_steal(*b, *cm, lambda_q16, n_lambda, max_iters, w.q_po, w.q_key, w.q_req, w.q_off,
                                             w.inst_status, n_pad, cres, trace,
                                             reinterpret_cast<const long long*>(trace_off), status, served_by,
                                             st))))

@@ -34,7 +34,7 @@ cudaError_t launch_lower_bound(const hos_batch& b, const hos_cost_model& cm, con
                                const InstInfo* info, int n_pad, hos_lb* out, cudaStream_t st);
 
 cudaError_t launch_queue_build(const hos_batch& b, const int32_t* assign, uint32_t p_max, int queue_order, uint2* q_po,
-                               uint32_t* q_req, int32_t* q_off, unsigned long long* inst_O,
+                               uint32_t* q_key, uint32_t* q_req, int32_t* q_off, unsigned long long* inst_O,
                                int32_t* inst_status, int n_pad, cudaStream_t st);
 cudaError_t launch_simulate(const hos_batch& b, const hos_cost_model& cm, const uint32_t* lambda_q16,
                             int n_lambda, uint32_t max_iters, const uint2* q_po, const int32_t* q_off,
@@ -43,7 +43,8 @@ cudaError_t launch_simulate(const hos_batch& b, const hos_cost_model& cm, const 
                             uint4* events, uint32_t* event_count, cudaStream_t st);
 size_t simulate_steal_smem(int n_clients, int cap, bool wide);
 cudaError_t launch_simulate_steal(const hos_batch& b, const hos_cost_model& cm, const uint32_t* lambda_q16,
-                                  int n_lambda, uint32_t max_iters, const uint2* q_po, const uint32_t* q_req,
+                                  int n_lambda, uint32_t max_iters, const uint2* q_po, const uint32_t* q_key,
+                                  const uint32_t* q_req,
                                   const int32_t* q_off, const int32_t* inst_status, int n_pad,
                                   hos_client_result* cres, hos_iter_rec* trace, const long long* trace_off,
                                   int32_t* status, int32_t* served_by, cudaStream_t st);

@@ -17,7 +17,8 @@ namespace hos {
 // ---------------------------------------------------------------------------------------
 template <typename IdxT>
 __global__ void __launch_bounds__(SORT_THREADS, 1)
-k_estimate_sort(const uint32_t* __restrict__ p, const uint32_t* __restrict__ o, int n_req,
+k_estimate_sort(const uint32_t* __restrict__ p, const uint32_t* __restrict__ o,
+                const uint32_t* __restrict__ o_est, int n_req,
                 long long kv_budget, uint32_t e_p, uint32_t e_o, uint32_t p_max,
                 uint32_t* __restrict__ T_sorted, uint32_t* __restrict__ order,
                 InstInfo* __restrict__ info, int32_t* __restrict__ status_out, int n_pad) {
@@ -27,12 +28,16 @@ k_estimate_sort(const uint32_t* __restrict__ p, const uint32_t* __restrict__ o, 
     const int inst = blockIdx.x;
     const uint32_t* pi = p + (size_t)inst * n_req;
     const uint32_t* oi = o + (size_t)inst * n_req;
+    const uint32_t* ei = o_est ? o_est + (size_t)inst * n_req : oi;   // the lengths the scheduler knows
 
+    // kv_budget here is the most KV one request may need: the fixed reservation, if there is one
     unsigned long long sum = 0, mx = 0, bad = 0;
     for (int i = threadIdx.x; i < n_req; i += SORT_THREADS) {
-        const uint32_t pp = pi[i], oo = oi[i];
-        const unsigned long long t = (unsigned long long)e_p * pp + (unsigned long long)e_o * oo;
-        if (pp == 0 || oo == 0 || pp > p_max || (long long)pp + (long long)oo > kv_budget || t > 0xFFFFFFFFull) bad = 1;
+        const uint32_t pp = pi[i], oo = oi[i], oe = ei[i];
+        const unsigned long long t = (unsigned long long)e_p * pp + (unsigned long long)e_o * oe;
+        if (pp == 0 || oo == 0 || oe == 0 || pp > p_max || (long long)pp + (long long)oo > kv_budget ||
+            t > 0xFFFFFFFFull)
+            bad = 1;
         s.key[i] = (uint32_t)t;
         sum += t;
         mx = t > mx ? t : mx;
@@ -1072,7 +1077,9 @@ cudaError_t launch_estimate_sort(const hos_batch& b, const hos_cost_model& cm, u
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     launch_hook("k_estimate_sort", 0, st);
-    kern<<<b.n_inst, SORT_THREADS, smem, st>>>(b.p, b.o, b.n_req, (long long)b.kv_budget,
+    kern<<<b.n_inst, SORT_THREADS, smem, st>>>(b.p, b.o, b.o_est, b.n_req,
+                                               b.kv_reserve_tokens ? (long long)b.kv_reserve_tokens
+                                                                   : (long long)b.kv_budget,
                                                cm.est_per_prompt_token, cm.est_per_output_token, stage_cap_tokens(cm),
                                                T_sorted, order, info, status_out, n_pad);
     launch_hook("k_estimate_sort", 1, st);

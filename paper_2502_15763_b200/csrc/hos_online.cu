@@ -19,8 +19,10 @@ constexpr int INST_WIDE = 0x100;         // internal flag in the workspace's per
 template <typename IdxT>
 __global__ void __launch_bounds__(SORT_THREADS, 1)
 k_queue_build(const uint32_t* __restrict__ p, const uint32_t* __restrict__ o,
+              const uint32_t* __restrict__ o_est,
               const int32_t* __restrict__ assign, int n_req, int n_clients, long long kv_budget,
-              uint32_t p_max, int queue_order, uint2* __restrict__ q_po, uint32_t* __restrict__ q_req,
+              uint32_t p_max, int queue_order, uint2* __restrict__ q_po, uint32_t* __restrict__ q_key,
+              uint32_t* __restrict__ q_req,
               int32_t* __restrict__ q_off, unsigned long long* __restrict__ inst_O,
               int32_t* __restrict__ inst_status, int n_pad) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -30,20 +32,27 @@ k_queue_build(const uint32_t* __restrict__ p, const uint32_t* __restrict__ o,
     const uint32_t* pi = p + (size_t)inst * n_req;
     const uint32_t* oi = o + (size_t)inst * n_req;
     const int32_t* ai = assign + (size_t)inst * n_req;
+    const uint32_t* ei = o_est ? o_est + (size_t)inst * n_req : oi;   // the lengths the scheduler sorts by
 
-    unsigned long long sumO = 0, mx = 0, bad = 0;
+    // kv_budget here is the most KV one request may need: the fixed reservation, if there is one
+    unsigned long long sumO = 0, mx = 0, mxk = 0, bad = 0;
     for (int i = threadIdx.x; i < n_req; i += SORT_THREADS) {
-        const uint32_t pp = pi[i], oo = oi[i];
+        const uint32_t pp = pi[i], oo = oi[i], oe = ei[i];
         const int c = ai[i];
         const unsigned long long tot = (unsigned long long)pp + oo;
-        if (pp == 0 || oo == 0 || pp > p_max || (long long)tot > kv_budget || c < 0 || c >= n_clients) bad = 1;
-        s.key[i] = (uint32_t)tot;
+        const unsigned long long totk = (unsigned long long)pp + oe;
+        if (pp == 0 || oo == 0 || oe == 0 || pp > p_max || (long long)tot > kv_budget || totk > 0xFFFFFFFFull ||
+            c < 0 || c >= n_clients)
+            bad = 1;
+        s.key[i] = (uint32_t)totk;
         s.buf1[i] = (IdxT)(c & 0xFF);                 // parked until the keys are composed
         sumO += oo;
         mx = tot > mx ? tot : mx;
+        mxk = totk > mxk ? totk : mxk;
     }
     sumO = block_sum_u64(sumO, red);
     mx = block_max_u64(mx, red);
+    mxk = block_max_u64(mxk, red);
     bad = block_max_u64(bad, red);
     __syncthreads();
     if (threadIdx.x == 0) {
@@ -53,7 +62,7 @@ k_queue_build(const uint32_t* __restrict__ p, const uint32_t* __restrict__ o,
     }
     if (bad) return;
 
-    const int kb = (queue_order == HOS_QUEUE_SORTED) ? bit_width_u32((uint32_t)mx) : 0;
+    const int kb = (queue_order == HOS_QUEUE_SORTED) ? bit_width_u32((uint32_t)mxk) : 0;
     const uint32_t kmask = kb >= 32 ? 0xFFFFFFFFu : ((1u << kb) - 1u);
     const int nbits = kb + bit_width_u32((uint32_t)(n_clients - 1));
     for (int i = threadIdx.x; i < n_req; i += SORT_THREADS) {
@@ -70,6 +79,7 @@ k_queue_build(const uint32_t* __restrict__ p, const uint32_t* __restrict__ o,
         const uint32_t id = sorted[r];
         qr[r] = id;
         qp[r] = make_uint2(pi[id], oi[id]);
+        if (q_key) q_key[(size_t)inst * n_pad + r] = pi[id] + ei[id];
         const int c = (int)(s.key[id] >> kb);
         const int cprev = r > 0 ? (int)(s.key[sorted[r - 1]] >> kb) : -1;
         for (int cc = cprev + 1; cc <= c; ++cc) qo[cc] = r;
@@ -333,7 +343,8 @@ k_simulate(const uint2* __restrict__ q_po, const int32_t* __restrict__ q_off,
 // ---------------------------------------------------------------------------------------
 template <typename E>
 __global__ void __launch_bounds__(MAX_CLIENTS)
-k_simulate_steal(const uint2* __restrict__ q_po, const uint32_t* __restrict__ q_req,
+k_simulate_steal(const uint2* __restrict__ q_po, const uint32_t* __restrict__ q_key,
+                 const uint32_t* __restrict__ q_req,
                  const int32_t* __restrict__ q_off, const int32_t* __restrict__ inst_status,
                  const uint32_t* __restrict__ lambda_q16, int n_lambda, int n_clients, int n_req,
                  int n_pad, int cap, uint32_t kv_budget, hos_cost_model cm, int q_shift,
@@ -371,6 +382,8 @@ k_simulate_steal(const uint2* __restrict__ q_po, const uint32_t* __restrict__ q_
     }
     const int32_t* qo = q_off + (size_t)inst * (n_clients + 1);
     const uint2* q = q_po + (size_t)inst * n_pad;          // all queues of the instance, CSR by client
+    // queued tokens as the scheduler counts them: p + estimated o when the lengths are estimated
+    const uint32_t* qk = q_key ? q_key + (size_t)inst * n_pad : nullptr;
     const uint32_t* qr = q_req + (size_t)inst * n_pad;
     int32_t* served = served_by ? served_by + (size_t)sim * n_req : nullptr;
     const int qend = is_client ? qo[c + 1] : 0;
@@ -380,7 +393,10 @@ k_simulate_steal(const uint2* __restrict__ q_po, const uint32_t* __restrict__ q_
 
     if (is_client) {
         unsigned long long r = 0;
-        for (int x = qo[c]; x < qend; ++x) { const uint2 po = q[x]; r += (unsigned long long)po.x + po.y; }
+        for (int x = qo[c]; x < qend; ++x) {
+            const uint2 po = q[x];
+            r += qk ? (unsigned long long)qk[x] : (unsigned long long)po.x + po.y;
+        }
         s_ustart[c] = qo[c];
         s_remain[c] = r;
     }
@@ -421,9 +437,10 @@ k_simulate_steal(const uint2* __restrict__ q_po, const uint32_t* __restrict__ q_
         heap_st(cap - 1 - (int)nA, E::make(po.y, tt));
         sumTot += tt; sumP += po.x; ++nA;
         if (!dry) {
+            const uint32_t tk = qk ? qk[x] : tt;
             s_ustart[owner] = x + 1;
-            s_remain[owner] -= tt;
-            atomicAdd(&s_total, 0ull - (unsigned long long)tt);
+            s_remain[owner] -= tk;
+            atomicAdd(&s_total, 0ull - (unsigned long long)tk);
             if (served) served[qr[x]] = c;
         }
         return true;
@@ -725,20 +742,30 @@ k_trace_offsets(const hos_client_result* __restrict__ cres, long long n_units,
 // ---------------------------------------------------------------------------------------
 // launchers
 // ---------------------------------------------------------------------------------------
+// Slots and KV budget the simulators run with (see launch_simulate).
+static int sim_slots(const hos_batch& b) {
+    if (!b.kv_reserve_tokens) return b.batch_cap;
+    const long long fit = b.kv_budget / (long long)b.kv_reserve_tokens;
+    return (int)(fit < (long long)b.batch_cap ? fit : (long long)b.batch_cap);
+}
+static uint32_t sim_budget(const hos_batch& b) { return b.kv_reserve_tokens ? 0x7FFFFFFFu : (uint32_t)b.kv_budget; }
+
 size_t queue_build_smem(int n_req) {
     return n_req <= 65536 ? sort_smem_bytes<uint16_t>(n_req) : sort_smem_bytes<uint32_t>(n_req);
 }
 
 cudaError_t launch_queue_build(const hos_batch& b, const int32_t* assign, uint32_t p_max, int queue_order, uint2* q_po,
-                               uint32_t* q_req, int32_t* q_off, unsigned long long* inst_O,
+                               uint32_t* q_key, uint32_t* q_req, int32_t* q_off, unsigned long long* inst_O,
                                int32_t* inst_status, int n_pad, cudaStream_t st) {
     const size_t smem = queue_build_smem(b.n_req);
     auto kern = b.n_req <= 65536 ? k_queue_build<uint16_t> : k_queue_build<uint32_t>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     launch_hook("k_queue_build", 0, st);
-    kern<<<b.n_inst, SORT_THREADS, smem, st>>>(b.p, b.o, assign, b.n_req, b.n_clients,
-                                               (long long)b.kv_budget, p_max, queue_order, q_po, q_req, q_off,
+    kern<<<b.n_inst, SORT_THREADS, smem, st>>>(b.p, b.o, b.o_est, assign, b.n_req, b.n_clients,
+                                               b.kv_reserve_tokens ? (long long)b.kv_reserve_tokens
+                                                                   : (long long)b.kv_budget,
+                                               p_max, queue_order, q_po, b.o_est ? q_key : nullptr, q_req, q_off,
                                                inst_O, inst_status, n_pad);
     launch_hook("k_queue_build", 1, st);
     return cudaGetLastError();
@@ -750,6 +777,10 @@ cudaError_t launch_simulate(const hos_batch& b, const hos_cost_model& cm, const 
                             hos_iter_rec* trace, const long long* trace_off, int32_t* status,
                             uint4* events, uint32_t* event_count, cudaStream_t st) {
     const long long n_units = (long long)b.n_inst * n_lambda * b.n_clients;
+    // A fixed reservation of R tokens per request admits floor(budget / R) requests at most and
+    // nothing else: the simulator runs with that many slots and no KV limit.
+    const int cap = sim_slots(b);
+    const uint32_t kv = sim_budget(b);
     const long long n_warps = (n_units + SIM_THREADS - 1) / SIM_THREADS;
     int q_shift = -1;                                    // power-of-two KV divisor -> shift
     if ((cm.decode_kv_div & (cm.decode_kv_div - 1)) == 0)
@@ -773,8 +804,8 @@ cudaError_t launch_simulate(const hos_batch& b, const hos_cost_model& cm, const 
         if (n_warps > cap_small && wide >= 1 && n_warps <= (long long)n_sm * wide) return (int)wide;
         return 1;
     };
-    const size_t warp_n = (size_t)b.batch_cap * SIM_THREADS * sizeof(uint32_t);
-    const size_t warp_w = (size_t)b.batch_cap * SIM_THREADS * sizeof(unsigned long long);
+    const size_t warp_n = (size_t)cap * SIM_THREADS * sizeof(uint32_t);
+    const size_t warp_w = (size_t)cap * SIM_THREADS * sizeof(unsigned long long);
     const int wpc_n = warps_per_cta(warp_n), wpc_w = warps_per_cta(warp_w);
     const size_t smem_n = warp_n * wpc_n, smem_w = warp_w * wpc_w;
     const unsigned grid_n = (unsigned)((n_warps + wpc_n - 1) / wpc_n);
@@ -785,14 +816,14 @@ cudaError_t launch_simulate(const hos_batch& b, const hos_cost_model& cm, const 
     if (e != cudaSuccess) return e;
     launch_hook("k_simulate", 0, st);
     k_simulate<NarrowEntry><<<grid_n, SIM_THREADS * wpc_n, smem_n, st>>>(
-        q_po, q_off, inst_status, lambda_q16, n_lambda, b.n_clients, n_pad, n_units, b.batch_cap,
-        (uint32_t)b.kv_budget, cm, q_shift, max_iters, cres, trace, trace_off, status, events, event_count);
+        q_po, q_off, inst_status, lambda_q16, n_lambda, b.n_clients, n_pad, n_units, cap,
+        kv, cm, q_shift, max_iters, cres, trace, trace_off, status, events, event_count);
     launch_hook("k_simulate", 1, st);
     if (b.kv_budget >= 65536) {                          // otherwise no p + o can reach 2^16
         launch_hook("k_simulate_wide", 0, st);
         k_simulate<WideEntry><<<grid_w, SIM_THREADS * wpc_w, smem_w, st>>>(
-            q_po, q_off, inst_status, lambda_q16, n_lambda, b.n_clients, n_pad, n_units, b.batch_cap,
-            (uint32_t)b.kv_budget, cm, q_shift, max_iters, cres, trace, trace_off, status, events, event_count);
+            q_po, q_off, inst_status, lambda_q16, n_lambda, b.n_clients, n_pad, n_units, cap,
+            kv, cm, q_shift, max_iters, cres, trace, trace_off, status, events, event_count);
         launch_hook("k_simulate_wide", 1, st);
     }
     return cudaGetLastError();
@@ -804,31 +835,34 @@ size_t simulate_steal_smem(int n_clients, int cap, bool wide) {
 }
 
 cudaError_t launch_simulate_steal(const hos_batch& b, const hos_cost_model& cm, const uint32_t* lambda_q16,
-                                  int n_lambda, uint32_t max_iters, const uint2* q_po, const uint32_t* q_req,
+                                  int n_lambda, uint32_t max_iters, const uint2* q_po, const uint32_t* q_key,
+                                  const uint32_t* q_req,
                                   const int32_t* q_off, const int32_t* inst_status, int n_pad,
                                   hos_client_result* cres, hos_iter_rec* trace, const long long* trace_off,
                                   int32_t* status, int32_t* served_by, cudaStream_t st) {
     const int threads = (b.n_clients + 31) & ~31;
+    const int cap = sim_slots(b);
+    const uint32_t kv = sim_budget(b);
     const unsigned grid = (unsigned)(b.n_inst * n_lambda);
     int q_shift = -1;
     if ((cm.decode_kv_div & (cm.decode_kv_div - 1)) == 0)
         for (q_shift = 0; (1u << q_shift) != cm.decode_kv_div; ++q_shift) {}
-    const size_t smem_n = simulate_steal_smem(b.n_clients, b.batch_cap, false);
-    const size_t smem_w = simulate_steal_smem(b.n_clients, b.batch_cap, true);
+    const size_t smem_n = simulate_steal_smem(b.n_clients, cap, false);
+    const size_t smem_w = simulate_steal_smem(b.n_clients, cap, true);
     cudaError_t e = cudaFuncSetAttribute(k_simulate_steal<NarrowEntry>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_n);
     if (e != cudaSuccess) return e;
     launch_hook("k_simulate_steal", 0, st);
     k_simulate_steal<NarrowEntry><<<grid, threads, smem_n, st>>>(
-        q_po, q_req, q_off, inst_status, lambda_q16, n_lambda, b.n_clients, b.n_req, n_pad, b.batch_cap,
-        (uint32_t)b.kv_budget, cm, q_shift, max_iters, cres, trace, trace_off, status, served_by);
+        q_po, b.o_est ? q_key : nullptr, q_req, q_off, inst_status, lambda_q16, n_lambda, b.n_clients, b.n_req, n_pad, cap,
+        kv, cm, q_shift, max_iters, cres, trace, trace_off, status, served_by);
     launch_hook("k_simulate_steal", 1, st);
     if (b.kv_budget >= 65536) {                          // otherwise no p + o can reach 2^16
         e = cudaFuncSetAttribute(k_simulate_steal<WideEntry>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_w);
         if (e != cudaSuccess) return e;
         launch_hook("k_simulate_steal_wide", 0, st);
         k_simulate_steal<WideEntry><<<grid, threads, smem_w, st>>>(
-            q_po, q_req, q_off, inst_status, lambda_q16, n_lambda, b.n_clients, b.n_req, n_pad, b.batch_cap,
-            (uint32_t)b.kv_budget, cm, q_shift, max_iters, cres, trace, trace_off, status, served_by);
+            q_po, b.o_est ? q_key : nullptr, q_req, q_off, inst_status, lambda_q16, n_lambda, b.n_clients, b.n_req, n_pad, cap,
+            kv, cm, q_shift, max_iters, cres, trace, trace_off, status, served_by);
         launch_hook("k_simulate_steal_wide", 1, st);
     }
     return cudaGetLastError();

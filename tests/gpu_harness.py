@@ -14,10 +14,11 @@ def to_dev(a, dtype=np.int32):
     return torch.from_numpy(a.astype(dtype, copy=False)).cuda()
 
 
-def gpu_offline(hos, p, o, M, cap, kv, cm, ls_rounds):
-    r = hos.hos_offline_pack(to_dev(p), to_dev(o), M, cap, kv, cm, ls_rounds, want_log=True, want_lb=True)
+def gpu_offline(hos, p, o, M, cap, kv, cm, ls_rounds, est=None, rsv=0):
+    ek = dict(o_est=None if est is None else to_dev(est), kv_reserve=rsv)
+    r = hos.hos_offline_pack(to_dev(p), to_dev(o), M, cap, kv, cm, ls_rounds, want_log=True, want_lb=True, **ek)
     import torch
-    sep = hos.hos_lower_bound(to_dev(p), to_dev(o), M, cap, kv, cm)
+    sep = hos.hos_lower_bound(to_dev(p), to_dev(o), M, cap, kv, cm, **ek)
     assert torch.equal(r["lb"], sep["lb"]), "bounds from hos_offline_pack differ from hos_lower_bound"
     out = {k: (v.cpu().numpy() if v is not None and k not in ("ls_log", "lb") else v) for k, v in r.items()}
     if r["ls_log"] is not None:
@@ -26,12 +27,12 @@ def gpu_offline(hos, p, o, M, cap, kv, cm, ls_rounds):
     return out
 
 
-def check_offline(hos, p, o, M, cap, kv, cm, ls_rounds, insts=None):
+def check_offline(hos, p, o, M, cap, kv, cm, ls_rounds, insts=None, est=None, rsv=0):
     """GPU offline pack of the whole batch against the oracle on `insts` (default: all)."""
-    g = gpu_offline(hos, p, o, M, cap, kv, cm, ls_rounds)
+    g = gpu_offline(hos, p, o, M, cap, kv, cm, ls_rounds, est, rsv)
     insts = range(p.shape[0]) if insts is None else insts
     for k in insts:
-        e = ora.offline_pack(p[k], o[k], M, cm, ls_rounds)
+        e = ora.offline_pack(p[k], o[k] if est is None else est[k], M, cm, ls_rounds)   # packed on what is known
         assert g["status"][k] == 0
         assert np.array_equal(g["assign"][k], e["assign"]), f"assign differs in instance {k}"
         assert np.array_equal(g["load"][k], e["load"]), f"load differs in instance {k}"
@@ -44,14 +45,18 @@ def check_offline(hos, p, o, M, cap, kv, cm, ls_rounds, insts=None):
     return g
 
 
-def check_lower_bound(hos, p, o, M, cap, kv, cm, insts=None):
+def check_lower_bound(hos, p, o, M, cap, kv, cm, insts=None, est=None, rsv=0):
     from paper_2502_15763_b200.binding import view_struct
-    r = hos.hos_lower_bound(to_dev(p), to_dev(o), M, cap, kv, cm)
+    r = hos.hos_lower_bound(to_dev(p), to_dev(o), M, cap, kv, cm, o_est=None if est is None else to_dev(est),
+                            kv_reserve=rsv)
     lb = view_struct(r["lb"], hos.LB_DTYPE)
     st = r["status"].cpu().numpy()
     insts = range(p.shape[0]) if insts is None else insts
     for k in insts:
         e = ora.lower_bound(p[k], o[k], M, cap, cm)
+        if est is not None:          # the packing bounds are in units of the estimated times
+            e.update({f: v for f, v in ora.lower_bound(p[k], est[k], M, cap, cm).items()
+                      if f in ("lb_pack", "sum_T", "max_T", "pair_T")})
         assert st[k] == 0
         for f, v in e.items():
             assert int(lb[k][f]) == v, f"lower bound field {f} differs in instance {k}"
@@ -59,7 +64,7 @@ def check_lower_bound(hos, p, o, M, cap, kv, cm, insts=None):
 
 
 def gpu_simulate(hos, p, o, M, cap, kv, cm, assign, lambdas, mode, max_iters=0x7FFFFFFF, want_trace=True,
-                 trace_slots=None):
+                 trace_slots=None, est=None, rsv=0):
     """Counts (with the event log), offsets, then the trace twice: rebuilt from the event log by
     hos_trace_fill and written directly by a traced simulation; the two must be the same bytes.
     Returns host-side views."""
@@ -67,7 +72,8 @@ def gpu_simulate(hos, p, o, M, cap, kv, cm, assign, lambdas, mode, max_iters=0x7
     from paper_2502_15763_b200.binding import view_struct
     dp, do, da = to_dev(p), to_dev(o), to_dev(assign)
     dl = to_dev(np.asarray(lambdas, dtype=np.uint32))
-    r = hos.hos_online_simulate(dp, do, M, cap, kv, cm, da, dl, mode, max_iters, keep_events=want_trace)
+    ek = dict(o_est=None if est is None else to_dev(est), kv_reserve=rsv)
+    r = hos.hos_online_simulate(dp, do, M, cap, kv, cm, da, dl, mode, max_iters, keep_events=want_trace, **ek)
     out = dict(cres=view_struct(r["cres"], hos.CLIENT_RESULT_DTYPE),
                sres=view_struct(r["sres"], hos.SIM_RESULT_DTYPE), status=r["status"].cpu().numpy())
     if want_trace:
@@ -78,14 +84,15 @@ def gpu_simulate(hos, p, o, M, cap, kv, cm, assign, lambdas, mode, max_iters=0x7
             off = torch.arange(n_units + 1, dtype=torch.int64, device="cuda") * int(trace_slots)
         total = int(off[-1].item())
         trace = torch.zeros((max(total, 1), 16), dtype=torch.uint8, device="cuda")
-        r2 = hos.hos_online_simulate(dp, do, M, cap, kv, cm, da, dl, mode, max_iters, trace=trace, trace_off=off)
+        r2 = hos.hos_online_simulate(dp, do, M, cap, kv, cm, da, dl, mode, max_iters, trace=trace, trace_off=off,
+                                     **ek)
         out2 = dict(cres=view_struct(r2["cres"], hos.CLIENT_RESULT_DTYPE),
                     sres=view_struct(r2["sres"], hos.SIM_RESULT_DTYPE), status=r2["status"].cpu().numpy())
         for f in out["cres"].dtype.names:
             assert np.array_equal(out["cres"][f], out2["cres"][f]), f"traced run changed cres.{f}"
         out["status_traced"] = out2["status"]
         filled = torch.zeros_like(trace)
-        hos.hos_trace_fill(dp, do, M, cap, kv, cm, len(lambdas), r, filled, off)
+        hos.hos_trace_fill(dp, do, M, cap, kv, cm, len(lambdas), r, filled, off, **ek)
         assert torch.equal(filled, trace), "trace rebuilt from the event log differs from the traced simulation"
         assert np.array_equal(r["status"].cpu().numpy(), out2["status"]), "status after hos_trace_fill differs"
         out["trace"] = view_struct(trace, hos.ITER_REC_DTYPE)
@@ -94,13 +101,14 @@ def gpu_simulate(hos, p, o, M, cap, kv, cm, assign, lambdas, mode, max_iters=0x7
 
 
 def check_simulate(hos, p, o, M, cap, kv, cm, assign, lambdas, mode, insts=None, max_iters=0x7FFFFFFF,
-                   want_trace=True):
-    g = gpu_simulate(hos, p, o, M, cap, kv, cm, assign, lambdas, mode, max_iters, want_trace)
+                   want_trace=True, est=None, rsv=0):
+    g = gpu_simulate(hos, p, o, M, cap, kv, cm, assign, lambdas, mode, max_iters, want_trace, est=est, rsv=rsv)
     insts = range(p.shape[0]) if insts is None else insts
     nl = len(lambdas)
     for k in insts:
         for li, lam in enumerate(lambdas):
-            e = ora.simulate(assign[k], p[k], o[k], M, cm, cap, kv, int(lam), mode, max_iters, want_trace)
+            e = ora.simulate(assign[k], p[k], o[k], M, cm, cap, kv, int(lam), mode, max_iters, want_trace,
+                             o_est=None if est is None else est[k], kv_reserve=rsv)
             s = g["sres"][k, li]
             assert int(s["makespan_us"]) == e.makespan_us, (k, li)
             assert int(s["busy_slot_us"]) == e.busy_slot_us
@@ -124,17 +132,19 @@ def check_simulate(hos, p, o, M, cap, kv, cm, assign, lambdas, mode, insts=None,
     return g
 
 
-def check_simulate_steal(hos, p, o, M, cap, kv, cm, assign, lambdas, mode, insts=None, max_iters=0x7FFFFFFF):
+def check_simulate_steal(hos, p, o, M, cap, kv, cm, assign, lambdas, mode, insts=None, max_iters=0x7FFFFFFF,
+                         est=None, rsv=0):
     """hos_online_simulate_steal (counts, then a traced run with exact slots) against the oracle."""
     import torch
     from paper_2502_15763_b200.binding import view_struct
     dp, do, da = to_dev(p), to_dev(o), to_dev(assign)
     dl = to_dev(np.asarray(lambdas, dtype=np.uint32))
-    r = hos.hos_online_simulate_steal(dp, do, M, cap, kv, cm, da, dl, mode, max_iters, want_served_by=True)
+    ek = dict(o_est=None if est is None else to_dev(est), kv_reserve=rsv)
+    r = hos.hos_online_simulate_steal(dp, do, M, cap, kv, cm, da, dl, mode, max_iters, want_served_by=True, **ek)
     off = hos.hos_trace_offsets(r["cres"])
     trace = torch.zeros((max(int(off[-1].item()), 1), 16), dtype=torch.uint8, device="cuda")
     r2 = hos.hos_online_simulate_steal(dp, do, M, cap, kv, cm, da, dl, mode, max_iters, trace=trace, trace_off=off,
-                                       want_served_by=True)
+                                       want_served_by=True, **ek)
     assert torch.equal(r["cres"][..., :32], r2["cres"][..., :32]) and torch.equal(r["served_by"], r2["served_by"])
     cres = view_struct(r2["cres"], hos.CLIENT_RESULT_DTYPE)
     sres = view_struct(r2["sres"], hos.SIM_RESULT_DTYPE)
@@ -146,7 +156,8 @@ def check_simulate_steal(hos, p, o, M, cap, kv, cm, assign, lambdas, mode, insts
     nl = len(lambdas)
     for k in insts:
         for li, lam in enumerate(lambdas):
-            e, eserved = ora.simulate_steal(assign[k], p[k], o[k], M, cm, cap, kv, int(lam), mode, max_iters, True)
+            e, eserved = ora.simulate_steal(assign[k], p[k], o[k], M, cm, cap, kv, int(lam), mode, max_iters, True,
+                                            o_est=None if est is None else est[k], kv_reserve=rsv)
             assert np.array_equal(served[k, li], eserved), f"served_by differs: inst {k} lambda {li}"
             s = sres[k, li]
             assert int(s["makespan_us"]) == e.makespan_us and int(s["busy_slot_us"]) == e.busy_slot_us

@@ -250,6 +250,39 @@ def test_paper_shaped_workload(hos):
     assert (hyb["sres"]["utilisation"][:, 0] > base["sres"]["utilisation"][:, 0]).mean() >= 0.5
 
 
+def test_estimated_output_lengths(hos):
+    """Packing, queues and queued-token counts on estimates, simulation on the true lengths, a fixed
+    reservation per request: batch of the c2e workload, plus small ragged cases with tight budgets."""
+    w = workload("c2e").subset(0, 12)
+    p, o = w.lengths()
+    est = w.estimates()
+    M, cap, kv, cm, R = w.n_clients, w.batch_cap, w.kv_budget, w.cost_model, w.kv_reserve
+    g = H.check_offline(hos, p, o, M, cap, kv, cm, 10, est=est, rsv=R)
+    H.check_lower_bound(hos, p, o, M, cap, kv, cm, est=est, rsv=R)
+    for mode in (ora.QUEUE_SORTED, ora.QUEUE_FCFS):
+        H.check_simulate(hos, p, o, M, cap, kv, cm, g["assign"], LAMS, mode, insts=range(0, 12, 3), est=est, rsv=R)
+    H.check_simulate_steal(hos, p, o, M, cap, kv, cm, g["assign"], (LAMBDA_ONE, 20000), ora.QUEUE_SORTED,
+                           insts=range(0, 12, 4), est=est, rsv=R)
+    rng = np.random.default_rng(77)
+    for n, M, cap, R, kv in ((37, 3, 5, 700, 2500), (130, 5, 4, 640, 640), (64, 2, 9, 900, 5000)):
+        p = rng.integers(1, 300, (3, n)).astype(np.uint32)
+        o = rng.integers(1, 300, (3, n)).astype(np.uint32)
+        est = np.clip(np.rint(o * np.exp(0.6 * rng.standard_normal((3, n)))), 1, 400).astype(np.uint32)
+        g = H.check_offline(hos, p, o, M, cap, kv, cm, 6, est=est, rsv=R)
+        H.check_simulate(hos, p, o, M, cap, kv, cm, g["assign"], LAMS, ora.QUEUE_SORTED, est=est, rsv=R)
+        H.check_simulate_steal(hos, p, o, M, cap, kv, cm, g["assign"], (LAMBDA_ONE,), ora.QUEUE_SORTED, est=est, rsv=R)
+    # estimates without a reservation, a reservation above the budget: refused on the host;
+    # a request longer than the reservation: the instance is marked invalid on the device
+    with pytest.raises(hos.HosError):
+        hos.hos_offline_pack(H.to_dev(p), H.to_dev(o), M, cap, kv, cm, 0, o_est=H.to_dev(est))
+    with pytest.raises(hos.HosError):
+        hos.hos_offline_pack(H.to_dev(p), H.to_dev(o), M, cap, 500, cm, 0, kv_reserve=600)
+    o2 = o.copy()
+    o2[1, 5] = 900
+    r = hos.hos_offline_pack(H.to_dev(p), H.to_dev(o2), M, cap, kv, cm, 0, o_est=H.to_dev(est), kv_reserve=R)
+    assert r["status"].cpu().tolist() == [0, hos.HOS_ST_INVALID, 0]
+
+
 def test_limits_and_bad_data(hos):
     w = workload("c0")
     p, o = w.lengths()
