@@ -35,7 +35,18 @@ L2_FLUSH_BYTES = 256 << 20
 
 # algorithmic bytes per unit of work of each kernel (what a streaming implementation of that
 # step alone must move once)
-BYTES_PER_REQ = {"k_estimate_sort": 16, "k_lpt": 12, "k_lower_bound": 8, "k_queue_build": 16}
+BYTES_PER_REQ = {"k_estimate_sort": 16, "k_lpt": 12, "k_lower_bound": 8, "k_queue_build": 16, "k_ls_lists": 15}
+# what bounds each kernel (counters in profiles/): streaming kernels against the measured copy
+# bandwidth, the two sequential recurrences against the integer issue rate
+BOUND = {"k_simulate": "alu", "k_simulate_steal": "alu", "k_lpt": "latency (dependent chain)",
+         "k_local_search": "latency / issue (instance resident on chip; bytes are those of a streaming round)"}
+# integer operations of one simulated iteration as the method states it: duration (3), busy slot
+# time (2), clock (1), waited decode time (2), sum of KV lengths (1), decision compare in Q16.16 (3),
+# trace hash (9), counters (3)
+INT_OPS_PER_ITERATION = 24
+# DRAM bytes per request and launch measured with ncu (dram__bytes_read.sum + dram__bytes_write.sum
+# over 296 instances of c4's shape, see profiles/); None for a kernel changed since its capture
+NCU_DRAM_BYTES_PER_REQ = {}
 
 
 def describe(w: Workload) -> str:
@@ -72,7 +83,7 @@ class ClockSampler:
     def start(self):
         try:
             self.proc = subprocess.Popen(
-                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "100",
+                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "50",
                  "-i", str(self.index)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             threading.Thread(target=self._read, daemon=True).start()
         except OSError:
@@ -123,6 +134,10 @@ class Pipeline:
         self.lam_host = torch.from_numpy(np.asarray(w.lambdas_q16, dtype=np.uint32).view(np.int32)).pin_memory()
         self.p = self.p_host.to(device)
         self.o = self.o_host.to(device)
+        est = w.estimates()                  # None unless the workload schedules on estimated lengths
+        self.est_host = None if est is None else torch.from_numpy(est.view(np.int32)).pin_memory()
+        self.est = None if est is None else self.est_host.to(device)
+        self.kw = dict(o_est=self.est, kv_reserve=w.kv_reserve)
         self.lam = self.lam_host.to(device)
         self.ws_off = None
         self.ws_on = None
@@ -141,14 +156,14 @@ class Pipeline:
         hos, w = self.hos, self.w
         sweep = len(w.lambdas_q16) > 1
         # a multiplier sweep runs its local-search rounds per (instance, multiplier) copy, below
-        pk = hos.hos_offline_pack(*self.args(), 0 if sweep else w.ls_rounds, ws=self.ws_off, want_lb=True)
+        pk = hos.hos_offline_pack(*self.args(), 0 if sweep else w.ls_rounds, ws=self.ws_off, want_lb=True, **self.kw)
         return self.online(pk)
 
     def prepare(self):
         """Workspaces (allocated once; the library itself allocates nothing)."""
         import ctypes as C
         from paper_2502_15763_b200 import binding as B
-        b = B._batch(*self.args()[:5])
+        b = B._batch(*self.args()[:5], self.est, self.w.kv_reserve)
         L = self.hos.lib()
         n_off = L.hos_offline_workspace_bytes(C.byref(b), len(self.w.lambdas_q16), self.w.ls_rounds)
         n_on = L.hos_online_workspace_bytes(C.byref(b), len(self.w.lambdas_q16), 1)
@@ -160,16 +175,16 @@ class Pipeline:
         hos, w = self.hos, self.w
         lb = dict(lb=pk["lb"])                      # Eq. 31-32 bounds, computed inside hos_offline_pack
         s1 = hos.hos_online_simulate(*self.args(), pk["assign"], self.lam, hos.HOS_QUEUE_SORTED,
-                                     keep_events=True, ws=self.ws_on)
+                                     keep_events=True, ws=self.ws_on, **self.kw)
         off = hos.hos_trace_offsets(s1["cres"])
         if self.trace is None:                      # first (warm-up) step sizes the trace buffer
             self.n_iters = int(off[-1].item())
             self.trace = self.torch.empty((max(self.n_iters, 1), 16), dtype=self.torch.uint8, device=self.dev)
-        hos.hos_trace_fill(*self.args(), len(w.lambdas_q16), s1, self.trace, off)
+        hos.hos_trace_fill(*self.args(), len(w.lambdas_q16), s1, self.trace, off, **self.kw)
         self.out = dict(pk=pk, lb=lb, sim=s1, off=off)
         if len(w.lambdas_q16) > 1 and w.ls_rounds > 0:
             copies = pk["assign"][:, None, :].expand(-1, len(w.lambdas_q16), -1).contiguous()
-            self.out["ls"] = hos.hos_local_search(*self.args(), copies, w.ls_rounds, ws=self.ws_off)
+            self.out["ls"] = hos.hos_local_search(*self.args(), copies, w.ls_rounds, ws=self.ws_off, **self.kw)
         return self.out
 
     def e2e_step(self, host_out):
@@ -203,6 +218,8 @@ class Pipeline:
             for f, n in self.chunks:
                 self.p[f:f + n].copy_(self.p_host[f:f + n], non_blocking=True)
                 self.o[f:f + n].copy_(self.o_host[f:f + n], non_blocking=True)
+                if self.est is not None:
+                    self.est[f:f + n].copy_(self.est_host[f:f + n], non_blocking=True)
                 ev = torch.cuda.Event()
                 ev.record(cs)
                 arrived.append(ev)
@@ -211,7 +228,8 @@ class Pipeline:
             main.wait_event(ev)
             hos.hos_offline_pack(self.p[f:f + n], self.o[f:f + n], w.n_clients, w.batch_cap, w.kv_budget,
                                  w.cost_model, 0 if sweep else w.ls_rounds, ws=self.ws_off,
-                                 out={k: v[f:f + n] for k, v in pk.items()})
+                                 out={k: v[f:f + n] for k, v in pk.items()},
+                                 o_est=None if self.est is None else self.est[f:f + n], kv_reserve=w.kv_reserve)
         packed = torch.cuda.Event()
         packed.record(main)
         early = (pk["assign"], pk["load"], pk["makespan_est"], pk["status"])
@@ -230,7 +248,8 @@ class Pipeline:
         for h, d in zip(host_out[4:], late):
             h.copy_(d, non_blocking=True)
         main.wait_stream(cs)
-        h2d = sum(t.numel() * t.element_size() for t in (self.p_host, self.o_host, self.lam_host))
+        h2d = sum(t.numel() * t.element_size() for t in (self.p_host, self.o_host, self.lam_host, self.est_host)
+                  if t is not None)
         d2h = sum(t.numel() * t.element_size() for t in early + late)
         return h2d, d2h
 
@@ -323,15 +342,18 @@ def oracle_sample(w: Workload, n_sample: int):
     from oracle import hos_oracle as ora
     sub = w.subset(0, n_sample)
     p, o = sub.lengths()
+    est = sub.estimates()
     t0 = time.perf_counter()
     iters = 0
     for k in range(sub.n_inst):
         sweep = len(w.lambdas_q16) > 1
-        pk = ora.offline_pack(p[k], o[k], w.n_clients, w.cost_model, 0 if sweep else w.ls_rounds)
+        pk = ora.offline_pack(p[k], o[k] if est is None else est[k], w.n_clients, w.cost_model,
+                              0 if sweep else w.ls_rounds)
         ora.lower_bound(p[k], o[k], w.n_clients, w.batch_cap, w.cost_model)
         for lam in w.lambdas_q16:
             s = ora.simulate(pk["assign"], p[k], o[k], w.n_clients, w.cost_model, w.batch_cap, w.kv_budget,
-                             lam, ora.QUEUE_SORTED, want_trace=True)
+                             lam, ora.QUEUE_SORTED, want_trace=True, o_est=None if est is None else est[k],
+                             kv_reserve=w.kv_reserve)
             iters += sum(c.n_prefill_iters + c.n_decode_iters for c in s.clients)
             if sweep and w.ls_rounds > 0:      # local search on a private copy per multiplier value
                 ora.local_search(pk["T"], pk["assign"], pk["load"], w.ls_rounds)
@@ -403,7 +425,7 @@ def run_ours(args):
     steal_ms = None
     if rank == 0 and not args.skip_steal:
         run_steal = lambda: hos.hos_online_simulate_steal(*pipe.args(), pipe.out["pk"]["assign"], pipe.lam,
-                                                          hos.HOS_QUEUE_SORTED, ws=pipe.ws_on)
+                                                          hos.HOS_QUEUE_SORTED, ws=pipe.ws_on, **pipe.kw)
         run_steal()
         torch.cuda.synchronize()
         steal_ms = timed_steps(torch, run_steal, 3, flush) / 3
@@ -422,10 +444,29 @@ def run_ours(args):
             gbs = by / (r["ms_per_launch"] * 1e-3) / 1e9
             rows[name] = dict(r, algorithmic_bytes=by, achieved_gbs=gbs, frac=gbs / peak,
                               ms_per_step=r["ms_per_launch"] * r["launches_per_step"])
+        for name in rows:
+            rows[name]["bound"] = BOUND.get(name, "hbm")
         top = max(rows, key=lambda n: rows[n]["ms_per_step"])
-        roofline = {"kernel": top, "bound": "hbm", "achieved": rows[top]["achieved_gbs"], "peak": peak,
-                    "unit": "GB/s", "frac": rows[top]["frac"], "traffic": None,
-                    "peak_source": f"of {peak_kind}", "ms_per_launch": rows[top]["ms_per_launch"]}
+        per_req = NCU_DRAM_BYTES_PER_REQ.get(top)
+        traffic = None if per_req is None else per_req * w.n_inst * w.n_req * len(w.lambdas_q16)
+        if BOUND.get(top) == "alu":
+            # the iteration recurrence is integer arithmetic: operations of the method per second
+            # against 128 int32 lanes per SM at the maximum SM clock
+            props = torch.cuda.get_device_properties(dev)
+            mhz = (clocks or {}).get("sm_max_mhz") or 1965.0
+            alu_peak = props.multi_processor_count * 128 * mhz * 1e6 / 1e12
+            ach = INT_OPS_PER_ITERATION * pipe.n_iters / (rows[top]["ms_per_launch"] * 1e-3) / 1e12
+            roofline = {"kernel": top, "bound": "alu", "achieved": ach, "peak": alu_peak, "unit": "Tint32op/s",
+                        "frac": ach / alu_peak, "traffic": traffic,
+                        "peak_source": "SMs x 128 int32 lanes x max SM clock",
+                        "ops_per_iteration": INT_OPS_PER_ITERATION, "ms_per_launch": rows[top]["ms_per_launch"]}
+        else:
+            roofline = {"kernel": top, "bound": "hbm", "achieved": rows[top]["achieved_gbs"], "peak": peak,
+                        "unit": "GB/s", "frac": rows[top]["frac"], "traffic": traffic,
+                        "peak_source": f"of {peak_kind}", "ms_per_launch": rows[top]["ms_per_launch"]}
+            if top == "k_local_search":
+                roofline["note"] = ("effective: bytes a streaming implementation would re-read every executed "
+                                    "round; this kernel reads the instance from HBM once")
         launches = sum(r["launches_per_step"] for r in prof.values())
         n_s = sample_size(w)
         if args.skip_cpu_baseline:
@@ -498,9 +539,9 @@ def run_reference(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=3)
-    ap.add_argument("--workload", default="c4", choices=["c0", "c1", "c2", "c3", "c4", "paper"])
+    ap.add_argument("--workload", default="c4", choices=["c0", "c1", "c2", "c3", "c4", "paper", "c1e", "c2e"])
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--instances", type=int, default=0,
                     help="use only the first N instances of the workload (profiling captures)")

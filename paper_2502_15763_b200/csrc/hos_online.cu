@@ -195,13 +195,86 @@ k_simulate(const uint2* __restrict__ q_po, const int32_t* __restrict__ q_off,
         if (it < tr_lim) tr[it] = make_uint4(dur, r1, r2, r3);
     };
 
-    // Every pass of this loop is one "event" iteration (a prefill, or a decode that may retire
-    // requests) followed by a quiet run of decode iterations in which nobody retires and the
-    // decision cannot change.  The lanes of a warp meet again at every event, so the heap and
-    // queue work is done by all of them together and the quiet runs are short scalar loops.
+    // One decode iteration (one token for every running request), popping every request that
+    // retires with it.  Returns the number retired; leaves duration and batch figures in dur, r1, r2.
     // The heap is 4-ary: half the depth of a binary heap, and the four children of a node are
     // independent loads.
+    uint32_t dur, r1, r2, r3;
+    auto decode_step = [&]() {
+        dur = ad + bd * B + (q_shift >= 0 ? (S >> q_shift) : (S / qd));
+        r1 = B; r2 = S;
+        uint32_t gone_n = 0;
+        busy += (long long)dur * B;
+        S += B;
+        if (cnt + 1 == next_fin) {
+            const uint32_t c1 = cnt + 1;
+            uint32_t n = B;
+            do {                                      // pop every request that retires now
+                const uint32_t gone = E::tot(heap_ld(0));
+                S -= gone;
+                reserved -= gone;
+                ++gone_n;
+                --n;
+                const entry_t x = heap_ld((int)n);
+                const entry_t xr = E::rel(x, c1);
+                uint32_t i = 0;
+                while (true) {
+                    const uint32_t ch = 4 * i + 1;
+                    if (ch >= n) break;
+                    // children beyond the heap's end compare as +infinity
+                    entry_t y0 = heap_ld((int)ch), ym = y0;
+                    entry_t m = E::rel(y0, c1);
+                    uint32_t at = ch;
+#pragma unroll
+                    for (uint32_t k = 1; k < 4; ++k) {
+                        if (ch + k < n) {
+                            const entry_t y = heap_ld((int)(ch + k));
+                            const entry_t r = E::rel(y, c1);
+                            if (r < m) { m = r; ym = y; at = ch + k; }
+                        }
+                    }
+                    if (xr <= m) break;
+                    heap_st((int)i, ym);
+                    i = at;
+                }
+                if (n > 0) heap_st((int)i, x);
+            } while (n > 0 && E::fin(heap_ld(0), c1) == c1);
+            B = n;
+            next_fin = n > 0 ? E::fin(heap_ld(0), c1) : EMPTY;
+            grow = head + (int)nA < qn;
+        }
+        r3 = gone_n;
+    };
+    // Bookkeeping of an event iteration (dur, r1, r2, r3): event log, clock, hash, trace, waited
+    // decode time.  False when the clock limit is reached.
+    auto finish_event = [&]() {
+        if (ev && ((r1 >> 31) || r3 != 0u)) {          // something changed: log it with the state after it
+            ev[2 * n_ev] = make_uint4(n_pre + cnt, B, S, 0u);
+            ev[2 * n_ev + 1] = make_uint4(dur, r1, r2, r3);
+            ++n_ev;
+        }
+        emit(dur, r1, r2, r3);
+        if (r1 >> 31) { Cd = 0; ++n_pre; }
+        else { ++cnt; Cd = min(Cd + dur, 0x7FFFFFFFu); }  // both below 2^31: no wrap
+        if (t >= (1ll << 39)) { status |= HOS_ST_LIMIT; return false; }
+        return true;
+    };
+
+    // Every pass of this loop is: a decode iteration that retires requests, if that is what comes
+    // next (the usual way a quiet run ends); then one general "event" iteration (a prefill, or any
+    // decode); then a quiet run of decode iterations in which nobody retires and the decision
+    // cannot change.  In steady state a client goes retire -> prefill -> quiet run, so a pass is a
+    // whole cycle and the lanes of a warp, which meet again at every pass, spend it in the same
+    // code.  The first part only does what the general part would do with that iteration.
     while (true) {
+        if (!grow && B > 0 && cnt + 1 == next_fin && n_pre + cnt != max_iters) {
+            // the candidate prefix is current (grow is false), so the decision can be taken here
+            const unsigned long long Cp16f = (unsigned long long)prefill_us(cm, sumP) << 16;
+            if (nA == 0 || (unsigned long long)lam * Cd <= Cp16f) {
+                decode_step();
+                if (!finish_event()) break;
+            }
+        }
         if (grow) {
             // candidates: the longest queue prefix that fits the free slots and the KV budget.
             // A retirement only loosens both limits, so the prefix found earlier stays valid.
@@ -223,7 +296,6 @@ k_simulate(const uint2* __restrict__ q_po, const int32_t* __restrict__ q_off,
 
         const uint32_t Cp = prefill_us(cm, sumP);
         const unsigned long long Cp16 = (unsigned long long)Cp << 16;
-        uint32_t dur, r1, r2, r3;
         if (nA > 0 && (B == 0 || (unsigned long long)lam * Cd > Cp16)) {
             // prefill: push the candidates, last staged first (its slot is the lowest, so the
             // growing heap never reaches a candidate that is still waiting)
@@ -249,59 +321,9 @@ k_simulate(const uint2* __restrict__ q_po, const int32_t* __restrict__ q_off,
             grow = stage_cap != 0xFFFFFFFFu && head < qn;
             next_fin = E::fin(heap_ld(0), cnt);
         } else {
-            dur = ad + bd * B + (q_shift >= 0 ? (S >> q_shift) : (S / qd));
-            r1 = B; r2 = S;
-            uint32_t gone_n = 0;
-            busy += (long long)dur * B;
-            S += B;
-            if (cnt + 1 == next_fin) {
-                const uint32_t c1 = cnt + 1;
-                uint32_t n = B;
-                do {                                      // pop every request that retires now
-                    const uint32_t gone = E::tot(heap_ld(0));
-                    S -= gone;
-                    reserved -= gone;
-                    ++gone_n;
-                    --n;
-                    const entry_t x = heap_ld((int)n);
-                    const entry_t xr = E::rel(x, c1);
-                    uint32_t i = 0;
-                    while (true) {
-                        const uint32_t ch = 4 * i + 1;
-                        if (ch >= n) break;
-                        // children beyond the heap's end compare as +infinity
-                        entry_t y0 = heap_ld((int)ch), ym = y0;
-                        entry_t m = E::rel(y0, c1);
-                        uint32_t at = ch;
-#pragma unroll
-                        for (uint32_t k = 1; k < 4; ++k) {
-                            if (ch + k < n) {
-                                const entry_t y = heap_ld((int)(ch + k));
-                                const entry_t r = E::rel(y, c1);
-                                if (r < m) { m = r; ym = y; at = ch + k; }
-                            }
-                        }
-                        if (xr <= m) break;
-                        heap_st((int)i, ym);
-                        i = at;
-                    }
-                    if (n > 0) heap_st((int)i, x);
-                } while (n > 0 && E::fin(heap_ld(0), c1) == c1);
-                B = n;
-                next_fin = n > 0 ? E::fin(heap_ld(0), c1) : EMPTY;
-                grow = head + (int)nA < qn;
-            }
-            r3 = gone_n;
+            decode_step();
         }
-        if (ev && ((r1 >> 31) || r3 != 0u)) {          // something changed: log it with the state after it
-            ev[2 * n_ev] = make_uint4(n_pre + cnt, B, S, 0u);
-            ev[2 * n_ev + 1] = make_uint4(dur, r1, r2, r3);
-            ++n_ev;
-        }
-        emit(dur, r1, r2, r3);
-        if (r1 >> 31) { Cd = 0; ++n_pre; }
-        else { ++cnt; Cd = min(Cd + dur, 0x7FFFFFFFu); }  // both below 2^31: no wrap
-        if (t >= (1ll << 39)) { status |= HOS_ST_LIMIT; break; }
+        if (!finish_event()) break;
         if (grow || B == 0) continue;
         // quiet run: at most `room` iterations -- up to the next retirement, the iteration limit,
         // and so few that only the last of them can take the clock past its limit (every
