@@ -46,7 +46,9 @@ BOUND = {"k_simulate": "alu", "k_simulate_steal": "alu", "k_lpt": "latency (depe
 INT_OPS_PER_ITERATION = 24
 # DRAM bytes per request and launch measured with ncu (dram__bytes_read.sum + dram__bytes_write.sum
 # over 296 instances of c4's shape, see profiles/); None for a kernel changed since its capture
-NCU_DRAM_BYTES_PER_REQ = {}
+NCU_DRAM_BYTES_PER_REQ = {"k_estimate_sort": 8.70, "k_lower_bound": 8.04, "k_lpt": 12.68, "k_ls_lists": 18.90,
+                          "k_local_search": 6.07, "k_queue_build": 17.41, "k_simulate": 41.67}
+NCU_DRAM_BYTES_PER_ITERATION = {"k_trace_fill": 20.93}
 
 
 def describe(w: Workload) -> str:
@@ -412,10 +414,12 @@ def run_ours(args):
 
     # end to end: pinned host tables in, pinned host results out, every step
     host_out = []
-    h2d, d2h = pipe.e2e_step(host_out)
-    barrier()
-    ms_e2e = timed_steps(torch, lambda: pipe.e2e_step(host_out), args.steps, flush)
-    barrier()
+    h2d, d2h, ms_e2e = 0, 0, 0.0
+    if not args.skip_e2e:
+        h2d, d2h = pipe.e2e_step(host_out)
+        barrier()
+        ms_e2e = timed_steps(torch, lambda: pipe.e2e_step(host_out), args.steps, flush)
+        barrier()
     e_t = torch.tensor([ms_e2e], dtype=torch.float64, device=dev)
     if world > 1:
         dist.all_reduce(e_t, op=dist.ReduceOp.MAX)
@@ -447,8 +451,19 @@ def run_ours(args):
         for name in rows:
             rows[name]["bound"] = BOUND.get(name, "hbm")
         top = max(rows, key=lambda n: rows[n]["ms_per_step"])
-        per_req = NCU_DRAM_BYTES_PER_REQ.get(top)
-        traffic = None if per_req is None else per_req * w.n_inst * w.n_req * len(w.lambdas_q16)
+        def dram_traffic(name):
+            # scaled from the capture by the units a launch processes (requests of every instance or
+            # simulation; iterations for the trace)
+            if name in NCU_DRAM_BYTES_PER_ITERATION:
+                return NCU_DRAM_BYTES_PER_ITERATION[name] * pipe.n_iters
+            per_req = NCU_DRAM_BYTES_PER_REQ.get(name)
+            if per_req is None:
+                return None
+            sims = len(w.lambdas_q16) if name in ("k_simulate", "k_local_search", "k_ls_lists") and len(w.lambdas_q16) > 1 else 1
+            return per_req * w.n_inst * w.n_req * sims
+        for name in rows:
+            rows[name]["traffic"] = dram_traffic(name)
+        traffic = dram_traffic(top)
         if BOUND.get(top) == "alu":
             # the iteration recurrence is integer arithmetic: operations of the method per second
             # against 128 int32 lanes per SM at the maximum SM clock
@@ -484,7 +499,7 @@ def run_ours(args):
             "sim_iterations_per_step": pipe.n_iters * world,
             "sim_iterations_per_s": pipe.n_iters * world * args.steps / (ms * 1e-3),
             "clocks": clocks,
-            "e2e": {"value": total_inst * args.steps / (ms_e2e * 1e-3), "unit": UNIT,
+            "e2e": {"value": None if args.skip_e2e else total_inst * args.steps / (ms_e2e * 1e-3), "unit": UNIT,
                     "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                     "note": "results copied back: assignment, loads, bounds, client and simulation results; "
                             "the iteration trace stays on the device; uploads and the offline part are pipelined by "
@@ -547,6 +562,8 @@ def main():
                     help="use only the first N instances of the workload (profiling captures)")
     ap.add_argument("--skip-steal", action="store_true",
                     help="do not time the request-stealing simulation (profiling captures)")
+    ap.add_argument("--skip-e2e", action="store_true",
+                    help="do not time the end-to-end step (profiling captures: one launch per kernel and step)")
     ap.add_argument("--skip-cpu-baseline", action="store_true",
                     help="do not time the CPU oracle (profiling captures)")
     args = ap.parse_args()
