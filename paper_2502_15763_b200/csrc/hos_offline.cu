@@ -480,6 +480,125 @@ __device__ inline void warp_patch_list(uint32_t* segT, IdxT* segI, int len, int 
     if (lane == 0) { segT[at] = valT; segI[at] = (IdxT)valI; }
 }
 
+// The same lists from the clients by rank that the packing kernel left (rcl), with coalesced
+// list writes.  Counts per (client, warp) and their scan give every warp the place of its members
+// in each client's list, as in build_member_lists.  Then a warp takes its ranks LSB_SUB at a time:
+// it counts them per client, lays them out by client in a staging area of its own (a client's
+// members of these ranks are consecutive in that client's list), and writes the staging area out
+// in order, so that neighbouring lanes write neighbouring list entries instead of one list each.
+// `stage` holds, per warp, LSB_SUB entries of T, index and client and two words per client.
+constexpr int LSB_SUB = 512;
+template <typename IdxT>
+__host__ __device__ constexpr size_t lists_stage_bytes_per_warp(int n_clients) {
+    return (size_t)LSB_SUB * (4 + sizeof(IdxT) + 1) + (size_t)((n_clients + 3) & ~3) * 8;
+}
+template <typename IdxT, int NT>
+__device__ inline void place_lists_staged(const uint8_t* __restrict__ rcl, const uint32_t* __restrict__ gO,
+                                          const uint32_t* __restrict__ gT, IdxT* clI, uint32_t* clT, int n,
+                                          int n_clients, uint32_t* cnt, uint32_t* wsum, int* off,
+                                          unsigned char* stage) {
+    constexpr int NW = NT / 32, STRIDE = NW + 1;
+    const int lane = lane_id(), warp = warp_id();
+    const int chunk = (((n + NW - 1) / NW) + 31) & ~31;
+    const int lo = warp * chunk, hi = min(n, lo + chunk);
+    const int nb = bit_width_u32((uint32_t)(n_clients - 1));
+    const int mpad = (n_clients + 3) & ~3;
+    unsigned char* mine = stage + (size_t)warp * lists_stage_bytes_per_warp<IdxT>(n_clients);
+    uint32_t* stT = reinterpret_cast<uint32_t*>(mine);
+    uint32_t* lcur = stT + LSB_SUB;                          // per client: next free staging slot
+    uint32_t* lbeg = lcur + mpad;                            // per client: its first staging slot
+    IdxT* stI = reinterpret_cast<IdxT*>(lbeg + mpad);
+    uint8_t* stC = reinterpret_cast<uint8_t*>(stI + LSB_SUB);
+
+    for (int x = threadIdx.x; x < n_clients * STRIDE; x += NT) cnt[x] = 0;
+    __syncthreads();
+    for (int r4 = lo + 4 * lane; r4 < hi; r4 += 128) {       // four ranks per lane and read
+        const uint32_t w = *reinterpret_cast<const uint32_t*>(rcl + r4);
+#pragma unroll
+        for (int e = 0; e < 4; ++e)
+            if (r4 + e < hi) atomicAdd(&cnt[((w >> (8 * e)) & 0xFFu) * STRIDE + warp], 1u);
+    }
+    __syncthreads();
+    block_scan_u32<NT>(cnt, n_clients * STRIDE, wsum);
+    for (int k = threadIdx.x; k <= n_clients; k += NT) off[k] = k < n_clients ? (int)cnt[k * STRIDE] : n;
+    __syncthreads();
+
+    const int per = (n_clients + 31) / 32;                  // clients per lane in the scan below
+    for (int sub = lo; sub < hi; sub += LSB_SUB) {
+        const int end = min(hi, sub + LSB_SUB);
+        for (int c = lane; c < n_clients; c += 32) lcur[c] = 0;
+        __syncwarp();
+        for (int r4 = sub + 4 * lane; r4 < end; r4 += 128) {
+            const uint32_t w = *reinterpret_cast<const uint32_t*>(rcl + r4);
+#pragma unroll
+            for (int e = 0; e < 4; ++e)
+                if (r4 + e < end) atomicAdd(&lcur[(w >> (8 * e)) & 0xFFu], 1u);
+        }
+        __syncwarp();
+        {   // exclusive scan of the counts over the clients: first staging slot of every client
+            uint32_t run = 0;
+            for (int k = 0; k < per; ++k) { const int c = lane * per + k; if (c < n_clients) run += lcur[c]; }
+            uint32_t inc = run;
+#pragma unroll
+            for (int d = 1; d < 32; d <<= 1) {
+                const uint32_t y = __shfl_up_sync(FULL, inc, d);
+                if (lane >= d) inc += y;
+            }
+            uint32_t acc = inc - run;
+            for (int k = 0; k < per; ++k) {
+                const int c = lane * per + k;
+                if (c < n_clients) { const uint32_t v = lcur[c]; lbeg[c] = acc; lcur[c] = acc; acc += v; }
+            }
+        }
+        __syncwarp();
+        for (int row = sub; row < end; row += 32 * LS_ROWS) {
+            uint32_t id[LS_ROWS], tr[LS_ROWS], dig[LS_ROWS];
+            unsigned m[LS_ROWS];
+#pragma unroll
+            for (int e = 0; e < LS_ROWS; ++e) {
+                const int r = row + e * 32 + lane;
+                const bool valid = r < end;
+                id[e] = valid ? __ldg(&gO[r]) : 0u;
+                tr[e] = valid ? __ldg(&gT[r]) : 0u;
+                dig[e] = valid ? (uint32_t)rcl[r] : 0u;
+                m[e] = __ballot_sync(FULL, valid);
+            }
+            for (int b = 0; b < nb; ++b) {                   // lanes of each row on my client
+#pragma unroll
+                for (int e = 0; e < LS_ROWS; ++e) {
+                    const bool bit = (dig[e] >> b) & 1u;
+                    const unsigned bal = __ballot_sync(FULL, bit);
+                    m[e] &= bit ? bal : ~bal;
+                }
+            }
+#pragma unroll
+            for (int e = 0; e < LS_ROWS; ++e) {
+                const bool valid = row + e * 32 + lane < end;
+                const uint32_t base = valid ? lcur[dig[e]] : 0u;
+                __syncwarp();
+                if (valid) {
+                    const uint32_t at = base + __popc(m[e] & ((1u << lane) - 1u));
+                    stT[at] = tr[e];
+                    stI[at] = (IdxT)id[e];
+                    stC[at] = (uint8_t)dig[e];
+                    if (lane == (__ffs(m[e]) - 1)) lcur[dig[e]] = base + __popc(m[e]);
+                }
+                __syncwarp();
+            }
+        }
+        for (int x = lane; x < end - sub; x += 32) {         // staging slot x -> its place in the client's list
+            const uint32_t c = stC[x];
+            const uint32_t g = cnt[c * STRIDE + warp] + ((uint32_t)x - lbeg[c]);
+            clT[g] = stT[x];
+            clI[g] = stI[x];
+        }
+        __syncwarp();
+        for (int c = lane; c < n_clients; c += 32) cnt[c * STRIDE + warp] += lcur[c] - lbeg[c];
+        __syncwarp();
+    }
+    __syncthreads();
+}
+
 // Member lists before the first round: one CTA per (instance, copy).  Leaves the lists (ws_T,
 // ws_I), their offsets (ws_off, n_clients + 1 per unit) and, for a caller's assignment, the
 // clients' loads; ws_bad[unit] != 0 marks an assignment outside [0, n_clients).
@@ -505,14 +624,15 @@ k_ls_lists(const uint32_t* __restrict__ T_sorted, const uint32_t* __restrict__ o
     for (int j = threadIdx.x; j < n_clients; j += LSB_THREADS) s_load[j] = 0;
     __syncthreads();
     // a caller's assignment is gathered and checked; the packing kernel's comes with the clients by rank
-    const bool failed =
-        load_from_assign
-            ? build_member_lists<IdxT, true, true, LSB_THREADS>(asg, ws_C + unit * n_pad, gO, gT, ws_I + unit * n_pad,
-                                                                ws_T + unit * n_pad, n_req, n_clients, cnt, s_wsum,
-                                                                s_off, s_load)
-            : build_member_lists<IdxT, false, false, LSB_THREADS>(asg, ws_C + unit * n_pad, gO, gT,
-                                                                  ws_I + unit * n_pad, ws_T + unit * n_pad, n_req,
-                                                                  n_clients, cnt, s_wsum, s_off, nullptr);
+    bool failed = false;
+    if (load_from_assign)
+        failed = build_member_lists<IdxT, true, true, LSB_THREADS>(asg, ws_C + unit * n_pad, gO, gT,
+                                                                   ws_I + unit * n_pad, ws_T + unit * n_pad, n_req,
+                                                                   n_clients, cnt, s_wsum, s_off, s_load);
+    else
+        place_lists_staged<IdxT, LSB_THREADS>(ws_C + unit * n_pad, gO, gT, ws_I + unit * n_pad, ws_T + unit * n_pad,
+                                              n_req, n_clients, cnt, s_wsum, s_off,
+                                              smem_raw + (((size_t)n_clients * (LSB_THREADS / 32 + 1) * 4 + 15) & ~(size_t)15));
     if (threadIdx.x == 0) ws_bad[unit] = failed ? 1 : 0;
     if (failed) return;
     for (int k = threadIdx.x; k <= n_clients; k += LSB_THREADS) ws_off[unit * (n_clients + 1) + k] = s_off[k];
@@ -972,16 +1092,17 @@ k_local_search(const uint32_t* __restrict__ T_sorted, const uint32_t* __restrict
 // Lower bounds.  One CTA per instance; reads p, o once, and T_(M), T_(M+1) from the sorted
 // table left by k_estimate_sort.
 // ---------------------------------------------------------------------------------------
-__device__ __forceinline__ unsigned long long floor_sum_below(uint32_t n, uint32_t q) {
+__device__ __forceinline__ unsigned long long floor_sum_below(uint32_t n, uint32_t q, int q_shift) {
     // sum over x in [0, n) of floor(x / q); n and q fit 32 bits, so one 32-bit division does
-    const uint32_t m = n / q, r = n - m * q;
+    // (a shift when q = 2^q_shift, q_shift >= 0)
+    const uint32_t m = q_shift >= 0 ? n >> q_shift : n / q, r = n - m * q;
     return (unsigned long long)q * (((unsigned long long)m * (m - 1u + (m == 0u))) >> 1) +
            (unsigned long long)m * r;                           // m = 0 -> 0
 }
 
 __global__ void __launch_bounds__(256)
 k_lower_bound(const uint32_t* __restrict__ p, const uint32_t* __restrict__ o, int n_req, int n_pad,
-              int n_clients, int cap, hos_cost_model cm, const uint32_t* __restrict__ T_sorted,
+              int n_clients, int cap, hos_cost_model cm, int q_shift, const uint32_t* __restrict__ T_sorted,
               const InstInfo* __restrict__ info, hos_lb* __restrict__ out) {
     __shared__ unsigned long long red[32];
     const int inst = blockIdx.x;
@@ -1000,8 +1121,8 @@ k_lower_bound(const uint32_t* __restrict__ p, const uint32_t* __restrict__ o, in
         O += oo;
         K += (unsigned long long)oo * pp + (((unsigned long long)oo * (oo - 1u)) >> 1);
         const unsigned long long alone = (unsigned long long)prefill_us(cm, pp) + oo * (ad + bd) +
-                                         floor_sum_below(pp + oo, cm.decode_kv_div) -
-                                         floor_sum_below(pp, cm.decode_kv_div);
+                                         floor_sum_below(pp + oo, cm.decode_kv_div, q_shift) -
+                                         floor_sum_below(pp, cm.decode_kv_div, q_shift);
         chain = alone > chain ? alone : chain;
     };
     constexpr int UN = 4;                                       // reads in flight per thread and table
@@ -1110,7 +1231,14 @@ cudaError_t launch_local_search(const hos_batch& b, const uint32_t* T_sorted, co
                                 int32_t* status, uint32_t* ws_T, void* ws_I, uint8_t* ws_C, int32_t* ws_off,
                                 int32_t* ws_bad, cudaStream_t st) {
     const size_t smem = local_search_smem(b.n_req, b.n_clients);
-    const size_t smem_lists = (size_t)b.n_clients * (LSB_THREADS / 32 + 1) * 4;
+    const bool narrow = b.n_req <= 65536;
+    const size_t smem_lists = (((size_t)b.n_clients * (LSB_THREADS / 32 + 1) * 4 + 15) & ~(size_t)15) +
+                              (load_from_assign ? 0
+                                                : (LSB_THREADS / 32) * (narrow ? lists_stage_bytes_per_warp<uint16_t>(b.n_clients)
+                                                                               : lists_stage_bytes_per_warp<uint32_t>(b.n_clients)));
+    cudaError_t ea = narrow ? cudaFuncSetAttribute(k_ls_lists<uint16_t>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_lists)
+                            : cudaFuncSetAttribute(k_ls_lists<uint32_t>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_lists);
+    if (ea != cudaSuccess) return ea;
     const unsigned grid = (unsigned)(b.n_inst * n_copies);
     launch_hook("k_ls_lists", 0, st);
     if (b.n_req <= 65536)
@@ -1139,8 +1267,11 @@ cudaError_t launch_local_search(const hos_batch& b, const uint32_t* T_sorted, co
 
 cudaError_t launch_lower_bound(const hos_batch& b, const hos_cost_model& cm, const uint32_t* T_sorted,
                                const InstInfo* info, int n_pad, hos_lb* out, cudaStream_t st) {
+    int q_shift = -1;                                    // power-of-two KV divisor -> shift
+    if ((cm.decode_kv_div & (cm.decode_kv_div - 1)) == 0)
+        for (q_shift = 0; (1u << q_shift) != cm.decode_kv_div; ++q_shift) {}
     launch_hook("k_lower_bound", 0, st);
-    k_lower_bound<<<b.n_inst, 256, 0, st>>>(b.p, b.o, b.n_req, n_pad, b.n_clients, b.batch_cap, cm,
+    k_lower_bound<<<b.n_inst, 256, 0, st>>>(b.p, b.o, b.n_req, n_pad, b.n_clients, b.batch_cap, cm, q_shift,
                                             T_sorted, info, out);
     launch_hook("k_lower_bound", 1, st);
     return cudaGetLastError();
