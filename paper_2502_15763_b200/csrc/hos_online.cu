@@ -99,6 +99,7 @@ k_queue_build(const uint32_t* __restrict__ p, const uint32_t* __restrict__ o,
 // sum KV is carried along: S += B - sum of retired tot.
 // ---------------------------------------------------------------------------------------
 constexpr uint32_t EMPTY = 0xFFFFFFFFu;
+constexpr int SIM_QUIET_MAX = 4;          // plain decode iterations per pass of the simulator's loop
 constexpr unsigned long long HASH_INIT = 0xCBF29CE484222325ull;
 constexpr uint32_t HASH_C1 = 0x9E3779B1u, HASH_C2 = 0x85EBCA77u, HASH_C3 = 0xC2B2AE3Du, HASH_M = 0x27D4EB2Fu;
 constexpr int SIM_THREADS = 32;          // heap stride: the 32 clients of one warp sit side by side
@@ -260,19 +261,18 @@ k_simulate(const uint2* __restrict__ q_po, const int32_t* __restrict__ q_off,
         return true;
     };
 
-    // Every pass of this loop is: a decode iteration that retires requests, if that is what comes
-    // next (the usual way a quiet run ends); then one general "event" iteration (a prefill, or any
-    // decode); then a quiet run of decode iterations in which nobody retires and the decision
-    // cannot change.  In steady state a client goes retire -> prefill -> quiet run, so a pass is a
-    // whole cycle and the lanes of a warp, which meet again at every pass, spend it in the same
-    // code.  The first part only does what the general part would do with that iteration.
-    while (true) {
+    // The event part of a pass: a decode iteration that retires requests, if that is what comes
+    // next (the usual way a quiet run ends), then one general "event" iteration (a prefill, or any
+    // decode).  The first only does what the second would do with that iteration.  Returns 0 when
+    // a quiet run may follow, 1 when the next pass must start with an event again, 2 when the client
+    // is done or has hit a limit.
+    auto event_part = [&]() -> int {
         if (!grow && B > 0 && cnt + 1 == next_fin && n_pre + cnt != max_iters) {
             // the candidate prefix is current (grow is false), so the decision can be taken here
             const unsigned long long Cp16f = (unsigned long long)prefill_us(cm, sumP) << 16;
             if (nA == 0 || (unsigned long long)lam * Cd <= Cp16f) {
                 decode_step();
-                if (!finish_event()) break;
+                if (!finish_event()) return 2;
             }
         }
         if (grow) {
@@ -291,8 +291,8 @@ k_simulate(const uint2* __restrict__ q_po, const int32_t* __restrict__ q_off,
             }
             grow = false;
         }
-        if (B == 0 && nA == 0) break;                    // queue empty and nothing running
-        if (n_pre + cnt == max_iters) { status |= HOS_ST_LIMIT; break; }
+        if (B == 0 && nA == 0) return 2;                 // queue empty and nothing running
+        if (n_pre + cnt == max_iters) { status |= HOS_ST_LIMIT; return 2; }
 
         const uint32_t Cp = prefill_us(cm, sumP);
         const unsigned long long Cp16 = (unsigned long long)Cp << 16;
@@ -323,13 +323,31 @@ k_simulate(const uint2* __restrict__ q_po, const int32_t* __restrict__ q_off,
         } else {
             decode_step();
         }
-        if (!finish_event()) break;
-        if (grow || B == 0) continue;
+        if (!finish_event()) return 2;
+        return (grow || B == 0) ? 1 : 0;
+    };
+
+    // Every pass of this loop is the event part, then a quiet run of decode iterations in which
+    // nobody retires and the decision cannot change.  In steady state a client goes retire ->
+    // prefill -> quiet run, so a pass is a whole cycle and the lanes of a warp, which meet again at
+    // every pass, spend it in the same code.  A quiet run is cut after SIM_QUIET_MAX iterations, so
+    // that the warp does not wait for its longest run; a client whose run was cut skips the event
+    // part of the next pass and goes on with its run.
+    bool cut = false;                                    // my quiet run was cut and goes on
+    while (true) {
+        if (!cut) {
+            const int act = event_part();
+            if (act == 2) break;
+            if (act == 1) continue;
+        }
         // quiet run: at most `room` iterations -- up to the next retirement, the iteration limit,
         // and so few that only the last of them can take the clock past its limit (every
         // iteration adds less than 2^31) -- and only while the rule keeps saying "decode"
+        const unsigned long long Cp16 = (unsigned long long)prefill_us(cm, sumP) << 16;
         const uint32_t room_t = (uint32_t)(((1ll << 39) - 1 - t) >> 31) + 1u;
         uint32_t room = min(min(next_fin - cnt - 1u, max_iters - (n_pre + cnt)), room_t);
+        const bool capped = room > (uint32_t)SIM_QUIET_MAX;
+        if (capped) room = SIM_QUIET_MAX;
         const uint32_t lam_run = nA > 0 ? lam : 0u;      // no candidates: nothing to prefill
         const uint32_t base = ad + bd * B;
         const long long t_run = t;
@@ -343,6 +361,7 @@ k_simulate(const uint2* __restrict__ q_po, const int32_t* __restrict__ q_off,
         }
         busy += (t - t_run) * (long long)B;
         if (t >= (1ll << 39)) { status |= HOS_ST_LIMIT; break; }
+        cut = capped && room == 0 && (unsigned long long)lam_run * Cd <= Cp16;   // the cap ended it, not the rule
     }
     if (tr && n_pre + cnt > tr_lim) status |= HOS_ST_TRACE;
     const uint32_t n_dec = cnt;
