@@ -99,7 +99,7 @@ k_queue_build(const uint32_t* __restrict__ p, const uint32_t* __restrict__ o,
 // sum KV is carried along: S += B - sum of retired tot.
 // ---------------------------------------------------------------------------------------
 constexpr uint32_t EMPTY = 0xFFFFFFFFu;
-constexpr int SIM_QUIET_MAX = 4;          // plain decode iterations per pass of the simulator's loop
+constexpr int SIM_QUIET_MAX = 16;         // plain decode iterations per pass of the simulator's loop
 constexpr unsigned long long HASH_INIT = 0xCBF29CE484222325ull;
 constexpr uint32_t HASH_C1 = 0x9E3779B1u, HASH_C2 = 0x85EBCA77u, HASH_C3 = 0xC2B2AE3Du, HASH_M = 0x27D4EB2Fu;
 constexpr int SIM_THREADS = 32;          // heap stride: the 32 clients of one warp sit side by side
