@@ -142,13 +142,16 @@ k_simulate(const uint2* __restrict__ q_po, const int32_t* __restrict__ q_off,
     auto heap_ld = [&](int sl) -> entry_t { return heap[sl * SIM_THREADS]; };
     auto heap_st = [&](int sl, entry_t v) { heap[sl * SIM_THREADS] = v; };
     const long long unit = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-    if (unit >= n_units) return;
-    const int c = (int)(unit % n_clients);
-    const int l = (int)((unit / n_clients) % n_lambda);
-    const int inst = (int)(unit / ((long long)n_clients * n_lambda));
+    const bool in_range = unit < n_units;
+    const int c = in_range ? (int)(unit % n_clients) : 0;
+    const int l = in_range ? (int)((unit / n_clients) % n_lambda) : 0;
+    const int inst = in_range ? (int)(unit / ((long long)n_clients * n_lambda)) : 0;
 
     const int ist = inst_status[inst];
-    if (((ist & INST_WIDE) != 0) != (sizeof(entry_t) == 8)) return;   // the other instantiation's instance
+    const bool mine = in_range && ((ist & INST_WIDE) != 0) == (sizeof(entry_t) == 8);   // else: the other instantiation's
+    // the lanes of this warp that simulate a client: they meet at the end of every pass of the loop
+    unsigned live = __ballot_sync(FULL, mine && !(ist & HOS_ST_INVALID));
+    if (!mine) return;
     if (ist & HOS_ST_INVALID) {
         cres[unit] = hos_client_result{0, 0, 0u, 0u, 0ull, 0.0};
         status_out[unit] = HOS_ST_INVALID;
@@ -335,33 +338,36 @@ k_simulate(const uint2* __restrict__ q_po, const int32_t* __restrict__ q_off,
     // part of the next pass and goes on with its run.
     bool cut = false;                                    // my quiet run was cut and goes on
     while (true) {
-        if (!cut) {
-            const int act = event_part();
-            if (act == 2) break;
-            if (act == 1) continue;
+        int act = 0;
+        if (!cut) act = event_part();
+        bool done = act == 2;
+        if (act == 0) {
+            // quiet run: at most `room` iterations -- up to the next retirement, the iteration limit,
+            // and so few that only the last of them can take the clock past its limit (every
+            // iteration adds less than 2^31) -- and only while the rule keeps saying "decode"
+            const unsigned long long Cp16 = (unsigned long long)prefill_us(cm, sumP) << 16;
+            const uint32_t room_t = (uint32_t)(((1ll << 39) - 1 - t) >> 31) + 1u;
+            uint32_t room = min(min(next_fin - cnt - 1u, max_iters - (n_pre + cnt)), room_t);
+            const bool capped = room > (uint32_t)SIM_QUIET_MAX;
+            if (capped) room = SIM_QUIET_MAX;
+            const uint32_t lam_run = nA > 0 ? lam : 0u;  // no candidates: nothing to prefill
+            const uint32_t base = ad + bd * B;
+            const long long t_run = t;
+            while (room > 0 && (unsigned long long)lam_run * Cd <= Cp16) {
+                const uint32_t dq = base + (q_shift >= 0 ? (S >> q_shift) : (S / qd));
+                emit(dq, B, S, 0u);
+                ++cnt;
+                S += B;
+                Cd = min(Cd + dq, 0x7FFFFFFFu);
+                --room;
+            }
+            busy += (t - t_run) * (long long)B;
+            if (t >= (1ll << 39)) { status |= HOS_ST_LIMIT; done = true; }
+            cut = capped && room == 0 && (unsigned long long)lam_run * Cd <= Cp16;   // the cap ended it, not the rule
         }
-        // quiet run: at most `room` iterations -- up to the next retirement, the iteration limit,
-        // and so few that only the last of them can take the clock past its limit (every
-        // iteration adds less than 2^31) -- and only while the rule keeps saying "decode"
-        const unsigned long long Cp16 = (unsigned long long)prefill_us(cm, sumP) << 16;
-        const uint32_t room_t = (uint32_t)(((1ll << 39) - 1 - t) >> 31) + 1u;
-        uint32_t room = min(min(next_fin - cnt - 1u, max_iters - (n_pre + cnt)), room_t);
-        const bool capped = room > (uint32_t)SIM_QUIET_MAX;
-        if (capped) room = SIM_QUIET_MAX;
-        const uint32_t lam_run = nA > 0 ? lam : 0u;      // no candidates: nothing to prefill
-        const uint32_t base = ad + bd * B;
-        const long long t_run = t;
-        while (room > 0 && (unsigned long long)lam_run * Cd <= Cp16) {
-            const uint32_t dq = base + (q_shift >= 0 ? (S >> q_shift) : (S / qd));
-            emit(dq, B, S, 0u);
-            ++cnt;
-            S += B;
-            Cd = min(Cd + dq, 0x7FFFFFFFu);
-            --room;
-        }
-        busy += (t - t_run) * (long long)B;
-        if (t >= (1ll << 39)) { status |= HOS_ST_LIMIT; break; }
-        cut = capped && room == 0 && (unsigned long long)lam_run * Cd <= Cp16;   // the cap ended it, not the rule
+        // every lane still simulating arrives here once per pass: the warp starts the next pass together
+        live = __ballot_sync(live, !done);
+        if (done) break;
     }
     if (tr && n_pre + cnt > tr_lim) status |= HOS_ST_TRACE;
     const uint32_t n_dec = cnt;
