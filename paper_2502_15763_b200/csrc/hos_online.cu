@@ -299,7 +299,10 @@ k_simulate(const uint2* __restrict__ q_po, const int32_t* __restrict__ q_off,
 
         const uint32_t Cp = prefill_us(cm, sumP);
         const unsigned long long Cp16 = (unsigned long long)Cp << 16;
-        if (nA > 0 && (B == 0 || (unsigned long long)lam * Cd > Cp16)) {
+        const bool want_prefill = nA > 0 && (B == 0 || (unsigned long long)lam * Cd > Cp16);
+        // plain decodes (nobody retires, the rule says decode) are the quiet run's business
+        if (!want_prefill && cnt + 1 != next_fin) return 0;
+        if (want_prefill) {
             // prefill: push the candidates, last staged first (its slot is the lowest, so the
             // growing heap never reaches a candidate that is still waiting)
             for (uint32_t j = 0; j < nA; ++j) {
