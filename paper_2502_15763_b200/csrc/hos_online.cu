@@ -35,7 +35,7 @@ k_queue_build(const uint32_t* __restrict__ p, const uint32_t* __restrict__ o,
     const uint32_t* ei = o_est ? o_est + (size_t)inst * n_req : oi;   // the lengths the scheduler sorts by
 
     // kv_budget here is the most KV one request may need: the fixed reservation, if there is one
-    unsigned long long sumO = 0, mx = 0, mxk = 0, bad = 0;
+    unsigned long long sumO = 0, mx = 0, mxk = 0, mxp = 0, bad = 0;
     for (int i = threadIdx.x; i < n_req; i += SORT_THREADS) {
         const uint32_t pp = pi[i], oo = oi[i], oe = ei[i];
         const int c = ai[i];
@@ -49,10 +49,12 @@ k_queue_build(const uint32_t* __restrict__ p, const uint32_t* __restrict__ o,
         sumO += oo;
         mx = tot > mx ? tot : mx;
         mxk = totk > mxk ? totk : mxk;
+        mxp = pp > mxp ? pp : mxp;
     }
     sumO = block_sum_u64(sumO, red);
     mx = block_max_u64(mx, red);
     mxk = block_max_u64(mxk, red);
+    mxp = block_max_u64(mxp, red);
     bad = block_max_u64(bad, red);
     __syncthreads();
     if (threadIdx.x == 0) {
@@ -65,9 +67,16 @@ k_queue_build(const uint32_t* __restrict__ p, const uint32_t* __restrict__ o,
     const int kb = (queue_order == HOS_QUEUE_SORTED) ? bit_width_u32((uint32_t)mxk) : 0;
     const uint32_t kmask = kb >= 32 ? 0xFFFFFFFFu : ((1u << kb) - 1u);
     const int nbits = kb + bit_width_u32((uint32_t)(n_clients - 1));
+    // The sort only looks at the low nbits of a key.  When the prompt length fits the bits above
+    // them it rides along there, so that the queue entries are written without going back to the
+    // request tables in queue order (a scattered read per request); with the key p + o the
+    // output length follows from it too.
+    const bool ride = nbits + bit_width_u32((uint32_t)mxp) <= 32;
+    const bool o_from_key = ride && kb > 0 && kb < 32 && !o_est;
     for (int i = threadIdx.x; i < n_req; i += SORT_THREADS) {
         const uint32_t c = (uint32_t)s.buf1[i];
-        s.key[i] = (kb >= 32 ? 0u : (c << kb)) | (kmask - (s.key[i] & kmask));
+        const uint32_t low = (kb >= 32 ? 0u : (c << kb)) | (kmask - (s.key[i] & kmask));
+        s.key[i] = ride ? (low | (nbits >= 32 ? 0u : (pi[i] << nbits))) : low;
     }
     __syncthreads();
     const IdxT* sorted = block_radix_sort_ids<IdxT>(s, n_req, nbits, 0u);
@@ -77,11 +86,16 @@ k_queue_build(const uint32_t* __restrict__ p, const uint32_t* __restrict__ o,
     int32_t* qo = q_off + (size_t)inst * (n_clients + 1);
     for (int r = threadIdx.x; r < n_req; r += SORT_THREADS) {
         const uint32_t id = sorted[r];
+        const uint32_t key = s.key[id];
+        const uint32_t low = (ride && nbits < 32) ? (key & ((1u << nbits) - 1u)) : key;
+        const uint32_t pp = (ride && nbits < 32) ? key >> nbits : pi[id];
+        const uint32_t totk = kmask - (low & kmask);             // p + (estimated) o, when it is the key
         qr[r] = id;
-        qp[r] = make_uint2(pi[id], oi[id]);
-        if (q_key) q_key[(size_t)inst * n_pad + r] = pi[id] + ei[id];
-        const int c = (int)(s.key[id] >> kb);
-        const int cprev = r > 0 ? (int)(s.key[sorted[r - 1]] >> kb) : -1;
+        qp[r] = make_uint2(pp, o_from_key ? totk - pp : oi[id]);
+        if (q_key) q_key[(size_t)inst * n_pad + r] = kb > 0 && kb < 32 ? totk : pp + ei[id];
+        const int c = (int)(low >> kb);
+        const uint32_t kprev = r > 0 ? s.key[sorted[r - 1]] : 0u;
+        const int cprev = r > 0 ? (int)(((ride && nbits < 32) ? (kprev & ((1u << nbits) - 1u)) : kprev) >> kb) : -1;
         for (int cc = cprev + 1; cc <= c; ++cc) qo[cc] = r;
         if (r == n_req - 1)
             for (int cc = c + 1; cc <= n_clients; ++cc) qo[cc] = n_req;
