@@ -81,6 +81,7 @@ k_lpt(const uint32_t* __restrict__ T_sorted, const uint32_t* __restrict__ order,
       int32_t* __restrict__ assign, long long* __restrict__ load_out,
       long long* __restrict__ makespan_out, uint8_t* __restrict__ rank_client) {
     constexpr int JB = (KPL == 1) ? 5 : (KPL == 2) ? 6 : (KPL == 4) ? 7 : 8;
+    __shared__ uint32_t s_perm[32];
     const int inst = blockIdx.x;
     const int lane = threadIdx.x;
     const InstInfo inf = info[inst];
@@ -134,21 +135,20 @@ k_lpt(const uint32_t* __restrict__ T_sorted, const uint32_t* __restrict__ order,
             while (pos < steps) {
                 // sort all 32 * KPL keys ascending: element e = k * 32 + lane.  After a wave that
                 // placed 32 items on 64 clients, the lower half (key[0]) is new and the upper half
-                // is still in order: sorting the lower half alone and merging the two (the upper
-                // half reversed makes the whole bitonic) takes 21 compare-exchange steps on single
-                // registers instead of 21 on both.
+                // is still in order: the lower half is sorted alone and merged with the upper one
+                // (reversed, which makes the whole bitonic): 6 dependent compare-exchange steps
+                // instead of 21.
                 if (KPL == 2 && half_sorted) {
+                    // the new half by rank: 32 independent compares instead of 15 dependent steps
+                    // (keys are distinct: they carry their client)
                     uint32_t x = key[0];
+                    int rank = 0;
 #pragma unroll
-                    for (int size = 2; size <= 32; size <<= 1) {
-#pragma unroll
-                        for (int stride = size >> 1; stride > 0; stride >>= 1) {
-                            const uint32_t other = __shfl_xor_sync(FULL, x, stride);
-                            const bool up = (lane & size) == 0;
-                            const bool lower = (lane & stride) == 0;
-                            x = (lower == up) ? min(x, other) : max(x, other);
-                        }
-                    }
+                    for (int b = 0; b < 32; ++b) rank += __shfl_sync(FULL, x, b) < x ? 1 : 0;
+                    s_perm[rank] = x;
+                    __syncwarp();
+                    x = s_perm[lane];
+                    __syncwarp();
                     const uint32_t y = __shfl_sync(FULL, key[KPL - 1], 31 - lane);
                     uint32_t lo2 = min(x, y), hi2 = max(x, y);
 #pragma unroll
