@@ -23,7 +23,7 @@
  *     base must be 256-byte aligned.  Two calls that share a workspace or an
  *     output buffer must be ordered on the stream.
  *   - Shape limits of this build: n_clients <= 256, batch_cap <= 256,
- *     n_req <= 24576, kv_budget < 2^31, estimated times T_i < 2^32.
+ *     n_req <= 24384, kv_budget < 2^31, estimated times T_i < 2^32.
  */
 #ifndef HOS_H
 #define HOS_H

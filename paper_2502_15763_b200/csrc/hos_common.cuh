@@ -15,7 +15,7 @@ constexpr int RADIX_BITS = 8;
 constexpr int RADIX = 1 << RADIX_BITS;
 constexpr int MAX_CLIENTS = 256;
 constexpr int MAX_CAP = 256;
-constexpr int MAX_REQ = 24576;
+constexpr int MAX_REQ = 24384;          // the request table, two id buffers and the radix counters fill one CTA's shared memory
 constexpr size_t SMEM_LIMIT = 227 * 1024;
 
 // Per-instance facts left in the workspace by the estimate+sort kernel.

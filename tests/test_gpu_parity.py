@@ -283,6 +283,26 @@ def test_estimated_output_lengths(hos):
     assert r["status"].cpu().tolist() == [0, hos.HOS_ST_INVALID, 0]
 
 
+def test_maximum_request_count(hos):
+    """The largest instance the library takes (24,384 requests, 256 clients of 256 slots): the
+    shared-memory sort is at its size limit and the lists span every client; one more request is
+    refused on the host."""
+    rng = np.random.default_rng(24576)
+    n, M, cap = 24384, 256, 256
+    p = rng.integers(1, 2000, size=(2, n)).astype(np.uint32)
+    o = rng.integers(1, 150, size=(2, n)).astype(np.uint32)
+    cm = (20000, 40, 15000, 300, 16, 40, 350)
+    kv = 1 << 20
+    g = H.check_offline(hos, p, o, M, cap, kv, cm, 4, insts=[1])
+    H.check_lower_bound(hos, p, o, M, cap, kv, cm)
+    H.check_simulate(hos, p, o, M, cap, kv, cm, g["assign"], (LAMBDA_ONE, LAMBDA_PREFILL_FIRST), ora.QUEUE_SORTED,
+                     insts=[0])
+    H.check_simulate_steal(hos, p, o, 64, 64, kv, cm, g["assign"] % 64, (LAMBDA_ONE,), ora.QUEUE_SORTED, insts=[1])
+    with pytest.raises(hos.HosError):
+        hos.hos_offline_pack(H.to_dev(np.ones((1, n + 1), np.uint32)), H.to_dev(np.ones((1, n + 1), np.uint32)),
+                             M, cap, kv, cm)
+
+
 def test_limits_and_bad_data(hos):
     w = workload("c0")
     p, o = w.lengths()
