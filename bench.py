@@ -46,9 +46,9 @@ BOUND = {"k_simulate": "alu", "k_simulate_steal": "alu", "k_lpt": "latency (depe
 INT_OPS_PER_ITERATION = 24
 # DRAM bytes per request and launch measured with ncu (dram__bytes_read.sum + dram__bytes_write.sum
 # over 296 instances of c4's shape, see profiles/); None for a kernel changed since its capture
-NCU_DRAM_BYTES_PER_REQ = {"k_estimate_sort": 8.77, "k_lower_bound": 8.04, "k_lpt": 12.71, "k_ls_lists": 18.15,
-                          "k_local_search": 6.07, "k_queue_build": 17.61, "k_simulate": 42.18}
-NCU_DRAM_BYTES_PER_ITERATION = {"k_trace_fill": 20.95}
+NCU_DRAM_BYTES_PER_REQ = {"k_estimate_sort": 8.77, "k_lower_bound": 8.04, "k_lpt": 12.68, "k_ls_lists": 18.33,
+                          "k_local_search": 6.07, "k_queue_build": 15.67, "k_simulate": 41.74}
+NCU_DRAM_BYTES_PER_ITERATION = {"k_trace_fill": 20.93}
 
 
 def describe(w: Workload) -> str:
@@ -364,8 +364,8 @@ def oracle_sample(w: Workload, n_sample: int):
 
 
 def sample_size(w: Workload) -> int:
-    # about 5 s of single-thread oracle work per instance at the largest size, milliseconds at the others
-    per_inst = 5.0 if w.n_req >= 10000 else 0.025 * max(1, len(w.lambdas_q16)) + 0.03
+    # about 3 s of single-thread oracle work per instance at the largest size, milliseconds at the others
+    per_inst = 3.0 if w.n_req >= 10000 else 0.025 * max(1, len(w.lambdas_q16)) + 0.03
     return max(1, min(w.n_inst, int(12.0 / per_inst)))
 
 
