@@ -95,7 +95,7 @@ struct OnlineWs {
     unsigned long long* inst_O;
     int32_t* inst_status;
     uint32_t* event_count;      // [n_units]                      (keep_events only)
-    uint4* events;              // [n_sims][n_pad][2 events][2]   (keep_events only)
+    uint4* events;              // [n_sims][n_pad][2 events]      (keep_events only)
     size_t bytes;
 };
 OnlineWs carve_online(const hos_batch* b, void* ws, int n_lambda, int keep_events) {
@@ -115,7 +115,7 @@ OnlineWs carve_online(const hos_batch* b, void* ws, int n_lambda, int keep_event
     if (keep_events) {
         const size_t sims = (size_t)b->n_inst * (size_t)n_lambda;
         w.event_count = reinterpret_cast<uint32_t*>(base + off);  off += up(sims * b->n_clients * 4);
-        w.events = reinterpret_cast<uint4*>(base + off);          off += up(sims * pad4(b->n_req) * 2 * 32);
+        w.events = reinterpret_cast<uint4*>(base + off);          off += up(sims * pad4(b->n_req) * 2 * 16);
     }
     w.bytes = off;
     return w;

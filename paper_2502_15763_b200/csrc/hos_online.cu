@@ -196,8 +196,8 @@ k_simulate(const uint2* __restrict__ q_po, const int32_t* __restrict__ q_off,
         tr = reinterpret_cast<uint4*>(trace + t0);
         tr_lim = capr > 0x7FFFFFFFll ? 0x7FFFFFFFu : (uint32_t)(capr < 0 ? 0 : capr);
     }
-    // event log of this client: two 16-byte words per logged iteration, at most 2 per request
-    uint4* ev = events ? events + ((size_t)(inst * n_lambda + l) * n_pad + q0) * 4 : nullptr;
+    // event log of this client: one 16-byte entry per logged iteration, at most 2 per request
+    uint4* ev = events ? events + ((size_t)(inst * n_lambda + l) * n_pad + q0) * 2 : nullptr;
     uint32_t n_ev = 0;
     uint2 nxt = make_uint2(0u, 0u);          // queue entries head + nA and head + nA + 1,
     uint2 nxt2 = make_uint2(0u, 0u);         // fetched ahead of their use
@@ -266,9 +266,14 @@ k_simulate(const uint2* __restrict__ q_po, const int32_t* __restrict__ q_off,
     // Bookkeeping of an event iteration (dur, r1, r2, r3): event log, clock, hash, trace, waited
     // decode time.  False when the clock limit is reached.
     auto finish_event = [&]() {
-        if (ev && ((r1 >> 31) || r3 != 0u)) {          // something changed: log it with the state after it
-            ev[2 * n_ev] = make_uint4(n_pre + cnt, B, S, 0u);
-            ev[2 * n_ev + 1] = make_uint4(dur, r1, r2, r3);
+        if (ev && ((r1 >> 31) || r3 != 0u)) {
+            // Something changed: one 16-byte log entry {iteration, tokens, sum KV after it, packed}.
+            // A prefill packs flag | head << 16 | (batch after - 1) << 8 | (admitted - 1); a retiring
+            // decode packs (retired - 1) << 8 | (batch before - 1).  Batches hold at most 256 requests
+            // and queue positions stay below 2^15, durations follow from the tokens.
+            const uint32_t packed = (r1 >> 31) ? (0x80000000u | (r3 << 16) | ((B - 1u) << 8) | ((r1 & 0x7FFFFFFFu) - 1u))
+                                               : (((r3 - 1u) << 8) | (r1 - 1u));
+            ev[n_ev] = make_uint4(n_pre + cnt, r2, S, packed);
             ++n_ev;
         }
         emit(dur, r1, r2, r3);
@@ -693,7 +698,7 @@ k_trace_fill(const int32_t* __restrict__ q_off, int n_lambda, int n_clients, int
     const int sim = (int)(unit / n_clients);
     const int inst = sim / n_lambda;
     const int q0 = q_off[(size_t)inst * (n_clients + 1) + c];
-    const uint4* ev = events + ((size_t)sim * n_pad + q0) * 4;
+    const uint4* ev = events + ((size_t)sim * n_pad + q0) * 2;
     const uint32_t n_ev = event_count[unit];
     const uint32_t n_total = cres[unit].n_prefill_iters + cres[unit].n_decode_iters;
     const long long t0 = trace_off[unit];
@@ -708,17 +713,21 @@ k_trace_fill(const int32_t* __restrict__ q_off, int n_lambda, int n_clients, int
         const uint32_t it = base + lane;
         // iteration numbers of the next 32 log entries
         const uint32_t kw = k_next + lane;
-        const uint32_t itw = kw < n_ev ? ev[2 * (size_t)kw].x : 0xFFFFFFFFu;
+        const uint32_t itw = kw < n_ev ? ev[kw].x : 0xFFFFFFFFu;
         const uint32_t dw = itw - base;                                  // >= 0 by construction
         const uint32_t mask = __reduce_or_sync(FULL, dw < 32u ? (1u << dw) : 0u);
         const uint32_t upto = mask & (0xFFFFFFFFu >> (31 - lane));       // logged iterations <= it
         const uint32_t k = k_next + __popc(upto) - 1u;                   // iteration 0 is always logged
         if (it < lim) {
-            const uint4 st = ev[2 * (size_t)k];
+            const uint4 st = ev[k];                    // {iteration, tokens, sum KV after it, packed}
+            const bool pre = st.w >> 31;
+            const uint32_t lo8 = (st.w & 0xFFu) + 1u, hi8 = ((st.w >> 8) & 0xFFu) + 1u;
             uint4 rec;
-            if (st.x == it) rec = ev[2 * (size_t)k + 1];
-            else {
-                const uint32_t Bk = st.y;
+            if (st.x == it) {
+                if (pre) rec = make_uint4(prefill_us(cm, st.y), 0x80000000u | lo8, st.y, (st.w >> 16) & 0x7FFFu);
+                else rec = make_uint4(ad + bd * lo8 + (q_shift >= 0 ? (st.y >> q_shift) : (st.y / qd)), lo8, st.y, hi8);
+            } else {
+                const uint32_t Bk = pre ? hi8 : lo8 - hi8;               // batch after the logged iteration
                 const uint32_t Sk = st.z + (it - st.x - 1u) * Bk;
                 rec = make_uint4(ad + bd * Bk + (q_shift >= 0 ? (Sk >> q_shift) : (Sk / qd)), Bk, Sk, 0u);
             }
