@@ -646,8 +646,11 @@ k_simulate_steal(const uint2* __restrict__ q_po, const uint32_t* __restrict__ q_
     // at most `cap` requests per iteration, so a client with u unclaimed own requests cannot use
     // them up -- and so cannot steal -- before es = clock + (ceil(u / cap) - 1) * d_min.  Nothing is
     // stolen before H = max(s_first, min es over the unfinished clients), hence every iteration that
-    // starts before H only touches its own client and all of them may run side by side.  When none
-    // starts before H, the client at the front of the global order may steal: it runs alone.
+    // starts before H only touches its own client and all of them may run side by side: a client
+    // goes on, iteration after iteration, until its clock reaches H (the bound is taken from the
+    // state at the start of the step and only gets more conservative as the clients claim their
+    // own requests).  When none starts before H, the client at the front of the global order may
+    // steal: it runs alone, one iteration.
     // shortest possible iteration: a prefill of one token, or a decode of one request
     const unsigned long long d_min = min((unsigned long long)prefill_us(cm, 1u), (unsigned long long)ad + bd);
     while (true) {
@@ -658,9 +661,19 @@ k_simulate_steal(const uint2* __restrict__ q_po, const uint32_t* __restrict__ q_
             const unsigned long long u = (unsigned long long)(qend - s_ustart[c]);
             const unsigned long long k = u > (unsigned long long)cap ? (u + cap - 1) / cap - 1 : 0ull;
             es_key = (((unsigned long long)t + k * d_min) << 9) | (unsigned)c;
-            atomicMin(&s_horizon, es_key);
         }
-        if (!finished) atomicMin(&s_front, key);
+        // minima per warp first: one shared-memory update per warp instead of one per client
+        unsigned long long wh = es_key, wf = finished ? ~0ull : key;
+#pragma unroll
+        for (int d = 16; d > 0; d >>= 1) {
+            const unsigned long long oh = __shfl_xor_sync(FULL, wh, d), of = __shfl_xor_sync(FULL, wf, d);
+            wh = oh < wh ? oh : wh;
+            wf = of < wf ? of : wf;
+        }
+        if ((c & 31) == 0) {
+            if (wh != ~0ull) atomicMin(&s_horizon, wh);
+            if (wf != ~0ull) atomicMin(&s_front, wf);
+        }
         if (__syncthreads_and(finished)) break;
         const unsigned long long H = max(s_horizon, s_first);
         const unsigned long long front = s_front;
@@ -668,7 +681,12 @@ k_simulate_steal(const uint2* __restrict__ q_po, const uint32_t* __restrict__ q_
         const int ahead = __syncthreads_or(run);           // also orders the reads of the shared keys
         if (!ahead) run = !finished && key == front;       // the front of the global order: may steal
         if (c == 0) { s_horizon = ~0ull; s_front = ~0ull; } // for the next step (after the barrier above)
-        if (run) advance(false);
+        if (run) {
+            if (ahead) {
+                do advance(false);
+                while (!finished && (((unsigned long long)t << 9) | (unsigned)c) < H);
+            } else advance(false);
+        }
     }
     if (is_client) {
         if (tr && n_pre + cnt > tr_lim) status |= HOS_ST_TRACE;
