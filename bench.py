@@ -527,7 +527,7 @@ def run_reference(args):
     if rank != 0:
         return
     w = workload(args.workload)
-    n_s = max(1, sample_size(w) // 2)
+    n_s = max(1, sample_size(w) // 4)        # per step; the default 50 steps then take about two minutes at c4
     for _ in range(args.warmup):
         oracle_sample(w, 1)
     t0 = time.perf_counter()
