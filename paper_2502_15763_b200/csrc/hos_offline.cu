@@ -1,6 +1,7 @@
 // Offline request scheduling kernels (Eq. 26-30 of arXiv 2502.15763):
 //   k_estimate_sort  T_i and the per-instance order (T descending, index ascending)
 //   k_lpt            longest-first list scheduling, one warp per instance
+//   k_ls_lists       the clients' member lists for the local search
 //   k_local_search   rounds of best move / pairwise swap off the critical client
 //   k_lower_bound    Eq. 31-32 and the packing relaxations
 #include "hos_common.cuh"

@@ -1,6 +1,8 @@
 // Online scheduling kernels (Section "Online requests and iteration scheduling"):
 //   k_queue_build    per-client queues in the order of Algorithm 1
-//   k_simulate       iteration-level simulation, one warp per (instance, multiplier, client)
+//   k_simulate       iteration-level simulation, one thread per (instance, multiplier, client)
+//   k_simulate_steal the same with Algorithm 1's request stealing, one CTA per simulation
+//   k_trace_fill     the iteration trace rebuilt from the simulator's event log
 //   k_finalize       per-simulation makespan, utilisation, generation speed
 //   k_trace_offsets  exclusive scan of the per-client iteration counts
 #include "hos_common.cuh"
@@ -105,7 +107,7 @@ k_queue_build(const uint32_t* __restrict__ p, const uint32_t* __restrict__ o,
 // ---------------------------------------------------------------------------------------
 // Iteration-level simulator.  One THREAD per (instance, multiplier, client): the per-client
 // recurrence (duration, clock, waited decode time, decision, hash) is scalar work, so every
-// lane of a warp runs a client of its own.  The running batch of a client is a binary
+// lane of a warp runs a client of its own.  The running batch of a client is a 4-ary
 // min-heap in shared memory, keyed by the decode-iteration count at which a request retires
 // (`fin`) with the request's p + o (`tot`) as payload, laid out [slot][lane] so that lanes
 // never collide on a bank whatever slots they touch.  The KV length of a request at count c
