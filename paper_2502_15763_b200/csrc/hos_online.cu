@@ -521,7 +521,79 @@ k_simulate_steal(const uint2* __restrict__ q_po, const uint32_t* __restrict__ q_
     // One event iteration of my client -- claims (and, when `may_steal`, requests taken from other
     // queues), the decision, the prefill or decode -- and the plain decodes that follow it while
     // nothing can be claimed.  Sets `finished` when the client is done or hits a limit.
-    auto advance = [&](bool dry) {
+    // One decode iteration (one token for every running request), popping every request that
+    // retires with it; leaves the record in dur, r1, r2, r3.
+    uint32_t dur, r1, r2, r3;
+    auto decode_step = [&]() {
+        dur = ad + bd * B + (q_shift >= 0 ? (S >> q_shift) : (S / qd));
+        r1 = B; r2 = S; r3 = 0;
+        busy += (long long)dur * B;
+        S += B;
+        if (cnt + 1 == next_fin) {
+            const uint32_t c1 = cnt + 1;
+            uint32_t n = B;
+            do {
+                const uint32_t gone = E::tot(heap_ld(0));
+                S -= gone;
+                reserved -= gone;
+                ++r3;
+                --n;
+                const entry_t x = heap_ld((int)n);
+                const entry_t xr = E::rel(x, c1);
+                uint32_t i = 0;
+                while (true) {
+                    const uint32_t ch = 4 * i + 1;
+                    if (ch >= n) break;
+                    entry_t y0 = heap_ld((int)ch), ym = y0;
+                    entry_t m = E::rel(y0, c1);
+                    uint32_t at = ch;
+#pragma unroll
+                    for (uint32_t k = 1; k < 4; ++k) {
+                        if (ch + k < n) {
+                            const entry_t y = heap_ld((int)(ch + k));
+                            const entry_t r = E::rel(y, c1);
+                            if (r < m) { m = r; ym = y; at = ch + k; }
+                        }
+                    }
+                    if (xr <= m) break;
+                    heap_st((int)i, ym);
+                    i = at;
+                }
+                if (n > 0) heap_st((int)i, x);
+            } while (n > 0 && E::fin(heap_ld(0), c1) == c1);
+            B = n;
+            next_fin = n > 0 ? E::fin(heap_ld(0), c1) : EMPTY;
+        }
+    };
+    // Clock, hash, trace and waited decode time of the iteration in dur, r1, r2, r3; false when the
+    // clock limit is reached.
+    auto finish_event = [&]() {
+        emit(dur, r1, r2, r3);
+        if (r1 >> 31) { Cd = 0; ++n_pre; }
+        else { ++cnt; Cd = min(Cd + dur, 0x7FFFFFFFu); }
+        if (t >= (1ll << 39)) { status |= HOS_ST_LIMIT; finished = true; return false; }
+        return true;
+    };
+    // `until`: while the client runs side by side with the others (or alone in the dry run), an
+    // advance may start with the retiring decode that ends a quiet run and go on to the next event,
+    // as long as that one still starts before `until`; 0 when the client runs in its turn of the
+    // global order, where every event has to wait for its turn.
+    auto advance = [&](bool dry, unsigned long long until) {
+        if (until != 0ull && B > 0 && cnt + 1 == next_fin && n_pre + cnt != max_iters) {
+            // nothing can be claimed now (no free slot, or the own queue is used up and nothing is
+            // left anywhere), so the candidates stay as they are and the rule decides on them
+            const int up0 = dry ? u_dry : s_ustart[c];
+            const bool no_claim = B + nA >= (uint32_t)cap || (up0 >= qend && (dry || s_total == 0));
+            const unsigned long long Cp16f = (unsigned long long)prefill_us(cm, sumP) << 16;
+            if (no_claim && (nA == 0 || (unsigned long long)lam * Cd <= Cp16f)) {
+                decode_step();
+                if (!finish_event()) return;
+                // the next event must still be mine to take: before the horizon, and (dry run) before
+                // the iteration in which the own queue could be used up
+                if ((((unsigned long long)t << 9) | (unsigned)c) >= until) return;
+                if (dry && (uint32_t)(qend - u_dry) <= (uint32_t)cap - B - nA) return;
+            }
+        }
         int up = dry ? u_dry : s_ustart[c];
         while (up < qend && B + nA < (uint32_t)cap) {
             if (!claim(c, up, dry)) break;
@@ -542,7 +614,6 @@ k_simulate_steal(const uint2* __restrict__ q_po, const uint32_t* __restrict__ q_
 
         const uint32_t Cp = prefill_us(cm, sumP);
         const unsigned long long Cp16 = (unsigned long long)Cp << 16;
-        uint32_t dur, r1, r2, r3;
         if (nA > 0 && (B == 0 || (unsigned long long)lam * Cd > Cp16)) {
             for (uint32_t j = 0; j < nA; ++j) {
                 const entry_t x = E::rebase(heap_ld(cap - (int)nA + (int)j), cnt);
@@ -563,50 +634,9 @@ k_simulate_steal(const uint2* __restrict__ q_po, const uint32_t* __restrict__ q_
             nA = 0; sumP = 0; sumTot = 0;
             next_fin = E::fin(heap_ld(0), cnt);
         } else {
-            dur = ad + bd * B + (q_shift >= 0 ? (S >> q_shift) : (S / qd));
-            r1 = B; r2 = S; r3 = 0;
-            busy += (long long)dur * B;
-            S += B;
-            if (cnt + 1 == next_fin) {
-                const uint32_t c1 = cnt + 1;
-                uint32_t n = B;
-                do {
-                    const uint32_t gone = E::tot(heap_ld(0));
-                    S -= gone;
-                    reserved -= gone;
-                    ++r3;
-                    --n;
-                    const entry_t x = heap_ld((int)n);
-                    const entry_t xr = E::rel(x, c1);
-                    uint32_t i = 0;
-                    while (true) {
-                        const uint32_t ch = 4 * i + 1;
-                        if (ch >= n) break;
-                        entry_t y0 = heap_ld((int)ch), ym = y0;
-                        entry_t m = E::rel(y0, c1);
-                        uint32_t at = ch;
-#pragma unroll
-                        for (uint32_t k = 1; k < 4; ++k) {
-                            if (ch + k < n) {
-                                const entry_t y = heap_ld((int)(ch + k));
-                                const entry_t r = E::rel(y, c1);
-                                if (r < m) { m = r; ym = y; at = ch + k; }
-                            }
-                        }
-                        if (xr <= m) break;
-                        heap_st((int)i, ym);
-                        i = at;
-                    }
-                    if (n > 0) heap_st((int)i, x);
-                } while (n > 0 && E::fin(heap_ld(0), c1) == c1);
-                B = n;
-                next_fin = n > 0 ? E::fin(heap_ld(0), c1) : EMPTY;
-            }
+            decode_step();
         }
-        emit(dur, r1, r2, r3);
-        if (r1 >> 31) { Cd = 0; ++n_pre; }
-        else { ++cnt; Cd = min(Cd + dur, 0x7FFFFFFFu); }
-        if (t >= (1ll << 39)) { status |= HOS_ST_LIMIT; finished = true; return; }
+        if (!finish_event()) return;
         // plain decodes may follow at once while nothing can be claimed: they touch no queue, so
         // their order against other clients' claims does not matter.  Nothing can be claimed when no
         // slot is free, or when the own queue is used up and no queue has anything left (s_total
@@ -636,7 +666,7 @@ k_simulate_steal(const uint2* __restrict__ q_po, const uint32_t* __restrict__ q_
     {
         const uint32_t keep_lim = tr_lim;
         tr_lim = 0;                                         // no trace from the dry run
-        while (!finished && (uint32_t)(qend - u_dry) > (uint32_t)cap - B - nA) advance(true);
+        while (!finished && (uint32_t)(qend - u_dry) > (uint32_t)cap - B - nA) advance(true, ~0ull);
         if (is_client) atomicMin(&s_first, ((unsigned long long)t << 9) | (unsigned)c);
         tr_lim = keep_lim;
         t = 0; busy = 0; Cd = 0; cnt = 0; B = 0; S = 0; reserved = 0; n_pre = 0;
@@ -685,9 +715,9 @@ k_simulate_steal(const uint2* __restrict__ q_po, const uint32_t* __restrict__ q_
         if (c == 0) { s_horizon = ~0ull; s_front = ~0ull; } // for the next step (after the barrier above)
         if (run) {
             if (ahead) {
-                do advance(false);
+                do advance(false, H);
                 while (!finished && (((unsigned long long)t << 9) | (unsigned)c) < H);
-            } else advance(false);
+            } else advance(false, 0ull);
         }
     }
     if (is_client) {
