@@ -146,20 +146,26 @@ class Pipeline:
         self.trace = None
         self.out = None
         self.n_iters = 0
-        self.copy_stream = None
-        self.chunks = None
-        self.pk_out = None
+        self.up = None
+        self.down = None
+        self.sets = None
 
-    def args(self):
+    def tables(self):
+        return dict(p=self.p, o=self.o, est=self.est, lam=self.lam)
+
+    def args(self, t=None):
         w = self.w
-        return (self.p, self.o, w.n_clients, w.batch_cap, w.kv_budget, w.cost_model)
+        t = t or self.tables()
+        return (t["p"], t["o"], w.n_clients, w.batch_cap, w.kv_budget, w.cost_model)
 
-    def step(self):
+    def step(self, t=None):
         hos, w = self.hos, self.w
+        t = t or self.tables()
         sweep = len(w.lambdas_q16) > 1
         # a multiplier sweep runs its local-search rounds per (instance, multiplier) copy, below
-        pk = hos.hos_offline_pack(*self.args(), 0 if sweep else w.ls_rounds, ws=self.ws_off, want_lb=True, **self.kw)
-        return self.online(pk)
+        pk = hos.hos_offline_pack(*self.args(t), 0 if sweep else w.ls_rounds, ws=self.ws_off, want_lb=True,
+                                  o_est=t["est"], kv_reserve=w.kv_reserve)
+        return self.online(pk, t)
 
     def prepare(self):
         """Workspaces (allocated once; the library itself allocates nothing)."""
@@ -172,88 +178,83 @@ class Pipeline:
         self.ws_off = self.torch.empty(n_off, dtype=self.torch.uint8, device=self.dev)
         self.ws_on = self.torch.empty(n_on, dtype=self.torch.uint8, device=self.dev)
 
-    def online(self, pk):
+    def online(self, pk, t=None):
         """Lower bound, simulation with event log, trace offsets, trace (and the sweep's local search)."""
         hos, w = self.hos, self.w
+        t = t or self.tables()
+        kw = dict(o_est=t["est"], kv_reserve=w.kv_reserve)
         lb = dict(lb=pk["lb"])                      # Eq. 31-32 bounds, computed inside hos_offline_pack
-        s1 = hos.hos_online_simulate(*self.args(), pk["assign"], self.lam, hos.HOS_QUEUE_SORTED,
-                                     keep_events=True, ws=self.ws_on, **self.kw)
+        s1 = hos.hos_online_simulate(*self.args(t), pk["assign"], t["lam"], hos.HOS_QUEUE_SORTED,
+                                     keep_events=True, ws=self.ws_on, **kw)
         off = hos.hos_trace_offsets(s1["cres"])
         if self.trace is None:                      # first (warm-up) step sizes the trace buffer
             self.n_iters = int(off[-1].item())
             self.trace = self.torch.empty((max(self.n_iters, 1), 16), dtype=self.torch.uint8, device=self.dev)
-        hos.hos_trace_fill(*self.args(), len(w.lambdas_q16), s1, self.trace, off, **self.kw)
+        hos.hos_trace_fill(*self.args(t), len(w.lambdas_q16), s1, self.trace, off, **kw)
         self.out = dict(pk=pk, lb=lb, sim=s1, off=off)
         if len(w.lambdas_q16) > 1 and w.ls_rounds > 0:
             copies = pk["assign"][:, None, :].expand(-1, len(w.lambdas_q16), -1).contiguous()
-            self.out["ls"] = hos.hos_local_search(*self.args(), copies, w.ls_rounds, ws=self.ws_off, **self.kw)
+            self.out["ls"] = hos.hos_local_search(*self.args(t), copies, w.ls_rounds, ws=self.ws_off, **kw)
         return self.out
 
-    def e2e_step(self, host_out):
-        """The same step from pinned host tables to pinned host results.
+    @staticmethod
+    def results(r):
+        """What a step hands back to the host: assignment, loads, estimate, status, bounds, client and
+        simulation results (the iteration trace stays on the device)."""
+        pk, sim = r["pk"], r["sim"]
+        return (pk["assign"], pk["load"], pk["makespan_est"], pk["status"], r["lb"]["lb"],
+                sim["cres"], sim["sres"], sim["status"])
 
-        The instances are independent, so the offline part runs on a first chunk (two full waves of
-        one-CTA-per-instance kernels) while the rest of the tables are still on their way up,
-        and the offline results go down while the simulation runs; everything is inside the step."""
-        torch, hos, w = self.torch, self.hos, self.w
-        sweep = len(w.lambdas_q16) > 1
+    def e2e_run(self, steps, host_out, flush):
+        """`steps` steps from pinned host tables to pinned host results, as a stream of batches.
+
+        Every step uploads its own tables and downloads its own results.  There are two sets of device
+        tables: while step k computes, the tables of step k+1 go up and the results of step k-1 go down
+        (separate streams, both copy directions at once).  Returns the device time from the start of
+        the first upload to the end of the last download (ms) and the bytes per step each way."""
+        torch = self.torch
         main = torch.cuda.current_stream()
-        if self.copy_stream is None:
-            self.copy_stream = torch.cuda.Stream()
-            sm = torch.cuda.get_device_properties(self.dev).multi_processor_count
-            # two chunks: a first one of two waves so that little of the upload is exposed, then the
-            # rest (every offline call pays the packing chain's latency once, so few chunks)
-            first = min(w.n_inst, 2 * sm)
-            self.chunks = [(0, first)] + ([(first, w.n_inst - first)] if w.n_inst > first else [])
-            self.pk_out = dict(
-                assign=torch.empty((w.n_inst, w.n_req), dtype=torch.int32, device=self.dev),
-                load=torch.empty((w.n_inst, w.n_clients), dtype=torch.int64, device=self.dev),
-                makespan_est=torch.empty((w.n_inst,), dtype=torch.int64, device=self.dev),
-                rounds_applied=torch.empty((w.n_inst,), dtype=torch.int32, device=self.dev),
-                status=torch.empty((w.n_inst,), dtype=torch.int32, device=self.dev),
-                lb=torch.empty((w.n_inst, hos.LB_DTYPE.itemsize), dtype=torch.uint8, device=self.dev))
-        cs = self.copy_stream
-        cs.wait_stream(main)
-        arrived = []
-        with torch.cuda.stream(cs):
-            self.lam.copy_(self.lam_host, non_blocking=True)
-            for f, n in self.chunks:
-                self.p[f:f + n].copy_(self.p_host[f:f + n], non_blocking=True)
-                self.o[f:f + n].copy_(self.o_host[f:f + n], non_blocking=True)
-                if self.est is not None:
-                    self.est[f:f + n].copy_(self.est_host[f:f + n], non_blocking=True)
-                ev = torch.cuda.Event()
-                ev.record(cs)
-                arrived.append(ev)
-        pk = self.pk_out
-        for (f, n), ev in zip(self.chunks, arrived):
-            main.wait_event(ev)
-            hos.hos_offline_pack(self.p[f:f + n], self.o[f:f + n], w.n_clients, w.batch_cap, w.kv_budget,
-                                 w.cost_model, 0 if sweep else w.ls_rounds, ws=self.ws_off,
-                                 out={k: v[f:f + n] for k, v in pk.items()},
-                                 o_est=None if self.est is None else self.est[f:f + n], kv_reserve=w.kv_reserve)
-        packed = torch.cuda.Event()
-        packed.record(main)
-        early = (pk["assign"], pk["load"], pk["makespan_est"], pk["status"])
-        r = None
-        if not host_out:                            # first call: run once to learn the result shapes
-            r = self.online(pk)
-            late = (r["lb"]["lb"], r["sim"]["cres"], r["sim"]["sres"], r["sim"]["status"])
-            host_out.extend(torch.empty(t.shape, dtype=t.dtype).pin_memory() for t in early + late)
-        with torch.cuda.stream(cs):                 # offline results go down while the simulation runs
-            cs.wait_event(packed)
-            for h, d in zip(host_out[:4], early):
-                h.copy_(d, non_blocking=True)
-        if r is None:
-            r = self.online(pk)
-        late = (r["lb"]["lb"], r["sim"]["cres"], r["sim"]["sres"], r["sim"]["status"])
-        for h, d in zip(host_out[4:], late):
-            h.copy_(d, non_blocking=True)
-        main.wait_stream(cs)
-        h2d = sum(t.numel() * t.element_size() for t in (self.p_host, self.o_host, self.lam_host, self.est_host)
-                  if t is not None)
-        d2h = sum(t.numel() * t.element_size() for t in early + late)
-        return h2d, d2h
+        if self.up is None:
+            self.up, self.down = torch.cuda.Stream(), torch.cuda.Stream()
+            spare = {k: (None if v is None else torch.empty_like(v)) for k, v in self.tables().items()}
+            self.sets = [self.tables(), spare]
+        host = dict(p=self.p_host, o=self.o_host, est=self.est_host, lam=self.lam_host)
+        read = [None, None]                         # the step that last read a set of tables has finished
+        start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        start.record(main)
+        self.up.wait_stream(main)
+        self.down.wait_stream(main)
+        for k in range(steps):
+            t = self.sets[k & 1]
+            with torch.cuda.stream(self.up):
+                if read[k & 1] is not None:
+                    self.up.wait_event(read[k & 1])
+                for name, h in host.items():
+                    if h is not None:
+                        t[name].copy_(h, non_blocking=True)
+                arrived = torch.cuda.Event()
+                arrived.record(self.up)
+            main.wait_event(arrived)
+            if flush is not None:
+                flush.fill_(1)
+            res = self.results(self.step(t))
+            done = torch.cuda.Event()
+            done.record(main)
+            read[k & 1] = done
+            if not host_out:                        # first call: learn the result shapes
+                host_out.extend(torch.empty(d.shape, dtype=d.dtype).pin_memory() for d in res)
+            with torch.cuda.stream(self.down):
+                self.down.wait_event(done)
+                for h, d in zip(host_out, res):
+                    h.copy_(d, non_blocking=True)
+                    d.record_stream(self.down)      # the allocator must not hand it out again before the copy ends
+        main.wait_stream(self.down)
+        main.wait_stream(self.up)
+        end.record(main)
+        torch.cuda.synchronize()
+        h2d = sum(h.numel() * h.element_size() for h in host.values() if h is not None)
+        d2h = sum(h.numel() * h.element_size() for h in host_out)
+        return start.elapsed_time(end), h2d, d2h
 
 
 def timed_steps(torch, fn, steps, flush):
@@ -416,10 +417,13 @@ def run_ours(args):
     host_out = []
     h2d, d2h, ms_e2e = 0, 0, 0.0
     if not args.skip_e2e:
-        h2d, d2h = pipe.e2e_step(host_out)
+        pipe.e2e_run(max(args.warmup, 3), host_out, flush)
         barrier()
-        ms_e2e = timed_steps(torch, lambda: pipe.e2e_step(host_out), args.steps, flush)
+        ms_e2e, h2d, d2h = pipe.e2e_run(args.steps, host_out, flush)
         barrier()
+        for h, d in zip(host_out, pipe.results(pipe.step())):
+            if not torch.equal(h, d.cpu()):
+                raise SystemExit("bench: the end-to-end results differ from those of the device-resident step")
     e_t = torch.tensor([ms_e2e], dtype=torch.float64, device=dev)
     if world > 1:
         dist.all_reduce(e_t, op=dist.ReduceOp.MAX)
@@ -501,9 +505,11 @@ def run_ours(args):
             "clocks": clocks,
             "e2e": {"value": None if args.skip_e2e else total_inst * args.steps / (ms_e2e * 1e-3), "unit": UNIT,
                     "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-                    "note": "results copied back: assignment, loads, bounds, client and simulation results; "
-                            "the iteration trace stays on the device; uploads and the offline part are pipelined by "
-                            "chunks of instances, offline results go down while the simulation runs"},
+                    "note": "every step uploads its tables from pinned host memory and downloads its results "
+                            "(assignment, loads, bounds, client and simulation results; the iteration trace stays "
+                            "on the device); two sets of device tables, so step k+1's upload and step k-1's "
+                            "download run beside step k's kernels; timed from the first upload to the last "
+                            "download" + ("" if flush is None else ", L2 flushes included")},
             "gpu_launches": int(round(launches * args.steps)),
             "roofline": roofline,
             "kernels": rows,

@@ -115,6 +115,8 @@ k_queue_build(const uint32_t* __restrict__ p, const uint32_t* __restrict__ o,
 // sum KV is carried along: S += B - sum of retired tot.
 // ---------------------------------------------------------------------------------------
 constexpr uint32_t EMPTY = 0xFFFFFFFFu;
+constexpr int TF_RING = 128;                // log entries in a warp's ring in k_trace_fill (a power of two)
+constexpr int TF_AHEAD = 64;                // entries that the ring is filled ahead of their use, at least
 constexpr int SIM_QUIET_MAX = 16;         // plain decode iterations per pass of the simulator's loop
 constexpr unsigned long long HASH_INIT = 0xCBF29CE484222325ull;
 constexpr uint32_t HASH_C1 = 0x9E3779B1u, HASH_C2 = 0x85EBCA77u, HASH_C3 = 0xC2B2AE3Du, HASH_M = 0x27D4EB2Fu;
@@ -758,18 +760,40 @@ k_trace_fill(const int32_t* __restrict__ q_off, int n_lambda, int n_clients, int
     if (lane == 0 && (long long)n_total > capr) atomicOr(&status_out[unit], HOS_ST_TRACE);
     const uint32_t ad = cm.decode_fixed_us, bd = cm.decode_per_seq_us, qd = cm.decode_kv_div;
 
+    // The log entries pass through a ring in shared memory, filled by asynchronous copies that
+    // run TF_AHEAD entries and more ahead of their use: a pass then waits for no load from the
+    // log.  The ring holds the entries [k_next - 1, filled); one group of 32 is in flight at most
+    // when a pass starts.
+    __shared__ uint4 s_ring[4][TF_RING];
+    uint4* ring = s_ring[warp_id()];
+    uint32_t filled = 0;                       // log entries before `filled` are in the ring or on their way
+    auto fill = [&]() {
+        const uint32_t kf = filled + lane;
+        uint4* dst = &ring[kf & (TF_RING - 1)];
+        if (kf < n_ev) {
+            const unsigned sa = (unsigned)__cvta_generic_to_shared(dst);
+            asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" :: "r"(sa), "l"(ev + kf) : "memory");
+        } else {
+            *dst = make_uint4(0xFFFFFFFFu, 0u, 0u, 0u);
+        }
+        asm volatile("cp.async.commit_group;" ::: "memory");
+        filled += 32;
+    };
+    for (int g = 0; g < TF_AHEAD / 32 + 1; ++g) fill();
+
     uint32_t k_next = 0;                       // log entries before k_next have it < base
     for (uint32_t base = 0; base < lim; base += 32) {
         const uint32_t it = base + lane;
+        asm volatile("cp.async.wait_group 1;" ::: "memory");
+        __syncwarp();
         // iteration numbers of the next 32 log entries
-        const uint32_t kw = k_next + lane;
-        const uint32_t itw = kw < n_ev ? ev[kw].x : 0xFFFFFFFFu;
+        const uint32_t itw = ring[(k_next + lane) & (TF_RING - 1)].x;       // 0xFFFFFFFF past the log's end
         const uint32_t dw = itw - base;                                  // >= 0 by construction
         const uint32_t mask = __reduce_or_sync(FULL, dw < 32u ? (1u << dw) : 0u);
         const uint32_t upto = mask & (0xFFFFFFFFu >> (31 - lane));       // logged iterations <= it
         const uint32_t k = k_next + __popc(upto) - 1u;                   // iteration 0 is always logged
         if (it < lim) {
-            const uint4 st = ev[k];                    // {iteration, tokens, sum KV after it, packed}
+            const uint4 st = ring[k & (TF_RING - 1)];  // {iteration, tokens, sum KV after it, packed}
             const bool pre = st.w >> 31;
             const uint32_t lo8 = (st.w & 0xFFu) + 1u, hi8 = ((st.w >> 8) & 0xFFu) + 1u;
             uint4 rec;
@@ -784,7 +808,11 @@ k_trace_fill(const int32_t* __restrict__ q_off, int n_lambda, int n_clients, int
             tr[it] = rec;
         }
         k_next += __popc(mask);
+        __syncwarp();                           // every lane has read its entries before slots are refilled
+        if (filled - k_next < (uint32_t)TF_AHEAD + 32u) fill();
+        else asm volatile("cp.async.commit_group;" ::: "memory");        // keeps "all but the newest group" exact
     }
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
 }
 
 
@@ -822,43 +850,62 @@ k_finalize(int n_sims, int n_lambda, int n_clients, int cap,
     }
 }
 
-// Exclusive scan of the iteration counts; one CTA walks the array in tiles of 1024.
+// Exclusive scan of the iteration counts.  Every CTA owns a slice of whole tiles of 1,024 units; it
+// first adds up all counts before its slice (no CTA waits for another and no scratch memory is
+// needed; the counts are a few MB in L2), then scans its slice tile by tile.
 __global__ void __launch_bounds__(1024)
-k_trace_offsets(const hos_client_result* __restrict__ cres, long long n_units,
+k_trace_offsets(const hos_client_result* __restrict__ cres, long long n_units, long long slice,
                 long long* __restrict__ trace_off) {
-    __shared__ unsigned long long wsum[32];
-    __shared__ unsigned long long carry_s;
-    if (threadIdx.x == 0) { carry_s = 0; trace_off[0] = 0; }
+    __shared__ unsigned long long wsum[2][32];
+    __shared__ unsigned long long s_before;
+    auto count = [&](long long x) {
+        return x < n_units ? (unsigned long long)cres[x].n_prefill_iters + cres[x].n_decode_iters : 0ull;
+    };
+    const long long x0 = slice * blockIdx.x, x1 = min(n_units, x0 + slice);
+    if (blockIdx.x == 0 && threadIdx.x == 0) trace_off[0] = 0;
+    if (x0 >= n_units) return;                                            // the whole CTA: a slice past the end
+    if (threadIdx.x == 0) s_before = 0;
     __syncthreads();
-    for (long long base = 0; base < n_units; base += 1024) {
+    {
+        unsigned long long part = 0;
+        long long x = threadIdx.x;
+        for (; x + 7 * 1024 < x0; x += 8 * 1024) {
+            unsigned long long v[8];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) v[j] = count(x + j * 1024);
+#pragma unroll
+            for (int j = 0; j < 8; ++j) part += v[j];
+        }
+        for (; x < x0; x += 1024) part += count(x);
+        part = warp_sum_u64(part);
+        if (lane_id() == 0 && part != 0) atomicAdd(&s_before, part);
+    }
+    __syncthreads();
+    unsigned long long carry = s_before;                                  // units before this tile
+    int buf = 0;
+    for (long long base = x0; base < x1; base += 1024, buf ^= 1) {
         const long long x = base + threadIdx.x;
-        const unsigned long long v =
-            x < n_units ? (unsigned long long)cres[x].n_prefill_iters + cres[x].n_decode_iters : 0ull;
-        unsigned long long inc = v;
+        const unsigned long long mine = count(x);
+        unsigned long long inc = mine;
 #pragma unroll
         for (int d = 1; d < 32; d <<= 1) {
             const unsigned long long y = __shfl_up_sync(FULL, inc, d);
             if (lane_id() >= d) inc += y;
         }
-        if (lane_id() == 31) wsum[warp_id()] = inc;
+        if (lane_id() == 31) wsum[buf][warp_id()] = inc;
         __syncthreads();
-        if (warp_id() == 0) {
-            const unsigned long long w = wsum[lane_id()];
-            unsigned long long winc = w;
+        // every warp scans the 32 warp sums itself: one barrier per tile (the two buffers keep a
+        // fast warp's next tile away from the sums that a slow warp still reads)
+        const unsigned long long w = wsum[buf][lane_id()];
+        unsigned long long winc = w;
 #pragma unroll
-            for (int d = 1; d < 32; d <<= 1) {
-                const unsigned long long y = __shfl_up_sync(FULL, winc, d);
-                if (lane_id() >= d) winc += y;
-            }
-            wsum[lane_id()] = winc - w;
+        for (int d = 1; d < 32; d <<= 1) {
+            const unsigned long long y = __shfl_up_sync(FULL, winc, d);
+            if (lane_id() >= d) winc += y;
         }
-        __syncthreads();
-        const unsigned long long carry = carry_s;
-        const unsigned long long mine = carry + wsum[warp_id()] + inc;       // inclusive
-        if (x < n_units) trace_off[x + 1] = (long long)mine;
-        __syncthreads();
-        if (threadIdx.x == 1023) carry_s = mine;
-        __syncthreads();
+        const unsigned long long before = __shfl_sync(FULL, winc - w, warp_id());
+        if (x < x1) trace_off[x + 1] = (long long)(carry + before + inc);
+        carry += __shfl_sync(FULL, winc, 31);
     }
 }
 
@@ -1020,7 +1067,11 @@ cudaError_t launch_finalize(const hos_batch& b, int n_lambda, const unsigned lon
 cudaError_t launch_trace_offsets(const hos_client_result* cres, long long n_units, long long* trace_off,
                                  cudaStream_t st) {
     launch_hook("k_trace_offsets", 0, st);
-    k_trace_offsets<<<1, 1024, 0, st>>>(cres, n_units, trace_off);
+    // at most one CTA per SM of the largest part, each with whole tiles of 1,024 units
+    const long long tiles = (n_units + 1023) / 1024;
+    const long long ctas = tiles < 1 ? 1 : (tiles < 148 ? tiles : 148);
+    const long long slice = (tiles + ctas - 1) / ctas * 1024;
+    k_trace_offsets<<<(unsigned)ctas, 1024, 0, st>>>(cres, n_units, slice, trace_off);
     launch_hook("k_trace_offsets", 1, st);
     return cudaGetLastError();
 }
