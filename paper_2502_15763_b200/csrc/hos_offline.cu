@@ -75,6 +75,7 @@ k_estimate_sort(const uint32_t* __restrict__ p, const uint32_t* __restrict__ o,
 // within max_T of their minimum (each item lands on the current minimum), which bounds the
 // packed field between re-basings; instances that do not fit use 64-bit loads.
 // ---------------------------------------------------------------------------------------
+constexpr int LPT_AHEAD = 4;                // chunks of 32 items that k_lpt fetches ahead of their use
 template <int KPL>
 __global__ void __launch_bounds__(32)
 k_lpt(const uint32_t* __restrict__ T_sorted, const uint32_t* __restrict__ order,
@@ -83,6 +84,7 @@ k_lpt(const uint32_t* __restrict__ T_sorted, const uint32_t* __restrict__ order,
       long long* __restrict__ makespan_out, uint8_t* __restrict__ rank_client) {
     constexpr int JB = (KPL == 1) ? 5 : (KPL == 2) ? 6 : (KPL == 4) ? 7 : 8;
     __shared__ uint32_t s_perm[32];
+    __shared__ uint32_t s_tv[32 * LPT_AHEAD], s_rq[32 * LPT_AHEAD];
     const int inst = blockIdx.x;
     const int lane = threadIdx.x;
     const InstInfo inf = info[inst];
@@ -121,15 +123,35 @@ k_lpt(const uint32_t* __restrict__ T_sorted, const uint32_t* __restrict__ order,
         }
         unsigned long long rebased = 0;                 // sum of the bases subtracted so far
         bool half_sorted = false;                       // key[0] is all new, key[1] still ascending
-        uint32_t tv_next = (lane < n_req) ? Ts[lane] : 0u;
-        uint32_t rq_next = (lane < n_req) ? od[lane] : 0u;
-        for (int r0 = 0; r0 < n_req; r0 += 32) {
+        // The items arrive LPT_AHEAD chunks ahead of their use: four chunks wait in shared memory
+        // while the next four are on their way in registers (a chunk is a few hundred cycles of
+        // dependent work and few warps share an SM, so one chunk ahead would leave most of a
+        // memory round trip in the open).
+        uint32_t tv_next[LPT_AHEAD], rq_next[LPT_AHEAD];
+#pragma unroll
+        for (int j = 0; j < LPT_AHEAD; ++j) {
+            const int rn = 32 * j + lane;
+            tv_next[j] = (rn < n_req) ? Ts[rn] : 0u;
+            rq_next[j] = (rn < n_req) ? od[rn] : 0u;
+        }
+        for (int R0 = 0; R0 < n_req; R0 += 32 * LPT_AHEAD) {
+        __syncwarp();                                   // the chunks before are used up
+#pragma unroll
+        for (int j = 0; j < LPT_AHEAD; ++j) {
+            s_tv[32 * j + lane] = tv_next[j];
+            s_rq[32 * j + lane] = rq_next[j];
+        }
+        __syncwarp();
+#pragma unroll
+        for (int j = 0; j < LPT_AHEAD; ++j) {
+            const int rn = R0 + 32 * (LPT_AHEAD + j) + lane;
+            tv_next[j] = (rn < n_req) ? Ts[rn] : 0u;
+            rq_next[j] = (rn < n_req) ? od[rn] : 0u;
+        }
+        for (int r0 = R0; r0 < min(n_req, R0 + 32 * LPT_AHEAD); r0 += 32) {
             const int r = r0 + lane;
-            const uint32_t tsh = tv_next << JB;         // this chunk's items, already in key units
-            const uint32_t rq = rq_next;
-            const int rn = r + 32;                      // prefetch the next chunk behind the chain
-            tv_next = (rn < n_req) ? Ts[rn] : 0u;
-            rq_next = (rn < n_req) ? od[rn] : 0u;
+            const uint32_t tsh = s_tv[r - R0] << JB;    // this chunk's items, already in key units
+            const uint32_t rq = s_rq[r - R0];
             const int steps = min(32, n_req - r0);
             uint32_t mine = 0;
             int pos = 0;
@@ -143,10 +165,10 @@ k_lpt(const uint32_t* __restrict__ T_sorted, const uint32_t* __restrict__ order,
                     // the new half by rank: 32 independent compares instead of 15 dependent steps
                     // (keys are distinct: they carry their client)
                     uint32_t x = key[0];
-                    int rank = 0;
+                    int rk[4] = {0, 0, 0, 0};           // four short chains of additions instead of one long
 #pragma unroll
-                    for (int b = 0; b < 32; ++b) rank += __shfl_sync(FULL, x, b) < x ? 1 : 0;
-                    s_perm[rank] = x;
+                    for (int b = 0; b < 32; ++b) rk[b & 3] += __shfl_sync(FULL, x, b) < x ? 1 : 0;
+                    s_perm[(rk[0] + rk[1]) + (rk[2] + rk[3])] = x;
                     __syncwarp();
                     x = s_perm[lane];
                     __syncwarp();
@@ -191,6 +213,22 @@ k_lpt(const uint32_t* __restrict__ T_sorted, const uint32_t* __restrict__ order,
                 }
                 }
                 // lane a now holds the a-th smallest key in key[0]; item pos + a is its candidate
+                if (pos == 0 && steps == 32) {
+                    // a whole chunk at once when even the largest of the 32 keys is below every updated
+                    // key (then it is below the updated keys of the lanes before it, and so are the
+                    // smaller ones): one warp minimum instead of the prefix minimum
+                    const uint32_t s_a = key[0];
+                    const uint32_t u_a = s_a + tsh;
+                    const uint32_t u_min = __reduce_min_sync(FULL, u_a);
+                    const uint32_t s_top = __shfl_sync(FULL, s_a, 31);
+                    if (s_top != 0xFFFFFFFFu && s_top < u_min) {
+                        key[0] = u_a;
+                        mine = s_a & ((1u << JB) - 1u);
+                        pos = 32;
+                        half_sorted = true;
+                        continue;
+                    }
+                }
                 const int src = pos + lane;
                 const bool have = src < steps;
                 const uint32_t t = __shfl_sync(FULL, tsh, src & 31);
@@ -226,6 +264,7 @@ k_lpt(const uint32_t* __restrict__ T_sorted, const uint32_t* __restrict__ order,
 #pragma unroll
             for (int k = 0; k < KPL; ++k)
                 if (key[k] != 0xFFFFFFFFu) key[k] -= base;
+        }
         }
         long long mx = 0;
 #pragma unroll
