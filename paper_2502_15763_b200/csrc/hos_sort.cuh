@@ -142,12 +142,24 @@ __device__ inline IdxT* block_radix_sort_ids(const SortSmem<IdxT>& s, int n, int
                 dig[g] = valid[g] ? (((s.key[id[g]] ^ flip) >> shift) & dmask) : 0u;
                 m[g] = __ballot_sync(FULL, valid[g]);        // lanes of this row with my digit
             }
-            for (int b = 0; b < nb; ++b) {
+            if (nb == RADIX_BITS) {                          // the usual digit: no loop, constant shifts
 #pragma unroll
-                for (int g = 0; g < G; ++g) {
-                    const bool bit = (dig[g] >> b) & 1u;
-                    const unsigned bal = __ballot_sync(FULL, bit);
-                    m[g] &= bit ? bal : ~bal;
+                for (int b = 0; b < RADIX_BITS; ++b) {
+#pragma unroll
+                    for (int g = 0; g < G; ++g) {
+                        const bool bit = (dig[g] >> b) & 1u;
+                        const unsigned bal = __ballot_sync(FULL, bit);
+                        m[g] &= bit ? bal : ~bal;
+                    }
+                }
+            } else {
+                for (int b = 0; b < nb; ++b) {
+#pragma unroll
+                    for (int g = 0; g < G; ++g) {
+                        const bool bit = (dig[g] >> b) & 1u;
+                        const unsigned bal = __ballot_sync(FULL, bit);
+                        m[g] &= bit ? bal : ~bal;
+                    }
                 }
             }
 #pragma unroll
