@@ -410,9 +410,9 @@ k_simulate(const uint2* __restrict__ q_po, const int32_t* __restrict__ q_off,
 //
 // Only a stealing client touches other clients' queues, so iterations that provably start
 // before any steal can happen run side by side, one thread each; the client at the front of
-// the global order runs alone when it might steal (see the horizon H below).  Plain decode
-// iterations claim nothing and commute with everything, so they follow their event iteration
-// at once.
+// the global order takes its turn alone when it might steal (see the horizon H below).
+// Iterations that claim nothing commute with everything: plain decodes follow their event
+// iteration at once, and a client without a free slot goes on without waiting for its turn.
 // ---------------------------------------------------------------------------------------
 template <typename E>
 __global__ void __launch_bounds__(MAX_CLIENTS)
@@ -678,7 +678,8 @@ k_simulate_steal(const uint2* __restrict__ q_po, const uint32_t* __restrict__ q_
 
     // After s_first the conservative bound: no iteration lasts less than d_min and a client claims
     // at most `cap` requests per iteration, so a client with u unclaimed own requests cannot use
-    // them up -- and so cannot steal -- before es = clock + (ceil(u / cap) - 1) * d_min.  Nothing is
+    // them up -- and so cannot steal -- before es = clock + (ceil(u / cap) - 1) * d_min; with u at least
+    // its free slots it cannot steal in its next iteration either, so es >= clock + d_min.  Nothing is
     // stolen before H = max(s_first, min es over the unfinished clients), hence every iteration that
     // starts before H only touches its own client and all of them may run side by side: a client
     // goes on, iteration after iteration, until its clock reaches H (the bound is taken from the
@@ -693,7 +694,10 @@ k_simulate_steal(const uint2* __restrict__ q_po, const uint32_t* __restrict__ q_
         unsigned long long es_key = ~0ull;
         if (!finished && s_total > s_remain[c]) {          // somebody else still has queued requests
             const unsigned long long u = (unsigned long long)(qend - s_ustart[c]);
-            const unsigned long long k = u > (unsigned long long)cap ? (u + cap - 1) / cap - 1 : 0ull;
+            unsigned long long k = u > (unsigned long long)cap ? (u + cap - 1) / cap - 1 : 0ull;
+            // and not in its next iteration when its free slots do not outnumber its own requests
+            // (it claims those first and steals only with a slot to spare)
+            if (k == 0ull && u >= (unsigned long long)((uint32_t)cap - B - nA)) k = 1ull;
             es_key = (((unsigned long long)t + k * d_min) << 9) | (unsigned)c;
         }
         // minima per warp first: one shared-memory update per warp instead of one per client
@@ -720,6 +724,13 @@ k_simulate_steal(const uint2* __restrict__ q_po, const uint32_t* __restrict__ q_
                 do advance(false, H);
                 while (!finished && (((unsigned long long)t << 9) | (unsigned)c) < H);
             } else advance(false, 0ull);
+        } else if (!finished) {
+            // A client without a free slot claims nothing in its next iteration, whatever that is
+            // (a prefill of what it has claimed already, or a decode): the iteration touches no
+            // queue and nobody looks at the state it changes, so it needs no turn in the global
+            // order.  (What it reads of the queues on the way only decides whether plain decodes
+            // may follow at once; a stale value there only postpones them.)
+            while (!finished && B + nA == (uint32_t)cap) advance(false, 0ull);
         }
     }
     if (is_client) {
