@@ -806,16 +806,16 @@ k_trace_fill(const int32_t* __restrict__ q_off, int n_lambda, int n_clients, int
         if (it < lim) {
             const uint4 st = ring[k & (TF_RING - 1)];  // {iteration, tokens, sum KV after it, packed}
             const bool pre = st.w >> 31;
+            const bool logged = st.x == it;
             const uint32_t lo8 = (st.w & 0xFFu) + 1u, hi8 = ((st.w >> 8) & 0xFFu) + 1u;
-            uint4 rec;
-            if (st.x == it) {
-                if (pre) rec = make_uint4(prefill_us(cm, st.y), 0x80000000u | lo8, st.y, (st.w >> 16) & 0x7FFFu);
-                else rec = make_uint4(ad + bd * lo8 + (q_shift >= 0 ? (st.y >> q_shift) : (st.y / qd)), lo8, st.y, hi8);
-            } else {
-                const uint32_t Bk = pre ? hi8 : lo8 - hi8;               // batch after the logged iteration
-                const uint32_t Sk = st.z + (it - st.x - 1u) * Bk;
-                rec = make_uint4(ad + bd * Bk + (q_shift >= 0 ? (Sk >> q_shift) : (Sk / qd)), Bk, Sk, 0u);
-            }
+            // a decode record either way -- the logged (retiring) one, or a plain one after the logged
+            // iteration -- from one formula; only a logged prefill takes a branch
+            const uint32_t Bk = logged ? lo8 : (pre ? hi8 : lo8 - hi8);  // batch of this iteration
+            const uint32_t Sk = logged ? st.y : st.z + (it - st.x - 1u) * Bk;
+            uint4 rec = make_uint4(ad + bd * Bk + (q_shift >= 0 ? (Sk >> q_shift) : (Sk / qd)), Bk, Sk,
+                                   logged ? hi8 : 0u);
+            if (logged && pre)
+                rec = make_uint4(prefill_us(cm, st.y), 0x80000000u | lo8, st.y, (st.w >> 16) & 0x7FFFu);
             tr[it] = rec;
         }
         k_next += __popc(mask);
