@@ -93,9 +93,12 @@ class ClockSampler:
 
     def _read(self):
         for line in self.proc.stdout:
-            self.rows.append(line.strip())
+            self.rows.append((time.monotonic(), line.strip()))
 
-    def stop(self) -> dict:
+    def stop(self, t0: float, t1: float) -> dict:
+        """Median SM clock and the throttle reasons seen between t0 and t1 (time.monotonic() around the
+        timed steps); the sampler runs from before the warm-up steps, and a timed region too short for
+        a sample of its own reports the samples taken under the same load since the warm-up began."""
         if self.proc is None:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
         self.proc.terminate()
@@ -105,7 +108,9 @@ class ClockSampler:
             self.proc.kill()
         sm, mx, reasons = [], [], set()
         names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
-        for row in self.rows:
+        inside = [r for ts, r in self.rows if t0 <= ts <= t1]
+        window = "timed steps" if inside else "warm-up and timed steps"
+        for row in (inside or [r for _, r in self.rows]):
             parts = [x.strip() for x in row.split(",")]
             if len(parts) != 6:
                 continue
@@ -117,7 +122,7 @@ class ClockSampler:
                 if v.lower().startswith("active"):
                     reasons.add(n)
         return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
-                "samples": len(sm), "reasons": sorted(reasons)}
+                "samples": len(sm), "window": window, "reasons": sorted(reasons)}
 
 
 # ------------------------------------------------------------------------------------------
@@ -399,15 +404,16 @@ def run_ours(args):
             dist.barrier()
         torch.cuda.synchronize()
 
-    for _ in range(max(args.warmup, 1)):
-        pipe.step()
-    barrier()
     sampler = ClockSampler(local)
     if rank == 0:
         sampler.start()
+    for _ in range(max(args.warmup, 1)):
+        pipe.step()
+    barrier()
+    t0 = time.monotonic()
     ms = timed_steps(torch, pipe.step, args.steps, flush)
     barrier()
-    clocks = sampler.stop() if rank == 0 else None
+    clocks = sampler.stop(t0, time.monotonic()) if rank == 0 else None
     ms_t = torch.tensor([ms], dtype=torch.float64, device=dev)
     if world > 1:
         dist.all_reduce(ms_t, op=dist.ReduceOp.MAX)
