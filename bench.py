@@ -163,14 +163,16 @@ class Pipeline:
         t = t or self.tables()
         return (t["p"], t["o"], w.n_clients, w.batch_cap, w.kv_budget, w.cost_model)
 
-    def step(self, t=None):
+    def offline(self, t=None):
         hos, w = self.hos, self.w
         t = t or self.tables()
         sweep = len(w.lambdas_q16) > 1
-        # a multiplier sweep runs its local-search rounds per (instance, multiplier) copy, below
-        pk = hos.hos_offline_pack(*self.args(t), 0 if sweep else w.ls_rounds, ws=self.ws_off, want_lb=True,
-                                  o_est=t["est"], kv_reserve=w.kv_reserve)
-        return self.online(pk, t)
+        # a multiplier sweep runs its local-search rounds per (instance, multiplier) copy, in online()
+        return hos.hos_offline_pack(*self.args(t), 0 if sweep else w.ls_rounds, ws=self.ws_off, want_lb=True,
+                                    o_est=t["est"], kv_reserve=w.kv_reserve)
+
+    def step(self, t=None):
+        return self.online(self.offline(t), t)
 
     def prepare(self):
         """Workspaces (allocated once; the library itself allocates nothing)."""
@@ -214,8 +216,9 @@ class Pipeline:
         """`steps` steps from pinned host tables to pinned host results, as a stream of batches.
 
         Every step uploads its own tables and downloads its own results.  There are two sets of device
-        tables: while step k computes, the tables of step k+1 go up and the results of step k-1 go down
-        (separate streams, both copy directions at once).  Returns the device time from the start of
+        tables: while step k computes, the tables of step k+1 go up and results go down (separate
+        streams, both copy directions at once; the offline results of step k already while its online
+        part runs).  Returns the device time from the start of
         the first upload to the end of the last download (ms) and the bytes per step each way."""
         torch = self.torch
         main = torch.cuda.current_stream()
@@ -242,15 +245,22 @@ class Pipeline:
             main.wait_event(arrived)
             if flush is not None:
                 flush.fill_(1)
-            res = self.results(self.step(t))
+            pk = self.offline(t)
+            packed = torch.cuda.Event()
+            packed.record(main)
+            res = self.results(self.online(pk, t))
             done = torch.cuda.Event()
             done.record(main)
             read[k & 1] = done
             if not host_out:                        # first call: learn the result shapes
                 host_out.extend(torch.empty(d.shape, dtype=d.dtype).pin_memory() for d in res)
+            n_early = 5                             # the offline results go down while the online part runs
             with torch.cuda.stream(self.down):
-                self.down.wait_event(done)
-                for h, d in zip(host_out, res):
+                for i, (h, d) in enumerate(zip(host_out, res)):
+                    if i == 0:
+                        self.down.wait_event(packed)
+                    if i == n_early:
+                        self.down.wait_event(done)
                     h.copy_(d, non_blocking=True)
                     d.record_stream(self.down)      # the allocator must not hand it out again before the copy ends
         main.wait_stream(self.down)
