@@ -379,7 +379,8 @@ constexpr int NO_I = 0x7FFFFFFF;
 constexpr int LS_THREADS = 128;
 constexpr int LS_WARPS = LS_THREADS / 32;
 constexpr int LS_STAGE = 512;             // longest critical list that is copied to shared memory
-constexpr int LS_BATCH = 4;               // work items a thread has in flight
+constexpr int LS_BATCH = 3;               // work items a thread has in flight (3 x 128 threads take a
+                                          // list of up to 383 members in one go: c4's have about 312)
 
 // Exclusive scan of a[0 .. len) in place by the whole CTA of NT threads; `wsum` holds NT / 32 words.
 template <int NT>
