@@ -379,8 +379,8 @@ constexpr int NO_I = 0x7FFFFFFF;
 constexpr int LS_THREADS = 128;
 constexpr int LS_WARPS = LS_THREADS / 32;
 constexpr int LS_STAGE = 512;             // longest critical list that is copied to shared memory
-constexpr int LS_BATCH = 3;               // work items a thread has in flight (3 x 128 threads take a
-                                          // list of up to 383 members in one go: c4's have about 312)
+constexpr int LS_BATCH_MAX = 4;           // work items a thread has in flight: 2, 3 or 4, chosen per launch so
+                                          // that a list of the usual length just fits one batch of the CTA
 
 // Exclusive scan of a[0 .. len) in place by the whole CTA of NT threads; `wsum` holds NT / 32 words.
 template <int NT>
@@ -724,22 +724,22 @@ struct LsListing {
     int na, nitems;
 };
 
-// b[u] += members with T >= thr[u], for LS_BATCH searches side by side.  A = s_T + 1 holds the
+// b[u] += members with T >= thr[u], for NB searches side by side.  A = s_T + 1 holds the
 // members' T (descending), then zeros up to 2^STEPS entries, and s_T[0] is all ones.
-template <int STEPS>
-__device__ __forceinline__ void count_ge_batch(const uint32_t* s_T, const uint32_t (&thr)[LS_BATCH],
-                                               int (&b)[LS_BATCH], int top) {
+template <int STEPS, int NB>
+__device__ __forceinline__ void count_ge_batch(const uint32_t* s_T, const uint32_t (&thr)[NB],
+                                               int (&b)[NB], int top) {
     if (STEPS > 0) {
 #pragma unroll
         for (int st = STEPS - 1; st >= 0; --st) {
 #pragma unroll
-            for (int u = 0; u < LS_BATCH; ++u)
+            for (int u = 0; u < NB; ++u)
                 if (s_T[b[u] + (1 << st)] >= thr[u]) b[u] += 1 << st;
         }
     } else {
         for (int step = top; step > 0; step >>= 1) {
 #pragma unroll
-            for (int u = 0; u < LS_BATCH; ++u)
+            for (int u = 0; u < NB; ++u)
                 if (s_T[b[u] + step] >= thr[u]) b[u] += step;
         }
     }
@@ -750,7 +750,7 @@ __device__ __forceinline__ void count_ge_batch(const uint32_t* s_T, const uint32
 __device__ __forceinline__ void pair_arrive() { asm volatile("bar.arrive 1, 64;" ::: "memory"); }
 __device__ __forceinline__ void pair_wait() { asm volatile("bar.sync 1, 64;" ::: "memory"); }
 
-template <typename IdxT>
+template <typename IdxT, int LS_BATCH>
 __global__ void __launch_bounds__(LS_THREADS, 7)
 k_local_search(const uint32_t* __restrict__ T_sorted, const uint32_t* __restrict__ order,
                const InstInfo* __restrict__ info, int n_req, int n_pad, int n_clients,
@@ -1034,7 +1034,7 @@ k_local_search(const uint32_t* __restrict__ T_sorted, const uint32_t* __restrict
                     // the next batch's reads are in flight during this batch's searches
                     if (i0 + LS_BATCH * LS_THREADS <= len) fetch(cb, len, i0 + LS_BATCH * LS_THREADS);
                     else if (ci + 1 < na) fetch(L.cb[ci + 1], L.as[ci + 2] - L.as[ci + 1] - 1, 0);
-                    count_ge_batch<STEPS>(s_T, thr, b, top);
+                    count_ge_batch<STEPS, LS_BATCH>(s_T, thr, b, top);
 #pragma unroll
                     for (int u = 0; u < LS_BATCH; ++u) {
                         const int idx = i0 + u * LS_THREADS + (int)threadIdx.x;
@@ -1323,17 +1323,21 @@ cudaError_t launch_local_search(const hos_batch& b, const uint32_t* T_sorted, co
             T_sorted, order, info, b.n_req, n_pad, b.n_clients, n_copies, load_from_assign, assign, load, ws_T,
             static_cast<uint32_t*>(ws_I), ws_C, ws_off, ws_bad);
     launch_hook("k_ls_lists", 1, st);
+    // searches in flight per thread: a list of the usual length (and a little more: the packing
+    // balances times, not counts), plus the move, should fit one batch of LS_THREADS x nb items
+    const long long usual = ((long long)b.n_req / b.n_clients + 1) * 115 / 100;
+    const int nb = usual <= 2 * LS_THREADS ? 2 : (usual <= 3 * LS_THREADS ? 3 : LS_BATCH_MAX);
     launch_hook("k_local_search", 0, st);
-    if (b.n_req <= 65536)
-        k_local_search<uint16_t><<<grid, LS_THREADS, smem, st>>>(
-            T_sorted, order, info, b.n_req, n_pad, b.n_clients, n_copies, rounds, load_from_assign, assign,
-            load, makespan, rounds_applied, ls_log, status, ws_T, static_cast<uint16_t*>(ws_I), ws_C, ws_off,
-            ws_bad);
-    else
-        k_local_search<uint32_t><<<grid, LS_THREADS, smem, st>>>(
-            T_sorted, order, info, b.n_req, n_pad, b.n_clients, n_copies, rounds, load_from_assign, assign,
-            load, makespan, rounds_applied, ls_log, status, ws_T, static_cast<uint32_t*>(ws_I), ws_C, ws_off,
-            ws_bad);
+#define HOS_LS(IDX, NB)                                                                              \
+    k_local_search<IDX, NB><<<grid, LS_THREADS, smem, st>>>(                                         \
+        T_sorted, order, info, b.n_req, n_pad, b.n_clients, n_copies, rounds, load_from_assign, assign, \
+        load, makespan, rounds_applied, ls_log, status, ws_T, static_cast<IDX*>(ws_I), ws_C, ws_off, ws_bad)
+    if (narrow) {
+        if (nb == 2) HOS_LS(uint16_t, 2); else if (nb == 3) HOS_LS(uint16_t, 3); else HOS_LS(uint16_t, 4);
+    } else {
+        if (nb == 2) HOS_LS(uint32_t, 2); else if (nb == 3) HOS_LS(uint32_t, 3); else HOS_LS(uint32_t, 4);
+    }
+#undef HOS_LS
     launch_hook("k_local_search", 1, st);
     return cudaGetLastError();
 }
