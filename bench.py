@@ -46,9 +46,9 @@ BOUND = {"k_simulate": "alu", "k_simulate_steal": "alu", "k_lpt": "latency (depe
 INT_OPS_PER_ITERATION = 24
 # DRAM bytes per request and launch measured with ncu (dram__bytes_read.sum + dram__bytes_write.sum
 # over 296 instances of c4's shape, see profiles/); None for a kernel changed since its capture
-NCU_DRAM_BYTES_PER_REQ = {"k_estimate_sort": 8.62, "k_lower_bound": 8.03, "k_lpt": 12.67, "k_ls_lists": 18.10,
-                          "k_local_search": 6.07, "k_queue_build": 15.73, "k_simulate": 21.10}
-NCU_DRAM_BYTES_PER_ITERATION = {"k_trace_fill": 18.77}
+NCU_DRAM_BYTES_PER_REQ = {"k_estimate_sort": 8.68, "k_lower_bound": 8.05, "k_lpt": 12.69, "k_ls_lists": 18.09,
+                          "k_local_search": 6.07, "k_queue_build": 15.77, "k_simulate": 20.75}
+NCU_DRAM_BYTES_PER_ITERATION = {"k_trace_fill": 18.79}
 
 
 def describe(w: Workload) -> str:
