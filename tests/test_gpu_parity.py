@@ -124,10 +124,12 @@ def test_local_search_from_bad_assignments(hos):
                 assert np.array_equal(log[k, c][f], elog[f])
 
 
-@pytest.mark.parametrize("n,M,scale", [(1530, 3, 1), (1024, 2, 1), (900, 5, 1), (600, 4, 10000)])
+@pytest.mark.parametrize("n,M,scale", [(1530, 3, 1), (1024, 2, 1), (900, 5, 1), (600, 4, 10000),
+                                       (1000, 3, 1), (1200, 4, 1)])
 def test_local_search_short_list_and_general_forms(hos, n, M, scale):
     # member lists around the length up to which the critical client's list is evaluated from
-    # on-chip memory (511), and loads above 2^31 (scale), which take the 64-bit form
+    # on-chip memory (511), loads above 2^31 (scale), which take the 64-bit form, and list lengths
+    # for which a thread runs two, three and four searches side by side
     rng = np.random.default_rng(n + M)
     n_inst = 2
     p = rng.integers(1, 3000, size=(n_inst, n)).astype(np.uint32)
