@@ -5,7 +5,7 @@
  * C ABI.  Conventions shared by every call:
  *   - `hos_batch`, `hos_cost_model` and every `const T*` marked HOST are read on
  *     the host during the call.  Every other pointer is DEVICE memory owned by
- *     the caller; the library allocates nothing, keeps no state between calls,
+ *     the caller; the library allocates nothing, keeps no results or data between calls,
  *     enqueues its kernels on `stream` (a cudaStream_t passed as void*) and
  *     returns without synchronising.  Results are valid once `stream` has
  *     reached the point of the call's return.
@@ -23,7 +23,13 @@
  *     base must be 256-byte aligned.  Two calls that share a workspace or an
  *     output buffer must be ordered on the stream.
  *   - Shape limits of this build: n_clients <= 256, batch_cap <= 256,
- *     n_req <= 24384, kv_budget < 2^31, estimated times T_i < 2^32.
+ *     n_req <= 24384, kv_budget < 2^31, estimated times T_i < 2^32; for the lower bounds
+ *     also n_req * R^2 / 2 < 2^63, R = the most KV tokens one request may need
+ *     (kv_reserve_tokens if set, else kv_budget).
+ *   - Calls may come from several host threads at once (each with its own stream, workspace
+ *     and outputs).  The only things the library remembers are idempotent per-device set-up
+ *     facts (a kernel's shared-memory allowance, the address of the built-in scratch), kept
+ *     under a lock.
  */
 #ifndef HOS_H
 #define HOS_H
@@ -48,8 +54,13 @@ enum {
 enum {
     HOS_ST_LIMIT   = 1,       /* iteration limit or 2^39 us clock limit reached; results partial */
     HOS_ST_TRACE   = 2,       /* more iterations than trace slots; extra records dropped         */
-    HOS_ST_INVALID = 4        /* instance data invalid (p_i = 0, o_i = 0, p_i + o_i > kv_budget,
-                                 T_i >= 2^32, assignment outside [0, n_clients))                */
+    HOS_ST_INVALID = 4,       /* instance data invalid (p_i = 0, o_i = 0, p_i + o_i > kv_budget,
+                                 T_i >= 2^32, assignment outside [0, n_clients), or a queue key
+                                 p_i + o_est_i too long to sit beside the client number in 32
+                                 bits: bit_width(max p + o_est) + bit_width(n_clients - 1) > 32) */
+    HOS_ST_RANGE   = 8        /* a lower bound of this instance does not fit 64 bits (products of
+                                 coefficients and token sums that are each inside their limits);
+                                 its hos_lb is zeroed, everything else is unaffected             */
 };
 
 enum { HOS_QUEUE_SORTED = 0, HOS_QUEUE_FCFS = 1 };
@@ -123,7 +134,8 @@ typedef struct hos_client_result {
     int64_t  makespan_us;        /* this client's clock when its last request retired        */
     int64_t  busy_slot_us;       /* sum over iterations of duration * requests advanced       */
     uint32_t n_prefill_iters, n_decode_iters;
-    uint64_t trace_hash;         /* polynomial hash of the trace, produced with or without it */
+    uint64_t trace_hash;         /* checksum of the trace records in order (a multiply-add
+                                    recurrence mod 2^64), produced with or without the trace  */
     double   utilisation;        /* busy_slot_us / (batch_cap * makespan of the simulation)   */
 } hos_client_result;
 
@@ -152,7 +164,7 @@ typedef struct hos_iter_rec { uint32_t dur_us, kind_n, tokens, aux; } hos_iter_r
  *   ls_log         [n_inst][ls_rounds] out, nullable
  *   lb             [n_inst]            out, nullable: the lower bounds of hos_lower_bound, from the
  *                                      sort this call does anyway (saves the separate call its own)
- *   status         [n_inst]            out  0 or HOS_ST_INVALID
+ *   status         [n_inst]            out  0, HOS_ST_INVALID, or HOS_ST_RANGE (with lb)
  */
 int hos_offline_pack(const hos_batch* batch, const hos_cost_model* cm, int ls_rounds,
                      int32_t* assign, int64_t* load, int64_t* makespan_est,
@@ -273,7 +285,8 @@ int hos_lower_bound_static(const hos_batch* batch, const hos_cost_model* cm, hos
 
 /* trace_off[0] = 0, trace_off[x+1] = trace_off[x] + iterations of unit x (exclusive scan of
  * n_prefill_iters + n_decode_iters over cres[0..n_units)).  The trace protocol of
- * hos_online_simulate; no counterpart in the paper beyond "the Gantt chart is recorded". */
+ * hos_online_simulate; no counterpart in the paper beyond the Gantt figures of its Numerical
+ * Experiment section. */
 int hos_trace_offsets(const hos_client_result* cres, int64_t n_units, int64_t* trace_off,
                       void* stream);
 
@@ -289,7 +302,7 @@ const char* hos_strerror(int code);
  * hook(kernel_name, 1, stream, user), called on the host from the launching thread, so that
  * a caller can record CUDA events on the launching stream and count launches.  Process-wide
  * and not thread-safe: set it only while no other thread is inside the library; pass NULL
- * to remove it.  With no hook set the library keeps no state between calls.
+ * to remove it.  It is never consulted for any decision of the hot path.
  */
 typedef void (*hos_launch_hook)(const char* kernel, int phase, void* stream, void* user);
 void hos_set_launch_hook(hos_launch_hook hook, void* user);

@@ -16,7 +16,7 @@ import numpy as np
 _PKG = os.path.dirname(os.path.abspath(__file__))
 
 HOS_QUEUE_SORTED, HOS_QUEUE_FCFS = 0, 1
-HOS_ST_LIMIT, HOS_ST_TRACE, HOS_ST_INVALID = 1, 2, 4
+HOS_ST_LIMIT, HOS_ST_TRACE, HOS_ST_INVALID, HOS_ST_RANGE = 1, 2, 4, 8
 
 LS_MOVE_DTYPE = np.dtype([("i", "<i4"), ("u", "<i4"), ("k", "<i4"), ("v", "<i8")], align=True)
 LB_DTYPE = np.dtype([(n, "<i8") for n in ("lb_pack", "sum_T", "max_T", "pair_T", "lb_sim_us",

@@ -1,6 +1,9 @@
 // C-ABI layer: argument validation, workspace carving, kernel sequencing.
 #include <cuda_runtime.h>
 
+#include <mutex>
+#include <unordered_map>
+
 #include "hos.h"
 #include "hos_common.cuh"
 #include "hos_kernels.h"
@@ -47,6 +50,14 @@ int check_cost(const hos_cost_model* cm, const hos_batch* b) {
                                    kv / cm->decode_kv_div;
     if (pre >= (1ull << 31) || dec >= (1ull << 31)) return HOS_E_INVALID;
     return HOS_OK;
+}
+
+// The lower bounds add up o_i * p_i + o_i (o_i - 1) / 2 <= (p_i + o_i)^2 / 2 over the requests of an
+// instance in 64 bits: the largest admissible request bounds that sum.
+int check_lb_range(const hos_batch* b) {
+    const unsigned long long most = b->kv_reserve_tokens ? b->kv_reserve_tokens : (unsigned long long)b->kv_budget;
+    const unsigned __int128 worst = (unsigned __int128)most * most / 2 * (unsigned long long)b->n_req;
+    return worst >> 63 ? HOS_E_UNSUPPORTED : HOS_OK;
 }
 
 int check_ws(const void* ws, size_t have, size_t need) {
@@ -129,6 +140,23 @@ void* g_hook_user = nullptr;
 }  // namespace
 
 namespace hos {
+cudaError_t allow_max_dynamic_smem(const void* func) {
+    static std::mutex mu;
+    static std::unordered_map<const void*, unsigned long long> done;      // kernel -> devices already set
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    std::lock_guard<std::mutex> lock(mu);
+    unsigned long long& mask = done[func];
+    if (dev >= 0 && dev < 64 && ((mask >> dev) & 1ull)) return cudaSuccess;
+    cudaFuncAttributes attr;
+    if ((e = cudaFuncGetAttributes(&attr, func)) != cudaSuccess) return e;
+    const int room = (int)SMEM_LIMIT - (int)attr.sharedSizeBytes;
+    if ((e = cudaFuncSetAttribute(func, cudaFuncAttributeMaxDynamicSharedMemorySize, room)) != cudaSuccess) return e;
+    if (dev >= 0 && dev < 64) mask |= 1ull << dev;
+    return cudaSuccess;
+}
+
 void launch_hook(const char* kernel, int phase, cudaStream_t st) {
     if (g_hook) g_hook(kernel, phase, static_cast<void*>(st), g_hook_user);
 }
@@ -157,13 +185,14 @@ int hos_offline_pack(const hos_batch* b, const hos_cost_model* cm, int ls_rounds
     if (rc) return rc;
     if ((rc = check_cost(cm, b))) return rc;
     if (!assign || !load || !makespan_est || !rounds_applied || !status || ls_rounds < 0) return HOS_E_INVALID;
+    if (lb && (rc = check_lb_range(b))) return rc;
     if (estimate_sort_smem(b->n_req) > SMEM_LIMIT) return HOS_E_UNSUPPORTED;
     if ((rc = check_ws(ws, ws_bytes, hos_offline_workspace_bytes(b, 1, ls_rounds)))) return rc;
     const OfflineWs w = carve_offline(b, ws, 1, ls_rounds);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const int n_pad = pad4(b->n_req);
     if ((rc = cuda_rc(launch_estimate_sort(*b, *cm, w.T_sorted, w.order, w.info, status, n_pad, st)))) return rc;
-    if (lb && (rc = cuda_rc(launch_lower_bound(*b, *cm, w.T_sorted, w.info, n_pad, lb, st)))) return rc;
+    if (lb && (rc = cuda_rc(launch_lower_bound(*b, *cm, w.T_sorted, w.info, n_pad, lb, status, st)))) return rc;
     if ((rc = cuda_rc(launch_lpt(*b, w.T_sorted, w.order, w.info, n_pad, assign,
                                  reinterpret_cast<long long*>(load),
                                  reinterpret_cast<long long*>(makespan_est), w.ls_C, st))))
@@ -203,13 +232,14 @@ int hos_lower_bound(const hos_batch* b, const hos_cost_model* cm, hos_lb* out, i
     if (rc) return rc;
     if ((rc = check_cost(cm, b))) return rc;
     if (!out || !status) return HOS_E_INVALID;
+    if ((rc = check_lb_range(b))) return rc;
     if (estimate_sort_smem(b->n_req) > SMEM_LIMIT) return HOS_E_UNSUPPORTED;
     if ((rc = check_ws(ws, ws_bytes, hos_lower_bound_workspace_bytes(b)))) return rc;
     const OfflineWs w = carve_offline(b, ws, 1, 0);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const int n_pad = pad4(b->n_req);
     if ((rc = cuda_rc(launch_estimate_sort(*b, *cm, w.T_sorted, w.order, w.info, status, n_pad, st)))) return rc;
-    return cuda_rc(launch_lower_bound(*b, *cm, w.T_sorted, w.info, n_pad, out, st));
+    return cuda_rc(launch_lower_bound(*b, *cm, w.T_sorted, w.info, n_pad, out, status, st));
 }
 
 int hos_online_simulate(const hos_batch* b, const int32_t* assign, const hos_cost_model* cm,

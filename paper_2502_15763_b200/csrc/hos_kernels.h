@@ -13,6 +13,11 @@ struct InstInfo;
 // Calls the user's launch hook, if one is set (see hos_set_launch_hook).
 void launch_hook(const char* kernel, int phase, cudaStream_t st);
 
+// Lets `func` be launched with any dynamic shared memory size up to what an SM offers beside the
+// kernel's static shared memory.  Done once per kernel and device and never lowered, so that
+// host threads that launch different shapes at the same time cannot undo each other's setting.
+cudaError_t allow_max_dynamic_smem(const void* func);
+
 size_t estimate_sort_smem(int n_req);
 size_t local_search_smem(int n_req, int n_clients);
 size_t queue_build_smem(int n_req);
@@ -31,7 +36,7 @@ cudaError_t launch_local_search(const hos_batch& b, const uint32_t* T_sorted, co
                                 int32_t* ws_bad, cudaStream_t st);
 size_t local_search_index_bytes(int n_req);
 cudaError_t launch_lower_bound(const hos_batch& b, const hos_cost_model& cm, const uint32_t* T_sorted,
-                               const InstInfo* info, int n_pad, hos_lb* out, cudaStream_t st);
+                               const InstInfo* info, int n_pad, hos_lb* out, int32_t* status, cudaStream_t st);
 
 cudaError_t launch_queue_build(const hos_batch& b, const int32_t* assign, uint32_t p_max, int queue_order, uint2* q_po,
                                uint32_t* q_key, uint32_t* q_req, int32_t* q_off, unsigned long long* inst_O,

@@ -1176,7 +1176,7 @@ __device__ __forceinline__ unsigned long long floor_sum_below(uint32_t n, uint32
 __global__ void __launch_bounds__(256)
 k_lower_bound(const uint32_t* __restrict__ p, const uint32_t* __restrict__ o, int n_req, int n_pad,
               int n_clients, int cap, hos_cost_model cm, int q_shift, const uint32_t* __restrict__ T_sorted,
-              const InstInfo* __restrict__ info, hos_lb* __restrict__ out) {
+              const InstInfo* __restrict__ info, hos_lb* __restrict__ out, int32_t* __restrict__ status_out) {
     __shared__ unsigned long long red[32];
     const int inst = blockIdx.x;
     const InstInfo inf = info[inst];
@@ -1226,27 +1226,39 @@ k_lower_bound(const uint32_t* __restrict__ p, const uint32_t* __restrict__ o, in
         lb = pairT > lb ? pairT : lb;
         const unsigned long long n_pre = ((unsigned long long)n_req + C - 1ull) / C;
         const unsigned long long n_dec = (O + C - 1ull) / C;
-        unsigned long long tp_star, tp_paper = 0;
+        // Scaled sums in 128 bits: coefficients and sums that are each inside their limits can still
+        // carry these products past 64 bits, and a bound that does not fit is flagged, not wrapped.
+        typedef unsigned __int128 u128;
+        const u128 lim = (u128)0x7FFFFFFFFFFFFFFFull;
+        u128 tp_wide, tp_paper_wide = 0;
         if (cm.n_levels == 0) {
-            tp_star = (unsigned long long)cm.prefill_fixed_us * n_pre + (unsigned long long)cm.prefill_per_token_us * P;
+            tp_wide = (u128)cm.prefill_fixed_us * n_pre + (u128)cm.prefill_per_token_us * P;
         } else {
             // at least n_pre stages of at least the smallest level's time; a stage of level l carries
             // at most N^cap_l tokens, so P tokens cost at least min_l floor(P / N^cap_l) T^p_l
-            const unsigned long long by_count = (unsigned long long)cm.level_time_us[0] * n_pre;
-            unsigned long long by_tokens = ~0ull;
+            const u128 by_count = (u128)cm.level_time_us[0] * n_pre;
+            u128 by_tokens = ~(u128)0;
             for (uint32_t l = 0; l < cm.n_levels; ++l) {
-                const unsigned long long v = (P / cm.level_cap_tokens[l]) * cm.level_time_us[l];
+                const u128 v = (u128)(P / cm.level_cap_tokens[l]) * cm.level_time_us[l];
                 by_tokens = v < by_tokens ? v : by_tokens;
             }
-            tp_star = by_count > by_tokens ? by_count : by_tokens;
-            tp_paper = (P / cm.level_cap_tokens[cm.n_levels - 1]) * cm.level_time_us[cm.n_levels - 1];
+            tp_wide = by_count > by_tokens ? by_count : by_tokens;
+            tp_paper_wide = (u128)(P / cm.level_cap_tokens[cm.n_levels - 1]) * cm.level_time_us[cm.n_levels - 1];
         }
-        r.tp_paper_us = (long long)tp_paper;
-        const unsigned long long td_q = q * ((ad - 1ull) * n_dec + bd * O) + K;
-        const unsigned long long work = (q * tp_star + td_q + q * M - 1ull) / (q * M);
+        const u128 td_q = (u128)q * ((u128)(ad - 1ull) * n_dec + (u128)bd * O) + K;
+        const u128 tot_q = (u128)q * tp_wide + td_q + (u128)(q * M - 1ull);
+        if (tp_wide > lim || tp_paper_wide > lim || td_q > lim || tot_q > lim) {
+            out[inst] = hos_lb{0, 0, 0, 0, 0, 0, 0, 0, 0};
+            if (status_out) atomicOr(&status_out[inst], HOS_ST_RANGE);
+            return;
+        }
+        const unsigned long long tp_star = (unsigned long long)tp_wide;
+        r.tp_paper_us = (long long)(unsigned long long)tp_paper_wide;
+        const unsigned long long td_q64 = (unsigned long long)td_q;
+        const unsigned long long work = (unsigned long long)tot_q / (q * M);
         r.lb_pack = (long long)lb; r.sum_T = (long long)sumT; r.max_T = (long long)maxT; r.pair_T = (long long)pairT;
         r.tp_star_us = (long long)((tp_star + M - 1ull) / M);
-        r.td_star_us = (long long)((td_q + q * M - 1ull) / (q * M));
+        r.td_star_us = (long long)((td_q64 + q * M - 1ull) / (q * M));
         r.chain_us = (long long)chain;
         r.lb_sim_us = (long long)(work > chain ? work : chain);
         out[inst] = r;
@@ -1268,7 +1280,7 @@ cudaError_t launch_estimate_sort(const hos_batch& b, const hos_cost_model& cm, u
                                  cudaStream_t st) {
     const size_t smem = estimate_sort_smem(b.n_req);
     auto kern = b.n_req <= 65536 ? k_estimate_sort<uint16_t> : k_estimate_sort<uint32_t>;
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    cudaError_t e = allow_max_dynamic_smem(reinterpret_cast<const void*>(kern));
     if (e != cudaSuccess) return e;
     launch_hook("k_estimate_sort", 0, st);
     kern<<<b.n_inst, SORT_THREADS, smem, st>>>(b.p, b.o, b.o_est, b.n_req,
@@ -1309,8 +1321,8 @@ cudaError_t launch_local_search(const hos_batch& b, const uint32_t* T_sorted, co
                               (load_from_assign ? 0
                                                 : (LSB_THREADS / 32) * (narrow ? lists_stage_bytes_per_warp<uint16_t>(b.n_clients)
                                                                                : lists_stage_bytes_per_warp<uint32_t>(b.n_clients)));
-    cudaError_t ea = narrow ? cudaFuncSetAttribute(k_ls_lists<uint16_t>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_lists)
-                            : cudaFuncSetAttribute(k_ls_lists<uint32_t>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_lists);
+    cudaError_t ea = narrow ? allow_max_dynamic_smem(reinterpret_cast<const void*>(k_ls_lists<uint16_t>))
+                            : allow_max_dynamic_smem(reinterpret_cast<const void*>(k_ls_lists<uint32_t>));
     if (ea != cudaSuccess) return ea;
     const unsigned grid = (unsigned)(b.n_inst * n_copies);
     launch_hook("k_ls_lists", 0, st);
@@ -1343,13 +1355,13 @@ cudaError_t launch_local_search(const hos_batch& b, const uint32_t* T_sorted, co
 }
 
 cudaError_t launch_lower_bound(const hos_batch& b, const hos_cost_model& cm, const uint32_t* T_sorted,
-                               const InstInfo* info, int n_pad, hos_lb* out, cudaStream_t st) {
+                               const InstInfo* info, int n_pad, hos_lb* out, int32_t* status, cudaStream_t st) {
     int q_shift = -1;                                    // power-of-two KV divisor -> shift
     if ((cm.decode_kv_div & (cm.decode_kv_div - 1)) == 0)
         for (q_shift = 0; (1u << q_shift) != cm.decode_kv_div; ++q_shift) {}
     launch_hook("k_lower_bound", 0, st);
     k_lower_bound<<<b.n_inst, 256, 0, st>>>(b.p, b.o, b.n_req, n_pad, b.n_clients, b.batch_cap, cm, q_shift,
-                                            T_sorted, info, out);
+                                            T_sorted, info, out, status);
     launch_hook("k_lower_bound", 1, st);
     return cudaGetLastError();
 }

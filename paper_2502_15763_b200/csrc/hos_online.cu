@@ -59,6 +59,10 @@ k_queue_build(const uint32_t* __restrict__ p, const uint32_t* __restrict__ o,
     mxp = block_max_u64(mxp, red);
     bad = block_max_u64(bad, red);
     __syncthreads();
+    const int kb = (queue_order == HOS_QUEUE_SORTED) ? bit_width_u32((uint32_t)mxk) : 0;
+    // the composite sort key, client above p + (estimated) o, has 32 bits: an estimate so long
+    // that it does not fit beside the client bits invalidates the instance (uniform over the CTA)
+    if (kb + bit_width_u32((uint32_t)(n_clients - 1)) > 32) bad = 1;
     if (threadIdx.x == 0) {
         inst_O[inst] = sumO;
         // bit 8 (internal): some p + o needs more than 16 bits -> the simulator's wide heap entries
@@ -66,7 +70,6 @@ k_queue_build(const uint32_t* __restrict__ p, const uint32_t* __restrict__ o,
     }
     if (bad) return;
 
-    const int kb = (queue_order == HOS_QUEUE_SORTED) ? bit_width_u32((uint32_t)mxk) : 0;
     const uint32_t kmask = kb >= 32 ? 0xFFFFFFFFu : ((1u << kb) - 1u);
     const int nbits = kb + bit_width_u32((uint32_t)(n_clients - 1));
     // The sort only looks at the low nbits of a key.  When the prompt length fits the bits above
@@ -95,9 +98,9 @@ k_queue_build(const uint32_t* __restrict__ p, const uint32_t* __restrict__ o,
         qr[r] = id;
         qp[r] = make_uint2(pp, o_from_key ? totk - pp : oi[id]);
         if (q_key) q_key[(size_t)inst * n_pad + r] = kb > 0 && kb < 32 ? totk : pp + ei[id];
-        const int c = (int)(low >> kb);
+        const int c = kb >= 32 ? 0 : (int)(low >> kb);            // 32 key bits leave none for the client: one client
         const uint32_t kprev = r > 0 ? s.key[sorted[r - 1]] : 0u;
-        const int cprev = r > 0 ? (int)(((ride && nbits < 32) ? (kprev & ((1u << nbits) - 1u)) : kprev) >> kb) : -1;
+        const int cprev = r > 0 ? (kb >= 32 ? 0 : (int)(((ride && nbits < 32) ? (kprev & ((1u << nbits) - 1u)) : kprev) >> kb)) : -1;
         for (int cc = cprev + 1; cc <= c; ++cc) qo[cc] = r;
         if (r == n_req - 1)
             for (int cc = c + 1; cc <= n_clients; ++cc) qo[cc] = n_req;
@@ -940,7 +943,7 @@ cudaError_t launch_queue_build(const hos_batch& b, const int32_t* assign, uint32
                                int32_t* inst_status, int n_pad, cudaStream_t st) {
     const size_t smem = queue_build_smem(b.n_req);
     auto kern = b.n_req <= 65536 ? k_queue_build<uint16_t> : k_queue_build<uint32_t>;
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    cudaError_t e = allow_max_dynamic_smem(reinterpret_cast<const void*>(kern));
     if (e != cudaSuccess) return e;
     launch_hook("k_queue_build", 0, st);
     kern<<<b.n_inst, SORT_THREADS, smem, st>>>(b.p, b.o, b.o_est, assign, b.n_req, b.n_clients,
@@ -991,9 +994,9 @@ cudaError_t launch_simulate(const hos_batch& b, const hos_cost_model& cm, const 
     const size_t smem_n = warp_n * wpc_n, smem_w = warp_w * wpc_w;
     const unsigned grid_n = (unsigned)((n_warps + wpc_n - 1) / wpc_n);
     const unsigned grid_w = (unsigned)((n_warps + wpc_w - 1) / wpc_w);
-    cudaError_t e = cudaFuncSetAttribute(k_simulate<NarrowEntry>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_n);
+    cudaError_t e = allow_max_dynamic_smem(reinterpret_cast<const void*>(k_simulate<NarrowEntry>));
     if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(k_simulate<WideEntry>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_w);
+    e = allow_max_dynamic_smem(reinterpret_cast<const void*>(k_simulate<WideEntry>));
     if (e != cudaSuccess) return e;
     launch_hook("k_simulate", 0, st);
     k_simulate<NarrowEntry><<<grid_n, SIM_THREADS * wpc_n, smem_n, st>>>(
@@ -1030,7 +1033,7 @@ cudaError_t launch_simulate_steal(const hos_batch& b, const hos_cost_model& cm, 
         for (q_shift = 0; (1u << q_shift) != cm.decode_kv_div; ++q_shift) {}
     const size_t smem_n = simulate_steal_smem(b.n_clients, cap, false);
     const size_t smem_w = simulate_steal_smem(b.n_clients, cap, true);
-    cudaError_t e = cudaFuncSetAttribute(k_simulate_steal<NarrowEntry>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_n);
+    cudaError_t e = allow_max_dynamic_smem(reinterpret_cast<const void*>(k_simulate_steal<NarrowEntry>));
     if (e != cudaSuccess) return e;
     launch_hook("k_simulate_steal", 0, st);
     k_simulate_steal<NarrowEntry><<<grid, threads, smem_n, st>>>(
@@ -1038,7 +1041,7 @@ cudaError_t launch_simulate_steal(const hos_batch& b, const hos_cost_model& cm, 
         kv, cm, q_shift, max_iters, cres, trace, trace_off, status, served_by);
     launch_hook("k_simulate_steal", 1, st);
     if (b.kv_budget >= 65536) {                          // otherwise no p + o can reach 2^16
-        e = cudaFuncSetAttribute(k_simulate_steal<WideEntry>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_w);
+        e = allow_max_dynamic_smem(reinterpret_cast<const void*>(k_simulate_steal<WideEntry>));
         if (e != cudaSuccess) return e;
         launch_hook("k_simulate_steal_wide", 0, st);
         k_simulate_steal<WideEntry><<<grid, threads, smem_w, st>>>(

@@ -132,9 +132,8 @@ def check_simulate(hos, p, o, M, cap, kv, cm, assign, lambdas, mode, insts=None,
     return g
 
 
-def check_simulate_steal(hos, p, o, M, cap, kv, cm, assign, lambdas, mode, insts=None, max_iters=0x7FFFFFFF,
-                         est=None, rsv=0):
-    """hos_online_simulate_steal (counts, then a traced run with exact slots) against the oracle."""
+def gpu_simulate_steal(hos, p, o, M, cap, kv, cm, assign, lambdas, mode, max_iters=0x7FFFFFFF, est=None, rsv=0):
+    """hos_online_simulate_steal: counts, then a traced run with exact slots.  Host-side views."""
     import torch
     from paper_2502_15763_b200.binding import view_struct
     dp, do, da = to_dev(p), to_dev(o), to_dev(assign)
@@ -146,12 +145,16 @@ def check_simulate_steal(hos, p, o, M, cap, kv, cm, assign, lambdas, mode, insts
     r2 = hos.hos_online_simulate_steal(dp, do, M, cap, kv, cm, da, dl, mode, max_iters, trace=trace, trace_off=off,
                                        want_served_by=True, **ek)
     assert torch.equal(r["cres"][..., :32], r2["cres"][..., :32]) and torch.equal(r["served_by"], r2["served_by"])
-    cres = view_struct(r2["cres"], hos.CLIENT_RESULT_DTYPE)
-    sres = view_struct(r2["sres"], hos.SIM_RESULT_DTYPE)
-    st = r2["status"].cpu().numpy()
-    served = r2["served_by"].cpu().numpy()
-    tr = view_struct(trace, hos.ITER_REC_DTYPE)
-    toff = off.cpu().numpy()
+    return dict(cres=view_struct(r2["cres"], hos.CLIENT_RESULT_DTYPE), sres=view_struct(r2["sres"], hos.SIM_RESULT_DTYPE),
+                status=r2["status"].cpu().numpy(), served_by=r2["served_by"].cpu().numpy(),
+                trace=view_struct(trace, hos.ITER_REC_DTYPE), trace_off=off.cpu().numpy())
+
+
+def check_simulate_steal(hos, p, o, M, cap, kv, cm, assign, lambdas, mode, insts=None, max_iters=0x7FFFFFFF,
+                         est=None, rsv=0):
+    """hos_online_simulate_steal (counts, then a traced run with exact slots) against the oracle."""
+    g = gpu_simulate_steal(hos, p, o, M, cap, kv, cm, assign, lambdas, mode, max_iters, est, rsv)
+    cres, sres, st, served, tr, toff = g["cres"], g["sres"], g["status"], g["served_by"], g["trace"], g["trace_off"]
     insts = range(p.shape[0]) if insts is None else insts
     nl = len(lambdas)
     for k in insts:
