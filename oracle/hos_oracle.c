@@ -123,6 +123,77 @@ int ora_local_search(int n, int M, const int64_t* T, int32_t* assign, int64_t* l
 }
 
 /* ------------------------------------------------------------------------- */
+/* A stronger packing for Eq. 26-30: MULTIFIT (Coffman, Garey and Johnson,    */
+/* "An application of bin-packing to multiprocessor scheduling", 1978)        */
+/* ------------------------------------------------------------------------- */
+
+/* First-fit decreasing with capacity C: every request, longest first, goes to the LOWEST client
+ * on which it still fits (load + T <= C).  Returns 1 when every request found a client. */
+static int first_fit_decreasing(int n, int M, const int64_t* T, const int32_t* order, int64_t C,
+                                int32_t* assign, int64_t* load)
+{
+    for (int j = 0; j < M; ++j) load[j] = 0;
+    for (int r = 0; r < n; ++r) {
+        int i = order[r];
+        int j = 0;
+        while (j < M && load[j] + T[i] > C) ++j;
+        if (j == M) return 0;
+        assign[i] = j;
+        load[j] += T[i];
+    }
+    return 1;
+}
+
+/* MULTIFIT: bisection on the capacity.  The search starts from the interval the authors give,
+ * C_L = max(ceil(sum T / M), max T) (no packing can do better) and C_U = max(ceil(2 sum T / M), max T)
+ * (first-fit decreasing always succeeds there), in integers: while C_L < C_U and steps remain,
+ * C = floor((C_L + C_U) / 2); success -> C_U = C, failure -> C_L = C + 1.  The packing is the
+ * first-fit decreasing one at the final C_U.  Returns 1 and fills assign/load when that packing
+ * exists (always, by the authors' result on C_U), 0 otherwise; *C_final gets the capacity. */
+int ora_multifit(int n, int M, const int64_t* T, const int32_t* order, int max_steps,
+                 int32_t* assign, int64_t* load, int64_t* C_final)
+{
+    int64_t sumT = 0, maxT = 0;
+    for (int i = 0; i < n; ++i) { sumT += T[i]; if (T[i] > maxT) maxT = T[i]; }
+    int64_t lo = (sumT + M - 1) / M;
+    if (maxT > lo) lo = maxT;
+    int64_t hi = (2 * sumT + M - 1) / M;
+    if (maxT > hi) hi = maxT;
+    for (int step = 0; step < max_steps && lo < hi; ++step) {
+        int64_t C = lo + (hi - lo) / 2;
+        if (first_fit_decreasing(n, M, T, order, C, assign, load)) hi = C;
+        else lo = C + 1;
+    }
+    if (C_final) *C_final = hi;
+    return first_fit_decreasing(n, M, T, order, hi, assign, load);
+}
+
+/* The optimum of Eq. 26-30 by trying every assignment (M^n of them): for tiny instances only. */
+static void optimum_rec(int n, int M, const int64_t* T, int i, int64_t* load, int64_t* best)
+{
+    if (i == n) {
+        int64_t m = 0;
+        for (int j = 0; j < M; ++j) if (load[j] > m) m = load[j];
+        if (*best < 0 || m < *best) *best = m;
+        return;
+    }
+    for (int j = 0; j < M; ++j) {
+        load[j] += T[i];
+        optimum_rec(n, M, T, i + 1, load, best);
+        load[j] -= T[i];
+    }
+}
+
+int64_t ora_optimal_makespan(int n, int M, const int64_t* T)
+{
+    int64_t* load = (int64_t*)calloc((size_t)M, sizeof(int64_t));
+    int64_t best = -1;
+    optimum_rec(n, M, T, 0, load, &best);
+    free(load);
+    return best < 0 ? 0 : best;
+}
+
+/* ------------------------------------------------------------------------- */
 /* Lower bounds, Eq. 31-32                                                    */
 /* ------------------------------------------------------------------------- */
 

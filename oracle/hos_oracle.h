@@ -73,6 +73,15 @@ void ora_lpt(int n, int M, const int64_t* T, const int32_t* order, int32_t* assi
 int ora_local_search(int n, int M, const int64_t* T, int32_t* assign, int64_t* load,
                      int rounds, ora_move* log);
 
+/* MULTIFIT (Coffman, Garey, Johnson 1978) for the same model: bisection on a common capacity C
+ * with first-fit decreasing as the feasibility test, at most max_steps probes; the packing is the
+ * first-fit decreasing one at the smallest capacity found.  Returns 1 when it exists. */
+int ora_multifit(int n, int M, const int64_t* T, const int32_t* order, int max_steps,
+                 int32_t* assign, int64_t* load, int64_t* C_final);
+
+/* Optimum of Eq. 26-30 by exhaustive enumeration (M^n assignments; tiny instances only). */
+int64_t ora_optimal_makespan(int n, int M, const int64_t* T);
+
 /* Lower bounds (Eq. 31-32 restated for the affine cost model and M clients of `cap` slots). */
 void ora_lower_bound(int n, int M, int cap, const uint32_t* p, const uint32_t* o,
                      const ora_cost* c, ora_lb* out);

@@ -70,6 +70,8 @@ def lib():
     if _lib is None:
         _lib = C.CDLL(build())
         _lib.ora_local_search.restype = C.c_int
+        _lib.ora_multifit.restype = C.c_int
+        _lib.ora_optimal_makespan.restype = C.c_int64
     return _lib
 
 
@@ -129,6 +131,24 @@ def local_search(T, assign, load, rounds: int):
         _ptr(load, C.c_int64), C.c_int(rounds),
         log.ctypes.data_as(C.POINTER(_Move)) if rounds > 0 else None)
     return assign, load, int(applied), log
+
+
+def multifit(T, order_, M: int, max_steps: int = 64):
+    """MULTIFIT packing: (assign, load, capacity found), or None if first-fit decreasing fails at it."""
+    T = np.ascontiguousarray(T, dtype=np.int64)
+    order_ = np.ascontiguousarray(order_, dtype=np.int32)
+    assign = np.empty(T.shape[0], dtype=np.int32)
+    load = np.zeros(M, dtype=np.int64)
+    cfin = C.c_int64(0)
+    ok = lib().ora_multifit(C.c_int(T.shape[0]), C.c_int(M), _ptr(T, C.c_int64), _ptr(order_, C.c_int32),
+                            C.c_int(max_steps), _ptr(assign, C.c_int32), _ptr(load, C.c_int64), C.byref(cfin))
+    return (assign, load, int(cfin.value)) if ok else None
+
+
+def optimal_makespan(T, M: int) -> int:
+    """Optimum of Eq. 26-30 by exhaustive enumeration (tiny instances only)."""
+    T = np.ascontiguousarray(T, dtype=np.int64)
+    return int(lib().ora_optimal_makespan(C.c_int(T.shape[0]), C.c_int(M), _ptr(T, C.c_int64)))
 
 
 def lower_bound(p, o, M: int, cap: int, cm) -> dict:
@@ -273,14 +293,22 @@ def simulate_steal(assign, p, o, M: int, cm, cap: int, kv_budget: int, lambda_q1
     return SimResult(makespan, busy, util, tps, clients), served
 
 
-def offline_pack(p, o, M: int, cm, ls_rounds: int = 0):
-    """estimate -> order -> LPT -> local search.  Returns dict with T, order, assign, load, ..."""
+def offline_pack(p, o, M: int, cm, ls_rounds: int = 0, multifit_steps: int = 0):
+    """estimate -> order -> LPT (-> MULTIFIT) -> local search.  Returns dict with T, order, assign, load, ...
+
+    multifit_steps > 0: the MULTIFIT packing with at most that many probes replaces the LPT one
+    when its largest load is strictly smaller; `packer` says which was kept (0 LPT, 1 MULTIFIT)."""
     T = estimate(p, o, cm)
     od = order(T)
     assign, load = lpt(T, od, M)
     lpt_assign, lpt_load = assign.copy(), load.copy()
+    packer = 0
+    if multifit_steps > 0:
+        mf = multifit(T, od, M, multifit_steps)
+        if mf is not None and int(mf[1].max()) < int(load.max()):
+            assign, load, packer = mf[0], mf[1], 1
     applied, log = 0, np.zeros(0, dtype=MOVE_DTYPE)
     if ls_rounds > 0:
         assign, load, applied, log = local_search(T, assign, load, ls_rounds)
     return dict(T=T, order=od, assign=assign, load=load, makespan_est=int(load.max()),
-                rounds_applied=applied, ls_log=log, lpt_assign=lpt_assign, lpt_load=lpt_load)
+                rounds_applied=applied, ls_log=log, lpt_assign=lpt_assign, lpt_load=lpt_load, packer=packer)
