@@ -172,6 +172,24 @@ int hos_offline_pack(const hos_batch* batch, const hos_cost_model* cm, int ls_ro
                      void* ws, size_t ws_bytes, void* stream);
 
 /*
+ * hos_offline_pack with a stronger packing before the local search.  The paper solves Eq. 26-30
+ * to optimality with a MIP solver (Numerical Experiment: "offline" and "offline + online" runs);
+ * this call narrows the gap to that optimum with MULTIFIT (Coffman, Garey, Johnson 1978):
+ * bisection on a common capacity C over [max(ceil(sum T / M), max T), max(ceil(2 sum T / M), max T)],
+ * at most `multifit_steps` probes (>= 1; 64 always converges), each probe a first-fit decreasing
+ * pass (every request, longest first, to the lowest client where load + T <= C; success halves the
+ * interval from above, failure from below).  The first-fit decreasing packing at the capacity found
+ * replaces the longest-first list schedule of an instance when its largest load is strictly
+ * smaller; the `ls_rounds` rounds then start from whichever was kept.
+ *   packer [n_inst] out, nullable: 1 where the MULTIFIT packing was kept, 0 where the list
+ *   schedule was.  Everything else as in hos_offline_pack (same workspace size).
+ */
+int hos_offline_pack_multifit(const hos_batch* batch, const hos_cost_model* cm, int multifit_steps,
+                              int ls_rounds, int32_t* assign, int64_t* load, int64_t* makespan_est,
+                              int32_t* rounds_applied, hos_ls_move* ls_log, hos_lb* lb, int32_t* status,
+                              int32_t* packer, void* ws, size_t ws_bytes, void* stream);
+
+/*
  * Local-search rounds only, from given assignments (same rule as in hos_offline_pack).
  * Every instance carries `n_copies` independent assignments (for instance one per
  * multiplier value of a sweep); request data are shared by the copies.

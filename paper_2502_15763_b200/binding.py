@@ -31,7 +31,8 @@ ITER_REC_DTYPE = np.dtype([("dur_us", "<u4"), ("kind_n", "<u4"), ("tokens", "<u4
 _SYMBOLS = ("hos_offline_pack", "hos_local_search", "hos_lower_bound", "hos_online_simulate",
             "hos_trace_offsets", "hos_offline_workspace_bytes", "hos_lower_bound_workspace_bytes",
             "hos_online_workspace_bytes", "hos_strerror", "hos_set_launch_hook",
-            "hos_lower_bound_static", "hos_trace_fill", "hos_online_simulate_steal")
+            "hos_lower_bound_static", "hos_trace_fill", "hos_online_simulate_steal",
+            "hos_offline_pack_multifit")
 
 LAUNCH_HOOK = C.CFUNCTYPE(None, C.c_char_p, C.c_int, C.c_void_p, C.c_void_p)
 
@@ -76,7 +77,7 @@ def lib():
         L.hos_strerror.restype = C.c_char_p
         for name in ("hos_offline_pack", "hos_local_search", "hos_lower_bound",
                      "hos_online_simulate", "hos_trace_offsets", "hos_lower_bound_static", "hos_trace_fill",
-                     "hos_online_simulate_steal"):
+                     "hos_online_simulate_steal", "hos_offline_pack_multifit"):
             getattr(L, name).restype = C.c_int
         _lib = L
     return _lib
@@ -172,8 +173,12 @@ def view_struct(t, dtype: np.dtype) -> np.ndarray:
 
 
 def hos_offline_pack(p, o, n_clients: int, batch_cap: int, kv_budget: int, cost_model, ls_rounds: int = 0,
-                     want_log: bool = False, ws=None, out=None, want_lb: bool = False, o_est=None, kv_reserve: int = 0):
+                     want_log: bool = False, ws=None, out=None, want_lb: bool = False, o_est=None, kv_reserve: int = 0,
+                     multifit_steps: int = 0):
     """Eq. 26-30: estimate, order, LPT, `ls_rounds` local-search rounds.  Returns a dict of tensors.
+
+    multifit_steps > 0 calls hos_offline_pack_multifit instead (MULTIFIT packing kept where it beats
+    the list schedule) and adds 'packer' (int32 [n_inst]) to the result.
 
     out: optional dict with preallocated 'assign', 'load', 'makespan_est', 'rounds_applied', 'status'
     (for instance row slices of larger tensors) to write into instead of new tensors, optionally 'lb'.
@@ -207,12 +212,21 @@ def hos_offline_pack(p, o, n_clients: int, batch_cap: int, kv_budget: int, cost_
         lb = _dev(out["lb"], torch.uint8, "out.lb")
     elif want_lb:
         lb = torch.empty((b.n_inst, LB_DTYPE.itemsize), dtype=torch.uint8, device=dev)
-    rc = L.hos_offline_pack(C.byref(b), C.byref(cm), C.c_int(ls_rounds), _ptr(assign), _ptr(load),
-                            _ptr(makespan), _ptr(applied), _ptr(log), _ptr(lb), _ptr(status), _ptr(ws),
-                            C.c_size_t(ws.numel()), _stream())
-    _check(rc, "hos_offline_pack")
+    packer = None
+    if multifit_steps > 0:
+        packer = torch.empty((b.n_inst,), dtype=torch.int32, device=dev)
+        rc = L.hos_offline_pack_multifit(C.byref(b), C.byref(cm), C.c_int(multifit_steps), C.c_int(ls_rounds),
+                                         _ptr(assign), _ptr(load), _ptr(makespan), _ptr(applied), _ptr(log),
+                                         _ptr(lb), _ptr(status), _ptr(packer), _ptr(ws), C.c_size_t(ws.numel()),
+                                         _stream())
+        _check(rc, "hos_offline_pack_multifit")
+    else:
+        rc = L.hos_offline_pack(C.byref(b), C.byref(cm), C.c_int(ls_rounds), _ptr(assign), _ptr(load),
+                                _ptr(makespan), _ptr(applied), _ptr(log), _ptr(lb), _ptr(status), _ptr(ws),
+                                C.c_size_t(ws.numel()), _stream())
+        _check(rc, "hos_offline_pack")
     return dict(assign=assign, load=load, makespan_est=makespan, rounds_applied=applied, ls_log=log,
-                lb=lb, status=status)
+                lb=lb, status=status, packer=packer)
 
 
 def hos_local_search(p, o, n_clients: int, batch_cap: int, kv_budget: int, cost_model, assign,

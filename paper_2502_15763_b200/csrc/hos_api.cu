@@ -177,14 +177,16 @@ size_t hos_online_workspace_bytes(const hos_batch* b, int n_lambda, int keep_eve
     return carve_online(b, nullptr, n_lambda, keep_events).bytes;
 }
 
-int hos_offline_pack(const hos_batch* b, const hos_cost_model* cm, int ls_rounds, int32_t* assign,
-                     int64_t* load, int64_t* makespan_est, int32_t* rounds_applied,
-                     hos_ls_move* ls_log, hos_lb* lb, int32_t* status, void* ws, size_t ws_bytes,
-                     void* stream) {
+namespace {
+int offline_pack_impl(const hos_batch* b, const hos_cost_model* cm, int multifit_steps, int ls_rounds,
+                      int32_t* assign, int64_t* load, int64_t* makespan_est, int32_t* rounds_applied,
+                      hos_ls_move* ls_log, hos_lb* lb, int32_t* status, int32_t* packer, void* ws,
+                      size_t ws_bytes, void* stream) {
     int rc = check_batch(b);
     if (rc) return rc;
     if ((rc = check_cost(cm, b))) return rc;
-    if (!assign || !load || !makespan_est || !rounds_applied || !status || ls_rounds < 0) return HOS_E_INVALID;
+    if (!assign || !load || !makespan_est || !rounds_applied || !status || ls_rounds < 0 || multifit_steps < 0)
+        return HOS_E_INVALID;
     if (lb && (rc = check_lb_range(b))) return rc;
     if (estimate_sort_smem(b->n_req) > SMEM_LIMIT) return HOS_E_UNSUPPORTED;
     if ((rc = check_ws(ws, ws_bytes, hos_offline_workspace_bytes(b, 1, ls_rounds)))) return rc;
@@ -197,12 +199,38 @@ int hos_offline_pack(const hos_batch* b, const hos_cost_model* cm, int ls_rounds
                                  reinterpret_cast<long long*>(load),
                                  reinterpret_cast<long long*>(makespan_est), w.ls_C, st))))
         return rc;
+    if (multifit_steps > 0) {
+        if ((rc = cuda_rc(launch_multifit(*b, w.T_sorted, w.order, w.info, n_pad, multifit_steps, assign,
+                                          reinterpret_cast<long long*>(load),
+                                          reinterpret_cast<long long*>(makespan_est), w.ls_C, packer, st))))
+            return rc;
+    } else if (packer) {
+        if ((rc = cuda_rc(cudaMemsetAsync(packer, 0, (size_t)b->n_inst * sizeof(int32_t), st)))) return rc;
+    }
     if (ls_rounds == 0)
         return cuda_rc(cudaMemsetAsync(rounds_applied, 0, (size_t)b->n_inst * sizeof(int32_t), st));
     return cuda_rc(launch_local_search(*b, w.T_sorted, w.order, w.info, n_pad, 1, ls_rounds, false, assign,
                                        reinterpret_cast<long long*>(load),
                                        reinterpret_cast<long long*>(makespan_est), rounds_applied,
                                        ls_log, status, w.ls_T, w.ls_I, w.ls_C, w.ls_off, w.ls_bad, st));
+}
+}  // namespace
+
+int hos_offline_pack(const hos_batch* b, const hos_cost_model* cm, int ls_rounds, int32_t* assign,
+                     int64_t* load, int64_t* makespan_est, int32_t* rounds_applied,
+                     hos_ls_move* ls_log, hos_lb* lb, int32_t* status, void* ws, size_t ws_bytes,
+                     void* stream) {
+    return offline_pack_impl(b, cm, 0, ls_rounds, assign, load, makespan_est, rounds_applied, ls_log, lb, status,
+                             nullptr, ws, ws_bytes, stream);
+}
+
+int hos_offline_pack_multifit(const hos_batch* b, const hos_cost_model* cm, int multifit_steps, int ls_rounds,
+                              int32_t* assign, int64_t* load, int64_t* makespan_est, int32_t* rounds_applied,
+                              hos_ls_move* ls_log, hos_lb* lb, int32_t* status, int32_t* packer, void* ws,
+                              size_t ws_bytes, void* stream) {
+    if (multifit_steps < 1) return HOS_E_INVALID;
+    return offline_pack_impl(b, cm, multifit_steps, ls_rounds, assign, load, makespan_est, rounds_applied, ls_log,
+                             lb, status, packer, ws, ws_bytes, stream);
 }
 
 int hos_local_search(const hos_batch* b, const hos_cost_model* cm, int n_copies, int ls_rounds,

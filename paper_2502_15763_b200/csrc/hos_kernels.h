@@ -28,6 +28,9 @@ cudaError_t launch_estimate_sort(const hos_batch& b, const hos_cost_model& cm, u
 cudaError_t launch_lpt(const hos_batch& b, const uint32_t* T_sorted, const uint32_t* order,
                        const InstInfo* info, int n_pad, int32_t* assign, long long* load,
                        long long* makespan, uint8_t* rank_client, cudaStream_t st);
+cudaError_t launch_multifit(const hos_batch& b, const uint32_t* T_sorted, const uint32_t* order,
+                            const InstInfo* info, int n_pad, int max_steps, int32_t* assign, long long* load,
+                            long long* makespan, uint8_t* rank_client, int32_t* packer, cudaStream_t st);
 cudaError_t launch_local_search(const hos_batch& b, const uint32_t* T_sorted, const uint32_t* order,
                                 const InstInfo* info, int n_pad, int n_copies, int rounds,
                                 bool load_from_assign, int32_t* assign, long long* load,

@@ -1,0 +1,192 @@
+// A stronger packing for the offline model (Eq. 26-30): MULTIFIT (Coffman, Garey and Johnson,
+// 1978) -- bisection on a common capacity C, first-fit decreasing as the feasibility test.
+//
+//   k_multifit   one CTA per instance.  The bisection's probes are first-fit decreasing passes
+//                over the whole sorted request table, each a dependent chain (a request goes to
+//                the LOWEST client with room, so every step needs the loads the step before
+//                left).  Seven warps run the seven probes of the next three levels of the
+//                bisection tree side by side -- the capacity that would be probed after
+//                success/success, success/failure, ... -- and one thread then walks the three
+//                levels: the same probe sequence as the step-by-step bisection, in a third of
+//                the passes.  A last pass packs at the capacity found; the result replaces
+//                the list-scheduling one only when its largest load is strictly smaller.
+#include "hos_common.cuh"
+#include "hos_kernels.h"
+
+namespace hos {
+
+constexpr int MF_WARPS = 8;
+constexpr int MF_THREADS = MF_WARPS * 32;
+constexpr int MF_LEVELS = 3;                         // bisection levels resolved per round
+constexpr int MF_NODES = (1 << MF_LEVELS) - 1;       // probes per round, one warp each
+
+// One first-fit decreasing pass by one warp: client j = k * 32 + lane keeps its load in load[k].
+// Returns false at the first request that fits nowhere.  With RECORD, rc[r] gets the client of
+// the request of rank r.  L is the load type: 32 bits when the capacity fits, else 64.
+template <int KPL, typename L, bool RECORD>
+__device__ __forceinline__ bool first_fit_pass(const uint32_t* __restrict__ Ts, int n, int n_clients, L C,
+                                               L (&load)[KPL], uint8_t* rc) {
+    const int lane = lane_id();
+    bool valid[KPL];
+#pragma unroll
+    for (int k = 0; k < KPL; ++k) { load[k] = 0; valid[k] = k * 32 + lane < n_clients; }
+    uint32_t tv_next = lane < n ? __ldg(&Ts[lane]) : 0u;
+    for (int r0 = 0; r0 < n; r0 += 32) {
+        const uint32_t tv = tv_next;
+        const int rn = r0 + 32 + lane;
+        tv_next = rn < n ? __ldg(&Ts[rn]) : 0u;      // the next 32 requests arrive during these
+        const int steps = min(32, n - r0);
+        uint32_t mine = 0;
+        for (int s = 0; s < steps; ++s) {
+            const L t = (L)__shfl_sync(FULL, tv, s);
+            int j = -1;
+#pragma unroll
+            for (int k = 0; k < KPL; ++k) {
+                // load <= C always, so C - load does not wrap whatever t is
+                const unsigned b = __ballot_sync(FULL, valid[k] && t <= C - load[k]);
+                if (j < 0 && b != 0u) {
+                    const int l = __ffs(b) - 1;
+                    j = k * 32 + l;
+                    if (lane == l) load[k] += t;
+                }
+            }
+            if (j < 0) return false;                 // uniform over the warp
+            if (RECORD && lane == s) mine = (uint32_t)j;
+        }
+        if (RECORD && r0 + lane < n) rc[r0 + lane] = (uint8_t)mine;
+    }
+    return true;
+}
+
+template <int KPL, typename L>
+__device__ void multifit_instance(const uint32_t* __restrict__ Ts, const uint32_t* __restrict__ od, int n,
+                                  int n_clients, unsigned long long sum_T, uint32_t max_T, int max_steps,
+                                  int32_t* __restrict__ asg, long long* __restrict__ load_out,
+                                  long long* __restrict__ makespan_out, uint8_t* __restrict__ rank_client,
+                                  int32_t* __restrict__ packer_out, uint8_t* s_rc) {
+    __shared__ unsigned long long s_lo, s_hi;
+    __shared__ int s_steps, s_ok[MF_NODES], s_take;
+    const int warp = warp_id(), lane = lane_id();
+    const unsigned long long M = (unsigned long long)n_clients;
+    if (threadIdx.x == 0) {
+        // the authors' interval: no packing beats C_L, first-fit decreasing always succeeds at C_U
+        const unsigned long long lo = max((sum_T + M - 1ull) / M, (unsigned long long)max_T);
+        const unsigned long long hi = max((2ull * sum_T + M - 1ull) / M, (unsigned long long)max_T);
+        s_lo = lo; s_hi = hi; s_steps = 0; s_take = 0;
+    }
+    __syncthreads();
+    L load[KPL];
+    while (true) {
+        const unsigned long long lo0 = s_lo, hi0 = s_hi;
+        const int steps0 = s_steps;
+        if (lo0 >= hi0 || steps0 >= max_steps) break;            // uniform: shared values
+        if (warp < MF_NODES) {
+            // my node of the tree: depth d, path bits from the top (0 = the probe above succeeded)
+            const int d = warp == 0 ? 0 : (warp < 3 ? 1 : 2);
+            const int path = warp - ((1 << d) - 1);
+            unsigned long long lo = lo0, hi = hi0;
+            bool active = steps0 + d < max_steps;
+            for (int e = d - 1; e >= 0 && active; --e) {
+                if (lo >= hi) { active = false; break; }
+                const unsigned long long C = lo + (hi - lo) / 2;
+                if ((path >> e) & 1) lo = C + 1; else hi = C;
+            }
+            active = active && lo < hi;
+            if (active) {
+                const unsigned long long C = lo + (hi - lo) / 2;
+                const bool ok = first_fit_pass<KPL, L, false>(Ts, n, n_clients, (L)C, load, nullptr);
+                if (lane == 0) s_ok[warp] = ok ? 1 : 0;
+            }
+        }
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            unsigned long long lo = lo0, hi = hi0;
+            int steps = steps0, node = 0;
+            for (int d = 0; d < MF_LEVELS && lo < hi && steps < max_steps; ++d) {
+                const unsigned long long C = lo + (hi - lo) / 2;
+                const bool ok = s_ok[node] != 0;
+                if (ok) hi = C; else lo = C + 1;
+                node = 2 * node + (ok ? 1 : 2);
+                ++steps;
+            }
+            s_lo = lo; s_hi = hi; s_steps = steps;
+        }
+        __syncthreads();
+    }
+    // the packing at the capacity found; taken only when strictly better than what is there
+    if (warp == 0) {
+        const bool ok = first_fit_pass<KPL, L, true>(Ts, n, n_clients, (L)s_hi, load, s_rc);
+        unsigned long long mx = 0;
+#pragma unroll
+        for (int k = 0; k < KPL; ++k)
+            if (k * 32 + lane < n_clients) mx = max(mx, (unsigned long long)load[k]);
+        mx = warp_max_u64(mx);
+        const bool take = ok && (long long)mx < makespan_out[blockIdx.x];
+        if (take) {
+#pragma unroll
+            for (int k = 0; k < KPL; ++k)
+                if (k * 32 + lane < n_clients) load_out[(size_t)blockIdx.x * n_clients + k * 32 + lane] = (long long)load[k];
+        }
+        __syncwarp();
+        if (lane == 0) {
+            if (take) makespan_out[blockIdx.x] = (long long)mx;
+            if (packer_out) packer_out[blockIdx.x] = take ? 1 : 0;
+            s_take = take ? 1 : 0;
+        }
+    }
+    __syncthreads();
+    if (s_take) {
+        for (int r = threadIdx.x; r < n; r += MF_THREADS) {
+            const uint8_t c = s_rc[r];
+            asg[od[r]] = (int32_t)c;
+            if (rank_client) rank_client[r] = c;
+        }
+    }
+}
+
+template <int KPL>
+__global__ void __launch_bounds__(MF_THREADS)
+k_multifit(const uint32_t* __restrict__ T_sorted, const uint32_t* __restrict__ order,
+           const InstInfo* __restrict__ info, int n_req, int n_pad, int n_clients, int max_steps,
+           int32_t* __restrict__ assign, long long* __restrict__ load_out, long long* __restrict__ makespan_out,
+           uint8_t* __restrict__ rank_client, int32_t* __restrict__ packer_out) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    const int inst = blockIdx.x;
+    const InstInfo inf = info[inst];
+    if (inf.status) {
+        if (threadIdx.x == 0 && packer_out) packer_out[inst] = 0;
+        return;
+    }
+    const uint32_t* Ts = T_sorted + (size_t)inst * n_pad;
+    const uint32_t* od = order + (size_t)inst * n_pad;
+    int32_t* asg = assign + (size_t)inst * n_req;
+    uint8_t* rc = rank_client ? rank_client + (size_t)inst * n_pad : nullptr;
+    const unsigned long long M = (unsigned long long)n_clients;
+    const unsigned long long hi = max((2ull * inf.sum_T + M - 1ull) / M, (unsigned long long)inf.max_T);
+    if (hi <= 0xFFFFFFFFull)
+        multifit_instance<KPL, uint32_t>(Ts, od, n_req, n_clients, inf.sum_T, inf.max_T, max_steps, asg, load_out,
+                                         makespan_out, rc, packer_out, smem_raw);
+    else
+        multifit_instance<KPL, unsigned long long>(Ts, od, n_req, n_clients, inf.sum_T, inf.max_T, max_steps, asg,
+                                                   load_out, makespan_out, rc, packer_out, smem_raw);
+}
+
+cudaError_t launch_multifit(const hos_batch& b, const uint32_t* T_sorted, const uint32_t* order,
+                            const InstInfo* info, int n_pad, int max_steps, int32_t* assign, long long* load,
+                            long long* makespan, uint8_t* rank_client, int32_t* packer, cudaStream_t st) {
+    const int M = b.n_clients;
+    const size_t smem = ((size_t)b.n_req + 15) & ~(size_t)15;
+#define HOS_MF(KPL)                                                                                        \
+    k_multifit<KPL><<<b.n_inst, MF_THREADS, smem, st>>>(T_sorted, order, info, b.n_req, n_pad, M, max_steps, \
+                                                        assign, load, makespan, rank_client, packer)
+    launch_hook("k_multifit", 0, st);
+    if (M <= 32) HOS_MF(1);
+    else if (M <= 64) HOS_MF(2);
+    else if (M <= 128) HOS_MF(4);
+    else HOS_MF(8);
+#undef HOS_MF
+    launch_hook("k_multifit", 1, st);
+    return cudaGetLastError();
+}
+
+}  // namespace hos

@@ -14,9 +14,10 @@ def to_dev(a, dtype=np.int32):
     return torch.from_numpy(a.astype(dtype, copy=False)).cuda()
 
 
-def gpu_offline(hos, p, o, M, cap, kv, cm, ls_rounds, est=None, rsv=0):
+def gpu_offline(hos, p, o, M, cap, kv, cm, ls_rounds, est=None, rsv=0, multifit_steps=0):
     ek = dict(o_est=None if est is None else to_dev(est), kv_reserve=rsv)
-    r = hos.hos_offline_pack(to_dev(p), to_dev(o), M, cap, kv, cm, ls_rounds, want_log=True, want_lb=True, **ek)
+    r = hos.hos_offline_pack(to_dev(p), to_dev(o), M, cap, kv, cm, ls_rounds, want_log=True, want_lb=True,
+                             multifit_steps=multifit_steps, **ek)
     import torch
     sep = hos.hos_lower_bound(to_dev(p), to_dev(o), M, cap, kv, cm, **ek)
     assert torch.equal(r["lb"], sep["lb"]), "bounds from hos_offline_pack differ from hos_lower_bound"
@@ -27,13 +28,16 @@ def gpu_offline(hos, p, o, M, cap, kv, cm, ls_rounds, est=None, rsv=0):
     return out
 
 
-def check_offline(hos, p, o, M, cap, kv, cm, ls_rounds, insts=None, est=None, rsv=0):
+def check_offline(hos, p, o, M, cap, kv, cm, ls_rounds, insts=None, est=None, rsv=0, multifit_steps=0):
     """GPU offline pack of the whole batch against the oracle on `insts` (default: all)."""
-    g = gpu_offline(hos, p, o, M, cap, kv, cm, ls_rounds, est, rsv)
+    g = gpu_offline(hos, p, o, M, cap, kv, cm, ls_rounds, est, rsv, multifit_steps)
     insts = range(p.shape[0]) if insts is None else insts
     for k in insts:
-        e = ora.offline_pack(p[k], o[k] if est is None else est[k], M, cm, ls_rounds)   # packed on what is known
+        e = ora.offline_pack(p[k], o[k] if est is None else est[k], M, cm, ls_rounds,
+                             multifit_steps=multifit_steps)                             # packed on what is known
         assert g["status"][k] == 0
+        if multifit_steps > 0:
+            assert int(g["packer"][k]) == e["packer"], f"packer differs in instance {k}"
         assert np.array_equal(g["assign"][k], e["assign"]), f"assign differs in instance {k}"
         assert np.array_equal(g["load"][k], e["load"]), f"load differs in instance {k}"
         assert int(g["makespan_est"][k]) == e["makespan_est"]

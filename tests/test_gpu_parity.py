@@ -363,3 +363,43 @@ def test_values_beyond_the_arithmetic_range_are_flagged(hos):
     assert pk["status"].cpu().tolist() == [hos.HOS_ST_RANGE, 0] and (pk["assign"][0] >= 0).all()
     with pytest.raises(hos.HosError):                          # the sums themselves could pass 64 bits
         hos.hos_lower_bound(H.to_dev(p), H.to_dev(o), 2, 1, (1 << 31) - 1, cm)
+
+
+@pytest.mark.parametrize("n,M,hi,scale,steps", [(7, 3, 6, 1, 64), (1, 1, 50, 1, 64), (40, 64, 300, 1, 64),
+                                                 (97, 5, 20, 1, 64), (300, 8, 2000, 1, 64), (300, 8, 2000, 1, 1),
+                                                 (300, 8, 2000, 1, 5), (1000, 33, 900, 1, 64), (700, 100, 400, 1, 7),
+                                                 (2050, 256, 3000, 1, 64), (500, 4, 3000, 1000, 64),
+                                                 (1300, 130, 60, 1, 64)])
+def test_multifit_packing(hos, n, M, hi, scale, steps):
+    """hos_offline_pack_multifit against the oracle's MULTIFIT: which packing is kept, the packing,
+    and the local search that starts from it; step limits, ties, 64-bit loads (scale)."""
+    rng = np.random.default_rng(n * 31 + M + steps)
+    n_inst = 4
+    p = rng.integers(1, hi + 1, size=(n_inst, n)).astype(np.uint32)
+    o = rng.integers(1, hi // 3 + 2, size=(n_inst, n)).astype(np.uint32)
+    p[1, ::3] = p[1, 0]                                            # runs of equal T
+    o[1, ::3] = o[1, 0]
+    cm = (20000, 40, 15000, 300, 16, 40 * scale, 350 * scale)
+    g = H.check_offline(hos, p, o, M, 16, 10 ** 7, cm, 8, multifit_steps=steps)
+    lb = H.check_lower_bound(hos, p, o, M, 16, 10 ** 7, cm)
+    assert (lb["lb_pack"] <= g["makespan_est"]).all()
+    plain = H.gpu_offline(hos, p, o, M, 16, 10 ** 7, cm, 0)
+    mf = H.gpu_offline(hos, p, o, M, 16, 10 ** 7, cm, 0, multifit_steps=steps)
+    assert (mf["makespan_est"] <= plain["makespan_est"]).all()
+    assert ((mf["makespan_est"] < plain["makespan_est"]) == (mf["packer"] == 1)).all()
+
+
+def test_multifit_on_the_configs(hos):
+    for name, count in (("c0", 1), ("c1", 1), ("c2", 100), ("c4", 6)):
+        w = workload(name).subset(0, count)
+        p, o = w.lengths()
+        H.check_offline(hos, p, o, w.n_clients, w.batch_cap, w.kv_budget, w.cost_model, min(w.ls_rounds, 30) or 10,
+                        multifit_steps=64)
+    # an invalid instance keeps its zeros and does not disturb its neighbour
+    w = workload("c0")
+    p, o = w.lengths()
+    p2 = np.concatenate([p, p]); o2 = np.concatenate([o, o]).copy(); o2[0, 3] = 0
+    g = H.gpu_offline(hos, p2, o2, w.n_clients, w.batch_cap, w.kv_budget, w.cost_model, 5, multifit_steps=64)
+    e = ora.offline_pack(p[0], o[0], w.n_clients, w.cost_model, 5, multifit_steps=64)
+    assert g["status"].tolist() == [hos.HOS_ST_INVALID, 0] and g["packer"][0] == 0
+    assert np.array_equal(g["assign"][1], e["assign"]) and (g["assign"][0] == -1).all()
