@@ -193,8 +193,7 @@ int offline_pack_impl(const hos_batch* b, const hos_cost_model* cm, int multifit
     const OfflineWs w = carve_offline(b, ws, 1, ls_rounds);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const int n_pad = pad4(b->n_req);
-    if ((rc = cuda_rc(launch_estimate_sort(*b, *cm, w.T_sorted, w.order, w.info, status, n_pad, st)))) return rc;
-    if (lb && (rc = cuda_rc(launch_lower_bound(*b, *cm, w.T_sorted, w.info, n_pad, lb, status, st)))) return rc;
+    if ((rc = cuda_rc(launch_estimate_sort(*b, *cm, w.T_sorted, w.order, w.info, status, lb, n_pad, st)))) return rc;
     if ((rc = cuda_rc(launch_lpt(*b, w.T_sorted, w.order, w.info, n_pad, assign,
                                  reinterpret_cast<long long*>(load),
                                  reinterpret_cast<long long*>(makespan_est), w.ls_C, st))))
@@ -247,7 +246,7 @@ int hos_local_search(const hos_batch* b, const hos_cost_model* cm, int n_copies,
     const OfflineWs w = carve_offline(b, ws, n_copies, ls_rounds);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const int n_pad = pad4(b->n_req);
-    if ((rc = cuda_rc(launch_estimate_sort(*b, *cm, w.T_sorted, w.order, w.info, status, n_pad, st)))) return rc;
+    if ((rc = cuda_rc(launch_estimate_sort(*b, *cm, w.T_sorted, w.order, w.info, status, nullptr, n_pad, st)))) return rc;
     return cuda_rc(launch_local_search(*b, w.T_sorted, w.order, w.info, n_pad, n_copies, ls_rounds, true,
                                        assign, reinterpret_cast<long long*>(load),
                                        reinterpret_cast<long long*>(makespan_est), rounds_applied,
@@ -266,8 +265,7 @@ int hos_lower_bound(const hos_batch* b, const hos_cost_model* cm, hos_lb* out, i
     const OfflineWs w = carve_offline(b, ws, 1, 0);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const int n_pad = pad4(b->n_req);
-    if ((rc = cuda_rc(launch_estimate_sort(*b, *cm, w.T_sorted, w.order, w.info, status, n_pad, st)))) return rc;
-    return cuda_rc(launch_lower_bound(*b, *cm, w.T_sorted, w.info, n_pad, out, status, st));
+    return cuda_rc(launch_estimate_sort(*b, *cm, w.T_sorted, w.order, w.info, status, out, n_pad, st));
 }
 
 int hos_online_simulate(const hos_batch* b, const int32_t* assign, const hos_cost_model* cm,

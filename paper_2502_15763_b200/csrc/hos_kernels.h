@@ -23,7 +23,7 @@ size_t local_search_smem(int n_req, int n_clients);
 size_t queue_build_smem(int n_req);
 
 cudaError_t launch_estimate_sort(const hos_batch& b, const hos_cost_model& cm, uint32_t* T_sorted,
-                                 uint32_t* order, InstInfo* info, int32_t* status_out, int n_pad,
+                                 uint32_t* order, InstInfo* info, int32_t* status_out, hos_lb* lb_out, int n_pad,
                                  cudaStream_t st);
 cudaError_t launch_lpt(const hos_batch& b, const uint32_t* T_sorted, const uint32_t* order,
                        const InstInfo* info, int n_pad, int32_t* assign, long long* load,
@@ -38,9 +38,6 @@ cudaError_t launch_local_search(const hos_batch& b, const uint32_t* T_sorted, co
                                 int32_t* status, uint32_t* ws_T, void* ws_I, uint8_t* ws_C, int32_t* ws_off,
                                 int32_t* ws_bad, cudaStream_t st);
 size_t local_search_index_bytes(int n_req);
-cudaError_t launch_lower_bound(const hos_batch& b, const hos_cost_model& cm, const uint32_t* T_sorted,
-                               const InstInfo* info, int n_pad, hos_lb* out, int32_t* status, cudaStream_t st);
-
 cudaError_t launch_queue_build(const hos_batch& b, const int32_t* assign, uint32_t p_max, int queue_order, uint2* q_po,
                                uint32_t* q_key, uint32_t* q_req, int32_t* q_off, unsigned long long* inst_O,
                                int32_t* inst_status, int n_pad, cudaStream_t st);

@@ -3,7 +3,7 @@
 //   k_lpt            longest-first list scheduling, one warp per instance
 //   k_ls_lists       the clients' member lists for the local search
 //   k_local_search   rounds of best move / pairwise swap off the critical client
-//   k_lower_bound    Eq. 31-32 and the packing relaxations
+//   (the lower bounds of Eq. 31-32 ride in k_estimate_sort's load pass)
 #include "hos_common.cuh"
 #include "hos_kernels.h"
 #include "hos_sort.cuh"
@@ -13,58 +13,197 @@
 namespace hos {
 
 // ---------------------------------------------------------------------------------------
-// Estimate + segmented sort.  One CTA per instance; the whole segment lives in shared
-// memory: the T table, two id buffers and the radix counters.
+// Lower bounds (Eq. 31-32 and the packing relaxations): the sums over an instance's requests
+// are taken in the load pass of the estimate + sort kernel, which reads p and o anyway, and
+// one thread finishes them once the sorted table gives T_(M) and T_(M+1).
 // ---------------------------------------------------------------------------------------
-template <typename IdxT>
+__device__ __forceinline__ unsigned long long floor_sum_below(uint32_t n, uint32_t q, int q_shift) {
+    // sum over x in [0, n) of floor(x / q); n and q fit 32 bits, so one 32-bit division does
+    // (a shift when q = 2^q_shift, q_shift >= 0)
+    const uint32_t m = q_shift >= 0 ? n >> q_shift : n / q, r = n - m * q;
+    return (unsigned long long)q * (((unsigned long long)m * (m - 1u + (m == 0u))) >> 1) +
+           (unsigned long long)m * r;                           // m = 0 -> 0
+}
+
+struct LbSums {
+    unsigned long long P, O, K, chain;      // sum p, sum o, sum of KV tokens attended, longest request alone
+};
+
+// a valid instance has p + o <= kv_budget < 2^31
+__device__ __forceinline__ void lb_take(LbSums& a, const hos_cost_model& cm, int q_shift, uint32_t pp, uint32_t oo) {
+    a.P += pp;
+    a.O += oo;
+    a.K += (unsigned long long)oo * pp + (((unsigned long long)oo * (oo - 1u)) >> 1);
+    const unsigned long long alone = (unsigned long long)prefill_us(cm, pp) +
+                                     oo * ((unsigned long long)cm.decode_fixed_us + cm.decode_per_seq_us) +
+                                     floor_sum_below(pp + oo, cm.decode_kv_div, q_shift) -
+                                     floor_sum_below(pp, cm.decode_kv_div, q_shift);
+    a.chain = alone > a.chain ? alone : a.chain;
+}
+
+// One thread: the bounds of an instance from its sums.  pairT = T_(M) + T_(M+1), 0 when n_req <= M.
+__device__ inline void lb_finish(const LbSums& a, const hos_cost_model& cm, int n_req, int n_clients, int cap,
+                                 unsigned long long sumT, unsigned long long maxT, unsigned long long pairT,
+                                 hos_lb* out, int32_t* status_word) {
+    const unsigned long long ad = cm.decode_fixed_us, bd = cm.decode_per_seq_us, q = cm.decode_kv_div;
+    const unsigned long long M = (unsigned long long)n_clients, C = (unsigned long long)cap;
+    hos_lb r;
+    unsigned long long lb = (sumT + M - 1ull) / M;
+    lb = maxT > lb ? maxT : lb;
+    lb = pairT > lb ? pairT : lb;
+    const unsigned long long n_pre = ((unsigned long long)n_req + C - 1ull) / C;
+    const unsigned long long n_dec = (a.O + C - 1ull) / C;
+    // Scaled sums in 128 bits: coefficients and sums that are each inside their limits can still
+    // carry these products past 64 bits, and a bound that does not fit is flagged, not wrapped.
+    typedef unsigned __int128 u128;
+    const u128 lim = (u128)0x7FFFFFFFFFFFFFFFull;
+    u128 tp_wide, tp_paper_wide = 0;
+    if (cm.n_levels == 0) {
+        tp_wide = (u128)cm.prefill_fixed_us * n_pre + (u128)cm.prefill_per_token_us * a.P;
+    } else {
+        // at least n_pre stages of at least the smallest level's time; a stage of level l carries
+        // at most N^cap_l tokens, so P tokens cost at least min_l floor(P / N^cap_l) T^p_l
+        const u128 by_count = (u128)cm.level_time_us[0] * n_pre;
+        u128 by_tokens = ~(u128)0;
+        for (uint32_t l = 0; l < cm.n_levels; ++l) {
+            const u128 v = (u128)(a.P / cm.level_cap_tokens[l]) * cm.level_time_us[l];
+            by_tokens = v < by_tokens ? v : by_tokens;
+        }
+        tp_wide = by_count > by_tokens ? by_count : by_tokens;
+        tp_paper_wide = (u128)(a.P / cm.level_cap_tokens[cm.n_levels - 1]) * cm.level_time_us[cm.n_levels - 1];
+    }
+    const u128 td_q = (u128)q * ((u128)(ad - 1ull) * n_dec + (u128)bd * a.O) + a.K;
+    const u128 tot_q = (u128)q * tp_wide + td_q + (u128)(q * M - 1ull);
+    if (tp_wide > lim || tp_paper_wide > lim || td_q > lim || tot_q > lim) {
+        *out = hos_lb{0, 0, 0, 0, 0, 0, 0, 0, 0};
+        if (status_word) *status_word |= HOS_ST_RANGE;
+        return;
+    }
+    const unsigned long long tp_star = (unsigned long long)tp_wide;
+    const unsigned long long td_q64 = (unsigned long long)td_q;
+    const unsigned long long work = (unsigned long long)tot_q / (q * M);
+    r.tp_paper_us = (long long)(unsigned long long)tp_paper_wide;
+    r.lb_pack = (long long)lb; r.sum_T = (long long)sumT; r.max_T = (long long)maxT; r.pair_T = (long long)pairT;
+    r.tp_star_us = (long long)((tp_star + M - 1ull) / M);
+    r.td_star_us = (long long)((td_q64 + q * M - 1ull) / (q * M));
+    r.chain_us = (long long)a.chain;
+    r.lb_sim_us = (long long)(work > a.chain ? work : a.chain);
+    *out = r;
+}
+
+// ---------------------------------------------------------------------------------------
+// Estimate + segmented sort (+ the lower bounds' sums).  One CTA per instance; the T table lives
+// in shared memory.  FAST: the bucket sort, one CTA per instance; when it declines an instance
+// (keys too wide or too bunched) it leaves SORT_PENDING in the instance's workspace status and
+// the second launch of this kernel, !FAST, a few persistent CTAs with the radix sort's larger
+// shared memory, takes exactly those instances.
+// ---------------------------------------------------------------------------------------
+constexpr int SORT_PENDING = 0x100;        // internal bit of InstInfo::status
+
+template <bool FAST>
 __global__ void __launch_bounds__(SORT_THREADS, 1)
 k_estimate_sort(const uint32_t* __restrict__ p, const uint32_t* __restrict__ o,
-                const uint32_t* __restrict__ o_est, int n_req,
-                long long kv_budget, uint32_t e_p, uint32_t e_o, uint32_t p_max,
+                const uint32_t* __restrict__ o_est, int n_inst, int n_req,
+                long long kv_budget, uint32_t p_max, hos_cost_model cm, int q_shift, int n_clients, int cap,
                 uint32_t* __restrict__ T_sorted, uint32_t* __restrict__ order,
-                InstInfo* __restrict__ info, int32_t* __restrict__ status_out, int n_pad) {
+                InstInfo* __restrict__ info, int32_t* __restrict__ status_out, hos_lb* __restrict__ lb_out,
+                int n_pad) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     __shared__ unsigned long long red[32];
-    SortSmem<IdxT> s = sort_smem_carve<IdxT>(smem_raw, n_req);
-    const int inst = blockIdx.x;
-    const uint32_t* pi = p + (size_t)inst * n_req;
-    const uint32_t* oi = o + (size_t)inst * n_req;
-    const uint32_t* ei = o_est ? o_est + (size_t)inst * n_req : oi;   // the lengths the scheduler knows
+    uint32_t* key = reinterpret_cast<uint32_t*>(smem_raw);
+    const uint32_t e_p = cm.est_per_prompt_token, e_o = cm.est_per_output_token;
+    for (int inst = blockIdx.x; inst < n_inst; inst += gridDim.x) {
+        if (!FAST) {
+            __syncthreads();                              // the instance before is finished with shared memory
+            if (!(info[inst].status & SORT_PENDING)) continue;      // uniform: one word read by every thread
+        }
+        const uint32_t* pi = p + (size_t)inst * n_req;
+        const uint32_t* oi = o + (size_t)inst * n_req;
+        const uint32_t* ei = o_est ? o_est + (size_t)inst * n_req : oi;   // the lengths the scheduler knows
 
-    // kv_budget here is the most KV one request may need: the fixed reservation, if there is one
-    unsigned long long sum = 0, mx = 0, bad = 0;
-    for (int i = threadIdx.x; i < n_req; i += SORT_THREADS) {
-        const uint32_t pp = pi[i], oo = oi[i], oe = ei[i];
-        const unsigned long long t = (unsigned long long)e_p * pp + (unsigned long long)e_o * oe;
-        if (pp == 0 || oo == 0 || oe == 0 || pp > p_max || (long long)pp + (long long)oo > kv_budget ||
-            t > 0xFFFFFFFFull)
-            bad = 1;
-        s.key[i] = (uint32_t)t;
-        sum += t;
-        mx = t > mx ? t : mx;
-    }
-    sum = block_sum_u64(sum, red);
-    mx = block_max_u64(mx, red);
-    bad = block_max_u64(bad, red);
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        info[inst].sum_T = sum;
-        info[inst].max_T = (uint32_t)mx;
-        info[inst].status = bad ? HOS_ST_INVALID : 0;
-        if (status_out) status_out[inst] = bad ? HOS_ST_INVALID : 0;
-    }
-    if (bad) return;                                  // uniform: every thread sees the same value
-
-    const int nbits = bit_width_u32((uint32_t)mx);
-    const uint32_t flip = nbits >= 32 ? 0xFFFFFFFFu : ((1u << nbits) - 1u);   // descending T
-    const IdxT* sorted = block_radix_sort_ids<IdxT>(s, n_req, nbits, flip);
-
-    uint32_t* Ts = T_sorted + (size_t)inst * n_pad;
-    uint32_t* od = order + (size_t)inst * n_pad;
-    for (int r = threadIdx.x; r < n_req; r += SORT_THREADS) {
-        const uint32_t id = sorted[r];
-        od[r] = id;
-        Ts[r] = s.key[id];
+        // kv_budget here is the most KV one request may need: the fixed reservation, if there is one
+        unsigned long long sum = 0, mx = 0, bad = 0;
+        LbSums a = {0ull, 0ull, 0ull, 0ull};
+        auto take = [&](int i, uint32_t pp, uint32_t oo, uint32_t oe) {
+            const unsigned long long t = (unsigned long long)e_p * pp + (unsigned long long)e_o * oe;
+            if (pp == 0 || oo == 0 || oe == 0 || pp > p_max || (long long)pp + (long long)oo > kv_budget ||
+                t > 0xFFFFFFFFull)
+                bad = 1;
+            else if (lb_out) lb_take(a, cm, q_shift, pp, oo);
+            key[i] = (uint32_t)t;
+            sum += t;
+            mx = t > mx ? t : mx;
+        };
+        // four requests per thread and read when the rows allow 16-byte loads
+        const bool vec = (n_req & 3) == 0 && ((reinterpret_cast<uintptr_t>(pi) | reinterpret_cast<uintptr_t>(oi) |
+                                               reinterpret_cast<uintptr_t>(ei)) & 15) == 0;
+        if (vec) {
+            const uint4* p4 = reinterpret_cast<const uint4*>(pi);
+            const uint4* o4 = reinterpret_cast<const uint4*>(oi);
+            const uint4* e4 = reinterpret_cast<const uint4*>(ei);
+            for (int i4 = threadIdx.x; i4 < (n_req >> 2); i4 += SORT_THREADS) {
+                const uint4 pv = __ldg(&p4[i4]), ov = __ldg(&o4[i4]);
+                const uint4 ev = o_est ? __ldg(&e4[i4]) : ov;
+                take(4 * i4 + 0, pv.x, ov.x, ev.x);
+                take(4 * i4 + 1, pv.y, ov.y, ev.y);
+                take(4 * i4 + 2, pv.z, ov.z, ev.z);
+                take(4 * i4 + 3, pv.w, ov.w, ev.w);
+            }
+        } else {
+            for (int i = threadIdx.x; i < n_req; i += SORT_THREADS) take(i, pi[i], oi[i], ei[i]);
+        }
+        sum = block_sum_u64(sum, red);
+        mx = block_max_u64(mx, red);
+        bad = block_max_u64(bad, red);
+        if (lb_out && !bad) {
+            a.P = block_sum_u64(a.P, red);
+            a.O = block_sum_u64(a.O, red);
+            a.K = block_sum_u64(a.K, red);
+            a.chain = block_max_u64(a.chain, red);
+        }
+        __syncthreads();
+        if (bad) {                                        // uniform: every thread sees the same value
+            if (threadIdx.x == 0) {
+                info[inst].sum_T = sum; info[inst].max_T = (uint32_t)mx; info[inst].status = HOS_ST_INVALID;
+                if (status_out) status_out[inst] = HOS_ST_INVALID;
+                if (lb_out) lb_out[inst] = hos_lb{0, 0, 0, 0, 0, 0, 0, 0, 0};
+            }
+            continue;
+        }
+        const int nbits = bit_width_u32((uint32_t)mx);
+        const uint32_t flip = nbits >= 32 ? 0xFFFFFFFFu : ((1u << nbits) - 1u);   // descending T
+        uint32_t* Ts = T_sorted + (size_t)inst * n_pad;
+        uint32_t* od = order + (size_t)inst * n_pad;
+        unsigned long long pairT = 0;
+        if (FAST) {
+            uint32_t* ent = reinterpret_cast<uint32_t*>(smem_raw + align16((size_t)n_req * 4));
+            uint32_t* cnt = reinterpret_cast<uint32_t*>(smem_raw + 2 * align16((size_t)n_req * 4));
+            if (!block_bucket_sort(key, ent, cnt, n_req, nbits, flip)) {
+                if (threadIdx.x == 0) info[inst].status = SORT_PENDING;
+                continue;
+            }
+            for (int r = threadIdx.x; r < n_req; r += SORT_THREADS) {
+                const uint32_t id = ent[r];
+                od[r] = id;
+                Ts[r] = key[id];
+            }
+            if (n_req > n_clients) pairT = (unsigned long long)key[ent[n_clients - 1]] + key[ent[n_clients]];
+        } else {
+            SortSmem<uint16_t> s = sort_smem_carve<uint16_t>(smem_raw, n_req);
+            const uint16_t* sorted = block_radix_sort_ids<uint16_t>(s, n_req, nbits, flip);
+            for (int r = threadIdx.x; r < n_req; r += SORT_THREADS) {
+                const uint32_t id = sorted[r];
+                od[r] = id;
+                Ts[r] = key[id];
+            }
+            if (n_req > n_clients) pairT = (unsigned long long)key[sorted[n_clients - 1]] + key[sorted[n_clients]];
+        }
+        if (threadIdx.x == 0) {
+            int32_t st = 0;
+            if (lb_out) lb_finish(a, cm, n_req, n_clients, cap, sum, mx, pairT, &lb_out[inst], &st);
+            info[inst].sum_T = sum; info[inst].max_T = (uint32_t)mx; info[inst].status = 0;
+            if (status_out) status_out[inst] = st;
+        }
     }
 }
 
@@ -1162,133 +1301,37 @@ k_local_search(const uint32_t* __restrict__ T_sorted, const uint32_t* __restrict
 }
 
 // ---------------------------------------------------------------------------------------
-// Lower bounds.  One CTA per instance; reads p, o once, and T_(M), T_(M+1) from the sorted
-// table left by k_estimate_sort.
-// ---------------------------------------------------------------------------------------
-__device__ __forceinline__ unsigned long long floor_sum_below(uint32_t n, uint32_t q, int q_shift) {
-    // sum over x in [0, n) of floor(x / q); n and q fit 32 bits, so one 32-bit division does
-    // (a shift when q = 2^q_shift, q_shift >= 0)
-    const uint32_t m = q_shift >= 0 ? n >> q_shift : n / q, r = n - m * q;
-    return (unsigned long long)q * (((unsigned long long)m * (m - 1u + (m == 0u))) >> 1) +
-           (unsigned long long)m * r;                           // m = 0 -> 0
-}
-
-__global__ void __launch_bounds__(256)
-k_lower_bound(const uint32_t* __restrict__ p, const uint32_t* __restrict__ o, int n_req, int n_pad,
-              int n_clients, int cap, hos_cost_model cm, int q_shift, const uint32_t* __restrict__ T_sorted,
-              const InstInfo* __restrict__ info, hos_lb* __restrict__ out, int32_t* __restrict__ status_out) {
-    __shared__ unsigned long long red[32];
-    const int inst = blockIdx.x;
-    const InstInfo inf = info[inst];
-    if (inf.status) {
-        if (threadIdx.x == 0) out[inst] = hos_lb{0, 0, 0, 0, 0, 0, 0, 0, 0};
-        return;
-    }
-    const uint32_t* pi = p + (size_t)inst * n_req;
-    const uint32_t* oi = o + (size_t)inst * n_req;
-    const unsigned long long ad = cm.decode_fixed_us, bd = cm.decode_per_seq_us, q = cm.decode_kv_div;
-    unsigned long long P = 0, O = 0, K = 0, chain = 0;
-    // a valid instance has p + o <= kv_budget < 2^31
-    auto take = [&](uint32_t pp, uint32_t oo) {
-        P += pp;
-        O += oo;
-        K += (unsigned long long)oo * pp + (((unsigned long long)oo * (oo - 1u)) >> 1);
-        const unsigned long long alone = (unsigned long long)prefill_us(cm, pp) + oo * (ad + bd) +
-                                         floor_sum_below(pp + oo, cm.decode_kv_div, q_shift) -
-                                         floor_sum_below(pp, cm.decode_kv_div, q_shift);
-        chain = alone > chain ? alone : chain;
-    };
-    constexpr int UN = 4;                                       // reads in flight per thread and table
-    int i = threadIdx.x;
-    for (; i + (UN - 1) * (int)blockDim.x < n_req; i += UN * blockDim.x) {
-        uint32_t pp[UN], oo[UN];
-#pragma unroll
-        for (int u = 0; u < UN; ++u) { pp[u] = pi[i + u * blockDim.x]; oo[u] = oi[i + u * blockDim.x]; }
-#pragma unroll
-        for (int u = 0; u < UN; ++u) take(pp[u], oo[u]);
-    }
-    for (; i < n_req; i += blockDim.x) take(pi[i], oi[i]);
-    P = block_sum_u64(P, red);
-    O = block_sum_u64(O, red);
-    K = block_sum_u64(K, red);
-    chain = block_max_u64(chain, red);
-    if (threadIdx.x == 0) {
-        const unsigned long long M = (unsigned long long)n_clients, C = (unsigned long long)cap;
-        hos_lb r;
-        const unsigned long long sumT = inf.sum_T, maxT = inf.max_T;
-        unsigned long long pairT = 0;
-        if (n_req > n_clients) {
-            const uint32_t* Ts = T_sorted + (size_t)inst * n_pad;
-            pairT = (unsigned long long)Ts[n_clients - 1] + (unsigned long long)Ts[n_clients];
-        }
-        unsigned long long lb = (sumT + M - 1ull) / M;
-        lb = maxT > lb ? maxT : lb;
-        lb = pairT > lb ? pairT : lb;
-        const unsigned long long n_pre = ((unsigned long long)n_req + C - 1ull) / C;
-        const unsigned long long n_dec = (O + C - 1ull) / C;
-        // Scaled sums in 128 bits: coefficients and sums that are each inside their limits can still
-        // carry these products past 64 bits, and a bound that does not fit is flagged, not wrapped.
-        typedef unsigned __int128 u128;
-        const u128 lim = (u128)0x7FFFFFFFFFFFFFFFull;
-        u128 tp_wide, tp_paper_wide = 0;
-        if (cm.n_levels == 0) {
-            tp_wide = (u128)cm.prefill_fixed_us * n_pre + (u128)cm.prefill_per_token_us * P;
-        } else {
-            // at least n_pre stages of at least the smallest level's time; a stage of level l carries
-            // at most N^cap_l tokens, so P tokens cost at least min_l floor(P / N^cap_l) T^p_l
-            const u128 by_count = (u128)cm.level_time_us[0] * n_pre;
-            u128 by_tokens = ~(u128)0;
-            for (uint32_t l = 0; l < cm.n_levels; ++l) {
-                const u128 v = (u128)(P / cm.level_cap_tokens[l]) * cm.level_time_us[l];
-                by_tokens = v < by_tokens ? v : by_tokens;
-            }
-            tp_wide = by_count > by_tokens ? by_count : by_tokens;
-            tp_paper_wide = (u128)(P / cm.level_cap_tokens[cm.n_levels - 1]) * cm.level_time_us[cm.n_levels - 1];
-        }
-        const u128 td_q = (u128)q * ((u128)(ad - 1ull) * n_dec + (u128)bd * O) + K;
-        const u128 tot_q = (u128)q * tp_wide + td_q + (u128)(q * M - 1ull);
-        if (tp_wide > lim || tp_paper_wide > lim || td_q > lim || tot_q > lim) {
-            out[inst] = hos_lb{0, 0, 0, 0, 0, 0, 0, 0, 0};
-            if (status_out) atomicOr(&status_out[inst], HOS_ST_RANGE);
-            return;
-        }
-        const unsigned long long tp_star = (unsigned long long)tp_wide;
-        r.tp_paper_us = (long long)(unsigned long long)tp_paper_wide;
-        const unsigned long long td_q64 = (unsigned long long)td_q;
-        const unsigned long long work = (unsigned long long)tot_q / (q * M);
-        r.lb_pack = (long long)lb; r.sum_T = (long long)sumT; r.max_T = (long long)maxT; r.pair_T = (long long)pairT;
-        r.tp_star_us = (long long)((tp_star + M - 1ull) / M);
-        r.td_star_us = (long long)((td_q64 + q * M - 1ull) / (q * M));
-        r.chain_us = (long long)chain;
-        r.lb_sim_us = (long long)(work > chain ? work : chain);
-        out[inst] = r;
-    }
-}
-
-// ---------------------------------------------------------------------------------------
 // launchers
 // ---------------------------------------------------------------------------------------
 
-size_t estimate_sort_smem(int n_req) {
-    return n_req <= 65536 ? sort_smem_bytes<uint16_t>(n_req) : sort_smem_bytes<uint32_t>(n_req);
-}
+size_t estimate_sort_smem(int n_req) { return sort_smem_bytes<uint16_t>(n_req); }
 size_t local_search_smem(int /*n_req*/, int n_clients) { return (size_t)n_clients * (LS_WARPS + 1) * 4; }
 size_t local_search_index_bytes(int n_req) { return n_req <= 65536 ? 2 : 4; }
 
 cudaError_t launch_estimate_sort(const hos_batch& b, const hos_cost_model& cm, uint32_t* T_sorted,
-                                 uint32_t* order, InstInfo* info, int32_t* status_out, int n_pad,
+                                 uint32_t* order, InstInfo* info, int32_t* status_out, hos_lb* lb_out, int n_pad,
                                  cudaStream_t st) {
-    const size_t smem = estimate_sort_smem(b.n_req);
-    auto kern = b.n_req <= 65536 ? k_estimate_sort<uint16_t> : k_estimate_sort<uint32_t>;
-    cudaError_t e = allow_max_dynamic_smem(reinterpret_cast<const void*>(kern));
+    cudaError_t e = allow_max_dynamic_smem(reinterpret_cast<const void*>(k_estimate_sort<true>));
     if (e != cudaSuccess) return e;
+    if ((e = allow_max_dynamic_smem(reinterpret_cast<const void*>(k_estimate_sort<false>))) != cudaSuccess) return e;
+    int q_shift = -1;                                    // power-of-two KV divisor -> shift
+    if ((cm.decode_kv_div & (cm.decode_kv_div - 1)) == 0)
+        for (q_shift = 0; (1u << q_shift) != cm.decode_kv_div; ++q_shift) {}
+    const long long most = b.kv_reserve_tokens ? (long long)b.kv_reserve_tokens : (long long)b.kv_budget;
     launch_hook("k_estimate_sort", 0, st);
-    kern<<<b.n_inst, SORT_THREADS, smem, st>>>(b.p, b.o, b.o_est, b.n_req,
-                                               b.kv_reserve_tokens ? (long long)b.kv_reserve_tokens
-                                                                   : (long long)b.kv_budget,
-                                               cm.est_per_prompt_token, cm.est_per_output_token, stage_cap_tokens(cm),
-                                               T_sorted, order, info, status_out, n_pad);
+    k_estimate_sort<true><<<b.n_inst, SORT_THREADS, bucket_sort_smem_bytes(b.n_req), st>>>(
+        b.p, b.o, b.o_est, b.n_inst, b.n_req, most, stage_cap_tokens(cm), cm, q_shift, b.n_clients, b.batch_cap,
+        T_sorted, order, info, status_out, lb_out, n_pad);
     launch_hook("k_estimate_sort", 1, st);
+    // the instances the bucket sort declined (none, as a rule): one CTA per SM at most, each
+    // walking the batch for pending instances
+    int n_sm = 148, dev = 0;
+    if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev);
+    launch_hook("k_estimate_sort_radix", 0, st);
+    k_estimate_sort<false><<<b.n_inst < n_sm ? b.n_inst : n_sm, SORT_THREADS, estimate_sort_smem(b.n_req), st>>>(
+        b.p, b.o, b.o_est, b.n_inst, b.n_req, most, stage_cap_tokens(cm), cm, q_shift, b.n_clients, b.batch_cap,
+        T_sorted, order, info, status_out, lb_out, n_pad);
+    launch_hook("k_estimate_sort_radix", 1, st);
     return cudaGetLastError();
 }
 
@@ -1351,18 +1394,6 @@ cudaError_t launch_local_search(const hos_batch& b, const uint32_t* T_sorted, co
     }
 #undef HOS_LS
     launch_hook("k_local_search", 1, st);
-    return cudaGetLastError();
-}
-
-cudaError_t launch_lower_bound(const hos_batch& b, const hos_cost_model& cm, const uint32_t* T_sorted,
-                               const InstInfo* info, int n_pad, hos_lb* out, int32_t* status, cudaStream_t st) {
-    int q_shift = -1;                                    // power-of-two KV divisor -> shift
-    if ((cm.decode_kv_div & (cm.decode_kv_div - 1)) == 0)
-        for (q_shift = 0; (1u << q_shift) != cm.decode_kv_div; ++q_shift) {}
-    launch_hook("k_lower_bound", 0, st);
-    k_lower_bound<<<b.n_inst, 256, 0, st>>>(b.p, b.o, b.n_req, n_pad, b.n_clients, b.batch_cap, cm, q_shift,
-                                            T_sorted, info, out, status);
-    launch_hook("k_lower_bound", 1, st);
     return cudaGetLastError();
 }
 

@@ -18,92 +18,129 @@ constexpr int INST_WIDE = 0x100;         // internal flag in the workspace's per
 // N^p + N^d descending, index ascending) -- one stable radix sort on the composite key
 // client << kb | (2^kb - 1 - (p + o)).  HOS_QUEUE_FCFS sorts by client only.
 // ---------------------------------------------------------------------------------------
-template <typename IdxT>
+// FAST: the bucket sort, one CTA per instance; an instance it declines keeps INST_PENDING in its
+// status word and the second launch (!FAST, persistent CTAs, radix sort) takes it.
+constexpr int INST_PENDING = 0x200;      // internal flag: queues not built yet
+
+template <bool FAST>
 __global__ void __launch_bounds__(SORT_THREADS, 1)
 k_queue_build(const uint32_t* __restrict__ p, const uint32_t* __restrict__ o,
               const uint32_t* __restrict__ o_est,
-              const int32_t* __restrict__ assign, int n_req, int n_clients, long long kv_budget,
+              const int32_t* __restrict__ assign, int n_inst, int n_req, int n_clients, long long kv_budget,
               uint32_t p_max, int queue_order, uint2* __restrict__ q_po, uint32_t* __restrict__ q_key,
               uint32_t* __restrict__ q_req,
               int32_t* __restrict__ q_off, unsigned long long* __restrict__ inst_O,
               int32_t* __restrict__ inst_status, int n_pad) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     __shared__ unsigned long long red[32];
-    SortSmem<IdxT> s = sort_smem_carve<IdxT>(smem_raw, n_req);
-    const int inst = blockIdx.x;
-    const uint32_t* pi = p + (size_t)inst * n_req;
-    const uint32_t* oi = o + (size_t)inst * n_req;
-    const int32_t* ai = assign + (size_t)inst * n_req;
-    const uint32_t* ei = o_est ? o_est + (size_t)inst * n_req : oi;   // the lengths the scheduler sorts by
+    uint32_t* key = reinterpret_cast<uint32_t*>(smem_raw);
+    // the clients wait here until the keys are composed (the sort's own buffer, not yet in use)
+    uint32_t* park = reinterpret_cast<uint32_t*>(smem_raw + align16((size_t)n_req * 4));
+    for (int inst = blockIdx.x; inst < n_inst; inst += gridDim.x) {
+        if (!FAST) {
+            __syncthreads();
+            if (!(inst_status[inst] & INST_PENDING)) continue;    // uniform
+        }
+        const uint32_t* pi = p + (size_t)inst * n_req;
+        const uint32_t* oi = o + (size_t)inst * n_req;
+        const int32_t* ai = assign + (size_t)inst * n_req;
+        const uint32_t* ei = o_est ? o_est + (size_t)inst * n_req : oi;   // the lengths the scheduler sorts by
 
-    // kv_budget here is the most KV one request may need: the fixed reservation, if there is one
-    unsigned long long sumO = 0, mx = 0, mxk = 0, mxp = 0, bad = 0;
-    for (int i = threadIdx.x; i < n_req; i += SORT_THREADS) {
-        const uint32_t pp = pi[i], oo = oi[i], oe = ei[i];
-        const int c = ai[i];
-        const unsigned long long tot = (unsigned long long)pp + oo;
-        const unsigned long long totk = (unsigned long long)pp + oe;
-        if (pp == 0 || oo == 0 || oe == 0 || pp > p_max || (long long)tot > kv_budget || totk > 0xFFFFFFFFull ||
-            c < 0 || c >= n_clients)
-            bad = 1;
-        s.key[i] = (uint32_t)totk;
-        s.buf1[i] = (IdxT)(c & 0xFF);                 // parked until the keys are composed
-        sumO += oo;
-        mx = tot > mx ? tot : mx;
-        mxk = totk > mxk ? totk : mxk;
-        mxp = pp > mxp ? pp : mxp;
-    }
-    sumO = block_sum_u64(sumO, red);
-    mx = block_max_u64(mx, red);
-    mxk = block_max_u64(mxk, red);
-    mxp = block_max_u64(mxp, red);
-    bad = block_max_u64(bad, red);
-    __syncthreads();
-    const int kb = (queue_order == HOS_QUEUE_SORTED) ? bit_width_u32((uint32_t)mxk) : 0;
-    // the composite sort key, client above p + (estimated) o, has 32 bits: an estimate so long
-    // that it does not fit beside the client bits invalidates the instance (uniform over the CTA)
-    if (kb + bit_width_u32((uint32_t)(n_clients - 1)) > 32) bad = 1;
-    if (threadIdx.x == 0) {
-        inst_O[inst] = sumO;
+        // kv_budget here is the most KV one request may need: the fixed reservation, if there is one
+        unsigned long long sumO = 0, mx = 0, mxk = 0, mxp = 0, bad = 0;
+        auto take = [&](int i, uint32_t pp, uint32_t oo, uint32_t oe, int c) {
+            const unsigned long long tot = (unsigned long long)pp + oo;
+            const unsigned long long totk = (unsigned long long)pp + oe;
+            if (pp == 0 || oo == 0 || oe == 0 || pp > p_max || (long long)tot > kv_budget || totk > 0xFFFFFFFFull ||
+                c < 0 || c >= n_clients)
+                bad = 1;
+            key[i] = (uint32_t)totk;
+            if (FAST) park[i] = (uint32_t)(c & 0xFF);
+            else reinterpret_cast<uint16_t*>(park)[i] = (uint16_t)(c & 0xFF);
+            sumO += oo;
+            mx = tot > mx ? tot : mx;
+            mxk = totk > mxk ? totk : mxk;
+            mxp = pp > mxp ? pp : mxp;
+        };
+        const bool vec = (n_req & 3) == 0 && ((reinterpret_cast<uintptr_t>(pi) | reinterpret_cast<uintptr_t>(oi) |
+                                               reinterpret_cast<uintptr_t>(ei) | reinterpret_cast<uintptr_t>(ai)) & 15) == 0;
+        if (vec) {
+            for (int i4 = threadIdx.x; i4 < (n_req >> 2); i4 += SORT_THREADS) {
+                const uint4 pv = __ldg(reinterpret_cast<const uint4*>(pi) + i4);
+                const uint4 ov = __ldg(reinterpret_cast<const uint4*>(oi) + i4);
+                const uint4 ev = o_est ? __ldg(reinterpret_cast<const uint4*>(ei) + i4) : ov;
+                const int4 av = __ldg(reinterpret_cast<const int4*>(ai) + i4);
+                take(4 * i4 + 0, pv.x, ov.x, ev.x, av.x);
+                take(4 * i4 + 1, pv.y, ov.y, ev.y, av.y);
+                take(4 * i4 + 2, pv.z, ov.z, ev.z, av.z);
+                take(4 * i4 + 3, pv.w, ov.w, ev.w, av.w);
+            }
+        } else {
+            for (int i = threadIdx.x; i < n_req; i += SORT_THREADS) take(i, pi[i], oi[i], ei[i], ai[i]);
+        }
+        sumO = block_sum_u64(sumO, red);
+        mx = block_max_u64(mx, red);
+        mxk = block_max_u64(mxk, red);
+        mxp = block_max_u64(mxp, red);
+        bad = block_max_u64(bad, red);
+        __syncthreads();
+        const int kb = (queue_order == HOS_QUEUE_SORTED) ? bit_width_u32((uint32_t)mxk) : 0;
+        // the composite sort key, client above p + (estimated) o, has 32 bits: an estimate so long
+        // that it does not fit beside the client bits invalidates the instance (uniform over the CTA)
+        if (kb + bit_width_u32((uint32_t)(n_clients - 1)) > 32) bad = 1;
         // bit 8 (internal): some p + o needs more than 16 bits -> the simulator's wide heap entries
-        inst_status[inst] = bad ? HOS_ST_INVALID : (mx >= 65536ull ? INST_WIDE : 0);
-    }
-    if (bad) return;
-
-    const uint32_t kmask = kb >= 32 ? 0xFFFFFFFFu : ((1u << kb) - 1u);
-    const int nbits = kb + bit_width_u32((uint32_t)(n_clients - 1));
-    // The sort only looks at the low nbits of a key.  When the prompt length fits the bits above
-    // them it rides along there, so that the queue entries are written without going back to the
-    // request tables in queue order (a scattered read per request); with the key p + o the
-    // output length follows from it too.
-    const bool ride = nbits + bit_width_u32((uint32_t)mxp) <= 32;
-    const bool o_from_key = ride && kb > 0 && kb < 32 && !o_est;
-    for (int i = threadIdx.x; i < n_req; i += SORT_THREADS) {
-        const uint32_t c = (uint32_t)s.buf1[i];
-        const uint32_t low = (kb >= 32 ? 0u : (c << kb)) | (kmask - (s.key[i] & kmask));
-        s.key[i] = ride ? (low | (nbits >= 32 ? 0u : (pi[i] << nbits))) : low;
-    }
-    __syncthreads();
-    const IdxT* sorted = block_radix_sort_ids<IdxT>(s, n_req, nbits, 0u);
-
-    uint2* qp = q_po + (size_t)inst * n_pad;
-    uint32_t* qr = q_req + (size_t)inst * n_pad;
-    int32_t* qo = q_off + (size_t)inst * (n_clients + 1);
-    for (int r = threadIdx.x; r < n_req; r += SORT_THREADS) {
-        const uint32_t id = sorted[r];
-        const uint32_t key = s.key[id];
-        const uint32_t low = (ride && nbits < 32) ? (key & ((1u << nbits) - 1u)) : key;
-        const uint32_t pp = (ride && nbits < 32) ? key >> nbits : pi[id];
-        const uint32_t totk = kmask - (low & kmask);             // p + (estimated) o, when it is the key
-        qr[r] = id;
-        qp[r] = make_uint2(pp, o_from_key ? totk - pp : oi[id]);
-        if (q_key) q_key[(size_t)inst * n_pad + r] = kb > 0 && kb < 32 ? totk : pp + ei[id];
-        const int c = kb >= 32 ? 0 : (int)(low >> kb);            // 32 key bits leave none for the client: one client
-        const uint32_t kprev = r > 0 ? s.key[sorted[r - 1]] : 0u;
-        const int cprev = r > 0 ? (kb >= 32 ? 0 : (int)(((ride && nbits < 32) ? (kprev & ((1u << nbits) - 1u)) : kprev) >> kb)) : -1;
-        for (int cc = cprev + 1; cc <= c; ++cc) qo[cc] = r;
-        if (r == n_req - 1)
-            for (int cc = c + 1; cc <= n_clients; ++cc) qo[cc] = n_req;
+        const int32_t st_done = bad ? HOS_ST_INVALID : (mx >= 65536ull ? INST_WIDE : 0);
+        if (bad) {
+            if (threadIdx.x == 0) { inst_O[inst] = sumO; inst_status[inst] = st_done; }
+            continue;
+        }
+        const uint32_t kmask = kb >= 32 ? 0xFFFFFFFFu : ((1u << kb) - 1u);
+        const int nbits = kb + bit_width_u32((uint32_t)(n_clients - 1));
+        // The sort only looks at the low nbits of a key.  When the prompt length fits the bits above
+        // them it rides along there, so that the queue entries are written without going back to the
+        // request tables in queue order (a scattered read per request); with the key p + o the
+        // output length follows from it too.
+        const bool ride = nbits + bit_width_u32((uint32_t)mxp) <= 32;
+        const bool o_from_key = ride && kb > 0 && kb < 32 && !o_est;
+        for (int i = threadIdx.x; i < n_req; i += SORT_THREADS) {
+            const uint32_t c = FAST ? park[i] : (uint32_t)reinterpret_cast<uint16_t*>(park)[i];
+            const uint32_t low = (kb >= 32 ? 0u : (c << kb)) | (kmask - (key[i] & kmask));
+            key[i] = ride ? (low | (nbits >= 32 ? 0u : (pi[i] << nbits))) : low;
+        }
+        __syncthreads();
+        uint2* qp = q_po + (size_t)inst * n_pad;
+        uint32_t* qr = q_req + (size_t)inst * n_pad;
+        int32_t* qo = q_off + (size_t)inst * (n_clients + 1);
+        auto write_out = [&](auto sorted) {
+            for (int r = threadIdx.x; r < n_req; r += SORT_THREADS) {
+                const uint32_t id = sorted[r];
+                const uint32_t kw = key[id];
+                const uint32_t low = (ride && nbits < 32) ? (kw & ((1u << nbits) - 1u)) : kw;
+                const uint32_t pp = (ride && nbits < 32) ? kw >> nbits : pi[id];
+                const uint32_t totk = kmask - (low & kmask);             // p + (estimated) o, when it is the key
+                qr[r] = id;
+                qp[r] = make_uint2(pp, o_from_key ? totk - pp : oi[id]);
+                if (q_key) q_key[(size_t)inst * n_pad + r] = kb > 0 && kb < 32 ? totk : pp + ei[id];
+                const int c = kb >= 32 ? 0 : (int)(low >> kb);            // 32 key bits leave none for the client: one client
+                const uint32_t kprev = r > 0 ? key[sorted[r - 1]] : 0u;
+                const int cprev = r > 0 ? (kb >= 32 ? 0 : (int)(((ride && nbits < 32) ? (kprev & ((1u << nbits) - 1u)) : kprev) >> kb)) : -1;
+                for (int cc = cprev + 1; cc <= c; ++cc) qo[cc] = r;
+                if (r == n_req - 1)
+                    for (int cc = c + 1; cc <= n_clients; ++cc) qo[cc] = n_req;
+            }
+        };
+        if (FAST) {
+            uint32_t* cnt = reinterpret_cast<uint32_t*>(smem_raw + 2 * align16((size_t)n_req * 4));
+            if (!block_bucket_sort(key, park, cnt, n_req, nbits, 0u)) {
+                if (threadIdx.x == 0) inst_status[inst] = INST_PENDING;
+                continue;
+            }
+            write_out(park);
+        } else {
+            SortSmem<uint16_t> s = sort_smem_carve<uint16_t>(smem_raw, n_req);
+            write_out(block_radix_sort_ids<uint16_t>(s, n_req, nbits, 0u));
+        }
+        if (threadIdx.x == 0) { inst_O[inst] = sumO; inst_status[inst] = st_done; }
     }
 }
 
@@ -934,24 +971,27 @@ static int sim_slots(const hos_batch& b) {
 }
 static uint32_t sim_budget(const hos_batch& b) { return b.kv_reserve_tokens ? 0x7FFFFFFFu : (uint32_t)b.kv_budget; }
 
-size_t queue_build_smem(int n_req) {
-    return n_req <= 65536 ? sort_smem_bytes<uint16_t>(n_req) : sort_smem_bytes<uint32_t>(n_req);
-}
+size_t queue_build_smem(int n_req) { return sort_smem_bytes<uint16_t>(n_req); }
 
 cudaError_t launch_queue_build(const hos_batch& b, const int32_t* assign, uint32_t p_max, int queue_order, uint2* q_po,
                                uint32_t* q_key, uint32_t* q_req, int32_t* q_off, unsigned long long* inst_O,
                                int32_t* inst_status, int n_pad, cudaStream_t st) {
-    const size_t smem = queue_build_smem(b.n_req);
-    auto kern = b.n_req <= 65536 ? k_queue_build<uint16_t> : k_queue_build<uint32_t>;
-    cudaError_t e = allow_max_dynamic_smem(reinterpret_cast<const void*>(kern));
+    cudaError_t e = allow_max_dynamic_smem(reinterpret_cast<const void*>(k_queue_build<true>));
     if (e != cudaSuccess) return e;
+    if ((e = allow_max_dynamic_smem(reinterpret_cast<const void*>(k_queue_build<false>))) != cudaSuccess) return e;
+    const long long most = b.kv_reserve_tokens ? (long long)b.kv_reserve_tokens : (long long)b.kv_budget;
     launch_hook("k_queue_build", 0, st);
-    kern<<<b.n_inst, SORT_THREADS, smem, st>>>(b.p, b.o, b.o_est, assign, b.n_req, b.n_clients,
-                                               b.kv_reserve_tokens ? (long long)b.kv_reserve_tokens
-                                                                   : (long long)b.kv_budget,
-                                               p_max, queue_order, q_po, b.o_est ? q_key : nullptr, q_req, q_off,
-                                               inst_O, inst_status, n_pad);
+    k_queue_build<true><<<b.n_inst, SORT_THREADS, bucket_sort_smem_bytes(b.n_req), st>>>(
+        b.p, b.o, b.o_est, assign, b.n_inst, b.n_req, b.n_clients, most, p_max, queue_order, q_po,
+        b.o_est ? q_key : nullptr, q_req, q_off, inst_O, inst_status, n_pad);
     launch_hook("k_queue_build", 1, st);
+    int n_sm = 148, dev = 0;
+    if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev);
+    launch_hook("k_queue_build_radix", 0, st);
+    k_queue_build<false><<<b.n_inst < n_sm ? b.n_inst : n_sm, SORT_THREADS, queue_build_smem(b.n_req), st>>>(
+        b.p, b.o, b.o_est, assign, b.n_inst, b.n_req, b.n_clients, most, p_max, queue_order, q_po,
+        b.o_est ? q_key : nullptr, q_req, q_off, inst_O, inst_status, n_pad);
+    launch_hook("k_queue_build_radix", 1, st);
     return cudaGetLastError();
 }
 

@@ -403,3 +403,34 @@ def test_multifit_on_the_configs(hos):
     e = ora.offline_pack(p[0], o[0], w.n_clients, w.cost_model, 5, multifit_steps=64)
     assert g["status"].tolist() == [hos.HOS_ST_INVALID, 0] and g["packer"][0] == 0
     assert np.array_equal(g["assign"][1], e["assign"]) and (g["assign"][0] == -1).all()
+
+
+@pytest.mark.parametrize("kind", ["all_equal", "two_values", "wide_keys", "wide_keys_short", "one_heavy_bucket"])
+def test_sort_falls_back_on_bunched_or_wide_keys(hos, kind):
+    """Instances whose keys bunch into a few buckets, or are too wide for a bucket entry, take the
+    radix sort instead of the bucket sort -- next to ordinary instances in the same batch."""
+    rng = np.random.default_rng(len(kind))
+    n_inst, n, M, cap = 3, 6000, 12, 24
+    p = rng.integers(16, 3000, size=(n_inst, n)).astype(np.uint32)
+    o = rng.integers(8, 900, size=(n_inst, n)).astype(np.uint32)
+    cm = (20000, 40, 15000, 300, 16, 40, 350)
+    if kind == "all_equal":
+        p[1] = 77; o[1] = 13
+    elif kind == "two_values":
+        p[1] = np.where(rng.random(n) < 0.5, 100, 101); o[1] = 50
+    elif kind == "wide_keys":                      # T up to ~2^31: rest of the key + id pass 32 bits at this size
+        n = 12000
+        p = rng.integers(16, 3000, size=(n_inst, n)).astype(np.uint32)
+        o = rng.integers(8, 900, size=(n_inst, n)).astype(np.uint32)
+        cm = (20000, 40, 15000, 300, 16, 500000, 500000)
+    elif kind == "wide_keys_short":                # the same keys still fit beside a 9-bit id
+        n = 500
+        p, o = p[:, :n].copy(), o[:, :n].copy()
+        cm = (20000, 40, 15000, 300, 16, 500000, 500000)
+    elif kind == "one_heavy_bucket":
+        p[2, : n // 2] = 500; o[2, : n // 2] = rng.integers(100, 102, size=n // 2)
+    kv = 10 ** 6
+    g = H.check_offline(hos, p, o, M, cap, kv, cm, 3)
+    H.check_lower_bound(hos, p, o, M, cap, kv, cm)
+    for mode in (ora.QUEUE_SORTED, ora.QUEUE_FCFS):
+        H.check_simulate(hos, p, o, M, cap, kv, cm, g["assign"], (LAMBDA_ONE,), mode)
