@@ -186,53 +186,67 @@ __device__ inline IdxT* block_radix_sort_ids(const SortSmem<IdxT>& s, int n, int
 //
 // The order wanted -- (key ^ flip) ascending over its low `nbits` bits, then id ascending -- is a
 // total order of distinct pairs, so it does not matter in which order the items of a bucket
-// arrive: the top BUCKET_BITS bits of the key choose a bucket (shared-memory histogram, scan,
-// scatter by atomic slot counters), every bucket entry is the rest of the key above the id in
-// one 32-bit word, and an item's final position is its bucket's start plus the number of
-// entries of that bucket below its own.  With keys that spread over the buckets this is a few
-// compares per item instead of a ranking vote per key bit and pass.  Returns false, with nothing
-// written, when the entries do not fit 32 bits or the buckets are so uneven that the compares
-// would cost more than the radix passes (sum of squared bucket sizes above BUCKET_WORK_MAX per
-// item); the caller then takes block_radix_sort_ids.
+// arrive: the top bits of the key choose a bucket (shared-memory histogram, scan, scatter by
+// atomic slot counters), every bucket entry is the rest of the key above the id in one 32-bit
+// word, and an item's final position is its bucket's start plus the number of entries of that
+// bucket below its own.  With about two buckets per item and keys that spread over them this
+// is a few compares per item instead of a ranking vote per key bit and pass.  The counters are
+// 16 bits wide, two to a word (no count or offset reaches 2^16), which buys twice the buckets
+// for the shared memory.  Returns false, with nothing written, when the entries do not fit 32
+// bits or the buckets are so uneven that the compares would cost more than the radix passes
+// (sum of squared bucket sizes above BUCKET_WORK_MAX per item); the caller then takes
+// block_radix_sort_ids.
 //
-// One CTA of SORT_THREADS threads; key[n] in shared memory; `ent` n words and `cnt` BUCKETS + 1
-// words of shared memory.  On success ent[r] is the id of the item of rank r.
+// One CTA of SORT_THREADS threads; key[n] in shared memory; `ent` n words and `cntw`
+// 2^(bucket bits - 1) words of shared memory.  On success ent[r] is the id of the item of rank r.
 // ---------------------------------------------------------------------------------------
-constexpr int BUCKET_BITS = 12;
-constexpr int BUCKETS = 1 << BUCKET_BITS;
+constexpr int BUCKET_BITS_MAX = 15;
 constexpr int BUCKET_WORK_MAX = 96;
 constexpr int BUCKET_ITEMS_PER_THREAD = (MAX_REQ + SORT_THREADS - 1) / SORT_THREADS;   // 24
 
+// Most bucket bits whose counters fit beside the two n-word arrays (host and device agree on it).
+__host__ __device__ inline int bucket_bits_cap(int n) {
+    const size_t room = SMEM_LIMIT - 2048 - 2 * align16(size_t(n) * 4);      // 2 KB left for static shared memory
+    int bb = BUCKET_BITS_MAX;
+    while (bb > 10 && (size_t(2) << bb) > room) --bb;
+    int want = 11;                                                           // about two buckets per item
+    while (want < BUCKET_BITS_MAX && (1 << want) < 2 * n) ++want;
+    return bb < want ? bb : want;
+}
 __host__ __device__ inline size_t bucket_sort_smem_bytes(int n) {
-    return 2 * align16(size_t(n) * 4) + size_t(BUCKETS + 32) * 4;
+    return 2 * align16(size_t(n) * 4) + (size_t(2) << bucket_bits_cap(n));
 }
 
-__device__ inline bool block_bucket_sort(const uint32_t* key, uint32_t* ent, uint32_t* cnt, int n, int nbits,
+__device__ inline bool block_bucket_sort(const uint32_t* key, uint32_t* ent, uint32_t* cntw, int n, int nbits,
                                          uint32_t flip) {
     __shared__ uint32_t s_wsum[SORT_WARPS];
     __shared__ unsigned long long s_work;
     const int t = threadIdx.x;
-    const int bbits = min(nbits, BUCKET_BITS);
-    const int low_bits = nbits - bbits;
+    const int bbits = max(1, min(nbits, bucket_bits_cap(n)));
+    const int low_bits = max(0, nbits - bbits);
     const int id_bits = n > 1 ? bit_width_u32((uint32_t)(n - 1)) : 1;
     if (low_bits + id_bits > 32) return false;                      // uniform: same arguments in every thread
     const uint32_t kmask = nbits >= 32 ? 0xFFFFFFFFu : ((1u << nbits) - 1u);
     const uint32_t lmask = (1u << low_bits) - 1u;                   // low_bits <= 31 here
-    for (int i = t; i < BUCKETS + 1; i += SORT_THREADS) cnt[i] = 0;
+    const int n_words = 1 << (bbits - 1);                           // two counters per word
+    const uint16_t* cnt16 = reinterpret_cast<const uint16_t*>(cntw);
+    for (int i = t; i < n_words; i += SORT_THREADS) cntw[i] = 0;
     if (t == 0) s_work = 0;
     __syncthreads();
-    for (int i = t; i < n; i += SORT_THREADS) atomicAdd(&cnt[((key[i] ^ flip) & kmask) >> low_bits], 1u);
+    for (int i = t; i < n; i += SORT_THREADS) {
+        const uint32_t b = ((key[i] ^ flip) & kmask) >> low_bits;
+        atomicAdd(&cntw[b >> 1], 1u << ((b & 1u) << 4));
+    }
     __syncthreads();
-    {   // exclusive scan of the bucket counts (BUCKETS / SORT_THREADS consecutive buckets per thread)
-        constexpr int PER = BUCKETS / SORT_THREADS;
-        uint32_t v[PER], run = 0;
+    {   // exclusive scan of the bucket counts: consecutive words per thread
+        const int per = (n_words + SORT_THREADS - 1) / SORT_THREADS;
+        const int w0 = min(n_words, t * per), w1 = min(n_words, w0 + per);
+        uint32_t run = 0;
         unsigned long long work = 0;
-#pragma unroll
-        for (int k = 0; k < PER; ++k) {
-            const uint32_t c = cnt[t * PER + k];
-            v[k] = run;
-            run += c;
-            work += (unsigned long long)c * c;
+        for (int w = w0; w < w1; ++w) {
+            const uint32_t c = cntw[w], a = c & 0xFFFFu, b = c >> 16;
+            run += a + b;
+            work += (unsigned long long)(a * a + b * b);
         }
         uint32_t inc = run;
 #pragma unroll
@@ -244,19 +258,21 @@ __device__ inline bool block_bucket_sort(const uint32_t* key, uint32_t* ent, uin
         if (lane_id() == 31) s_wsum[warp_id()] = inc;
         if (lane_id() == 0 && work) atomicAdd(&s_work, work);
         __syncthreads();
-        uint32_t before = 0;
         const uint32_t wv = s_wsum[lane_id()];
-        before = __reduce_add_sync(FULL, lane_id() < warp_id() ? wv : 0u);
-        const uint32_t base = before + inc - run;
-#pragma unroll
-        for (int k = 0; k < PER; ++k) cnt[t * PER + k] = base + v[k];
+        uint32_t acc = __reduce_add_sync(FULL, lane_id() < warp_id() ? wv : 0u) + inc - run;
+        for (int w = w0; w < w1; ++w) {
+            const uint32_t c = cntw[w], a = c & 0xFFFFu, b = c >> 16;
+            cntw[w] = acc | ((acc + a) << 16);
+            acc += a + b;
+        }
         __syncthreads();
     }
     if (s_work > (unsigned long long)BUCKET_WORK_MAX * (unsigned long long)n) return false;   // uniform
-    // scatter: cnt[b] walks from the start of bucket b to its end
+    // scatter: counter b walks from the start of bucket b to its end
     for (int i = t; i < n; i += SORT_THREADS) {
         const uint32_t fk = (key[i] ^ flip) & kmask;
-        const uint32_t slot = atomicAdd(&cnt[fk >> low_bits], 1u);
+        const uint32_t b = fk >> low_bits, sh = (b & 1u) << 4;
+        const uint32_t slot = (atomicAdd(&cntw[b >> 1], 1u << sh) >> sh) & 0xFFFFu;
         ent[slot] = ((fk & lmask) << id_bits) | (uint32_t)i;
     }
     __syncthreads();
@@ -270,9 +286,10 @@ __device__ inline bool block_bucket_sort(const uint32_t* key, uint32_t* ent, uin
             const uint32_t fk = (key[i] ^ flip) & kmask;
             const uint32_t b = fk >> low_bits;
             const uint32_t mine = ((fk & lmask) << id_bits) | (uint32_t)i;
-            const uint32_t start = b ? cnt[b - 1] : 0u, end = cnt[b];
-            uint32_t r = start;
-            for (uint32_t s = start; s < end; ++s) r += ent[s] < mine ? 1u : 0u;
+            const uint32_t start = b ? cnt16[b - 1] : 0u, end = cnt16[b];
+            uint32_t r = start, s2 = start;
+            for (; s2 + 1 < end; s2 += 2) r += (ent[s2] < mine ? 1u : 0u) + (ent[s2 + 1] < mine ? 1u : 0u);
+            if (s2 < end) r += ent[s2] < mine ? 1u : 0u;
             rank[e] = r;
         }
     }
