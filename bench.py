@@ -34,21 +34,33 @@ DTYPE = "int64"            # integer microseconds / Q16.16; utilisation is one f
 L2_FLUSH_BYTES = 256 << 20
 
 # algorithmic bytes per unit of work of each kernel (what a streaming implementation of that
-# step alone must move once)
-BYTES_PER_REQ = {"k_estimate_sort": 16, "k_lpt": 12, "k_lower_bound": 8, "k_queue_build": 16, "k_ls_lists": 15}
-# what bounds each kernel (counters in profiles/): streaming kernels against the measured copy
-# bandwidth, the two sequential recurrences against the integer issue rate
-BOUND = {"k_simulate": "alu", "k_simulate_steal": "alu", "k_lpt": "latency (dependent chain)",
-         "k_local_search": "latency / issue (instance resident on chip; bytes are those of a streaming round)"}
+# step alone must move once); the estimate + sort kernel also carries the lower bounds' 64 B per instance
+BYTES_PER_REQ = {"k_estimate_sort": 16, "k_lpt": 12, "k_queue_build": 16, "k_ls_lists": 15, "k_multifit": 9}
+# What bounds each kernel (counters in profiles/).  "hbm": streaming, set against the measured copy
+# bandwidth.  "alu": the iteration recurrence, integer operations of the method against the int32
+# lanes.  "issue": dependent chains on data that stays on chip (DRAM idle); warp instructions
+# issued against the schedulers' issue slots.
+BOUND = {"k_simulate": "alu", "k_simulate_steal": "alu", "k_lpt": "issue", "k_local_search": "issue",
+         "k_multifit": "issue"}
 # integer operations of one simulated iteration as the method states it: duration (3), busy slot
 # time (2), clock (1), waited decode time (2), sum of KV lengths (1), decision compare in Q16.16 (3),
 # trace hash (9), counters (3)
 INT_OPS_PER_ITERATION = 24
-# DRAM bytes per request and launch measured with ncu (dram__bytes_read.sum + dram__bytes_write.sum
-# over 296 instances of c4's shape, see profiles/); None for a kernel changed since its capture
-NCU_DRAM_BYTES_PER_REQ = {"k_estimate_sort": 8.68, "k_lower_bound": 8.05, "k_lpt": 12.69, "k_ls_lists": 18.09,
-                          "k_local_search": 6.07, "k_queue_build": 15.77, "k_simulate": 20.75}
-NCU_DRAM_BYTES_PER_ITERATION = {"k_trace_fill": 18.79}
+# Counters of one ncu capture (DRAM bytes and warp instructions per unit of work and kernel),
+# written by paper_2502_15763_b200/profile_summary.py; ignored once the library sources changed.
+NCU_COUNTERS = os.path.join(ROOT, "profiles", "ncu_counters_c4x296.json")
+
+
+def ncu_counters():
+    """(counters per kernel, note): {} with the reason when the file is missing or stale."""
+    try:
+        doc = json.load(open(NCU_COUNTERS))
+    except (OSError, ValueError):
+        return {}, "no counter file"
+    from paper_2502_15763_b200 import _build
+    if doc.get("source_hash") != _build.source_hash():
+        return {}, "kernels changed since the counters were taken"
+    return doc.get("kernels", {}), "ncu capture of " + doc.get("workload", "?")
 
 
 def describe(w: Workload) -> str:
@@ -154,6 +166,8 @@ class Pipeline:
         self.up = None
         self.down = None
         self.sets = None
+        self.trace_free = None
+        self.trace_host = None
 
     def tables(self):
         return dict(p=self.p, o=self.o, est=self.est, lam=self.lam)
@@ -197,6 +211,8 @@ class Pipeline:
         if self.trace is None:                      # first (warm-up) step sizes the trace buffer
             self.n_iters = int(off[-1].item())
             self.trace = self.torch.empty((max(self.n_iters, 1), 16), dtype=self.torch.uint8, device=self.dev)
+        if self.trace_free is not None:             # the last step's trace is still on its way to the host
+            self.torch.cuda.current_stream().wait_event(self.trace_free)
         hos.hos_trace_fill(*self.args(t), len(w.lambdas_q16), s1, self.trace, off, **kw)
         self.out = dict(pk=pk, lb=lb, sim=s1, off=off)
         if len(w.lambdas_q16) > 1 and w.ls_rounds > 0:
@@ -212,7 +228,7 @@ class Pipeline:
         return (pk["assign"], pk["load"], pk["makespan_est"], pk["status"], r["lb"]["lb"],
                 sim["cres"], sim["sres"], sim["status"])
 
-    def e2e_run(self, steps, host_out, flush):
+    def e2e_run(self, steps, host_out, flush, with_trace=False):
         """`steps` steps from pinned host tables to pinned host results, as a stream of batches.
 
         Every step uploads its own tables and downloads its own results.  There are two sets of device
@@ -263,12 +279,21 @@ class Pipeline:
                         self.down.wait_event(done)
                     h.copy_(d, non_blocking=True)
                     d.record_stream(self.down)      # the allocator must not hand it out again before the copy ends
+                if with_trace:                      # the iteration trace too: the next fill waits for this copy
+                    if self.trace_host is None:
+                        self.trace_host = torch.empty(self.trace.shape, dtype=torch.uint8).pin_memory()
+                    self.trace_host.copy_(self.trace, non_blocking=True)
+                    self.trace_free = torch.cuda.Event()
+                    self.trace_free.record(self.down)
         main.wait_stream(self.down)
         main.wait_stream(self.up)
         end.record(main)
         torch.cuda.synchronize()
+        self.trace_free = None
         h2d = sum(h.numel() * h.element_size() for h in host.values() if h is not None)
         d2h = sum(h.numel() * h.element_size() for h in host_out)
+        if with_trace:
+            d2h += self.trace_host.numel()
         return start.elapsed_time(end), h2d, d2h
 
 
@@ -325,13 +350,11 @@ def algorithmic_bytes(w: Workload, name: str, pipe) -> float:
     """Bytes one launch of `name` must move at least (see the design notes for the per-unit figures)."""
     n_req_total = w.n_inst * w.n_req
     if name in BYTES_PER_REQ:
-        extra = 64 * w.n_inst if name == "k_lower_bound" else 0
-        return BYTES_PER_REQ[name] * n_req_total + extra
+        extra = 64 * w.n_inst if name == "k_estimate_sort" else 0
+        copies = len(w.lambdas_q16) if name == "k_ls_lists" and len(w.lambdas_q16) > 1 else 1
+        return BYTES_PER_REQ[name] * n_req_total * copies + extra
     if name == "k_local_search":
-        src = pipe.out["ls"] if "ls" in pipe.out else pipe.out["pk"]
-        applied = src["rounds_applied"].to("cpu").numpy().astype(np.int64)
-        executed = np.minimum(applied + 1, w.ls_rounds).sum()          # the no-op round is evaluated too
-        return float(executed) * (8 * w.n_req + 8 * w.n_clients)
+        return float(executed_rounds(w, pipe)) * (8 * w.n_req + 8 * w.n_clients)
     if name == "k_simulate":
         n_sims = w.n_inst * len(w.lambdas_q16)
         # reads the queue entries, writes the client results
@@ -345,6 +368,117 @@ def algorithmic_bytes(w: Workload, name: str, pipe) -> float:
     return 0.0
 
 
+def executed_rounds(w: Workload, pipe) -> int:
+    """Local-search rounds that were evaluated in the last step (the round that finds nothing counts)."""
+    src = pipe.out.get("ls") or pipe.out["pk"]
+    if w.ls_rounds <= 0:
+        return 0
+    applied = src["rounds_applied"].to("cpu").numpy().astype(np.int64)
+    return int(np.minimum(applied + 1, w.ls_rounds).sum())
+
+
+# Shortest a local-search round can be with its phases in sequence and nothing else on the SM
+# (cycles; the derivation is in the design notes): copy of the critical list (one global round
+# trip, ~600), nine dependent shared-memory probes (~270), evaluation of both neighbours (~100),
+# two CTA-wide minima with a barrier between (~300), load update and next extremes (~300), list
+# patch by search and shift (~550), two barriers (~100).
+LS_ROUND_MIN_CYCLES = 2200
+
+
+def input_sha256(pipe) -> str:
+    """SHA-256 of the request tables this rank evaluates (p, o and, if used, the estimates)."""
+    import hashlib
+    h = hashlib.sha256()
+    for t in (pipe.p_host, pipe.o_host, pipe.est_host):
+        if t is not None:
+            h.update(t.numpy().tobytes())
+    return h.hexdigest()
+
+
+def struct_view(t, dtype):
+    from paper_2502_15763_b200.binding import view_struct
+    return view_struct(t, dtype)
+
+
+def study_report(hos, pipe, w: Workload) -> dict:
+    """The 100-case study (Section "Numerical experiment"): hybrid scheduling (longest-first packing,
+    queues sorted by length, multiplier 1.0) against the two baselines (requests dealt round-robin
+    in arrival order, first-come-first-served queues; prefill-first, and never preempting a decode)."""
+    import torch
+    from workload import LAMBDA_NEVER_PREEMPT, LAMBDA_ONE, LAMBDA_PREFILL_FIRST
+    args = pipe.args()
+    pk = hos.hos_offline_pack(*args, w.ls_rounds, want_lb=True, **pipe.kw)
+    lam = lambda *v: torch.from_numpy(np.asarray(v, dtype=np.uint32).view(np.int32)).to(pipe.dev)
+    hyb = hos.hos_online_simulate(*args, pk["assign"], lam(LAMBDA_ONE), hos.HOS_QUEUE_SORTED, **pipe.kw)
+    rr = (torch.arange(w.n_req, dtype=torch.int32, device=pipe.dev) % w.n_clients)[None, :].repeat(w.n_inst, 1).contiguous()
+    base = hos.hos_online_simulate(*args, rr, lam(LAMBDA_PREFILL_FIRST, LAMBDA_NEVER_PREEMPT), hos.HOS_QUEUE_FCFS,
+                                   **pipe.kw)
+    h = struct_view(hyb["sres"], hos.SIM_RESULT_DTYPE)[:, 0]
+    b = struct_view(base["sres"], hos.SIM_RESULT_DTYPE)
+    lb = struct_view(pk["lb"], hos.LB_DTYPE)
+    uh, up, un = h["utilisation"], b["utilisation"][:, 0], b["utilisation"][:, 1]
+    r4 = lambda a: [round(float(x), 4) for x in a]
+    return {
+        "instances": w.n_inst,
+        "mean_utilisation": {"hybrid": float(uh.mean()), "fcfs_prefill_first": float(up.mean()),
+                             "fcfs_never_preempt": float(un.mean())},
+        "mean_makespan_s": {"hybrid": float(h["makespan_us"].mean()) / 1e6,
+                            "fcfs_prefill_first": float(b["makespan_us"][:, 0].mean()) / 1e6,
+                            "fcfs_never_preempt": float(b["makespan_us"][:, 1].mean()) / 1e6,
+                            "lower_bound": float(lb["lb_sim_us"].mean()) / 1e6},
+        "gain_vs_prefill_first": {"percentage_points": float((uh - up).mean() * 100), "ratio": float((uh / up).mean()),
+                                  "instances_improved": int((uh > up).sum())},
+        "gain_vs_never_preempt": {"percentage_points": float((uh - un).mean() * 100), "ratio": float((uh / un).mean()),
+                                  "instances_improved": int((uh > un).sum())},
+        "tokens_per_s_gain_vs_prefill_first": float((h["tokens_per_s"] - b["tokens_per_s"][:, 0]).mean()),
+        "paper_context": "the paper's own 100-case study on its data reports +8.0 % utilisation and +100.63 tokens/s",
+        "per_instance": {"utilisation_hybrid": r4(uh), "utilisation_fcfs_prefill_first": r4(up),
+                         "utilisation_fcfs_never_preempt": r4(un),
+                         "makespan_over_lower_bound": r4(h["makespan_us"] / lb["lb_sim_us"])},
+    }
+
+
+def sweep_report(torch, hos, pipe, w: Workload, flush) -> dict:
+    """The multiplier sweep's local search both ways: one private copy of the packing per (instance,
+    multiplier), as the workload states it, and once per instance (the copies agree bit for bit)."""
+    pk = pipe.out["pk"]
+    nl = len(w.lambdas_q16)
+    copies = pk["assign"][:, None, :].expand(-1, nl, -1).contiguous()
+    one = pk["assign"][:, None, :].contiguous()
+    run_all = lambda: hos.hos_local_search(*pipe.args(), copies.clone(), w.ls_rounds, ws=pipe.ws_off, **pipe.kw)
+    run_one = lambda: hos.hos_local_search(*pipe.args(), one.clone(), w.ls_rounds, ws=pipe.ws_off, **pipe.kw)
+    run_all(); run_one()
+    torch.cuda.synchronize()
+    ms_all = timed_steps(torch, run_all, 5, flush) / 5
+    ms_one = timed_steps(torch, run_one, 5, flush) / 5
+    return {"as_executed": {"searches": w.n_inst * nl, "rounds_each": w.ls_rounds, "ms": ms_all,
+                            "rounds_per_s": w.n_inst * nl * w.ls_rounds / (ms_all * 1e-3)},
+            "deduplicated": {"searches": w.n_inst, "rounds_each": w.ls_rounds, "ms": ms_one,
+                             "rounds_per_s": w.n_inst * w.ls_rounds / (ms_one * 1e-3)},
+            "note": "times include the clone of the assignments and the sort that hos_local_search does itself"}
+
+
+def packing_gap_report(torch, hos, pipe, w: Workload, flush) -> dict:
+    """makespan_est - lb_pack with the list schedule and with MULTIFIT before the same local search."""
+    rounds = w.ls_rounds if len(w.lambdas_q16) == 1 else 0
+    out = {}
+    for key, steps in (("lpt", 0), ("multifit", 64)):
+        run = lambda: hos.hos_offline_pack(*pipe.args(), rounds, ws=pipe.ws_off, want_lb=True, multifit_steps=steps,
+                                           **pipe.kw)
+        r = run()
+        torch.cuda.synchronize()
+        ms_ = timed_steps(torch, run, 3, flush) / 3
+        lb = struct_view(r["lb"], hos.LB_DTYPE)["lb_pack"]
+        mk = r["makespan_est"].cpu().numpy()
+        gap = mk - lb
+        out[key] = {"ms_per_call": ms_, "mean_gap": float(gap.mean()), "max_gap": int(gap.max()),
+                    "mean_relative_gap": float((gap / np.maximum(lb, 1)).mean()), "at_lower_bound": int((gap == 0).sum()),
+                    "local_search_rounds": rounds}
+        if steps:
+            out[key]["instances_taking_multifit"] = int(r["packer"].sum().item())
+    return out
+
+
 def measured_peak():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
@@ -355,15 +489,15 @@ def measured_peak():
     return 6650.0, "fallback"
 
 
-def oracle_sample(w: Workload, n_sample: int):
-    """Time the CPU oracle (one thread) on the first n_sample instances: the whole path."""
+def oracle_sample(w: Workload, n_sample: int, repeats: int = 1):
+    """Time the CPU oracle (one thread) on the first n_sample instances, `repeats` times over: the whole path."""
     from oracle import hos_oracle as ora
     sub = w.subset(0, n_sample)
     p, o = sub.lengths()
     est = sub.estimates()
     t0 = time.perf_counter()
     iters = 0
-    for k in range(sub.n_inst):
+    for k in [k for _ in range(repeats) for k in range(sub.n_inst)]:
         sweep = len(w.lambdas_q16) > 1
         pk = ora.offline_pack(p[k], o[k] if est is None else est[k], w.n_clients, w.cost_model,
                               0 if sweep else w.ls_rounds)
@@ -376,13 +510,16 @@ def oracle_sample(w: Workload, n_sample: int):
             if sweep and w.ls_rounds > 0:      # local search on a private copy per multiplier value
                 ora.local_search(pk["T"], pk["assign"], pk["load"], w.ls_rounds)
     dt = time.perf_counter() - t0
-    return sub.n_inst / dt, iters / dt, dt
+    return sub.n_inst * repeats / dt, iters / dt, dt
 
 
-def sample_size(w: Workload) -> int:
-    # about 3 s of single-thread oracle work per instance at the largest size, milliseconds at the others
-    per_inst = 3.0 if w.n_req >= 10000 else 0.025 * max(1, len(w.lambdas_q16)) + 0.03
-    return max(1, min(w.n_inst, int(12.0 / per_inst)))
+def sample_size(w: Workload, budget_s: float = 12.0) -> int:
+    """Instances of the workload (from its start, at most all of them) that take the oracle about
+    budget_s seconds on one core, from the time of the first one."""
+    t0 = time.perf_counter()
+    oracle_sample(w, 1)
+    per_inst = max(time.perf_counter() - t0, 1e-4)
+    return max(1, min(w.n_inst, int(budget_s / per_inst)))
 
 
 def run_ours(args):
@@ -454,6 +591,24 @@ def run_ours(args):
         torch.cuda.synchronize()
         steal_ms = timed_steps(torch, run_steal, 3, flush) / 3
 
+    e2e_trace = None
+    if rank == 0 and not args.skip_e2e and not args.skip_e2e_trace:
+        pipe.e2e_run(1, host_out, flush, with_trace=True)
+        n_t = max(2, min(args.steps, 5))
+        ms_t, h2d_t, d2h_t = pipe.e2e_run(n_t, host_out, flush, with_trace=True)
+        e2e_trace = {"value": w.n_inst * n_t / (ms_t * 1e-3), "unit": UNIT, "steps": n_t, "n_gpus": 1,
+                     "h2d_bytes_per_step": h2d_t, "d2h_bytes_per_step": d2h_t,
+                     "note": "as e2e, with the full iteration trace delivered to pinned host memory every step"}
+        pipe.step()
+    study = sweep = gap = None
+    if rank == 0 and not args.skip_reports:
+        if len(w.lambdas_q16) == 1 and w.n_inst >= 8 and (args.study or w.name in ("c2", "c2e", "paper")):
+            study = study_report(hos, pipe, w)
+        if len(w.lambdas_q16) > 1 and w.ls_rounds > 0:
+            sweep = sweep_report(torch, hos, pipe, w, flush)
+        gap = packing_gap_report(torch, hos, pipe, w, flush)
+        pipe.step()
+
     st = pipe.out
     bad = int((st["pk"]["status"] != 0).sum().item()) + int((st["sim"]["status"] != 0).sum().item())
     if bad:
@@ -462,52 +617,85 @@ def run_ours(args):
     if rank == 0:
         prof = kernel_profile(torch, hos, pipe, max(2, min(args.steps, 5)), flush)
         peak, peak_kind = measured_peak()
+        counters, counters_note = ncu_counters()
+        props = torch.cuda.get_device_properties(dev)
+        mhz = (clocks or {}).get("sm_max_mhz") or 1965.0
+        alu_peak = props.multi_processor_count * 128 * mhz * 1e6 / 1e12       # T int32 op/s
+        issue_peak = props.multi_processor_count * 4 * mhz * 1e6 / 1e9        # G warp instructions/s
+        units = {"request": w.n_inst * w.n_req, "iteration": pipe.n_iters,
+                 "round": executed_rounds(w, pipe)}
+
+        def scaled(name, field):
+            """Counter of the capture scaled to this launch by the units it processes."""
+            c = counters.get(name)
+            if not c:
+                return None
+            n = units[c["unit"]]
+            if c["unit"] == "request" and len(w.lambdas_q16) > 1 and name in ("k_simulate", "k_ls_lists"):
+                n *= len(w.lambdas_q16)                  # one pass over the requests per multiplier value
+            return c[field] * n
+
         rows = {}
         for name, r in prof.items():
+            sec = r["ms_per_launch"] * 1e-3
             by = algorithmic_bytes(w, name, pipe)
-            gbs = by / (r["ms_per_launch"] * 1e-3) / 1e9
-            rows[name] = dict(r, algorithmic_bytes=by, achieved_gbs=gbs, frac=gbs / peak,
-                              ms_per_step=r["ms_per_launch"] * r["launches_per_step"])
-        for name in rows:
-            rows[name]["bound"] = BOUND.get(name, "hbm")
+            row = dict(r, ms_per_step=r["ms_per_launch"] * r["launches_per_step"], bound=BOUND.get(name, "hbm"),
+                       algorithmic_bytes=by, traffic=scaled(name, "dram_bytes_per_unit"))
+            if row["bound"] == "hbm":
+                row.update(achieved=by / sec / 1e9, peak=peak, unit="GB/s", peak_source=f"of {peak_kind}")
+            elif row["bound"] == "alu":
+                row.update(achieved=INT_OPS_PER_ITERATION * pipe.n_iters / sec / 1e12, peak=alu_peak,
+                           unit="Tint32op/s", peak_source="SMs x 128 int32 lanes x max SM clock",
+                           ops_per_iteration=INT_OPS_PER_ITERATION)
+            else:
+                inst = scaled(name, "warp_inst_per_unit")
+                row.update(achieved=None if inst is None else inst / sec / 1e9, peak=issue_peak,
+                           unit="Gwarp-inst/s", peak_source="SMs x 4 schedulers x max SM clock",
+                           warp_inst_per_launch=inst)
+                row["effective_gbs"] = by / sec / 1e9     # what a streaming form of the step would have to sustain
+            row["frac"] = None if row["achieved"] is None else row["achieved"] / row["peak"]
+            rows[name] = row
+        if "k_local_search" in rows and units["round"]:
+            r, n_ctas = rows["k_local_search"], w.n_inst * (len(w.lambdas_q16) if len(w.lambdas_q16) > 1 else 1)
+            inst = r.get("warp_inst_per_launch")
+            # rounds run side by side, one CTA per (instance, copy): a CTA's rounds follow each other
+            r["round"] = {"executed_rounds": units["round"], "rounds_per_cta": units["round"] / n_ctas,
+                          "us_per_round_per_cta": r["ms_per_launch"] * 1e3 / (units["round"] / n_ctas),
+                          "cycles_per_round_per_cta": r["ms_per_launch"] * 1e-3 * mhz * 1e6 / (units["round"] / n_ctas),
+                          "warp_inst_per_round": None if inst is None else inst / units["round"],
+                          "min_cycles_dependent_phases": LS_ROUND_MIN_CYCLES}
         top = max(rows, key=lambda n: rows[n]["ms_per_step"])
-        def dram_traffic(name):
-            # scaled from the capture by the units a launch processes (requests of every instance or
-            # simulation; iterations for the trace)
-            if name in NCU_DRAM_BYTES_PER_ITERATION:
-                return NCU_DRAM_BYTES_PER_ITERATION[name] * pipe.n_iters
-            per_req = NCU_DRAM_BYTES_PER_REQ.get(name)
-            if per_req is None:
-                return None
-            sims = len(w.lambdas_q16) if name in ("k_simulate", "k_local_search", "k_ls_lists") and len(w.lambdas_q16) > 1 else 1
-            return per_req * w.n_inst * w.n_req * sims
-        for name in rows:
-            rows[name]["traffic"] = dram_traffic(name)
-        traffic = dram_traffic(top)
-        if BOUND.get(top) == "alu":
-            # the iteration recurrence is integer arithmetic: operations of the method per second
-            # against 128 int32 lanes per SM at the maximum SM clock
-            props = torch.cuda.get_device_properties(dev)
-            mhz = (clocks or {}).get("sm_max_mhz") or 1965.0
-            alu_peak = props.multi_processor_count * 128 * mhz * 1e6 / 1e12
-            ach = INT_OPS_PER_ITERATION * pipe.n_iters / (rows[top]["ms_per_launch"] * 1e-3) / 1e12
-            roofline = {"kernel": top, "bound": "alu", "achieved": ach, "peak": alu_peak, "unit": "Tint32op/s",
-                        "frac": ach / alu_peak, "traffic": traffic,
-                        "peak_source": "SMs x 128 int32 lanes x max SM clock",
-                        "ops_per_iteration": INT_OPS_PER_ITERATION, "ms_per_launch": rows[top]["ms_per_launch"]}
-        else:
-            roofline = {"kernel": top, "bound": "hbm", "achieved": rows[top]["achieved_gbs"], "peak": peak,
-                        "unit": "GB/s", "frac": rows[top]["frac"], "traffic": traffic,
-                        "peak_source": f"of {peak_kind}", "ms_per_launch": rows[top]["ms_per_launch"]}
-            if top == "k_local_search":
-                roofline["note"] = ("effective: bytes a streaming implementation would re-read every executed "
-                                    "round; this kernel reads the instance from HBM once")
+        t = rows[top]
+        roofline = {"kernel": top, "bound": "alu" if t["bound"] == "issue" else t["bound"],
+                    "model": {"hbm": "algorithmic bytes", "alu": "int32 operations of the method",
+                              "issue": "warp instructions issued"}[t["bound"]],
+                    "achieved": t["achieved"], "peak": t["peak"],
+                    "unit": t["unit"], "frac": t["frac"], "traffic": t["traffic"], "peak_source": t["peak_source"],
+                    "ms_per_launch": t["ms_per_launch"], "counters": counters_note}
+        if t["bound"] == "issue":
+            roofline["note"] = ("latency-bound chain on data resident on chip: warp instructions issued (ncu "
+                                "count per unit of work x units of this launch) against the issue slots; "
+                                "effective_gbs is what a streaming form re-reading the instance every round "
+                                "would have to sustain, not a bandwidth this kernel reaches")
+            roofline["effective_gbs"] = t["effective_gbs"]
+            if "round" in t:
+                roofline["round"] = t["round"]
+        # the step as a whole against the HBM roofline: algorithmic bytes of every kernel, local search once
+        step_bytes = sum(r["algorithmic_bytes"] for n, r in rows.items() if r["bound"] != "issue" or n == "k_lpt")
+        step_bytes += 8.0 * w.n_inst * w.n_req if "k_local_search" in rows else 0.0
+        step_roofline = {"algorithmic_bytes": step_bytes, "achieved_gbs": step_bytes / (ms / args.steps * 1e-3) / 1e9,
+                         "frac_of_hbm": step_bytes / (ms / args.steps * 1e-3) / 1e9 / peak}
         launches = sum(r["launches_per_step"] for r in prof.values())
-        n_s = sample_size(w)
+        n_s, reps = 0, 1
         if args.skip_cpu_baseline:
             cpu_inst, cpu_iters, cpu_dt = None, None, 0.0
         else:
-            cpu_inst, cpu_iters, cpu_dt = oracle_sample(w, n_s)
+            n_s = sample_size(w)
+            if n_s == w.n_inst:                         # a small workload: over and over, for about 12 s in all
+                t1 = time.perf_counter()
+                oracle_sample(w, n_s)
+                reps = max(1, int(12.0 / max(time.perf_counter() - t1, 1e-3)))
+            cpu_inst, cpu_iters, cpu_dt = oracle_sample(w, n_s, reps)
         total_inst = w.n_inst * world
         line = {
             "metric": METRIC, "value": total_inst * args.steps / (ms * 1e-3), "unit": UNIT,
@@ -526,15 +714,21 @@ def run_ours(args):
                             "on the device); two sets of device tables, so step k+1's upload and step k-1's "
                             "download run beside step k's kernels; timed from the first upload to the last "
                             "download" + ("" if flush is None else ", L2 flushes included")},
+            "e2e_with_trace": e2e_trace,
             "gpu_launches": int(round(launches * args.steps)),
+            "requests_per_step": w.n_inst * w.n_req,
+            "ls_rounds_executed_per_step": units["round"],
+            "input_sha256": input_sha256(pipe),
             "roofline": roofline,
+            "step_roofline": step_roofline,
+            "study": study, "sweep_local_search": sweep, "packing_gap": gap,
             "kernels": rows,
             "request_stealing": None if steal_ms is None else {
                 "call": "hos_online_simulate_steal", "ms_per_call": steal_ms,
                 "simulations_per_s": w.n_inst * len(w.lambdas_q16) / (steal_ms * 1e-3),
                 "plain_simulate_ms": rows.get("k_simulate", {}).get("ms_per_launch")},
             "cpu_baseline": {"value": cpu_inst, "unit": UNIT, "cores": 1, "kind": "oracle",
-                             "sample": f"first {n_s} instance(s) of the workload, whole path, {cpu_dt:.1f} s",
+                             "sample": f"first {n_s} instance(s) of the workload x {reps}, whole path, {cpu_dt:.1f} s",
                              "sim_iterations_per_s": cpu_iters},
         }
         print(json.dumps(line))
@@ -549,7 +743,7 @@ def run_reference(args):
     if rank != 0:
         return
     w = workload(args.workload)
-    n_s = max(1, sample_size(w) // 4)        # per step; the default 50 steps then take about two minutes at c4
+    n_s = max(1, sample_size(w, 3.0))        # per step: about three seconds of oracle work
     for _ in range(args.warmup):
         oracle_sample(w, 1)
     t0 = time.perf_counter()
@@ -586,6 +780,12 @@ def main():
                     help="do not time the request-stealing simulation (profiling captures)")
     ap.add_argument("--skip-e2e", action="store_true",
                     help="do not time the end-to-end step (profiling captures: one launch per kernel and step)")
+    ap.add_argument("--skip-e2e-trace", action="store_true",
+                    help="do not time the end-to-end step that also delivers the trace to the host")
+    ap.add_argument("--skip-reports", action="store_true",
+                    help="leave out the study / sweep / packing-gap reports (profiling captures)")
+    ap.add_argument("--study", action="store_true",
+                    help="hybrid-vs-baseline study on this workload too (default: c2, c2e, paper)")
     ap.add_argument("--skip-cpu-baseline", action="store_true",
                     help="do not time the CPU oracle (profiling captures)")
     args = ap.parse_args()
