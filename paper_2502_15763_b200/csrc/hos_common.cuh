@@ -75,6 +75,31 @@ __device__ __forceinline__ unsigned long long block_max_u64(unsigned long long v
 
 __device__ __forceinline__ int bit_width_u32(uint32_t v) { return 32 - __clz(v); }
 
+// One pass of a CTA over the request tables of an instance: f(i, p_i, o_i, e_i, a_i) for every
+// request, four requests per thread and 16-byte loads when the rows allow it.  ei may be oi
+// itself (no separate estimates); ai may be null (then a_i = 0).
+template <typename F>
+__device__ __forceinline__ void for_each_request(const uint32_t* __restrict__ pi, const uint32_t* __restrict__ oi,
+                                                 const uint32_t* __restrict__ ei, const int32_t* __restrict__ ai,
+                                                 int n, F&& f) {
+    const uintptr_t bits = reinterpret_cast<uintptr_t>(pi) | reinterpret_cast<uintptr_t>(oi) |
+                           reinterpret_cast<uintptr_t>(ei) | reinterpret_cast<uintptr_t>(ai);
+    if ((n & 3) == 0 && (bits & 15) == 0) {
+        for (int i4 = threadIdx.x; i4 < (n >> 2); i4 += blockDim.x) {
+            const uint4 pv = __ldg(reinterpret_cast<const uint4*>(pi) + i4);
+            const uint4 ov = __ldg(reinterpret_cast<const uint4*>(oi) + i4);
+            const uint4 ev = ei != oi ? __ldg(reinterpret_cast<const uint4*>(ei) + i4) : ov;
+            const int4 av = ai ? __ldg(reinterpret_cast<const int4*>(ai) + i4) : make_int4(0, 0, 0, 0);
+            f(4 * i4 + 0, pv.x, ov.x, ev.x, av.x);
+            f(4 * i4 + 1, pv.y, ov.y, ev.y, av.y);
+            f(4 * i4 + 2, pv.z, ov.z, ev.z, av.z);
+            f(4 * i4 + 3, pv.w, ov.w, ev.w, av.w);
+        }
+    } else {
+        for (int i = threadIdx.x; i < n; i += blockDim.x) f(i, pi[i], oi[i], ei[i], ai ? ai[i] : 0);
+    }
+}
+
 // Duration of a prefill stage over `tokens` prompt tokens: affine, or by level (Eq. 5-7).
 __device__ __forceinline__ uint32_t prefill_us(const hos_cost_model& cm, uint32_t tokens) {
     if (cm.n_levels == 0) return cm.prefill_fixed_us + cm.prefill_per_token_us * tokens;

@@ -33,12 +33,17 @@ struct LbSums {
 __device__ __forceinline__ void lb_take(LbSums& a, const hos_cost_model& cm, int q_shift, uint32_t pp, uint32_t oo) {
     a.P += pp;
     a.O += oo;
-    a.K += (unsigned long long)oo * pp + (((unsigned long long)oo * (oo - 1u)) >> 1);
-    const unsigned long long alone = (unsigned long long)prefill_us(cm, pp) +
-                                     oo * ((unsigned long long)cm.decode_fixed_us + cm.decode_per_seq_us) +
-                                     floor_sum_below(pp + oo, cm.decode_kv_div, q_shift) -
-                                     floor_sum_below(pp, cm.decode_kv_div, q_shift);
-    a.chain = alone > a.chain ? alone : a.chain;
+    a.K += ((unsigned long long)oo * (2ull * pp + oo - 1ull)) >> 1;      // o p + o (o - 1) / 2
+    // the request served alone: a maximum, so the exact value (two floor sums) is only taken when
+    // an upper bound of it, sum of floor((p + s) / q) <= o (p + o) / q, beats the running maximum
+    const unsigned long long fixed = (unsigned long long)prefill_us(cm, pp) +
+                                     oo * ((unsigned long long)cm.decode_fixed_us + cm.decode_per_seq_us);
+    const unsigned long long kv_hi = (unsigned long long)oo * (pp + oo);
+    if (fixed + (q_shift >= 0 ? kv_hi >> q_shift : kv_hi / cm.decode_kv_div) > a.chain) {
+        const unsigned long long alone = fixed + floor_sum_below(pp + oo, cm.decode_kv_div, q_shift) -
+                                         floor_sum_below(pp, cm.decode_kv_div, q_shift);
+        a.chain = alone > a.chain ? alone : a.chain;
+    }
 }
 
 // One thread: the bounds of an instance from its sums.  pairT = T_(M) + T_(M+1), 0 when n_req <= M.
@@ -110,7 +115,7 @@ k_estimate_sort(const uint32_t* __restrict__ p, const uint32_t* __restrict__ o,
                 int n_pad) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     __shared__ unsigned long long red[32];
-    uint32_t* key = reinterpret_cast<uint32_t*>(smem_raw);
+    __shared__ uint32_t s_pair[2];                        // T_(M), T_(M+1)
     const uint32_t e_p = cm.est_per_prompt_token, e_o = cm.est_per_output_token;
     for (int inst = blockIdx.x; inst < n_inst; inst += gridDim.x) {
         if (!FAST) {
@@ -120,38 +125,22 @@ k_estimate_sort(const uint32_t* __restrict__ p, const uint32_t* __restrict__ o,
         const uint32_t* pi = p + (size_t)inst * n_req;
         const uint32_t* oi = o + (size_t)inst * n_req;
         const uint32_t* ei = o_est ? o_est + (size_t)inst * n_req : oi;   // the lengths the scheduler knows
+        uint32_t* key = reinterpret_cast<uint32_t*>(smem_raw);            // the radix path keeps T here
 
-        // kv_budget here is the most KV one request may need: the fixed reservation, if there is one
+        // first pass: checks, sums, the largest T (and the lower bounds' sums).  kv_budget here is
+        // the most KV one request may need: the fixed reservation, if there is one
         unsigned long long sum = 0, mx = 0, bad = 0;
         LbSums a = {0ull, 0ull, 0ull, 0ull};
-        auto take = [&](int i, uint32_t pp, uint32_t oo, uint32_t oe) {
+        for_each_request(pi, oi, ei, nullptr, n_req, [&](int i, uint32_t pp, uint32_t oo, uint32_t oe, int) {
             const unsigned long long t = (unsigned long long)e_p * pp + (unsigned long long)e_o * oe;
             if (pp == 0 || oo == 0 || oe == 0 || pp > p_max || (long long)pp + (long long)oo > kv_budget ||
                 t > 0xFFFFFFFFull)
                 bad = 1;
             else if (lb_out) lb_take(a, cm, q_shift, pp, oo);
-            key[i] = (uint32_t)t;
+            if (!FAST) key[i] = (uint32_t)t;
             sum += t;
             mx = t > mx ? t : mx;
-        };
-        // four requests per thread and read when the rows allow 16-byte loads
-        const bool vec = (n_req & 3) == 0 && ((reinterpret_cast<uintptr_t>(pi) | reinterpret_cast<uintptr_t>(oi) |
-                                               reinterpret_cast<uintptr_t>(ei)) & 15) == 0;
-        if (vec) {
-            const uint4* p4 = reinterpret_cast<const uint4*>(pi);
-            const uint4* o4 = reinterpret_cast<const uint4*>(oi);
-            const uint4* e4 = reinterpret_cast<const uint4*>(ei);
-            for (int i4 = threadIdx.x; i4 < (n_req >> 2); i4 += SORT_THREADS) {
-                const uint4 pv = __ldg(&p4[i4]), ov = __ldg(&o4[i4]);
-                const uint4 ev = o_est ? __ldg(&e4[i4]) : ov;
-                take(4 * i4 + 0, pv.x, ov.x, ev.x);
-                take(4 * i4 + 1, pv.y, ov.y, ev.y);
-                take(4 * i4 + 2, pv.z, ov.z, ev.z);
-                take(4 * i4 + 3, pv.w, ov.w, ev.w);
-            }
-        } else {
-            for (int i = threadIdx.x; i < n_req; i += SORT_THREADS) take(i, pi[i], oi[i], ei[i]);
-        }
+        });
         sum = block_sum_u64(sum, red);
         mx = block_max_u64(mx, red);
         bad = block_max_u64(bad, red);
@@ -174,20 +163,34 @@ k_estimate_sort(const uint32_t* __restrict__ p, const uint32_t* __restrict__ o,
         const uint32_t flip = nbits >= 32 ? 0xFFFFFFFFu : ((1u << nbits) - 1u);   // descending T
         uint32_t* Ts = T_sorted + (size_t)inst * n_pad;
         uint32_t* od = order + (size_t)inst * n_pad;
-        unsigned long long pairT = 0;
+        if (threadIdx.x < 2) s_pair[threadIdx.x] = 0;
         if (FAST) {
-            uint32_t* ent = reinterpret_cast<uint32_t*>(smem_raw + align16((size_t)n_req * 4));
-            uint32_t* cnt = reinterpret_cast<uint32_t*>(smem_raw + 2 * align16((size_t)n_req * 4));
-            if (!block_bucket_sort(key, ent, cnt, n_req, nbits, flip)) {
+            // two more passes over the tables (now in L2): count, then place; T is taken again
+            BucketSort B;
+            bool ok = bucket_sort_plan(B, smem_raw, n_req, nbits, 0);
+            if (ok) {
+                bucket_sort_clear(B);
+                for_each_request(pi, oi, ei, nullptr, n_req, [&](int, uint32_t pp, uint32_t, uint32_t oe, int) {
+                    bucket_sort_count(B, (e_p * pp + e_o * oe) ^ flip);
+                });
+                ok = bucket_sort_scan(B, n_req);
+            }
+            if (!ok) {
                 if (threadIdx.x == 0) info[inst].status = SORT_PENDING;
                 continue;
             }
-            for (int r = threadIdx.x; r < n_req; r += SORT_THREADS) {
-                const uint32_t id = ent[r];
+            for_each_request(pi, oi, ei, nullptr, n_req, [&](int i, uint32_t pp, uint32_t, uint32_t oe, int) {
+                bucket_sort_place(B, (e_p * pp + e_o * oe) ^ flip, (uint32_t)i, 0u);
+            });
+            __syncthreads();
+            for (int s = threadIdx.x; s < n_req; s += SORT_THREADS) {
+                uint32_t fk, id, extra;
+                const uint32_t r = bucket_sort_rank(B, s, fk, id, extra);
+                const uint32_t T = fk ^ flip;             // T < 2^nbits: the flip is its own inverse there
                 od[r] = id;
-                Ts[r] = key[id];
+                Ts[r] = T;
+                if (r + 1 == (uint32_t)n_clients || r == (uint32_t)n_clients) s_pair[r + 1 - n_clients] = T;
             }
-            if (n_req > n_clients) pairT = (unsigned long long)key[ent[n_clients - 1]] + key[ent[n_clients]];
         } else {
             SortSmem<uint16_t> s = sort_smem_carve<uint16_t>(smem_raw, n_req);
             const uint16_t* sorted = block_radix_sort_ids<uint16_t>(s, n_req, nbits, flip);
@@ -195,11 +198,13 @@ k_estimate_sort(const uint32_t* __restrict__ p, const uint32_t* __restrict__ o,
                 const uint32_t id = sorted[r];
                 od[r] = id;
                 Ts[r] = key[id];
+                if (r + 1 == n_clients || r == n_clients) s_pair[r + 1 - n_clients] = key[id];
             }
-            if (n_req > n_clients) pairT = (unsigned long long)key[sorted[n_clients - 1]] + key[sorted[n_clients]];
         }
+        __syncthreads();
         if (threadIdx.x == 0) {
             int32_t st = 0;
+            const unsigned long long pairT = n_req > n_clients ? (unsigned long long)s_pair[0] + s_pair[1] : 0ull;
             if (lb_out) lb_finish(a, cm, n_req, n_clients, cap, sum, mx, pairT, &lb_out[inst], &st);
             info[inst].sum_T = sum; info[inst].max_T = (uint32_t)mx; info[inst].status = 0;
             if (status_out) status_out[inst] = st;

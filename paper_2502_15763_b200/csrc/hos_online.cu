@@ -33,9 +33,7 @@ k_queue_build(const uint32_t* __restrict__ p, const uint32_t* __restrict__ o,
               int32_t* __restrict__ inst_status, int n_pad) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     __shared__ unsigned long long red[32];
-    uint32_t* key = reinterpret_cast<uint32_t*>(smem_raw);
-    // the clients wait here until the keys are composed (the sort's own buffer, not yet in use)
-    uint32_t* park = reinterpret_cast<uint32_t*>(smem_raw + align16((size_t)n_req * 4));
+    const int cbits = bit_width_u32((uint32_t)(n_clients - 1));
     for (int inst = blockIdx.x; inst < n_inst; inst += gridDim.x) {
         if (!FAST) {
             __syncthreads();
@@ -45,39 +43,25 @@ k_queue_build(const uint32_t* __restrict__ p, const uint32_t* __restrict__ o,
         const uint32_t* oi = o + (size_t)inst * n_req;
         const int32_t* ai = assign + (size_t)inst * n_req;
         const uint32_t* ei = o_est ? o_est + (size_t)inst * n_req : oi;   // the lengths the scheduler sorts by
+        // the radix path keeps the keys here, and the clients beside them until the keys are composed
+        uint32_t* key = reinterpret_cast<uint32_t*>(smem_raw);
+        uint16_t* park = reinterpret_cast<uint16_t*>(smem_raw + align16((size_t)n_req * 4));
 
-        // kv_budget here is the most KV one request may need: the fixed reservation, if there is one
+        // first pass: checks and sums.  kv_budget here is the most KV one request may need: the
+        // fixed reservation, if there is one
         unsigned long long sumO = 0, mx = 0, mxk = 0, mxp = 0, bad = 0;
-        auto take = [&](int i, uint32_t pp, uint32_t oo, uint32_t oe, int c) {
+        for_each_request(pi, oi, ei, ai, n_req, [&](int i, uint32_t pp, uint32_t oo, uint32_t oe, int c) {
             const unsigned long long tot = (unsigned long long)pp + oo;
             const unsigned long long totk = (unsigned long long)pp + oe;
             if (pp == 0 || oo == 0 || oe == 0 || pp > p_max || (long long)tot > kv_budget || totk > 0xFFFFFFFFull ||
                 c < 0 || c >= n_clients)
                 bad = 1;
-            key[i] = (uint32_t)totk;
-            if (FAST) park[i] = (uint32_t)(c & 0xFF);
-            else reinterpret_cast<uint16_t*>(park)[i] = (uint16_t)(c & 0xFF);
+            if (!FAST) { key[i] = (uint32_t)totk; park[i] = (uint16_t)(c & 0xFF); }
             sumO += oo;
             mx = tot > mx ? tot : mx;
             mxk = totk > mxk ? totk : mxk;
             mxp = pp > mxp ? pp : mxp;
-        };
-        const bool vec = (n_req & 3) == 0 && ((reinterpret_cast<uintptr_t>(pi) | reinterpret_cast<uintptr_t>(oi) |
-                                               reinterpret_cast<uintptr_t>(ei) | reinterpret_cast<uintptr_t>(ai)) & 15) == 0;
-        if (vec) {
-            for (int i4 = threadIdx.x; i4 < (n_req >> 2); i4 += SORT_THREADS) {
-                const uint4 pv = __ldg(reinterpret_cast<const uint4*>(pi) + i4);
-                const uint4 ov = __ldg(reinterpret_cast<const uint4*>(oi) + i4);
-                const uint4 ev = o_est ? __ldg(reinterpret_cast<const uint4*>(ei) + i4) : ov;
-                const int4 av = __ldg(reinterpret_cast<const int4*>(ai) + i4);
-                take(4 * i4 + 0, pv.x, ov.x, ev.x, av.x);
-                take(4 * i4 + 1, pv.y, ov.y, ev.y, av.y);
-                take(4 * i4 + 2, pv.z, ov.z, ev.z, av.z);
-                take(4 * i4 + 3, pv.w, ov.w, ev.w, av.w);
-            }
-        } else {
-            for (int i = threadIdx.x; i < n_req; i += SORT_THREADS) take(i, pi[i], oi[i], ei[i], ai[i]);
-        }
+        });
         sumO = block_sum_u64(sumO, red);
         mx = block_max_u64(mx, red);
         mxk = block_max_u64(mxk, red);
@@ -87,7 +71,7 @@ k_queue_build(const uint32_t* __restrict__ p, const uint32_t* __restrict__ o,
         const int kb = (queue_order == HOS_QUEUE_SORTED) ? bit_width_u32((uint32_t)mxk) : 0;
         // the composite sort key, client above p + (estimated) o, has 32 bits: an estimate so long
         // that it does not fit beside the client bits invalidates the instance (uniform over the CTA)
-        if (kb + bit_width_u32((uint32_t)(n_clients - 1)) > 32) bad = 1;
+        if (kb + cbits > 32) bad = 1;
         // bit 8 (internal): some p + o needs more than 16 bits -> the simulator's wide heap entries
         const int32_t st_done = bad ? HOS_ST_INVALID : (mx >= 65536ull ? INST_WIDE : 0);
         if (bad) {
@@ -95,23 +79,69 @@ k_queue_build(const uint32_t* __restrict__ p, const uint32_t* __restrict__ o,
             continue;
         }
         const uint32_t kmask = kb >= 32 ? 0xFFFFFFFFu : ((1u << kb) - 1u);
-        const int nbits = kb + bit_width_u32((uint32_t)(n_clients - 1));
-        // The sort only looks at the low nbits of a key.  When the prompt length fits the bits above
-        // them it rides along there, so that the queue entries are written without going back to the
-        // request tables in queue order (a scattered read per request); with the key p + o the
-        // output length follows from it too.
-        const bool ride = nbits + bit_width_u32((uint32_t)mxp) <= 32;
-        const bool o_from_key = ride && kb > 0 && kb < 32 && !o_est;
-        for (int i = threadIdx.x; i < n_req; i += SORT_THREADS) {
-            const uint32_t c = FAST ? park[i] : (uint32_t)reinterpret_cast<uint16_t*>(park)[i];
-            const uint32_t low = (kb >= 32 ? 0u : (c << kb)) | (kmask - (key[i] & kmask));
-            key[i] = ride ? (low | (nbits >= 32 ? 0u : (pi[i] << nbits))) : low;
-        }
-        __syncthreads();
         uint2* qp = q_po + (size_t)inst * n_pad;
         uint32_t* qr = q_req + (size_t)inst * n_pad;
+        uint32_t* qk = q_key ? q_key + (size_t)inst * n_pad : nullptr;
         int32_t* qo = q_off + (size_t)inst * (n_clients + 1);
-        auto write_out = [&](auto sorted) {
+        if (FAST) {
+            // Sort key: the client above the length key 2^kb - 1 - (p + o) (longest first), or above
+            // the request index for first-come-first-served queues; ties never arise beyond the
+            // index.  The prompt length rides in an entry's spare bits when it fits, so that the queue
+            // entries are written without going back to the request tables in queue order (a
+            // scattered read per request); with the key p + o the output length follows from it too.
+            const bool by_len = kb > 0;
+            const int sbits = by_len ? kb : (n_req > 1 ? bit_width_u32((uint32_t)(n_req - 1)) : 1);
+            const int nbits = sbits + cbits;             // <= 32 (checked above; 15 + 8 for the index form)
+            BucketSort B;
+            const int pbits = bit_width_u32((uint32_t)mxp);
+            bool ok = bucket_sort_plan(B, smem_raw, n_req, nbits, pbits);
+            const bool ride = ok;
+            if (!ok) ok = bucket_sort_plan(B, smem_raw, n_req, nbits, 0);
+            const bool o_from_key = ride && by_len && kb < 32 && !o_est;
+            auto sort_key = [&](int i, uint32_t pp, uint32_t oe, int c) -> uint32_t {
+                const uint32_t low = by_len ? kmask - ((pp + oe) & kmask) : (uint32_t)i;
+                return (sbits >= 32 ? 0u : ((uint32_t)c << sbits)) | low;
+            };
+            if (ok) {
+                bucket_sort_clear(B);
+                for_each_request(pi, oi, ei, ai, n_req, [&](int i, uint32_t pp, uint32_t, uint32_t oe, int c) {
+                    bucket_sort_count(B, sort_key(i, pp, oe, c));
+                });
+                ok = bucket_sort_scan(B, n_req);
+            }
+            if (!ok) {
+                if (threadIdx.x == 0) inst_status[inst] = INST_PENDING;
+                continue;
+            }
+            // the clients' bits are the top bits of the bucket number: a queue starts where its first bucket does
+            for (int c = threadIdx.x; c <= n_clients; c += SORT_THREADS)
+                qo[c] = c < n_clients ? (int32_t)bucket_sort_start(B, (uint32_t)c << (B.bbits - cbits)) : n_req;
+            __syncthreads();
+            for_each_request(pi, oi, ei, ai, n_req, [&](int i, uint32_t pp, uint32_t, uint32_t oe, int c) {
+                bucket_sort_place(B, sort_key(i, pp, oe, c), (uint32_t)i, ride ? pp : 0u);
+            });
+            __syncthreads();
+            for (int s = threadIdx.x; s < n_req; s += SORT_THREADS) {
+                uint32_t k, id, extra;
+                const uint32_t r = bucket_sort_rank(B, s, k, id, extra);
+                const uint32_t pp = ride ? extra : pi[id];
+                const uint32_t totk = by_len ? kmask - (k & kmask) : 0u;     // p + (estimated) o, when it is the key
+                qr[r] = id;
+                qp[r] = make_uint2(pp, o_from_key ? totk - pp : oi[id]);
+                if (qk) qk[r] = (by_len && kb < 32) ? totk : pp + ei[id];
+            }
+        } else {
+            const int nbits = kb + cbits;
+            const bool ride = nbits + bit_width_u32((uint32_t)mxp) <= 32;
+            const bool o_from_key = ride && kb > 0 && kb < 32 && !o_est;
+            for (int i = threadIdx.x; i < n_req; i += SORT_THREADS) {
+                const uint32_t c = (uint32_t)park[i];
+                const uint32_t low = (kb >= 32 ? 0u : (c << kb)) | (kmask - (key[i] & kmask));
+                key[i] = ride ? (low | (nbits >= 32 ? 0u : (pi[i] << nbits))) : low;
+            }
+            __syncthreads();
+            SortSmem<uint16_t> ss = sort_smem_carve<uint16_t>(smem_raw, n_req);
+            const uint16_t* sorted = block_radix_sort_ids<uint16_t>(ss, n_req, nbits, 0u);
             for (int r = threadIdx.x; r < n_req; r += SORT_THREADS) {
                 const uint32_t id = sorted[r];
                 const uint32_t kw = key[id];
@@ -120,7 +150,7 @@ k_queue_build(const uint32_t* __restrict__ p, const uint32_t* __restrict__ o,
                 const uint32_t totk = kmask - (low & kmask);             // p + (estimated) o, when it is the key
                 qr[r] = id;
                 qp[r] = make_uint2(pp, o_from_key ? totk - pp : oi[id]);
-                if (q_key) q_key[(size_t)inst * n_pad + r] = kb > 0 && kb < 32 ? totk : pp + ei[id];
+                if (qk) qk[r] = kb > 0 && kb < 32 ? totk : pp + ei[id];
                 const int c = kb >= 32 ? 0 : (int)(low >> kb);            // 32 key bits leave none for the client: one client
                 const uint32_t kprev = r > 0 ? key[sorted[r - 1]] : 0u;
                 const int cprev = r > 0 ? (kb >= 32 ? 0 : (int)(((ride && nbits < 32) ? (kprev & ((1u << nbits) - 1u)) : kprev) >> kb)) : -1;
@@ -128,17 +158,6 @@ k_queue_build(const uint32_t* __restrict__ p, const uint32_t* __restrict__ o,
                 if (r == n_req - 1)
                     for (int cc = c + 1; cc <= n_clients; ++cc) qo[cc] = n_req;
             }
-        };
-        if (FAST) {
-            uint32_t* cnt = reinterpret_cast<uint32_t*>(smem_raw + 2 * align16((size_t)n_req * 4));
-            if (!block_bucket_sort(key, park, cnt, n_req, nbits, 0u)) {
-                if (threadIdx.x == 0) inst_status[inst] = INST_PENDING;
-                continue;
-            }
-            write_out(park);
-        } else {
-            SortSmem<uint16_t> s = sort_smem_carve<uint16_t>(smem_raw, n_req);
-            write_out(block_radix_sort_ids<uint16_t>(s, n_req, nbits, 0u));
         }
         if (threadIdx.x == 0) { inst_O[inst] = sumO; inst_status[inst] = st_done; }
     }

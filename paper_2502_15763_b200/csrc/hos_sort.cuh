@@ -182,31 +182,34 @@ __device__ inline IdxT* block_radix_sort_ids(const SortSmem<IdxT>& s, int n, int
 
 
 // ---------------------------------------------------------------------------------------
-// Bucket sort of item ids by the same keys, for keys that spread out (the usual case).
+// Bucket sort of items by a 32-bit key, for keys that spread out (the usual case).
 //
-// The order wanted -- (key ^ flip) ascending over its low `nbits` bits, then id ascending -- is a
-// total order of distinct pairs, so it does not matter in which order the items of a bucket
-// arrive: the top bits of the key choose a bucket (shared-memory histogram, scan, scatter by
-// atomic slot counters), every bucket entry is the rest of the key above the id in one 32-bit
-// word, and an item's final position is its bucket's start plus the number of entries of that
-// bucket below its own.  With about two buckets per item and keys that spread over them this
-// is a few compares per item instead of a ranking vote per key bit and pass.  The counters are
-// 16 bits wide, two to a word (no count or offset reaches 2^16), which buys twice the buckets
-// for the shared memory.  Returns false, with nothing written, when the entries do not fit 32
+// The order wanted -- key ascending over its low `nbits` bits, then id ascending -- is a total
+// order of distinct pairs, so it does not matter in which order the items of a bucket arrive:
+// the top bits of the key choose a bucket (shared-memory histogram, scan, scatter by atomic slot
+// counters); a bucket entry is the rest of the key above the id (and, below both, whatever
+// the caller wants to carry along) in one 32-bit word, with the bucket number in a 16-bit table
+// beside it; and an item's final position is its bucket's start plus the number of entries of
+// that bucket below its own.  Ranks are taken in SLOT order: the 32 lanes of a warp look at
+// neighbouring buckets, so their reads of a bucket's entries fall on the same or on
+// neighbouring words (no bank conflicts, equal trip counts), and their results land on
+// neighbouring positions, so the caller can write them straight to global memory.  With about
+// two buckets per item this is a few compares per item instead of a ranking vote per key bit
+// and pass.  The counters are 16 bits wide, two to a word (no count or offset reaches 2^16).
+// The keys themselves are not kept in shared memory: the caller passes over its data once to
+// count and once to place (bucket_sort_count / bucket_sort_place).
+//
+// The sort declines (plan or scan return false, nothing written) when an entry does not fit 32
 // bits or the buckets are so uneven that the compares would cost more than the radix passes
 // (sum of squared bucket sizes above BUCKET_WORK_MAX per item); the caller then takes
-// block_radix_sort_ids.
-//
-// One CTA of SORT_THREADS threads; key[n] in shared memory; `ent` n words and `cntw`
-// 2^(bucket bits - 1) words of shared memory.  On success ent[r] is the id of the item of rank r.
+// block_radix_sort_ids.  One CTA of SORT_THREADS threads.
 // ---------------------------------------------------------------------------------------
 constexpr int BUCKET_BITS_MAX = 15;
 constexpr int BUCKET_WORK_MAX = 96;
-constexpr int BUCKET_ITEMS_PER_THREAD = (MAX_REQ + SORT_THREADS - 1) / SORT_THREADS;   // 24
 
-// Most bucket bits whose counters fit beside the two n-word arrays (host and device agree on it).
+// Most bucket bits whose counters fit beside the entry and bucket tables (host and device agree).
 __host__ __device__ inline int bucket_bits_cap(int n) {
-    const size_t room = SMEM_LIMIT - 2048 - 2 * align16(size_t(n) * 4);      // 2 KB left for static shared memory
+    const size_t room = SMEM_LIMIT - 2048 - align16(size_t(n) * 4) - align16(size_t(n) * 2);   // 2 KB for static shared memory
     int bb = BUCKET_BITS_MAX;
     while (bb > 10 && (size_t(2) << bb) > room) --bb;
     int want = 11;                                                           // about two buckets per item
@@ -214,93 +217,111 @@ __host__ __device__ inline int bucket_bits_cap(int n) {
     return bb < want ? bb : want;
 }
 __host__ __device__ inline size_t bucket_sort_smem_bytes(int n) {
-    return 2 * align16(size_t(n) * 4) + (size_t(2) << bucket_bits_cap(n));
+    return align16(size_t(n) * 4) + align16(size_t(n) * 2) + (size_t(2) << bucket_bits_cap(n));
 }
 
-__device__ inline bool block_bucket_sort(const uint32_t* key, uint32_t* ent, uint32_t* cntw, int n, int nbits,
-                                         uint32_t flip) {
+struct BucketSort {
+    int bbits, low_bits, id_bits, xbits, n_words;
+    uint32_t kmask, lmask;
+    uint32_t* ent;              // [n]  (rest of key << id_bits | id) << xbits | extra, in slot order
+    uint16_t* bkt;              // [n]  bucket of every slot
+    uint32_t* cntw;             // [2^(bbits-1)] two 16-bit counters per word
+};
+
+// Layout and bit budget for n items with `nbits` significant key bits and `xbits` extra bits per
+// entry.  False when an entry does not fit.  Uniform over the CTA.
+__device__ inline bool bucket_sort_plan(BucketSort& B, unsigned char* smem, int n, int nbits, int xbits) {
+    B.bbits = max(1, min(nbits, bucket_bits_cap(n)));
+    B.low_bits = max(0, nbits - B.bbits);
+    B.id_bits = n > 1 ? bit_width_u32((uint32_t)(n - 1)) : 1;
+    B.xbits = xbits;
+    B.n_words = 1 << (B.bbits - 1);
+    B.kmask = nbits >= 32 ? 0xFFFFFFFFu : ((1u << nbits) - 1u);
+    B.lmask = B.low_bits >= 32 ? 0xFFFFFFFFu : ((1u << B.low_bits) - 1u);
+    B.ent = reinterpret_cast<uint32_t*>(smem);
+    B.bkt = reinterpret_cast<uint16_t*>(smem + align16(size_t(n) * 4));
+    B.cntw = reinterpret_cast<uint32_t*>(smem + align16(size_t(n) * 4) + align16(size_t(n) * 2));
+    return B.low_bits + B.id_bits + xbits <= 32;
+}
+
+// Zeroes the counters.  Ends with a __syncthreads().
+__device__ inline void bucket_sort_clear(const BucketSort& B) {
+    for (int i = threadIdx.x; i < B.n_words; i += SORT_THREADS) B.cntw[i] = 0;
+    __syncthreads();
+}
+
+__device__ __forceinline__ void bucket_sort_count(const BucketSort& B, uint32_t key) {
+    const uint32_t b = (key & B.kmask) >> B.low_bits;
+    atomicAdd(&B.cntw[b >> 1], 1u << ((b & 1u) << 4));
+}
+
+// Exclusive scan of the bucket counts (after every bucket_sort_count).  Starts and ends with a
+// __syncthreads().  False when the buckets are too uneven.
+__device__ inline bool bucket_sort_scan(const BucketSort& B, int n) {
     __shared__ uint32_t s_wsum[SORT_WARPS];
     __shared__ unsigned long long s_work;
     const int t = threadIdx.x;
-    const int bbits = max(1, min(nbits, bucket_bits_cap(n)));
-    const int low_bits = max(0, nbits - bbits);
-    const int id_bits = n > 1 ? bit_width_u32((uint32_t)(n - 1)) : 1;
-    if (low_bits + id_bits > 32) return false;                      // uniform: same arguments in every thread
-    const uint32_t kmask = nbits >= 32 ? 0xFFFFFFFFu : ((1u << nbits) - 1u);
-    const uint32_t lmask = (1u << low_bits) - 1u;                   // low_bits <= 31 here
-    const int n_words = 1 << (bbits - 1);                           // two counters per word
-    const uint16_t* cnt16 = reinterpret_cast<const uint16_t*>(cntw);
-    for (int i = t; i < n_words; i += SORT_THREADS) cntw[i] = 0;
     if (t == 0) s_work = 0;
     __syncthreads();
-    for (int i = t; i < n; i += SORT_THREADS) {
-        const uint32_t b = ((key[i] ^ flip) & kmask) >> low_bits;
-        atomicAdd(&cntw[b >> 1], 1u << ((b & 1u) << 4));
+    const int per = (B.n_words + SORT_THREADS - 1) / SORT_THREADS;   // consecutive words per thread
+    const int w0 = min(B.n_words, t * per), w1 = min(B.n_words, w0 + per);
+    uint32_t run = 0;
+    unsigned long long work = 0;
+    for (int w = w0; w < w1; ++w) {
+        const uint32_t c = B.cntw[w], a = c & 0xFFFFu, b = c >> 16;
+        run += a + b;
+        work += (unsigned long long)(a * a + b * b);
     }
-    __syncthreads();
-    {   // exclusive scan of the bucket counts: consecutive words per thread
-        const int per = (n_words + SORT_THREADS - 1) / SORT_THREADS;
-        const int w0 = min(n_words, t * per), w1 = min(n_words, w0 + per);
-        uint32_t run = 0;
-        unsigned long long work = 0;
-        for (int w = w0; w < w1; ++w) {
-            const uint32_t c = cntw[w], a = c & 0xFFFFu, b = c >> 16;
-            run += a + b;
-            work += (unsigned long long)(a * a + b * b);
-        }
-        uint32_t inc = run;
+    uint32_t inc = run;
 #pragma unroll
-        for (int d = 1; d < 32; d <<= 1) {
-            const uint32_t y = __shfl_up_sync(FULL, inc, d);
-            if (lane_id() >= d) inc += y;
-        }
-        work = warp_sum_u64(work);
-        if (lane_id() == 31) s_wsum[warp_id()] = inc;
-        if (lane_id() == 0 && work) atomicAdd(&s_work, work);
-        __syncthreads();
-        const uint32_t wv = s_wsum[lane_id()];
-        uint32_t acc = __reduce_add_sync(FULL, lane_id() < warp_id() ? wv : 0u) + inc - run;
-        for (int w = w0; w < w1; ++w) {
-            const uint32_t c = cntw[w], a = c & 0xFFFFu, b = c >> 16;
-            cntw[w] = acc | ((acc + a) << 16);
-            acc += a + b;
-        }
-        __syncthreads();
+    for (int d = 1; d < 32; d <<= 1) {
+        const uint32_t y = __shfl_up_sync(FULL, inc, d);
+        if (lane_id() >= d) inc += y;
     }
-    if (s_work > (unsigned long long)BUCKET_WORK_MAX * (unsigned long long)n) return false;   // uniform
-    // scatter: counter b walks from the start of bucket b to its end
-    for (int i = t; i < n; i += SORT_THREADS) {
-        const uint32_t fk = (key[i] ^ flip) & kmask;
-        const uint32_t b = fk >> low_bits, sh = (b & 1u) << 4;
-        const uint32_t slot = (atomicAdd(&cntw[b >> 1], 1u << sh) >> sh) & 0xFFFFu;
-        ent[slot] = ((fk & lmask) << id_bits) | (uint32_t)i;
+    work = warp_sum_u64(work);
+    if (lane_id() == 31) s_wsum[warp_id()] = inc;
+    if (lane_id() == 0 && work) atomicAdd(&s_work, work);
+    __syncthreads();
+    const uint32_t wv = s_wsum[lane_id()];
+    uint32_t acc = __reduce_add_sync(FULL, lane_id() < warp_id() ? wv : 0u) + inc - run;
+    for (int w = w0; w < w1; ++w) {
+        const uint32_t c = B.cntw[w], a = c & 0xFFFFu, b = c >> 16;
+        B.cntw[w] = acc | ((acc + a) << 16);
+        acc += a + b;
     }
     __syncthreads();
-    // rank of every item inside its bucket; the ranks wait in registers until all reads are done
-    uint32_t rank[BUCKET_ITEMS_PER_THREAD];
-#pragma unroll
-    for (int e = 0; e < BUCKET_ITEMS_PER_THREAD; ++e) {
-        const int i = t + e * SORT_THREADS;
-        rank[e] = 0;
-        if (i < n) {
-            const uint32_t fk = (key[i] ^ flip) & kmask;
-            const uint32_t b = fk >> low_bits;
-            const uint32_t mine = ((fk & lmask) << id_bits) | (uint32_t)i;
-            const uint32_t start = b ? cnt16[b - 1] : 0u, end = cnt16[b];
-            uint32_t r = start, s2 = start;
-            for (; s2 + 1 < end; s2 += 2) r += (ent[s2] < mine ? 1u : 0u) + (ent[s2 + 1] < mine ? 1u : 0u);
-            if (s2 < end) r += ent[s2] < mine ? 1u : 0u;
-            rank[e] = r;
-        }
-    }
-    __syncthreads();
-#pragma unroll
-    for (int e = 0; e < BUCKET_ITEMS_PER_THREAD; ++e) {
-        const int i = t + e * SORT_THREADS;
-        if (i < n) ent[rank[e]] = (uint32_t)i;
-    }
-    __syncthreads();
-    return true;
+    return s_work <= (unsigned long long)BUCKET_WORK_MAX * (unsigned long long)n;
+}
+
+// First slot of bucket b; valid between bucket_sort_scan and the first bucket_sort_place.
+__device__ __forceinline__ uint32_t bucket_sort_start(const BucketSort& B, uint32_t b) {
+    return reinterpret_cast<const uint16_t*>(B.cntw)[b];
+}
+
+// Scatter: the counter of the item's bucket walks from the bucket's start to its end.
+__device__ __forceinline__ void bucket_sort_place(const BucketSort& B, uint32_t key, uint32_t id, uint32_t extra) {
+    const uint32_t fk = key & B.kmask;
+    const uint32_t b = fk >> B.low_bits, sh = (b & 1u) << 4;
+    const uint32_t slot = (atomicAdd(&B.cntw[b >> 1], 1u << sh) >> sh) & 0xFFFFu;
+    B.ent[slot] = ((((fk & B.lmask) << B.id_bits) | id) << B.xbits) | extra;
+    B.bkt[slot] = (uint16_t)b;
+}
+
+// Final position of the item in slot s (after every bucket_sort_place and a __syncthreads());
+// its key, id and extra bits come back through the references.
+__device__ __forceinline__ uint32_t bucket_sort_rank(const BucketSort& B, int s, uint32_t& key, uint32_t& id,
+                                                     uint32_t& extra) {
+    const uint16_t* cnt16 = reinterpret_cast<const uint16_t*>(B.cntw);
+    const uint32_t mine = B.ent[s], b = B.bkt[s];
+    const uint32_t start = b ? cnt16[b - 1] : 0u, end = cnt16[b];
+    uint32_t r = start, j = start;
+    for (; j + 1 < end; j += 2) r += (B.ent[j] < mine ? 1u : 0u) + (B.ent[j + 1] < mine ? 1u : 0u);
+    if (j < end) r += B.ent[j] < mine ? 1u : 0u;
+    const uint32_t body = B.xbits >= 32 ? 0u : mine >> B.xbits;
+    extra = B.xbits >= 32 ? mine : (mine & ((1u << B.xbits) - 1u));
+    id = body & ((1u << B.id_bits) - 1u);                       // id_bits <= 15 for any supported n
+    key = (b << B.low_bits) | (B.id_bits >= 32 ? 0u : body >> B.id_bits);
+    return r;
 }
 
 }  // namespace hos
