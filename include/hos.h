@@ -322,6 +322,16 @@ const char* hos_strerror(int code);
  * and not thread-safe: set it only while no other thread is inside the library; pass NULL
  * to remove it.  It is never consulted for any decision of the hot path.
  */
+/*
+ * Memory-safety aid (no counterpart in the paper).  The library can be built with
+ * -DHOS_DEBUG_BOUNDS (libhos_debug.so): every data-dependent index into shared or global
+ * memory is then checked, an index out of range is counted and its access skipped -- nothing
+ * faults -- and this call synchronises the device and returns the number of violations on the
+ * current device since the library was loaded (first, nullable: {site number, index, limit} of
+ * the first one).  The ordinary build has no checks and returns -1.
+ */
+long long hos_debug_bounds_violations(long long* first);
+
 typedef void (*hos_launch_hook)(const char* kernel, int phase, void* stream, void* user);
 void hos_set_launch_hook(hos_launch_hook hook, void* user);
 

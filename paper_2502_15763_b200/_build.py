@@ -10,6 +10,7 @@ _ROOT = os.path.dirname(_PKG)
 CSRC = os.path.join(_PKG, "csrc")
 INCLUDE = os.path.join(_ROOT, "include")
 LIB_PATH = os.path.join(_PKG, "libhos.so")
+DEBUG_LIB_PATH = os.path.join(_PKG, "libhos_debug.so")   # the bounds-checked build (-DHOS_DEBUG_BOUNDS)
 
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-shared", "-Xcompiler", "-fPIC", "--expt-relaxed-constexpr"]
@@ -36,26 +37,29 @@ def source_hash() -> str:
     return h.hexdigest()
 
 
-def is_stale() -> bool:
-    if not os.path.exists(LIB_PATH):
+def is_stale(debug: bool = False) -> bool:
+    path = DEBUG_LIB_PATH if debug else LIB_PATH
+    if not os.path.exists(path):
         return True
-    t = os.path.getmtime(LIB_PATH)
+    t = os.path.getmtime(path)
     return any(os.path.getmtime(f) > t for f in _deps())
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
-    """Compile every .cu under csrc/ into libhos.so; returns its path."""
-    if not force and not is_stale():
-        return LIB_PATH
+def build(force: bool = False, verbose: bool = False, debug: bool = False) -> str:
+    """Compile every .cu under csrc/ into libhos.so (debug: the bounds-checked libhos_debug.so);
+    returns its path."""
+    path = DEBUG_LIB_PATH if debug else LIB_PATH
+    if not force and not is_stale(debug):
+        return path
     nvcc = os.environ.get("NVCC", "nvcc")
-    tmp = LIB_PATH + f".{os.getpid()}.tmp"
-    cmd = [nvcc] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + \
+    tmp = path + f".{os.getpid()}.tmp"
+    cmd = [nvcc] + NVCC_FLAGS + (["-DHOS_DEBUG_BOUNDS"] if debug else []) + (["-Xptxas", "-v"] if verbose else []) + \
         ["-I", INCLUDE, "-I", CSRC, "-o", tmp] + _sources()
     subprocess.check_call(cmd)
-    os.replace(tmp, LIB_PATH)
-    return LIB_PATH
+    os.replace(tmp, path)
+    return path
 
 
 if __name__ == "__main__":
     import sys
-    print(build(force=True, verbose="-v" in sys.argv))
+    print(build(force=True, verbose="-v" in sys.argv, debug="--debug" in sys.argv))

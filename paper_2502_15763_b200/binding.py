@@ -32,7 +32,7 @@ _SYMBOLS = ("hos_offline_pack", "hos_local_search", "hos_lower_bound", "hos_onli
             "hos_trace_offsets", "hos_offline_workspace_bytes", "hos_lower_bound_workspace_bytes",
             "hos_online_workspace_bytes", "hos_strerror", "hos_set_launch_hook",
             "hos_lower_bound_static", "hos_trace_fill", "hos_online_simulate_steal",
-            "hos_offline_pack_multifit")
+            "hos_offline_pack_multifit", "hos_debug_bounds_violations")
 
 LAUNCH_HOOK = C.CFUNCTYPE(None, C.c_char_p, C.c_int, C.c_void_p, C.c_void_p)
 
@@ -65,12 +65,16 @@ def lib_path() -> str:
 
 
 def lib():
-    """Load libhos.so (building it first if the sources are newer).  Raises if it cannot be had."""
+    """Load libhos.so (building it first if the sources are newer).  Raises if it cannot be had.
+    With HOS_LIB_VARIANT=debug in the environment the bounds-checked build libhos_debug.so is
+    loaded instead (see hos_debug_bounds_violations)."""
     global _lib
     if _lib is None:
         from . import _build
-        path = _build.build() if _build.is_stale() else lib_path()
+        debug = os.environ.get("HOS_LIB_VARIANT", "") == "debug"
+        path = _build.build(debug=debug)
         L = C.CDLL(path)
+        L.hos_debug_bounds_violations.restype = C.c_longlong
         for name in ("hos_offline_workspace_bytes", "hos_lower_bound_workspace_bytes",
                      "hos_online_workspace_bytes"):
             getattr(L, name).restype = C.c_size_t
@@ -94,6 +98,14 @@ def hos_set_launch_hook(fn):
     cb = LAUNCH_HOOK(fn)
     L.hos_set_launch_hook(cb, None)
     return cb
+
+
+def hos_debug_bounds_violations():
+    """(count, (site, index, limit) of the first) out-of-range indexes caught by the bounds-checked
+    build on the current device since it was loaded; count is -1 in the ordinary build."""
+    first = (C.c_longlong * 3)()
+    n = lib().hos_debug_bounds_violations(first)
+    return int(n), tuple(int(x) for x in first)
 
 
 def exported_symbols() -> Sequence[str]:

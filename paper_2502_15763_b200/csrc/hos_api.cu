@@ -354,6 +354,22 @@ int hos_trace_offsets(const hos_client_result* cres, int64_t n_units, int64_t* t
                                         static_cast<cudaStream_t>(stream)));
 }
 
+long long hos_debug_bounds_violations(long long* first) {
+#ifdef HOS_DEBUG_BOUNDS
+    unsigned long long count = 0;
+    long long f[3] = {0, 0, 0};
+    if (cudaDeviceSynchronize() != cudaSuccess) return HOS_E_CUDA;
+    debug_bounds_offline(&count, f);
+    debug_bounds_online(&count, f);
+    debug_bounds_multifit(&count, f);
+    if (first) { first[0] = f[0]; first[1] = f[1]; first[2] = f[2]; }
+    return (long long)count;
+#else
+    (void)first;
+    return -1;
+#endif
+}
+
 void hos_set_launch_hook(hos_launch_hook hook, void* user) {
     g_hook = hook;
     g_hook_user = user;

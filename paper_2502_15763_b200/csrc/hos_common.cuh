@@ -25,6 +25,41 @@ struct InstInfo {
     int32_t status;
 };
 
+// ---------------------------------------------------------------------------------------
+// Bounds-checked build (-DHOS_DEBUG_BOUNDS; libhos_debug.so).  Every data-dependent index into
+// shared or global memory goes through HOS_IN(index, limit, site): in the ordinary build it is
+// the constant `true`; in the checked build an index outside [0, limit) is counted, the first
+// one is kept with its site number, and the access is skipped -- nothing faults or traps.  The
+// counters are per translation unit (no relocatable device code); hos_debug_bounds_violations()
+// adds them up.
+// ---------------------------------------------------------------------------------------
+#ifdef HOS_DEBUG_BOUNDS
+static __device__ unsigned int g_bounds_count;
+static __device__ long long g_bounds_first[3];           // site, index, limit of the first violation
+__device__ __forceinline__ bool bounds_ok(long long idx, long long limit, int site) {
+    if (idx >= 0 && idx < limit) return true;
+    if (atomicAdd(&g_bounds_count, 1u) == 0u) {
+        g_bounds_first[0] = site; g_bounds_first[1] = idx; g_bounds_first[2] = limit;
+    }
+    return false;
+}
+#define HOS_IN(idx, limit, site) (::hos::bounds_ok((long long)(idx), (long long)(limit), (site)))
+// one per translation unit with kernels: adds this unit's count, keeps the first violation seen
+#define HOS_DEFINE_BOUNDS_READER(name)                                                        \
+    void name(unsigned long long* count, long long* first) {                                  \
+        unsigned int c = 0;                                                                   \
+        long long f[3] = {0, 0, 0};                                                           \
+        cudaMemcpyFromSymbol(&c, g_bounds_count, sizeof(c));                                  \
+        cudaMemcpyFromSymbol(f, g_bounds_first, sizeof(f));                                   \
+        if (c && !*count) { first[0] = f[0]; first[1] = f[1]; first[2] = f[2]; }              \
+        *count += c;                                                                          \
+    }
+#else
+#define HOS_IN(idx, limit, site) (true)
+#define HOS_DEFINE_BOUNDS_READER(name) \
+    void name(unsigned long long*, long long*) {}
+#endif
+
 __device__ __forceinline__ int lane_id() { return threadIdx.x & 31; }
 __device__ __forceinline__ int warp_id() { return threadIdx.x >> 5; }
 

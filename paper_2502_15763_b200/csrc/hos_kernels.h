@@ -10,6 +10,11 @@ namespace hos {
 
 struct InstInfo;
 
+// Bounds-checked build: add this translation unit's violation count (no-ops otherwise).
+void debug_bounds_offline(unsigned long long* count, long long* first);
+void debug_bounds_online(unsigned long long* count, long long* first);
+void debug_bounds_multifit(unsigned long long* count, long long* first);
+
 // Calls the user's launch hook, if one is set (see hos_set_launch_hook).
 void launch_hook(const char* kernel, int phase, cudaStream_t st);
 

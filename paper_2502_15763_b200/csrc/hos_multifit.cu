@@ -138,6 +138,7 @@ __device__ void multifit_instance(const uint32_t* __restrict__ Ts, const uint32_
     if (s_take) {
         for (int r = threadIdx.x; r < n; r += MF_THREADS) {
             const uint8_t c = s_rc[r];
+            if (!HOS_IN(od[r], n, 401) || !HOS_IN(c, n_clients, 402)) continue;
             asg[od[r]] = (int32_t)c;
             if (rank_client) rank_client[r] = c;
         }
@@ -170,6 +171,8 @@ k_multifit(const uint32_t* __restrict__ T_sorted, const uint32_t* __restrict__ o
         multifit_instance<KPL, unsigned long long>(Ts, od, n_req, n_clients, inf.sum_T, inf.max_T, max_steps, asg,
                                                    load_out, makespan_out, rc, packer_out, smem_raw);
 }
+
+HOS_DEFINE_BOUNDS_READER(debug_bounds_multifit)
 
 cudaError_t launch_multifit(const hos_batch& b, const uint32_t* T_sorted, const uint32_t* order,
                             const InstInfo* info, int n_pad, int max_steps, int32_t* assign, long long* load,

@@ -187,6 +187,7 @@ k_estimate_sort(const uint32_t* __restrict__ p, const uint32_t* __restrict__ o,
                 uint32_t fk, id, extra;
                 const uint32_t r = bucket_sort_rank(B, s, fk, id, extra);
                 const uint32_t T = fk ^ flip;             // T < 2^nbits: the flip is its own inverse there
+                if (!HOS_IN(r, n_req, 201) || !HOS_IN(id, n_req, 202)) continue;
                 od[r] = id;
                 Ts[r] = T;
                 if (r + 1 == (uint32_t)n_clients || r == (uint32_t)n_clients) s_pair[r + 1 - n_clients] = T;
@@ -312,7 +313,7 @@ k_lpt(const uint32_t* __restrict__ T_sorted, const uint32_t* __restrict__ order,
                     int rk[4] = {0, 0, 0, 0};           // four short chains of additions instead of one long
 #pragma unroll
                     for (int b = 0; b < 32; ++b) rk[b & 3] += __shfl_sync(FULL, x, b) < x ? 1 : 0;
-                    s_perm[(rk[0] + rk[1]) + (rk[2] + rk[3])] = x;
+                    if (HOS_IN((rk[0] + rk[1]) + (rk[2] + rk[3]), 32, 212)) s_perm[(rk[0] + rk[1]) + (rk[2] + rk[3])] = x;
                     __syncwarp();
                     x = s_perm[lane];
                     __syncwarp();
@@ -395,7 +396,7 @@ k_lpt(const uint32_t* __restrict__ T_sorted, const uint32_t* __restrict__ order,
                 pos += W;
                 half_sorted = W == 32;
             }
-            if (r < n_req) {
+            if (r < n_req && HOS_IN(rq, n_req, 211) && HOS_IN(mine, n_clients, 213)) {
                 asg[rq] = (int32_t)mine;
                 if (rc) rc[r] = (uint8_t)mine;
             }
@@ -413,7 +414,7 @@ k_lpt(const uint32_t* __restrict__ T_sorted, const uint32_t* __restrict__ order,
         long long mx = 0;
 #pragma unroll
         for (int k = 0; k < KPL; ++k) {
-            if (key[k] != 0xFFFFFFFFu) {
+            if (key[k] != 0xFFFFFFFFu && HOS_IN(key[k] & ((1u << JB) - 1u), n_clients, 213)) {
                 const long long l = (long long)(rebased + (key[k] >> JB));
                 load_out[(size_t)inst * n_clients + (key[k] & ((1u << JB) - 1u))] = l;
                 mx = l > mx ? l : mx;
@@ -449,7 +450,7 @@ k_lpt(const uint32_t* __restrict__ T_sorted, const uint32_t* __restrict__ order,
                 for (int k = 0; k < KPL; ++k) load[k] += (own && (bj >> 5) == k) ? (long long)t : 0ll;
                 mine = (lane == sidx) ? (uint32_t)bj : mine;
             }
-            if (r < n_req) {
+            if (r < n_req && HOS_IN(rq, n_req, 211) && HOS_IN(mine, n_clients, 213)) {
                 asg[rq] = (int32_t)mine;
                 if (rc) rc[r] = (uint8_t)mine;
             }
@@ -647,6 +648,7 @@ __device__ inline bool build_member_lists(const int32_t* asg, uint8_t* rcl, cons
             __syncwarp();
             if (valid) {
                 const uint32_t at = base + __popc(m[e] & ((1u << lane) - 1u));
+                if (!HOS_IN(at, n, 222)) continue;
                 clI[at] = (IdxT)id[e];
                 clT[at] = tr[e];
                 if (lane == (__ffs(m[e]) - 1)) cnt[dig[e] * (NT / 32 + 1) + warp] = base + __popc(m[e]);
@@ -671,6 +673,7 @@ __device__ inline void warp_patch_list(uint32_t* segT, IdxT* segI, int len, int 
         const bool before = t > valT || (t == valT && (uint32_t)segI[mid] < valI);
         if (before) a = mid + 1; else z = mid;
     }
+    if (!HOS_IN(gone, len, 232) || !HOS_IN(a, len + 1, 231)) return;
     const uint32_t tg = segT[gone];
     const bool gone_before = tg > valT || (tg == valT && (uint32_t)segI[gone] < valI);
     const int at = a - (gone_before ? 1 : 0);                // position among the remaining entries
@@ -795,6 +798,7 @@ __device__ inline void place_lists_staged(const uint8_t* __restrict__ rcl, const
                 __syncwarp();
                 if (valid) {
                     const uint32_t at = base + __popc(m[e] & ((1u << lane) - 1u));
+                    if (!HOS_IN(at, LSB_SUB, 224)) continue;
                     stT[at] = tr[e];
                     stI[at] = (IdxT)id[e];
                     stC[at] = (uint8_t)dig[e];
@@ -805,7 +809,9 @@ __device__ inline void place_lists_staged(const uint8_t* __restrict__ rcl, const
         }
         for (int x = lane; x < end - sub; x += 32) {         // staging slot x -> its place in the client's list
             const uint32_t c = stC[x];
+            if (!HOS_IN(c, n_clients, 223)) continue;
             const uint32_t g = cnt[c * STRIDE + warp] + ((uint32_t)x - lbeg[c]);
+            if (!HOS_IN(g, n, 225)) continue;
             clT[g] = stT[x];
             clI[g] = stI[x];
         }
@@ -1146,6 +1152,7 @@ k_local_search(const uint32_t* __restrict__ T_sorted, const uint32_t* __restrict
             const int na = L.na;
             int best_at = -1;                                   // where the best partner's index is, if not read yet
             auto consider = [&](uint32_t inv, int pi, uint32_t k, bool move, int at, int idx) {
+                if (!HOS_IN(pi, LS_STAGE, 242)) return;
                 const uint32_t ik = ((uint32_t)s_I[pi] << 8) | k;
                 if (inv < best.inv || (inv == best.inv && ik < best.ik)) {
                     best.inv = inv; best.ik = ik; best.pi = pi; best.pu = move ? -1 : idx;
@@ -1183,6 +1190,7 @@ k_local_search(const uint32_t* __restrict__ T_sorted, const uint32_t* __restrict
                     for (int u = 0; u < LS_BATCH; ++u) {
                         const int idx = i0 + u * LS_THREADS + (int)threadIdx.x;
                         if (idx > len) continue;
+                        if (!HOS_IN(b[u] + 1, LS_STAGE + 1, 241) || !HOS_IN(cb + idx, n_req + 1, 246)) continue;
                         const uint32_t Ti = s_T[b[u]];          // A[b - 1]: smallest T >= thr (rising side)
                         const uint32_t d = Ti - Tu[u];
                         const uint32_t inv_r = d < slack ? ~(slack - d) : NO_CAND;
@@ -1247,6 +1255,7 @@ k_local_search(const uint32_t* __restrict__ T_sorted, const uint32_t* __restrict
         //     client, copies its list unless that is one of the two being patched; warps 2 and 3 patch
         //     one member list each.  (A move rebuilds the lists, so nothing is prepared ahead.)
         const int base_k = s_off[best_k];
+        if (!HOS_IN(base_j + best.pi, n_req, 247) || !HOS_IN(base_k + (swap ? best.pu : 0), n_req + 1, 247)) break;   // uniform
         const uint32_t Ti_w = clT[base_j + best.pi];            // read by every warp before any list changes
         const uint32_t Tu_w = swap ? clT[base_k + best.pu] : 0u;
         __syncthreads();
@@ -1264,7 +1273,7 @@ k_local_search(const uint32_t* __restrict__ T_sorted, const uint32_t* __restrict
                 list_clients(s_ls[buf ^ 1], nj, nL, floor_of_min(nj, nL) + margin, false);
             }
         } else if (warp == 1) {
-            if (lane == 0) {
+            if (lane == 0 && HOS_IN(best_i, n_req, 243) && HOS_IN(best_k, n_clients, 244) && HOS_IN(best_u + 1, n_req + 1, 243)) {
                 asg[best_i] = best_k;
                 if (best_u >= 0) asg[best_u] = jmax;
                 if (log) log[round] = hos_ls_move{best_i, best_u, best_k, best_v};
@@ -1339,6 +1348,8 @@ cudaError_t launch_estimate_sort(const hos_batch& b, const hos_cost_model& cm, u
     launch_hook("k_estimate_sort_radix", 1, st);
     return cudaGetLastError();
 }
+
+HOS_DEFINE_BOUNDS_READER(debug_bounds_offline)
 
 cudaError_t launch_lpt(const hos_batch& b, const uint32_t* T_sorted, const uint32_t* order,
                        const InstInfo* info, int n_pad, int32_t* assign, long long* load,

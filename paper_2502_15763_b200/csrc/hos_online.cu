@@ -124,6 +124,7 @@ k_queue_build(const uint32_t* __restrict__ p, const uint32_t* __restrict__ o,
             for (int s = threadIdx.x; s < n_req; s += SORT_THREADS) {
                 uint32_t k, id, extra;
                 const uint32_t r = bucket_sort_rank(B, s, k, id, extra);
+                if (!HOS_IN(r, n_req, 301) || !HOS_IN(id, n_req, 302)) continue;
                 const uint32_t pp = ride ? extra : pi[id];
                 const uint32_t totk = by_len ? kmask - (k & kmask) : 0u;     // p + (estimated) o, when it is the key
                 qr[r] = id;
@@ -179,7 +180,8 @@ constexpr int TF_AHEAD = 64;                // entries that the ring is filled a
 constexpr int SIM_QUIET_MAX = 16;         // plain decode iterations per pass of the simulator's loop
 constexpr unsigned long long HASH_INIT = 0xCBF29CE484222325ull;
 constexpr uint32_t HASH_C1 = 0x9E3779B1u, HASH_C2 = 0x85EBCA77u, HASH_C3 = 0xC2B2AE3Du, HASH_M = 0x27D4EB2Fu;
-constexpr int SIM_THREADS = 32;          // heap stride: the 32 clients of one warp sit side by side
+constexpr int SIM_MAX_WARPS_PER_SM = 16;  // simulator warps an SM is given at most when clients are spread thin (four per
+                                          // scheduler: at c4's size 28 warps of 16 clients took 1.74 ms, 14 warps of 32 1.48 ms)
 
 // Heap entries.  Narrow: (fin mod 2^16) << 16 | tot, usable when every p + o of the instance is
 // below 2^16 (then fin - cnt < 2^16 too, and entries compare correctly after subtracting
@@ -202,11 +204,11 @@ struct WideEntry {
     static __device__ __forceinline__ T rebase(T staged, uint32_t cnt) { return staged + ((T)cnt << 32); }
 };
 
-template <typename E>
+template <typename E, bool FULL_WARP>
 __global__ void __launch_bounds__(1024)
 k_simulate(const uint2* __restrict__ q_po, const int32_t* __restrict__ q_off,
            const int32_t* __restrict__ inst_status, const uint32_t* __restrict__ lambda_q16,
-           int n_lambda, int n_clients, int n_pad, long long n_units, int cap, uint32_t kv_budget,
+           int n_lambda, int n_clients, int n_pad, long long n_units, int lanes, int cap, uint32_t kv_budget,
            hos_cost_model cm, int q_shift, uint32_t max_iters,
            hos_client_result* __restrict__ cres,
            hos_iter_rec* __restrict__ trace, const long long* __restrict__ trace_off,
@@ -214,12 +216,16 @@ k_simulate(const uint2* __restrict__ q_po, const int32_t* __restrict__ q_off,
            uint32_t* __restrict__ event_count) {
     typedef typename E::T entry_t;
     extern __shared__ __align__(16) unsigned char smem_raw[];
-    // warps of a CTA are independent; each has its own block of cap * 32 heap entries
-    entry_t* heap = reinterpret_cast<entry_t*>(smem_raw) + (size_t)warp_id() * cap * SIM_THREADS + lane_id();
-    auto heap_ld = [&](int sl) -> entry_t { return heap[sl * SIM_THREADS]; };
-    auto heap_st = [&](int sl, entry_t v) { heap[sl * SIM_THREADS] = v; };
-    const long long unit = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-    const bool in_range = unit < n_units;
+    // warps of a CTA are independent; each has its own block of cap * lanes heap entries.  Only the
+    // first `lanes` lanes of a warp simulate a client: with fewer clients per warp the lanes wait
+    // less for each other's events, and a small batch spreads over more SMs.
+    // (FULL_WARP: lanes == 32 as a compile-time stride)
+    const int stride = FULL_WARP ? 32 : lanes;
+    entry_t* heap = reinterpret_cast<entry_t*>(smem_raw) + (size_t)warp_id() * cap * stride + lane_id();
+    auto heap_ld = [&](int sl) -> entry_t { return HOS_IN(sl, cap, 311) ? heap[sl * stride] : (entry_t)0; };
+    auto heap_st = [&](int sl, entry_t v) { if (HOS_IN(sl, cap, 311)) heap[sl * stride] = v; };
+    const long long unit = ((long long)blockIdx.x * (blockDim.x >> 5) + warp_id()) * stride + lane_id();
+    const bool in_range = lane_id() < stride && unit < n_units;
     const int c = in_range ? (int)(unit % n_clients) : 0;
     const int l = in_range ? (int)((unit / n_clients) % n_lambda) : 0;
     const int inst = in_range ? (int)(unit / ((long long)n_clients * n_lambda)) : 0;
@@ -336,7 +342,7 @@ k_simulate(const uint2* __restrict__ q_po, const int32_t* __restrict__ q_off,
             // and queue positions stay below 2^15, durations follow from the tokens.
             const uint32_t packed = (r1 >> 31) ? (0x80000000u | (r3 << 16) | ((B - 1u) << 8) | ((r1 & 0x7FFFFFFFu) - 1u))
                                                : (((r3 - 1u) << 8) | (r1 - 1u));
-            ev[n_ev] = make_uint4(n_pre + cnt, r2, S, packed);
+            if (HOS_IN(n_ev, 2 * qn, 313)) ev[n_ev] = make_uint4(n_pre + cnt, r2, S, packed);
             ++n_ev;
         }
         emit(dur, r1, r2, r3);
@@ -372,7 +378,7 @@ k_simulate(const uint2* __restrict__ q_po, const int32_t* __restrict__ q_off,
                 heap_st(cap - 1 - (int)nA, E::make(nxt.y, tt));
                 sumTot += tt; sumP += nxt.x; ++nA;
                 nxt = nxt2;
-                if (head + (int)nA + 1 < qn) nxt2 = __ldg(&q[head + nA + 1]);
+                if (head + (int)nA + 1 < qn && HOS_IN(q0 + head + (int)nA + 1, n_pad, 312)) nxt2 = __ldg(&q[head + nA + 1]);
             }
             grow = false;
         }
@@ -498,8 +504,8 @@ k_simulate_steal(const uint2* __restrict__ q_po, const uint32_t* __restrict__ q_
     const long long unit = (long long)sim * n_clients + c;
     const bool is_client = c < n_clients;
     entry_t* heap = reinterpret_cast<entry_t*>(smem_raw) + c;
-    auto heap_ld = [&](int sl) -> entry_t { return heap[sl * stride]; };
-    auto heap_st = [&](int sl, entry_t v) { heap[sl * stride] = v; };
+    auto heap_ld = [&](int sl) -> entry_t { return HOS_IN(sl, cap, 321) ? heap[sl * stride] : (entry_t)0; };
+    auto heap_st = [&](int sl, entry_t v) { if (HOS_IN(sl, cap, 321)) heap[sl * stride] = v; };
 
     const int ist = inst_status[inst];
     if (((ist & INST_WIDE) != 0) != (sizeof(entry_t) == 8)) return;   // the other instantiation's instance
@@ -562,6 +568,7 @@ k_simulate_steal(const uint2* __restrict__ q_po, const uint32_t* __restrict__ q_
     // claim the request at position x of some queue as my next candidate, if it fits.  A dry run
     // keeps its hands off everything the clients share.
     auto claim = [&](int owner, int x, bool dry) -> bool {
+        if (!HOS_IN(x, n_req, 322) || !HOS_IN(owner, n_clients, 324)) return false;
         const uint2 po = q[x];
         const uint32_t tt = po.x + po.y;
         if (reserved + sumTot + tt > kv_budget) return false;
@@ -573,7 +580,7 @@ k_simulate_steal(const uint2* __restrict__ q_po, const uint32_t* __restrict__ q_
             s_ustart[owner] = x + 1;
             s_remain[owner] -= tk;
             atomicAdd(&s_total, 0ull - (unsigned long long)tk);
-            if (served) served[qr[x]] = c;
+            if (served && HOS_IN(qr[x], n_req, 323)) served[qr[x]] = c;
         }
         return true;
     };
@@ -990,6 +997,8 @@ static int sim_slots(const hos_batch& b) {
 }
 static uint32_t sim_budget(const hos_batch& b) { return b.kv_reserve_tokens ? 0x7FFFFFFFu : (uint32_t)b.kv_budget; }
 
+HOS_DEFINE_BOUNDS_READER(debug_bounds_online)
+
 size_t queue_build_smem(int n_req) { return sort_smem_bytes<uint16_t>(n_req); }
 
 cudaError_t launch_queue_build(const hos_batch& b, const int32_t* assign, uint32_t p_max, int queue_order, uint2* q_po,
@@ -1024,48 +1033,60 @@ cudaError_t launch_simulate(const hos_batch& b, const hos_cost_model& cm, const 
     // nothing else: the simulator runs with that many slots and no KV limit.
     const int cap = sim_slots(b);
     const uint32_t kv = sim_budget(b);
-    const long long n_warps = (n_units + SIM_THREADS - 1) / SIM_THREADS;
     int q_shift = -1;                                    // power-of-two KV divisor -> shift
     if ((cm.decode_kv_div & (cm.decode_kv_div - 1)) == 0)
         for (q_shift = 0; (1u << q_shift) != cm.decode_kv_div; ++q_shift) {}
     // Both instantiations are launched; each one runs the instances whose entries it can hold and
     // returns at once for the others (the flag is per instance, on the device).
     //
-    // Warps per CTA.  The recurrence is latency-bound and shared memory (one heap per client) limits
-    // the resident warps, so what matters is how many fit at once.  Every CTA costs 1 KB of shared
-    // memory on top of its own: one-warp CTAs free their SM slot as soon as they finish, which is
-    // best over many waves, but when all the work fits the GPU at once only with fewer, larger
-    // CTAs (one per SM), those are used.
+    // Launch shape.  The recurrence is latency-bound and shared memory (one heap per client) limits
+    // what is resident, so what matters is that everything runs at once, on as many SMs as possible,
+    // with as few clients per warp as that allows (the lanes of a warp wait for each other's events).
+    // `lanes` clients per warp: the smallest power of two for which all warps are resident in one
+    // wave and an SM holds at most SIM_MAX_WARPS_PER_SM of them (more warps than that and they only
+    // compete for the issue slots).  Every CTA
+    // costs 1 KB of shared memory on top of its heaps; if not even 32 lanes make one wave, one-warp
+    // CTAs are used, which free their SM slot as soon as they finish.
     int n_sm = 148, dev = 0;
     if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev);
-    auto warps_per_cta = [&](size_t per_warp) {
+    struct Shape { int lanes, wpc; unsigned grid; size_t smem; };
+    auto shape_for = [&](size_t entry_bytes) {
         const size_t budget = 227 * 1024, fixed = 1024;
-        const long long small_ctas = (long long)(budget / (per_warp + fixed));
-        const long long cap_small = (long long)n_sm * (small_ctas < 32 ? small_ctas : 32);
-        long long wide = (long long)((budget - fixed) / per_warp);
-        if (wide > 32) wide = 32;
-        if (n_warps > cap_small && wide >= 1 && n_warps <= (long long)n_sm * wide) return (int)wide;
-        return 1;
+        Shape best{32, 1, 0, 0};
+        bool found = false;
+        for (int lanes = 32; lanes >= 1; lanes >>= 1) {
+            const long long n_warps = (n_units + lanes - 1) / lanes;
+            const size_t per_warp = (size_t)cap * lanes * entry_bytes;
+            const long long per_sm = (n_warps + n_sm - 1) / n_sm;              // warps an SM must hold
+            if (per_sm > SIM_MAX_WARPS_PER_SM) break;
+            const long long ctas = (per_sm + 31) / 32;                         // CTAs per SM
+            const long long wpc = (per_sm + ctas - 1) / ctas;
+            if ((size_t)ctas * ((size_t)wpc * per_warp + fixed) > budget) break;
+            best = Shape{lanes, (int)wpc, (unsigned)((n_warps + wpc - 1) / wpc), (size_t)wpc * per_warp};
+            found = true;
+        }
+        if (!found) {
+            const long long n_warps = (n_units + 31) / 32;
+            best = Shape{32, 1, (unsigned)n_warps, (size_t)cap * 32 * entry_bytes};
+        }
+        return best;
     };
-    const size_t warp_n = (size_t)cap * SIM_THREADS * sizeof(uint32_t);
-    const size_t warp_w = (size_t)cap * SIM_THREADS * sizeof(unsigned long long);
-    const int wpc_n = warps_per_cta(warp_n), wpc_w = warps_per_cta(warp_w);
-    const size_t smem_n = warp_n * wpc_n, smem_w = warp_w * wpc_w;
-    const unsigned grid_n = (unsigned)((n_warps + wpc_n - 1) / wpc_n);
-    const unsigned grid_w = (unsigned)((n_warps + wpc_w - 1) / wpc_w);
-    cudaError_t e = allow_max_dynamic_smem(reinterpret_cast<const void*>(k_simulate<NarrowEntry>));
+    const Shape sn = shape_for(sizeof(uint32_t)), sw = shape_for(sizeof(unsigned long long));
+    auto kern_n = sn.lanes == 32 ? k_simulate<NarrowEntry, true> : k_simulate<NarrowEntry, false>;
+    auto kern_w = sw.lanes == 32 ? k_simulate<WideEntry, true> : k_simulate<WideEntry, false>;
+    cudaError_t e = allow_max_dynamic_smem(reinterpret_cast<const void*>(kern_n));
     if (e != cudaSuccess) return e;
-    e = allow_max_dynamic_smem(reinterpret_cast<const void*>(k_simulate<WideEntry>));
+    e = allow_max_dynamic_smem(reinterpret_cast<const void*>(kern_w));
     if (e != cudaSuccess) return e;
     launch_hook("k_simulate", 0, st);
-    k_simulate<NarrowEntry><<<grid_n, SIM_THREADS * wpc_n, smem_n, st>>>(
-        q_po, q_off, inst_status, lambda_q16, n_lambda, b.n_clients, n_pad, n_units, cap,
+    kern_n<<<sn.grid, 32 * sn.wpc, sn.smem, st>>>(
+        q_po, q_off, inst_status, lambda_q16, n_lambda, b.n_clients, n_pad, n_units, sn.lanes, cap,
         kv, cm, q_shift, max_iters, cres, trace, trace_off, status, events, event_count);
     launch_hook("k_simulate", 1, st);
     if (b.kv_budget >= 65536) {                          // otherwise no p + o can reach 2^16
         launch_hook("k_simulate_wide", 0, st);
-        k_simulate<WideEntry><<<grid_w, SIM_THREADS * wpc_w, smem_w, st>>>(
-            q_po, q_off, inst_status, lambda_q16, n_lambda, b.n_clients, n_pad, n_units, cap,
+        kern_w<<<sw.grid, 32 * sw.wpc, sw.smem, st>>>(
+            q_po, q_off, inst_status, lambda_q16, n_lambda, b.n_clients, n_pad, n_units, sw.lanes, cap,
             kv, cm, q_shift, max_iters, cres, trace, trace_off, status, events, event_count);
         launch_hook("k_simulate_wide", 1, st);
     }

@@ -118,7 +118,7 @@ __device__ inline IdxT* block_radix_sort_ids(const SortSmem<IdxT>& s, int n, int
             if (pos < hi) {
                 const uint32_t id = natural ? (uint32_t)pos : (uint32_t)src[pos];
                 const uint32_t dig = ((s.key[id] ^ flip) >> shift) & dmask;
-                atomicAdd(&s.cnt[dig * CNT_STRIDE + warp], 1u);
+                if (HOS_IN(id, n, 103) && HOS_IN(dig * CNT_STRIDE + warp, CNT_WORDS, 101)) atomicAdd(&s.cnt[dig * CNT_STRIDE + warp], 1u);
             }
         }
         __syncthreads();
@@ -167,7 +167,7 @@ __device__ inline IdxT* block_radix_sort_ids(const SortSmem<IdxT>& s, int n, int
                 const uint32_t base = valid[g] ? s.cnt[dig[g] * CNT_STRIDE + warp] : 0u;
                 __syncwarp();
                 if (valid[g]) {
-                    dst[base + __popc(m[g] & ((1u << lane) - 1u))] = (IdxT)id[g];
+                    if (HOS_IN(base + __popc(m[g] & ((1u << lane) - 1u)), n, 102)) dst[base + __popc(m[g] & ((1u << lane) - 1u))] = (IdxT)id[g];
                     if (lane == (__ffs(m[g]) - 1)) s.cnt[dig[g] * CNT_STRIDE + warp] = base + __popc(m[g]);
                 }
                 __syncwarp();
@@ -221,7 +221,7 @@ __host__ __device__ inline size_t bucket_sort_smem_bytes(int n) {
 }
 
 struct BucketSort {
-    int bbits, low_bits, id_bits, xbits, n_words;
+    int bbits, low_bits, id_bits, xbits, n_words, n;
     uint32_t kmask, lmask;
     uint32_t* ent;              // [n]  (rest of key << id_bits | id) << xbits | extra, in slot order
     uint16_t* bkt;              // [n]  bucket of every slot
@@ -235,6 +235,7 @@ __device__ inline bool bucket_sort_plan(BucketSort& B, unsigned char* smem, int 
     B.low_bits = max(0, nbits - B.bbits);
     B.id_bits = n > 1 ? bit_width_u32((uint32_t)(n - 1)) : 1;
     B.xbits = xbits;
+    B.n = n;
     B.n_words = 1 << (B.bbits - 1);
     B.kmask = nbits >= 32 ? 0xFFFFFFFFu : ((1u << nbits) - 1u);
     B.lmask = B.low_bits >= 32 ? 0xFFFFFFFFu : ((1u << B.low_bits) - 1u);
@@ -252,7 +253,7 @@ __device__ inline void bucket_sort_clear(const BucketSort& B) {
 
 __device__ __forceinline__ void bucket_sort_count(const BucketSort& B, uint32_t key) {
     const uint32_t b = (key & B.kmask) >> B.low_bits;
-    atomicAdd(&B.cntw[b >> 1], 1u << ((b & 1u) << 4));
+    if (HOS_IN(b >> 1, B.n_words, 111)) atomicAdd(&B.cntw[b >> 1], 1u << ((b & 1u) << 4));
 }
 
 // Exclusive scan of the bucket counts (after every bucket_sort_count).  Starts and ends with a
@@ -302,7 +303,9 @@ __device__ __forceinline__ uint32_t bucket_sort_start(const BucketSort& B, uint3
 __device__ __forceinline__ void bucket_sort_place(const BucketSort& B, uint32_t key, uint32_t id, uint32_t extra) {
     const uint32_t fk = key & B.kmask;
     const uint32_t b = fk >> B.low_bits, sh = (b & 1u) << 4;
+    if (!HOS_IN(b >> 1, B.n_words, 111)) return;
     const uint32_t slot = (atomicAdd(&B.cntw[b >> 1], 1u << sh) >> sh) & 0xFFFFu;
+    if (!HOS_IN(slot, B.n, 112)) return;
     B.ent[slot] = ((((fk & B.lmask) << B.id_bits) | id) << B.xbits) | extra;
     B.bkt[slot] = (uint16_t)b;
 }
@@ -313,7 +316,9 @@ __device__ __forceinline__ uint32_t bucket_sort_rank(const BucketSort& B, int s,
                                                      uint32_t& extra) {
     const uint16_t* cnt16 = reinterpret_cast<const uint16_t*>(B.cntw);
     const uint32_t mine = B.ent[s], b = B.bkt[s];
-    const uint32_t start = b ? cnt16[b - 1] : 0u, end = cnt16[b];
+    const bool b_ok = HOS_IN(b, 1 << B.bbits, 113);
+    uint32_t start = (b_ok && b) ? cnt16[b - 1] : 0u, end = b_ok ? cnt16[b] : 0u;
+    if (!HOS_IN(end, B.n + 1, 114) || !HOS_IN(start, end + 1, 114)) start = end = 0;
     uint32_t r = start, j = start;
     for (; j + 1 < end; j += 2) r += (B.ent[j] < mine ? 1u : 0u) + (B.ent[j + 1] < mine ? 1u : 0u);
     if (j < end) r += B.ent[j] < mine ? 1u : 0u;
