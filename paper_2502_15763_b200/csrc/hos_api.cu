@@ -265,7 +265,7 @@ int hos_lower_bound(const hos_batch* b, const hos_cost_model* cm, hos_lb* out, i
     const OfflineWs w = carve_offline(b, ws, 1, 0);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const int n_pad = pad4(b->n_req);
-    return cuda_rc(launch_estimate_sort(*b, *cm, w.T_sorted, w.order, w.info, status, out, n_pad, st));
+    return cuda_rc(launch_estimate_sort(*b, *cm, nullptr, nullptr, w.info, status, out, n_pad, st));
 }
 
 int hos_online_simulate(const hos_batch* b, const int32_t* assign, const hos_cost_model* cm,

@@ -161,8 +161,8 @@ k_estimate_sort(const uint32_t* __restrict__ p, const uint32_t* __restrict__ o,
         }
         const int nbits = bit_width_u32((uint32_t)mx);
         const uint32_t flip = nbits >= 32 ? 0xFFFFFFFFu : ((1u << nbits) - 1u);   // descending T
-        uint32_t* Ts = T_sorted + (size_t)inst * n_pad;
-        uint32_t* od = order + (size_t)inst * n_pad;
+        uint32_t* Ts = T_sorted ? T_sorted + (size_t)inst * n_pad : nullptr;
+        uint32_t* od = T_sorted ? order + (size_t)inst * n_pad : nullptr;
         if (threadIdx.x < 2) s_pair[threadIdx.x] = 0;
         if (FAST) {
             // two more passes over the tables (now in L2): count, then place; T is taken again
@@ -179,6 +179,33 @@ k_estimate_sort(const uint32_t* __restrict__ p, const uint32_t* __restrict__ o,
                 if (threadIdx.x == 0) info[inst].status = SORT_PENDING;
                 continue;
             }
+            if (!T_sorted) {
+                // Bounds only: no order is wanted, just T_(M) and T_(M+1).  The buckets that hold
+                // those two ranks are known from the scan; their items alone are collected and
+                // ranked among themselves.
+                if (n_req > n_clients) {
+                    __shared__ uint32_t s_ncand;
+                    if (threadIdx.x == 0) s_ncand = 0;
+                    __syncthreads();
+                    const uint32_t M = (uint32_t)n_clients, nb = 1u << B.bbits;
+                    for_each_request(pi, oi, ei, nullptr, n_req, [&](int i, uint32_t pp, uint32_t, uint32_t oe, int) {
+                        const uint32_t fk = ((e_p * pp + e_o * oe) ^ flip) & B.kmask, b = fk >> B.low_bits;
+                        const uint32_t start = bucket_sort_start(B, b), end = b + 1 < nb ? bucket_sort_start(B, b + 1) : (uint32_t)n_req;
+                        if (start <= M && M - 1 < end) {             // the bucket holds rank M - 1 or M
+                            const uint32_t at = atomicAdd(&s_ncand, 1u);
+                            if (HOS_IN(at, n_req, 203)) { B.ent[at] = ((fk & B.lmask) << B.id_bits) | (uint32_t)i; B.bkt[at] = (uint16_t)b; }
+                        }
+                    });
+                    __syncthreads();
+                    const uint32_t nc = s_ncand;
+                    for (uint32_t c = threadIdx.x; c < nc; c += SORT_THREADS) {
+                        const uint32_t mine = B.ent[c], b = B.bkt[c];
+                        uint32_t r = bucket_sort_start(B, b);
+                        for (uint32_t j = 0; j < nc; ++j) r += (B.bkt[j] == b && B.ent[j] < mine) ? 1u : 0u;
+                        if (r + 1 == M || r == M) s_pair[r + 1 - M] = ((b << B.low_bits) | (mine >> B.id_bits)) ^ flip;
+                    }
+                }
+            } else {
             for_each_request(pi, oi, ei, nullptr, n_req, [&](int i, uint32_t pp, uint32_t, uint32_t oe, int) {
                 bucket_sort_place(B, (e_p * pp + e_o * oe) ^ flip, (uint32_t)i, 0u);
             });
@@ -192,13 +219,13 @@ k_estimate_sort(const uint32_t* __restrict__ p, const uint32_t* __restrict__ o,
                 Ts[r] = T;
                 if (r + 1 == (uint32_t)n_clients || r == (uint32_t)n_clients) s_pair[r + 1 - n_clients] = T;
             }
+            }
         } else {
             SortSmem<uint16_t> s = sort_smem_carve<uint16_t>(smem_raw, n_req);
             const uint16_t* sorted = block_radix_sort_ids<uint16_t>(s, n_req, nbits, flip);
             for (int r = threadIdx.x; r < n_req; r += SORT_THREADS) {
                 const uint32_t id = sorted[r];
-                od[r] = id;
-                Ts[r] = key[id];
+                if (T_sorted) { od[r] = id; Ts[r] = key[id]; }
                 if (r + 1 == n_clients || r == n_clients) s_pair[r + 1 - n_clients] = key[id];
             }
         }
@@ -1325,6 +1352,7 @@ size_t local_search_index_bytes(int n_req) { return n_req <= 65536 ? 2 : 4; }
 cudaError_t launch_estimate_sort(const hos_batch& b, const hos_cost_model& cm, uint32_t* T_sorted,
                                  uint32_t* order, InstInfo* info, int32_t* status_out, hos_lb* lb_out, int n_pad,
                                  cudaStream_t st) {
+    // T_sorted == nullptr: the bounds only (no order is written; T_(M), T_(M+1) come from a selection)
     cudaError_t e = allow_max_dynamic_smem(reinterpret_cast<const void*>(k_estimate_sort<true>));
     if (e != cudaSuccess) return e;
     if ((e = allow_max_dynamic_smem(reinterpret_cast<const void*>(k_estimate_sort<false>))) != cudaSuccess) return e;
