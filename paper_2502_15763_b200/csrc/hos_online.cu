@@ -180,8 +180,12 @@ constexpr int TF_AHEAD = 64;                // entries that the ring is filled a
 constexpr int SIM_QUIET_MAX = 16;         // plain decode iterations per pass of the simulator's loop
 constexpr unsigned long long HASH_INIT = 0xCBF29CE484222325ull;
 constexpr uint32_t HASH_C1 = 0x9E3779B1u, HASH_C2 = 0x85EBCA77u, HASH_C3 = 0xC2B2AE3Du, HASH_M = 0x27D4EB2Fu;
-constexpr int SIM_MAX_WARPS_PER_SM = 16;  // simulator warps an SM is given at most when clients are spread thin (four per
-                                          // scheduler: at c4's size 28 warps of 16 clients took 1.74 ms, 14 warps of 32 1.48 ms)
+// Clients are spread over more warps (fewer than 32 per warp) only while an SM gets at most this
+// many warps, two per scheduler: spreading pays as long as schedulers would otherwise sit empty
+// (800 clients: 0.54 ms as 25 full warps, 0.25 ms one client per warp), not beyond (18,944
+// clients: 1.03 ms as 4 full warps per SM, 1.07 ms as 16 warps of 8; 65,536 clients: 1.48 ms
+// as 14 full warps per SM, 1.74 ms as 28 warps of 16).
+constexpr int SIM_SPREAD_WARPS_PER_SM = 8;
 
 // Heap entries.  Narrow: (fin mod 2^16) << 16 | tot, usable when every p + o of the instance is
 // below 2^16 (then fin - cnt < 2^16 too, and entries compare correctly after subtracting
@@ -1043,8 +1047,7 @@ cudaError_t launch_simulate(const hos_batch& b, const hos_cost_model& cm, const 
     // what is resident, so what matters is that everything runs at once, on as many SMs as possible,
     // with as few clients per warp as that allows (the lanes of a warp wait for each other's events).
     // `lanes` clients per warp: the smallest power of two for which all warps are resident in one
-    // wave and an SM holds at most SIM_MAX_WARPS_PER_SM of them (more warps than that and they only
-    // compete for the issue slots).  Every CTA
+    // wave and, below 32, an SM holds at most SIM_SPREAD_WARPS_PER_SM of them.  Every CTA
     // costs 1 KB of shared memory on top of its heaps; if not even 32 lanes make one wave, one-warp
     // CTAs are used, which free their SM slot as soon as they finish.
     int n_sm = 148, dev = 0;
@@ -1058,7 +1061,7 @@ cudaError_t launch_simulate(const hos_batch& b, const hos_cost_model& cm, const 
             const long long n_warps = (n_units + lanes - 1) / lanes;
             const size_t per_warp = (size_t)cap * lanes * entry_bytes;
             const long long per_sm = (n_warps + n_sm - 1) / n_sm;              // warps an SM must hold
-            if (per_sm > SIM_MAX_WARPS_PER_SM) break;
+            if (lanes < 32 && per_sm > SIM_SPREAD_WARPS_PER_SM) break;
             const long long ctas = (per_sm + 31) / 32;                         // CTAs per SM
             const long long wpc = (per_sm + ctas - 1) / ctas;
             if ((size_t)ctas * ((size_t)wpc * per_warp + fixed) > budget) break;
