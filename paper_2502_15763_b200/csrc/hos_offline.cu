@@ -586,7 +586,7 @@ __device__ inline void block_scan_u32(uint32_t* a, int len, uint32_t* wsum) {
 // LS_ROWS rows of 32 ranks at a time, so that their reads are in flight together.
 constexpr int LS_ROWS = 4;
 template <typename IdxT, bool CHECK, bool GATHER, int NT>
-__device__ inline bool build_member_lists(const int32_t* asg, uint8_t* rcl, const uint32_t* __restrict__ gO,
+__device__ __noinline__ bool build_member_lists(const int32_t* asg, uint8_t* rcl, const uint32_t* __restrict__ gO,
                                           const uint32_t* __restrict__ gT, IdxT* clI, uint32_t* clT,
                                           int n, int n_clients, uint32_t* cnt, uint32_t* wsum, int* off,
                                           long long* load) {
@@ -690,7 +690,7 @@ __device__ inline bool build_member_lists(const int32_t* asg, uint8_t* rcl, cons
 // One warp: in the list (segT, segI)[0 .. len), ordered by (T descending, index ascending),
 // drop the entry at position `gone` and insert (valT, valI) at its place in the order.
 template <typename IdxT>
-__device__ inline void warp_patch_list(uint32_t* segT, IdxT* segI, int len, int gone, uint32_t valT,
+__device__ __noinline__ void warp_patch_list(uint32_t* segT, IdxT* segI, int len, int gone, uint32_t valT,
                                        uint32_t valI) {
     const int lane = lane_id();
     int a = 0, z = len;                                      // entries that come before the new one
@@ -926,6 +926,9 @@ __device__ __forceinline__ void count_ge_batch(const uint32_t* s_T, const uint32
 // that client's list) while the other warps patch the lists.
 __device__ __forceinline__ void pair_arrive() { asm volatile("bar.arrive 1, 64;" ::: "memory"); }
 __device__ __forceinline__ void pair_wait() { asm volatile("bar.sync 1, 64;" ::: "memory"); }
+// Named barrier 2 lets warps 2 and 3, once their lists are patched, help with that copy.
+__device__ __forceinline__ void trio_arrive() { asm volatile("bar.arrive 2, 96;" ::: "memory"); }
+__device__ __forceinline__ void trio_wait() { asm volatile("bar.sync 2, 96;" ::: "memory"); }
 
 template <typename IdxT, int LS_BATCH>
 __global__ void __launch_bounds__(LS_THREADS, 7)
@@ -1066,13 +1069,30 @@ k_local_search(const uint32_t* __restrict__ T_sorted, const uint32_t* __restrict
             if (!skip_listed) L.min_unlisted = min_out;
         }
     };
-    // Copy of a critical client's list to shared memory by `nthr` threads (this one is number `t`).
-    auto copy_list = [&](int base, int nmem, int t, int nthr) {
+    // Copy of a critical client's list to shared memory by `nthr` threads (this one is number `t`):
+    // the T entries by asynchronous 4-byte copies (all in flight at once, no registers) with the
+    // guard values written by hand, and the 2-byte request indices.  Each part ends when this
+    // thread's share of it has landed.
+    auto copy_list_T = [&](int base, int nmem, int t, int nthr) {
         const int top2 = 2 << (31 - __clz(nmem));
         for (int x = t; x <= top2; x += nthr) {
-            s_T[x] = x == 0 ? 0xFFFFFFFFu : (x <= nmem ? clT[base + x - 1] : 0u);
-            if (x < nmem) s_I[x] = clI[base + x];
+            if (x >= 1 && x <= nmem) {
+                const unsigned sa = (unsigned)__cvta_generic_to_shared(&s_T[x]);
+                asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" :: "r"(sa), "l"(clT + base + x - 1) : "memory");
+            } else {
+                s_T[x] = x == 0 ? 0xFFFFFFFFu : 0u;
+            }
         }
+        asm volatile("cp.async.commit_group;" ::: "memory");
+        asm volatile("cp.async.wait_group 0;" ::: "memory");
+    };
+    auto copy_list_I = [&](int base, int nmem, int t, int nthr) {
+#pragma unroll 4
+        for (int x = t; x < nmem; x += nthr) s_I[x] = clI[base + x];
+    };
+    auto copy_list = [&](int base, int nmem, int t, int nthr) {
+        copy_list_I(base, nmem, t, nthr);
+        copy_list_T(base, nmem, t, nthr);
     };
     auto is_fast = [&](int nmem, long long Lmax) { return nmem >= 1 && nmem < LS_STAGE && Lmax <= 0x7FFFFFFFll; };
     auto floor_of_min = [&](int jmax, long long Lmax) {
@@ -1246,8 +1266,6 @@ k_local_search(const uint32_t* __restrict__ T_sorted, const uint32_t* __restrict
         long long best_v = Lmax;
         for (int pass = 0; pass < 2; ++pass) {
             if (!fast) evaluate_listed(best);
-            else if (top == 256) evaluate_listed_fast(best, std::integral_constant<int, 9>());
-            else if (top == 128) evaluate_listed_fast(best, std::integral_constant<int, 8>());
             else evaluate_listed_fast(best, std::integral_constant<int, 0>());
             // CTA-wide lexicographic minimum: per warp, then every warp reduces the warps' records
             best = cand_warp_min(best);
@@ -1294,6 +1312,7 @@ k_local_search(const uint32_t* __restrict__ T_sorted, const uint32_t* __restrict
             __syncwarp();
             __threadfence_block();                              // the extremes are written before warp 1 is let go
             pair_arrive();
+            if (swap) trio_arrive();
             if (swap) {
                 const int nj = s_jmax;
                 const long long nL = s_lmax;
@@ -1310,13 +1329,19 @@ k_local_search(const uint32_t* __restrict__ T_sorted, const uint32_t* __restrict
             const int nj = s_jmax;
             if (swap && nj != jmax && nj != best_k) {
                 const int nb = s_off[nj], nn = s_off[nj + 1] - nb;
-                if (is_fast(nn, s_lmax)) copy_list(nb, nn, lane, 32);
+                if (is_fast(nn, s_lmax)) copy_list_T(nb, nn, lane, 32);   // warps 2 and 3 bring the indices
             }
         } else if (swap) {
             if (warp == 2) warp_patch_list<IdxT>(clT + base_j, clI + base_j, nm, best.pi, Tu_w, (uint32_t)best_u);
             else if (warp == 3)
                 warp_patch_list<IdxT>(clT + base_k, clI + base_k, s_off[best_k + 1] - base_k, best.pu, Ti_w,
                                       (uint32_t)best_i);
+            trio_wait();                                        // warp 0 has found the next critical client
+            const int nj = s_jmax;
+            if (nj != jmax && nj != best_k) {
+                const int nb = s_off[nj], nn = s_off[nj + 1] - nb;
+                if (is_fast(nn, s_lmax)) copy_list_I(nb, nn, (int)threadIdx.x - 64, 64);
+            }
         }
         __syncthreads();
         if (!swap)
