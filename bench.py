@@ -52,15 +52,16 @@ NCU_COUNTERS = os.path.join(ROOT, "profiles", "ncu_counters_c4x296.json")
 
 
 def ncu_counters():
-    """(counters per kernel, note): {} with the reason when the file is missing or stale."""
+    """(counters per kernel, shape of the captured workload, note): {} with the reason when the file
+    is missing or stale."""
     try:
         doc = json.load(open(NCU_COUNTERS))
     except (OSError, ValueError):
-        return {}, "no counter file"
+        return {}, None, "no counter file"
     from paper_2502_15763_b200 import _build
     if doc.get("source_hash") != _build.source_hash():
-        return {}, "kernels changed since the counters were taken"
-    return doc.get("kernels", {}), "ncu capture of " + doc.get("workload", "?")
+        return {}, None, "kernels changed since the counters were taken"
+    return doc.get("kernels", {}), doc.get("shape"), "ncu capture of " + doc.get("workload", "?")
 
 
 def describe(w: Workload) -> str:
@@ -617,7 +618,8 @@ def run_ours(args):
     if rank == 0:
         prof = kernel_profile(torch, hos, pipe, max(2, min(args.steps, 5)), flush)
         peak, peak_kind = measured_peak()
-        counters, counters_note = ncu_counters()
+        counters, counters_shape, counters_note = ncu_counters()
+        shape = {"n_req": w.n_req, "n_clients": w.n_clients, "batch_cap": w.batch_cap}
         props = torch.cuda.get_device_properties(dev)
         mhz = (clocks or {}).get("sm_max_mhz") or 1965.0
         alu_peak = props.multi_processor_count * 128 * mhz * 1e6 / 1e12       # T int32 op/s
@@ -629,6 +631,9 @@ def run_ours(args):
             """Counter of the capture scaled to this launch by the units it processes."""
             c = counters.get(name)
             if not c:
+                return None
+            # instructions per unit depend on the lists' lengths and the batch size: only for the captured shape
+            if field == "warp_inst_per_unit" and counters_shape != shape:
                 return None
             n = units[c["unit"]]
             if c["unit"] == "request" and len(w.lambdas_q16) > 1 and name in ("k_simulate", "k_ls_lists"):
@@ -716,7 +721,7 @@ def run_ours(args):
                             "download" + ("" if flush is None else ", L2 flushes included")},
             "e2e_with_trace": e2e_trace,
             "gpu_launches": int(round(launches * args.steps)),
-            "requests_per_step": w.n_inst * w.n_req,
+            "requests_per_step": w.n_inst * w.n_req, "shape": shape,
             "ls_rounds_executed_per_step": units["round"],
             "input_sha256": input_sha256(pipe),
             "roofline": roofline,

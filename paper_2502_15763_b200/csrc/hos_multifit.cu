@@ -8,17 +8,19 @@
 //                bisection tree side by side -- the capacity that would be probed after
 //                success/success, success/failure, ... -- and one thread then walks the three
 //                levels: the same probe sequence as the step-by-step bisection, in a third of
-//                the passes.  A last pass packs at the capacity found; the result replaces
-//                the list-scheduling one only when its largest load is strictly smaller.
+//                the passes.  That is for small batches, where the chain's latency is all there
+//                is; a batch that fills the GPU anyway is bound by instruction issue, and there
+//                the four speculative probes in seven that are thrown away cost more than the
+//                shorter chain saves, so it runs one warp per instance, one level per round.
+//                A last pass packs at the capacity found; the result replaces the
+//                list-scheduling one only when its largest load is strictly smaller.
 #include "hos_common.cuh"
 #include "hos_kernels.h"
 
 namespace hos {
 
-constexpr int MF_WARPS = 8;
-constexpr int MF_THREADS = MF_WARPS * 32;
-constexpr int MF_LEVELS = 3;                         // bisection levels resolved per round
-constexpr int MF_NODES = (1 << MF_LEVELS) - 1;       // probes per round, one warp each
+constexpr int MF_LEVELS_MAX = 3;                     // bisection levels resolved per round, at most
+constexpr int MF_NODES_MAX = (1 << MF_LEVELS_MAX) - 1;   // probes per round, one warp each
 
 // One first-fit decreasing pass by one warp: client j = k * 32 + lane keeps its load in load[k].
 // Returns false at the first request that fits nowhere.  With RECORD, rc[r] gets the client of
@@ -60,12 +62,13 @@ __device__ __forceinline__ bool first_fit_pass(const uint32_t* __restrict__ Ts, 
 
 template <int KPL, typename L>
 __device__ void multifit_instance(const uint32_t* __restrict__ Ts, const uint32_t* __restrict__ od, int n,
-                                  int n_clients, unsigned long long sum_T, uint32_t max_T, int max_steps,
+                                  int n_clients, unsigned long long sum_T, uint32_t max_T, int max_steps, int levels,
                                   int32_t* __restrict__ asg, long long* __restrict__ load_out,
                                   long long* __restrict__ makespan_out, uint8_t* __restrict__ rank_client,
                                   int32_t* __restrict__ packer_out, uint8_t* s_rc) {
     __shared__ unsigned long long s_lo, s_hi;
-    __shared__ int s_steps, s_ok[MF_NODES], s_take;
+    __shared__ int s_steps, s_ok[MF_NODES_MAX], s_take;
+    const int nodes = (1 << levels) - 1;
     const int warp = warp_id(), lane = lane_id();
     const unsigned long long M = (unsigned long long)n_clients;
     if (threadIdx.x == 0) {
@@ -80,7 +83,7 @@ __device__ void multifit_instance(const uint32_t* __restrict__ Ts, const uint32_
         const unsigned long long lo0 = s_lo, hi0 = s_hi;
         const int steps0 = s_steps;
         if (lo0 >= hi0 || steps0 >= max_steps) break;            // uniform: shared values
-        if (warp < MF_NODES) {
+        if (warp < nodes) {
             // my node of the tree: depth d, path bits from the top (0 = the probe above succeeded)
             const int d = warp == 0 ? 0 : (warp < 3 ? 1 : 2);
             const int path = warp - ((1 << d) - 1);
@@ -102,7 +105,7 @@ __device__ void multifit_instance(const uint32_t* __restrict__ Ts, const uint32_
         if (threadIdx.x == 0) {
             unsigned long long lo = lo0, hi = hi0;
             int steps = steps0, node = 0;
-            for (int d = 0; d < MF_LEVELS && lo < hi && steps < max_steps; ++d) {
+            for (int d = 0; d < levels && lo < hi && steps < max_steps; ++d) {
                 const unsigned long long C = lo + (hi - lo) / 2;
                 const bool ok = s_ok[node] != 0;
                 if (ok) hi = C; else lo = C + 1;
@@ -136,7 +139,7 @@ __device__ void multifit_instance(const uint32_t* __restrict__ Ts, const uint32_
     }
     __syncthreads();
     if (s_take) {
-        for (int r = threadIdx.x; r < n; r += MF_THREADS) {
+        for (int r = threadIdx.x; r < n; r += blockDim.x) {
             const uint8_t c = s_rc[r];
             if (!HOS_IN(od[r], n, 401) || !HOS_IN(c, n_clients, 402)) continue;
             asg[od[r]] = (int32_t)c;
@@ -146,9 +149,9 @@ __device__ void multifit_instance(const uint32_t* __restrict__ Ts, const uint32_
 }
 
 template <int KPL>
-__global__ void __launch_bounds__(MF_THREADS)
+__global__ void __launch_bounds__(32 * MF_NODES_MAX)
 k_multifit(const uint32_t* __restrict__ T_sorted, const uint32_t* __restrict__ order,
-           const InstInfo* __restrict__ info, int n_req, int n_pad, int n_clients, int max_steps,
+           const InstInfo* __restrict__ info, int n_req, int n_pad, int n_clients, int max_steps, int levels,
            int32_t* __restrict__ assign, long long* __restrict__ load_out, long long* __restrict__ makespan_out,
            uint8_t* __restrict__ rank_client, int32_t* __restrict__ packer_out) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -165,10 +168,10 @@ k_multifit(const uint32_t* __restrict__ T_sorted, const uint32_t* __restrict__ o
     const unsigned long long M = (unsigned long long)n_clients;
     const unsigned long long hi = max((2ull * inf.sum_T + M - 1ull) / M, (unsigned long long)inf.max_T);
     if (hi <= 0xFFFFFFFFull)
-        multifit_instance<KPL, uint32_t>(Ts, od, n_req, n_clients, inf.sum_T, inf.max_T, max_steps, asg, load_out,
+        multifit_instance<KPL, uint32_t>(Ts, od, n_req, n_clients, inf.sum_T, inf.max_T, max_steps, levels, asg, load_out,
                                          makespan_out, rc, packer_out, smem_raw);
     else
-        multifit_instance<KPL, unsigned long long>(Ts, od, n_req, n_clients, inf.sum_T, inf.max_T, max_steps, asg,
+        multifit_instance<KPL, unsigned long long>(Ts, od, n_req, n_clients, inf.sum_T, inf.max_T, max_steps, levels, asg,
                                                    load_out, makespan_out, rc, packer_out, smem_raw);
 }
 
@@ -179,9 +182,16 @@ cudaError_t launch_multifit(const hos_batch& b, const uint32_t* T_sorted, const 
                             long long* makespan, uint8_t* rank_client, int32_t* packer, cudaStream_t st) {
     const int M = b.n_clients;
     const size_t smem = ((size_t)b.n_req + 15) & ~(size_t)15;
+    // as many levels per round (1, 3 or 7 warps per instance) as leave the schedulers room: up to
+    // about six warps per scheduler over the whole batch
+    int n_sm = 148, dev = 0;
+    if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev);
+    int levels = MF_LEVELS_MAX;
+    while (levels > 1 && (long long)b.n_inst * ((1 << levels) - 1) > 24ll * n_sm) --levels;
+    const int threads = 32 * ((1 << levels) - 1);
 #define HOS_MF(KPL)                                                                                        \
-    k_multifit<KPL><<<b.n_inst, MF_THREADS, smem, st>>>(T_sorted, order, info, b.n_req, n_pad, M, max_steps, \
-                                                        assign, load, makespan, rank_client, packer)
+    k_multifit<KPL><<<b.n_inst, threads, smem, st>>>(T_sorted, order, info, b.n_req, n_pad, M, max_steps,  \
+                                                     levels, assign, load, makespan, rank_client, packer)
     launch_hook("k_multifit", 0, st);
     if (M <= 32) HOS_MF(1);
     else if (M <= 64) HOS_MF(2);

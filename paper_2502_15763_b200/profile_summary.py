@@ -98,7 +98,8 @@ def main():
         kernels[name] = dict(unit=UNIT[name], units_in_capture=n,
                              dram_bytes_per_unit=(rec.get("dram_read", 0.0) + rec.get("dram_write", 0.0)) / n,
                              warp_inst_per_unit=rec.get("warp_inst", 0.0) / n, **rec)
-    doc = dict(source_hash=_build.source_hash(), workload=line["config"]["workload"], command=a.command,
+    doc = dict(source_hash=_build.source_hash(), workload=line["config"]["workload"], shape=line.get("shape"),
+               command=a.command,
                note="one launch of each kernel; per-launch times under the profiler are cold-cache and serialised",
                kernels=kernels)
     with open(a.out, "w") as fh:

@@ -434,3 +434,15 @@ def test_sort_falls_back_on_bunched_or_wide_keys(hos, kind):
     H.check_lower_bound(hos, p, o, M, cap, kv, cm)
     for mode in (ora.QUEUE_SORTED, ora.QUEUE_FCFS):
         H.check_simulate(hos, p, o, M, cap, kv, cm, g["assign"], (LAMBDA_ONE,), mode)
+
+
+@pytest.mark.parametrize("n_inst", [600, 1300])
+def test_multifit_on_large_batches(hos, n_inst):
+    """Batches large enough that the packing kernel resolves two levels, or one level, of the
+    bisection per round instead of three (the probe sequence must not depend on that)."""
+    rng = np.random.default_rng(n_inst)
+    n, M = 90, 7
+    p = rng.integers(1, 900, size=(n_inst, n)).astype(np.uint32)
+    o = rng.integers(1, 300, size=(n_inst, n)).astype(np.uint32)
+    cm = (20000, 40, 15000, 300, 16, 40, 350)
+    H.check_offline(hos, p, o, M, 8, 10 ** 6, cm, 4, multifit_steps=64)
