@@ -178,11 +178,14 @@ int hos_offline_pack(const hos_batch* batch, const hos_cost_model* cm, int ls_ro
  * bisection on a common capacity C over [max(ceil(sum T / M), max T), max(ceil(2 sum T / M), max T)],
  * at most `multifit_steps` probes (>= 1; 64 always converges), each probe a first-fit decreasing
  * pass (every request, longest first, to the lowest client where load + T <= C; success halves the
- * interval from above, failure from below).  The first-fit decreasing packing at the capacity found
- * replaces the longest-first list schedule of an instance when its largest load is strictly
- * smaller; the `ls_rounds` rounds then start from whichever was kept.
+ * interval from above, failure from below).  Both packings -- the longest-first list schedule and
+ * the first-fit decreasing one at the capacity found -- are improved by the same `ls_rounds`
+ * rounds of local search, and every instance keeps the better result: the list schedule's unless
+ * the other's largest load is strictly smaller (so the result is never worse than
+ * hos_offline_pack's).
  *   packer [n_inst] out, nullable: 1 where the MULTIFIT packing was kept, 0 where the list
- *   schedule was.  Everything else as in hos_offline_pack (same workspace size).
+ *   schedule was.  Everything else as in hos_offline_pack, except the workspace:
+ *   hos_offline_multifit_workspace_bytes (room for the second packing).
  */
 int hos_offline_pack_multifit(const hos_batch* batch, const hos_cost_model* cm, int multifit_steps,
                               int ls_rounds, int32_t* assign, int64_t* load, int64_t* makespan_est,
@@ -309,6 +312,7 @@ int hos_trace_offsets(const hos_client_result* cres, int64_t n_units, int64_t* t
                       void* stream);
 
 size_t hos_offline_workspace_bytes(const hos_batch* batch, int n_copies, int ls_rounds);
+size_t hos_offline_multifit_workspace_bytes(const hos_batch* batch, int ls_rounds);
 size_t hos_lower_bound_workspace_bytes(const hos_batch* batch);
 size_t hos_online_workspace_bytes(const hos_batch* batch, int n_lambda, int keep_events);
 

@@ -296,8 +296,9 @@ def simulate_steal(assign, p, o, M: int, cm, cap: int, kv_budget: int, lambda_q1
 def offline_pack(p, o, M: int, cm, ls_rounds: int = 0, multifit_steps: int = 0):
     """estimate -> order -> LPT (-> MULTIFIT) -> local search.  Returns dict with T, order, assign, load, ...
 
-    multifit_steps > 0: the MULTIFIT packing with at most that many probes replaces the LPT one
-    when its largest load is strictly smaller; `packer` says which was kept (0 LPT, 1 MULTIFIT)."""
+    multifit_steps > 0: the MULTIFIT packing with at most that many probes is improved by the same
+    local search, and the better of the two final packings is kept (the longest-first one unless the
+    other's largest load is strictly smaller); `packer` says which (0 LPT, 1 MULTIFIT)."""
     T = estimate(p, o, cm)
     od = order(T)
     assign, load = lpt(T, od, M)
@@ -305,8 +306,15 @@ def offline_pack(p, o, M: int, cm, ls_rounds: int = 0, multifit_steps: int = 0):
     packer = 0
     if multifit_steps > 0:
         mf = multifit(T, od, M, multifit_steps)
-        if mf is not None and int(mf[1].max()) < int(load.max()):
-            assign, load, packer = mf[0], mf[1], 1
+        if mf is not None:
+            a1, l1, ap1, lg1 = (local_search(T, assign, load, ls_rounds) if ls_rounds > 0
+                                else (assign, load, 0, np.zeros(0, dtype=MOVE_DTYPE)))
+            a2, l2, ap2, lg2 = (local_search(T, mf[0], mf[1], ls_rounds) if ls_rounds > 0
+                                else (mf[0], mf[1], 0, np.zeros(0, dtype=MOVE_DTYPE)))
+            if int(l2.max()) < int(l1.max()):
+                a1, l1, ap1, lg1, packer = a2, l2, ap2, lg2, 1
+            return dict(T=T, order=od, assign=a1, load=l1, makespan_est=int(l1.max()), rounds_applied=ap1,
+                        ls_log=lg1, lpt_assign=lpt_assign, lpt_load=lpt_load, packer=packer)
     applied, log = 0, np.zeros(0, dtype=MOVE_DTYPE)
     if ls_rounds > 0:
         assign, load, applied, log = local_search(T, assign, load, ls_rounds)

@@ -32,7 +32,7 @@ _SYMBOLS = ("hos_offline_pack", "hos_local_search", "hos_lower_bound", "hos_onli
             "hos_trace_offsets", "hos_offline_workspace_bytes", "hos_lower_bound_workspace_bytes",
             "hos_online_workspace_bytes", "hos_strerror", "hos_set_launch_hook",
             "hos_lower_bound_static", "hos_trace_fill", "hos_online_simulate_steal",
-            "hos_offline_pack_multifit", "hos_debug_bounds_violations")
+            "hos_offline_pack_multifit", "hos_debug_bounds_violations", "hos_offline_multifit_workspace_bytes")
 
 LAUNCH_HOOK = C.CFUNCTYPE(None, C.c_char_p, C.c_int, C.c_void_p, C.c_void_p)
 
@@ -76,7 +76,7 @@ def lib():
         L = C.CDLL(path)
         L.hos_debug_bounds_violations.restype = C.c_longlong
         for name in ("hos_offline_workspace_bytes", "hos_lower_bound_workspace_bytes",
-                     "hos_online_workspace_bytes"):
+                     "hos_online_workspace_bytes", "hos_offline_multifit_workspace_bytes"):
             getattr(L, name).restype = C.c_size_t
         L.hos_strerror.restype = C.c_char_p
         for name in ("hos_offline_pack", "hos_local_search", "hos_lower_bound",
@@ -199,8 +199,9 @@ def hos_offline_pack(p, o, n_clients: int, batch_cap: int, kv_budget: int, cost_
     b = _batch(p, o, n_clients, batch_cap, kv_budget, o_est, kv_reserve)
     cm = _cost(cost_model)
     L = lib()
-    need = L.hos_offline_workspace_bytes(C.byref(b), C.c_int(1), C.c_int(ls_rounds))
-    ws = ws if ws is not None else _workspace(need, p)
+    need = (L.hos_offline_multifit_workspace_bytes(C.byref(b), C.c_int(ls_rounds)) if multifit_steps > 0
+            else L.hos_offline_workspace_bytes(C.byref(b), C.c_int(1), C.c_int(ls_rounds)))
+    ws = ws if ws is not None and ws.numel() >= need else _workspace(need, p)
     dev = p.device
     if out is not None:
         assign = _dev(out["assign"], torch.int32, "out.assign")

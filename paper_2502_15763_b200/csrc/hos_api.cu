@@ -178,6 +178,26 @@ size_t hos_online_workspace_bytes(const hos_batch* b, int n_lambda, int keep_eve
 }
 
 namespace {
+// Buffers of the alternative packing (MULTIFIT start), behind the ordinary offline workspace.
+struct AltWs {
+    int32_t* assign; long long* load; long long* makespan; int32_t* rounds; hos_ls_move* log; int32_t* ok;
+    size_t bytes;
+};
+AltWs carve_alt(const hos_batch* b, void* ws, size_t at, int ls_rounds) {
+    AltWs a;
+    unsigned char* base = static_cast<unsigned char*>(ws);
+    size_t off = at;
+    const size_t n = (size_t)b->n_inst;
+    a.assign = reinterpret_cast<int32_t*>(base + off);      off += up(n * (size_t)b->n_req * 4);
+    a.load = reinterpret_cast<long long*>(base + off);      off += up(n * (size_t)b->n_clients * 8);
+    a.makespan = reinterpret_cast<long long*>(base + off);  off += up(n * 8);
+    a.rounds = reinterpret_cast<int32_t*>(base + off);      off += up(n * 4);
+    a.ok = reinterpret_cast<int32_t*>(base + off);          off += up(n * 4);
+    a.log = reinterpret_cast<hos_ls_move*>(base + off);     off += up(n * (size_t)(ls_rounds > 0 ? ls_rounds : 0) * sizeof(hos_ls_move));
+    a.bytes = off;
+    return a;
+}
+
 int offline_pack_impl(const hos_batch* b, const hos_cost_model* cm, int multifit_steps, int ls_rounds,
                       int32_t* assign, int64_t* load, int64_t* makespan_est, int32_t* rounds_applied,
                       hos_ls_move* ls_log, hos_lb* lb, int32_t* status, int32_t* packer, void* ws,
@@ -189,29 +209,32 @@ int offline_pack_impl(const hos_batch* b, const hos_cost_model* cm, int multifit
         return HOS_E_INVALID;
     if (lb && (rc = check_lb_range(b))) return rc;
     if (estimate_sort_smem(b->n_req) > SMEM_LIMIT) return HOS_E_UNSUPPORTED;
-    if ((rc = check_ws(ws, ws_bytes, hos_offline_workspace_bytes(b, 1, ls_rounds)))) return rc;
     const OfflineWs w = carve_offline(b, ws, 1, ls_rounds);
+    const AltWs alt = carve_alt(b, ws, w.bytes, ls_rounds);
+    if ((rc = check_ws(ws, ws_bytes, multifit_steps > 0 ? alt.bytes : w.bytes))) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const int n_pad = pad4(b->n_req);
+    long long* ld = reinterpret_cast<long long*>(load);
+    long long* mk = reinterpret_cast<long long*>(makespan_est);
+    auto search = [&](int32_t* a, long long* l, long long* m, int32_t* applied, hos_ls_move* log) {
+        if (ls_rounds == 0) return cuda_rc(cudaMemsetAsync(applied, 0, (size_t)b->n_inst * sizeof(int32_t), st));
+        return cuda_rc(launch_local_search(*b, w.T_sorted, w.order, w.info, n_pad, 1, ls_rounds, false, a, l, m, applied,
+                                           log, status, w.ls_T, w.ls_I, w.ls_C, w.ls_off, w.ls_bad, st));
+    };
     if ((rc = cuda_rc(launch_estimate_sort(*b, *cm, w.T_sorted, w.order, w.info, status, lb, n_pad, st)))) return rc;
-    if ((rc = cuda_rc(launch_lpt(*b, w.T_sorted, w.order, w.info, n_pad, assign,
-                                 reinterpret_cast<long long*>(load),
-                                 reinterpret_cast<long long*>(makespan_est), w.ls_C, st))))
+    if ((rc = cuda_rc(launch_lpt(*b, w.T_sorted, w.order, w.info, n_pad, assign, ld, mk, w.ls_C, st)))) return rc;
+    if ((rc = search(assign, ld, mk, rounds_applied, ls_log))) return rc;
+    if (multifit_steps == 0) return HOS_OK;
+    // The MULTIFIT packing, improved by the same local search, in buffers of its own; then the better
+    // of the two per instance.  (The packing kernel writes where its result beats the makespan it
+    // finds: with that preset to the largest value, wherever first-fit decreasing succeeded.)
+    if ((rc = cuda_rc(cudaMemsetAsync(alt.makespan, 0x7F, (size_t)b->n_inst * sizeof(long long), st)))) return rc;
+    if ((rc = cuda_rc(launch_multifit(*b, w.T_sorted, w.order, w.info, n_pad, multifit_steps, alt.assign, alt.load,
+                                      alt.makespan, w.ls_C, alt.ok, st))))
         return rc;
-    if (multifit_steps > 0) {
-        if ((rc = cuda_rc(launch_multifit(*b, w.T_sorted, w.order, w.info, n_pad, multifit_steps, assign,
-                                          reinterpret_cast<long long*>(load),
-                                          reinterpret_cast<long long*>(makespan_est), w.ls_C, packer, st))))
-            return rc;
-    } else if (packer) {
-        if ((rc = cuda_rc(cudaMemsetAsync(packer, 0, (size_t)b->n_inst * sizeof(int32_t), st)))) return rc;
-    }
-    if (ls_rounds == 0)
-        return cuda_rc(cudaMemsetAsync(rounds_applied, 0, (size_t)b->n_inst * sizeof(int32_t), st));
-    return cuda_rc(launch_local_search(*b, w.T_sorted, w.order, w.info, n_pad, 1, ls_rounds, false, assign,
-                                       reinterpret_cast<long long*>(load),
-                                       reinterpret_cast<long long*>(makespan_est), rounds_applied,
-                                       ls_log, status, w.ls_T, w.ls_I, w.ls_C, w.ls_off, w.ls_bad, st));
+    if ((rc = search(alt.assign, alt.load, alt.makespan, alt.rounds, ls_log ? alt.log : nullptr))) return rc;
+    return cuda_rc(launch_pick_packing(*b, ls_rounds, alt.ok, alt.assign, alt.load, alt.makespan, alt.rounds, alt.log,
+                                       assign, ld, mk, rounds_applied, ls_log, packer, st));
 }
 }  // namespace
 
@@ -221,6 +244,11 @@ int hos_offline_pack(const hos_batch* b, const hos_cost_model* cm, int ls_rounds
                      void* stream) {
     return offline_pack_impl(b, cm, 0, ls_rounds, assign, load, makespan_est, rounds_applied, ls_log, lb, status,
                              nullptr, ws, ws_bytes, stream);
+}
+
+size_t hos_offline_multifit_workspace_bytes(const hos_batch* b, int ls_rounds) {
+    if (!b || b->n_inst < 1 || b->n_req < 1 || b->n_clients < 1 || ls_rounds < 0) return 0;
+    return carve_alt(b, nullptr, carve_offline(b, nullptr, 1, ls_rounds).bytes, ls_rounds).bytes;
 }
 
 int hos_offline_pack_multifit(const hos_batch* b, const hos_cost_model* cm, int multifit_steps, int ls_rounds,

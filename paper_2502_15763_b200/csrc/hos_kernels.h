@@ -36,6 +36,10 @@ cudaError_t launch_lpt(const hos_batch& b, const uint32_t* T_sorted, const uint3
 cudaError_t launch_multifit(const hos_batch& b, const uint32_t* T_sorted, const uint32_t* order,
                             const InstInfo* info, int n_pad, int max_steps, int32_t* assign, long long* load,
                             long long* makespan, uint8_t* rank_client, int32_t* packer, cudaStream_t st);
+cudaError_t launch_pick_packing(const hos_batch& b, int rounds, const int32_t* alt_ok, const int32_t* alt_assign,
+                                const long long* alt_load, const long long* alt_makespan, const int32_t* alt_rounds,
+                                const hos_ls_move* alt_log, int32_t* assign, long long* load, long long* makespan,
+                                int32_t* rounds_applied, hos_ls_move* ls_log, int32_t* packer, cudaStream_t st);
 cudaError_t launch_local_search(const hos_batch& b, const uint32_t* T_sorted, const uint32_t* order,
                                 const InstInfo* info, int n_pad, int n_copies, int rounds,
                                 bool load_from_assign, int32_t* assign, long long* load,

@@ -175,6 +175,38 @@ k_multifit(const uint32_t* __restrict__ T_sorted, const uint32_t* __restrict__ o
                                                    load_out, makespan_out, rc, packer_out, smem_raw);
 }
 
+// Keeps, per instance, the better of two finished packings: the alternative replaces the primary
+// one when its packing exists (alt_ok) and its largest load is strictly smaller.
+__global__ void __launch_bounds__(256)
+k_pick_packing(int n_req, int n_clients, int rounds, const int32_t* __restrict__ alt_ok,
+               const int32_t* __restrict__ alt_assign, const long long* __restrict__ alt_load,
+               const long long* __restrict__ alt_makespan, const int32_t* __restrict__ alt_rounds,
+               const hos_ls_move* __restrict__ alt_log, int32_t* __restrict__ assign, long long* __restrict__ load,
+               long long* __restrict__ makespan, int32_t* __restrict__ rounds_applied,
+               hos_ls_move* __restrict__ ls_log, int32_t* __restrict__ packer) {
+    const int inst = blockIdx.x;
+    const bool take = alt_ok[inst] != 0 && alt_makespan[inst] < makespan[inst];   // uniform over the CTA
+    __syncthreads();                                     // everyone has read the old makespan
+    if (threadIdx.x == 0 && packer) packer[inst] = take ? 1 : 0;
+    if (!take) return;
+    for (int i = threadIdx.x; i < n_req; i += blockDim.x) assign[(size_t)inst * n_req + i] = alt_assign[(size_t)inst * n_req + i];
+    for (int j = threadIdx.x; j < n_clients; j += blockDim.x) load[(size_t)inst * n_clients + j] = alt_load[(size_t)inst * n_clients + j];
+    if (ls_log)
+        for (int r = threadIdx.x; r < rounds; r += blockDim.x) ls_log[(size_t)inst * rounds + r] = alt_log[(size_t)inst * rounds + r];
+    if (threadIdx.x == 0) { makespan[inst] = alt_makespan[inst]; rounds_applied[inst] = alt_rounds[inst]; }
+}
+
+cudaError_t launch_pick_packing(const hos_batch& b, int rounds, const int32_t* alt_ok, const int32_t* alt_assign,
+                                const long long* alt_load, const long long* alt_makespan, const int32_t* alt_rounds,
+                                const hos_ls_move* alt_log, int32_t* assign, long long* load, long long* makespan,
+                                int32_t* rounds_applied, hos_ls_move* ls_log, int32_t* packer, cudaStream_t st) {
+    launch_hook("k_pick_packing", 0, st);
+    k_pick_packing<<<b.n_inst, 256, 0, st>>>(b.n_req, b.n_clients, rounds, alt_ok, alt_assign, alt_load, alt_makespan,
+                                             alt_rounds, alt_log, assign, load, makespan, rounds_applied, ls_log, packer);
+    launch_hook("k_pick_packing", 1, st);
+    return cudaGetLastError();
+}
+
 HOS_DEFINE_BOUNDS_READER(debug_bounds_multifit)
 
 cudaError_t launch_multifit(const hos_batch& b, const uint32_t* T_sorted, const uint32_t* order,

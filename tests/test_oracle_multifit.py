@@ -106,16 +106,28 @@ def test_bounds_against_the_exhaustive_optimum(seed):
         assert np.array_equal(both["assign"], lpt["assign"])
 
 
-def test_multifit_then_local_search_keeps_the_books():
+def test_better_of_two_finished_packings():
+    """With local-search rounds both starts are improved and the better final packing is kept: never
+    worse than the list schedule with the same rounds, the books stay consistent, and the MULTIFIT
+    start does win on some instances."""
     rng = np.random.default_rng(5)
     taken = 0
-    for _ in range(30):
+    for case in range(40):
         n, M = int(rng.integers(20, 200)), int(rng.integers(2, 9))
+        rounds = (0, 1, 3, 10)[case % 4]
         p = rng.integers(1, 400, size=n).astype(np.uint32)
         o = rng.integers(1, 400, size=n).astype(np.uint32)
-        r = ora.offline_pack(p, o, M, CM, 10, multifit_steps=64)
+        r = ora.offline_pack(p, o, M, CM, rounds, multifit_steps=64)
+        plain = ora.offline_pack(p, o, M, CM, rounds)
         T = ora.estimate(p, o, CM)
         assert all(int(r["load"][j]) == int(T[r["assign"] == j].sum()) for j in range(M))
-        assert r["makespan_est"] <= ora.offline_pack(p, o, M, CM, 0)["makespan_est"]
+        assert r["makespan_est"] <= plain["makespan_est"]
+        assert (r["packer"] == 1) == (r["makespan_est"] < plain["makespan_est"])
+        if r["packer"] == 0:
+            assert np.array_equal(r["assign"], plain["assign"]) and r["rounds_applied"] == plain["rounds_applied"]
+        else:                       # the kept packing is the search started from the MULTIFIT one
+            mf = ora.multifit(T, ora.order(T), M, 64)
+            a, l, applied, _ = ora.local_search(T, mf[0], mf[1], rounds)
+            assert np.array_equal(r["assign"], a) and r["rounds_applied"] == applied
         taken += r["packer"]
-    assert taken > 0            # the stronger packing does get used on such instances
+    assert taken > 0
