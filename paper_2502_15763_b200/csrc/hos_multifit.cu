@@ -11,9 +11,10 @@
 //                the passes.  That is for small batches, where the chain's latency is all there
 //                is; a batch that fills the GPU anyway is bound by instruction issue, and there
 //                the four speculative probes in seven that are thrown away cost more than the
-//                shorter chain saves, so it runs one warp per instance, one level per round.
-//                A last pass packs at the capacity found; the result replaces the
-//                list-scheduling one only when its largest load is strictly smaller.
+//                shorter chain saves, so larger batches resolve two levels per round (three
+//                warps) or one (the plain bisection).  A last pass packs at the capacity found
+//                and writes it where it beats the makespan it finds there (the caller presets
+//                that to the largest value and chooses between the packings afterwards).
 #include "hos_common.cuh"
 #include "hos_kernels.h"
 
