@@ -22,7 +22,7 @@
  *   - Workspaces are scratch: contents are undefined before and after a call;
  *     base must be 256-byte aligned.  Two calls that share a workspace or an
  *     output buffer must be ordered on the stream.
- *   - Shape limits of this build: n_clients <= 256, batch_cap <= 256,
+ *   - Shape limits of this library: n_clients <= 256, batch_cap <= 256,
  *     n_req <= 24384, kv_budget < 2^31, estimated times T_i < 2^32; for the lower bounds
  *     also n_req * R^2 / 2 < 2^63, R = the most KV tokens one request may need
  *     (kv_reserve_tokens if set, else kv_budget).
@@ -66,7 +66,7 @@ enum {
 enum { HOS_QUEUE_SORTED = 0, HOS_QUEUE_FCFS = 1 };
 
 /* Integer-microsecond cost model.  The paper profiles both stage times as affine in the
- * token counts (Numerical Experiment, "Experiment settings"); the KV term is this build's
+ * token counts (Numerical Experiment, "Experiment settings"); the KV term is the synthetic workloads'
  * workload definition.  prefill iteration = prefill_fixed_us + prefill_per_token_us * sum p;
  * decode iteration = decode_fixed_us + decode_per_seq_us * B + floor(sum KV / decode_kv_div);
  * estimated request time T_i = est_per_prompt_token * p_i + est_per_output_token * o_i.
@@ -252,7 +252,7 @@ int hos_online_simulate(const hos_batch* batch, const int32_t* assign, const hos
  * candidate for its next prefill.  Everything else -- queues, iteration rule, results, trace,
  * status bits -- is as in hos_online_simulate.
  *   served_by [n_inst][n_lambda][n_req]  out, nullable: the client that served each request.
- * Limit of this build: n_clients (rounded up to 32) * batch_cap heap entries of one simulation
+ * Limit of this library: n_clients (rounded up to 32) * batch_cap heap entries of one simulation
  * must fit one CTA's shared memory (HOS_E_UNSUPPORTED otherwise).
  */
 int hos_online_simulate_steal(const hos_batch* batch, const int32_t* assign, const hos_cost_model* cm,

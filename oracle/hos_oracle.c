@@ -301,7 +301,7 @@ void ora_queue_build(int n, int M, const int32_t* assign, const uint32_t* p, con
     free(a);
 }
 
-/* Trace hash (this build's own definition; the paper has none): h <- (h + dur + C1 kind_n +
+/* Trace hash (a definition made for this checker and the library; the paper has none): h <- (h + dur + C1 kind_n +
  * C2 tokens + C3 aux) * M  mod 2^64 per record, in trace order, from h = INIT. */
 #define ORA_HASH_INIT  0xCBF29CE484222325ull
 #define ORA_HASH_C1    0x9E3779B1ull
