@@ -66,8 +66,8 @@ enum {
 enum { HOS_QUEUE_SORTED = 0, HOS_QUEUE_FCFS = 1 };
 
 /* Integer-microsecond cost model.  The paper profiles both stage times as affine in the
- * token counts (Numerical Experiment, "Experiment settings"); the KV term is the synthetic workloads'
- * workload definition.  prefill iteration = prefill_fixed_us + prefill_per_token_us * sum p;
+ * token counts (Numerical Experiment, "Experiment settings"); the KV term comes from the
+ * synthetic workloads' definition.  prefill iteration = prefill_fixed_us + prefill_per_token_us * sum p;
  * decode iteration = decode_fixed_us + decode_per_seq_us * B + floor(sum KV / decode_kv_div);
  * estimated request time T_i = est_per_prompt_token * p_i + est_per_output_token * o_i.
  * Requires decode_fixed_us >= 1, decode_kv_div >= 1, and both iteration durations < 2^31
