@@ -591,6 +591,27 @@ def run_ours(args):
         run_steal()
         torch.cuda.synchronize()
         steal_ms = timed_steps(torch, run_steal, 3, flush) / 3
+        # the traced form: the same call with its event log, offsets, and the trace rebuilt from the log
+        state = {}
+
+        def run_steal_logged():
+            state["sim"] = hos.hos_online_simulate_steal(*pipe.args(), pipe.out["pk"]["assign"], pipe.lam,
+                                                         hos.HOS_QUEUE_SORTED, keep_events=True, ws=pipe.ws_on,
+                                                         **pipe.kw)
+            state["off"] = hos.hos_trace_offsets(state["sim"]["cres"])
+
+        run_steal_logged()
+        n_steal_iters = int(state["off"][-1].item())
+        steal_trace = pipe.trace if n_steal_iters <= pipe.trace.shape[0] else \
+            torch.empty((n_steal_iters, 16), dtype=torch.uint8, device=dev)
+        run_steal_fill = lambda: hos.hos_trace_fill(*pipe.args(), len(w.lambdas_q16), state["sim"], steal_trace,
+                                                    state["off"], **pipe.kw)
+        run_steal_fill()
+        torch.cuda.synchronize()
+        steal_log_ms = timed_steps(torch, run_steal_logged, 3, flush) / 3
+        steal_fill_ms = timed_steps(torch, run_steal_fill, 3, flush) / 3
+        del steal_trace
+        pipe.step()                                   # the plain simulator's log is back in the workspace
 
     e2e_trace = None
     if rank == 0 and not args.skip_e2e and not args.skip_e2e_trace:
@@ -730,6 +751,9 @@ def run_ours(args):
             "kernels": rows,
             "request_stealing": None if steal_ms is None else {
                 "call": "hos_online_simulate_steal", "ms_per_call": steal_ms,
+                "ms_per_call_with_event_log_and_offsets": steal_log_ms,
+                "trace_fill_ms": steal_fill_ms, "trace_iterations": n_steal_iters,
+                "trace_fill_gbs": 16.0 * n_steal_iters / (steal_fill_ms * 1e-3) / 1e9,
                 "simulations_per_s": w.n_inst * len(w.lambdas_q16) / (steal_ms * 1e-3),
                 "plain_simulate_ms": rows.get("k_simulate", {}).get("ms_per_launch")},
             "cpu_baseline": {"value": cpu_inst, "unit": UNIT, "cores": 1, "kind": "oracle",

@@ -252,6 +252,10 @@ int hos_online_simulate(const hos_batch* batch, const int32_t* assign, const hos
  * candidate for its next prefill.  Everything else -- queues, iteration rule, results, trace,
  * status bits -- is as in hos_online_simulate.
  *   served_by [n_inst][n_lambda][n_req]  out, nullable: the client that served each request.
+ *   keep_events  as in hos_online_simulate: the event log stays in `ws` for hos_trace_fill.  Here
+ *              a client's logged iterations are not bounded by its own queue, only all clients'
+ *              together by two per request of the instance; the log is handed out in chunks.
+ *              Same workspace size as for hos_online_simulate with keep_events.
  * Limit of this library: n_clients (rounded up to 32) * batch_cap heap entries of one simulation
  * must fit one CTA's shared memory (HOS_E_UNSUPPORTED otherwise).
  */
@@ -259,11 +263,12 @@ int hos_online_simulate_steal(const hos_batch* batch, const int32_t* assign, con
                               const uint32_t* lambda_q16, int n_lambda, int queue_order,
                               uint32_t max_iters, hos_client_result* cres, hos_sim_result* sres,
                               hos_iter_rec* trace, const int64_t* trace_off, int32_t* status,
-                              int32_t* served_by, void* ws, size_t ws_bytes, void* stream);
+                              int32_t* served_by, int keep_events, void* ws, size_t ws_bytes,
+                              void* stream);
 
 /*
- * The iteration trace from the event log of a hos_online_simulate call made with
- * keep_events != 0: between two logged iterations a client only decodes, with a constant
+ * The iteration trace from the event log of a hos_online_simulate or hos_online_simulate_steal
+ * call made with keep_events != 0 (the workspace records which of the two wrote it): between two logged iterations a client only decodes, with a constant
  * batch and sum KV growing by B per iteration, so every record in between follows from the
  * log (same records, bit for bit, as a traced simulation).  `batch`, `cm`, `n_lambda`, `cres`
  * and `ws` must be those of that call, and `ws` untouched since.  trace / trace_off as in

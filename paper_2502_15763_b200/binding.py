@@ -348,8 +348,12 @@ def hos_online_simulate(p, o, n_clients: int, batch_cap: int, kv_budget: int, co
 
 def hos_online_simulate_steal(p, o, n_clients: int, batch_cap: int, kv_budget: int, cost_model, assign,
                               lambda_q16, queue_order: int = HOS_QUEUE_SORTED, max_iters: int = 0x7FFFFFFF,
-                              trace=None, trace_off=None, want_served_by: bool = False, ws=None, o_est=None, kv_reserve: int = 0):
-    """hos_online_simulate with Algorithm 1's request stealing between the clients of an instance."""
+                              trace=None, trace_off=None, want_served_by: bool = False, keep_events: bool = False,
+                              ws=None, o_est=None, kv_reserve: int = 0):
+    """hos_online_simulate with Algorithm 1's request stealing between the clients of an instance.
+
+    keep_events: leave the event log in the returned workspace `ws` for hos_trace_fill.
+    """
     torch = _torch()
     b = _batch(p, o, n_clients, batch_cap, kv_budget, o_est, kv_reserve)
     cm = _cost(cost_model)
@@ -359,7 +363,7 @@ def hos_online_simulate_steal(p, o, n_clients: int, batch_cap: int, kv_budget: i
     lambda_q16 = _dev(lambda_q16, torch.int32, "lambda_q16")
     n_lambda = int(lambda_q16.numel())
     L = lib()
-    need = L.hos_online_workspace_bytes(C.byref(b), C.c_int(n_lambda), C.c_int(0))
+    need = L.hos_online_workspace_bytes(C.byref(b), C.c_int(n_lambda), C.c_int(int(keep_events)))
     ws = ws if ws is not None else _workspace(need, p)
     dev = p.device
     cres = torch.empty((b.n_inst, n_lambda, n_clients, CLIENT_RESULT_DTYPE.itemsize), dtype=torch.uint8, device=dev)
@@ -373,8 +377,8 @@ def hos_online_simulate_steal(p, o, n_clients: int, batch_cap: int, kv_budget: i
             raise ValueError("trace_off must have n_units + 1 entries")
     rc = L.hos_online_simulate_steal(C.byref(b), _ptr(assign), C.byref(cm), _ptr(lambda_q16), C.c_int(n_lambda),
                                      C.c_int(queue_order), C.c_uint32(max_iters), _ptr(cres), _ptr(sres),
-                                     _ptr(trace), _ptr(trace_off), _ptr(status), _ptr(served), _ptr(ws),
-                                     C.c_size_t(ws.numel()), _stream())
+                                     _ptr(trace), _ptr(trace_off), _ptr(status), _ptr(served),
+                                     C.c_int(int(keep_events)), _ptr(ws), C.c_size_t(ws.numel()), _stream())
     _check(rc, "hos_online_simulate_steal")
     return dict(cres=cres, sres=sres, status=status, served_by=served, ws=ws)
 
@@ -382,7 +386,7 @@ def hos_online_simulate_steal(p, o, n_clients: int, batch_cap: int, kv_budget: i
 def hos_trace_fill(p, o, n_clients: int, batch_cap: int, kv_budget: int, cost_model, n_lambda: int,
                    sim, trace, trace_off, o_est=None, kv_reserve: int = 0):
     """The full iteration trace from the event log of `sim`, the dict returned by
-    hos_online_simulate(..., keep_events=True) for the same batch.  ORs HOS_ST_TRACE into
+    hos_online_simulate or hos_online_simulate_steal (..., keep_events=True) for the same batch.  ORs HOS_ST_TRACE into
     sim["status"] where the slots are too few.  Returns `trace`."""
     torch = _torch()
     b = _batch(p, o, n_clients, batch_cap, kv_budget, o_est, kv_reserve)

@@ -105,8 +105,7 @@ struct OnlineWs {
     int32_t* q_off;
     unsigned long long* inst_O;
     int32_t* inst_status;
-    uint32_t* event_count;      // [n_units]                      (keep_events only)
-    uint4* events;              // [n_sims][n_pad][2 events]      (keep_events only)
+    EventLog log;               // all null without keep_events
     size_t bytes;
 };
 OnlineWs carve_online(const hos_batch* b, void* ws, int n_lambda, int keep_events) {
@@ -121,12 +120,18 @@ OnlineWs carve_online(const hos_batch* b, void* ws, int n_lambda, int keep_event
     w.q_off = reinterpret_cast<int32_t*>(base + off);             off += up((size_t)b->n_inst * (b->n_clients + 1) * 4);
     w.inst_O = reinterpret_cast<unsigned long long*>(base + off); off += up((size_t)b->n_inst * 8);
     w.inst_status = reinterpret_cast<int32_t*>(base + off);       off += up((size_t)b->n_inst * 4);
-    w.event_count = nullptr;
-    w.events = nullptr;
+    w.log = EventLog{nullptr, 0, nullptr, nullptr, 0, nullptr, nullptr, nullptr};
     if (keep_events) {
         const size_t sims = (size_t)b->n_inst * (size_t)n_lambda;
-        w.event_count = reinterpret_cast<uint32_t*>(base + off);  off += up(sims * b->n_clients * 4);
-        w.events = reinterpret_cast<uint4*>(base + off);          off += up(sims * pad4(b->n_req) * 2 * 16);
+        const size_t chunks = (size_t)event_log_chunks(pad4(b->n_req), b->n_clients);
+        w.log.pool_chunks = (int)chunks;
+        w.log.ev_stride = (long long)(chunks * event_log_chunk_entries());
+        w.log.kind = reinterpret_cast<uint32_t*>(base + off);         off += up(4);
+        w.log.event_count = reinterpret_cast<uint32_t*>(base + off);  off += up(sims * b->n_clients * 4);
+        w.log.dir_start = reinterpret_cast<uint32_t*>(base + off);    off += up(sims * b->n_clients * 4);
+        w.log.chunk_tag = reinterpret_cast<uint32_t*>(base + off);    off += up(sims * chunks * 4);
+        w.log.chunk_dir = reinterpret_cast<uint32_t*>(base + off);    off += up(sims * chunks * 4);
+        w.log.events = reinterpret_cast<uint4*>(base + off);          off += up(sims * (size_t)w.log.ev_stride * 16);
     }
     w.bytes = off;
     return w;
@@ -321,8 +326,7 @@ int hos_online_simulate(const hos_batch* b, const int32_t* assign, const hos_cos
         return rc;
     if ((rc = cuda_rc(launch_simulate(*b, *cm, lambda_q16, n_lambda, max_iters, w.q_po, w.q_off,
                                       w.inst_status, n_pad, cres, trace,
-                                      reinterpret_cast<const long long*>(trace_off), status, w.events,
-                                      w.event_count, st))))
+                                      reinterpret_cast<const long long*>(trace_off), status, w.log, st))))
         return rc;
     return cuda_rc(launch_finalize(*b, n_lambda, w.inst_O, cres, sres, st));
 }
@@ -330,8 +334,8 @@ int hos_online_simulate(const hos_batch* b, const int32_t* assign, const hos_cos
 int hos_online_simulate_steal(const hos_batch* b, const int32_t* assign, const hos_cost_model* cm,
                               const uint32_t* lambda_q16, int n_lambda, int queue_order, uint32_t max_iters,
                               hos_client_result* cres, hos_sim_result* sres, hos_iter_rec* trace,
-                              const int64_t* trace_off, int32_t* status, int32_t* served_by, void* ws,
-                              size_t ws_bytes, void* stream) {
+                              const int64_t* trace_off, int32_t* status, int32_t* served_by, int keep_events,
+                              void* ws, size_t ws_bytes, void* stream) {
     int rc = check_batch(b);
     if (rc) return rc;
     if ((rc = check_cost(cm, b))) return rc;
@@ -345,8 +349,8 @@ int hos_online_simulate_steal(const hos_batch* b, const int32_t* assign, const h
     // every client's heap of one simulation shares a CTA's shared memory
     const bool may_be_wide = b->kv_budget >= 65536;
     if (simulate_steal_smem(b->n_clients, b->batch_cap, may_be_wide) + 8 * 1024 > SMEM_LIMIT) return HOS_E_UNSUPPORTED;
-    if ((rc = check_ws(ws, ws_bytes, hos_online_workspace_bytes(b, n_lambda, 0)))) return rc;
-    const OnlineWs w = carve_online(b, ws, n_lambda, 0);
+    if ((rc = check_ws(ws, ws_bytes, hos_online_workspace_bytes(b, n_lambda, keep_events)))) return rc;
+    const OnlineWs w = carve_online(b, ws, n_lambda, keep_events);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const int n_pad = pad4(b->n_req);
     if (max_iters > 0x7FFFFFFFu) max_iters = 0x7FFFFFFFu;
@@ -356,7 +360,7 @@ int hos_online_simulate_steal(const hos_batch* b, const int32_t* assign, const h
     if ((rc = cuda_rc(launch_simulate_steal(*b, *cm, lambda_q16, n_lambda, max_iters, w.q_po, w.q_key, w.q_req, w.q_off,
                                             w.inst_status, n_pad, cres, trace,
                                             reinterpret_cast<const long long*>(trace_off), status, served_by,
-                                            st))))
+                                            w.log, st))))
         return rc;
     return cuda_rc(launch_finalize(*b, n_lambda, w.inst_O, cres, sres, st));
 }
@@ -371,7 +375,7 @@ int hos_trace_fill(const hos_batch* b, const hos_cost_model* cm, int n_lambda, c
     if ((long long)b->n_inst * n_lambda > 0x7FFFFFFFll / 4) return HOS_E_UNSUPPORTED;
     if ((rc = check_ws(ws, ws_bytes, hos_online_workspace_bytes(b, n_lambda, 1)))) return rc;
     const OnlineWs w = carve_online(b, const_cast<void*>(ws), n_lambda, 1);
-    return cuda_rc(launch_trace_fill(*b, *cm, n_lambda, w.q_off, pad4(b->n_req), cres, w.events, w.event_count,
+    return cuda_rc(launch_trace_fill(*b, *cm, n_lambda, w.q_off, pad4(b->n_req), cres, w.log,
                                      trace, reinterpret_cast<const long long*>(trace_off), status,
                                      static_cast<cudaStream_t>(stream)));
 }

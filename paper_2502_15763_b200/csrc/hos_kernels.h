@@ -50,21 +50,37 @@ size_t local_search_index_bytes(int n_req);
 cudaError_t launch_queue_build(const hos_batch& b, const int32_t* assign, uint32_t p_max, int queue_order, uint2* q_po,
                                uint32_t* q_key, uint32_t* q_req, int32_t* q_off, unsigned long long* inst_O,
                                int32_t* inst_status, int n_pad, cudaStream_t st);
+// The event log of a simulation call, in the caller's workspace (all null without a log).  A
+// simulation owns `ev_stride` = pool_chunks * event_log_chunk_entries() entries of `events`: the
+// plain simulator gives client c the entries from 2 * q_off[c] on; the stealing simulator hands
+// them out in chunks and lists every client's chunks in `chunk_dir` from `dir_start[unit]` on.
+struct EventLog {
+    uint4* events;              // [n_sims][ev_stride]
+    long long ev_stride;
+    uint32_t* event_count;      // [n_units]
+    uint32_t* kind;             // one word: which simulator wrote the log
+    int pool_chunks;            // chunks per simulation
+    uint32_t* chunk_tag;        // [n_sims][pool_chunks]  owner << 16 | number within the owner's log
+    uint32_t* chunk_dir;        // [n_sims][pool_chunks]  chunks by owner, then by number
+    uint32_t* dir_start;        // [n_units]
+};
+int event_log_chunks(int n_pad, int n_clients);
+int event_log_chunk_entries();
 cudaError_t launch_simulate(const hos_batch& b, const hos_cost_model& cm, const uint32_t* lambda_q16,
                             int n_lambda, uint32_t max_iters, const uint2* q_po, const int32_t* q_off,
                             const int32_t* inst_status, int n_pad, hos_client_result* cres,
                             hos_iter_rec* trace, const long long* trace_off, int32_t* status,
-                            uint4* events, uint32_t* event_count, cudaStream_t st);
+                            const EventLog& log, cudaStream_t st);
 size_t simulate_steal_smem(int n_clients, int cap, bool wide);
 cudaError_t launch_simulate_steal(const hos_batch& b, const hos_cost_model& cm, const uint32_t* lambda_q16,
                                   int n_lambda, uint32_t max_iters, const uint2* q_po, const uint32_t* q_key,
                                   const uint32_t* q_req,
                                   const int32_t* q_off, const int32_t* inst_status, int n_pad,
                                   hos_client_result* cres, hos_iter_rec* trace, const long long* trace_off,
-                                  int32_t* status, int32_t* served_by, cudaStream_t st);
+                                  int32_t* status, int32_t* served_by, const EventLog& log, cudaStream_t st);
 cudaError_t launch_trace_fill(const hos_batch& b, const hos_cost_model& cm, int n_lambda,
                               const int32_t* q_off, int n_pad, const hos_client_result* cres,
-                              const uint4* events, const uint32_t* event_count, hos_iter_rec* trace,
+                              const EventLog& log, hos_iter_rec* trace,
                               const long long* trace_off, int32_t* status, cudaStream_t st);
 cudaError_t launch_finalize(const hos_batch& b, int n_lambda, const unsigned long long* inst_O,
                             hos_client_result* cres, hos_sim_result* sres, cudaStream_t st);

@@ -177,6 +177,14 @@ k_queue_build(const uint32_t* __restrict__ p, const uint32_t* __restrict__ o,
 constexpr uint32_t EMPTY = 0xFFFFFFFFu;
 constexpr int TF_RING = 128;                // log entries in a warp's ring in k_trace_fill (a power of two)
 constexpr int TF_AHEAD = 64;                // entries that the ring is filled ahead of their use, at least
+// Event logs (what k_trace_fill rebuilds a trace from).  The plain simulator logs at most two
+// events per request of the client's own queue, so client c of a simulation owns the entries
+// [2 * q_off[c], 2 * q_off[c + 1]) of the simulation's log.  Under stealing a client's events
+// are not bounded by its own queue, only their sum over the clients is (every request is
+// admitted once and retired once): the clients take chunks of LOG_CHUNK entries from the
+// simulation's log as they need them, and a directory lists every client's chunks in order.
+constexpr uint32_t LOG_PER_QUEUE = 1u, LOG_CHUNKED = 2u;   // which form a workspace's log has
+constexpr int LOG_CHUNK = 32;
 constexpr int SIM_QUIET_MAX = 16;         // plain decode iterations per pass of the simulator's loop
 constexpr unsigned long long HASH_INIT = 0xCBF29CE484222325ull;
 constexpr uint32_t HASH_C1 = 0x9E3779B1u, HASH_C2 = 0x85EBCA77u, HASH_C3 = 0xC2B2AE3Du, HASH_M = 0x27D4EB2Fu;
@@ -216,10 +224,11 @@ k_simulate(const uint2* __restrict__ q_po, const int32_t* __restrict__ q_off,
            hos_cost_model cm, int q_shift, uint32_t max_iters,
            hos_client_result* __restrict__ cres,
            hos_iter_rec* __restrict__ trace, const long long* __restrict__ trace_off,
-           int32_t* __restrict__ status_out, uint4* __restrict__ events,
-           uint32_t* __restrict__ event_count) {
+           int32_t* __restrict__ status_out, uint4* __restrict__ events, long long ev_stride,
+           uint32_t* __restrict__ event_count, uint32_t* __restrict__ log_kind) {
     typedef typename E::T entry_t;
     extern __shared__ __align__(16) unsigned char smem_raw[];
+    if (log_kind && blockIdx.x == 0 && threadIdx.x == 0) *log_kind = LOG_PER_QUEUE;
     // warps of a CTA are independent; each has its own block of cap * lanes heap entries.  Only the
     // first `lanes` lanes of a warp simulate a client: with fewer clients per warp the lanes wait
     // less for each other's events, and a small batch spreads over more SMs.
@@ -270,7 +279,7 @@ k_simulate(const uint2* __restrict__ q_po, const int32_t* __restrict__ q_off,
         tr_lim = capr > 0x7FFFFFFFll ? 0x7FFFFFFFu : (uint32_t)(capr < 0 ? 0 : capr);
     }
     // event log of this client: one 16-byte entry per logged iteration, at most 2 per request
-    uint4* ev = events ? events + ((size_t)(inst * n_lambda + l) * n_pad + q0) * 2 : nullptr;
+    uint4* ev = events ? events + (size_t)(inst * n_lambda + l) * ev_stride + (size_t)q0 * 2 : nullptr;
     uint32_t n_ev = 0;
     uint2 nxt = make_uint2(0u, 0u);          // queue entries head + nA and head + nA + 1,
     uint2 nxt2 = make_uint2(0u, 0u);         // fetched ahead of their use
@@ -492,9 +501,16 @@ k_simulate_steal(const uint2* __restrict__ q_po, const uint32_t* __restrict__ q_
                  int n_pad, int cap, uint32_t kv_budget, hos_cost_model cm, int q_shift,
                  uint32_t max_iters, hos_client_result* __restrict__ cres,
                  hos_iter_rec* __restrict__ trace, const long long* __restrict__ trace_off,
-                 int32_t* __restrict__ status_out, int32_t* __restrict__ served_by) {
+                 int32_t* __restrict__ status_out, int32_t* __restrict__ served_by,
+                 uint4* __restrict__ events, long long ev_stride, int pool_chunks,
+                 uint32_t* __restrict__ chunk_tag, uint32_t* __restrict__ chunk_dir,
+                 uint32_t* __restrict__ dir_start, uint32_t* __restrict__ event_count,
+                 uint32_t* __restrict__ log_kind) {
     typedef typename E::T entry_t;
     extern __shared__ __align__(16) unsigned char smem_raw[];
+    __shared__ unsigned s_chunks;                         // chunks of the event log handed out so far
+    __shared__ uint32_t s_dstart[MAX_CLIENTS];            // first directory entry of each client
+    __shared__ uint32_t s_wchunks[MAX_CLIENTS / 32];
     __shared__ int s_ustart[MAX_CLIENTS];                 // first unclaimed position of each queue
     __shared__ unsigned long long s_remain[MAX_CLIENTS];  // p+o still unclaimed in each queue
     __shared__ unsigned long long s_total;                // sum of s_remain
@@ -512,11 +528,13 @@ k_simulate_steal(const uint2* __restrict__ q_po, const uint32_t* __restrict__ q_
     auto heap_st = [&](int sl, entry_t v) { if (HOS_IN(sl, cap, 321)) heap[sl * stride] = v; };
 
     const int ist = inst_status[inst];
+    if (log_kind && blockIdx.x == 0 && threadIdx.x == 0) *log_kind = LOG_CHUNKED;
     if (((ist & INST_WIDE) != 0) != (sizeof(entry_t) == 8)) return;   // the other instantiation's instance
     if (ist & HOS_ST_INVALID) {
         if (is_client) {
             cres[unit] = hos_client_result{0, 0, 0u, 0u, 0ull, 0.0};
             status_out[unit] = HOS_ST_INVALID;
+            if (events) { event_count[unit] = 0; dir_start[unit] = 0; }
         }
         if (served_by)
             for (int i = c; i < n_req; i += stride) served_by[(size_t)sim * n_req + i] = -1;
@@ -542,7 +560,7 @@ k_simulate_steal(const uint2* __restrict__ q_po, const uint32_t* __restrict__ q_
         s_ustart[c] = qo[c];
         s_remain[c] = r;
     }
-    if (c == 0) { s_total = 0; s_horizon = ~0ull; s_first = ~0ull; s_front = ~0ull; }
+    if (c == 0) { s_total = 0; s_horizon = ~0ull; s_first = ~0ull; s_front = ~0ull; s_chunks = 0u; }
     if (served)                                           // requests nobody gets to (iteration limit)
         for (int i = c; i < n_req; i += stride) served[i] = -1;
     __syncthreads();
@@ -562,6 +580,12 @@ k_simulate_steal(const uint2* __restrict__ q_po, const uint32_t* __restrict__ q_
         tr = reinterpret_cast<uint4*>(trace + t0);
         tr_lim = capr > 0x7FFFFFFFll ? 0x7FFFFFFFu : (uint32_t)(capr < 0 ? 0 : capr);
     }
+    // event log: this simulation's pool of chunks, the chunk I am filling, my entries so far
+    uint4* const ev_pool = events ? events + (size_t)sim * ev_stride : nullptr;
+    uint32_t* const tag_sim = events ? chunk_tag + (size_t)sim * pool_chunks : nullptr;
+    uint4* ev_chunk = nullptr;
+    uint32_t n_ev = 0;
+    bool log_on = false;                                  // not during the dry run
     auto emit = [&](uint32_t dur, uint32_t r1, uint32_t r2, uint32_t r3) {
         const uint32_t it = n_pre + cnt;
         t += dur;
@@ -640,6 +664,24 @@ k_simulate_steal(const uint2* __restrict__ q_po, const uint32_t* __restrict__ q_
     // Clock, hash, trace and waited decode time of the iteration in dur, r1, r2, r3; false when the
     // clock limit is reached.
     auto finish_event = [&]() {
+        if (log_on && ((r1 >> 31) || r3 != 0u)) {
+            // Something changed: a log entry as in k_simulate, {iteration, tokens, sum KV after it,
+            // packed}.  Every prefill admits a request and every logged decode retires one, so all
+            // the clients' entries together are at most two per request of the instance, and the
+            // chunks they start at most that / LOG_CHUNK + one per client: the pool's size.
+            if ((n_ev & (LOG_CHUNK - 1)) == 0u) {
+                const unsigned ch = atomicAdd(&s_chunks, 1u);
+                ev_chunk = nullptr;
+                if (HOS_IN(ch, pool_chunks, 325) && ch < (unsigned)pool_chunks) {
+                    tag_sim[ch] = ((uint32_t)c << 16) | (n_ev / LOG_CHUNK);
+                    ev_chunk = ev_pool + (size_t)ch * LOG_CHUNK;
+                }
+            }
+            const uint32_t packed = (r1 >> 31) ? (0x80000000u | (r3 << 16) | ((B - 1u) << 8) | ((r1 & 0x7FFFFFFFu) - 1u))
+                                               : (((r3 - 1u) << 8) | (r1 - 1u));
+            if (ev_chunk) ev_chunk[n_ev & (LOG_CHUNK - 1)] = make_uint4(n_pre + cnt, r2, S, packed);
+            ++n_ev;
+        }
         emit(dur, r1, r2, r3);
         if (r1 >> 31) { Cd = 0; ++n_pre; }
         else { ++cnt; Cd = min(Cd + dur, 0x7FFFFFFFu); }
@@ -744,6 +786,7 @@ k_simulate_steal(const uint2* __restrict__ q_po, const uint32_t* __restrict__ q_
         t = 0; busy = 0; Cd = 0; cnt = 0; B = 0; S = 0; reserved = 0; n_pre = 0;
         next_fin = EMPTY; nA = 0; sumP = 0; sumTot = 0; head = 0;
         hash = HASH_INIT; status = 0; finished = !is_client;
+        log_on = events != nullptr;
     }
 
     // After s_first the conservative bound: no iteration lasts less than d_min and a client claims
@@ -808,6 +851,36 @@ k_simulate_steal(const uint2* __restrict__ q_po, const uint32_t* __restrict__ q_
         cres[unit] = hos_client_result{t, busy, n_pre, cnt, hash, 0.0};
         status_out[unit] = status;
     }
+    if (events) {
+        // The directory: every client's chunks in the order it filled them, the clients one after
+        // the other.  (The loop above ends at a barrier, so every tag written is visible here.)
+        const uint32_t mine = is_client ? (n_ev + LOG_CHUNK - 1) / LOG_CHUNK : 0u;
+        uint32_t inc = mine;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const uint32_t y = __shfl_up_sync(FULL, inc, d);
+            if (lane_id() >= d) inc += y;
+        }
+        if (lane_id() == 31) s_wchunks[warp_id()] = inc;
+        __syncthreads();
+        uint32_t before = 0;
+        for (int w = 0; w < warp_id(); ++w) before += s_wchunks[w];
+        s_dstart[c] = before + inc - mine;
+        if (is_client) {
+            event_count[unit] = n_ev;
+            dir_start[unit] = before + inc - mine;
+        }
+        __syncthreads();
+        const unsigned total = min(s_chunks, (unsigned)pool_chunks);
+        uint32_t* const dir_sim = chunk_dir + (size_t)sim * pool_chunks;
+        for (unsigned ch = c; ch < total; ch += stride) {
+            const uint32_t tag = tag_sim[ch];
+            const uint32_t owner = tag >> 16, seq = tag & 0xFFFFu;
+            if (!HOS_IN(owner, n_clients, 326) || owner >= (uint32_t)n_clients) continue;
+            const uint32_t at = s_dstart[owner] + seq;
+            if (HOS_IN(at, pool_chunks, 327) && at < (uint32_t)pool_chunks) dir_sim[at] = ch;
+        }
+    }
 }
 
 // ---------------------------------------------------------------------------------------
@@ -821,7 +894,9 @@ k_simulate_steal(const uint2* __restrict__ q_po, const uint32_t* __restrict__ q_
 __global__ void __launch_bounds__(128)
 k_trace_fill(const int32_t* __restrict__ q_off, int n_lambda, int n_clients, int n_pad, long long n_units,
              hos_cost_model cm, int q_shift, const hos_client_result* __restrict__ cres,
-             const uint4* __restrict__ events, const uint32_t* __restrict__ event_count,
+             const uint4* __restrict__ events, long long ev_stride, const uint32_t* __restrict__ event_count,
+             const uint32_t* __restrict__ log_kind, int pool_chunks, const uint32_t* __restrict__ chunk_dir,
+             const uint32_t* __restrict__ dir_start,
              hos_iter_rec* __restrict__ trace, const long long* __restrict__ trace_off,
              int32_t* __restrict__ status_out) {
     const long long unit = (long long)blockIdx.x * 4 + warp_id();
@@ -831,7 +906,12 @@ k_trace_fill(const int32_t* __restrict__ q_off, int n_lambda, int n_clients, int
     const int sim = (int)(unit / n_clients);
     const int inst = sim / n_lambda;
     const int q0 = q_off[(size_t)inst * (n_clients + 1) + c];
-    const uint4* ev = events + ((size_t)sim * n_pad + q0) * 2;
+    // the client's log: its own stretch of the simulation's log, or (stealing simulator) chunks of
+    // LOG_CHUNK entries listed in the directory
+    const bool chunked = __ldg(log_kind) == LOG_CHUNKED;
+    const uint4* ev = events + (size_t)sim * ev_stride + (chunked ? (size_t)0 : (size_t)q0 * 2);
+    const uint32_t* dir = chunk_dir + (size_t)sim * pool_chunks;
+    const uint32_t d0 = chunked ? dir_start[unit] : 0u;
     const uint32_t n_ev = event_count[unit];
     const uint32_t n_total = cres[unit].n_prefill_iters + cres[unit].n_decode_iters;
     const long long t0 = trace_off[unit];
@@ -852,8 +932,15 @@ k_trace_fill(const int32_t* __restrict__ q_off, int n_lambda, int n_clients, int
         const uint32_t kf = filled + lane;
         uint4* dst = &ring[kf & (TF_RING - 1)];
         if (kf < n_ev) {
+            const uint4* src = ev + kf;
+            if (chunked) {
+                // `filled` is a multiple of LOG_CHUNK = 32: the warp's 32 entries are one chunk
+                const uint32_t at = d0 + filled / LOG_CHUNK;
+                const uint32_t ch = HOS_IN(at, pool_chunks, 341) && at < (uint32_t)pool_chunks ? __ldg(&dir[at]) : 0u;
+                src = HOS_IN(ch, pool_chunks, 342) && ch < (uint32_t)pool_chunks ? ev + (size_t)ch * LOG_CHUNK + lane : ev;
+            }
             const unsigned sa = (unsigned)__cvta_generic_to_shared(dst);
-            asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" :: "r"(sa), "l"(ev + kf) : "memory");
+            asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" :: "r"(sa), "l"(src) : "memory");
         } else {
             *dst = make_uint4(0xFFFFFFFFu, 0u, 0u, 0u);
         }
@@ -1031,7 +1118,7 @@ cudaError_t launch_simulate(const hos_batch& b, const hos_cost_model& cm, const 
                             int n_lambda, uint32_t max_iters, const uint2* q_po, const int32_t* q_off,
                             const int32_t* inst_status, int n_pad, hos_client_result* cres,
                             hos_iter_rec* trace, const long long* trace_off, int32_t* status,
-                            uint4* events, uint32_t* event_count, cudaStream_t st) {
+                            const EventLog& log, cudaStream_t st) {
     const long long n_units = (long long)b.n_inst * n_lambda * b.n_clients;
     // A fixed reservation of R tokens per request admits floor(budget / R) requests at most and
     // nothing else: the simulator runs with that many slots and no KV limit.
@@ -1084,17 +1171,22 @@ cudaError_t launch_simulate(const hos_batch& b, const hos_cost_model& cm, const 
     launch_hook("k_simulate", 0, st);
     kern_n<<<sn.grid, 32 * sn.wpc, sn.smem, st>>>(
         q_po, q_off, inst_status, lambda_q16, n_lambda, b.n_clients, n_pad, n_units, sn.lanes, cap,
-        kv, cm, q_shift, max_iters, cres, trace, trace_off, status, events, event_count);
+        kv, cm, q_shift, max_iters, cres, trace, trace_off, status, log.events, log.ev_stride, log.event_count,
+        log.kind);
     launch_hook("k_simulate", 1, st);
     if (b.kv_budget >= 65536) {                          // otherwise no p + o can reach 2^16
         launch_hook("k_simulate_wide", 0, st);
         kern_w<<<sw.grid, 32 * sw.wpc, sw.smem, st>>>(
             q_po, q_off, inst_status, lambda_q16, n_lambda, b.n_clients, n_pad, n_units, sw.lanes, cap,
-            kv, cm, q_shift, max_iters, cres, trace, trace_off, status, events, event_count);
+            kv, cm, q_shift, max_iters, cres, trace, trace_off, status, log.events, log.ev_stride,
+            log.event_count, log.kind);
         launch_hook("k_simulate_wide", 1, st);
     }
     return cudaGetLastError();
 }
+
+int event_log_chunks(int n_pad, int n_clients) { return (2 * n_pad + LOG_CHUNK - 1) / LOG_CHUNK + n_clients; }
+int event_log_chunk_entries() { return LOG_CHUNK; }
 
 size_t simulate_steal_smem(int n_clients, int cap, bool wide) {
     const int threads = (n_clients + 31) & ~31;
@@ -1106,7 +1198,7 @@ cudaError_t launch_simulate_steal(const hos_batch& b, const hos_cost_model& cm, 
                                   const uint32_t* q_req,
                                   const int32_t* q_off, const int32_t* inst_status, int n_pad,
                                   hos_client_result* cres, hos_iter_rec* trace, const long long* trace_off,
-                                  int32_t* status, int32_t* served_by, cudaStream_t st) {
+                                  int32_t* status, int32_t* served_by, const EventLog& log, cudaStream_t st) {
     const int threads = (b.n_clients + 31) & ~31;
     const int cap = sim_slots(b);
     const uint32_t kv = sim_budget(b);
@@ -1121,7 +1213,8 @@ cudaError_t launch_simulate_steal(const hos_batch& b, const hos_cost_model& cm, 
     launch_hook("k_simulate_steal", 0, st);
     k_simulate_steal<NarrowEntry><<<grid, threads, smem_n, st>>>(
         q_po, b.o_est ? q_key : nullptr, q_req, q_off, inst_status, lambda_q16, n_lambda, b.n_clients, b.n_req, n_pad, cap,
-        kv, cm, q_shift, max_iters, cres, trace, trace_off, status, served_by);
+        kv, cm, q_shift, max_iters, cres, trace, trace_off, status, served_by, log.events, log.ev_stride,
+        log.pool_chunks, log.chunk_tag, log.chunk_dir, log.dir_start, log.event_count, log.kind);
     launch_hook("k_simulate_steal", 1, st);
     if (b.kv_budget >= 65536) {                          // otherwise no p + o can reach 2^16
         e = allow_max_dynamic_smem(reinterpret_cast<const void*>(k_simulate_steal<WideEntry>));
@@ -1129,7 +1222,8 @@ cudaError_t launch_simulate_steal(const hos_batch& b, const hos_cost_model& cm, 
         launch_hook("k_simulate_steal_wide", 0, st);
         k_simulate_steal<WideEntry><<<grid, threads, smem_w, st>>>(
             q_po, b.o_est ? q_key : nullptr, q_req, q_off, inst_status, lambda_q16, n_lambda, b.n_clients, b.n_req, n_pad, cap,
-            kv, cm, q_shift, max_iters, cres, trace, trace_off, status, served_by);
+            kv, cm, q_shift, max_iters, cres, trace, trace_off, status, served_by, log.events, log.ev_stride,
+            log.pool_chunks, log.chunk_tag, log.chunk_dir, log.dir_start, log.event_count, log.kind);
         launch_hook("k_simulate_steal_wide", 1, st);
     }
     return cudaGetLastError();
@@ -1137,7 +1231,7 @@ cudaError_t launch_simulate_steal(const hos_batch& b, const hos_cost_model& cm, 
 
 cudaError_t launch_trace_fill(const hos_batch& b, const hos_cost_model& cm, int n_lambda,
                               const int32_t* q_off, int n_pad, const hos_client_result* cres,
-                              const uint4* events, const uint32_t* event_count, hos_iter_rec* trace,
+                              const EventLog& log, hos_iter_rec* trace,
                               const long long* trace_off, int32_t* status, cudaStream_t st) {
     const long long n_units = (long long)b.n_inst * n_lambda * b.n_clients;
     int q_shift = -1;
@@ -1145,7 +1239,9 @@ cudaError_t launch_trace_fill(const hos_batch& b, const hos_cost_model& cm, int 
         for (q_shift = 0; (1u << q_shift) != cm.decode_kv_div; ++q_shift) {}
     launch_hook("k_trace_fill", 0, st);
     k_trace_fill<<<(unsigned)((n_units + 3) / 4), 128, 0, st>>>(q_off, n_lambda, b.n_clients, n_pad, n_units,
-                                                                cm, q_shift, cres, events, event_count,
+                                                                cm, q_shift, cres, log.events, log.ev_stride,
+                                                                log.event_count, log.kind, log.pool_chunks,
+                                                                log.chunk_dir, log.dir_start,
                                                                 trace, trace_off, status);
     launch_hook("k_trace_fill", 1, st);
     return cudaGetLastError();

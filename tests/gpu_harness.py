@@ -137,18 +137,25 @@ def check_simulate(hos, p, o, M, cap, kv, cm, assign, lambdas, mode, insts=None,
 
 
 def gpu_simulate_steal(hos, p, o, M, cap, kv, cm, assign, lambdas, mode, max_iters=0x7FFFFFFF, est=None, rsv=0):
-    """hos_online_simulate_steal: counts, then a traced run with exact slots.  Host-side views."""
+    """hos_online_simulate_steal: counts (with the event log), offsets, then the trace twice: rebuilt
+    from the event log by hos_trace_fill and written directly by a traced run with exact slots; the
+    two must be the same bytes.  Host-side views."""
     import torch
     from paper_2502_15763_b200.binding import view_struct
     dp, do, da = to_dev(p), to_dev(o), to_dev(assign)
     dl = to_dev(np.asarray(lambdas, dtype=np.uint32))
     ek = dict(o_est=None if est is None else to_dev(est), kv_reserve=rsv)
-    r = hos.hos_online_simulate_steal(dp, do, M, cap, kv, cm, da, dl, mode, max_iters, want_served_by=True, **ek)
+    r = hos.hos_online_simulate_steal(dp, do, M, cap, kv, cm, da, dl, mode, max_iters, want_served_by=True,
+                                      keep_events=True, **ek)
     off = hos.hos_trace_offsets(r["cres"])
     trace = torch.zeros((max(int(off[-1].item()), 1), 16), dtype=torch.uint8, device="cuda")
     r2 = hos.hos_online_simulate_steal(dp, do, M, cap, kv, cm, da, dl, mode, max_iters, trace=trace, trace_off=off,
                                        want_served_by=True, **ek)
     assert torch.equal(r["cres"][..., :32], r2["cres"][..., :32]) and torch.equal(r["served_by"], r2["served_by"])
+    filled = torch.zeros_like(trace)
+    hos.hos_trace_fill(dp, do, M, cap, kv, cm, len(lambdas), r, filled, off, **ek)
+    assert torch.equal(filled, trace), "trace rebuilt from the stealing simulator's event log differs from the traced run"
+    assert torch.equal(r["status"], r2["status"]), "status after hos_trace_fill differs"
     return dict(cres=view_struct(r2["cres"], hos.CLIENT_RESULT_DTYPE), sres=view_struct(r2["sres"], hos.SIM_RESULT_DTYPE),
                 status=r2["status"].cpu().numpy(), served_by=r2["served_by"].cpu().numpy(),
                 trace=view_struct(trace, hos.ITER_REC_DTYPE), trace_off=off.cpu().numpy())

@@ -185,6 +185,58 @@ def test_request_stealing(hos, n, M, cap):
     H.check_simulate_steal(hos, p, o, M, cap, kv, cm, g["assign"], (LAMBDA_ONE,), ora.QUEUE_SORTED, max_iters=25)
 
 
+def test_request_stealing_event_log_edges(hos):
+    import torch
+    # one slot per client: every request is a prefill and a retiring decode of its own, so the log is
+    # as long as it can get (two entries per request) and nearly all of it sits with the clients that
+    # took the requests from client 0's queue
+    rng = np.random.default_rng(77)
+    n_inst, n, M, cap = 3, 257, 7, 1
+    p = rng.integers(1, 300, size=(n_inst, n)).astype(np.uint32)
+    o = rng.integers(1, 40, size=(n_inst, n)).astype(np.uint32)
+    cm = (20000, 40, 15000, 300, 16, 40, 350)
+    assign = np.zeros((n_inst, n), dtype=np.int32)
+    r = H.check_simulate_steal(hos, p, o, M, cap, 10 ** 6, cm, assign, (LAMBDA_ONE, LAMBDA_PREFILL_FIRST), ora.QUEUE_SORTED)
+    assert int(r["cres"]["n_prefill_iters"].sum()) == 2 * n_inst * n          # one prefill per request and multiplier
+    assert (r["cres"]["n_prefill_iters"][:, :, 1:] > 0).all()                   # the others served stolen requests
+    # an invalid instance beside valid ones: no log entries, no trace records, neighbours untouched
+    o2 = o.copy(); o2[1, 9] = 0
+    dp, do, da = H.to_dev(p), H.to_dev(o2), H.to_dev(assign)
+    dl = H.to_dev(np.asarray([LAMBDA_ONE], np.uint32))
+    s = hos.hos_online_simulate_steal(dp, do, M, cap, 10 ** 6, cm, da, dl, ora.QUEUE_SORTED, keep_events=True)
+    off = hos.hos_trace_offsets(s["cres"])
+    offs = off.cpu().numpy()
+    assert offs[M] == offs[2 * M]                                               # instance 1 has no iterations
+    filled = torch.zeros((int(offs[-1]), 16), dtype=torch.uint8, device="cuda")
+    hos.hos_trace_fill(dp, do, M, cap, 10 ** 6, cm, 1, s, filled, off)
+    direct = torch.zeros_like(filled)
+    hos.hos_online_simulate_steal(dp, do, M, cap, 10 ** 6, cm, da, dl, ora.QUEUE_SORTED, trace=direct, trace_off=off)
+    assert torch.equal(filled, direct)
+    st = s["status"].cpu().numpy()
+    assert (st[1] == hos.HOS_ST_INVALID).all() and (st[0] == 0).all() and (st[2] == 0).all()
+    # too few trace slots: the records that fit are the first ones, the status bit is set
+    small = torch.arange(n_inst * M + 1, dtype=torch.int64, device="cuda") * 5
+    part = torch.zeros((n_inst * M * 5, 16), dtype=torch.uint8, device="cuda")
+    s = hos.hos_online_simulate_steal(dp, H.to_dev(o), M, cap, 10 ** 6, cm, da, dl, ora.QUEUE_SORTED, keep_events=True)
+    hos.hos_trace_fill(dp, H.to_dev(o), M, cap, 10 ** 6, cm, 1, s, part, small)
+    assert (s["status"].cpu().numpy() == hos.HOS_ST_TRACE).all()
+    full_off = hos.hos_trace_offsets(s["cres"]).cpu().numpy()
+    full = torch.zeros((int(full_off[-1]), 16), dtype=torch.uint8, device="cuda")
+    hos.hos_online_simulate_steal(dp, H.to_dev(o), M, cap, 10 ** 6, cm, da, dl, ora.QUEUE_SORTED, trace=full,
+                                  trace_off=H.to_dev(full_off, np.int64))
+    for x in range(n_inst * M):
+        assert torch.equal(part[5 * x:5 * x + 5], full[int(full_off[x]):int(full_off[x]) + 5])
+    # the same workspace used by the plain simulator afterwards: the log's form follows the last call
+    ws = s["ws"]
+    s3 = hos.hos_online_simulate(dp, H.to_dev(o), M, cap, 10 ** 6, cm, da, dl, ora.QUEUE_SORTED, keep_events=True, ws=ws)
+    off3 = hos.hos_trace_offsets(s3["cres"])
+    f3 = torch.zeros((int(off3[-1].item()), 16), dtype=torch.uint8, device="cuda")
+    hos.hos_trace_fill(dp, H.to_dev(o), M, cap, 10 ** 6, cm, 1, s3, f3, off3)
+    d3 = torch.zeros_like(f3)
+    hos.hos_online_simulate(dp, H.to_dev(o), M, cap, 10 ** 6, cm, da, dl, ora.QUEUE_SORTED, trace=d3, trace_off=off3)
+    assert torch.equal(f3, d3)
+
+
 def test_request_stealing_config1_and_wide(hos):
     w = workload("c1")
     p, o = w.lengths()
