@@ -114,7 +114,6 @@ k_estimate_sort(const uint32_t* __restrict__ p, const uint32_t* __restrict__ o,
                 InstInfo* __restrict__ info, int32_t* __restrict__ status_out, hos_lb* __restrict__ lb_out,
                 int n_pad) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
-    __shared__ unsigned long long red[32];
     __shared__ uint32_t s_pair[2];                        // T_(M), T_(M+1)
     const uint32_t e_p = cm.est_per_prompt_token, e_o = cm.est_per_output_token;
     for (int inst = blockIdx.x; inst < n_inst; inst += gridDim.x) {
@@ -130,6 +129,7 @@ k_estimate_sort(const uint32_t* __restrict__ p, const uint32_t* __restrict__ o,
         // first pass: checks, sums, the largest T (and the lower bounds' sums).  kv_budget here is
         // the most KV one request may need: the fixed reservation, if there is one
         unsigned long long sum = 0, mx = 0, bad = 0;
+        uint32_t mx32 = 0;                                // a T beyond 32 bits marks the instance bad: mx is not used then
         LbSums a = {0ull, 0ull, 0ull, 0ull};
         for_each_request(pi, oi, ei, nullptr, n_req, [&](int i, uint32_t pp, uint32_t oo, uint32_t oe, int) {
             const unsigned long long t = (unsigned long long)e_p * pp + (unsigned long long)e_o * oe;
@@ -139,18 +139,31 @@ k_estimate_sort(const uint32_t* __restrict__ p, const uint32_t* __restrict__ o,
             else if (lb_out) lb_take(a, cm, q_shift, pp, oo);
             if (!FAST) key[i] = (uint32_t)t;
             sum += t;
-            mx = t > mx ? t : mx;
+            mx32 = max(mx32, (uint32_t)t);
         });
-        sum = block_sum_u64(sum, red);
-        mx = block_max_u64(mx, red);
-        bad = block_max_u64(bad, red);
-        if (lb_out && !bad) {
-            a.P = block_sum_u64(a.P, red);
-            a.O = block_sum_u64(a.O, red);
-            a.K = block_sum_u64(a.K, red);
-            a.chain = block_max_u64(a.chain, red);
+        mx = mx32;
+        // all of them in one go: per warp, then warp k finishes value k (four sums, two maxima).  The
+        // scratch is a part of the sort's shared memory that nothing uses before the sort starts.
+        {
+            typedef unsigned long long red_row[SORT_WARPS];
+            red_row* red = reinterpret_cast<red_row*>(
+                FAST ? smem_raw : reinterpret_cast<unsigned char*>(sort_smem_carve<uint16_t>(smem_raw, n_req).cnt));
+            unsigned long long v[6] = {sum, a.P, a.O, a.K, mx, a.chain};
+#pragma unroll
+            for (int k = 0; k < 6; ++k) {
+                v[k] = k < 4 ? warp_sum_u64(v[k]) : warp_max_u64(v[k]);
+                if (lane_id() == 0) red[k][warp_id()] = v[k];
+            }
+            bad = __syncthreads_or(bad != 0);
+            if (warp_id() < 6) {
+                const unsigned long long t = red[warp_id()][lane_id()];
+                const unsigned long long r = warp_id() < 4 ? warp_sum_u64(t) : warp_max_u64(t);
+                if (lane_id() == 0) red[warp_id()][0] = r;
+            }
+            __syncthreads();
+            sum = red[0][0]; a.P = red[1][0]; a.O = red[2][0]; a.K = red[3][0]; mx = red[4][0]; a.chain = red[5][0];
+            __syncthreads();                              // the scratch is the sort's again
         }
-        __syncthreads();
         if (bad) {                                        // uniform: every thread sees the same value
             if (threadIdx.x == 0) {
                 info[inst].sum_T = sum; info[inst].max_T = (uint32_t)mx; info[inst].status = HOS_ST_INVALID;

@@ -32,7 +32,6 @@ k_queue_build(const uint32_t* __restrict__ p, const uint32_t* __restrict__ o,
               int32_t* __restrict__ q_off, unsigned long long* __restrict__ inst_O,
               int32_t* __restrict__ inst_status, int n_pad) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
-    __shared__ unsigned long long red[32];
     const int cbits = bit_width_u32((uint32_t)(n_clients - 1));
     for (int inst = blockIdx.x; inst < n_inst; inst += gridDim.x) {
         if (!FAST) {
@@ -49,7 +48,10 @@ k_queue_build(const uint32_t* __restrict__ p, const uint32_t* __restrict__ o,
 
         // first pass: checks and sums.  kv_budget here is the most KV one request may need: the
         // fixed reservation, if there is one
-        unsigned long long sumO = 0, mx = 0, mxk = 0, mxp = 0, bad = 0;
+        // (the maxima in 32 bits: a sum that does not fit marks the instance bad, and then they are not used)
+        unsigned long long sumO = 0;
+        uint32_t mx = 0, mxk = 0, mxp = 0;
+        int bad = 0;
         for_each_request(pi, oi, ei, ai, n_req, [&](int i, uint32_t pp, uint32_t oo, uint32_t oe, int c) {
             const unsigned long long tot = (unsigned long long)pp + oo;
             const unsigned long long totk = (unsigned long long)pp + oe;
@@ -58,22 +60,32 @@ k_queue_build(const uint32_t* __restrict__ p, const uint32_t* __restrict__ o,
                 bad = 1;
             if (!FAST) { key[i] = (uint32_t)totk; park[i] = (uint16_t)(c & 0xFF); }
             sumO += oo;
-            mx = tot > mx ? tot : mx;
-            mxk = totk > mxk ? totk : mxk;
-            mxp = pp > mxp ? pp : mxp;
+            mx = max(mx, (uint32_t)tot);
+            mxk = max(mxk, (uint32_t)totk);
+            mxp = max(mxp, pp);
         });
-        sumO = block_sum_u64(sumO, red);
-        mx = block_max_u64(mx, red);
-        mxk = block_max_u64(mxk, red);
-        mxp = block_max_u64(mxp, red);
-        bad = block_max_u64(bad, red);
-        __syncthreads();
+        // per warp, one barrier, then every warp finishes all four from the warps' values.  The scratch
+        // is a part of the sort's shared memory that nothing uses before the sort starts.
+        unsigned long long* red = reinterpret_cast<unsigned long long*>(
+            FAST ? smem_raw : reinterpret_cast<unsigned char*>(sort_smem_carve<uint16_t>(smem_raw, n_req).cnt));
+        uint32_t (*redm)[SORT_WARPS] = reinterpret_cast<uint32_t (*)[SORT_WARPS]>(red + SORT_WARPS);
+        sumO = warp_sum_u64(sumO);
+        mx = __reduce_max_sync(FULL, mx);
+        mxk = __reduce_max_sync(FULL, mxk);
+        mxp = __reduce_max_sync(FULL, mxp);
+        if (lane_id() == 0) { red[warp_id()] = sumO; redm[0][warp_id()] = mx; redm[1][warp_id()] = mxk; redm[2][warp_id()] = mxp; }
+        bad = __syncthreads_or(bad);
+        sumO = warp_sum_u64(red[lane_id()]);
+        mx = __reduce_max_sync(FULL, redm[0][lane_id()]);
+        mxk = __reduce_max_sync(FULL, redm[1][lane_id()]);
+        mxp = __reduce_max_sync(FULL, redm[2][lane_id()]);
+        __syncthreads();                                  // the scratch is the sort's again
         const int kb = (queue_order == HOS_QUEUE_SORTED) ? bit_width_u32((uint32_t)mxk) : 0;
         // the composite sort key, client above p + (estimated) o, has 32 bits: an estimate so long
         // that it does not fit beside the client bits invalidates the instance (uniform over the CTA)
         if (kb + cbits > 32) bad = 1;
         // bit 8 (internal): some p + o needs more than 16 bits -> the simulator's wide heap entries
-        const int32_t st_done = bad ? HOS_ST_INVALID : (mx >= 65536ull ? INST_WIDE : 0);
+        const int32_t st_done = bad ? HOS_ST_INVALID : (mx >= 65536u ? INST_WIDE : 0);
         if (bad) {
             if (threadIdx.x == 0) { inst_O[inst] = sumO; inst_status[inst] = st_done; }
             continue;

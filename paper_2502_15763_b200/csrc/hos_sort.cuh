@@ -196,6 +196,9 @@ __device__ inline IdxT* block_radix_sort_ids(const SortSmem<IdxT>& s, int n, int
 // neighbouring positions, so the caller can write them straight to global memory.  With about
 // two buckets per item this is a few compares per item instead of a ranking vote per key bit
 // and pass.  The counters are 16 bits wide, two to a word (no count or offset reaches 2^16).
+// In the scan every thread owns a run of consecutive counter words; a spare word after each such
+// run keeps the threads of a warp on different banks (without it their runs, a power of two long,
+// start on two banks in all: at 2^15 buckets the scan alone took a quarter of the sort).
 // The keys themselves are not kept in shared memory: the caller passes over its data once to
 // count and once to place (bucket_sort_count / bucket_sort_place).
 //
@@ -208,8 +211,10 @@ constexpr int BUCKET_BITS_MAX = 15;
 constexpr int BUCKET_WORK_MAX = 96;
 
 // Most bucket bits whose counters fit beside the entry and bucket tables (host and device agree).
+constexpr size_t BUCKET_PAD_BYTES = 4 * SORT_THREADS;      // one spare counter word per thread
 __host__ __device__ inline int bucket_bits_cap(int n) {
-    const size_t room = SMEM_LIMIT - 2048 - align16(size_t(n) * 4) - align16(size_t(n) * 2);   // 2 KB for static shared memory
+    // 2 KB for static shared memory
+    const size_t room = SMEM_LIMIT - 2048 - BUCKET_PAD_BYTES - align16(size_t(n) * 4) - align16(size_t(n) * 2);
     int bb = BUCKET_BITS_MAX;
     while (bb > 10 && (size_t(2) << bb) > room) --bb;
     int want = 11;                                                           // about two buckets per item
@@ -217,15 +222,16 @@ __host__ __device__ inline int bucket_bits_cap(int n) {
     return bb < want ? bb : want;
 }
 __host__ __device__ inline size_t bucket_sort_smem_bytes(int n) {
-    return align16(size_t(n) * 4) + align16(size_t(n) * 2) + (size_t(2) << bucket_bits_cap(n));
+    return align16(size_t(n) * 4) + align16(size_t(n) * 2) + (size_t(2) << bucket_bits_cap(n)) + BUCKET_PAD_BYTES;
 }
 
 struct BucketSort {
     int bbits, low_bits, id_bits, xbits, n_words, n;
+    int pad_shift;              // counter word w lives at cntw[w + (w >> pad_shift)]
     uint32_t kmask, lmask;
     uint32_t* ent;              // [n]  (rest of key << id_bits | id) << xbits | extra, in slot order
     uint16_t* bkt;              // [n]  bucket of every slot
-    uint32_t* cntw;             // [2^(bbits-1)] two 16-bit counters per word
+    uint32_t* cntw;             // [2^(bbits-1) + spares] two 16-bit counters per word
 };
 
 // Layout and bit budget for n items with `nbits` significant key bits and `xbits` extra bits per
@@ -237,6 +243,8 @@ __device__ inline bool bucket_sort_plan(BucketSort& B, unsigned char* smem, int 
     B.xbits = xbits;
     B.n = n;
     B.n_words = 1 << (B.bbits - 1);
+    // a thread's run in the scan is n_words / SORT_THREADS words (a power of two); no spares for runs of one
+    B.pad_shift = B.n_words > SORT_THREADS ? B.bbits - 1 - (31 - __clz(SORT_THREADS)) : 31;
     B.kmask = nbits >= 32 ? 0xFFFFFFFFu : ((1u << nbits) - 1u);
     B.lmask = B.low_bits >= 32 ? 0xFFFFFFFFu : ((1u << B.low_bits) - 1u);
     B.ent = reinterpret_cast<uint32_t*>(smem);
@@ -245,15 +253,22 @@ __device__ inline bool bucket_sort_plan(BucketSort& B, unsigned char* smem, int 
     return B.low_bits + B.id_bits + xbits <= 32;
 }
 
+// Where counter word w is kept, and bucket b's 16-bit counter.
+__device__ __forceinline__ uint32_t bucket_word_at(const BucketSort& B, uint32_t w) { return w + (w >> B.pad_shift); }
+__device__ __forceinline__ uint32_t bucket_half_at(const BucketSort& B, uint32_t b) {
+    return (bucket_word_at(B, b >> 1) << 1) | (b & 1u);
+}
+
 // Zeroes the counters.  Ends with a __syncthreads().
 __device__ inline void bucket_sort_clear(const BucketSort& B) {
-    for (int i = threadIdx.x; i < B.n_words; i += SORT_THREADS) B.cntw[i] = 0;
+    const int n_kept = (int)bucket_word_at(B, (uint32_t)B.n_words);
+    for (int i = threadIdx.x; i < n_kept; i += SORT_THREADS) B.cntw[i] = 0;
     __syncthreads();
 }
 
 __device__ __forceinline__ void bucket_sort_count(const BucketSort& B, uint32_t key) {
     const uint32_t b = (key & B.kmask) >> B.low_bits;
-    if (HOS_IN(b >> 1, B.n_words, 111)) atomicAdd(&B.cntw[b >> 1], 1u << ((b & 1u) << 4));
+    if (HOS_IN(b >> 1, B.n_words, 111)) atomicAdd(&B.cntw[bucket_word_at(B, b >> 1)], 1u << ((b & 1u) << 4));
 }
 
 // Exclusive scan of the bucket counts (after every bucket_sort_count).  Starts and ends with a
@@ -268,8 +283,9 @@ __device__ inline bool bucket_sort_scan(const BucketSort& B, int n) {
     const int w0 = min(B.n_words, t * per), w1 = min(B.n_words, w0 + per);
     uint32_t run = 0;
     unsigned long long work = 0;
+    const int at0 = (int)bucket_word_at(B, (uint32_t)w0);   // a run never crosses a spare word
     for (int w = w0; w < w1; ++w) {
-        const uint32_t c = B.cntw[w], a = c & 0xFFFFu, b = c >> 16;
+        const uint32_t c = B.cntw[at0 + (w - w0)], a = c & 0xFFFFu, b = c >> 16;
         run += a + b;
         work += (unsigned long long)(a * a + b * b);
     }
@@ -286,8 +302,8 @@ __device__ inline bool bucket_sort_scan(const BucketSort& B, int n) {
     const uint32_t wv = s_wsum[lane_id()];
     uint32_t acc = __reduce_add_sync(FULL, lane_id() < warp_id() ? wv : 0u) + inc - run;
     for (int w = w0; w < w1; ++w) {
-        const uint32_t c = B.cntw[w], a = c & 0xFFFFu, b = c >> 16;
-        B.cntw[w] = acc | ((acc + a) << 16);
+        const uint32_t c = B.cntw[at0 + (w - w0)], a = c & 0xFFFFu, b = c >> 16;
+        B.cntw[at0 + (w - w0)] = acc | ((acc + a) << 16);
         acc += a + b;
     }
     __syncthreads();
@@ -296,7 +312,7 @@ __device__ inline bool bucket_sort_scan(const BucketSort& B, int n) {
 
 // First slot of bucket b; valid between bucket_sort_scan and the first bucket_sort_place.
 __device__ __forceinline__ uint32_t bucket_sort_start(const BucketSort& B, uint32_t b) {
-    return reinterpret_cast<const uint16_t*>(B.cntw)[b];
+    return reinterpret_cast<const uint16_t*>(B.cntw)[bucket_half_at(B, b)];
 }
 
 // Scatter: the counter of the item's bucket walks from the bucket's start to its end.
@@ -304,7 +320,7 @@ __device__ __forceinline__ void bucket_sort_place(const BucketSort& B, uint32_t 
     const uint32_t fk = key & B.kmask;
     const uint32_t b = fk >> B.low_bits, sh = (b & 1u) << 4;
     if (!HOS_IN(b >> 1, B.n_words, 111)) return;
-    const uint32_t slot = (atomicAdd(&B.cntw[b >> 1], 1u << sh) >> sh) & 0xFFFFu;
+    const uint32_t slot = (atomicAdd(&B.cntw[bucket_word_at(B, b >> 1)], 1u << sh) >> sh) & 0xFFFFu;
     if (!HOS_IN(slot, B.n, 112)) return;
     B.ent[slot] = ((((fk & B.lmask) << B.id_bits) | id) << B.xbits) | extra;
     B.bkt[slot] = (uint16_t)b;
@@ -317,7 +333,7 @@ __device__ __forceinline__ uint32_t bucket_sort_rank(const BucketSort& B, int s,
     const uint16_t* cnt16 = reinterpret_cast<const uint16_t*>(B.cntw);
     const uint32_t mine = B.ent[s], b = B.bkt[s];
     const bool b_ok = HOS_IN(b, 1 << B.bbits, 113);
-    uint32_t start = (b_ok && b) ? cnt16[b - 1] : 0u, end = b_ok ? cnt16[b] : 0u;
+    uint32_t start = (b_ok && b) ? cnt16[bucket_half_at(B, b - 1)] : 0u, end = b_ok ? cnt16[bucket_half_at(B, b)] : 0u;
     if (!HOS_IN(end, B.n + 1, 114) || !HOS_IN(start, end + 1, 114)) start = end = 0;
     uint32_t r = start, j = start;
     for (; j + 1 < end; j += 2) r += (B.ent[j] < mine ? 1u : 0u) + (B.ent[j + 1] < mine ? 1u : 0u);
