@@ -1225,6 +1225,11 @@ k_local_search(const uint32_t* __restrict__ T_sorted, const uint32_t* __restrict
             };
             // The listed clients one after the other, so that client, list start and slack are the
             // same for the whole CTA; item idx of a client is its idx-th member, idx = len is the move.
+            // Nothing worse than the best step any lane of this warp has found so far can be the CTA's
+            // minimum, so that (one warp minimum per batch) is what a candidate is held against first:
+            // against its own best alone nearly every item would send some lane of the warp down the
+            // bookkeeping path.  Equal values pass: the order among them is decided by (i, k, u).
+            uint32_t wbest = NO_CAND;
             uint32_t nTu[LS_BATCH];                             // next batch: partner T (0 for the move)
             auto fetch = [&](int cb, int len, int i0) {
 #pragma unroll
@@ -1256,7 +1261,7 @@ k_local_search(const uint32_t* __restrict__ T_sorted, const uint32_t* __restrict
                         const uint32_t inv_r = d < slack ? ~(slack - d) : NO_CAND;
                         const int d2 = (int)(s_T[b[u] + 1] - Tu[u]);   // A[b]: largest T < thr (falling side)
                         const uint32_t inv_f = d2 > 0 ? ~(uint32_t)d2 : NO_CAND;
-                        if (min(inv_r, inv_f) > best.inv) continue;     // NO_CAND is the largest value
+                        if (min(inv_r, inv_f) > wbest) continue;        // NO_CAND is the largest value
                         const bool move = idx == len;
                         if (inv_r != NO_CAND && inv_r <= best.inv) {
                             // first member of the run of equal T: b - 1 itself unless its predecessor ties
@@ -1265,6 +1270,7 @@ k_local_search(const uint32_t* __restrict__ T_sorted, const uint32_t* __restrict
                         }
                         if (inv_f != NO_CAND && inv_f <= best.inv) consider(inv_f, b[u], k, move, cb + idx, idx);
                     }
+                    wbest = __reduce_min_sync(FULL, best.inv);
                 }
             }
             if (best_at >= 0) best.u1 = (uint32_t)clI[best_at] + 1u;
